@@ -1,0 +1,244 @@
+"""fp64 CPU oracle for Eigen Attention (rank-r attention) -- TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain statement of what the GPU library must compute.
+It is imported only by the tests, by the smoke check and by the benchmark's
+CPU-baseline leg; the product path never routes through it.  It shares no code
+with the CUDA sources and never sees a value produced by them.
+
+Everything is numpy float64.  The result has a closed-form definition
+(Eq. 7 of the paper), so the oracle is that definition written out: project,
+score, ordinary three-pass softmax, weighted sum, lift.  No tiling, no
+splitting of the key axis, no online softmax.
+
+Notation follows the paper: d_h head dimension, r rank, U^K / U^V bases with
+orthonormal columns (d_h x r), n cached length, per-head index i dropped where
+one head is handled.
+
+Parity pins (see tests): the functions here are pinned against an independent
+library routine for softmax attention applied to the d_h-wide low-rank inputs
+Q', K', V' of Eq. 6, brute-force Python loops on tiny inputs, closed-form
+special cases, and the numbers the paper prints for cache sizes.  Nothing in
+this file is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# Building blocks
+# --------------------------------------------------------------------------
+
+def softmax_rows(S: np.ndarray) -> np.ndarray:
+    """Row-wise Softmax of Eq. 2/3: max, exp-sum, normalise (three passes)."""
+    S = np.asarray(S, dtype=F64)
+    m = S.max(axis=-1, keepdims=True)
+    E = np.exp(S - m)
+    return E / E.sum(axis=-1, keepdims=True)
+
+
+def to_rank_space(X: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """Coordinates of the rows of X in the basis U: X U  (the r-wide factor of Eq. 6;
+    the merged weights W U of Eq. 8 produce exactly these rows)."""
+    return np.asarray(X, dtype=F64) @ np.asarray(U, dtype=F64)
+
+
+def lift(Y: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """Back to d_h dimensions: Y U^T  (the trailing (U^V)^T of Eq. 7)."""
+    return np.asarray(Y, dtype=F64) @ np.asarray(U, dtype=F64).T
+
+
+# --------------------------------------------------------------------------
+# One head, stateless: the definition
+# --------------------------------------------------------------------------
+
+def decode_head(q: np.ndarray, K: np.ndarray, V: np.ndarray,
+                U_K: np.ndarray, U_V: np.ndarray, lowrank_out: bool = False) -> np.ndarray:
+    """Generation-phase Eigen Attention for one head (Eq. 3 in the space of Eq. 7).
+
+    q [d_h]; K, V [n, d_h] are the un-projected rows of the n cached tokens
+    (the new token's row included: the cache is extended first, then attended,
+    Section 2 "LLM Inference").  Returns [d_h] (or [r_V] with lowrank_out).
+    The softmax scale is 1/sqrt(d_h) -- Eq. 7 keeps d_h although the vectors
+    are r wide.
+    """
+    d_h = U_K.shape[0]
+    qp = to_rank_space(q, U_K)                    # [r_K]
+    Kp = to_rank_space(K, U_K)                    # [n, r_K]
+    Vp = to_rank_space(V, U_V)                    # [n, r_V]
+    s = (Kp @ qp) / math.sqrt(d_h)                # [n]
+    p = softmax_rows(s[None, :])[0]
+    o = p @ Vp                                    # [r_V]
+    return o if lowrank_out else lift(o, U_V)
+
+
+def prefill_head(Q: np.ndarray, K: np.ndarray, V: np.ndarray,
+                 U_K: np.ndarray, U_V: np.ndarray, len0: int = 0,
+                 lowrank_out: bool = False) -> np.ndarray:
+    """Causal Eigen Attention for one head over a prompt.
+
+    Q [T, d_h] are the T new queries; K, V [len0+T, d_h] are all rows cached
+    after the call (len0 earlier rows followed by the T new ones).  Query t
+    attends rows 0..len0+t inclusive (decoder-only models; masked entries are
+    excluded from the softmax).  Returns [T, d_h] (or [T, r_V]).
+    """
+    d_h = U_K.shape[0]
+    T = Q.shape[0]
+    Qp = to_rank_space(Q, U_K)
+    Kp = to_rank_space(K, U_K)
+    Vp = to_rank_space(V, U_V)
+    O = np.zeros((T, Vp.shape[1]), dtype=F64)
+    for t in range(T):
+        n_t = len0 + t + 1
+        s = (Kp[:n_t] @ Qp[t]) / math.sqrt(d_h)
+        p = softmax_rows(s[None, :])[0]
+        O[t] = p @ Vp[:n_t]
+    return O if lowrank_out else lift(O, U_V)
+
+
+# --------------------------------------------------------------------------
+# One decoder layer with a rank-r KV cache (stateful, mirrors the library calls)
+# --------------------------------------------------------------------------
+
+class LayerOracle:
+    """Rank-r KV cache of one layer plus the calls of the library, in fp64.
+
+    U_K[h] is d_h x r_K[h], U_V[h] is d_h x r_V[h]  (per layer and head,
+    Section 4.1).  `tracked` optionally restricts the state to a list of
+    (b, h) units so that very large workloads can be checked on a subset.
+    """
+
+    def __init__(self, batch: int, n_heads: int, d_head: int,
+                 U_K: Sequence[np.ndarray], U_V: Sequence[np.ndarray],
+                 tracked: Optional[Sequence[Tuple[int, int]]] = None):
+        assert len(U_K) == n_heads and len(U_V) == n_heads
+        self.B, self.H, self.d_h = batch, n_heads, d_head
+        self.U_K = [np.asarray(u, dtype=F64) for u in U_K]
+        self.U_V = [np.asarray(u, dtype=F64) for u in U_V]
+        for u in self.U_K + self.U_V:
+            assert u.shape[0] == d_head
+        self.units = list(tracked) if tracked is not None else [
+            (b, h) for b in range(batch) for h in range(n_heads)]
+        self.Kp = {u: np.zeros((0, self.U_K[u[1]].shape[1]), dtype=F64) for u in self.units}
+        self.Vp = {u: np.zeros((0, self.U_V[u[1]].shape[1]), dtype=F64) for u in self.units}
+        self.len = 0
+        # counters for the closed forms of Table 1
+        self.cache_elements = 0       # stored numbers, all tracked units
+        self.projection_macs = 0      # run-time U multiplications
+        self.attention_macs = 0       # q'K'^T and pV' of the last decode call
+
+    # -- Section 2 "LLM Inference": K <- Concat(K, k), V <- Concat(V, v), in rank space (Eq. 6/8)
+    def append_kv(self, k: np.ndarray, v: np.ndarray) -> None:
+        """k, v: [B, T, H, d_h].  Projects each new row and extends the cache."""
+        k = np.asarray(k, dtype=F64)
+        v = np.asarray(v, dtype=F64)
+        T = k.shape[1]
+        for (b, h) in self.units:
+            kp = to_rank_space(k[b, :, h, :], self.U_K[h])
+            vp = to_rank_space(v[b, :, h, :], self.U_V[h])
+            self.Kp[(b, h)] = np.concatenate([self.Kp[(b, h)], kp], axis=0)
+            self.Vp[(b, h)] = np.concatenate([self.Vp[(b, h)], vp], axis=0)
+            self.cache_elements += kp.size + vp.size
+            self.projection_macs += T * self.d_h * (kp.shape[1] + vp.shape[1])
+        self.len += T
+
+    def append_unit_rows(self, unit: Tuple[int, int], k_rows: np.ndarray, v_rows: np.ndarray) -> None:
+        """Same as append_kv for one tracked unit given its rows [T, d_h] (large workloads
+        hand the history over unit by unit); the caller advances `len` with set_len."""
+        b, h = unit
+        kp = to_rank_space(k_rows, self.U_K[h])
+        vp = to_rank_space(v_rows, self.U_V[h])
+        self.Kp[unit] = np.concatenate([self.Kp[unit], kp], axis=0)
+        self.Vp[unit] = np.concatenate([self.Vp[unit], vp], axis=0)
+        self.cache_elements += kp.size + vp.size
+        self.projection_macs += k_rows.shape[0] * self.d_h * (kp.shape[1] + vp.shape[1])
+
+    def set_len(self, n: int) -> None:
+        self.len = n
+
+    # -- Eq. 3 in the rank-r space of Eq. 7
+    def decode(self, q: np.ndarray, lowrank_out: bool = False) -> dict:
+        """q: [B, 1, H, d_h] (or [B, H, d_h]).  Returns {(b,h): out[d_h]} for tracked units."""
+        q = np.asarray(q, dtype=F64).reshape(self.B, self.H, self.d_h)
+        out = {}
+        self.attention_macs = 0
+        for (b, h) in self.units:
+            Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]
+            assert Kp.shape[0] == self.len and self.len > 0
+            qp = to_rank_space(q[b, h], self.U_K[h])
+            self.projection_macs += self.d_h * qp.shape[0]
+            s = (Kp @ qp) / math.sqrt(self.d_h)
+            p = softmax_rows(s[None, :])[0]
+            o = p @ Vp
+            self.attention_macs += Kp.size + Vp.size
+            if lowrank_out:
+                out[(b, h)] = o
+            else:
+                out[(b, h)] = lift(o, self.U_V[h])
+                self.projection_macs += self.d_h * o.shape[0]
+        return out
+
+    def decode_dense(self, q: np.ndarray) -> np.ndarray:
+        """decode() gathered into [B, 1, H, d_h] (all units must be tracked)."""
+        res = self.decode(q)
+        out = np.zeros((self.B, 1, self.H, self.d_h), dtype=F64)
+        for (b, h), o in res.items():
+            out[b, 0, h] = o
+        return out
+
+    # -- prefill: cache the prompt's rank-r K/V, causal attention of its queries
+    def prefill(self, q: np.ndarray, k: np.ndarray, v: np.ndarray) -> dict:
+        """q, k, v: [B, T, H, d_h].  Returns {(b,h): out[T, d_h]}."""
+        q = np.asarray(q, dtype=F64)
+        len0 = self.len
+        self.append_kv(k, v)
+        T = q.shape[1]
+        out = {}
+        for (b, h) in self.units:
+            Qp = to_rank_space(q[b, :, h, :], self.U_K[h])
+            Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]
+            O = np.zeros((T, Vp.shape[1]), dtype=F64)
+            for t in range(T):
+                n_t = len0 + t + 1
+                s = (Kp[:n_t] @ Qp[t]) / math.sqrt(self.d_h)
+                p = softmax_rows(s[None, :])[0]
+                O[t] = p @ Vp[:n_t]
+            out[(b, h)] = lift(O, self.U_V[h])
+        return out
+
+    def prefill_dense(self, q, k, v) -> np.ndarray:
+        res = self.prefill(q, k, v)
+        T = np.asarray(q).shape[1]
+        out = np.zeros((self.B, T, self.H, self.d_h), dtype=F64)
+        for (b, h), o in res.items():
+            out[b, :, h, :] = o
+        return out
+
+
+# --------------------------------------------------------------------------
+# Closed forms the paper states (Table 1, Section 2)
+# --------------------------------------------------------------------------
+
+def kv_cache_bits(b: int, n: int, d: int, L: int, p: int) -> int:
+    """KV-cache size in bits: 2 * b * n * d * L * p with d the model width.
+
+    Section 2 prints an extra factor h; since d = h * d_h already covers all
+    heads, the paper's own worked example (batch 16, 32k context, 7B model,
+    16 bit -> 256 GB, Section 1) fixes the formula without it.
+    """
+    return 2 * b * n * d * L * p
+
+
+def table1_standard(n: int, d: int) -> dict:
+    """Table 1, standard attention column (per token, per layer; FLOPs are multiply-accumulates)."""
+    return {"kv_cache": 2 * n * d, "params": 4 * d * d, "flops": 4 * d * d + 2 * n * d}
+
+
+def table1_eigen(n: int, d: int, r: int) -> dict:
+    """Table 1, Eigen Attention column; r is the layer-wide rank (sum over heads)."""
+    return {"kv_cache": 2 * n * r, "params": 4 * d * r, "flops": 4 * d * r + 2 * n * r}
