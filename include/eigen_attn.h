@@ -1,0 +1,163 @@
+/*
+ * eigen_attn.h -- C ABI of libeigenattn: Eigen Attention (attention in a per-head rank-r space)
+ * for one decoder layer on one NVIDIA B200 (sm_100a).
+ *
+ * What is computed (paper: "Eigen Attention", Sections 2 and 4.2):
+ *   - every new key/value row is projected onto the head's orthonormal bases,
+ *       k' = k U^K_i ,  v' = v U^V_i                      (the r-wide factor of Eq. 6; Eq. 8 merged form)
+ *     and appended to a rank-r KV cache, K'_i <- Concat(K'_i, k'), V'_i <- Concat(V'_i, v')
+ *                                                          (Section 2, "LLM Inference")
+ *   - a decode step attends one query per sequence over the n cached rows,
+ *       h_i = Softmax( (q U^K_i) K'_i^T / sqrt(d_h) ) V'_i (U^V_i)^T          (Eq. 3 in the space of Eq. 7)
+ *     the scale is 1/sqrt(d_head) although the vectors are r wide (Eq. 7);
+ *   - a prefill call does the same for T prompt tokens at once with a causal mask
+ *     (query t sees rows 0..len0+t) and leaves their rank-r rows in the cache (Section 2, prefill phase).
+ *
+ * Conventions
+ *   - "d_" pointers are DEVICE pointers, "h_" pointers are HOST pointers.  Token tensors are
+ *     [batch][T][n_heads][d_head] in the layer's IO dtype; the head and d_head axes are contiguous,
+ *     the batch and token strides are passed in ELEMENTS.  The packed rank-space tensors selected by
+ *     the *_PREPROJECTED / EA_OUT_LOWRANK flags are always contiguous; strides do not apply to them.
+ *   - The caller owns every buffer, including the cache and the workspace (sizes from
+ *     eigen_attn_cache_bytes).  The library allocates no device memory; a handle owns host memory only.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All calls
+ *     are asynchronous with respect to that stream unless stated otherwise.
+ *   - Every function returns an ea_status.  Argument, shape and capacity errors are found on the
+ *     host before anything is launched and leave the handle unchanged.  Kernels never trap: a wait that
+ *     exceeds its bound records EA_ERR_TIMEOUT in a device status word read by eigen_attn_poll_status.
+ *   - A handle is not thread-safe.  All sequences of a handle share one length (`len`).
+ */
+#ifndef EIGEN_ATTN_H_
+#define EIGEN_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eigen_attn* eigen_attn_t;   /* opaque; one per decoder layer */
+
+typedef enum {
+  EA_OK = 0,
+  EA_ERR_INVALID_ARG = -1,      /* NULL pointer, bad enum, bad flag combination            */
+  EA_ERR_SHAPE = -2,            /* a dimension out of the supported range, len == 0 decode */
+  EA_ERR_CAPACITY = -3,         /* cache / workspace too small, len + T > n_max            */
+  EA_ERR_UNSUPPORTED = -4,      /* a valid request this version does not implement         */
+  EA_ERR_CUDA = -5,             /* a CUDA runtime call failed; see eigen_attn_last_error   */
+  EA_ERR_TIMEOUT = -6,          /* a bounded device-side wait gave up                      */
+  EA_ERR_NOT_ORTHONORMAL = -7   /* EA_CHECK_ORTHONORMAL: max|U^T U - I| > 1e-4             */
+} ea_status;
+
+typedef enum { EA_BF16 = 0, EA_FP32 = 1 } ea_dtype;   /* cache + IO dtype; accumulation is always fp32 */
+
+/* ea_desc.flags */
+#define EA_CHECK_ORTHONORMAL 0x1u   /* verify U^T U = I on the host at create (Section 4.2 assumes it) */
+
+/* per-call flags */
+#define EA_Q_PREPROJECTED  0x1u  /* d_q already holds q U^K (merged W^Q', Eq. 8): [B][T][sum_h rp_k[h]]      */
+#define EA_OUT_LOWRANK     0x2u  /* write o' without the (U^V)^T lift (merged W^O', Eq. 8): [B][T][sum rp_v] */
+#define EA_KV_PREPROJECTED 0x4u  /* d_k/d_v already hold k U^K, v U^V (merged W^K', W^V'): packed like q above */
+
+typedef struct {
+  int32_t batch;               /* B >= 1                                                             */
+  int32_t n_heads;             /* H, 1..256 (multi-head attention: one K/V head per query head)      */
+  int32_t d_head;              /* d_h, multiple of 8, 8..128                                          */
+  int32_t n_max;               /* cache capacity in rows per sequence                                 */
+  int32_t dtype;               /* ea_dtype                                                            */
+  int32_t max_prefill_tokens;  /* largest T of one eigen_attn_prefill call (sizes its scratch); 0 = none */
+  const int32_t* r_k;          /* HOST [H]: rank of U^K per head, 1..d_head                           */
+  const int32_t* r_v;          /* HOST [H] or NULL (= r_k): rank of U^V per head                      */
+  const float* U_k;            /* HOST fp32, heads back to back; head h is row-major d_head x r_k[h], */
+  const float* U_v;            /*   columns = basis vectors u_1..u_r (Section 4.1)                    */
+  uint32_t flags;
+} ea_desc;
+
+/* Cache rows are padded to rp = 8*ceil(r/8) elements; padding columns hold zeros. */
+
+/* Sizes of the two device buffers the caller must provide for this layer.  Pure host arithmetic. */
+ea_status eigen_attn_cache_bytes(const ea_desc* desc, size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Builds a handle: validates desc, pads and uploads the bases into the workspace (synchronises
+ * `cuda_stream` before returning; desc's host arrays are not retained), sets len = 0.
+ * d_cache and d_workspace must be 256-byte aligned and stay valid for the life of the handle. */
+ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_bytes,
+                            void* d_workspace, size_t workspace_bytes,
+                            void* cuda_stream, eigen_attn_t* out);
+
+/* Frees host memory only.  NULL is allowed. */
+void eigen_attn_destroy(eigen_attn_t h);
+
+/* Section 2 (generation phase) + Eq. 6: project T new rows per sequence and write them at rows
+ * len..len+T-1 of the rank-r cache; then len += T.  d_k, d_v: [B][T][H][d_head].
+ * flags: EA_KV_PREPROJECTED. */
+ea_status eigen_attn_append_kv(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
+                               int64_t stride_b, int64_t stride_t, uint32_t flags, void* cuda_stream);
+
+/* Eq. 3 in the rank-r space of Eq. 7: one query per sequence against rows [0, len).  Call it after
+ * the append of the same token (the new token attends to itself).  d_q, d_out: [B][1][H][d_head]
+ * with batch stride `stride_b`.  flags: EA_Q_PREPROJECTED, EA_OUT_LOWRANK.  len == 0 -> EA_ERR_SHAPE. */
+ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out,
+                            uint32_t flags, void* cuda_stream);
+
+/* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token). */
+ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
+                                 int64_t stride_b, void* d_out, uint32_t flags, void* cuda_stream);
+
+/* The same step for HOST tensors (contiguous [B][1][H][d_head], ideally pinned): copies q, k, v to a
+ * staging area of the workspace, runs the step, copies the result back and synchronises the stream. */
+ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const void* h_k, const void* h_v,
+                                      void* h_out, uint32_t flags, void* cuda_stream);
+
+/* Section 2 (prefill phase) with Eq. 7 and a causal mask: append T rows (as eigen_attn_append_kv) and
+ * compute the attention output of the T queries, query t over rows [0, len0 + t] where len0 is the
+ * length before the call.  T <= max_prefill_tokens.  d_q, d_k, d_v, d_out: [B][T][H][d_head].
+ * flags: EA_OUT_LOWRANK. */
+ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
+                             int32_t T, int64_t stride_b, int64_t stride_t, void* d_out,
+                             uint32_t flags, void* cuda_stream);
+
+/* Current number of cached rows; set_len truncates or rewinds (0 <= len <= n_max), e.g. to re-run
+ * a step at a fixed context length.  Rows beyond the previous length hold whatever was last written. */
+ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len);
+ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
+
+/* Synchronises the stream and returns the device status word (EA_OK or EA_ERR_TIMEOUT), then clears it. */
+ea_status eigen_attn_poll_status(eigen_attn_t h, void* cuda_stream);
+
+/* Text of the last error of this handle (never NULL; valid until the next call on the handle). */
+const char* eigen_attn_last_error(eigen_attn_t h);
+
+/* Element offsets of each head inside the packed low-rank vectors used by the *_PREPROJECTED and
+ * EA_OUT_LOWRANK flags: prefix sums of rp_k / rp_v.  offs arrays: HOST [H+1] (last = total width). */
+ea_status eigen_attn_head_offsets(eigen_attn_t h, int32_t* offs_k, int32_t* offs_v);
+
+/* Where head `head` lives in the cache buffer: byte offsets of its K' and V' slabs, each laid out
+ * [B][n_max][rp] row-major in the cache dtype, and the padded widths. */
+ea_status eigen_attn_cache_layout(eigen_attn_t h, int32_t head, size_t* k_offset, size_t* v_offset,
+                                  int32_t* rp_k, int32_t* rp_v);
+
+/* Tuning / instrumentation knobs (all optional). */
+typedef enum {
+  EA_OPT_DECODE_CTAS = 1,     /* CTAs of the split-KV decode kernel; 0 = one per SM                      */
+  EA_OPT_DECODE_TILE_ROWS = 2,/* rows per shared-memory tile (multiple of 16, <= 128); 0 = automatic     */
+  EA_OPT_DECODE_STAGES = 3,   /* depth of the shared-memory ring (2..12); 0 = as many as fit              */
+  EA_OPT_PREFILL_IMPL = 4     /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel      */
+} ea_option;
+ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value);
+
+/* Number of kernels this handle has launched since create. */
+ea_status eigen_attn_launch_count(eigen_attn_t h, uint64_t* count);
+
+/* If both are non-NULL cudaEvent_t handles, every later decode records `start` immediately before
+ * and `stop` immediately after the split-KV attention kernel on the call's stream (NULL, NULL = off). */
+ea_status eigen_attn_set_decode_events(eigen_attn_t h, void* start_event, void* stop_event);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int32_t eigen_attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* EIGEN_ATTN_H_ */

@@ -1,0 +1,497 @@
+// Host side of libeigenattn: the C ABI declared in include/eigen_attn.h.  Validates arguments,
+// lays out the cache and the workspace, plans each launch and calls the kernels.  No device memory is
+// allocated here: the cache and the workspace belong to the caller.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/eigen_attn.h"
+#include "internal.h"
+
+using ea::HeadInfo;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxDecodeCtas = 1024;
+constexpr int kSmemLimit = 227 * 1024;
+
+size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+int ceil8(int r) { return (r + 7) / 8 * 8; }
+
+struct Layout {
+  std::vector<HeadInfo> heads;
+  size_t cache_bytes = 0;
+  // workspace
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_staging = 0, off_qp = 0;
+  size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
+  int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
+  int part_stride = 0;
+  int64_t sum_w = 0;
+  int es = 2;
+};
+
+ea_status check_desc(const ea_desc* d) {
+  if (!d || !d->r_k) return EA_ERR_INVALID_ARG;
+  if (d->dtype != EA_BF16 && d->dtype != EA_FP32) return EA_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->n_heads < 1 || d->n_heads > ea::kMaxHeads || d->n_max < 1) return EA_ERR_SHAPE;
+  if (d->d_head < 8 || d->d_head > 128 || d->d_head % 8) return EA_ERR_SHAPE;
+  if (d->max_prefill_tokens < 0 || d->max_prefill_tokens > d->n_max) return EA_ERR_SHAPE;
+  for (int h = 0; h < d->n_heads; ++h) {
+    const int rk = d->r_k[h], rv = d->r_v ? d->r_v[h] : d->r_k[h];
+    if (rk < 1 || rk > d->d_head || rv < 1 || rv > d->d_head) return EA_ERR_SHAPE;
+  }
+  if (static_cast<int64_t>(d->batch) * d->n_max > (1ll << 40)) return EA_ERR_SHAPE;
+  return EA_OK;
+}
+
+void make_layout(const ea_desc* d, Layout* L) {
+  const int H = d->n_heads, dh = d->d_head;
+  L->es = d->dtype == EA_BF16 ? 2 : 4;
+  L->heads.resize(H);
+  size_t cache = 0, basis = 0;
+  int64_t wsum = 0;
+  int lk = 0, lv = 0;
+  for (int h = 0; h < H; ++h) {
+    HeadInfo& hi = L->heads[h];
+    memset(&hi, 0, sizeof(hi));
+    hi.r_k = d->r_k[h];
+    hi.r_v = d->r_v ? d->r_v[h] : d->r_k[h];
+    hi.rp_k = ceil8(hi.r_k);
+    hi.rp_v = ceil8(hi.r_v);
+    hi.k_off = static_cast<int64_t>(cache);
+    cache = align_up(cache + static_cast<size_t>(d->batch) * d->n_max * hi.rp_k * L->es);
+    hi.v_off = static_cast<int64_t>(cache);
+    cache = align_up(cache + static_cast<size_t>(d->batch) * d->n_max * hi.rp_v * L->es);
+    hi.uk_off = static_cast<int32_t>(basis);  basis += static_cast<size_t>(dh) * hi.rp_k;
+    hi.uv_off = static_cast<int32_t>(basis);  basis += static_cast<size_t>(dh) * hi.rp_v;
+    hi.uvt_off = static_cast<int32_t>(basis); basis += static_cast<size_t>(dh) * hi.rp_v;
+    hi.lr_k_off = lk; lk += hi.rp_k;
+    hi.lr_v_off = lv; lv += hi.rp_v;
+    hi.w_prefix = wsum; wsum += hi.rp_k + hi.rp_v;
+    if (hi.rp_k > L->max_rp_k) L->max_rp_k = hi.rp_k;
+    if (hi.rp_v > L->max_rp_v) L->max_rp_v = hi.rp_v;
+    if (hi.rp_k + hi.rp_v > L->max_w) L->max_w = hi.rp_k + hi.rp_v;
+  }
+  L->cache_bytes = cache;
+  L->basis_floats = basis;
+  L->sum_rp_k = lk; L->sum_rp_v = lv; L->sum_w = wsum;
+  L->part_stride = 4 + L->max_rp_v;
+  size_t off = 0;
+  L->off_status = off;   off = align_up(off + 64);
+  L->off_heads = off;    off = align_up(off + sizeof(HeadInfo) * H);
+  L->off_basis = off;    off = align_up(off + basis * sizeof(float));
+  L->off_partials = off;
+  off = align_up(off + (static_cast<size_t>(d->batch) * H + kMaxDecodeCtas) * L->part_stride * sizeof(float));
+  L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
+  L->off_staging = off;  off += 4 * L->staging_each;
+  L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
+  L->workspace_bytes = off;
+}
+
+}  // namespace
+
+struct eigen_attn {
+  ea_desc desc;           // the host array pointers are cleared after create
+  Layout L;
+  char* cache = nullptr;
+  char* ws = nullptr;
+  int32_t len = 0;
+  int sm_count = 148;
+  int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0;
+  uint64_t launches = 0;
+  cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  char err[256];
+};
+
+namespace {
+
+ea_status fail(eigen_attn_t h, ea_status st, const char* fmt, ...) {
+  if (h) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(h->err, sizeof(h->err), fmt, ap);
+    va_end(ap);
+  }
+  return st;
+}
+ea_status cuda_fail(eigen_attn_t h, cudaError_t e, const char* what) {
+  return fail(h, EA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+const HeadInfo* dev_heads(eigen_attn_t h) { return reinterpret_cast<const HeadInfo*>(h->ws + h->L.off_heads); }
+const float* dev_basis(eigen_attn_t h) { return reinterpret_cast<const float*>(h->ws + h->L.off_basis); }
+int* dev_status(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_status); }
+
+ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T, int64_t stride_b,
+                    int64_t stride_t, uint32_t flags, cudaStream_t s) {
+  if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "append_kv: NULL k or v");
+  if (flags & ~EA_KV_PREPROJECTED) return fail(h, EA_ERR_INVALID_ARG, "append_kv: unknown flag 0x%x", flags);
+  if (T < 1) return fail(h, EA_ERR_SHAPE, "append_kv: T = %d", T);
+  if (static_cast<int64_t>(h->len) + T > h->desc.n_max)
+    return fail(h, EA_ERR_CAPACITY, "append_kv: len %d + T %d exceeds n_max %d", h->len, T, h->desc.n_max);
+  ea::ProjectParams p{};
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.k = d_k; p.v = d_v; p.cache = h->cache;
+  p.stride_b = stride_b; p.stride_t = stride_t;
+  p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head;
+  p.n_max = h->desc.n_max; p.row0 = h->len; p.flags = flags;
+  const cudaError_t e = ea::launch_project_append(p, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "append_kv launch");
+  h->len += T;
+  return EA_OK;
+}
+
+ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, uint32_t flags,
+                    cudaStream_t s) {
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
+    return fail(h, EA_ERR_INVALID_ARG, "decode: unknown flag 0x%x", flags);
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
+  const Layout& L = h->L;
+  const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
+  const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
+  const int sms = h->opt_ctas > 0 ? static_cast<int>(h->opt_ctas) : h->sm_count;
+
+  // rows per tile: 128 unless the context is short (keep a few tiles per CTA) or a stage would be too big
+  int tile_rows = 128;
+  if (h->opt_tile_rows > 0) {
+    tile_rows = static_cast<int>(h->opt_tile_rows);
+  } else {
+    while (tile_rows > 16 && static_cast<int64_t>(B) * H * ((n + tile_rows - 1) / tile_rows) < 4ll * sms)
+      tile_rows >>= 1;
+  }
+  int stage_bytes = 0, stages = 0;
+  for (;;) {
+    stage_bytes = static_cast<int>(align_up(static_cast<size_t>(tile_rows) * (L.max_rp_k + L.max_rp_v) * L.es, 128));
+    stages = (kSmemLimit - fixed) / stage_bytes;
+    if (stages >= 3 || tile_rows <= 16) break;
+    tile_rows >>= 1;
+  }
+  if (stages > 12) stages = 12;
+  if (h->opt_stages > 0 && h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
+  if (stages < 1)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode: a tile of %d rows does not fit in shared memory", tile_rows);
+
+  const int nt = (n + tile_rows - 1) / tile_rows;
+  const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
+  int grid = sms;
+  const int64_t cap = w_total / L.max_w;          // every CTA must own at least one tile
+  if (grid > cap) grid = static_cast<int>(cap);
+  if (grid < 1) grid = 1;
+
+  ea::DecodeParams p{};
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
+  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b;
+  p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
+  p.status = dev_status(h);
+  p.part_stride = L.part_stride;
+  p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
+  p.tile_rows = tile_rows; p.nt = nt; p.stages = stages; p.stage_bytes = stage_bytes;
+  p.v_tile_off = tile_rows * L.max_rp_k * L.es;
+  p.w_total = w_total;
+  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  p.flags = flags;
+  const size_t smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
+
+  if (h->ev_start) cudaEventRecord(h->ev_start, s);
+  cudaError_t e = ea::launch_decode(p, h->desc.dtype, grid, smem, s, &h->launches);
+  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode launch");
+
+  ea::CombineParams c{};
+  c.heads = p.heads; c.basis = p.basis; c.partials = p.partials; c.out = d_out;
+  c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b;
+  c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
+  c.w_total = w_total; c.flags = flags;
+  e = ea::launch_combine(c, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "combine launch");
+  return EA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t eigen_attn_version(void) { return 100; }
+
+ea_status eigen_attn_cache_bytes(const ea_desc* desc, size_t* cache_bytes, size_t* workspace_bytes) {
+  if (!cache_bytes || !workspace_bytes) return EA_ERR_INVALID_ARG;
+  const ea_status st = check_desc(desc);
+  if (st != EA_OK) return st;
+  Layout L;
+  make_layout(desc, &L);
+  *cache_bytes = L.cache_bytes;
+  *workspace_bytes = L.workspace_bytes;
+  return EA_OK;
+}
+
+ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_bytes, void* d_workspace,
+                            size_t workspace_bytes, void* cuda_stream, eigen_attn_t* out) {
+  if (!out) return EA_ERR_INVALID_ARG;
+  *out = nullptr;
+  ea_status st = check_desc(desc);
+  if (st != EA_OK) return st;
+  if (!desc->U_k || !desc->U_v || !d_cache || !d_workspace) return EA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_cache) % kAlign) || (reinterpret_cast<uintptr_t>(d_workspace) % kAlign))
+    return EA_ERR_INVALID_ARG;
+  eigen_attn* h = new (std::nothrow) eigen_attn();
+  if (!h) return EA_ERR_INVALID_ARG;
+  h->err[0] = 0;
+  h->desc = *desc;
+  make_layout(desc, &h->L);
+  const Layout& L = h->L;
+  if (cache_bytes < L.cache_bytes || workspace_bytes < L.workspace_bytes) {
+    delete h;
+    return EA_ERR_CAPACITY;
+  }
+  const int H = desc->n_heads, dh = desc->d_head;
+
+  // pad the bases (zero columns), build (U^V)^T, optionally check orthonormality
+  std::vector<float> basis(L.basis_floats, 0.f);
+  const float* uk = desc->U_k;
+  const float* uv = desc->U_v;
+  for (int hh = 0; hh < H; ++hh) {
+    const HeadInfo& hi = L.heads[hh];
+    for (int d = 0; d < dh; ++d) {
+      for (int c = 0; c < hi.r_k; ++c)
+        basis[hi.uk_off + static_cast<size_t>(d) * hi.rp_k + c] = uk[static_cast<size_t>(d) * hi.r_k + c];
+      for (int c = 0; c < hi.r_v; ++c) {
+        const float x = uv[static_cast<size_t>(d) * hi.r_v + c];
+        basis[hi.uv_off + static_cast<size_t>(d) * hi.rp_v + c] = x;
+        basis[hi.uvt_off + static_cast<size_t>(c) * dh + d] = x;
+      }
+    }
+    if (desc->flags & EA_CHECK_ORTHONORMAL) {
+      for (int pass = 0; pass < 2; ++pass) {
+        const float* U = pass ? uv : uk;
+        const int r = pass ? hi.r_v : hi.r_k;
+        for (int a = 0; a < r; ++a)
+          for (int b = a; b < r; ++b) {
+            double dot = 0;
+            for (int d = 0; d < dh; ++d)
+              dot += static_cast<double>(U[static_cast<size_t>(d) * r + a]) * U[static_cast<size_t>(d) * r + b];
+            if (fabs(dot - (a == b ? 1.0 : 0.0)) > 1e-4) {
+              delete h;
+              return EA_ERR_NOT_ORTHONORMAL;
+            }
+          }
+      }
+    }
+    uk += static_cast<size_t>(dh) * hi.r_k;
+    uv += static_cast<size_t>(dh) * hi.r_v;
+  }
+  h->cache = static_cast<char*>(d_cache);
+  h->ws = static_cast<char*>(d_workspace);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemsetAsync(h->ws + L.off_status, 0, 64, s);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(h->ws + L.off_heads, L.heads.data(), sizeof(HeadInfo) * H, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(h->ws + L.off_basis, basis.data(), basis.size() * sizeof(float), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  int dev = 0;
+  if (e == cudaSuccess) e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = ea::decode_configure(desc->dtype);
+  if (e != cudaSuccess) {
+    delete h;
+    return EA_ERR_CUDA;
+  }
+  h->desc.r_k = nullptr; h->desc.r_v = nullptr; h->desc.U_k = nullptr; h->desc.U_v = nullptr;
+  h->len = 0;
+  *out = h;
+  return EA_OK;
+}
+
+void eigen_attn_destroy(eigen_attn_t h) { delete h; }
+
+ea_status eigen_attn_append_kv(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T, int64_t stride_b,
+                               int64_t stride_t, uint32_t flags, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  return do_append(h, d_k, d_v, T, stride_b, stride_t, flags, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, uint32_t flags,
+                            void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  return do_decode(h, d_q, stride_b, d_out, flags, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
+                                 int64_t stride_b, void* d_out, uint32_t flags, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL q or out");
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
+    return fail(h, EA_ERR_INVALID_ARG, "decode_step: unknown flag 0x%x", flags);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const ea_status st = do_append(h, d_k, d_v, 1, stride_b, stride_b, 0, s);
+  if (st != EA_OK) return st;
+  return do_decode(h, d_q, stride_b, d_out, flags, s);
+}
+
+ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const void* h_k, const void* h_v,
+                                      void* h_out, uint32_t flags, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!h_q || !h_k || !h_v || !h_out) return fail(h, EA_ERR_INVALID_ARG, "decode_step_host: NULL buffer");
+  if (flags) return fail(h, EA_ERR_INVALID_ARG, "decode_step_host: flags must be 0");
+  if (h->len + 1 > h->desc.n_max) return fail(h, EA_ERR_CAPACITY, "decode_step_host: cache full");
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const Layout& L = h->L;
+  const size_t bytes = static_cast<size_t>(h->desc.batch) * h->desc.n_heads * h->desc.d_head * L.es;
+  char* sq = h->ws + L.off_staging;
+  char* sk = sq + L.staging_each;
+  char* sv = sk + L.staging_each;
+  char* so = sv + L.staging_each;
+  cudaError_t e = cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(sk, h_k, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(sv, h_v, bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_step_host H2D");
+  const int64_t sb = static_cast<int64_t>(h->desc.n_heads) * h->desc.d_head;
+  ea_status st = do_append(h, sk, sv, 1, sb, sb, 0, s);
+  if (st != EA_OK) return st;
+  st = do_decode(h, sq, sb, so, 0, s);
+  if (st != EA_OK) return st;
+  e = cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_step_host D2H");
+  return EA_OK;
+}
+
+ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v, int32_t T,
+                             int64_t stride_b, int64_t stride_t, void* d_out, uint32_t flags,
+                             void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
+  if (flags & ~EA_OUT_LOWRANK) return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
+  if (T < 1) return fail(h, EA_ERR_SHAPE, "prefill: T = %d", T);
+  if (T > h->desc.max_prefill_tokens)
+    return fail(h, EA_ERR_CAPACITY, "prefill: T %d exceeds max_prefill_tokens %d", T, h->desc.max_prefill_tokens);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int len0 = h->len;
+  const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, 0, s);
+  if (st != EA_OK) return st;
+  const Layout& L = h->L;
+  ea::QProjectParams qp{};
+  qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
+  qp.stride_b = stride_b; qp.stride_t = stride_t;
+  qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
+  cudaError_t e = ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "prefill q projection launch");
+  ea::PrefillParams p{};
+  p.heads = qp.heads; p.basis = qp.basis; p.cache = h->cache; p.qp = qp.qp; p.out = d_out;
+  if (flags & EA_OUT_LOWRANK) {
+    p.out_stride_t = L.sum_rp_v;
+    p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
+  } else {
+    p.out_stride_b = stride_b; p.out_stride_t = stride_t;
+  }
+  p.B = qp.B; p.T = T; p.H = qp.H; p.d_head = qp.d_head; p.n_max = h->desc.n_max; p.len0 = len0;
+  p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
+  p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  p.flags = flags; p.status = dev_status(h);
+  e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch");
+  return EA_OK;
+}
+
+ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len) {
+  if (!h || !len) return EA_ERR_INVALID_ARG;
+  *len = h->len;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (len < 0 || len > h->desc.n_max)
+    return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %d]", len, h->desc.n_max);
+  h->len = len;
+  return EA_OK;
+}
+
+ea_status eigen_attn_poll_status(eigen_attn_t h, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, dev_status(h), sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(dev_status(h), 0, sizeof(int), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "poll_status");
+  if (word == ea::kStatusTimeout) return fail(h, EA_ERR_TIMEOUT, "a device-side wait exceeded its bound");
+  return EA_OK;
+}
+
+const char* eigen_attn_last_error(eigen_attn_t h) { return h ? h->err : "null handle"; }
+
+ea_status eigen_attn_head_offsets(eigen_attn_t h, int32_t* offs_k, int32_t* offs_v) {
+  if (!h || !offs_k || !offs_v) return EA_ERR_INVALID_ARG;
+  const int H = h->desc.n_heads;
+  for (int i = 0; i < H; ++i) {
+    offs_k[i] = h->L.heads[i].lr_k_off;
+    offs_v[i] = h->L.heads[i].lr_v_off;
+  }
+  offs_k[H] = h->L.sum_rp_k;
+  offs_v[H] = h->L.sum_rp_v;
+  return EA_OK;
+}
+
+ea_status eigen_attn_cache_layout(eigen_attn_t h, int32_t head, size_t* k_offset, size_t* v_offset,
+                                  int32_t* rp_k, int32_t* rp_v) {
+  if (!h || !k_offset || !v_offset || !rp_k || !rp_v) return EA_ERR_INVALID_ARG;
+  if (head < 0 || head >= h->desc.n_heads) return fail(h, EA_ERR_SHAPE, "cache_layout: head %d", head);
+  const HeadInfo& hi = h->L.heads[head];
+  *k_offset = static_cast<size_t>(hi.k_off);
+  *v_offset = static_cast<size_t>(hi.v_off);
+  *rp_k = hi.rp_k;
+  *rp_v = hi.rp_v;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  switch (option) {
+    case EA_OPT_DECODE_CTAS:
+      if (value < 0 || value > kMaxDecodeCtas)
+        return fail(h, EA_ERR_INVALID_ARG, "DECODE_CTAS %lld", static_cast<long long>(value));
+      h->opt_ctas = value;
+      return EA_OK;
+    case EA_OPT_DECODE_TILE_ROWS:
+      if (value < 0 || value > 128 || value % 16)
+        return fail(h, EA_ERR_INVALID_ARG, "DECODE_TILE_ROWS %lld", static_cast<long long>(value));
+      h->opt_tile_rows = value;
+      return EA_OK;
+    case EA_OPT_DECODE_STAGES:
+      if (value != 0 && (value < 2 || value > 12))
+        return fail(h, EA_ERR_INVALID_ARG, "DECODE_STAGES %lld", static_cast<long long>(value));
+      h->opt_stages = value;
+      return EA_OK;
+    case EA_OPT_PREFILL_IMPL:
+      if (value < 0 || value > 2)
+        return fail(h, EA_ERR_INVALID_ARG, "PREFILL_IMPL %lld", static_cast<long long>(value));
+      h->opt_prefill = value;
+      return EA_OK;
+    default:
+      return fail(h, EA_ERR_INVALID_ARG, "unknown option %d", option);
+  }
+}
+
+ea_status eigen_attn_launch_count(eigen_attn_t h, uint64_t* count) {
+  if (!h || !count) return EA_ERR_INVALID_ARG;
+  *count = h->launches;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_decode_events(eigen_attn_t h, void* start_event, void* stop_event) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if ((start_event == nullptr) != (stop_event == nullptr))
+    return fail(h, EA_ERR_INVALID_ARG, "set_decode_events: pass both or neither");
+  h->ev_start = static_cast<cudaEvent_t>(start_event);
+  h->ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return EA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,494 @@
+// Split-KV decode attention in the rank-r space (Eq. 3 of the paper evaluated in the space of Eq. 7)
+// and the cross-split combine + lift through (U^V)^T.
+//
+// Kernel 1 (decode_splitkv_kernel): persistent CTAs, one per SM.  The (head, sequence) units are laid
+// end to end as a list of row tiles weighted by their bytes (rp_k + rp_v per row); every CTA takes an
+// equal share of that weight, i.e. a contiguous run of tiles that may start and end inside a unit.
+// One producer thread streams the K' and V' tiles of the run from HBM into a shared-memory ring with
+// bulk asynchronous copies (mbarrier completion); eight consumer warps take the scores, an online
+// softmax and the weighted sum of value rows from shared memory.  A lane pair owns one row of a tile.
+// For every (CTA, unit) piece the CTA writes an un-normalised partial (max, sum, o'[rp_v]).
+//
+// Kernel 2 (combine_lift_kernel): merges the partials of a unit (exact re-association of the
+// softmax), normalises, multiplies by (U^V)^T and stores the d_head-wide output.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace ea {
+namespace {
+
+constexpr int kMaxStages = 12;
+constexpr uint64_t kWaitBoundNs = 2000000000ull;   // every device-side wait gives up after 2 s
+
+struct __align__(128) DecodeSmemFixed {
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
+  long long range[2];
+  int abort_flag;
+  int pad_[3];
+  float qraw[128];
+  float qpart[4][128];
+  float qp[128];
+  float wmax[kDecodeConsumerWarps];
+  float wsum[kDecodeConsumerWarps];
+  float stage_o[kDecodeConsumerWarps][4][128];
+};
+
+// ---------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false (and the status word set) if the phase did not complete within the bound.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kWaitBoundNs) {
+      atomicExch(status, kStatusTimeout);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, void* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void consumer_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerWarps * 32) : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------- element access
+
+template <typename T>
+struct Elem;
+template <>
+struct Elem<__nv_bfloat16> {
+  static constexpr int kPerChunk = 8;   // elements in 16 bytes
+  static __device__ __forceinline__ void load_chunk(const unsigned char* p, float (&f)[8]) {
+    const uint4 x = *reinterpret_cast<const uint4*>(p);
+    f[0] = __uint_as_float(x.x << 16); f[1] = __uint_as_float(x.x & 0xffff0000u);
+    f[2] = __uint_as_float(x.y << 16); f[3] = __uint_as_float(x.y & 0xffff0000u);
+    f[4] = __uint_as_float(x.z << 16); f[5] = __uint_as_float(x.z & 0xffff0000u);
+    f[6] = __uint_as_float(x.w << 16); f[7] = __uint_as_float(x.w & 0xffff0000u);
+  }
+  static __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ __nv_bfloat16 from_float(float v) { return __float2bfloat16_rn(v); }
+};
+template <>
+struct Elem<float> {
+  static constexpr int kPerChunk = 4;
+  static __device__ __forceinline__ void load_chunk(const unsigned char* p, float (&f)[4]) {
+    const float4 x = *reinterpret_cast<const float4*>(p);
+    f[0] = x.x; f[1] = x.y; f[2] = x.z; f[3] = x.w;
+  }
+  static __device__ __forceinline__ float to_float(float v) { return v; }
+  static __device__ __forceinline__ float from_float(float v) { return v; }
+};
+
+// ---------------------------------------------------------------- work decomposition
+
+// First tile (in the flat order head-major, then sequence, then tile) whose start weight x
+// satisfies x * grid >= c * w_total.  Tiles of head h weigh (rp_k + rp_v).
+__device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
+  const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
+  if (c >= grid) return per_head_tiles * p.H;
+  const long long num = static_cast<long long>(c) * p.w_total;
+  const long long target = (num + grid - 1) / grid;
+  int h = 0;
+  for (int j = 1; j < p.H; ++j)
+    if (per_head_tiles * p.heads[j].w_prefix <= target) h = j;
+  const long long base = per_head_tiles * p.heads[h].w_prefix;
+  const long long w = p.heads[h].rp_k + p.heads[h].rp_v;
+  long long idx = (target - base + w - 1) / w;
+  if (idx > per_head_tiles) idx = per_head_tiles;
+  return per_head_tiles * h + idx;
+}
+
+// ---------------------------------------------------------------- one (CTA, unit) piece
+
+template <typename T, int NCH>
+__device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
+                                            unsigned char* ring, const HeadInfo& hd, int i0, int i1,
+                                            uint32_t& it, int warp, int lane, int slot) {
+  constexpr int EPC = Elem<T>::kPerChunk;
+  const int pair = lane >> 1, half = lane & 1;
+  const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
+  const int rowb_v = hd.rp_v * static_cast<int>(sizeof(T));
+  const int nch_k = rowb_k >> 4, nch_v = rowb_v >> 4;
+
+  // Chunk rotation that spreads the four lane pairs of a quarter warp over all banks when the
+  // row pitch is a multiple of 64 bytes.
+  auto rotation = [&](int rowb) {
+    const int s = (rowb >> 2) & 31;
+    return s == 0 ? (pair & 3) : (s == 16 ? ((pair >> 1) & 1) : 0);
+  };
+  const int rot_k = rotation(rowb_k), rot_v = rotation(rowb_v);
+
+  int off_k[NCH], off_v[NCH];
+  float q[NCH][EPC];
+  float o[NCH][EPC];
+#pragma unroll
+  for (int j = 0; j < NCH; ++j) {
+    const int ck = ((j ^ rot_k) << 1) + half;
+    const int cv = ((j ^ rot_v) << 1) + half;
+    const bool vk = ck < nch_k;
+    off_k[j] = vk ? (ck << 4) : 0;
+    off_v[j] = cv < nch_v ? (cv << 4) : 0;
+#pragma unroll
+    for (int e = 0; e < EPC; ++e) {
+      q[j][e] = vk ? fx->qp[ck * EPC + e] : 0.f;
+      o[j][e] = 0.f;
+    }
+  }
+
+  volatile int* abort_flag = &fx->abort_flag;
+  float m = -INFINITY, l = 0.f;
+  for (int i = i0; i < i1; ++i) {
+    const int stage = it % p.stages;
+    const uint32_t parity = (it / p.stages) & 1u;
+    ++it;
+    if (*abort_flag) continue;
+    if (!mbar_wait(&fx->full[stage], parity, p.status)) {
+      *abort_flag = 1;
+      continue;
+    }
+    const unsigned char* kt = ring + static_cast<size_t>(stage) * p.stage_bytes;
+    const unsigned char* vt = kt + p.v_tile_off;
+    const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
+    for (int row = warp * 16 + pair; row < rows; row += kDecodeConsumerWarps * 16) {
+      const unsigned char* kr = kt + row * rowb_k;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+      for (int j = 0; j < NCH; ++j) {
+        float x[EPC];
+        Elem<T>::load_chunk(kr + off_k[j], x);
+#pragma unroll
+        for (int e = 0; e < EPC; e += 4) {
+          a0 = fmaf(x[e + 0], q[j][e + 0], a0); a1 = fmaf(x[e + 1], q[j][e + 1], a1);
+          a2 = fmaf(x[e + 2], q[j][e + 2], a2); a3 = fmaf(x[e + 3], q[j][e + 3], a3);
+        }
+      }
+      float s = (a0 + a1) + (a2 + a3);
+      s += __shfl_xor_sync(0xffffffffu, s, 1);
+      if (s > m) {                      // rare after the first rows: rescale the running state
+        const float c = fast_exp2(m - s);
+        l *= c;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j)
+#pragma unroll
+          for (int e = 0; e < EPC; ++e) o[j][e] *= c;
+        m = s;
+      }
+      const float pr = fast_exp2(s - m);
+      l += pr;
+      const unsigned char* vr = vt + row * rowb_v;
+#pragma unroll
+      for (int j = 0; j < NCH; ++j) {
+        float x[EPC];
+        Elem<T>::load_chunk(vr + off_v[j], x);
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, x[e], o[j][e]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&fx->empty[stage]);
+  }
+
+  // ---- merge the 128 lane pairs of the CTA into one partial
+  float wm = m;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+  if (lane == 0) fx->wmax[warp] = wm;
+  consumer_sync();
+  float M = fx->wmax[0];
+#pragma unroll
+  for (int w = 1; w < kDecodeConsumerWarps; ++w) M = fmaxf(M, fx->wmax[w]);
+  const float f = (m == -INFINITY) ? 0.f : fast_exp2(m - M);
+  float ls = half == 0 ? l * f : 0.f;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+  if (lane == 0) fx->wsum[warp] = ls;
+#pragma unroll
+  for (int j = 0; j < NCH; ++j)
+#pragma unroll
+    for (int e = 0; e < EPC; ++e) {
+      float v = o[j][e] * f;
+      v += __shfl_xor_sync(0xffffffffu, v, 8);    // pairs p, p+4, p+8, p+12 hold the same columns
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      o[j][e] = v;
+    }
+  if (lane < 8) {
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      const int cv = ((j ^ rot_v) << 1) + half;
+      if (cv < nch_v) {
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) fx->stage_o[warp][pair][cv * EPC + e] = o[j][e];
+      }
+    }
+  }
+  consumer_sync();
+  const int t = warp * 32 + lane;
+  float* part = p.partials + static_cast<size_t>(slot) * p.part_stride;
+  if (t < hd.rp_v) {
+    float acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecodeConsumerWarps; ++w)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc += fx->stage_o[w][c][t];
+    part[4 + t] = acc;
+  }
+  if (t == 0) {
+    float L = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecodeConsumerWarps; ++w) L += fx->wsum[w];
+    part[0] = M;
+    part[1] = L;
+  }
+  consumer_sync();   // the staging area and q' are reused by the next piece
+}
+
+// q' = q U^K * log2(e)/sqrt(d_head) for one unit, left in fx->qp (all consumer threads take part).
+template <typename T>
+__device__ __forceinline__ void project_query(const DecodeParams& p, DecodeSmemFixed* fx,
+                                              const HeadInfo& hd, int h, int b, int t) {
+  const T* q = static_cast<const T*>(p.q);
+  const int rp = hd.rp_k;
+  if (p.flags & 0x1u) {   // rank-space query supplied by the caller (merged W^Q')
+    if (t < rp) fx->qp[t] = Elem<T>::to_float(q[b * p.q_stride_b + hd.lr_k_off + t]) * p.q_scale;
+    consumer_sync();
+    return;
+  }
+  const int d_head = p.d_head;
+  if (t < d_head) fx->qraw[t] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + t]);
+  consumer_sync();
+  const int nthreads = kDecodeConsumerWarps * 32;
+  int ngrp = nthreads / rp;
+  if (ngrp > 4) ngrp = 4;
+  const int g = t / rp, c = t - g * rp;
+  if (g < ngrp) {
+    const int per = (d_head + ngrp - 1) / ngrp;
+    const int d0 = g * per, d1 = min(d_head, d0 + per);
+    const float* U = p.basis + hd.uk_off;
+    float acc = 0.f;
+#pragma unroll 8
+    for (int d = d0; d < d1; ++d) acc = fmaf(fx->qraw[d], __ldg(U + d * rp + c), acc);
+    fx->qpart[g][c] = acc;
+  }
+  consumer_sync();
+  if (t < rp) {
+    float acc = 0.f;
+    for (int gg = 0; gg < ngrp; ++gg) acc += fx->qpart[gg][t];
+    fx->qp[t] = acc * p.q_scale;
+  }
+  consumer_sync();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const DecodeParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  DecodeSmemFixed* fx = reinterpret_cast<DecodeSmemFixed*>(smem_raw);
+  unsigned char* ring = smem_raw + sizeof(DecodeSmemFixed);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int grid = gridDim.x, cta = blockIdx.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&fx->full[s], 1);
+      mbar_init(&fx->empty[s], kDecodeConsumerWarps);
+    }
+    fx->abort_flag = 0;
+    fx->range[0] = first_tile_of_cta(p, grid, cta);
+    fx->range[1] = first_tile_of_cta(p, grid, cta + 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const long long f_lo = fx->range[0], f_hi = fx->range[1];
+  volatile int* abort_flag = &fx->abort_flag;
+
+  if (warp == kDecodeConsumerWarps) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      int cur_h = -1;
+      HeadInfo hd{};
+      for (long long F = f_lo; F < f_hi; ++F, ++it) {
+        if (*abort_flag) break;
+        const int unit = static_cast<int>(F / p.nt);
+        const int i = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
+        const int h = unit / p.B, b = unit - h * p.B;
+        if (h != cur_h) { hd = p.heads[h]; cur_h = h; }
+        const int stage = it % p.stages;
+        const uint32_t k = it / p.stages;
+        if (k > 0 && !mbar_wait(&fx->empty[stage], (k - 1) & 1u, p.status)) {
+          *abort_flag = 1;
+          break;
+        }
+        const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
+        const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i) * p.tile_rows;
+        const uint32_t bytes_k = static_cast<uint32_t>(rows) * hd.rp_k * sizeof(T);
+        const uint32_t bytes_v = static_cast<uint32_t>(rows) * hd.rp_v * sizeof(T);
+        unsigned char* dst = ring + static_cast<size_t>(stage) * p.stage_bytes;
+        mbar_arrive_expect_tx(&fx->full[stage], bytes_k + bytes_v);
+        bulk_g2s(dst, p.cache + hd.k_off + row0 * hd.rp_k * sizeof(T), bytes_k, &fx->full[stage]);
+        bulk_g2s(dst + p.v_tile_off, p.cache + hd.v_off + row0 * hd.rp_v * sizeof(T), bytes_v,
+                 &fx->full[stage]);
+      }
+      // Make sure every copy this thread issued has landed before the CTA can exit.
+      const uint32_t first = it > static_cast<uint32_t>(p.stages) ? it - p.stages : 0u;
+      for (uint32_t j = first; j < it; ++j)
+        mbar_wait(&fx->full[j % p.stages], (j / p.stages) & 1u, p.status);
+    }
+  } else {
+    // ------------------------------------------------------------ consumers
+    uint32_t it = 0;
+    long long F = f_lo;
+    while (F < f_hi) {
+      const int unit = static_cast<int>(F / p.nt);
+      const int i0 = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
+      const long long left = f_hi - F;
+      const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + left));
+      const int h = unit / p.B, b = unit - h * p.B;
+      const HeadInfo hd = p.heads[h];
+      project_query<T>(p, fx, hd, h, b, tid);
+      const int slot = unit + cta;
+      const int mx = max(hd.rp_k, hd.rp_v);
+      const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
+      constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
+      switch (cls) {
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+      }
+      F += i1 - i0;
+    }
+  }
+  __syncthreads();
+}
+
+// ---------------------------------------------------------------- combine + lift
+
+// CTA that owns the tile with start weight x: floor(x * grid / w_total).
+__device__ __forceinline__ int owner_cta(long long x, int grid, long long w_total) {
+  return static_cast<int>((x * grid) / w_total);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) combine_lift_kernel(const CombineParams p) {
+  __shared__ float o_sm[128];
+  const int unit = blockIdx.x;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
+  const long long w = hd.rp_k + hd.rp_v;
+  const long long x0 = per_head_tiles * hd.w_prefix + static_cast<long long>(b) * p.nt * w;
+  const long long x1 = x0 + static_cast<long long>(p.nt - 1) * w;
+  const int c0 = owner_cta(x0, p.grid, p.w_total);
+  const int c1 = owner_cta(x1, p.grid, p.w_total);
+  const int t = threadIdx.x;
+
+  // global max and denominator (every thread computes them; the piece count is small)
+  float M = -INFINITY;
+  for (int c = c0; c <= c1; ++c)
+    M = fmaxf(M, p.partials[static_cast<size_t>(unit + c) * p.part_stride]);
+  float L = 0.f, acc = 0.f;
+  for (int c = c0; c <= c1; ++c) {
+    const float* part = p.partials + static_cast<size_t>(unit + c) * p.part_stride;
+    const float f = fast_exp2(part[0] - M);
+    L = fmaf(part[1], f, L);
+    if (t < hd.rp_v) acc = fmaf(part[4 + t], f, acc);
+  }
+  const float o = acc / L;
+  T* out = static_cast<T*>(p.out);
+  if (p.flags & 0x2u) {   // rank-space output for a merged W^O'
+    if (t < hd.rp_v) out[b * p.out_stride_b + hd.lr_v_off + t] = Elem<T>::from_float(o);
+    return;
+  }
+  if (t < hd.rp_v) o_sm[t] = o;
+  __syncthreads();
+  if (t < p.d_head) {
+    const float* Ut = p.basis + hd.uvt_off;   // (U^V)^T: rp_v x d_head
+    float y = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < hd.rp_v; ++c) y = fmaf(o_sm[c], __ldg(Ut + c * p.d_head + t), y);
+    out[b * p.out_stride_b + static_cast<int64_t>(h) * p.d_head + t] = Elem<T>::from_float(y);
+  }
+}
+
+}  // namespace
+
+size_t decode_fixed_smem_bytes() { return sizeof(DecodeSmemFixed); }
+
+cudaError_t decode_configure(int dtype) {
+  const int max_smem = 227 * 1024;
+  if (dtype == 0)
+    return cudaFuncSetAttribute(decode_splitkv_kernel<__nv_bfloat16>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+  return cudaFuncSetAttribute(decode_splitkv_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              max_smem);
+}
+
+cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t smem_bytes, cudaStream_t s,
+                          uint64_t* launches) {
+  if (dtype == 0)
+    decode_splitkv_kernel<__nv_bfloat16><<<grid, kDecodeThreads, smem_bytes, s>>>(p);
+  else
+    decode_splitkv_kernel<float><<<grid, kDecodeThreads, smem_bytes, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches) {
+  const int units = p.B * p.H;
+  if (dtype == 0)
+    combine_lift_kernel<__nv_bfloat16><<<units, 128, 0, s>>>(p);
+  else
+    combine_lift_kernel<float><<<units, 128, 0, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace ea

@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libeigenattn (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ea {
+
+// One entry per head, resident in the workspace; every kernel reads it.
+struct HeadInfo {
+  int64_t k_off;      // byte offset of the head's K' slab [B][n_max][rp_k] in the cache
+  int64_t v_off;      // byte offset of the head's V' slab [B][n_max][rp_v]
+  int64_t w_prefix;   // sum over earlier heads of (rp_k + rp_v): decode work weight prefix
+  int32_t r_k, r_v;   // ranks
+  int32_t rp_k, rp_v; // ranks padded to a multiple of 8
+  int32_t uk_off;     // float offset of U^K  (d_head x rp_k, row-major, zero padded) in the basis area
+  int32_t uv_off;     // float offset of U^V  (d_head x rp_v)
+  int32_t uvt_off;    // float offset of (U^V)^T (rp_v x d_head)
+  int32_t lr_k_off;   // element offset of the head in packed rank-space K/Q vectors (prefix of rp_k)
+  int32_t lr_v_off;   // same for V / O
+  int32_t pad_;
+};
+
+constexpr int kDecodeConsumerWarps = 8;
+constexpr int kDecodeThreads = (kDecodeConsumerWarps + 1) * 32;   // + one producer warp
+constexpr int kMaxHeads = 256;
+constexpr int kStatusTimeout = -6;
+
+struct DecodeParams {
+  const HeadInfo* heads;
+  const float* basis;       // basis area of the workspace
+  const char* cache;
+  const void* q;            // [B][1][H][d_head] or packed rank-space [B][sum rp_k]
+  int64_t q_stride_b;       // elements
+  float* partials;          // [(B*H + grid)][part_stride]: m, l, pad, pad, o'[rp_v]
+  int* status;
+  int32_t part_stride;      // floats per partial slot (multiple of 4)
+  int32_t B, H, d_head;
+  int32_t n;                // rows to attend
+  int32_t n_max;
+  int32_t tile_rows;        // rows per tile
+  int32_t nt;               // tiles per unit = ceil(n / tile_rows)
+  int32_t stages;
+  int32_t stage_bytes;      // bytes per ring stage (K tile then V tile)
+  int32_t v_tile_off;       // byte offset of the V tile inside a stage
+  int64_t w_total;          // nt * B * sum_h (rp_k + rp_v)
+  float q_scale;            // log2(e) / sqrt(d_head)
+  uint32_t flags;
+};
+
+struct CombineParams {
+  const HeadInfo* heads;
+  const float* basis;
+  const float* partials;
+  void* out;                // [B][1][H][d_head] or packed [B][sum rp_v]
+  int64_t out_stride_b;
+  int32_t part_stride;
+  int32_t B, H, d_head;
+  int32_t nt;
+  int32_t grid;             // CTAs of the split-KV kernel that produced the partials
+  int64_t w_total;
+  uint32_t flags;
+};
+
+struct ProjectParams {       // project rows with U and scatter them into the cache
+  const HeadInfo* heads;
+  const float* basis;
+  const void* k;            // [B][T][H][d_head]   (or packed rank-space rows)
+  const void* v;
+  char* cache;
+  int64_t stride_b, stride_t;
+  int32_t B, T, H, d_head;
+  int32_t n_max;
+  int32_t row0;             // first cache row to write (= len before the call)
+  uint32_t flags;
+};
+
+struct QProjectParams {      // prefill: Q' = Q U^K into a scratch buffer (IO dtype)
+  const HeadInfo* heads;
+  const float* basis;
+  const void* q;
+  char* qp;                 // scratch base: head h at lr_k_off[h] * B * T elements, then [B][T][rp_k]
+  int64_t stride_b, stride_t;
+  int32_t B, T, H, d_head;
+};
+
+struct PrefillParams {
+  const HeadInfo* heads;
+  const float* basis;
+  const char* cache;
+  const char* qp;           // Q' scratch (layout as in QProjectParams)
+  void* out;                // [B][T][H][d_head] or packed [B][T][sum rp_v]
+  int64_t out_stride_b, out_stride_t;
+  int32_t B, T, H, d_head;
+  int32_t n_max;
+  int32_t len0;
+  int32_t max_rp;           // widest padded rank over heads and over K/V
+  float scale_log2;         // log2(e) / sqrt(d_head)
+  uint32_t flags;
+  int* status;
+};
+
+// Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.
+cudaError_t launch_project_append(const ProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t smem_bytes,
+                          cudaStream_t s, uint64_t* launches);
+cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+
+size_t decode_fixed_smem_bytes();         // shared memory the decode kernel needs besides the ring
+cudaError_t decode_configure(int dtype);  // opt in to large dynamic shared memory (once per device)
+
+}  // namespace ea
