@@ -1,0 +1,309 @@
+"""ctypes binding of libeigenattn.so: the same calls as include/eigen_attn.h, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; torch is used for device memory and
+streams.  There is no fallback: if the library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libeigenattn.so")
+
+EA_OK = 0
+EA_ERR_INVALID_ARG, EA_ERR_SHAPE, EA_ERR_CAPACITY, EA_ERR_UNSUPPORTED = -1, -2, -3, -4
+EA_ERR_CUDA, EA_ERR_TIMEOUT, EA_ERR_NOT_ORTHONORMAL = -5, -6, -7
+EA_BF16, EA_FP32 = 0, 1
+EA_CHECK_ORTHONORMAL = 0x1
+EA_Q_PREPROJECTED, EA_OUT_LOWRANK, EA_KV_PREPROJECTED = 0x1, 0x2, 0x4
+EA_OPT_DECODE_CTAS, EA_OPT_DECODE_TILE_ROWS, EA_OPT_DECODE_STAGES, EA_OPT_PREFILL_IMPL = 1, 2, 3, 4
+
+STATUS_NAMES = {0: "EA_OK", -1: "EA_ERR_INVALID_ARG", -2: "EA_ERR_SHAPE", -3: "EA_ERR_CAPACITY",
+                -4: "EA_ERR_UNSUPPORTED", -5: "EA_ERR_CUDA", -6: "EA_ERR_TIMEOUT",
+                -7: "EA_ERR_NOT_ORTHONORMAL"}
+
+
+class EigenAttnError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} {detail}".strip())
+
+
+class ea_desc(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("n_heads", ctypes.c_int32), ("d_head", ctypes.c_int32),
+        ("n_max", ctypes.c_int32), ("dtype", ctypes.c_int32), ("max_prefill_tokens", ctypes.c_int32),
+        ("r_k", ctypes.POINTER(ctypes.c_int32)), ("r_v", ctypes.POINTER(ctypes.c_int32)),
+        ("U_k", ctypes.POINTER(ctypes.c_float)), ("U_v", ctypes.POINTER(ctypes.c_float)),
+        ("flags", ctypes.c_uint32),
+    ]
+
+
+# name -> (restype, argtypes); the list mirrors include/eigen_attn.h
+_vp, _i32, _i64, _u32, _sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_size_t
+SYMBOLS = {
+    "eigen_attn_cache_bytes": (_i32, [ctypes.POINTER(ea_desc), ctypes.POINTER(_sz), ctypes.POINTER(_sz)]),
+    "eigen_attn_create": (_i32, [ctypes.POINTER(ea_desc), _vp, _sz, _vp, _sz, _vp, ctypes.POINTER(_vp)]),
+    "eigen_attn_destroy": (None, [_vp]),
+    "eigen_attn_append_kv": (_i32, [_vp, _vp, _vp, _i32, _i64, _i64, _u32, _vp]),
+    "eigen_attn_decode": (_i32, [_vp, _vp, _i64, _vp, _u32, _vp]),
+    "eigen_attn_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _u32, _vp]),
+    "eigen_attn_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _u32, _vp]),
+    "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _u32, _vp]),
+    "eigen_attn_get_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
+    "eigen_attn_set_len": (_i32, [_vp, _i32]),
+    "eigen_attn_poll_status": (_i32, [_vp, _vp]),
+    "eigen_attn_last_error": (ctypes.c_char_p, [_vp]),
+    "eigen_attn_head_offsets": (_i32, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "eigen_attn_cache_layout": (_i32, [_vp, _i32, ctypes.POINTER(_sz), ctypes.POINTER(_sz),
+                                       ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "eigen_attn_set_option": (_i32, [_vp, _i32, _i64]),
+    "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
+    "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
+    "eigen_attn_version": (_i32, []),
+}
+
+
+def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
+    if not os.path.exists(path):
+        raise ImportError(f"{path} not found: build it with `python -m paper_2408_05646_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
+    for name, (res, args) in SYMBOLS.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    return lib
+
+
+lib = load_library()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _make_desc(batch, n_heads, d_head, n_max, dtype, r_k, r_v, U_k, U_v, max_prefill_tokens, flags):
+    """Returns (desc, keepalive): ctypes arrays must outlive the call that reads them."""
+    rk = (ctypes.c_int32 * n_heads)(*[int(r) for r in r_k])
+    rv = (ctypes.c_int32 * n_heads)(*[int(r) for r in (r_v if r_v is not None else r_k)])
+    keep = [rk, rv]
+    d = ea_desc()
+    d.batch, d.n_heads, d.d_head, d.n_max = batch, n_heads, d_head, n_max
+    d.dtype = dtype
+    d.max_prefill_tokens = max_prefill_tokens
+    d.r_k = rk
+    d.r_v = rv
+    if U_k is not None:
+        uk = np.ascontiguousarray(np.concatenate([np.asarray(u, dtype=np.float32).reshape(-1) for u in U_k]))
+        uv = np.ascontiguousarray(np.concatenate([np.asarray(u, dtype=np.float32).reshape(-1) for u in U_v]))
+        keep += [uk, uv]
+        d.U_k = uk.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+        d.U_v = uv.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+    d.flags = flags
+    return d, keep
+
+
+def cache_bytes(batch, n_heads, d_head, n_max, dtype, r_k, r_v=None, max_prefill_tokens=0):
+    """eigen_attn_cache_bytes: (cache_bytes, workspace_bytes).  Host arithmetic only."""
+    d, _keep = _make_desc(batch, n_heads, d_head, n_max, dtype, r_k, r_v, None, None, max_prefill_tokens, 0)
+    cb, wb = _sz(0), _sz(0)
+    st = lib.eigen_attn_cache_bytes(ctypes.byref(d), ctypes.byref(cb), ctypes.byref(wb))
+    if st != EA_OK:
+        raise EigenAttnError(st, "eigen_attn_cache_bytes")
+    return cb.value, wb.value
+
+
+class EigenAttnLayer:
+    """One decoder layer's rank-r KV cache and the library calls on it (eigen_attn_t)."""
+
+    def __init__(self, batch: int, n_heads: int, d_head: int, n_max: int, dtype: torch.dtype,
+                 U_k: Sequence[np.ndarray], U_v: Sequence[np.ndarray], max_prefill_tokens: int = 0,
+                 device: str | torch.device = "cuda:0", check_orthonormal: bool = False,
+                 stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("EigenAttnLayer needs a CUDA device; there is no CPU fallback")
+        self.B, self.H, self.d_head, self.n_max = batch, n_heads, d_head, n_max
+        self.torch_dtype = dtype
+        self.ea_dtype = {torch.bfloat16: EA_BF16, torch.float32: EA_FP32}[dtype]
+        self.device = torch.device(device)
+        self.r_k = [int(u.shape[1]) for u in U_k]
+        self.r_v = [int(u.shape[1]) for u in U_v]
+        for u in list(U_k) + list(U_v):
+            assert u.shape[0] == d_head
+        desc, keep = _make_desc(batch, n_heads, d_head, n_max, self.ea_dtype, self.r_k, self.r_v, U_k, U_v,
+                                max_prefill_tokens, EA_CHECK_ORTHONORMAL if check_orthonormal else 0)
+        cb, wb = _sz(0), _sz(0)
+        st = lib.eigen_attn_cache_bytes(ctypes.byref(desc), ctypes.byref(cb), ctypes.byref(wb))
+        if st != EA_OK:
+            raise EigenAttnError(st, "eigen_attn_cache_bytes")
+        with torch.cuda.device(self.device):
+            self.cache = torch.empty(cb.value, dtype=torch.uint8, device=self.device)
+            self.workspace = torch.empty(wb.value, dtype=torch.uint8, device=self.device)
+            handle = _vp(0)
+            st = lib.eigen_attn_create(ctypes.byref(desc), self.cache.data_ptr(), cb.value,
+                                       self.workspace.data_ptr(), wb.value, _stream_ptr(stream),
+                                       ctypes.byref(handle))
+        del keep
+        if st != EA_OK:
+            raise EigenAttnError(st, "eigen_attn_create")
+        self.handle = handle
+        offs_k = (ctypes.c_int32 * (n_heads + 1))()
+        offs_v = (ctypes.c_int32 * (n_heads + 1))()
+        self._check(lib.eigen_attn_head_offsets(self.handle, offs_k, offs_v), "eigen_attn_head_offsets")
+        self.offs_k, self.offs_v = list(offs_k), list(offs_v)
+
+    # -- plumbing
+    def _check(self, st: int, where: str) -> None:
+        if st != EA_OK:
+            raise EigenAttnError(st, where, lib.eigen_attn_last_error(self.handle).decode())
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            lib.eigen_attn_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _tok(self, x: torch.Tensor, T: Optional[int] = None):
+        """Checks a [B][T][H][d_head] tensor and returns (ptr, T, stride_b, stride_t)."""
+        assert x.is_cuda and x.dtype == self.torch_dtype and x.dim() == 4
+        assert x.shape[0] == self.B and x.shape[2] == self.H and x.shape[3] == self.d_head
+        assert x.stride(3) == 1 and x.stride(2) == self.d_head
+        if T is not None:
+            assert x.shape[1] == T
+        return x.data_ptr(), x.shape[1], x.stride(0), x.stride(1)
+
+    # -- the calls of include/eigen_attn.h
+    def append_kv(self, k: torch.Tensor, v: torch.Tensor, preprojected: bool = False, stream=None) -> None:
+        if preprojected:
+            assert k.is_contiguous() and v.is_contiguous() and k.dtype == self.torch_dtype
+            assert k.shape == (self.B, k.shape[1], self.offs_k[-1]) and v.shape == (self.B, k.shape[1], self.offs_v[-1])
+            T = k.shape[1]
+            st = lib.eigen_attn_append_kv(self.handle, k.data_ptr(), v.data_ptr(), T, k.stride(0), k.stride(1),
+                                          EA_KV_PREPROJECTED, _stream_ptr(stream))
+            self._check(st, "eigen_attn_append_kv")
+            return
+        pk, T, sb, stt = self._tok(k)
+        pv, _, sb2, st2 = self._tok(v, T)
+        assert (sb, stt) == (sb2, st2)
+        self._check(lib.eigen_attn_append_kv(self.handle, pk, pv, T, sb, stt, 0, _stream_ptr(stream)),
+                    "eigen_attn_append_kv")
+
+    def decode(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, q_preprojected: bool = False,
+               out_lowrank: bool = False, stream=None) -> torch.Tensor:
+        flags = 0
+        if q_preprojected:
+            assert q.is_contiguous() and q.shape == (self.B, 1, self.offs_k[-1]) and q.dtype == self.torch_dtype
+            flags |= EA_Q_PREPROJECTED
+            pq, sb = q.data_ptr(), self.H * self.d_head
+        else:
+            pq, _, sb, _ = self._tok(q, 1)
+        if out_lowrank:
+            flags |= EA_OUT_LOWRANK
+            if out is None:
+                out = torch.empty((self.B, 1, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
+            assert out.is_contiguous()
+        else:
+            if out is None:
+                out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+            po, _, sbo, _ = self._tok(out, 1)
+            if q_preprojected:
+                sb = sbo
+            assert sbo == sb
+        self._check(lib.eigen_attn_decode(self.handle, pq, sb, out.data_ptr(), flags, _stream_ptr(stream)),
+                    "eigen_attn_decode")
+        return out
+
+    def decode_step(self, q, k, v, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        pq, _, sb, _ = self._tok(q, 1)
+        pk, _, sbk, _ = self._tok(k, 1)
+        pv, _, sbv, _ = self._tok(v, 1)
+        if out is None:
+            out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+        po, _, sbo, _ = self._tok(out, 1)
+        assert sb == sbk == sbv == sbo
+        self._check(lib.eigen_attn_decode_step(self.handle, pq, pk, pv, sb, po, 0, _stream_ptr(stream)),
+                    "eigen_attn_decode_step")
+        return out
+
+    def decode_step_host(self, h_q, h_k, h_v, h_out, stream=None) -> torch.Tensor:
+        """Host tensors (contiguous, ideally pinned) in, host tensor out; synchronises the stream."""
+        for x in (h_q, h_k, h_v, h_out):
+            assert not x.is_cuda and x.is_contiguous() and x.dtype == self.torch_dtype
+            assert x.numel() == self.B * self.H * self.d_head
+        self._check(lib.eigen_attn_decode_step_host(self.handle, h_q.data_ptr(), h_k.data_ptr(), h_v.data_ptr(),
+                                                    h_out.data_ptr(), 0, _stream_ptr(stream)),
+                    "eigen_attn_decode_step_host")
+        return h_out
+
+    def prefill(self, q, k, v, out: Optional[torch.Tensor] = None, out_lowrank: bool = False, stream=None):
+        pq, T, sb, stt = self._tok(q)
+        pk, _, sbk, stk = self._tok(k, T)
+        pv, _, sbv, stv = self._tok(v, T)
+        assert (sb, stt) == (sbk, stk) == (sbv, stv)
+        flags = 0
+        if out_lowrank:
+            flags = EA_OUT_LOWRANK
+            if out is None:
+                out = torch.empty((self.B, T, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
+            assert out.is_contiguous()
+            po = out.data_ptr()
+        else:
+            if out is None:
+                out = torch.empty((self.B, T, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+            po, _, sbo, sto = self._tok(out, T)
+            assert (sbo, sto) == (sb, stt)
+        self._check(lib.eigen_attn_prefill(self.handle, pq, pk, pv, T, sb, stt, po, flags, _stream_ptr(stream)),
+                    "eigen_attn_prefill")
+        return out
+
+    @property
+    def len(self) -> int:
+        n = ctypes.c_int32(0)
+        self._check(lib.eigen_attn_get_len(self.handle, ctypes.byref(n)), "eigen_attn_get_len")
+        return n.value
+
+    def set_len(self, n: int) -> None:
+        self._check(lib.eigen_attn_set_len(self.handle, int(n)), "eigen_attn_set_len")
+
+    def poll_status(self, stream=None) -> None:
+        self._check(lib.eigen_attn_poll_status(self.handle, _stream_ptr(stream)), "eigen_attn_poll_status")
+
+    def set_option(self, option: int, value: int) -> None:
+        self._check(lib.eigen_attn_set_option(self.handle, option, int(value)), "eigen_attn_set_option")
+
+    def launch_count(self) -> int:
+        n = ctypes.c_uint64(0)
+        self._check(lib.eigen_attn_launch_count(self.handle, ctypes.byref(n)), "eigen_attn_launch_count")
+        return n.value
+
+    def set_decode_events(self, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+        a = start.cuda_event if start is not None else None
+        b = stop.cuda_event if stop is not None else None
+        self._check(lib.eigen_attn_set_decode_events(self.handle, a, b), "eigen_attn_set_decode_events")
+
+    def cache_layout(self, head: int):
+        ko, vo, rk, rv = _sz(0), _sz(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        self._check(lib.eigen_attn_cache_layout(self.handle, head, ctypes.byref(ko), ctypes.byref(vo),
+                                                ctypes.byref(rk), ctypes.byref(rv)), "eigen_attn_cache_layout")
+        return ko.value, vo.value, rk.value, rv.value
+
+    def cache_rows(self, head: int, which: str = "k") -> torch.Tensor:
+        """View of head `head`'s slab [B][n_max][rp] inside the cache buffer (for inspection)."""
+        ko, vo, rk, rv = self.cache_layout(head)
+        off, rp = (ko, rk) if which == "k" else (vo, rv)
+        es = 2 if self.torch_dtype == torch.bfloat16 else 4
+        nbytes = self.B * self.n_max * rp * es
+        return self.cache[off:off + nbytes].view(self.torch_dtype).view(self.B, self.n_max, rp)

@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "libeigenattn.so")
 SOURCES = ["api.cu", "append.cu", "decode.cu", "prefill_simt.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-    "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
+    "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
 ]
 
 

@@ -140,6 +140,7 @@ ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
   p.stride_b = stride_b; p.stride_t = stride_t;
   p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head;
   p.n_max = h->desc.n_max; p.row0 = h->len; p.flags = flags;
+  p.lr_k_width = h->L.sum_rp_k; p.lr_v_width = h->L.sum_rp_v;
   const cudaError_t e = ea::launch_project_append(p, h->desc.dtype, s, &h->launches);
   if (e != cudaSuccess) return cuda_fail(h, e, "append_kv launch");
   h->len += T;

@@ -111,7 +111,8 @@ __global__ void __launch_bounds__(256) copy_lowrank_rows_kernel(const ProjectPar
     const int col = is_k ? c : c - hd.rp_k;
     const int r = is_k ? hd.r_k : hd.r_v;
     const int rp = is_k ? hd.rp_k : hd.rp_v;
-    const T* src = (is_k ? k : v) + b * p.stride_b + t * p.stride_t + (is_k ? hd.lr_k_off : hd.lr_v_off);
+    const int width = is_k ? p.lr_k_width : p.lr_v_width;   // packed rows are contiguous [B][T][width]
+    const T* src = (is_k ? k : v) + (static_cast<int64_t>(b) * p.T + t) * width + (is_k ? hd.lr_k_off : hd.lr_v_off);
     T* dst = reinterpret_cast<T*>(p.cache + (is_k ? hd.k_off : hd.v_off)) + crow * rp;
     dst[col] = col < r ? src[col] : from_f<T>(0.f);
   }

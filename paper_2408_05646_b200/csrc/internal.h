@@ -72,6 +72,7 @@ struct ProjectParams {       // project rows with U and scatter them into the ca
   int32_t B, T, H, d_head;
   int32_t n_max;
   int32_t row0;             // first cache row to write (= len before the call)
+  int32_t lr_k_width, lr_v_width;   // widths of the packed rank-space rows (sum of rp_k / rp_v)
   uint32_t flags;
 };
 

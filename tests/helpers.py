@@ -1,0 +1,52 @@
+"""Shared helpers of the GPU parity tests: build a layer on both sides from the same seeded inputs
+and compare with the tolerances the workloads state."""
+import numpy as np
+import torch
+
+from oracle import eigen_attention as orc
+from paper_2408_05646_b200 import synth
+
+# bf16 storage / fp32 accumulation: max-abs <= 2e-2 and mean-abs <= 2e-3 against the fp64 oracle
+# (outputs are O(1) convex combinations of unit-variance value rows; one bf16 ulp at 1.0 is 7.8e-3).
+BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
+# fp32 mode: 1e-5 relative, taken per tensor (max-abs / max|ref| and the relative L2 norm); an
+# element-wise ratio is meaningless near zeros.
+FP32_REL = 1e-5
+
+
+def assert_close(got: torch.Tensor, ref: np.ndarray, dtype: torch.dtype, what: str = "", fp32_rel: float = FP32_REL):
+    g = got.detach().double().cpu().numpy().reshape(ref.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite output"
+    diff = np.abs(g - ref)
+    if dtype == torch.bfloat16:
+        assert diff.max() <= BF16_MAX_ABS, f"{what}: max-abs {diff.max():.3e}"
+        assert diff.mean() <= BF16_MEAN_ABS, f"{what}: mean-abs {diff.mean():.3e}"
+    else:
+        scale = max(np.abs(ref).max(), 1e-30)
+        assert diff.max() / scale <= fp32_rel, f"{what}: rel max {diff.max() / scale:.3e}"
+        l2 = np.linalg.norm(g - ref) / max(np.linalg.norm(ref), 1e-30)
+        assert l2 <= fp32_rel, f"{what}: rel l2 {l2:.3e}"
+
+
+def make_case(B, H, d_head, ranks_k, ranks_v, n, dtype, seed_cfg=90, rho=16, sigma=0.1, q_scale=1.0,
+              device="cuda:0", T_q=1):
+    """Seeded bases and K/V/Q tensors on `device` (values already rounded to the IO dtype)."""
+    U_k = [synth.orthonormal_basis(d_head, r, synth.stream_seed(seed_cfg, "U_K", h)).astype(np.float32)
+           for h, r in enumerate(ranks_k)]
+    U_v = [synth.orthonormal_basis(d_head, r, synth.stream_seed(seed_cfg, "U_V", h)).astype(np.float32)
+           for h, r in enumerate(ranks_v)]
+    W_k = synth.mixing_matrices(H, rho, d_head, seed_cfg, "W_K")
+    W_v = synth.mixing_matrices(H, rho, d_head, seed_cfg, "W_V")
+    W_q = synth.mixing_matrices(H, rho, d_head, seed_cfg, "W_Q")
+    k = synth.lowrank_rows(W_k, B, n, sigma, seed_cfg, "K", dtype=dtype, device=device)
+    v = synth.lowrank_rows(W_v, B, n, sigma, seed_cfg, "V", dtype=dtype, device=device)
+    q = (synth.lowrank_rows(W_q, B, T_q, sigma, seed_cfg, "Q", dtype=torch.float32, device=device) * q_scale).to(dtype)
+    return U_k, U_v, q, k, v
+
+
+def oracle_layer(B, H, d_head, U_k, U_v, tracked=None):
+    return orc.LayerOracle(B, H, d_head, U_k, U_v, tracked)
+
+
+def to_np(x: torch.Tensor) -> np.ndarray:
+    return x.detach().double().cpu().numpy()

@@ -1,0 +1,276 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element, on the
+same seeded inputs.  Sizes span several shared-memory tiles, ragged tails and several CTAs' splits."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, make_case, oracle_layer, to_np
+
+pytestmark = pytest.mark.gpu
+
+BF16, FP32 = torch.bfloat16, torch.float32
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    return binding
+
+
+def run_decode_case(B_, bnd, H, d_head, rk, rv, n, dtype, seed=90, q_scale=1.0, opts=None):
+    U_k, U_v, q, k, v = make_case(B_, H, d_head, rk, rv, n, dtype, seed_cfg=seed, q_scale=q_scale)
+    lay = bnd.EigenAttnLayer(B_, H, d_head, n + 4, dtype, U_k, U_v)
+    for o, val in (opts or {}).items():
+        lay.set_option(o, val)
+    lay.append_kv(k, v)
+    out = lay.decode(q)
+    lay.poll_status()
+    ref = oracle_layer(B_, H, d_head, U_k, U_v)
+    ref.append_kv(to_np(k), to_np(v))
+    expect = ref.decode_dense(to_np(q))
+    assert_close(out, expect, dtype, f"decode B{B_} H{H} d{d_head} n{n}")
+    return lay, ref, (U_k, U_v, q, k, v), out
+
+
+def test_tiny_fp32_workload(B):
+    # the small reference workload: 1 x 4 heads, d_head 64, r 32, 512 cached rows + 1 new token
+    from paper_2408_05646_b200 import synth
+    wl = synth.WORKLOADS["tiny_fp32"]
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
+    W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
+    k = synth.lowrank_rows(W_k, wl.batch, wl.context + 1, wl.sigma, wl.index, "K", dtype=FP32, device="cuda:0")
+    v = synth.lowrank_rows(W_v, wl.batch, wl.context + 1, wl.sigma, wl.index, "V", dtype=FP32, device="cuda:0")
+    q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=FP32, device="cuda:0")
+    lay = B.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + 1, FP32, U_k, U_v)
+    lay.append_kv(k[:, :wl.context], v[:, :wl.context])
+    out = lay.decode_step(q, k[:, wl.context:], v[:, wl.context:])      # one new token appended, then attended
+    assert lay.len == wl.context + 1
+    ref = oracle_layer(wl.batch, wl.n_heads, wl.d_head, U_k, U_v)
+    ref.append_kv(to_np(k), to_np(v))
+    assert_close(out, ref.decode_dense(to_np(q)), FP32, "tiny fp32")
+    # cache contents == the oracle's projected rows
+    for h in range(wl.n_heads):
+        Kc = lay.cache_rows(h, "k")[:, :wl.context + 1, :ranks[h]]
+        Vc = lay.cache_rows(h, "v")[:, :wl.context + 1, :ranks[h]]
+        for b in range(wl.batch):
+            assert_close(Kc[b], ref.Kp[(b, h)], FP32, "K' rows")
+            assert_close(Vc[b], ref.Vp[(b, h)], FP32, "V' rows")
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP32])
+@pytest.mark.parametrize("r", [8, 16, 32, 48, 64, 80, 96, 112, 128])
+def test_decode_uniform_ranks(B, dtype, r):
+    # every lane-pair width class and both bank-rotation cases; n spans tiles with a ragged tail
+    run_decode_case(2, B, 3, 128, [r] * 3, [r] * 3, 700, dtype)
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP32])
+def test_decode_heterogeneous_and_unpadded_ranks(B, dtype):
+    rk = [5, 48, 80, 33, 112, 64, 17, 96]
+    rv = [9, 64, 80, 128, 40, 7, 100, 24]
+    lay, ref, _, _ = run_decode_case(3, B, 8, 128, rk, rv, 1111, dtype)
+    # padding columns of the cache hold zeros
+    for h in (0, 3):
+        assert float(lay.cache_rows(h, "k")[:, :1111, rk[h]:].abs().max()) == 0.0
+        assert float(lay.cache_rows(h, "v")[:, :1111, rv[h]:].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("n", [1, 2, 15, 16, 17, 127, 128, 129, 513])
+def test_decode_short_contexts(B, n):
+    run_decode_case(2, B, 4, 64, [32] * 4, [24] * 4, n, BF16)
+    run_decode_case(1, B, 2, 64, [32] * 2, [32] * 2, n, FP32)
+
+
+@pytest.mark.parametrize("d_head", [8, 64, 96, 128])
+def test_decode_head_dims(B, d_head):
+    r = max(8, d_head // 2)
+    run_decode_case(2, B, 2, d_head, [r, d_head], [d_head, r], 300, FP32)
+
+
+def test_long_context_split_over_all_ctas_matches_single_cta(B):
+    # few units, long context: every unit is split over many CTAs and merged by the combine kernel
+    B_, H, n = 1, 2, 40000
+    lay, ref, (U_k, U_v, q, k, v), out = run_decode_case(B_, B, H, 128, [64, 64], [64, 64], n, BF16)
+    for ctas, tile, stages in [(1, 0, 0), (7, 64, 2), (148, 32, 3), (300, 128, 0)]:
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        lay.set_option(B.EA_OPT_DECODE_TILE_ROWS, tile)
+        lay.set_option(B.EA_OPT_DECODE_STAGES, stages)
+        o2 = lay.decode(q)
+        lay.poll_status()
+        assert_close(o2, ref.decode_dense(to_np(q)), BF16, f"ctas={ctas}")
+        assert float((o2.float() - out.float()).abs().max()) < 2e-2
+
+
+def test_split_consistency_fp32(B):
+    # the split-KV result is an exact re-association: in fp32 mode any CTA count agrees to 1e-5
+    B_, H, n = 2, 3, 9000
+    lay, ref, (U_k, U_v, q, k, v), out = run_decode_case(B_, B, H, 64, [32, 16, 48], [32, 64, 8], n, FP32)
+    for ctas in (1, 2, 5, 33, 148, 512):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        o2 = lay.decode(q)
+        assert_close(o2, ref.decode_dense(to_np(q)), FP32, f"ctas={ctas}")
+
+
+def test_append_T_tokens_equals_T_single_appends_and_64_steps(B):
+    # long-context workload shape in miniature: 64 consecutive single-token append+decode steps
+    B_, H, d, r, n0, steps = 2, 4, 128, 64, 1000, 64
+    U_k, U_v, q, k, v = make_case(B_, H, d, [r] * H, [r] * H, n0 + steps, BF16, seed_cfg=94, T_q=steps)
+    a = B.EigenAttnLayer(B_, H, d, n0 + steps, BF16, U_k, U_v)
+    b = B.EigenAttnLayer(B_, H, d, n0 + steps, BF16, U_k, U_v)
+    a.append_kv(k[:, :n0], v[:, :n0])
+    b.append_kv(k[:, :n0], v[:, :n0])
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    ref.append_kv(to_np(k[:, :n0]), to_np(v[:, :n0]))
+    for t in range(steps):
+        out = a.decode_step(q[:, t:t + 1], k[:, n0 + t:n0 + t + 1], v[:, n0 + t:n0 + t + 1])
+        ref.append_kv(to_np(k[:, n0 + t:n0 + t + 1]), to_np(v[:, n0 + t:n0 + t + 1]))
+        if t % 9 == 0 or t == steps - 1:
+            assert_close(out, ref.decode_dense(to_np(q[:, t:t + 1])), BF16, f"step {t}")
+    b.append_kv(k[:, n0:], v[:, n0:])
+    assert a.len == b.len == n0 + steps
+    assert torch.equal(a.cache, b.cache)          # identical cache bytes either way
+
+
+def test_adversarial_softmax_inputs(B):
+    B_, H, d, r, n = 1, 2, 64, 32, 600
+    U_k, U_v, q, k, v = make_case(B_, H, d, [r] * H, [r] * H, n, FP32, seed_cfg=95)
+    Uk0 = torch.from_numpy(U_k[0]).cuda()
+    cases = {}
+    # scores increasing with position: a rescale of the running state at every row
+    dirn = (Uk0 @ torch.ones(r, device="cuda")).float()
+    dirn = dirn / dirn.norm()
+    k_inc = k.clone()
+    k_inc[0, :, 0, :] = dirn[None, :] * torch.linspace(-40, 40, n, device="cuda")[:, None]
+    q_inc = q.clone()
+    q_inc[0, 0, 0, :] = dirn * 8.0
+    cases["increasing"] = (q_inc, k_inc)
+    # one dominant key
+    k_dom = k.clone()
+    k_dom[0, 77, 1, :] = (Uk0 @ torch.ones(r, device="cuda")) * 3
+    q_dom = q.clone()
+    q_dom[0, 0, 1, :] = k_dom[0, 77, 1, :] * 4
+    cases["dominant"] = (q_dom, k_dom)
+    # all-equal scores (q = 0) and very large |scores| (~ +-80 before the softmax)
+    cases["uniform"] = (torch.zeros_like(q), k)
+    cases["large"] = (q * 60.0, k)
+    for name, (qq, kk) in cases.items():
+        lay = B.EigenAttnLayer(B_, H, d, n, FP32, U_k, U_v)
+        lay.append_kv(kk, v)
+        out = lay.decode(qq)
+        ref = oracle_layer(B_, H, d, U_k, U_v)
+        ref.append_kv(to_np(kk), to_np(v))
+        # a score s carries an absolute fp32 error of about |s| * 2^-23 * sqrt(r), which the softmax turns
+        # into the same relative error of a weight: with |s| up to ~300 here the bound is 2e-4, not 1e-5
+        tol = 2e-4 if name in ("large", "increasing", "dominant") else 1e-5
+        assert_close(out, ref.decode_dense(to_np(qq)), FP32, name, fp32_rel=tol)
+
+
+def test_merged_weight_flags(B):
+    # rank-space inputs/outputs for callers whose projection weights already contain U (Eq. 8)
+    B_, H, d, n = 2, 3, 64, 257
+    rk, rv = [16, 24, 30], [8, 40, 21]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, FP32, seed_cfg=96)
+    lay = B.EigenAttnLayer(B_, H, d, n, FP32, U_k, U_v)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    ref.append_kv(to_np(k), to_np(v))
+    # packed rank-space tensors built on the host from the same fp32 bases
+    def pack(x, U, offs):
+        out = torch.zeros((B_, x.shape[1], offs[-1]), dtype=torch.float32)
+        xn = to_np(x)
+        for h in range(H):
+            y = xn[:, :, h, :] @ U[h].astype(np.float64)
+            out[:, :, offs[h]:offs[h] + U[h].shape[1]] = torch.from_numpy(y).float()
+        return out.cuda()
+    kp, vp, qp = pack(k, U_k, lay.offs_k), pack(v, U_v, lay.offs_v), pack(q, U_k, lay.offs_k)
+    lay.append_kv(kp, vp, preprojected=True)
+    out = lay.decode(qp, q_preprojected=True)
+    assert_close(out, ref.decode_dense(to_np(q)), FP32, "preprojected q,k,v")
+    low = lay.decode(q, out_lowrank=True)
+    res = ref.decode(to_np(q), lowrank_out=True)
+    for b in range(B_):
+        for h in range(H):
+            got = low[b, 0, lay.offs_v[h]:lay.offs_v[h] + rv[h]]
+            assert_close(got, res[(b, h)], FP32, "lowrank out")
+
+
+@pytest.mark.parametrize("dtype,H,d,rk,rv,T", [
+    (FP32, 2, 64, [32, 20], [16, 40], 75),
+    (BF16, 4, 128, [80, 48, 128, 64], [80, 112, 8, 64], 200),
+    (BF16, 1, 128, [80], [80], 33),
+])
+def test_prefill_matches_oracle_and_feeds_decode(B, dtype, H, d, rk, rv, T):
+    B_ = 2
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + 1, dtype, seed_cfg=97, T_q=T + 1)
+    lay = B.EigenAttnLayer(B_, H, d, T + 1, dtype, U_k, U_v, max_prefill_tokens=T)
+    out = lay.prefill(q[:, :T], k[:, :T], v[:, :T])
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    expect = ref.prefill_dense(to_np(q[:, :T]), to_np(k[:, :T]), to_np(v[:, :T]))
+    assert_close(out, expect, dtype, "prefill")
+    # the cache the prefill wrote serves the next decode step
+    o1 = lay.decode_step(q[:, T:], k[:, T:], v[:, T:])
+    ref.append_kv(to_np(k[:, T:]), to_np(v[:, T:]))
+    assert_close(o1, ref.decode_dense(to_np(q[:, T:])), dtype, "decode after prefill")
+
+
+def test_chunked_prefill_and_lowrank_output(B):
+    B_, H, d, T = 1, 2, 64, 90
+    rk, rv = [32, 24], [16, 32]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, FP32, seed_cfg=98, T_q=T)
+    lay = B.EigenAttnLayer(B_, H, d, T, FP32, U_k, U_v, max_prefill_tokens=64)
+    o1 = lay.prefill(q[:, :50].contiguous(), k[:, :50].contiguous(), v[:, :50].contiguous())
+    o2 = lay.prefill(q[:, 50:].contiguous(), k[:, 50:].contiguous(), v[:, 50:].contiguous())
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
+    assert_close(torch.cat([o1, o2], dim=1), expect, FP32, "chunked prefill")
+    lay.set_len(0)
+    low = lay.prefill(q[:, :64].contiguous(), k[:, :64].contiguous(), v[:, :64].contiguous(), out_lowrank=True)
+    for h in range(H):
+        got = to_np(low[0, :, lay.offs_v[h]:lay.offs_v[h] + rv[h]]) @ U_v[h].astype(np.float64).T
+        assert np.abs(got - expect[0, :64, h, :]).max() < 1e-5
+
+
+def test_strided_inputs_and_host_step(B):
+    B_, H, d, n = 2, 2, 64, 100
+    U_k, U_v, q, k, v = make_case(B_, H, d, [32] * H, [32] * H, n, BF16, seed_cfg=99)
+    # q/k/v as slices of a fused [B][T][3][H][d] projection output (non-contiguous batch/token strides)
+    fused = torch.stack([k, v, k], dim=2).contiguous()
+    ks, vs = fused[:, :, 0], fused[:, :, 1]
+    lay = B.EigenAttnLayer(B_, H, d, n + 1, BF16, U_k, U_v)
+    lay.append_kv(ks[:, :n - 1], vs[:, :n - 1])
+    hq, hk, hv = q.cpu().pin_memory(), k[:, n - 1:].cpu().contiguous().pin_memory(), v[:, n - 1:].cpu().contiguous().pin_memory()
+    hout = torch.empty_like(hq).pin_memory()
+    lay.decode_step_host(hq, hk, hv, hout)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    ref.append_kv(to_np(k), to_np(v))
+    assert_close(hout, ref.decode_dense(to_np(q)), BF16, "host step")
+    assert lay.launch_count() >= 4
+
+
+def test_errors_leave_state_unchanged(B):
+    B_, H, d = 1, 2, 64
+    U_k, U_v, q, k, v = make_case(B_, H, d, [32] * H, [32] * H, 8, BF16, seed_cfg=100)
+    lay = B.EigenAttnLayer(B_, H, d, 8, BF16, U_k, U_v, max_prefill_tokens=4, check_orthonormal=True)
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.decode(q)
+    assert e.value.status == B.EA_ERR_SHAPE and "empty" in str(e.value)
+    lay.append_kv(k, v)
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.append_kv(k[:, :1], v[:, :1])
+    assert e.value.status == B.EA_ERR_CAPACITY and lay.len == 8
+    lay.set_len(0)
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.prefill(q.expand(B_, 8, H, d).contiguous(), k, v)
+    assert e.value.status == B.EA_ERR_CAPACITY and lay.len == 0
+    with pytest.raises(B.EigenAttnError):
+        lay.set_option(B.EA_OPT_DECODE_TILE_ROWS, 24)
+    bad = [u.copy() for u in U_k]
+    bad[1][:, 0] *= 1.5
+    with pytest.raises(B.EigenAttnError) as e:
+        B.EigenAttnLayer(B_, H, d, 8, BF16, bad, U_v, check_orthonormal=True)
+    assert e.value.status == B.EA_ERR_NOT_ORTHONORMAL
+    lay.poll_status()
