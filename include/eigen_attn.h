@@ -97,13 +97,16 @@ ea_status eigen_attn_append_kv(eigen_attn_t h, const void* d_k, const void* d_v,
 
 /* Eq. 3 in the rank-r space of Eq. 7: one query per sequence against rows [0, len).  Call it after
  * the append of the same token (the new token attends to itself).  d_q, d_out: [B][1][H][d_head]
- * with batch stride `stride_b`.  flags: EA_Q_PREPROJECTED, EA_OUT_LOWRANK.  len == 0 -> EA_ERR_SHAPE. */
-ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out,
-                            uint32_t flags, void* cuda_stream);
+ * with batch strides `stride_b_q`, `stride_b_out`.  flags: EA_Q_PREPROJECTED, EA_OUT_LOWRANK.
+ * len == 0 -> EA_ERR_SHAPE. */
+ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                            int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
-/* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token). */
-ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
-                                 int64_t stride_b, void* d_out, uint32_t flags, void* cuda_stream);
+/* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token).
+ * d_k and d_v share the batch stride `stride_b_kv`. */
+ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q,
+                                 const void* d_k, const void* d_v, int64_t stride_b_kv,
+                                 void* d_out, int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
 /* The same step for HOST tensors (contiguous [B][1][H][d_head], ideally pinned): copies q, k, v to a
  * staging area of the workspace, runs the step, copies the result back and synchronises the stream. */

@@ -51,8 +51,8 @@ SYMBOLS = {
     "eigen_attn_create": (_i32, [ctypes.POINTER(ea_desc), _vp, _sz, _vp, _sz, _vp, ctypes.POINTER(_vp)]),
     "eigen_attn_destroy": (None, [_vp]),
     "eigen_attn_append_kv": (_i32, [_vp, _vp, _vp, _i32, _i64, _i64, _u32, _vp]),
-    "eigen_attn_decode": (_i32, [_vp, _vp, _i64, _vp, _u32, _vp]),
-    "eigen_attn_decode_step": (_i32, [_vp, _vp, _vp, _vp, _i64, _vp, _u32, _vp]),
+    "eigen_attn_decode": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
+    "eigen_attn_decode_step": (_i32, [_vp, _vp, _i64, _vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _u32, _vp]),
     "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _u32, _vp]),
     "eigen_attn_get_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
@@ -207,34 +207,35 @@ class EigenAttnLayer:
         if q_preprojected:
             assert q.is_contiguous() and q.shape == (self.B, 1, self.offs_k[-1]) and q.dtype == self.torch_dtype
             flags |= EA_Q_PREPROJECTED
-            pq, sb = q.data_ptr(), self.H * self.d_head
+            pq, sbq = q.data_ptr(), self.offs_k[-1]
         else:
-            pq, _, sb, _ = self._tok(q, 1)
+            pq, _, sbq, _ = self._tok(q, 1)
         if out_lowrank:
             flags |= EA_OUT_LOWRANK
             if out is None:
                 out = torch.empty((self.B, 1, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
-            assert out.is_contiguous()
+            assert out.is_contiguous() and out.dtype == self.torch_dtype
+            sbo = self.offs_v[-1]
         else:
             if out is None:
                 out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
-            po, _, sbo, _ = self._tok(out, 1)
-            if q_preprojected:
-                sb = sbo
-            assert sbo == sb
-        self._check(lib.eigen_attn_decode(self.handle, pq, sb, out.data_ptr(), flags, _stream_ptr(stream)),
+            _, _, sbo, _ = self._tok(out, 1)
+        self._check(lib.eigen_attn_decode(self.handle, pq, sbq, out.data_ptr(), sbo, flags, _stream_ptr(stream)),
                     "eigen_attn_decode")
         return out
 
     def decode_step(self, q, k, v, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-        pq, _, sb, _ = self._tok(q, 1)
+        pq, _, sbq, _ = self._tok(q, 1)
         pk, _, sbk, _ = self._tok(k, 1)
         pv, _, sbv, _ = self._tok(v, 1)
+        if sbk != sbv:
+            k, v = k.contiguous(), v.contiguous()
+            pk, _, sbk, _ = self._tok(k, 1)
+            pv, _, sbv, _ = self._tok(v, 1)
         if out is None:
             out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
         po, _, sbo, _ = self._tok(out, 1)
-        assert sb == sbk == sbv == sbo
-        self._check(lib.eigen_attn_decode_step(self.handle, pq, pk, pv, sb, po, 0, _stream_ptr(stream)),
+        self._check(lib.eigen_attn_decode_step(self.handle, pq, sbq, pk, pv, sbk, po, sbo, 0, _stream_ptr(stream)),
                     "eigen_attn_decode_step")
         return out
 

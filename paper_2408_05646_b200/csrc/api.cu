@@ -147,8 +147,8 @@ ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
   return EA_OK;
 }
 
-ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, uint32_t flags,
-                    cudaStream_t s) {
+ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
+                    uint32_t flags, cudaStream_t s) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
     return fail(h, EA_ERR_INVALID_ARG, "decode: unknown flag 0x%x", flags);
@@ -206,7 +206,7 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
 
   ea::CombineParams c{};
   c.heads = p.heads; c.basis = p.basis; c.partials = p.partials; c.out = d_out;
-  c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b;
+  c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
   c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
   c.w_total = w_total; c.flags = flags;
   e = ea::launch_combine(c, h->desc.dtype, s, &h->launches);
@@ -317,22 +317,23 @@ ea_status eigen_attn_append_kv(eigen_attn_t h, const void* d_k, const void* d_v,
   return do_append(h, d_k, d_v, T, stride_b, stride_t, flags, static_cast<cudaStream_t>(cuda_stream));
 }
 
-ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, uint32_t flags,
-                            void* cuda_stream) {
+ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                            int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  return do_decode(h, d_q, stride_b, d_out, flags, static_cast<cudaStream_t>(cuda_stream));
+  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags, static_cast<cudaStream_t>(cuda_stream));
 }
 
-ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
-                                 int64_t stride_b, void* d_out, uint32_t flags, void* cuda_stream) {
+ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q, const void* d_k,
+                                 const void* d_v, int64_t stride_b_kv, void* d_out, int64_t stride_b_out,
+                                 uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL q or out");
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
     return fail(h, EA_ERR_INVALID_ARG, "decode_step: unknown flag 0x%x", flags);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  const ea_status st = do_append(h, d_k, d_v, 1, stride_b, stride_b, 0, s);
+  const ea_status st = do_append(h, d_k, d_v, 1, stride_b_kv, stride_b_kv, 0, s);
   if (st != EA_OK) return st;
-  return do_decode(h, d_q, stride_b, d_out, flags, s);
+  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags, s);
 }
 
 ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const void* h_k, const void* h_v,
@@ -355,7 +356,7 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   const int64_t sb = static_cast<int64_t>(h->desc.n_heads) * h->desc.d_head;
   ea_status st = do_append(h, sk, sv, 1, sb, sb, 0, s);
   if (st != EA_OK) return st;
-  st = do_decode(h, sq, sb, so, 0, s);
+  st = do_decode(h, sq, sb, so, sb, 0, s);
   if (st != EA_OK) return st;
   e = cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);

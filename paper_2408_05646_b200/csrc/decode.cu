@@ -193,7 +193,11 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     const unsigned char* kt = ring + static_cast<size_t>(stage) * p.stage_bytes;
     const unsigned char* vt = kt + p.v_tile_off;
     const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
-    for (int row = warp * 16 + pair; row < rows; row += kDecodeConsumerWarps * 16) {
+    // The loop bound is the same for all lanes of a warp (the shuffle below needs every lane);
+    // lane pairs past the last row recompute the group's first row and drop the result.
+    for (int rbase = warp * 16; rbase < rows; rbase += kDecodeConsumerWarps * 16) {
+      const bool valid = rbase + pair < rows;
+      const int row = valid ? rbase + pair : rbase;
       const unsigned char* kr = kt + row * rowb_k;
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -208,24 +212,26 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
       }
       float s = (a0 + a1) + (a2 + a3);
       s += __shfl_xor_sync(0xffffffffu, s, 1);
-      if (s > m) {                      // rare after the first rows: rescale the running state
-        const float c = fast_exp2(m - s);
-        l *= c;
+      if (valid) {
+        if (s > m) {                    // rare after the first rows: rescale the running state
+          const float c = fast_exp2(m - s);
+          l *= c;
 #pragma unroll
-        for (int j = 0; j < NCH; ++j)
+          for (int j = 0; j < NCH; ++j)
 #pragma unroll
-          for (int e = 0; e < EPC; ++e) o[j][e] *= c;
-        m = s;
-      }
-      const float pr = fast_exp2(s - m);
-      l += pr;
-      const unsigned char* vr = vt + row * rowb_v;
+            for (int e = 0; e < EPC; ++e) o[j][e] *= c;
+          m = s;
+        }
+        const float pr = fast_exp2(s - m);
+        l += pr;
+        const unsigned char* vr = vt + row * rowb_v;
 #pragma unroll
-      for (int j = 0; j < NCH; ++j) {
-        float x[EPC];
-        Elem<T>::load_chunk(vr + off_v[j], x);
+        for (int j = 0; j < NCH; ++j) {
+          float x[EPC];
+          Elem<T>::load_chunk(vr + off_v[j], x);
 #pragma unroll
-        for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, x[e], o[j][e]);
+          for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, x[e], o[j][e]);
+        }
       }
     }
     __syncwarp();

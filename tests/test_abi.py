@@ -64,6 +64,6 @@ def test_null_arguments(binding):
     lib = binding.lib
     assert lib.eigen_attn_cache_bytes(None, None, None) == binding.EA_ERR_INVALID_ARG
     assert lib.eigen_attn_get_len(None, None) == binding.EA_ERR_INVALID_ARG
-    assert lib.eigen_attn_decode(None, None, 0, None, 0, None) == binding.EA_ERR_INVALID_ARG
+    assert lib.eigen_attn_decode(None, None, 0, None, 0, 0, None) == binding.EA_ERR_INVALID_ARG
     assert lib.eigen_attn_last_error(None) == b"null handle"
     lib.eigen_attn_destroy(None)
