@@ -115,10 +115,11 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
 
 /* Section 2 (prefill phase) with Eq. 7 and a causal mask: append T rows (as eigen_attn_append_kv) and
  * compute the attention output of the T queries, query t over rows [0, len0 + t] where len0 is the
- * length before the call.  T <= max_prefill_tokens.  d_q, d_k, d_v, d_out: [B][T][H][d_head].
- * flags: EA_OUT_LOWRANK. */
+ * length before the call.  T <= max_prefill_tokens.  d_q, d_k, d_v: [B][T][H][d_head] sharing
+ * (stride_b, stride_t); d_out: [B][T][H][d_head] with its own strides.  flags: EA_OUT_LOWRANK. */
 ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
                              int32_t T, int64_t stride_b, int64_t stride_t, void* d_out,
+                             int64_t out_stride_b, int64_t out_stride_t,
                              uint32_t flags, void* cuda_stream);
 
 /* Current number of cached rows; set_len truncates or rewinds (0 <= len <= n_max), e.g. to re-run

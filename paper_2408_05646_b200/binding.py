@@ -54,7 +54,7 @@ SYMBOLS = {
     "eigen_attn_decode": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_decode_step": (_i32, [_vp, _vp, _i64, _vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _u32, _vp]),
-    "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _u32, _vp]),
+    "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _i64, _i64, _u32, _vp]),
     "eigen_attn_get_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "eigen_attn_set_len": (_i32, [_vp, _i32]),
     "eigen_attn_poll_status": (_i32, [_vp, _vp]),
@@ -260,13 +260,12 @@ class EigenAttnLayer:
             if out is None:
                 out = torch.empty((self.B, T, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
             assert out.is_contiguous()
-            po = out.data_ptr()
+            po, sbo, sto = out.data_ptr(), T * self.offs_v[-1], self.offs_v[-1]
         else:
             if out is None:
                 out = torch.empty((self.B, T, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
             po, _, sbo, sto = self._tok(out, T)
-            assert (sbo, sto) == (sb, stt)
-        self._check(lib.eigen_attn_prefill(self.handle, pq, pk, pv, T, sb, stt, po, flags, _stream_ptr(stream)),
+        self._check(lib.eigen_attn_prefill(self.handle, pq, pk, pv, T, sb, stt, po, sbo, sto, flags, _stream_ptr(stream)),
                     "eigen_attn_prefill")
         return out
 

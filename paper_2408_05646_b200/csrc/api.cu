@@ -365,8 +365,8 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
 }
 
 ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v, int32_t T,
-                             int64_t stride_b, int64_t stride_t, void* d_out, uint32_t flags,
-                             void* cuda_stream) {
+                             int64_t stride_b, int64_t stride_t, void* d_out, int64_t out_stride_b,
+                             int64_t out_stride_t, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
   if (flags & ~EA_OUT_LOWRANK) return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
@@ -390,7 +390,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     p.out_stride_t = L.sum_rp_v;
     p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
   } else {
-    p.out_stride_b = stride_b; p.out_stride_t = stride_t;
+    p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
   }
   p.B = qp.B; p.T = T; p.H = qp.H; p.d_head = qp.d_head; p.n_max = h->desc.n_max; p.len0 = len0;
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;

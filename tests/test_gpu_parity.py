@@ -75,7 +75,7 @@ def test_decode_heterogeneous_and_unpadded_ranks(B, dtype):
     rv = [9, 64, 80, 128, 40, 7, 100, 24]
     lay, ref, _, _ = run_decode_case(3, B, 8, 128, rk, rv, 1111, dtype)
     # padding columns of the cache hold zeros
-    for h in (0, 3):
+    for h in (0, 6):
         assert float(lay.cache_rows(h, "k")[:, :1111, rk[h]:].abs().max()) == 0.0
         assert float(lay.cache_rows(h, "v")[:, :1111, rv[h]:].abs().max()) == 0.0
 
