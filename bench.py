@@ -1,0 +1,400 @@
+"""Benchmark of the rank-r decode attention step (append one token, attend over the whole rank-r cache).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the decode hot path over one batch: project + append the new K/V row of every
+sequence, project q, split-KV attention over all cached rank-r rows, cross-split combine and lift.
+Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank runs its own batch (the path shards by
+sequence with no exchange), timings are the max over ranks.  `--impl reference` times the fp64 CPU
+oracle on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2408_05646_b200 import synth
+
+METRIC = "rank-r decode attention KV GB/s (B=16, n=32k, 7B layer; us/step alongside)"
+UNIT = "GB/s"
+FILL_CHUNK = 1024          # tokens per append call while filling the cache
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, torch copy read+write)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def algorithmic_bytes(wl, ranks_k, ranks_v, n):
+    """K' and V' rows that one decode step must read: B * n * sum_h (r_k + r_v) * element size."""
+    es = 2 if wl.dtype == "bf16" else 4
+    return wl.batch * n * (sum(ranks_k) + sum(ranks_v)) * es
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# the CPU oracle leg (also the --impl reference arm)
+# ----------------------------------------------------------------------------------------------
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, sample_heads, history=None):
+    """Oracle state for the units (0, h), h in sample_heads: projects their whole history once.
+    `history` maps h -> (k_rows, v_rows) [n, d_head] float64; if None it is drawn on the CPU."""
+    from oracle import eigen_attention as orc
+    units = [(0, h) for h in sample_heads]
+    lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units)
+    if history is None:
+        W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
+        W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
+        dt = synth.torch_dtype(wl.dtype)
+        for ci, c in enumerate(range(0, wl.context, FILL_CHUNK)):
+            t = min(FILL_CHUNK, wl.context - c)
+            k = synth.lowrank_rows(W_k, 1, t, wl.sigma, wl.index, "K", chunk=ci, dtype=dt).double().numpy()
+            v = synth.lowrank_rows(W_v, 1, t, wl.sigma, wl.index, "V", chunk=ci, dtype=dt).double().numpy()
+            for h in sample_heads:
+                lay.append_unit_rows((0, h), k[0, :, h, :], v[0, :, h, :])
+    else:
+        for h in sample_heads:
+            lay.append_unit_rows((0, h), history[h][0], history[h][1])
+    lay.set_len(wl.context)
+    return lay
+
+
+def oracle_timed_steps(lay, wl, q, k_new, v_new, steps, warmup):
+    """Times `steps` oracle decode steps (append the new row, attend) on the tracked units.
+    Returns (seconds per step, outputs of the last step)."""
+    n0 = wl.context
+    times, out = [], None
+    for i in range(warmup + steps):
+        for u in lay.units:                                   # rewind to the fixed context length
+            lay.Kp[u] = lay.Kp[u][:n0]
+            lay.Vp[u] = lay.Vp[u][:n0]
+        lay.set_len(n0)
+        t0 = time.perf_counter()
+        lay.append_kv(k_new, v_new)
+        out = lay.decode(q)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    return sum(times) / len(times), out
+
+
+def run_reference(args, wl):
+    """The fp64 oracle as it stands on the host cores; each step covers a bounded sample of units."""
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    sample_heads = list(range(wl.n_heads))                  # all heads of sequence 0
+    lay = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, sample_heads)
+    dt = synth.torch_dtype(wl.dtype)
+    W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
+    W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
+    k_new = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt).double().numpy()
+    v_new = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt).double().numpy()
+    q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt).double().numpy()
+    sec, _ = oracle_timed_steps(lay, wl, q, k_new, v_new, args.steps, args.warmup)
+    es = 2 if wl.dtype == "bf16" else 4
+    sample_bytes = (wl.context + 1) * sum(2 * ranks[h] for h in sample_heads) * es
+    gbs = sample_bytes / sec / 1e9
+    cores = blas_threads()
+    sample = (f"{len(sample_heads)} of {wl.batch * wl.n_heads} (sequence, head) units per step "
+              f"(all heads of sequence 0), full context {wl.context}+1; GB/s counts the same "
+              f"{es}-byte rank-r elements as the GPU metric")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
+                   "rank": list(wl.ranks), "context": wl.context, "sampled_units": len(sample_heads)},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# the CUDA arm
+# ----------------------------------------------------------------------------------------------
+
+def build_layer(wl, device, binding, keep_heads=()):
+    """Creates the layer and fills `context` rows through eigen_attn_append_kv.  Returns the layer, the
+    bases, and for the units (0, h), h in keep_heads, the raw K/V history as float64 arrays."""
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    dt = synth.torch_dtype(wl.dtype)
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + 1, dt, U_k, U_v, device=device)
+    W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K", device=device)
+    W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V", device=device)
+    hist = {h: ([], []) for h in keep_heads}
+    for ci, c in enumerate(range(0, wl.context, FILL_CHUNK)):
+        t = min(FILL_CHUNK, wl.context - c)
+        k = synth.lowrank_rows(W_k, wl.batch, t, wl.sigma, wl.index, "K", chunk=ci, dtype=dt, device=device)
+        v = synth.lowrank_rows(W_v, wl.batch, t, wl.sigma, wl.index, "V", chunk=ci, dtype=dt, device=device)
+        lay.append_kv(k, v)
+        for h in keep_heads:
+            hist[h][0].append(k[0, :, h, :].double().cpu().numpy())
+            hist[h][1].append(v[0, :, h, :].double().cpu().numpy())
+    hist = {h: (np.concatenate(a), np.concatenate(b)) for h, (a, b) in hist.items()}
+    k_new = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device=device)
+    v_new = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt, device=device)
+    q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt, device=device)
+    torch.cuda.synchronize(device)
+    return lay, ranks, U_k, U_v, hist, q, k_new, v_new
+
+
+def run_ours(args, wl):
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2408_05646_b200 import build
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        dist.barrier()
+    from paper_2408_05646_b200 import binding
+
+    do_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+    keep_heads = list(range(0, wl.n_heads, 2)) if do_cpu else []      # 16 sampled units of sequence 0
+    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep_heads)
+    n0 = wl.context
+    assert lay.len == n0
+    stream = torch.cuda.current_stream(device)
+    out = torch.empty_like(q)
+
+    def step():
+        lay.set_len(n0)
+        lay.decode_step(q, k_new, v_new, out=out)
+
+    def sync_all():
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(device)
+
+    # ---- device-resident timing, with per-step events around the split-KV kernel
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for e0, e1 in ev:           # create the underlying CUDA events
+        e0.record(stream)
+        e1.record(stream)
+    for _ in range(args.warmup):
+        step()
+    sync_all()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = lay.launch_count()
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    t_start.record(stream)
+    for i in range(args.steps):
+        lay.set_decode_events(ev[i][0], ev[i][1])
+        step()
+    t_stop.record(stream)
+    sync_all()
+    lay.set_decode_events(None, None)
+    launches = lay.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    lay.poll_status()
+    ms_total = t_start.elapsed_time(t_stop)
+    kern_ms = [a.elapsed_time(b) for a, b in ev]
+    if world > 1:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    bytes_step = algorithmic_bytes(wl, ranks, ranks, n0 + 1)
+    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    kern_avg_ms = sum(kern_ms) / len(kern_ms)
+    peak, peak_src = measured_peaks()
+    achieved = bytes_step / (kern_avg_ms * 1e-3) / 1e9
+
+    # ---- end to end: host tensors in, host tensor out, through the C ABI
+    hq, hk, hv = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+    hout = torch.empty_like(hq).pin_memory()
+    for _ in range(args.warmup):
+        lay.set_len(n0)
+        lay.decode_step_host(hq, hk, hv, hout)
+    sync_all()
+    t0 = time.perf_counter()
+    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_start.record(stream)
+    for _ in range(args.steps):
+        lay.set_len(n0)
+        lay.decode_step_host(hq, hk, hv, hout)
+    e_stop.record(stream)
+    sync_all()
+    e2e_ms = e_start.elapsed_time(e_stop)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_ms_step = e2e_ms / args.steps
+    e2e_value = world * bytes_step / (e2e_ms_step * 1e-3) / 1e9
+    io_bytes = hq.numel() * hq.element_size()
+    same = bool(torch.equal(hout, out.cpu()))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- the oracle on the host cores: a bounded sample, also a full-size parity check
+    cpu = None
+    parity = None
+    if do_cpu:
+        ref = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, keep_heads, history=hist)
+        qn, kn, vn = q.double().cpu().numpy(), k_new.double().cpu().numpy(), v_new.double().cpu().numpy()
+        sec, res = oracle_timed_steps(ref, wl, qn, kn, vn, steps=20, warmup=2)
+        es = 2 if wl.dtype == "bf16" else 4
+        sample_bytes = (n0 + 1) * sum(2 * ranks[h] for h in keep_heads) * es
+        cpu = {"value": sample_bytes / sec / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "us_per_step_sample": sec * 1e6,
+               "us_per_step_scaled_to_all_units": sec * 1e6 * wl.batch * wl.n_heads / len(keep_heads),
+               "sample": f"{len(keep_heads)} of {wl.batch * wl.n_heads} (sequence, head) units (sequence 0, every "
+                         f"second head), full context, 20 timed steps; history projected beforehand"}
+        g = out.double().cpu().numpy()
+        errs = [np.abs(g[0, 0, h] - res[(0, h)]) for h in keep_heads]
+        parity = {"units": len(keep_heads), "max_abs": float(max(e.max() for e in errs)),
+                  "mean_abs": float(np.mean([e.mean() for e in errs])),
+                  "tolerance": "max_abs <= 2e-2, mean_abs <= 2e-3 (bf16 storage)"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
+        "tokens_per_s": world * wl.batch / (ms_step * 1e-3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 storage, f32 accumulate" if wl.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "batch_per_gpu": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
+                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1,
+                   "cache_gb_per_gpu": bytes_step / 1e9, "parallelism": f"{world} independent batch shard(s)",
+                   "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
+        "frac_of_nominal_8TBs": value / world / 8000.0,
+        "roofline": {"bound": "hbm", "kernel": "decode_splitkv_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                     "kernel_us": kern_avg_ms * 1e3, "algorithmic_bytes": bytes_step, "traffic": None},
+        "e2e": {"value": e2e_value, "unit": UNIT, "us_per_step": e2e_ms_step * 1e3,
+                "h2d_bytes_per_step": 3 * io_bytes, "d2h_bytes_per_step": io_bytes,
+                "matches_device_path": same},
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+        line["parity_full_size"] = parity
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, wl)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
