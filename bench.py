@@ -65,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -171,7 +171,8 @@ def run_reference(args, wl):
     k_new = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt).double().numpy()
     v_new = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt).double().numpy()
     q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt).double().numpy()
-    sec, _ = oracle_timed_steps(lay, wl, q, k_new, v_new, args.steps, args.warmup)
+    steps = min(args.steps, 40)          # ~0.3 s of host work per step: keep the whole run to a minute
+    sec, _ = oracle_timed_steps(lay, wl, q, k_new, v_new, steps, min(args.warmup, 5))
     es = 2 if wl.dtype == "bf16" else 4
     sample_bytes = (wl.context + 1) * sum(2 * ranks[h] for h in sample_heads) * es
     gbs = sample_bytes / sec / 1e9
@@ -181,7 +182,7 @@ def run_reference(args, wl):
               f"{es}-byte rank-r elements as the GPU metric")
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": min(args.warmup, 5), "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
                    "rank": list(wl.ranks), "context": wl.context, "sampled_units": len(sample_heads)},
@@ -378,8 +379,8 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
