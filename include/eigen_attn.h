@@ -102,6 +102,26 @@ ea_status eigen_attn_append_kv(eigen_attn_t h, const void* d_k, const void* d_v,
 ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                             int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
+/* (No counterpart in the paper: an engineering variant of eigen_attn_decode.)
+ * Same result as eigen_attn_decode, but the split-KV partial results (per-piece max, sum and
+ * un-normalised o') are kept in an array built into the library image instead of the workspace.
+ * It is meant for callers that must not obtain device memory while they run -- e.g. a plugin inside
+ * an inference engine whose memory plan is frozen, a real-time loop where cudaMalloc's device-wide
+ * synchronisation is unacceptable, or a process whose memory pool is already handed out in full --
+ * and that therefore want the decode call itself to depend on no scratch they have to provide.
+ *   - Limit: (batch * n_heads + decode CTAs) * (4 + widest rp_v) <= 270336 floats (2048 slots of 132
+ *     floats, 1.03 MiB, resident on every GPU that loads the library until the process exits).
+ *     Larger layers get EA_ERR_CAPACITY and a message; use eigen_attn_decode for them.
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query, no
+ *     allocation); make that first call outside any stream capture.  The call itself never calls
+ *     cudaMalloc/cudaFree or any allocating routine.
+ *   - All handles and all calls on a device share the one array, and it keeps whatever the previous
+ *     call left.  Nothing in it has to start at zero: every slot the combine step reads is written
+ *     earlier in the same call.  Two calls that may overlap on the GPU (different streams, or several
+ *     host threads) race on the array and give undefined results; serialise them. */
+ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                                   int64_t stride_b_out, uint32_t flags, void* cuda_stream);
+
 /* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token).
  * d_k and d_v share the batch stride `stride_b_kv`. */
 ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q,

@@ -52,6 +52,7 @@ SYMBOLS = {
     "eigen_attn_destroy": (None, [_vp]),
     "eigen_attn_append_kv": (_i32, [_vp, _vp, _vp, _i32, _i64, _i64, _u32, _vp]),
     "eigen_attn_decode": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
+    "eigen_attn_decode_static": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_decode_step": (_i32, [_vp, _vp, _i64, _vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_decode_step_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _u32, _vp]),
     "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _i64, _i64, _u32, _vp]),
@@ -222,6 +223,18 @@ class EigenAttnLayer:
             _, _, sbo, _ = self._tok(out, 1)
         self._check(lib.eigen_attn_decode(self.handle, pq, sbq, out.data_ptr(), sbo, flags, _stream_ptr(stream)),
                     "eigen_attn_decode")
+        return out
+
+    def decode_static(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """eigen_attn_decode_static: decode with the partials in the library's built-in scratch array
+        (for callers that cannot hand the call any scratch memory).  Calls that could overlap on the
+        GPU share that array and must be serialised."""
+        pq, _, sbq, _ = self._tok(q, 1)
+        if out is None:
+            out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+        _, _, sbo, _ = self._tok(out, 1)
+        self._check(lib.eigen_attn_decode_static(self.handle, pq, sbq, out.data_ptr(), sbo, 0,
+                                                 _stream_ptr(stream)), "eigen_attn_decode_static")
         return out
 
     def decode_step(self, q, k, v, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

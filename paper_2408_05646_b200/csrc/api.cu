@@ -364,6 +364,80 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   return EA_OK;
 }
 
+// Same computation and launch plan as eigen_attn_decode, with the split-KV partials in the library's
+// built-in device array instead of the caller's workspace.  Kept apart from do_decode on purpose.
+ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                                   int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_static: NULL q or out");
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
+    return fail(h, EA_ERR_INVALID_ARG, "decode_static: unknown flag 0x%x", flags);
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_static: the cache is empty");
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const Layout& L = h->L;
+  const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
+  const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
+  const int sms = h->opt_ctas > 0 ? static_cast<int>(h->opt_ctas) : h->sm_count;
+  int tile_rows = 128;
+  if (h->opt_tile_rows > 0) {
+    tile_rows = static_cast<int>(h->opt_tile_rows);
+  } else {
+    while (tile_rows > 16 && static_cast<int64_t>(B) * H * ((n + tile_rows - 1) / tile_rows) < 4ll * sms)
+      tile_rows >>= 1;
+  }
+  int stage_bytes = 0, stages = 0;
+  for (;;) {
+    stage_bytes = static_cast<int>(align_up(static_cast<size_t>(tile_rows) * (L.max_rp_k + L.max_rp_v) * L.es, 128));
+    stages = (kSmemLimit - fixed) / stage_bytes;
+    if (stages >= 3 || tile_rows <= 16) break;
+    tile_rows >>= 1;
+  }
+  if (stages > 12) stages = 12;
+  if (h->opt_stages > 0 && h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
+  if (stages < 1)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode_static: a tile of %d rows does not fit in shared memory", tile_rows);
+  const int nt = (n + tile_rows - 1) / tile_rows;
+  const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
+  int grid = sms;
+  const int64_t cap = w_total / L.max_w;
+  if (grid > cap) grid = static_cast<int>(cap);
+  if (grid < 1) grid = 1;
+
+  const size_t need = (static_cast<size_t>(B) * H + grid) * L.part_stride;
+  if (need > ea::kStaticPartialFloats)
+    return fail(h, EA_ERR_CAPACITY,
+                "decode_static: (batch*heads + CTAs) * (4 + widest rp_v) = %zu floats exceeds the built-in "
+                "scratch of %zu floats; use eigen_attn_decode with a workspace",
+                need, static_cast<size_t>(ea::kStaticPartialFloats));
+  float* scratch = nullptr;
+  cudaError_t e = ea::static_partials(&scratch);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_static: address of the built-in scratch");
+
+  ea::DecodeParams p{};
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
+  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
+  p.partials = scratch;
+  p.status = dev_status(h);
+  p.part_stride = L.part_stride;
+  p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
+  p.tile_rows = tile_rows; p.nt = nt; p.stages = stages; p.stage_bytes = stage_bytes;
+  p.v_tile_off = tile_rows * L.max_rp_k * L.es;
+  p.w_total = w_total;
+  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  p.flags = flags;
+  const size_t smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
+  e = ea::launch_decode(p, h->desc.dtype, grid, smem, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_static launch");
+  ea::CombineParams c{};
+  c.heads = p.heads; c.basis = p.basis; c.partials = scratch; c.out = d_out;
+  c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
+  c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
+  c.w_total = w_total; c.flags = flags;
+  e = ea::launch_combine(c, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_static combine launch");
+  return EA_OK;
+}
+
 ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v, int32_t T,
                              int64_t stride_b, int64_t stride_t, void* d_out, int64_t out_stride_b,
                              int64_t out_stride_t, uint32_t flags, void* cuda_stream) {

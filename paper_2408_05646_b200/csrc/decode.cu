@@ -464,7 +464,31 @@ __global__ void __launch_bounds__(128) combine_lift_kernel(const CombineParams p
   }
 }
 
+// Scratch of eigen_attn_decode_static: split-KV partials kept inside the library image, so that the
+// call needs no caller-provided scratch.  2048 slots x (4 + 128) floats = 1.03 MiB on every GPU that
+// loads the library.  Host code must not pass this name to a kernel: on the host it is only a stand-in
+// for the device object; static_partials() asks the runtime for the real device address.
+static __device__ __align__(256) float g_static_partials[kStaticPartialFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_static_partials_addr[kMaxDevices] = {};
+
 }  // namespace
+
+cudaError_t static_partials(float** ptr) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_static_partials_addr[dev]) {
+    float* p = nullptr;
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials);   // `dev` is current
+    if (e != cudaSuccess) return e;
+    g_static_partials_addr[dev] = p;
+  }
+  *ptr = g_static_partials_addr[dev];
+  return cudaSuccess;
+}
 
 size_t decode_fixed_smem_bytes() { return sizeof(DecodeSmemFixed); }
 

@@ -109,6 +109,11 @@ cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, ui
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 
+// Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
+// library's own partials array on the current device.  Resolves the address on first use per device.
+constexpr size_t kStaticPartialFloats = 2048 * 132;
+cudaError_t static_partials(float** ptr);
+
 size_t decode_fixed_smem_bytes();         // shared memory the decode kernel needs besides the ring
 cudaError_t decode_configure(int dtype);  // opt in to large dynamic shared memory (once per device)
 
