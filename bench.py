@@ -384,10 +384,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
+    ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = synth.WORKLOADS[args.workload]
+    if args.batch or args.context:
+        import dataclasses
+        wl = dataclasses.replace(wl, batch=args.batch or wl.batch, context=args.context or wl.context,
+                                 name=f"{wl.name}[batch={args.batch or wl.batch},context={args.context or wl.context}]")
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:
             run_reference(args, wl)
