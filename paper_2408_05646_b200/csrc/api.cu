@@ -20,6 +20,7 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr int kMaxDecodeCtas = 1024;
 constexpr int kSmemLimit = 227 * 1024;
+constexpr int kInFlightBytes = 120 * 1024;   // target bytes of bulk copies in flight per SM (decode)
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 int ceil8(int r) { return (r + 7) / 8 * 8; }
@@ -147,12 +148,20 @@ ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
   return EA_OK;
 }
 
-ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
-                    uint32_t flags, cudaStream_t s) {
-  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
+struct DecodePlan {
+  ea::DecodeParams p;
+  ea::CombineParams c;
+  int grid = 0;
+  size_t smem = 0;
+};
+
+// Validates a decode request and plans its two launches; `partials` is where the split-KV pieces go.
+ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t stride_b_q, void* d_out,
+                      int64_t stride_b_out, uint32_t flags, float* partials, DecodePlan* plan) {
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "%s: NULL q or out", who);
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
-    return fail(h, EA_ERR_INVALID_ARG, "decode: unknown flag 0x%x", flags);
-  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
+    return fail(h, EA_ERR_INVALID_ARG, "%s: unknown flag 0x%x", who, flags);
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "%s: the cache is empty", who);
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
@@ -174,9 +183,17 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
     tile_rows >>= 1;
   }
   if (stages > 12) stages = 12;
-  if (h->opt_stages > 0 && h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
+  if (h->opt_stages > 0) {
+    if (h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
+  } else {
+    // Measured on B200: about 120 KB of copies in flight per SM saturates HBM; deeper rings lose
+    // bandwidth again (more concurrent DRAM streams), so the ring is not simply made as deep as fits.
+    int want = (kInFlightBytes + stage_bytes - 1) / stage_bytes;
+    if (want < 3) want = 3;
+    if (want < stages) stages = want;
+  }
   if (stages < 1)
-    return fail(h, EA_ERR_UNSUPPORTED, "decode: a tile of %d rows does not fit in shared memory", tile_rows);
+    return fail(h, EA_ERR_UNSUPPORTED, "%s: a tile of %d rows does not fit in shared memory", who, tile_rows);
 
   const int nt = (n + tile_rows - 1) / tile_rows;
   const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
@@ -185,10 +202,11 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
   if (grid > cap) grid = static_cast<int>(cap);
   if (grid < 1) grid = 1;
 
-  ea::DecodeParams p{};
+  ea::DecodeParams& p = plan->p;
+  p = ea::DecodeParams{};
   p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
-  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b;
-  p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
+  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
+  p.partials = partials;
   p.status = dev_status(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
@@ -197,21 +215,35 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
   p.w_total = w_total;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
-  const size_t smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
+  plan->grid = grid;
+  plan->smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
 
-  if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  cudaError_t e = ea::launch_decode(p, h->desc.dtype, grid, smem, s, &h->launches);
-  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
-  if (e != cudaSuccess) return cuda_fail(h, e, "decode launch");
-
-  ea::CombineParams c{};
-  c.heads = p.heads; c.basis = p.basis; c.partials = p.partials; c.out = d_out;
+  ea::CombineParams& c = plan->c;
+  c = ea::CombineParams{};
+  c.heads = p.heads; c.basis = p.basis; c.partials = partials; c.out = d_out;
   c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
   c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
   c.w_total = w_total; c.flags = flags;
-  e = ea::launch_combine(c, h->desc.dtype, s, &h->launches);
-  if (e != cudaSuccess) return cuda_fail(h, e, "combine launch");
   return EA_OK;
+}
+
+ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, bool events, cudaStream_t s) {
+  if (events && h->ev_start) cudaEventRecord(h->ev_start, s);
+  cudaError_t e = ea::launch_decode(plan.p, h->desc.dtype, plan.grid, plan.smem, s, &h->launches);
+  if (events && h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, who);
+  e = ea::launch_combine(plan.c, h->desc.dtype, s, &h->launches);
+  if (e != cudaSuccess) return cuda_fail(h, e, who);
+  return EA_OK;
+}
+
+ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
+                    uint32_t flags, cudaStream_t s) {
+  DecodePlan plan;
+  const ea_status st = plan_decode(h, "decode", d_q, stride_b, d_out, stride_b_out, flags,
+                                   reinterpret_cast<float*>(h->ws + h->L.off_partials), &plan);
+  if (st != EA_OK) return st;
+  return launch_plan(h, "decode launch", plan, true, s);
 }
 
 }  // namespace
@@ -365,77 +397,25 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
 }
 
 // Same computation and launch plan as eigen_attn_decode, with the split-KV partials in the library's
-// built-in device array instead of the caller's workspace.  Kept apart from do_decode on purpose.
+// built-in device array instead of the caller's workspace.
 ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                    int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_static: NULL q or out");
-  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
-    return fail(h, EA_ERR_INVALID_ARG, "decode_static: unknown flag 0x%x", flags);
-  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_static: the cache is empty");
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  const Layout& L = h->L;
-  const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
-  const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
-  const int sms = h->opt_ctas > 0 ? static_cast<int>(h->opt_ctas) : h->sm_count;
-  int tile_rows = 128;
-  if (h->opt_tile_rows > 0) {
-    tile_rows = static_cast<int>(h->opt_tile_rows);
-  } else {
-    while (tile_rows > 16 && static_cast<int64_t>(B) * H * ((n + tile_rows - 1) / tile_rows) < 4ll * sms)
-      tile_rows >>= 1;
-  }
-  int stage_bytes = 0, stages = 0;
-  for (;;) {
-    stage_bytes = static_cast<int>(align_up(static_cast<size_t>(tile_rows) * (L.max_rp_k + L.max_rp_v) * L.es, 128));
-    stages = (kSmemLimit - fixed) / stage_bytes;
-    if (stages >= 3 || tile_rows <= 16) break;
-    tile_rows >>= 1;
-  }
-  if (stages > 12) stages = 12;
-  if (h->opt_stages > 0 && h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
-  if (stages < 1)
-    return fail(h, EA_ERR_UNSUPPORTED, "decode_static: a tile of %d rows does not fit in shared memory", tile_rows);
-  const int nt = (n + tile_rows - 1) / tile_rows;
-  const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
-  int grid = sms;
-  const int64_t cap = w_total / L.max_w;
-  if (grid > cap) grid = static_cast<int>(cap);
-  if (grid < 1) grid = 1;
-
-  const size_t need = (static_cast<size_t>(B) * H + grid) * L.part_stride;
+  DecodePlan plan;
+  ea_status st = plan_decode(h, "decode_static", d_q, stride_b_q, d_out, stride_b_out, flags, nullptr, &plan);
+  if (st != EA_OK) return st;
+  const size_t need = (static_cast<size_t>(plan.p.B) * plan.p.H + plan.grid) * plan.p.part_stride;
   if (need > ea::kStaticPartialFloats)
     return fail(h, EA_ERR_CAPACITY,
                 "decode_static: (batch*heads + CTAs) * (4 + widest rp_v) = %zu floats exceeds the built-in "
                 "scratch of %zu floats; use eigen_attn_decode with a workspace",
                 need, static_cast<size_t>(ea::kStaticPartialFloats));
   float* scratch = nullptr;
-  cudaError_t e = ea::static_partials(&scratch);
+  const cudaError_t e = ea::static_partials(&scratch);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_static: address of the built-in scratch");
-
-  ea::DecodeParams p{};
-  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
-  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
-  p.partials = scratch;
-  p.status = dev_status(h);
-  p.part_stride = L.part_stride;
-  p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
-  p.tile_rows = tile_rows; p.nt = nt; p.stages = stages; p.stage_bytes = stage_bytes;
-  p.v_tile_off = tile_rows * L.max_rp_k * L.es;
-  p.w_total = w_total;
-  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
-  p.flags = flags;
-  const size_t smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
-  e = ea::launch_decode(p, h->desc.dtype, grid, smem, s, &h->launches);
-  if (e != cudaSuccess) return cuda_fail(h, e, "decode_static launch");
-  ea::CombineParams c{};
-  c.heads = p.heads; c.basis = p.basis; c.partials = scratch; c.out = d_out;
-  c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
-  c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
-  c.w_total = w_total; c.flags = flags;
-  e = ea::launch_combine(c, h->desc.dtype, s, &h->launches);
-  if (e != cudaSuccess) return cuda_fail(h, e, "decode_static combine launch");
-  return EA_OK;
+  plan.p.partials = scratch;
+  plan.c.partials = scratch;
+  return launch_plan(h, "decode_static launch", plan, false, static_cast<cudaStream_t>(cuda_stream));
 }
 
 ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v, int32_t T,

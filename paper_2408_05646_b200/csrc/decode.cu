@@ -95,6 +95,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Position in the shared-memory ring: slot index and the parity of the slot's current fill.
+struct RingPos {
+  int stage = 0;
+  uint32_t parity = 0;
+  uint32_t count = 0;     // tiles so far
+  __device__ __forceinline__ void advance(int stages) {
+    ++count;
+    if (++stage == stages) { stage = 0; parity ^= 1u; }
+  }
+};
+
+// L2 policy for data that is read once: evict it first.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void* dst, const void* src, uint32_t bytes, void* bar,
+                                              uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+
 // ---------------------------------------------------------------- element access
 
 template <typename T>
@@ -147,7 +173,7 @@ __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
 template <typename T, int NCH>
 __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
                                             unsigned char* ring, const HeadInfo& hd, int i0, int i1,
-                                            uint32_t& it, int warp, int lane, int slot) {
+                                            RingPos& pos, int warp, int lane, int slot) {
   constexpr int EPC = Elem<T>::kPerChunk;
   const int pair = lane >> 1, half = lane & 1;
   const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
@@ -182,9 +208,9 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   volatile int* abort_flag = &fx->abort_flag;
   float m = -INFINITY, l = 0.f;
   for (int i = i0; i < i1; ++i) {
-    const int stage = it % p.stages;
-    const uint32_t parity = (it / p.stages) & 1u;
-    ++it;
+    const int stage = pos.stage;
+    const uint32_t parity = pos.parity;
+    pos.advance(p.stages);
     if (*abort_flag) continue;
     if (!mbar_wait(&fx->full[stage], parity, p.status)) {
       *abort_flag = 1;
@@ -353,39 +379,60 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
   if (warp == kDecodeConsumerWarps) {
     // ------------------------------------------------------------ producer
     if (lane == 0) {
-      uint32_t it = 0;
-      int cur_h = -1;
-      HeadInfo hd{};
-      for (long long F = f_lo; F < f_hi; ++F, ++it) {
-        if (*abort_flag) break;
+      const uint64_t policy = policy_evict_first();
+      RingPos pos;
+      bool ok = true;
+      long long F = f_lo;
+      while (F < f_hi && ok) {
+        // one (CTA, unit) piece: tiles [i0, i1) of `unit`; everything per tile below is incremental
         const int unit = static_cast<int>(F / p.nt);
-        const int i = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
+        const int i0 = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
+        const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + (f_hi - F)));
         const int h = unit / p.B, b = unit - h * p.B;
-        if (h != cur_h) { hd = p.heads[h]; cur_h = h; }
-        const int stage = it % p.stages;
-        const uint32_t k = it / p.stages;
-        if (k > 0 && !mbar_wait(&fx->empty[stage], (k - 1) & 1u, p.status)) {
-          *abort_flag = 1;
-          break;
+        const HeadInfo hd = p.heads[h];
+        const uint32_t rowb_k = hd.rp_k * sizeof(T), rowb_v = hd.rp_v * sizeof(T);
+        const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i0) * p.tile_rows;
+        const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
+        const char* src_v = p.cache + hd.v_off + row0 * rowb_v;
+        const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
+        for (int i = i0; i < i1; ++i) {
+          if (*abort_flag) { ok = false; break; }
+          if (pos.count >= static_cast<uint32_t>(p.stages) &&
+              !mbar_wait(&fx->empty[pos.stage], pos.parity ^ 1u, p.status)) {
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+          uint32_t bytes_k = tile_k, bytes_v = tile_v;
+          if (i == p.nt - 1) {            // ragged last tile of the unit
+            const uint32_t rows = p.n - i * p.tile_rows;
+            bytes_k = rows * rowb_k;
+            bytes_v = rows * rowb_v;
+          }
+          unsigned char* dst = ring + static_cast<size_t>(pos.stage) * p.stage_bytes;
+          void* bar = &fx->full[pos.stage];
+          mbar_arrive_expect_tx(bar, bytes_k + bytes_v);
+          bulk_g2s_hint(dst, src_k, bytes_k, bar, policy);
+          bulk_g2s_hint(dst + p.v_tile_off, src_v, bytes_v, bar, policy);
+          src_k += tile_k;
+          src_v += tile_v;
+          pos.advance(p.stages);
         }
-        const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
-        const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i) * p.tile_rows;
-        const uint32_t bytes_k = static_cast<uint32_t>(rows) * hd.rp_k * sizeof(T);
-        const uint32_t bytes_v = static_cast<uint32_t>(rows) * hd.rp_v * sizeof(T);
-        unsigned char* dst = ring + static_cast<size_t>(stage) * p.stage_bytes;
-        mbar_arrive_expect_tx(&fx->full[stage], bytes_k + bytes_v);
-        bulk_g2s(dst, p.cache + hd.k_off + row0 * hd.rp_k * sizeof(T), bytes_k, &fx->full[stage]);
-        bulk_g2s(dst + p.v_tile_off, p.cache + hd.v_off + row0 * hd.rp_v * sizeof(T), bytes_v,
-                 &fx->full[stage]);
+        F += i1 - i0;
       }
-      // Make sure every copy this thread issued has landed before the CTA can exit.
-      const uint32_t first = it > static_cast<uint32_t>(p.stages) ? it - p.stages : 0u;
-      for (uint32_t j = first; j < it; ++j)
-        mbar_wait(&fx->full[j % p.stages], (j / p.stages) & 1u, p.status);
+      // Make sure every copy this thread issued has landed before the CTA can exit: walk back over
+      // the last min(count, stages) fills.
+      const uint32_t pending = pos.count < static_cast<uint32_t>(p.stages) ? pos.count : p.stages;
+      int st = pos.stage;
+      uint32_t par = pos.parity;
+      for (uint32_t j = 0; j < pending; ++j) {
+        if (st == 0) { st = p.stages - 1; par ^= 1u; } else { --st; }
+        mbar_wait(&fx->full[st], par, p.status);
+      }
     }
   } else {
     // ------------------------------------------------------------ consumers
-    uint32_t it = 0;
+    RingPos pos;
     long long F = f_lo;
     while (F < f_hi) {
       const int unit = static_cast<int>(F / p.nt);
@@ -400,14 +447,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, it, warp, lane, slot); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
       }
       F += i1 - i0;
     }
