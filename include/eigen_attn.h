@@ -122,7 +122,8 @@ ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b_q,
 ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                    int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
-/* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token).
+/* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token), fused into a
+ * single launch when the cache already holds at least one row.
  * d_k and d_v share the batch stride `stride_b_kv`. */
 ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q,
                                  const void* d_k, const void* d_v, int64_t stride_b_kv,
@@ -167,7 +168,9 @@ typedef enum {
   EA_OPT_DECODE_CTAS = 1,     /* CTAs of the split-KV decode kernel; 0 = one per SM                      */
   EA_OPT_DECODE_TILE_ROWS = 2,/* rows per shared-memory tile (multiple of 16, <= 128); 0 = automatic     */
   EA_OPT_DECODE_STAGES = 3,   /* depth of the shared-memory ring (2..12); 0 = as many as fit              */
-  EA_OPT_PREFILL_IMPL = 4     /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel      */
+  EA_OPT_PREFILL_IMPL = 4,    /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel      */
+  EA_OPT_DECODE_FUSED = 5     /* 1 (default): a decode step is one launch (append row, attend, merge the
+                                 splits, lift); 0: separate append / attention / merge launches           */
 } ea_option;
 ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value);
 

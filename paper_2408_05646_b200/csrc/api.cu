@@ -29,7 +29,7 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_staging = 0, off_qp = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0;
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -89,6 +89,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_basis = off;    off = align_up(off + basis * sizeof(float));
   L->off_partials = off;
   off = align_up(off + (static_cast<size_t>(d->batch) * H + kMaxDecodeCtas) * L->part_stride * sizeof(float));
+  L->off_counters = off; off = align_up(off + static_cast<size_t>(d->batch) * H * sizeof(int));
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
   L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
@@ -104,7 +105,7 @@ struct eigen_attn {
   char* ws = nullptr;
   int32_t len = 0;
   int sm_count = 148;
-  int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0;
+  int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   char err[256];
@@ -128,6 +129,7 @@ ea_status cuda_fail(eigen_attn_t h, cudaError_t e, const char* what) {
 const HeadInfo* dev_heads(eigen_attn_t h) { return reinterpret_cast<const HeadInfo*>(h->ws + h->L.off_heads); }
 const float* dev_basis(eigen_attn_t h) { return reinterpret_cast<const float*>(h->ws + h->L.off_basis); }
 int* dev_status(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_status); }
+int* dev_counters(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_counters); }
 
 ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T, int64_t stride_b,
                     int64_t stride_t, uint32_t flags, cudaStream_t s) {
@@ -156,8 +158,11 @@ struct DecodePlan {
 };
 
 // Validates a decode request and plans its two launches; `partials` is where the split-KV pieces go.
+// With k_new/v_new the cache holds len rows and the new token's row is projected, stored at row len and
+// attended inside the same launch; otherwise the len cached rows are attended.
 ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t stride_b_q, void* d_out,
-                      int64_t stride_b_out, uint32_t flags, float* partials, DecodePlan* plan) {
+                      int64_t stride_b_out, uint32_t flags, float* partials, const void* k_new,
+                      const void* v_new, int64_t kv_stride_b, DecodePlan* plan) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "%s: NULL q or out", who);
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
     return fail(h, EA_ERR_INVALID_ARG, "%s: unknown flag 0x%x", who, flags);
@@ -206,7 +211,10 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p = ea::DecodeParams{};
   p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
   p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
+  p.k_new = k_new; p.v_new = v_new; p.kv_stride_b = kv_stride_b;
+  p.out = d_out; p.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
   p.partials = partials;
+  p.counters = h->opt_fused ? dev_counters(h) : nullptr;
   p.status = dev_status(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
@@ -232,8 +240,10 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
   cudaError_t e = ea::launch_decode(plan.p, h->desc.dtype, plan.grid, plan.smem, s, &h->launches);
   if (events && h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, who);
-  e = ea::launch_combine(plan.c, h->desc.dtype, s, &h->launches);
-  if (e != cudaSuccess) return cuda_fail(h, e, who);
+  if (plan.p.counters == nullptr) {   // the merge + lift as its own launch
+    e = ea::launch_combine(plan.c, h->desc.dtype, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, who);
+  }
   return EA_OK;
 }
 
@@ -241,9 +251,33 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
                     uint32_t flags, cudaStream_t s) {
   DecodePlan plan;
   const ea_status st = plan_decode(h, "decode", d_q, stride_b, d_out, stride_b_out, flags,
-                                   reinterpret_cast<float*>(h->ws + h->L.off_partials), &plan);
+                                   reinterpret_cast<float*>(h->ws + h->L.off_partials), nullptr, nullptr, 0,
+                                   &plan);
   if (st != EA_OK) return st;
   return launch_plan(h, "decode launch", plan, true, s);
+}
+
+// One generated token.  Fused form: a single launch projects and stores the new row, attends over the
+// cached rows plus that row, merges the splits and lifts.  It needs at least one cached row (the work
+// decomposition is over cached rows); otherwise, or with fusion switched off, append then decode.
+ea_status do_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q, const void* d_k, const void* d_v,
+                  int64_t stride_b_kv, void* d_out, int64_t stride_b_out, uint32_t flags, cudaStream_t s) {
+  if (h->opt_fused && h->len >= 1) {
+    if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL k or v");
+    if (h->len + 1 > h->desc.n_max)
+      return fail(h, EA_ERR_CAPACITY, "decode_step: len %d + 1 exceeds n_max %d", h->len, h->desc.n_max);
+    DecodePlan plan;
+    const ea_status st = plan_decode(h, "decode_step", d_q, stride_b_q, d_out, stride_b_out, flags,
+                                     reinterpret_cast<float*>(h->ws + h->L.off_partials), d_k, d_v, stride_b_kv,
+                                     &plan);
+    if (st != EA_OK) return st;
+    const ea_status sl = launch_plan(h, "decode_step launch", plan, true, s);
+    if (sl == EA_OK) h->len += 1;
+    return sl;
+  }
+  const ea_status st = do_append(h, d_k, d_v, 1, stride_b_kv, stride_b_kv, 0, s);
+  if (st != EA_OK) return st;
+  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags, s);
 }
 
 }  // namespace
@@ -322,6 +356,7 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
   h->ws = static_cast<char*>(d_workspace);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = cudaMemsetAsync(h->ws + L.off_status, 0, 64, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + L.off_counters, 0, static_cast<size_t>(desc->batch) * H * sizeof(int), s);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(h->ws + L.off_heads, L.heads.data(), sizeof(HeadInfo) * H, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess)
@@ -363,9 +398,7 @@ ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
     return fail(h, EA_ERR_INVALID_ARG, "decode_step: unknown flag 0x%x", flags);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  const ea_status st = do_append(h, d_k, d_v, 1, stride_b_kv, stride_b_kv, 0, s);
-  if (st != EA_OK) return st;
-  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags, s);
+  return do_step(h, d_q, stride_b_q, d_k, d_v, stride_b_kv, d_out, stride_b_out, flags, s);
 }
 
 ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const void* h_k, const void* h_v,
@@ -386,9 +419,7 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   if (e == cudaSuccess) e = cudaMemcpyAsync(sv, h_v, bytes, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_step_host H2D");
   const int64_t sb = static_cast<int64_t>(h->desc.n_heads) * h->desc.d_head;
-  ea_status st = do_append(h, sk, sv, 1, sb, sb, 0, s);
-  if (st != EA_OK) return st;
-  st = do_decode(h, sq, sb, so, sb, 0, s);
+  const ea_status st = do_step(h, sq, sb, sk, sv, sb, so, sb, 0, s);
   if (st != EA_OK) return st;
   e = cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -402,7 +433,8 @@ ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stri
                                    int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   DecodePlan plan;
-  ea_status st = plan_decode(h, "decode_static", d_q, stride_b_q, d_out, stride_b_out, flags, nullptr, &plan);
+  ea_status st = plan_decode(h, "decode_static", d_q, stride_b_q, d_out, stride_b_out, flags, nullptr, nullptr,
+                             nullptr, 0, &plan);
   if (st != EA_OK) return st;
   const size_t need = (static_cast<size_t>(plan.p.B) * plan.p.H + plan.grid) * plan.p.part_stride;
   if (need > ea::kStaticPartialFloats)
@@ -477,7 +509,12 @@ ea_status eigen_attn_poll_status(eigen_attn_t h, void* cuda_stream) {
   if (e == cudaSuccess) e = cudaMemsetAsync(dev_status(h), 0, sizeof(int), s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return cuda_fail(h, e, "poll_status");
-  if (word == ea::kStatusTimeout) return fail(h, EA_ERR_TIMEOUT, "a device-side wait exceeded its bound");
+  if (word == ea::kStatusTimeout) {
+    // an aborted launch may have left arrival counters half way: clear them for the next call
+    cudaMemsetAsync(dev_counters(h), 0, static_cast<size_t>(h->desc.batch) * h->desc.n_heads * sizeof(int), s);
+    cudaStreamSynchronize(s);
+    return fail(h, EA_ERR_TIMEOUT, "a device-side wait exceeded its bound");
+  }
   return EA_OK;
 }
 
@@ -529,6 +566,10 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
       if (value < 0 || value > 2)
         return fail(h, EA_ERR_INVALID_ARG, "PREFILL_IMPL %lld", static_cast<long long>(value));
       h->opt_prefill = value;
+      return EA_OK;
+    case EA_OPT_DECODE_FUSED:
+      if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "DECODE_FUSED %lld", static_cast<long long>(value));
+      h->opt_fused = value;
       return EA_OK;
     default:
       return fail(h, EA_ERR_INVALID_ARG, "unknown option %d", option);

@@ -7,10 +7,15 @@
 // One producer thread streams the K' and V' tiles of the run from HBM into a shared-memory ring with
 // bulk asynchronous copies (mbarrier completion); eight consumer warps take the scores, an online
 // softmax and the weighted sum of value rows from shared memory.  A lane pair owns one row of a tile.
-// For every (CTA, unit) piece the CTA writes an un-normalised partial (max, sum, o'[rp_v]).
+// A piece that covers its whole unit is normalised and lifted through (U^V)^T on the spot.  Otherwise
+// the CTA writes an un-normalised partial (max, sum, o'[rp_v]) and bumps a per-unit counter; the CTA
+// that arrives last merges the unit's partials (exact re-association of the softmax), normalises and
+// lifts.  The new token's row can be handed to the kernel directly (k_new/v_new): the CTA that owns
+// the end of a unit projects it, stores it in the cache and attends to it from shared memory, so a
+// whole decode step (append + attend + combine + lift) is one launch.
 //
-// Kernel 2 (combine_lift_kernel): merges the partials of a unit (exact re-association of the
-// softmax), normalises, multiplies by (U^V)^T and stores the d_head-wide output.
+// Kernel 2 (combine_lift_kernel): the same merge + lift as a separate launch, used when the fused
+// merge is switched off.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -26,12 +31,16 @@ struct __align__(128) DecodeSmemFixed {
   unsigned long long empty[kMaxStages];
   long long range[2];
   int abort_flag;
-  int pad_[3];
-  float qraw[128];
-  float qpart[4][128];
-  float qp[128];
+  int is_last;
+  float piece_m, piece_l;
+  float qraw[128], kraw[128], vraw[128];   // the unit's q (and new k, v) as fp32
+  float proj_part[256];                    // partial sums of the projections
+  float qp[128];                           // q' * log2(e)/sqrt(d_head)
+  __align__(16) unsigned char new_k[512];  // the new token's k', v' in cache format (one row each)
+  __align__(16) unsigned char new_v[512];
   float wmax[kDecodeConsumerWarps];
   float wsum[kDecodeConsumerWarps];
+  float o_acc[128];                        // the piece's (later the unit's) o'
   float stage_o[kDecodeConsumerWarps][4][128];
 };
 
@@ -78,13 +87,6 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* statu
       return false;
     }
   }
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, void* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          smem_u32(dst)),
-      "l"(src), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
 }
 __device__ __forceinline__ void consumer_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerWarps * 32) : "memory");
@@ -173,7 +175,7 @@ __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
 template <typename T, int NCH>
 __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
                                             unsigned char* ring, const HeadInfo& hd, int i0, int i1,
-                                            RingPos& pos, int warp, int lane, int slot) {
+                                            RingPos& pos, int warp, int lane, bool with_new_row) {
   constexpr int EPC = Elem<T>::kPerChunk;
   const int pair = lane >> 1, half = lane & 1;
   const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
@@ -207,62 +209,71 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
 
   volatile int* abort_flag = &fx->abort_flag;
   float m = -INFINITY, l = 0.f;
+
+  // score of one cached row against q', online-softmax update, weighted accumulation of its value row
+  auto process_row = [&](const unsigned char* kr, const unsigned char* vr, bool valid) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NCH; ++j) {
+      float x[EPC];
+      Elem<T>::load_chunk(kr + off_k[j], x);
+#pragma unroll
+      for (int e = 0; e < EPC; e += 4) {
+        a0 = fmaf(x[e + 0], q[j][e + 0], a0); a1 = fmaf(x[e + 1], q[j][e + 1], a1);
+        a2 = fmaf(x[e + 2], q[j][e + 2], a2); a3 = fmaf(x[e + 3], q[j][e + 3], a3);
+      }
+    }
+    float s = (a0 + a1) + (a2 + a3);
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    if (valid) {
+      if (s > m) {                      // rare after the first rows: rescale the running state
+        const float c = fast_exp2(m - s);
+        l *= c;
+#pragma unroll
+        for (int j = 0; j < NCH; ++j)
+#pragma unroll
+          for (int e = 0; e < EPC; ++e) o[j][e] *= c;
+        m = s;
+      }
+      const float pr = fast_exp2(s - m);
+      l += pr;
+#pragma unroll
+      for (int j = 0; j < NCH; ++j) {
+        float x[EPC];
+        Elem<T>::load_chunk(vr + off_v[j], x);
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, x[e], o[j][e]);
+      }
+    }
+  };
+
   for (int i = i0; i < i1; ++i) {
     const int stage = pos.stage;
     const uint32_t parity = pos.parity;
     pos.advance(p.stages);
-    if (*abort_flag) continue;
-    if (!mbar_wait(&fx->full[stage], parity, p.status)) {
+    // warp-uniform decisions: the row code below shuffles across the whole warp
+    if (__any_sync(0xffffffffu, *abort_flag != 0)) continue;
+    if (__any_sync(0xffffffffu, !mbar_wait(&fx->full[stage], parity, p.status))) {
       *abort_flag = 1;
       continue;
     }
     const unsigned char* kt = ring + static_cast<size_t>(stage) * p.stage_bytes;
     const unsigned char* vt = kt + p.v_tile_off;
     const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
-    // The loop bound is the same for all lanes of a warp (the shuffle below needs every lane);
+    // The loop bound is the same for all lanes of a warp (the shuffle inside needs every lane);
     // lane pairs past the last row recompute the group's first row and drop the result.
     for (int rbase = warp * 16; rbase < rows; rbase += kDecodeConsumerWarps * 16) {
       const bool valid = rbase + pair < rows;
       const int row = valid ? rbase + pair : rbase;
-      const unsigned char* kr = kt + row * rowb_k;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-      for (int j = 0; j < NCH; ++j) {
-        float x[EPC];
-        Elem<T>::load_chunk(kr + off_k[j], x);
-#pragma unroll
-        for (int e = 0; e < EPC; e += 4) {
-          a0 = fmaf(x[e + 0], q[j][e + 0], a0); a1 = fmaf(x[e + 1], q[j][e + 1], a1);
-          a2 = fmaf(x[e + 2], q[j][e + 2], a2); a3 = fmaf(x[e + 3], q[j][e + 3], a3);
-        }
-      }
-      float s = (a0 + a1) + (a2 + a3);
-      s += __shfl_xor_sync(0xffffffffu, s, 1);
-      if (valid) {
-        if (s > m) {                    // rare after the first rows: rescale the running state
-          const float c = fast_exp2(m - s);
-          l *= c;
-#pragma unroll
-          for (int j = 0; j < NCH; ++j)
-#pragma unroll
-            for (int e = 0; e < EPC; ++e) o[j][e] *= c;
-          m = s;
-        }
-        const float pr = fast_exp2(s - m);
-        l += pr;
-        const unsigned char* vr = vt + row * rowb_v;
-#pragma unroll
-        for (int j = 0; j < NCH; ++j) {
-          float x[EPC];
-          Elem<T>::load_chunk(vr + off_v[j], x);
-#pragma unroll
-          for (int e = 0; e < EPC; ++e) o[j][e] = fmaf(pr, x[e], o[j][e]);
-        }
-      }
+      process_row(kt + row * rowb_k, vt + row * rowb_v, valid);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&fx->empty[stage]);
   }
+
+  // the new token's row (already projected, in shared memory) is attended by one lane pair
+  if (with_new_row && warp == 0 && !__any_sync(0xffffffffu, *abort_flag != 0))
+    process_row(fx->new_k, fx->new_v, pair == 0);
 
   // ---- merge the 128 lane pairs of the CTA into one partial
   float wm = m;
@@ -299,59 +310,165 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   }
   consumer_sync();
   const int t = warp * 32 + lane;
-  float* part = p.partials + static_cast<size_t>(slot) * p.part_stride;
   if (t < hd.rp_v) {
     float acc = 0.f;
 #pragma unroll
     for (int w = 0; w < kDecodeConsumerWarps; ++w)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc += fx->stage_o[w][c][t];
-    part[4 + t] = acc;
+    fx->o_acc[t] = acc;
   }
   if (t == 0) {
     float L = 0.f;
 #pragma unroll
     for (int w = 0; w < kDecodeConsumerWarps; ++w) L += fx->wsum[w];
-    part[0] = M;
-    part[1] = L;
+    fx->piece_m = M;
+    fx->piece_l = L;
   }
-  consumer_sync();   // the staging area and q' are reused by the next piece
+  consumer_sync();
 }
 
-// q' = q U^K * log2(e)/sqrt(d_head) for one unit, left in fx->qp (all consumer threads take part).
+// Projections at the head of a piece (all consumer threads): q' = q U^K * log2(e)/sqrt(d_head) into
+// fx->qp, and, when the piece ends its unit and a new token is supplied, k' = k U^K and v' = v U^V,
+// rounded to the cache dtype, into fx->new_k / fx->new_v and into row p.n of the cache.
 template <typename T>
-__device__ __forceinline__ void project_query(const DecodeParams& p, DecodeSmemFixed* fx,
-                                              const HeadInfo& hd, int h, int b, int t) {
+__device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmemFixed* fx,
+                                               const HeadInfo& hd, int h, int b, int t, bool with_new_row) {
+  constexpr int kThreads = kDecodeConsumerWarps * 32;
   const T* q = static_cast<const T*>(p.q);
-  const int rp = hd.rp_k;
-  if (p.flags & 0x1u) {   // rank-space query supplied by the caller (merged W^Q')
-    if (t < rp) fx->qp[t] = Elem<T>::to_float(q[b * p.q_stride_b + hd.lr_k_off + t]) * p.q_scale;
-    consumer_sync();
-    return;
-  }
   const int d_head = p.d_head;
-  if (t < d_head) fx->qraw[t] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + t]);
-  consumer_sync();
-  const int nthreads = kDecodeConsumerWarps * 32;
-  int ngrp = nthreads / rp;
-  if (ngrp > 4) ngrp = 4;
-  const int g = t / rp, c = t - g * rp;
-  if (g < ngrp) {
-    const int per = (d_head + ngrp - 1) / ngrp;
-    const int d0 = g * per, d1 = min(d_head, d0 + per);
-    const float* U = p.basis + hd.uk_off;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int d = d0; d < d1; ++d) acc = fmaf(fx->qraw[d], __ldg(U + d * rp + c), acc);
-    fx->qpart[g][c] = acc;
+  const bool q_lowrank = (p.flags & 0x1u) != 0;   // rank-space query supplied by the caller (merged W^Q')
+  if (q_lowrank) {
+    if (t < hd.rp_k) fx->qp[t] = Elem<T>::to_float(q[b * p.q_stride_b + hd.lr_k_off + t]) * p.q_scale;
+  } else if (t < d_head) {
+    fx->qraw[t] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + t]);
+  }
+  if (with_new_row && t < d_head) {
+    const int64_t src = b * p.kv_stride_b + static_cast<int64_t>(h) * d_head + t;
+    fx->kraw[t] = Elem<T>::to_float(static_cast<const T*>(p.k_new)[src]);
+    fx->vraw[t] = Elem<T>::to_float(static_cast<const T*>(p.v_new)[src]);
   }
   consumer_sync();
-  if (t < rp) {
+  // outputs: [0, nq) = q' columns, [nq, nq + rp_k) = k' columns, then rp_v v' columns
+  const int nq = q_lowrank ? 0 : hd.rp_k;
+  const int total = nq + (with_new_row ? hd.rp_k + hd.rp_v : 0);
+  if (total == 0) return;
+  int groups = kThreads / total;                  // split the d_head sum when few outputs are needed
+  if (groups > 4) groups = 4;
+  // k' and v' are summed over d_head in one fixed order (the append kernel's), so that a row stored by
+  // this kernel is bit-identical to the same row stored by eigen_attn_append_kv
+  if (groups < 1 || with_new_row) groups = 1;
+  const int per = (d_head + groups - 1) / groups;
+  T* knew = reinterpret_cast<T*>(fx->new_k);
+  T* vnew = reinterpret_cast<T*>(fx->new_v);
+  const int64_t crow = static_cast<int64_t>(b) * p.n_max + p.n;
+  auto finish = [&](int o, float acc) {
+    if (o < nq) {
+      fx->qp[o] = acc * p.q_scale;
+    } else if (o < nq + hd.rp_k) {
+      const int c = o - nq;
+      const T val = Elem<T>::from_float(acc);
+      knew[c] = val;
+      reinterpret_cast<T*>(p.cache + hd.k_off)[crow * hd.rp_k + c] = val;
+    } else {
+      const int c = o - nq - hd.rp_k;
+      const T val = Elem<T>::from_float(acc);
+      vnew[c] = val;
+      reinterpret_cast<T*>(p.cache + hd.v_off)[crow * hd.rp_v + c] = val;
+    }
+  };
+  auto dot = [&](int o, int d0, int d1) {
+    const float* x;
+    const float* U;
+    int rp;
+    if (o < nq) { x = fx->qraw; U = p.basis + hd.uk_off + o; rp = hd.rp_k; }
+    else if (o < nq + hd.rp_k) { x = fx->kraw; U = p.basis + hd.uk_off + (o - nq); rp = hd.rp_k; }
+    else { x = fx->vraw; U = p.basis + hd.uv_off + (o - nq - hd.rp_k); rp = hd.rp_v; }
     float acc = 0.f;
-    for (int gg = 0; gg < ngrp; ++gg) acc += fx->qpart[gg][t];
-    fx->qp[t] = acc * p.q_scale;
+#pragma unroll 16
+    for (int d = d0; d < d1; ++d) acc = fmaf(x[d], __ldg(U + d * rp), acc);
+    return acc;
+  };
+  if (groups == 1) {
+    for (int o = t; o < total; o += kThreads) finish(o, dot(o, 0, d_head));
+  } else {
+    const int g = t / total, o = t - g * total;
+    if (g < groups) fx->proj_part[g * total + o] = dot(o, g * per, min(d_head, (g + 1) * per));
+    consumer_sync();
+    if (t < total) {
+      float acc = 0.f;
+      for (int gg = 0; gg < groups; ++gg) acc += fx->proj_part[gg * total + t];
+      finish(t, acc);
+    }
   }
   consumer_sync();
+}
+
+// CTA that owns the tile with start weight x: floor(x * grid / w_total).
+__device__ __forceinline__ int owner_cta(long long x, int grid, long long w_total) {
+  return static_cast<int>((x * grid) / w_total);
+}
+
+// After run_segment: turn the piece in shared memory (o_acc, piece_m, piece_l) into the unit's output,
+// directly if the piece is the whole unit, else through the partial slots and the arrival counter.
+template <typename T>
+__device__ __forceinline__ void finish_piece(const DecodeParams& p, DecodeSmemFixed* fx, const HeadInfo& hd,
+                                             int unit, int h, int b, int cta, int grid, bool whole, int t) {
+  bool finalize = whole && p.counters != nullptr;
+  float inv_l = 1.f / fx->piece_l;
+  if (!finalize) {
+    float* part = p.partials + static_cast<size_t>(unit + cta) * p.part_stride;
+    if (t < hd.rp_v) part[4 + t] = fx->o_acc[t];
+    if (t == 0) { part[0] = fx->piece_m; part[1] = fx->piece_l; }
+    if (p.counters == nullptr) {      // a separate combine launch follows
+      consumer_sync();
+      return;
+    }
+    const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
+    const long long w = hd.rp_k + hd.rp_v;
+    const long long x0 = per_head_tiles * hd.w_prefix + static_cast<long long>(b) * p.nt * w;
+    const int c0 = owner_cta(x0, grid, p.w_total);
+    const int c1 = owner_cta(x0 + static_cast<long long>(p.nt - 1) * w, grid, p.w_total);
+    __threadfence();                  // this thread's partial is visible before the arrival is counted
+    consumer_sync();
+    if (t == 0) {
+      const int arrived = atomicAdd(&p.counters[unit], 1);
+      const int last = arrived == c1 - c0;
+      if (last) p.counters[unit] = 0; // ready for the next call
+      fx->is_last = last;
+    }
+    consumer_sync();
+    if (fx->is_last) {
+      __threadfence();
+      float M = -INFINITY;
+      for (int c = c0; c <= c1; ++c)
+        M = fmaxf(M, __ldcg(p.partials + static_cast<size_t>(unit + c) * p.part_stride));
+      float L = 0.f, acc = 0.f;
+      for (int c = c0; c <= c1; ++c) {
+        const float* pc = p.partials + static_cast<size_t>(unit + c) * p.part_stride;
+        const float f = fast_exp2(__ldcg(pc) - M);
+        L = fmaf(__ldcg(pc + 1), f, L);
+        if (t < hd.rp_v) acc = fmaf(__ldcg(pc + 4 + t), f, acc);
+      }
+      if (t < hd.rp_v) fx->o_acc[t] = acc;
+      inv_l = 1.f / L;
+      finalize = true;
+    }
+    consumer_sync();
+  }
+  if (finalize) {
+    T* out = static_cast<T*>(p.out);
+    if (p.flags & 0x2u) {             // rank-space output for a merged W^O'
+      if (t < hd.rp_v) out[b * p.out_stride_b + hd.lr_v_off + t] = Elem<T>::from_float(fx->o_acc[t] * inv_l);
+    } else if (t < p.d_head) {
+      const float* Ut = p.basis + hd.uvt_off + t;   // (U^V)^T: rp_v x d_head
+      float y = 0.f;
+#pragma unroll 16
+      for (int c = 0; c < hd.rp_v; ++c) y = fmaf(fx->o_acc[c], __ldg(Ut + c * p.d_head), y);
+      out[b * p.out_stride_b + static_cast<int64_t>(h) * p.d_head + t] = Elem<T>::from_float(y * inv_l);
+    }
+  }
+  consumer_sync();                    // o_acc, q' and the staging area are reused by the next piece
 }
 
 template <typename T>
@@ -441,21 +558,23 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + left));
       const int h = unit / p.B, b = unit - h * p.B;
       const HeadInfo hd = p.heads[h];
-      project_query<T>(p, fx, hd, h, b, tid);
-      const int slot = unit + cta;
+      const bool whole = i0 == 0 && i1 == p.nt;
+      const bool with_new_row = p.k_new != nullptr && i1 == p.nt;
+      project_inputs<T>(p, fx, hd, h, b, tid, with_new_row);
       const int mx = max(hd.rp_k, hd.rp_v);
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, slot); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
       }
+      finish_piece<T>(p, fx, hd, unit, h, b, cta, grid, whole, tid);
       F += i1 - i0;
     }
   }
@@ -463,11 +582,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
 }
 
 // ---------------------------------------------------------------- combine + lift
-
-// CTA that owns the tile with start weight x: floor(x * grid / w_total).
-__device__ __forceinline__ int owner_cta(long long x, int grid, long long w_total) {
-  return static_cast<int>((x * grid) / w_total);
-}
 
 template <typename T>
 __global__ void __launch_bounds__(128) combine_lift_kernel(const CombineParams p) {

@@ -29,14 +29,20 @@ constexpr int kStatusTimeout = -6;
 struct DecodeParams {
   const HeadInfo* heads;
   const float* basis;       // basis area of the workspace
-  const char* cache;
+  char* cache;
   const void* q;            // [B][1][H][d_head] or packed rank-space [B][sum rp_k]
   int64_t q_stride_b;       // elements
+  const void* k_new;        // [B][1][H][d_head] new token to project, store at row n and attend; or NULL
+  const void* v_new;
+  int64_t kv_stride_b;
+  void* out;                // [B][1][H][d_head] or packed [B][sum rp_v]
+  int64_t out_stride_b;
   float* partials;          // [(B*H + grid)][part_stride]: m, l, pad, pad, o'[rp_v]
+  int* counters;            // [B*H] arrivals per unit (all zero between calls); NULL = separate combine launch
   int* status;
   int32_t part_stride;      // floats per partial slot (multiple of 4)
   int32_t B, H, d_head;
-  int32_t n;                // rows to attend
+  int32_t n;                // cached rows to stream (the new token's row, if any, comes on top)
   int32_t n_max;
   int32_t tile_rows;        // rows per tile
   int32_t nt;               // tiles per unit = ceil(n / tile_rows)
