@@ -482,7 +482,16 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags; p.status = dev_status(h);
-  e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);
+  // tensor-core kernel for bf16 layers whose output rows can be stored 16 bytes at a time
+  const bool aligned = (flags & EA_OUT_LOWRANK) ||
+                       (reinterpret_cast<uintptr_t>(d_out) % 16 == 0 && out_stride_b % 8 == 0 && out_stride_t % 8 == 0);
+  const bool tc_ok = ea::prefill_tc_supported(p, h->desc.dtype) && aligned;
+  if (h->opt_prefill == 2 && !tc_ok)
+    return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
+  if (tc_ok && h->opt_prefill != 1)
+    e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+  else
+    e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);
   if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch");
   return EA_OK;
 }

@@ -114,6 +114,9 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+bool prefill_tc_supported(const PrefillParams& p, int dtype);       // bf16, d_head a multiple of 16
+cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s,
+                              uint64_t* launches);
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
 // library's own partials array on the current device.  Resolves the address on first use per device.

@@ -267,6 +267,47 @@ def test_prefill_matches_oracle_and_feeds_decode(B, dtype, H, d, rk, rv, T):
     assert_close(o1, ref.decode_dense(to_np(q[:, T:])), dtype, "decode after prefill")
 
 
+@pytest.mark.parametrize("H,d,rk,rv,T", [
+    (1, 128, [80], [80], 128),                       # exactly one query tile and one key tile
+    (2, 128, [80, 64], [80, 96], 300),               # several tiles, ragged tail, K and V ranks differ
+    (3, 64, [24, 64, 40], [56, 8, 64], 517),         # small d_head, ranks that are not multiples of 16
+    (2, 128, [128, 16], [16, 128], 1000),            # widest and narrowest ranks
+])
+def test_tensor_core_prefill_matches_oracle_and_cuda_core_kernel(B, H, d, rk, rv, T):
+    B_ = 2
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, BF16, seed_cfg=101, T_q=T)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
+    outs = {}
+    for impl in (2, 1):                              # 2 = tcgen05 kernel, 1 = CUDA-core kernel
+        lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
+        lay.set_option(B.EA_OPT_PREFILL_IMPL, impl)
+        outs[impl] = lay.prefill(q, k, v)
+        lay.poll_status()
+        assert_close(outs[impl], expect, BF16, f"prefill impl {impl}")
+    assert float((outs[1].float() - outs[2].float()).abs().max()) < 3e-2
+
+
+def test_tensor_core_prefill_chunked_and_lowrank(B):
+    B_, H, d, T = 1, 2, 128, 700
+    rk, rv = [80, 48], [64, 80]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, BF16, seed_cfg=102, T_q=T)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
+    lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=400)
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, 2)
+    cuts = [0, 130, 530, 700]                        # len0 > 0 and not a multiple of the tile
+    parts = [lay.prefill(q[:, a:b_].contiguous(), k[:, a:b_].contiguous(), v[:, a:b_].contiguous())
+             for a, b_ in zip(cuts[:-1], cuts[1:])]
+    lay.poll_status()
+    assert_close(torch.cat(parts, dim=1), expect, BF16, "chunked tensor-core prefill")
+    lay.set_len(0)
+    low = lay.prefill(q[:, :400].contiguous(), k[:, :400].contiguous(), v[:, :400].contiguous(), out_lowrank=True)
+    for h in range(H):
+        got = to_np(low[0, :, lay.offs_v[h]:lay.offs_v[h] + rv[h]]) @ U_v[h].astype(np.float64).T
+        assert np.abs(got - expect[0, :400, h, :]).max() < 2e-2
+
+
 def test_chunked_prefill_and_lowrank_output(B):
     B_, H, d, T = 1, 2, 64, 90
     rk, rv = [32, 24], [16, 32]
