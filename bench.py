@@ -376,6 +376,79 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_prefill(args, wl):
+    """Causal rank-r prefill of the whole prompt (project K/V and write the cache, project Q, attention on the
+    tensor cores, lift): one JSON line with time, TFLOP/s of the causal contractions and the tensor roofline."""
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    dt = synth.torch_dtype(wl.dtype)
+    T = wl.context
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device)
+    if args.prefill_impl:
+        lay.set_option(binding.EA_OPT_PREFILL_IMPL, args.prefill_impl)
+    W = {t: synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_" + t, device=device) for t in "KVQ"}
+    k = synth.lowrank_rows(W["K"], wl.batch, T, wl.sigma, wl.index, "K", dtype=dt, device=device)
+    v = synth.lowrank_rows(W["V"], wl.batch, T, wl.sigma, wl.index, "V", dtype=dt, device=device)
+    q = synth.lowrank_rows(W["Q"], wl.batch, T, wl.sigma, wl.index, "Q", dtype=dt, device=device)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream(device)
+    steps, warmup = min(args.steps, 20), min(args.warmup, 5)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        a.record(stream); b.record(stream)
+    for _ in range(warmup):
+        lay.set_len(0); lay.prefill(q, k, v, out=out)
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(device.index or 0)
+    sampler.start(); time.sleep(0.2)
+    l0 = lay.launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        lay.set_decode_events(ev[i][0], ev[i][1])
+        lay.set_len(0); lay.prefill(q, k, v, out=out)
+    t1.record(stream)
+    torch.cuda.synchronize(device)
+    lay.set_decode_events(None, None)
+    clocks = sampler.stop()
+    lay.poll_status()
+    ms = t0.elapsed_time(t1) / steps
+    kern = sum(a.elapsed_time(b) for a, b in ev) / steps
+    pairs = wl.batch * T * (T + 1) // 2                       # causal (query, key) pairs per head, summed over the batch
+    flop = 2 * pairs * sum(2 * r for r in ranks)             # Q'K'^T and PV' over the lower triangle
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak, src = 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+    if os.path.exists(peaks_path):
+        peak, src = float(json.load(open(peaks_path))["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    # parity of sampled rows of two units against the oracle (one by one)
+    from oracle import eigen_attention as orc
+    errs = []
+    for (b, h) in [(0, 0), (wl.batch - 1, wl.n_heads - 1)]:
+        rows = [0, 1, 127, 128, 1000, T - 1]
+        kk, vv = k[b, :, h].double().cpu().numpy(), v[b, :, h].double().cpu().numpy()
+        for t in rows:
+            ref = orc.decode_head(q[b, t, h].double().cpu().numpy(), kk[:t + 1], vv[:t + 1], U_k[h], U_v[h])
+            errs.append(float(np.abs(out[b, t, h].double().cpu().numpy() - ref).max()))
+    achieved = flop / (kern * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "causal rank-r prefill attention TFLOP/s (B=4, T=4096, 7B layer)", "value": flop / (ms * 1e-3) / 1e12,
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 operands, f32 accumulate", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head, "rank": sorted(set(ranks)),
+                   "prompt": T, "flop_counted": "2*pairs*(r_k+r_v) over the causal triangle; projections and lift excluded"},
+        "roofline": {"bound": "tensor", "kernel": "prefill attention kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "peak_source": src, "kernel_ms": kern, "traffic": None},
+        "gpu_launches": lay.launch_count() - l0, "clocks": clocks,
+        "parity_sampled_rows": {"rows": len(errs), "max_abs": max(errs), "tolerance": "max_abs <= 2e-2"},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -386,6 +459,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
+    ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -400,7 +474,10 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
-    run_ours(args, wl)
+    if wl.name.startswith("prefill"):
+        run_prefill(args, wl)
+    else:
+        run_ours(args, wl)
 
 
 if __name__ == "__main__":

@@ -177,8 +177,9 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value);
 /* Number of kernels this handle has launched since create. */
 ea_status eigen_attn_launch_count(eigen_attn_t h, uint64_t* count);
 
-/* If both are non-NULL cudaEvent_t handles, every later decode records `start` immediately before
- * and `stop` immediately after the split-KV attention kernel on the call's stream (NULL, NULL = off). */
+/* If both are non-NULL cudaEvent_t handles, every later decode, decode_step or prefill call records
+ * `start` immediately before and `stop` immediately after its attention kernel (the split-KV kernel, or
+ * the causal prefill kernel) on the call's stream (NULL, NULL = off). */
 ea_status eigen_attn_set_decode_events(eigen_attn_t h, void* start_event, void* stop_event);
 
 /* Library version: major*10000 + minor*100 + patch. */

@@ -488,10 +488,12 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   const bool tc_ok = ea::prefill_tc_supported(p, h->desc.dtype) && aligned;
   if (h->opt_prefill == 2 && !tc_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
+  if (h->ev_start) cudaEventRecord(h->ev_start, s);
   if (tc_ok && h->opt_prefill != 1)
     e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
   else
     e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);
+  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch");
   return EA_OK;
 }
