@@ -23,6 +23,17 @@ constexpr int kSmemLimit = 227 * 1024;
 constexpr int kInFlightBytes = 120 * 1024;   // target bytes of bulk copies in flight per SM (decode)
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+uint16_t bf16_rne(float x) {          // round to nearest even; inputs are finite
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  return static_cast<uint16_t>((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+float bf16_to_float(uint16_t b) {
+  const uint32_t u = static_cast<uint32_t>(b) << 16;
+  float x;
+  memcpy(&x, &u, 4);
+  return x;
+}
 int ceil8(int r) { return (r + 7) / 8 * 8; }
 
 struct Layout {
@@ -72,6 +83,11 @@ void make_layout(const ea_desc* d, Layout* L) {
     hi.uk_off = static_cast<int32_t>(basis);  basis += static_cast<size_t>(dh) * hi.rp_k;
     hi.uv_off = static_cast<int32_t>(basis);  basis += static_cast<size_t>(dh) * hi.rp_v;
     hi.uvt_off = static_cast<int32_t>(basis); basis += static_cast<size_t>(dh) * hi.rp_v;
+    if (dh % 16 == 0) {   // bf16 high/low images of U^T for the tensor-core projections (2 bytes per element)
+      basis = (basis + 3) & ~static_cast<size_t>(3);
+      hi.ukt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_k + 15) & ~15) * dh;
+      hi.uvt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_v + 15) & ~15) * dh;
+    }
     hi.lr_k_off = lk; lk += hi.rp_k;
     hi.lr_v_off = lv; lv += hi.rp_v;
     hi.w_prefix = wsum; wsum += hi.rp_k + hi.rp_v;
@@ -333,6 +349,25 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
         basis[hi.uvt_off + static_cast<size_t>(c) * dh + d] = x;
       }
     }
+    if (dh % 16 == 0) {
+      for (int pass = 0; pass < 2; ++pass) {
+        const float* U = pass ? uv : uk;
+        const int r = pass ? hi.r_v : hi.r_k;
+        const int rp16 = ((pass ? hi.rp_v : hi.rp_k) + 15) & ~15;
+        uint16_t* img_hi = reinterpret_cast<uint16_t*>(basis.data() + (pass ? hi.uvt16_off : hi.ukt16_off));
+        uint16_t* img_lo = img_hi + static_cast<size_t>(rp16) * dh;
+        const int grp = (dh / 8) * 128;                       // bytes per group of 8 rank columns
+        for (int c = 0; c < rp16; ++c)
+          for (int d = 0; d < dh; ++d) {
+            const float x = c < r ? U[static_cast<size_t>(d) * r + c] : 0.f;
+            const uint16_t xh = bf16_rne(x);
+            const uint16_t xl = bf16_rne(x - bf16_to_float(xh));
+            const size_t off = (static_cast<size_t>(c >> 3) * grp + (d >> 3) * 128 + (c & 7) * 16 + (d & 7) * 2) / 2;
+            img_hi[off] = xh;
+            img_lo[off] = xl;
+          }
+      }
+    }
     if (desc->flags & EA_CHECK_ORTHONORMAL) {
       for (int pass = 0; pass < 2; ++pass) {
         const float* U = pass ? uv : uk;
@@ -461,35 +496,56 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     return fail(h, EA_ERR_CAPACITY, "prefill: T %d exceeds max_prefill_tokens %d", T, h->desc.max_prefill_tokens);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const int len0 = h->len;
-  const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, 0, s);
-  if (st != EA_OK) return st;
   const Layout& L = h->L;
-  ea::QProjectParams qp{};
-  qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
-  qp.stride_b = stride_b; qp.stride_t = stride_t;
-  qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
-  cudaError_t e = ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
-  if (e != cudaSuccess) return cuda_fail(h, e, "prefill q projection launch");
+  const bool tc_shape = h->desc.dtype == EA_BF16 && h->desc.d_head % 16 == 0;
+  // tensor-core kernels need 16-byte aligned rows on both sides
+  const bool in_aligned = reinterpret_cast<uintptr_t>(d_q) % 16 == 0 && reinterpret_cast<uintptr_t>(d_k) % 16 == 0 &&
+                          reinterpret_cast<uintptr_t>(d_v) % 16 == 0 && stride_b % 8 == 0 && stride_t % 8 == 0;
+  const bool out_aligned = (flags & EA_OUT_LOWRANK) || (reinterpret_cast<uintptr_t>(d_out) % 16 == 0 &&
+                                                        out_stride_b % 8 == 0 && out_stride_t % 8 == 0);
+  const bool tc_attn = tc_shape && out_aligned;
+  if (h->opt_prefill == 2 && !tc_attn)
+    return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
+  cudaError_t e;
+  if (tc_shape && in_aligned && h->opt_prefill != 1) {
+    // Q', K', V' in one tensor-core launch.  Its rows equal eigen_attn_append_kv's except where the two
+    // fp32 summation orders round to different bf16 values (one unit in the last place).
+    if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
+    if (static_cast<int64_t>(len0) + T > h->desc.n_max)
+      return fail(h, EA_ERR_CAPACITY, "prefill: len %d + T %d exceeds n_max %d", len0, T, h->desc.n_max);
+    ea::ProjectTcParams pp{};
+    pp.heads = dev_heads(h); pp.basis = dev_basis(h); pp.q = d_q; pp.k = d_k; pp.v = d_v;
+    pp.cache = h->cache; pp.qp = h->ws + L.off_qp; pp.stride_b = stride_b; pp.stride_t = stride_t;
+    pp.B = h->desc.batch; pp.T = T; pp.H = h->desc.n_heads; pp.d_head = h->desc.d_head;
+    pp.n_max = h->desc.n_max; pp.row0 = len0; pp.status = dev_status(h);
+    e = ea::launch_project_tc(pp, L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill projection launch");
+    h->len += T;
+  } else {
+    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, 0, s);
+    if (st != EA_OK) return st;
+    ea::QProjectParams qp{};
+    qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
+    qp.stride_b = stride_b; qp.stride_t = stride_t;
+    qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
+    e = ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill q projection launch");
+  }
   ea::PrefillParams p{};
-  p.heads = qp.heads; p.basis = qp.basis; p.cache = h->cache; p.qp = qp.qp; p.out = d_out;
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache; p.qp = h->ws + L.off_qp; p.out = d_out;
   if (flags & EA_OUT_LOWRANK) {
     p.out_stride_t = L.sum_rp_v;
     p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
   } else {
     p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
   }
-  p.B = qp.B; p.T = T; p.H = qp.H; p.d_head = qp.d_head; p.n_max = h->desc.n_max; p.len0 = len0;
+  p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
+  p.len0 = len0;
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags; p.status = dev_status(h);
-  // tensor-core kernel for bf16 layers whose output rows can be stored 16 bytes at a time
-  const bool aligned = (flags & EA_OUT_LOWRANK) ||
-                       (reinterpret_cast<uintptr_t>(d_out) % 16 == 0 && out_stride_b % 8 == 0 && out_stride_t % 8 == 0);
-  const bool tc_ok = ea::prefill_tc_supported(p, h->desc.dtype) && aligned;
-  if (h->opt_prefill == 2 && !tc_ok)
-    return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  if (tc_ok && h->opt_prefill != 1)
+  if (tc_attn && h->opt_prefill != 1)
     e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
   else
     e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);

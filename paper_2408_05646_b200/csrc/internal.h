@@ -18,7 +18,9 @@ struct HeadInfo {
   int32_t uvt_off;    // float offset of (U^V)^T (rp_v x d_head)
   int32_t lr_k_off;   // element offset of the head in packed rank-space K/Q vectors (prefix of rp_k)
   int32_t lr_v_off;   // same for V / O
-  int32_t pad_;
+  int32_t ukt16_off;  // float offset of the tensor-core image of (U^K)^T: bf16 high part then low part, each
+  int32_t uvt16_off;  //   [rp16][d_head] in the canonical core-matrix order (rp16 = rank padded to 16); same for U^V
+  int32_t pad_[3];
 };
 
 constexpr int kDecodeConsumerWarps = 8;
@@ -91,6 +93,21 @@ struct QProjectParams {      // prefill: Q' = Q U^K into a scratch buffer (IO dt
   int32_t B, T, H, d_head;
 };
 
+struct ProjectTcParams {     // prefill: Q', K', V' projections on the tensor cores (bf16 layers)
+  const HeadInfo* heads;
+  const float* basis;
+  const void* q;            // [B][T][H][d_head], shared strides
+  const void* k;
+  const void* v;
+  char* cache;
+  char* qp;                 // Q' scratch (layout as in QProjectParams)
+  int64_t stride_b, stride_t;
+  int32_t B, T, H, d_head;
+  int32_t n_max;
+  int32_t row0;
+  int* status;
+};
+
 struct PrefillParams {
   const HeadInfo* heads;
   const float* basis;
@@ -114,7 +131,7 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
-bool prefill_tc_supported(const PrefillParams& p, int dtype);       // bf16, d_head a multiple of 16
+cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s,
                               uint64_t* launches);
 

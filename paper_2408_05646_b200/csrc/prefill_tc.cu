@@ -13,157 +13,12 @@
 #include <cuda_bf16.h>
 
 #include "internal.h"
+#include "tc_common.cuh"
 
 namespace ea {
 namespace {
 
-constexpr int kTile = 128;                 // query rows per CTA = key rows per tile = MMA M
-constexpr int kThreads = 128;
-constexpr uint64_t kWaitBoundNs = 2000000000ull;
-
-// ---------------------------------------------------------------- PTX wrappers
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > kWaitBoundNs) {
-      atomicExch(status, kStatusTimeout);
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(void* dst_smem, uint32_t ncols) {   // one full warp
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
-               "r"(ncols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  // one full warp
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem], M = 128, K = 16, bf16 x bf16 -> f32; issued by one thread.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       bool accumulate) {
-  const uint32_t acc = accumulate ? 1u : 0u;
-  const uint32_t zero = 0u;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(zero), "r"(zero), "r"(zero), "r"(zero)
-      : "memory");
-}
-// The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void mma_commit(void* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-
-#define EA_R16(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
-  "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]),               \
-  "=r"(r[o + 12]), "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
-#define EA_W16(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]),       \
-  "r"(r[o + 6]), "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]),      \
-  "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15])
-
-// 16 consecutive fp32 columns of this thread's TMEM lane (warp w reads lanes 32w..32w+31).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : EA_R16(r, 0)
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
-      ::EA_W16(r, 0),
-      "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-
-// ---------------------------------------------------------------- descriptors
-
-// Shared-memory matrix descriptor, no swizzle: start address, leading-dimension byte offset (LBO),
-// stride-dimension byte offset (SBO), all in units of 16 bytes; bits 46-47 hold the descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return static_cast<uint64_t>((saddr >> 4) & 0x3FFFu) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-         (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
-}
-// Instruction descriptor, kind::f16: f32 accumulator, bf16 A and B, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
-         (static_cast<uint32_t>(kTile >> 4) << 24);
-}
-
-// Canonical tile: chunk (row, c) of 16 bytes lives at (row/8) * group_stride + c * 128 + (row%8) * 16,
-// i.e. the core matrices of an 8-row group are contiguous.
-__device__ __forceinline__ uint32_t chunk_off(int row, int c, int group_stride) {
-  return static_cast<uint32_t>((row >> 3) * group_stride + (c << 7) + ((row & 7) << 4));
-}
-
-// Copies `rows_valid` rows of a row-major bf16 matrix (row pitch `rp` elements) into a canonical tile of
-// 128 rows x `nch` chunks; rows and chunks past the source are zero.
-__device__ __forceinline__ void load_tile(unsigned char* dst, const __nv_bfloat16* src, int rp, int rows_valid,
-                                          int nch, int tid) {
-  const int src_chunks = rp >> 3;
-  const int group_stride = nch << 7;
-  for (int idx = tid; idx < kTile * nch; idx += kThreads) {
-    const int c = idx >> 7, row = idx & (kTile - 1);
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row < rows_valid && c < src_chunks)
-      v = __ldg(reinterpret_cast<const uint4*>(src + static_cast<int64_t>(row) * rp) + c);
-    *reinterpret_cast<uint4*>(dst + chunk_off(row, c, group_stride)) = v;
-  }
-}
-
-struct __align__(16) TcSmemHeader {
-  unsigned long long bar;
-  uint32_t tmem_base;
-  int abort_flag;
-};
+using namespace tc;
 
 // ---------------------------------------------------------------- the kernel
 
@@ -418,10 +273,6 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
 }
 
 }  // namespace
-
-bool prefill_tc_supported(const PrefillParams& p, int dtype) {
-  return dtype == 0 && p.d_head % 16 == 0 && p.d_head >= 16 && p.d_head <= 128;
-}
 
 size_t prefill_tc_smem_bytes(int max_rp_k, int max_rp_v) {
   const size_t k16 = (max_rp_k + 15) & ~15, v16 = (max_rp_v + 15) & ~15;
