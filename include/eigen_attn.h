@@ -168,7 +168,9 @@ typedef enum {
   EA_OPT_DECODE_CTAS = 1,     /* CTAs of the split-KV decode kernel; 0 = one per SM                      */
   EA_OPT_DECODE_TILE_ROWS = 2,/* rows per shared-memory tile (multiple of 16, <= 128); 0 = automatic     */
   EA_OPT_DECODE_STAGES = 3,   /* depth of the shared-memory ring (2..12); 0 = as many as fit              */
-  EA_OPT_PREFILL_IMPL = 4,    /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernel      */
+  EA_OPT_PREFILL_IMPL = 4,    /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernels, 3 = the
+                                 single-tile tcgen05 kernel (otherwise only used for ranks too wide for the
+                                 warp-specialised one)                                                     */
   EA_OPT_DECODE_FUSED = 5     /* 1 (default): a decode step is one launch (append row, attend, merge the
                                  splits, lift); 0: separate append / attention / merge launches           */
 } ea_option;

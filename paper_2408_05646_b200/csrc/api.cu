@@ -87,6 +87,7 @@ void make_layout(const ea_desc* d, Layout* L) {
       basis = (basis + 3) & ~static_cast<size_t>(3);
       hi.ukt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_k + 15) & ~15) * dh;
       hi.uvt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_v + 15) & ~15) * dh;
+      hi.uvl16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_v + 15) & ~15) * dh;
     }
     hi.lr_k_off = lk; lk += hi.rp_k;
     hi.lr_v_off = lv; lv += hi.rp_v;
@@ -368,6 +369,21 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
           }
       }
     }
+    if (dh % 16 == 0) {   // lift image of U^V: rows = d (the N index of the lift product), contraction over the rank
+      const int rv16 = (hi.rp_v + 15) & ~15;
+      uint16_t* img_hi = reinterpret_cast<uint16_t*>(basis.data() + hi.uvl16_off);
+      uint16_t* img_lo = img_hi + static_cast<size_t>(rv16) * dh;
+      const int grp = (rv16 / 8) * 128;                       // bytes per group of 8 rows (d values)
+      for (int d = 0; d < dh; ++d)
+        for (int c = 0; c < rv16; ++c) {
+          const float x = c < hi.r_v ? uv[static_cast<size_t>(d) * hi.r_v + c] : 0.f;
+          const uint16_t xh = bf16_rne(x);
+          const uint16_t xl = bf16_rne(x - bf16_to_float(xh));
+          const size_t off = (static_cast<size_t>(d >> 3) * grp + (c >> 3) * 128 + (d & 7) * 16 + (c & 7) * 2) / 2;
+          img_hi[off] = xh;
+          img_lo[off] = xl;
+        }
+    }
     if (desc->flags & EA_CHECK_ORTHONORMAL) {
       for (int pass = 0; pass < 2; ++pass) {
         const float* U = pass ? uv : uk;
@@ -545,8 +561,12 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags; p.status = dev_status(h);
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  if (tc_attn && h->opt_prefill != 1)
-    e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+  size_t ws_smem = 0;
+  const int ws_stages = tc_attn ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
+  if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 2)
+    e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, s, &h->launches);   // warp-specialised, 256 query rows per CTA
+  else if (tc_attn && h->opt_prefill != 1)
+    e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);  // single query tile per CTA (wide ranks)
   else
     e = ea::launch_prefill_simt(p, h->desc.dtype, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
@@ -630,7 +650,7 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
       h->opt_stages = value;
       return EA_OK;
     case EA_OPT_PREFILL_IMPL:
-      if (value < 0 || value > 2)
+      if (value < 0 || value > 3)
         return fail(h, EA_ERR_INVALID_ARG, "PREFILL_IMPL %lld", static_cast<long long>(value));
       h->opt_prefill = value;
       return EA_OK;

@@ -20,7 +20,8 @@ struct HeadInfo {
   int32_t lr_v_off;   // same for V / O
   int32_t ukt16_off;  // float offset of the tensor-core image of (U^K)^T: bf16 high part then low part, each
   int32_t uvt16_off;  //   [rp16][d_head] in the canonical core-matrix order (rp16 = rank padded to 16); same for U^V
-  int32_t pad_[3];
+  int32_t uvl16_off;  // float offset of the lift image of U^V: bf16 high then low part, each [d_head][rv16] canonical
+  int32_t pad_[2];
 };
 
 constexpr int kDecodeConsumerWarps = 8;
@@ -131,6 +132,8 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
+cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s,
                               uint64_t* launches);

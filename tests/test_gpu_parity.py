@@ -279,13 +279,14 @@ def test_tensor_core_prefill_matches_oracle_and_cuda_core_kernel(B, H, d, rk, rv
     ref = oracle_layer(B_, H, d, U_k, U_v)
     expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
     outs = {}
-    for impl in (2, 1):                              # 2 = tcgen05 kernel, 1 = CUDA-core kernel
+    for impl in (2, 3, 1):                           # 2 = tcgen05 (warp-specialised if it fits), 3 = single-tile tcgen05, 1 = CUDA cores
         lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
         lay.set_option(B.EA_OPT_PREFILL_IMPL, impl)
         outs[impl] = lay.prefill(q, k, v)
         lay.poll_status()
         assert_close(outs[impl], expect, BF16, f"prefill impl {impl}")
     assert float((outs[1].float() - outs[2].float()).abs().max()) < 3e-2
+    assert float((outs[3].float() - outs[2].float()).abs().max()) < 3e-2
 
 
 def test_tensor_core_prefill_chunked_and_lowrank(B):
