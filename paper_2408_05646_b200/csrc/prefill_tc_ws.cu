@@ -120,10 +120,24 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
                       q_rows, nch_k, ld, lane);
     }
     cp_async_commit();
+    // Copy groups in issue order: group 0 = the Q tiles, group j + 1 = key tile j.  `signalled` groups have
+    // been announced on their barrier; a group may be announced once cp.async.wait_group says it landed.
+    int committed = 1, signalled = 0;
+    auto announce = [&](int upto) {                          // groups [signalled, upto) have landed
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0)
+        for (int g = signalled; g < upto; ++g) mbar_arrive(g == 0 ? &hdr->q_full : &hdr->kv_full[(g - 1) % stages]);
+      signalled = max(signalled, upto);
+    };
     bool ok = true;
     for (int j = 0; j < n_max_tiles; ++j) {
       const int stage = j % stages;
       if (j >= stages) {
+        // everything issued so far must be announced before blocking on a free stage: the MMA warp frees
+        // stages only after it has seen the tiles that are still in flight here
+        cp_async_wait<0>();
+        announce(committed);
         if (lane == 0) ok = mbar_wait(&hdr->kv_empty[stage], ((j / stages) - 1) & 1u, p.status) && !*abort_flag;
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;   // one decision for the whole warp
         if (!ok) { *abort_flag = 1; break; }
@@ -134,15 +148,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       load_tile_async(st, Kg + static_cast<int64_t>(key0) * hd.rp_k, hd.rp_k, k_valid, nch_k, ld, lane);
       load_tile_async(st + k_bytes, Vg + static_cast<int64_t>(key0) * hd.rp_v, hd.rp_v, k_valid, nch_v, ld, lane);
       cp_async_commit();
+      ++committed;
       cp_async_wait<1>();                                    // everything but the newest group has landed
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(j == 0 ? &hdr->q_full : &hdr->kv_full[(j - 1) % stages]);
+      announce(committed - 1);
     }
     cp_async_wait<0>();
-    fence_async_smem();
-    __syncwarp();
-    if (ok && lane == 0) mbar_arrive(&hdr->kv_full[(n_max_tiles - 1) % stages]);
+    if (ok) announce(committed);
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
