@@ -217,60 +217,76 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       if (!ok) break;
       tc_fence_after();
       const bool diag = key0 + kTile - 1 > p.len0 + tx;      // some (row, key) pair of the tile is masked
+      // pass 1: row maximum, 64 columns per TMEM round trip
       float row_max = -INFINITY;
 #pragma unroll 1
-      for (int c0 = 0; c0 < kTile; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(tS + c0, r);
+      for (int c0 = 0; c0 < kTile; c0 += 64) {
+        uint32_t r[64];
+        tmem_ld64(tS + c0, r);
         tmem_wait_ld();
+        if (diag) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float s = __uint_as_float(r[i]) * p.scale_log2;
-          if (diag && key0 + c0 + i > my_pos) s = -INFINITY;
-          row_max = fmaxf(row_max, s);
+          for (int i = 0; i < 64; ++i)
+            if (key0 + c0 + i <= my_pos) row_max = fmaxf(row_max, __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 64; ++i) row_max = fmaxf(row_max, __uint_as_float(r[i]));
         }
       }
-      const float m_new = fmaxf(m_run, row_max);
-      const float alpha = ex2(m_run - m_new);
+      row_max *= p.scale_log2;                               // the scale is positive: max and scale commute
+      // Lazy reference: the exponentials use m_run, which follows the true maximum only when that has grown
+      // by more than 8 (a factor 256 that fp32 sums and bf16 P absorb); O' is rescaled only then.
+      float alpha = 1.f;
+      if (row_max > m_run + 8.f) {
+        alpha = ex2(m_run - row_max);
+        m_run = row_max;
+      }
       if (j > 0) {                                           // P_x and O'_x are free once PV_x(j-1) is done
         ok = mbar_wait(&hdr->o_done[x], (j - 1) & 1u, p.status);
         ok = __all_sync(0xffffffffu, ok && !*abort_flag);
         if (!ok) break;
         tc_fence_after();
       }
+      // pass 2: exponentials, row sum, P as bf16 into the A-operand tile
       float row_sum = 0.f;
+      const float neg_m = -m_run;
 #pragma unroll 1
-      for (int c0 = 0; c0 < kTile; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(tS + c0, r);
+      for (int c0 = 0; c0 < kTile; c0 += 64) {
+        uint32_t r[64];
+        tmem_ld64(tS + c0, r);
         tmem_wait_ld();
-        float pr[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float s = __uint_as_float(r[i]) * p.scale_log2 - m_new;
-          if (diag && key0 + c0 + i > my_pos) s = -INFINITY;
-          pr[i] = ex2(s);
-          row_sum += pr[i];
+        for (int g = 0; g < 8; ++g) {
+          float pr[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float e = ex2(fmaf(__uint_as_float(r[g * 8 + i]), p.scale_log2, neg_m));
+            if (diag && key0 + c0 + g * 8 + i > my_pos) e = 0.f;
+            pr[i] = e;
+            row_sum += e;
+          }
+          uint4 w;
+          w.x = pack_bf16(pr[0], pr[1]); w.y = pack_bf16(pr[2], pr[3]);
+          w.z = pack_bf16(pr[4], pr[5]); w.w = pack_bf16(pr[6], pr[7]);
+          *reinterpret_cast<uint4*>(Px + chunk_off(row, (c0 >> 3) + g, grp_p)) = w;
         }
-        uint4 w0, w1;
-        w0.x = pack_bf16(pr[0], pr[1]);   w0.y = pack_bf16(pr[2], pr[3]);
-        w0.z = pack_bf16(pr[4], pr[5]);   w0.w = pack_bf16(pr[6], pr[7]);
-        w1.x = pack_bf16(pr[8], pr[9]);   w1.y = pack_bf16(pr[10], pr[11]);
-        w1.z = pack_bf16(pr[12], pr[13]); w1.w = pack_bf16(pr[14], pr[15]);
-        *reinterpret_cast<uint4*>(Px + chunk_off(row, c0 >> 3, grp_p)) = w0;
-        *reinterpret_cast<uint4*>(Px + chunk_off(row, (c0 >> 3) + 1, grp_p)) = w1;
       }
       l_run = l_run * alpha + row_sum;
-      m_run = m_new;
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale this row of O'
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale this row of O' (rare after the first tiles)
 #pragma unroll 1
-        for (int c0 = 0; c0 < rpv16; c0 += 16) {
-          uint32_t r[16];
-          tmem_ld16(tO + c0, r);
+        for (int h0 = 0; h0 < rpv16; h0 += 64) {             // up to 64 columns per round trip
+          uint32_t r[64];
+#pragma unroll
+          for (int c0 = 0; c0 < 64; c0 += 16)
+            if (h0 + c0 < rpv16) tmem_ld16(tO + h0 + c0, *reinterpret_cast<uint32_t(*)[16]>(&r[c0]));
           tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-          tmem_st16(tO + c0, r);
+          for (int c0 = 0; c0 < 64; c0 += 16)
+            if (h0 + c0 < rpv16) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) r[c0 + i] = __float_as_uint(__uint_as_float(r[c0 + i]) * alpha);
+              tmem_st16(tO + h0 + c0, *reinterpret_cast<const uint32_t(*)[16]>(&r[c0]));
+            }
         }
         tmem_wait_st();
       }

@@ -115,6 +115,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       "r"(taddr)
       : "memory");
 }
+// 64 consecutive columns: four loads in flight before the caller waits once.
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) tmem_ld16(taddr + 16 * k, *reinterpret_cast<uint32_t(*)[16]>(&r[16 * k]));
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
