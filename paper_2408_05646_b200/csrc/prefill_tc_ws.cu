@@ -157,14 +157,22 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      // One thread feeds the tensor pipe, so its per-instruction overhead is on the critical path: all
+      // descriptors are built once and advanced by adding 16-byte units to their address field.
       const uint32_t idesc_s = instr_desc(kTile, false);
       const uint32_t idesc_o = instr_desc(rpv16, true);
       const uint32_t qa = smem_u32(Qs), ra = smem_u32(ring), pa = smem_u32(Ps);
-      auto issue_s = [&](int x, int j) {                     // S_x = Q_x K_j^T
-        const uint32_t ka = ra + (j % stages) * stage_bytes;
-        for (int s = 0; s < rpk16 / 16; ++s)
-          mma_ss(tmem + x * kTile, smem_desc(qa + x * q_bytes + s * 256, 128, grp_k),
-                 smem_desc(ka + s * 256, 128, grp_k), idesc_s, s > 0);
+      const uint64_t dq[2] = {smem_desc(qa, 128, grp_k), smem_desc(qa + q_bytes, 128, grp_k)};
+      const uint64_t dp[2] = {smem_desc(pa, 128, grp_p), smem_desc(pa + p_bytes, 128, grp_p)};
+      const uint64_t dk0 = smem_desc(ra, 128, grp_k);                 // K tile of stage 0 (K-major B operand)
+      const uint64_t dv0 = smem_desc(ra + k_bytes, grp_v, 128);       // V tile of stage 0 (MN-major B operand)
+      const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
+      const uint64_t v_step = static_cast<uint64_t>((2 * grp_v) >> 4); // 16 keys = two 8-row groups
+      const int ks_steps = rpk16 >> 4;
+      const uint32_t ts[2] = {tmem, tmem + kTile}, to[2] = {tmem + 256, tmem + 256 + kTile};
+      auto issue_s = [&](int x, int stage) {                 // S_x = Q_x K^T, contraction over the rank
+        uint64_t a = dq[x], bk = dk0 + stage * stage_step;
+        for (int s = 0; s < ks_steps; ++s, a += 16, bk += 16) mma_ss(ts[x], a, bk, idesc_s, s > 0);
         mma_commit(&hdr->s_full[x]);
       };
       bool ok = mbar_wait(&hdr->q_full, 0, p.status) && mbar_wait(&hdr->kv_full[0], 0, p.status);
@@ -173,26 +181,29 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         for (int x = 0; x < 2; ++x)
           if (n_tiles[x] > 0) issue_s(x, 0);
       }
+      int stage = 0, nstage = stages > 1 ? 1 : 0;            // ring slots of key tiles j and j + 1
+      uint32_t nparity = stages > 1 ? 0u : 1u;               // kv_full parity of tile j + 1
       for (int j = 0; j < n_max_tiles && ok; ++j) {
-        const int stage = j % stages;
         for (int x = 0; x < 2 && ok; ++x) {
           if (j >= n_tiles[x]) continue;
           ok = mbar_wait(&hdr->p_full[x], j & 1u, p.status) && !*abort_flag;
           if (!ok) break;
           tc_fence_after();
-          const uint32_t va = ra + stage * stage_bytes + k_bytes;
-          for (int s = 0; s < kTile / 16; ++s)               // O'_x += P_x V_j
-            mma_ss(tmem + 256 + x * kTile, smem_desc(pa + x * p_bytes + s * 256, 128, grp_p),
-                   smem_desc(va + s * 2 * grp_v, grp_v, 128), idesc_o, j > 0 || s > 0);
+          uint64_t a = dp[x], bv = dv0 + stage * stage_step;
+#pragma unroll
+          for (int s = 0; s < kTile / 16; ++s, a += 16, bv += v_step)   // O'_x += P_x V_j over the 128 keys
+            mma_ss(to[x], a, bv, idesc_o, j > 0 || s > 0);
           mma_commit(&hdr->o_done[x]);
           if (j + 1 < n_tiles[x]) {
-            ok = mbar_wait(&hdr->kv_full[(j + 1) % stages], ((j + 1) / stages) & 1u, p.status);
+            ok = mbar_wait(&hdr->kv_full[nstage], nparity, p.status);
             if (!ok) break;
             tc_fence_after();
-            issue_s(x, j + 1);
+            issue_s(x, nstage);
           }
         }
         if (ok) mma_commit(&hdr->kv_empty[stage]);           // stage free once everything issued so far is done
+        stage = nstage;
+        if (++nstage == stages) { nstage = 0; nparity ^= 1u; }
       }
       // the last commit's arrival must have landed before the CTA may leave
       if (ok) ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
