@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libeigenattn.so")
+LIB_PATH = os.environ.get("EIGEN_ATTN_LIB", os.path.join(_HERE, "libeigenattn.so"))   # override: another build of the library
 
 EA_OK = 0
 EA_ERR_INVALID_ARG, EA_ERR_SHAPE, EA_ERR_CAPACITY, EA_ERR_UNSUPPORTED = -1, -2, -3, -4
