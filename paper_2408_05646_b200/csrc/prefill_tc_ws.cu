@@ -25,7 +25,8 @@ constexpr int kSoftmaxWarps = 8;
 constexpr int kMmaWarp = 8;
 constexpr int kLoadWarp0 = 9;
 constexpr int kLoadWarps = 2;
-constexpr int kWsThreads = (kSoftmaxWarps + 1 + kLoadWarps) * 32;
+constexpr int kSIssueWarp = 11;               // issues the S products; kMmaWarp issues the PV products
+constexpr int kWsThreads = (kSoftmaxWarps + 1 + kLoadWarps + 1) * 32;
 constexpr int kMaxStages = 3;
 
 struct __align__(16) WsHeader {
@@ -104,7 +105,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int n_keys = p.len0 + min(p.T, t0 + 2 * kTile);      // rows of K'/V' the CTA may touch
   const int total_rows = p.B * p.T;
 
-  if (warp >= kLoadWarp0) {
+  if (warp >= kLoadWarp0 && warp < kLoadWarp0 + kLoadWarps) {
     // ------------------------------------------------------------------ loaders
     const int ld = warp - kLoadWarp0;
     const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.qp) +
@@ -154,11 +155,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     }
     cp_async_wait<0>();
     if (ok) announce(committed);
-  } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == kMmaWarp || warp == kSIssueWarp) {
+    // ------------------------------------------------------------------ MMA issuers
+    // Two threads feed the tensor pipe so that their per-instruction latencies overlap: one issues the
+    // PV products, the other the S products of the next key tile.  Both start a tile's work when the
+    // softmax group has written P (which also means it has consumed S).  Descriptors are built once
+    // and advanced by adding 16-byte units to their address field.
     if (lane == 0) {
-      // One thread feeds the tensor pipe, so its per-instruction overhead is on the critical path: all
-      // descriptors are built once and advanced by adding 16-byte units to their address field.
+      const bool pv_role = warp == kMmaWarp;
       const uint32_t idesc_s = instr_desc(kTile, false);
       const uint32_t idesc_o = instr_desc(rpv16, true);
       const uint32_t qa = smem_u32(Qs), ra = smem_u32(ring), pa = smem_u32(Ps);
@@ -175,38 +179,45 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         for (int s = 0; s < ks_steps; ++s, a += 16, bk += 16) mma_ss(ts[x], a, bk, idesc_s, s > 0);
         mma_commit(&hdr->s_full[x]);
       };
-      bool ok = mbar_wait(&hdr->q_full, 0, p.status) && mbar_wait(&hdr->kv_full[0], 0, p.status);
-      if (ok) {
-        tc_fence_after();
-        for (int x = 0; x < 2; ++x)
-          if (n_tiles[x] > 0) issue_s(x, 0);
+      bool ok = true;
+      if (!pv_role) {
+        ok = mbar_wait(&hdr->q_full, 0, p.status) && mbar_wait(&hdr->kv_full[0], 0, p.status);
+        if (ok) {
+          tc_fence_after();
+          for (int x = 0; x < 2; ++x)
+            if (n_tiles[x] > 0) issue_s(x, 0);
+        }
       }
       int stage = 0, nstage = stages > 1 ? 1 : 0;            // ring slots of key tiles j and j + 1
       uint32_t nparity = stages > 1 ? 0u : 1u;               // kv_full parity of tile j + 1
       for (int j = 0; j < n_max_tiles && ok; ++j) {
         for (int x = 0; x < 2 && ok; ++x) {
           if (j >= n_tiles[x]) continue;
+          if (!pv_role && j + 1 >= n_tiles[x]) continue;     // no further S product for this tile
           ok = mbar_wait(&hdr->p_full[x], j & 1u, p.status) && !*abort_flag;
           if (!ok) break;
           tc_fence_after();
-          uint64_t a = dp[x], bv = dv0 + stage * stage_step;
+          if (pv_role) {
+            uint64_t a = dp[x], bv = dv0 + stage * stage_step;
 #pragma unroll
-          for (int s = 0; s < kTile / 16; ++s, a += 16, bv += v_step)   // O'_x += P_x V_j over the 128 keys
-            mma_ss(to[x], a, bv, idesc_o, j > 0 || s > 0);
-          mma_commit(&hdr->o_done[x]);
-          if (j + 1 < n_tiles[x]) {
+            for (int s = 0; s < kTile / 16; ++s, a += 16, bv += v_step)   // O'_x += P_x V_j over the 128 keys
+              mma_ss(to[x], a, bv, idesc_o, j > 0 || s > 0);
+            mma_commit(&hdr->o_done[x]);
+          } else {
             ok = mbar_wait(&hdr->kv_full[nstage], nparity, p.status);
             if (!ok) break;
             tc_fence_after();
             issue_s(x, nstage);
           }
         }
-        if (ok) mma_commit(&hdr->kv_empty[stage]);           // stage free once everything issued so far is done
+        // the PV products are the last readers of a stage (its S products completed before the softmax ran)
+        if (ok && pv_role) mma_commit(&hdr->kv_empty[stage]);
         stage = nstage;
         if (++nstage == stages) { nstage = 0; nparity ^= 1u; }
       }
       // the last commit's arrival must have landed before the CTA may leave
-      if (ok) ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
+      if (ok && pv_role)
+        ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
       if (!ok) *abort_flag = 1;
     }
   } else {
@@ -268,17 +279,19 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         tmem_wait_ld();
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
-          float pr[8];
+          // P is cut to bf16 by truncation with integer ops, and the row sum adds the truncated values, so
+          // numerator and denominator of the softmax use identical weights.
+          uint32_t pt[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             float e = ex2(fmaf(__uint_as_float(r[g * 8 + i]), p.scale_log2, neg_m));
             if (diag && key0 + c0 + g * 8 + i > my_pos) e = 0.f;
-            pr[i] = e;
-            row_sum += e;
+            pt[i] = __float_as_uint(e) & 0xffff0000u;
+            row_sum += __uint_as_float(pt[i]);
           }
           uint4 w;
-          w.x = pack_bf16(pr[0], pr[1]); w.y = pack_bf16(pr[2], pr[3]);
-          w.z = pack_bf16(pr[4], pr[5]); w.w = pack_bf16(pr[6], pr[7]);
+          w.x = __byte_perm(pt[0], pt[1], 0x7632); w.y = __byte_perm(pt[2], pt[3], 0x7632);
+          w.z = __byte_perm(pt[4], pt[5], 0x7632); w.w = __byte_perm(pt[6], pt[7], 0x7632);
           *reinterpret_cast<uint4*>(Px + chunk_off(row, (c0 >> 3) + g, grp_p)) = w;
         }
       }
@@ -394,7 +407,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int img16 = p.d_head * rpv16 * 2 / 16;               // 16-byte words per image
   if (run) {
     const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.uvl16_off);
-    for (int idx = tid - kMmaWarp * 32; idx < 2 * img16; idx += (1 + kLoadWarps) * 32)
+    for (int idx = tid - kMmaWarp * 32; idx < 2 * img16; idx += (2 + kLoadWarps) * 32)
       reinterpret_cast<uint4*>(Uh)[idx] = __ldg(Ug + idx);
   }
   fence_async_smem();
