@@ -1,0 +1,152 @@
+"""GPU parity at the sizes of the reference workloads, in the launch configuration the benchmark times:
+the cache is filled on the GPU chunk by chunk, and the outputs of a seeded sample of (sequence, head)
+units are compared one by one with the fp64 oracle, which receives the same rows."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import BF16_MAX_ABS, BF16_MEAN_ABS, to_np
+from oracle import eigen_attention as orc
+from paper_2408_05646_b200 import synth
+
+pytestmark = pytest.mark.gpu
+FILL = 1024
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    return binding
+
+
+def build_and_fill(B, wl, units, extra_rows=1):
+    """Layer filled with wl.context rows; returns the raw rows of the sampled units for the oracle."""
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    dt = synth.torch_dtype(wl.dtype)
+    lay = B.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + extra_rows, dt, U_k, U_v)
+    W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K", device="cuda:0")
+    W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V", device="cuda:0")
+    hist = {u: ([], []) for u in units}
+    for ci, c in enumerate(range(0, wl.context, FILL)):
+        t = min(FILL, wl.context - c)
+        k = synth.lowrank_rows(W_k, wl.batch, t, wl.sigma, wl.index, "K", chunk=ci, dtype=dt, device="cuda:0")
+        v = synth.lowrank_rows(W_v, wl.batch, t, wl.sigma, wl.index, "V", chunk=ci, dtype=dt, device="cuda:0")
+        lay.append_kv(k, v)
+        for (b, h) in units:
+            hist[(b, h)][0].append(to_np(k[b, :, h, :]))
+            hist[(b, h)][1].append(to_np(v[b, :, h, :]))
+    hist = {u: (np.concatenate(a), np.concatenate(b_)) for u, (a, b_) in hist.items()}
+    return lay, ranks, U_k, U_v, W_k, W_v, hist
+
+
+def check_units(out, q, hist, new_rows, units, U_k, U_v):
+    """out[b, 0, h] against the definition for every sampled unit (history + the new rows)."""
+    errs = []
+    for (b, h) in units:
+        K = np.concatenate([hist[(b, h)][0]] + [to_np(r[0][b, :, h, :]) for r in new_rows])
+        V = np.concatenate([hist[(b, h)][1]] + [to_np(r[1][b, :, h, :]) for r in new_rows])
+        ref = orc.decode_head(to_np(q[b, 0, h]), K, V, U_k[h], U_v[h])
+        errs.append(np.abs(to_np(out[b, 0, h]) - ref))
+    e = np.stack(errs)
+    assert np.isfinite(to_np(out)).all()
+    assert e.max() <= BF16_MAX_ABS and e.mean() <= BF16_MEAN_ABS, (e.max(), e.mean())
+
+
+def test_llama2_7b_b16_n32k_full_size_sampled_units(B):
+    wl = synth.WORKLOADS["llama2_7b_b16_n32k"]
+    ranks0 = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    units = synth.sample_units(wl.batch, wl.n_heads, ranks0, 18, wl.index)[:18]
+    lay, ranks, U_k, U_v, W_k, W_v, hist = build_and_fill(B, wl, units)
+    dt = torch.bfloat16
+    k1 = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device="cuda:0")
+    v1 = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt, device="cuda:0")
+    q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt, device="cuda:0")
+    out = lay.decode_step(q, k1, v1)                        # the step the benchmark times (one fused launch)
+    lay.poll_status()
+    assert lay.len == wl.context + 1
+    check_units(out, q, hist, [(k1, v1)], units, U_k, U_v)
+    # the separate-launch path and the plain decode entry point give the same rows
+    lay.set_option(B.EA_OPT_DECODE_FUSED, 0)
+    out2 = lay.decode(q)
+    assert float((out2.float() - out.float()).abs().max()) <= 1e-2
+
+
+@pytest.mark.parametrize("batch,context", [(1, 2048), (4, 8192), (16, 2048)])
+def test_opt_6p7b_hetero_ranks_sampled_units(B, batch, context):
+    wl = dataclasses.replace(synth.WORKLOADS["opt_6p7b_hetero"], batch=batch, context=context)
+    ranks0 = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    assert len(set(ranks0)) == 5                            # every rank of the set occurs
+    units = synth.sample_units(wl.batch, wl.n_heads, ranks0, 24, wl.index)[:24]
+    lay, ranks, U_k, U_v, W_k, W_v, hist = build_and_fill(B, wl, units)
+    dt = torch.bfloat16
+    k1 = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device="cuda:0")
+    v1 = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt, device="cuda:0")
+    q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt, device="cuda:0")
+    out = lay.decode_step(q, k1, v1)
+    lay.poll_status()
+    check_units(out, q, hist, [(k1, v1)], units, U_k, U_v)
+
+
+@pytest.mark.parametrize("batch", [1, 2])
+def test_mpt_7b_long_context_64_steps(B, batch):
+    # 131072 cached rows, r = 64: every unit is split over many CTAs; then 64 single-token steps, and the
+    # same 64 rows appended in one call give the identical cache
+    wl = dataclasses.replace(synth.WORKLOADS["mpt_7b_long"], batch=batch)
+    ranks0 = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    units = [(0, 0), (batch - 1, wl.n_heads - 1), (0, 13), (batch - 1, 20)]
+    steps = 64
+    lay, ranks, U_k, U_v, W_k, W_v, hist = build_and_fill(B, wl, units, extra_rows=steps)
+    dt = torch.bfloat16
+    kn = synth.lowrank_rows(W_k, wl.batch, steps, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device="cuda:0")
+    vn = synth.lowrank_rows(W_v, wl.batch, steps, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt, device="cuda:0")
+    new_rows = []
+    for t in range(steps):
+        q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, step=t, dtype=dt, device="cuda:0")
+        out = lay.decode_step(q, kn[:, t:t + 1], vn[:, t:t + 1])
+        new_rows.append((kn[:, t:t + 1], vn[:, t:t + 1]))
+        if t in (0, 31, 63):
+            check_units(out, q, hist, new_rows, units, U_k, U_v)
+    lay.poll_status()
+    assert lay.len == wl.context + steps
+    tail = {h: (lay.cache_rows(h, "k")[:, wl.context:].clone(), lay.cache_rows(h, "v")[:, wl.context:].clone())
+            for h in (0, 13, 31)}
+    lay.set_len(wl.context)
+    lay.append_kv(kn, vn)                                   # the same 64 tokens in one call
+    for h, (kk, vv) in tail.items():
+        assert torch.equal(lay.cache_rows(h, "k")[:, wl.context:], kk)
+        assert torch.equal(lay.cache_rows(h, "v")[:, wl.context:], vv)
+
+
+def test_prefill_b4_t4096_sampled_rows_then_decode(B):
+    wl = synth.WORKLOADS["prefill_b4_t4096"]
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    T, dt = wl.context, torch.bfloat16
+    lay = B.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T)
+    W = {t: synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_" + t, device="cuda:0") for t in "KVQ"}
+    k = synth.lowrank_rows(W["K"], wl.batch, T + 1, wl.sigma, wl.index, "K", dtype=dt, device="cuda:0")
+    v = synth.lowrank_rows(W["V"], wl.batch, T + 1, wl.sigma, wl.index, "V", dtype=dt, device="cuda:0")
+    q = synth.lowrank_rows(W["Q"], wl.batch, T + 1, wl.sigma, wl.index, "Q", dtype=dt, device="cuda:0")
+    out = lay.prefill(q[:, :T], k[:, :T], v[:, :T])
+    lay.poll_status()
+    assert np.isfinite(to_np(out)).all()
+    errs = []
+    for (b, h) in [(0, 0), (3, 31), (1, 7), (2, 19)]:
+        kk, vv = to_np(k[b, :, h]), to_np(v[b, :, h])
+        for t in (0, 1, 127, 128, 255, 256, 1000, 2047, 2048, T - 1):
+            ref = orc.decode_head(to_np(q[b, t, h]), kk[:t + 1], vv[:t + 1], U_k[h], U_v[h])
+            errs.append(np.abs(to_np(out[b, t, h]) - ref))
+    e = np.stack(errs)
+    assert e.max() <= BF16_MAX_ABS and e.mean() <= BF16_MEAN_ABS, (e.max(), e.mean())
+    # the cache written by the prefill serves the next decode step
+    o1 = lay.decode_step(q[:, T:], k[:, T:], v[:, T:])
+    for (b, h) in [(0, 0), (3, 31)]:
+        ref = orc.decode_head(to_np(q[b, T, h]), to_np(k[b, :, h]), to_np(v[b, :, h]), U_k[h], U_v[h])
+        assert np.abs(to_np(o1[b, 0, h]) - ref).max() <= BF16_MAX_ABS
