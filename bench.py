@@ -31,6 +31,10 @@ from paper_2408_05646_b200 import synth
 METRIC = "rank-r decode attention KV GB/s (B=16, n=32k, 7B layer; us/step alongside)"
 UNIT = "GB/s"
 FILL_CHUNK = 1024          # tokens per append call while filling the cache
+# DRAM bytes moved per algorithmic byte by decode_splitkv_kernel, from the ncu capture summarised in
+# profiles/decode_splitkv_llama2_7b_b2_n32k_full.md (B = 2 case: 680.7 MB for 671.1 MB; traffic grows in
+# proportion to the number of units).  Set to None whenever that kernel changes after the capture.
+DECODE_TRAFFIC_RATIO = 680.78 / 671.11
 
 
 def measured_peaks():
@@ -361,19 +365,71 @@ def run_ours(args, wl):
         "frac_of_nominal_8TBs": value / world / 8000.0,
         "roofline": {"bound": "hbm", "kernel": "decode_splitkv_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                     "kernel_us": kern_avg_ms * 1e3, "algorithmic_bytes": bytes_step, "traffic": None},
+                     "kernel_us": kern_avg_ms * 1e3, "algorithmic_bytes": bytes_step,
+                     "traffic": (bytes_step * DECODE_TRAFFIC_RATIO
+                                 if DECODE_TRAFFIC_RATIO and wl.name == "llama2_7b_b16_n32k" else None),
+                     "traffic_source": "ncu dram bytes of the B=2 case scaled by units (profiles/)"},
         "e2e": {"value": e2e_value, "unit": UNIT, "us_per_step": e2e_ms_step * 1e3,
                 "h2d_bytes_per_step": 3 * io_bytes, "d2h_bytes_per_step": io_bytes,
                 "matches_device_path": same},
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    if not args.no_prefill and world == 1:
+        del lay
+        torch.cuda.empty_cache()
+        line["prefill"] = prefill_measure(synth.WORKLOADS["prefill_b4_t4096"], device, steps=10, warmup=3)
     if cpu is not None:
         line["cpu_baseline"] = cpu
         line["parity_full_size"] = parity
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def prefill_measure(wl, device, steps, warmup, impl=0):
+    """Times eigen_attn_prefill on the prompt workload; returns a small dict (call time, attention-kernel time,
+    TFLOP/s of the causal contractions, fraction of the measured bf16 peak)."""
+    from paper_2408_05646_b200 import binding
+    ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
+    U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
+    dt = synth.torch_dtype(wl.dtype)
+    T = wl.context
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device)
+    if impl:
+        lay.set_option(binding.EA_OPT_PREFILL_IMPL, impl)
+    W = {t: synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_" + t, device=device) for t in "KVQ"}
+    k = synth.lowrank_rows(W["K"], wl.batch, T, wl.sigma, wl.index, "K", dtype=dt, device=device)
+    v = synth.lowrank_rows(W["V"], wl.batch, T, wl.sigma, wl.index, "V", dtype=dt, device=device)
+    q = synth.lowrank_rows(W["Q"], wl.batch, T, wl.sigma, wl.index, "Q", dtype=dt, device=device)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream(device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        a.record(stream); b.record(stream)
+    for _ in range(warmup):
+        lay.set_len(0); lay.prefill(q, k, v, out=out)
+    torch.cuda.synchronize(device)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        lay.set_decode_events(ev[i][0], ev[i][1])
+        lay.set_len(0); lay.prefill(q, k, v, out=out)
+    t1.record(stream)
+    torch.cuda.synchronize(device)
+    lay.set_decode_events(None, None)
+    lay.poll_status()
+    ms = t0.elapsed_time(t1) / steps
+    kern = sum(a.elapsed_time(b) for a, b in ev) / steps
+    flop = 2 * (wl.batch * T * (T + 1) // 2) * sum(2 * r for r in ranks)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["bf16_tflops"]) if os.path.exists(peaks_path) else 1590.0
+    tf = flop / (kern * 1e-3) / 1e12
+    return {"workload": wl.name, "ms_per_call": ms, "attention_kernel_ms": kern, "attention_tflops": tf,
+            "bound": "tensor", "peak_tflops": peak, "frac": tf / peak,
+            "peak_source": "measured burst" if os.path.exists(peaks_path) else "fallback",
+            "flop_counted": "causal Q'K'^T + PV' (projections and lift excluded)"}
 
 
 def run_prefill(args, wl):
@@ -457,6 +513,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")
