@@ -197,25 +197,23 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
     while (tile_rows > 16 && static_cast<int64_t>(B) * H * ((n + tile_rows - 1) / tile_rows) < 4ll * sms)
       tile_rows >>= 1;
   }
-  int stage_bytes = 0, stages = 0;
+  // The ring: slots are sized per head inside the kernel.  Measured on B200: about 120 KB of copies in
+  // flight per SM saturates HBM and deeper rings lose bandwidth again (more concurrent DRAM streams), so
+  // the ring holds max(3 slots, 120 KB) of the widest head, as far as shared memory allows.
+  int ring_bytes = 0;
   for (;;) {
-    stage_bytes = static_cast<int>(align_up(static_cast<size_t>(tile_rows) * (L.max_rp_k + L.max_rp_v) * L.es, 128));
-    stages = (kSmemLimit - fixed) / stage_bytes;
-    if (stages >= 3 || tile_rows <= 16) break;
+    const int widest = static_cast<int>(align_up(static_cast<size_t>(tile_rows) * L.max_w * L.es, 128));
+    const int avail = kSmemLimit - fixed;
+    if (3 * widest <= avail || tile_rows <= 16) {
+      int want = 3 * widest > kInFlightBytes + widest ? 3 * widest : kInFlightBytes + widest;
+      if (h->opt_stages > 0) want = static_cast<int>(h->opt_stages) * widest;
+      ring_bytes = want < avail ? want : avail;
+      if (ring_bytes < widest)
+        return fail(h, EA_ERR_UNSUPPORTED, "%s: a tile of %d rows does not fit in shared memory", who, tile_rows);
+      break;
+    }
     tile_rows >>= 1;
   }
-  if (stages > 12) stages = 12;
-  if (h->opt_stages > 0) {
-    if (h->opt_stages < stages) stages = static_cast<int>(h->opt_stages);
-  } else {
-    // Measured on B200: about 120 KB of copies in flight per SM saturates HBM; deeper rings lose
-    // bandwidth again (more concurrent DRAM streams), so the ring is not simply made as deep as fits.
-    int want = (kInFlightBytes + stage_bytes - 1) / stage_bytes;
-    if (want < 3) want = 3;
-    if (want < stages) stages = want;
-  }
-  if (stages < 1)
-    return fail(h, EA_ERR_UNSUPPORTED, "%s: a tile of %d rows does not fit in shared memory", who, tile_rows);
 
   const int nt = (n + tile_rows - 1) / tile_rows;
   const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
@@ -235,13 +233,13 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.status = dev_status(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
-  p.tile_rows = tile_rows; p.nt = nt; p.stages = stages; p.stage_bytes = stage_bytes;
-  p.v_tile_off = tile_rows * L.max_rp_k * L.es;
+  p.tile_rows = tile_rows; p.nt = nt; p.ring_bytes = ring_bytes; p.inflight_bytes = kInFlightBytes;
+  p.fixed_stages = static_cast<int>(h->opt_stages);
   p.w_total = w_total;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
   plan->grid = grid;
-  plan->smem = static_cast<size_t>(fixed) + static_cast<size_t>(stages) * stage_bytes;
+  plan->smem = static_cast<size_t>(fixed) + static_cast<size_t>(ring_bytes);
 
   ea::CombineParams& c = plan->c;
   c = ea::CombineParams{};

@@ -97,16 +97,36 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// Position in the shared-memory ring: slot index and the parity of the slot's current fill.
-struct RingPos {
-  int stage = 0;
-  uint32_t parity = 0;
-  uint32_t count = 0;     // tiles so far
-  __device__ __forceinline__ void advance(int stages) {
-    ++count;
-    if (++stage == stages) { stage = 0; parity ^= 1u; }
-  }
+// The shared-memory ring as one role sees it.  Slots are sized for the head being streamed (a narrow
+// head gets more, smaller slots, so the bytes in flight stay the same), hence the slot count can change
+// from one piece to the next; every slot's mbarriers keep their own phase, tracked as one parity bit per
+// slot.  Producer and consumers derive the same geometry from the head and walk the slots in the same order.
+struct Ring {
+  int stage = 0;            // next slot
+  int stages = 0;           // slots of the current geometry
+  int stage_bytes = 0;      // bytes per slot: K tile, then V tile at v_off
+  int v_off = 0;
+  uint32_t full_bits = 0;   // bit s: parity of slot s's next "full" phase
+  uint32_t empty_bits = 0;  // bit s: parity of slot s's next "empty" phase (producer only)
+  uint32_t filled = 0;      // bit s: the slot holds a tile not yet known to be released (producer only)
+  __device__ __forceinline__ void advance() { if (++stage == stages) stage = 0; }
 };
+
+// Slot geometry for a head: about p.inflight_bytes of copies in flight, at least three slots if they fit.
+template <typename T>
+__device__ __forceinline__ void ring_geometry(const DecodeParams& p, const HeadInfo& hd, int* stage_bytes,
+                                              int* v_off, int* stages) {
+  const int kb = p.tile_rows * hd.rp_k * static_cast<int>(sizeof(T));
+  const int vb = p.tile_rows * hd.rp_v * static_cast<int>(sizeof(T));
+  const int sb = (kb + vb + 127) & ~127;
+  int fit = p.ring_bytes / sb;
+  if (fit > kMaxStages) fit = kMaxStages;
+  int want = p.fixed_stages > 0 ? p.fixed_stages : (p.inflight_bytes + sb - 1) / sb;
+  if (want < 3 && p.fixed_stages == 0) want = 3;
+  *stage_bytes = sb;
+  *v_off = kb;
+  *stages = want < fit ? want : fit;
+}
 
 // L2 policy for data that is read once: evict it first.
 __device__ __forceinline__ uint64_t policy_evict_first() {
@@ -175,7 +195,7 @@ __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
 template <typename T, int NCH>
 __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
                                             unsigned char* ring, const HeadInfo& hd, int i0, int i1,
-                                            RingPos& pos, int warp, int lane, bool with_new_row) {
+                                            Ring& ring_state, int warp, int lane, bool with_new_row) {
   constexpr int EPC = Elem<T>::kPerChunk;
   const int pair = lane >> 1, half = lane & 1;
   const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
@@ -248,17 +268,18 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   };
 
   for (int i = i0; i < i1; ++i) {
-    const int stage = pos.stage;
-    const uint32_t parity = pos.parity;
-    pos.advance(p.stages);
+    const int stage = ring_state.stage;
+    const uint32_t parity = (ring_state.full_bits >> stage) & 1u;
+    ring_state.full_bits ^= 1u << stage;
+    ring_state.advance();
     // warp-uniform decisions: the row code below shuffles across the whole warp
     if (__any_sync(0xffffffffu, *abort_flag != 0)) continue;
     if (__any_sync(0xffffffffu, !mbar_wait(&fx->full[stage], parity, p.status))) {
       *abort_flag = 1;
       continue;
     }
-    const unsigned char* kt = ring + static_cast<size_t>(stage) * p.stage_bytes;
-    const unsigned char* vt = kt + p.v_tile_off;
+    const unsigned char* kt = ring + static_cast<size_t>(stage) * ring_state.stage_bytes;
+    const unsigned char* vt = kt + ring_state.v_off;
     const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
     // The loop bound is the same for all lanes of a warp (the shuffle inside needs every lane);
     // lane pairs past the last row recompute the group's first row and drop the result.
@@ -480,7 +501,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
   const int grid = gridDim.x, cta = blockIdx.x;
 
   if (tid == 0) {
-    for (int s = 0; s < p.stages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(&fx->full[s], 1);
       mbar_init(&fx->empty[s], kDecodeConsumerWarps);
     }
@@ -497,7 +518,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
     // ------------------------------------------------------------ producer
     if (lane == 0) {
       const uint64_t policy = policy_evict_first();
-      RingPos pos;
+      Ring rg;
       bool ok = true;
       long long F = f_lo;
       while (F < f_hi && ok) {
@@ -507,6 +528,20 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + (f_hi - F)));
         const int h = unit / p.B, b = unit - h * p.B;
         const HeadInfo hd = p.heads[h];
+        int sb, voff, nst;
+        ring_geometry<T>(p, hd, &sb, &voff, &nst);
+        if (sb != rg.stage_bytes || nst != rg.stages) {
+          // New slot layout: the new slots overlap the old ones differently, so every tile still in the
+          // ring must have been released before the first copy into the new layout.
+          for (int s2 = 0; s2 < kMaxStages && ok; ++s2)
+            if (rg.filled & (1u << s2)) {
+              ok = mbar_wait(&fx->empty[s2], (rg.empty_bits >> s2) & 1u, p.status);
+              rg.empty_bits ^= 1u << s2;
+              rg.filled &= ~(1u << s2);
+            }
+          if (!ok) { *abort_flag = 1; break; }
+          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb; rg.v_off = voff;
+        }
         const uint32_t rowb_k = hd.rp_k * sizeof(T), rowb_v = hd.rp_v * sizeof(T);
         const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i0) * p.tile_rows;
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
@@ -514,11 +549,15 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
         for (int i = i0; i < i1; ++i) {
           if (*abort_flag) { ok = false; break; }
-          if (pos.count >= static_cast<uint32_t>(p.stages) &&
-              !mbar_wait(&fx->empty[pos.stage], pos.parity ^ 1u, p.status)) {
-            *abort_flag = 1;
-            ok = false;
-            break;
+          const int st = rg.stage;
+          const uint32_t bit = 1u << st;
+          if (rg.filled & bit) {          // the slot's previous tile must have been released
+            if (!mbar_wait(&fx->empty[st], (rg.empty_bits >> st) & 1u, p.status)) {
+              *abort_flag = 1;
+              ok = false;
+              break;
+            }
+            rg.empty_bits ^= bit;
           }
           uint32_t bytes_k = tile_k, bytes_v = tile_v;
           if (i == p.nt - 1) {            // ragged last tile of the unit
@@ -526,30 +565,27 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
             bytes_k = rows * rowb_k;
             bytes_v = rows * rowb_v;
           }
-          unsigned char* dst = ring + static_cast<size_t>(pos.stage) * p.stage_bytes;
-          void* bar = &fx->full[pos.stage];
+          unsigned char* dst = ring + static_cast<size_t>(st) * rg.stage_bytes;
+          void* bar = &fx->full[st];
           mbar_arrive_expect_tx(bar, bytes_k + bytes_v);
           bulk_g2s_hint(dst, src_k, bytes_k, bar, policy);
-          bulk_g2s_hint(dst + p.v_tile_off, src_v, bytes_v, bar, policy);
+          bulk_g2s_hint(dst + rg.v_off, src_v, bytes_v, bar, policy);
+          rg.filled |= bit;
+          rg.full_bits ^= bit;            // bit now holds the parity of the slot's next fill
           src_k += tile_k;
           src_v += tile_v;
-          pos.advance(p.stages);
+          rg.advance();
         }
         F += i1 - i0;
       }
-      // Make sure every copy this thread issued has landed before the CTA can exit: walk back over
-      // the last min(count, stages) fills.
-      const uint32_t pending = pos.count < static_cast<uint32_t>(p.stages) ? pos.count : p.stages;
-      int st = pos.stage;
-      uint32_t par = pos.parity;
-      for (uint32_t j = 0; j < pending; ++j) {
-        if (st == 0) { st = p.stages - 1; par ^= 1u; } else { --st; }
-        mbar_wait(&fx->full[st], par, p.status);
-      }
+      // Make sure every copy this thread issued has landed before the CTA can exit: the latest fill of
+      // every slot in use (its phase parity is the opposite of the slot's next one).
+      for (int s2 = 0; s2 < kMaxStages; ++s2)
+        if (rg.filled & (1u << s2)) mbar_wait(&fx->full[s2], ((rg.full_bits >> s2) & 1u) ^ 1u, p.status);
     }
   } else {
     // ------------------------------------------------------------ consumers
-    RingPos pos;
+    Ring rg;
     long long F = f_lo;
     while (F < f_hi) {
       const int unit = static_cast<int>(F / p.nt);
@@ -558,6 +594,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + left));
       const int h = unit / p.B, b = unit - h * p.B;
       const HeadInfo hd = p.heads[h];
+      {
+        int sb, voff, nst;
+        ring_geometry<T>(p, hd, &sb, &voff, &nst);
+        if (sb != rg.stage_bytes || nst != rg.stages) {      // same decision as the producer's
+          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb; rg.v_off = voff;
+        }
+      }
       const bool whole = i0 == 0 && i1 == p.nt;
       const bool with_new_row = p.k_new != nullptr && i1 == p.nt;
       project_inputs<T>(p, fx, hd, h, b, tid, with_new_row);
@@ -565,14 +608,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, pos, warp, lane, with_new_row); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
       }
       finish_piece<T>(p, fx, hd, unit, h, b, cta, grid, whole, tid);
       F += i1 - i0;

@@ -49,9 +49,9 @@ struct DecodeParams {
   int32_t n_max;
   int32_t tile_rows;        // rows per tile
   int32_t nt;               // tiles per unit = ceil(n / tile_rows)
-  int32_t stages;
-  int32_t stage_bytes;      // bytes per ring stage (K tile then V tile)
-  int32_t v_tile_off;       // byte offset of the V tile inside a stage
+  int32_t ring_bytes;       // shared memory of the tile ring; slots are sized per head inside the kernel
+  int32_t inflight_bytes;   // target bytes of copies in flight per SM (sets the slot count per head)
+  int32_t fixed_stages;     // > 0: use this many slots (if they fit) instead of the in-flight target
   int64_t w_total;          // nt * B * sum_h (rp_k + rp_v)
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
