@@ -198,10 +198,39 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------------------------
+# multi-rank plumbing (one process per GPU; the path shards by sequence, so ranks never exchange data)
+# ----------------------------------------------------------------------------------------------
+
+def rank_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's time: the only collective of the benchmark (timing, not data)."""
+    if world == 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank streams its own batch shard's cache; the job's rate is the sum."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
+def rank_chunk_base(rank: int) -> int:
+    """Offset of a rank's random sub-streams, so that batch shards hold different sequences."""
+    return rank * 100000
+
+
+# ----------------------------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------
 
-def build_layer(wl, device, binding, keep_heads=()):
+def build_layer(wl, device, binding, keep_heads=(), rank=0):
     """Creates the layer and fills `context` rows through eigen_attn_append_kv.  Returns the layer, the
     bases, and for the units (0, h), h in keep_heads, the raw K/V history as float64 arrays."""
     ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
@@ -214,8 +243,9 @@ def build_layer(wl, device, binding, keep_heads=()):
     hist = {h: ([], []) for h in keep_heads}
     for ci, c in enumerate(range(0, wl.context, FILL_CHUNK)):
         t = min(FILL_CHUNK, wl.context - c)
-        k = synth.lowrank_rows(W_k, wl.batch, t, wl.sigma, wl.index, "K", chunk=ci, dtype=dt, device=device)
-        v = synth.lowrank_rows(W_v, wl.batch, t, wl.sigma, wl.index, "V", chunk=ci, dtype=dt, device=device)
+        cid = ci + rank_chunk_base(rank)
+        k = synth.lowrank_rows(W_k, wl.batch, t, wl.sigma, wl.index, "K", chunk=cid, dtype=dt, device=device)
+        v = synth.lowrank_rows(W_v, wl.batch, t, wl.sigma, wl.index, "V", chunk=cid, dtype=dt, device=device)
         lay.append_kv(k, v)
         for h in keep_heads:
             hist[h][0].append(k[0, :, h, :].double().cpu().numpy())
@@ -230,9 +260,7 @@ def build_layer(wl, device, binding, keep_heads=()):
 
 def run_ours(args, wl):
     import torch.distributed as dist
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     if world > 1:
@@ -247,7 +275,7 @@ def run_ours(args, wl):
 
     do_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     keep_heads = list(range(0, wl.n_heads, 2)) if do_cpu else []      # 16 sampled units of sequence 0
-    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep_heads)
+    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep_heads, rank=rank)
     n0 = wl.context
     assert lay.len == n0
     stream = torch.cuda.current_stream(device)
@@ -290,13 +318,10 @@ def run_ours(args, wl):
     lay.poll_status()
     ms_total = t_start.elapsed_time(t_stop)
     kern_ms = [a.elapsed_time(b) for a, b in ev]
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, device)
     ms_step = ms_total / args.steps
     bytes_step = algorithmic_bytes(wl, ranks, ranks, n0 + 1)
-    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    value = whole_job_gbs(bytes_step, world, ms_step)
     kern_avg_ms = sum(kern_ms) / len(kern_ms)
     peak, peak_src = measured_peaks()
     achieved = bytes_step / (kern_avg_ms * 1e-3) / 1e9
@@ -317,12 +342,9 @@ def run_ours(args, wl):
     e_stop.record(stream)
     sync_all()
     e2e_ms = e_start.elapsed_time(e_stop)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
     e2e_ms_step = e2e_ms / args.steps
-    e2e_value = world * bytes_step / (e2e_ms_step * 1e-3) / 1e9
+    e2e_value = whole_job_gbs(bytes_step, world, e2e_ms_step)
     io_bytes = hq.numel() * hq.element_size()
     same = bool(torch.equal(hout, out.cpu()))
 
