@@ -79,8 +79,9 @@ typedef struct {
 /* Sizes of the two device buffers the caller must provide for this layer.  Pure host arithmetic. */
 ea_status eigen_attn_cache_bytes(const ea_desc* desc, size_t* cache_bytes, size_t* workspace_bytes);
 
-/* Builds a handle: validates desc, pads and uploads the bases into the workspace (synchronises
- * `cuda_stream` before returning; desc's host arrays are not retained), sets len = 0.
+/* Builds a handle: validates desc, pads and uploads the bases into the workspace, fills the cache
+ * with zeros (rows that no call has written must hold finite values) and sets len = 0.  Synchronises
+ * `cuda_stream` before returning; desc's host arrays are not retained.
  * d_cache and d_workspace must be 256-byte aligned and stay valid for the life of the handle. */
 ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_bytes,
                             void* d_workspace, size_t workspace_bytes,

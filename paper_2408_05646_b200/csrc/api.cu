@@ -10,6 +10,8 @@
 #include <new>
 #include <vector>
 
+#include <cuda.h>   // CUtensorMap and its enums only; the encoder is resolved at run time, libcuda is not linked
+
 #include "../../include/eigen_attn.h"
 #include "internal.h"
 
@@ -40,7 +42,7 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0;
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -110,7 +112,40 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
   L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
+  L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->workspace_bytes = off;
+}
+
+// Tensor maps of the K' and V' slabs of every head for the prefill kernel's TMA loads: a 3-D view
+// {rank (inner), n_max rows, batch} of bf16, box = 64 elements x 64 rows with the 128-byte swizzle.  Elements
+// past the rank and rows past n_max read as zero.  Returns false when the driver's encoder is unavailable or
+// rejects a shape; the caller then keeps the prefill kernels that do not use TMA.
+bool encode_tensor_maps(const ea_desc* d, const Layout& L, char* cache, std::vector<CUtensorMap>* maps) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return false;
+  const EncodeFn encode = reinterpret_cast<EncodeFn>(fn);
+  maps->resize(2 * static_cast<size_t>(d->n_heads));
+  for (int h = 0; h < d->n_heads; ++h)
+    for (int which = 0; which < 2; ++which) {
+      const HeadInfo& hi = L.heads[h];
+      const cuuint64_t rp = which ? hi.rp_v : hi.rp_k;
+      const cuuint64_t dims[3] = {rp, static_cast<cuuint64_t>(d->n_max), static_cast<cuuint64_t>(d->batch)};
+      const cuuint64_t strides[2] = {rp * 2, static_cast<cuuint64_t>(d->n_max) * rp * 2};
+      const cuuint32_t box[3] = {64, 64, 1};
+      const cuuint32_t estr[3] = {1, 1, 1};
+      void* base = cache + (which ? hi.v_off : hi.k_off);
+      if (encode(&(*maps)[2 * h + which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    }
+  return true;
 }
 
 }  // namespace
@@ -122,6 +157,7 @@ struct eigen_attn {
   char* ws = nullptr;
   int32_t len = 0;
   int sm_count = 148;
+  bool tmaps_ok = false;  // the workspace holds tensor maps of the cache slabs
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
@@ -410,6 +446,16 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
     e = cudaMemcpyAsync(h->ws + L.off_heads, L.heads.data(), sizeof(HeadInfo) * H, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(h->ws + L.off_basis, basis.data(), basis.size() * sizeof(float), cudaMemcpyHostToDevice, s);
+  // Rows of the cache that no call has written yet must hold finite values: the tensor-core prefill loads
+  // whole 64-row tiles and multiplies the rows past the current length by zero weights.
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->cache, 0, L.cache_bytes, s);
+  std::vector<CUtensorMap> tmaps;
+  if (e == cudaSuccess && desc->dtype == EA_BF16 && dh % 16 == 0 &&
+      static_cast<int64_t>(desc->n_max) * L.max_rp_k * 2 < (1ll << 40) &&
+      encode_tensor_maps(desc, L, h->cache, &tmaps)) {
+    e = cudaMemcpyAsync(h->ws + L.off_tmaps, tmaps.data(), tmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s);
+    h->tmaps_ok = true;
+  }
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
@@ -558,9 +604,10 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags; p.status = dev_status(h);
+  p.tmaps = h->ws + L.off_tmaps;
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   size_t ws_smem = 0;
-  const int ws_stages = tc_attn ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
+  const int ws_stages = tc_attn && h->tmaps_ok ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
   if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 2)
     e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, s, &h->launches);   // warp-specialised, 256 query rows per CTA
   else if (tc_attn && h->opt_prefill != 1)

@@ -123,6 +123,7 @@ struct PrefillParams {
   float scale_log2;         // log2(e) / sqrt(d_head)
   uint32_t flags;
   int* status;
+  const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head (warp-specialised kernel only)
 };
 
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.

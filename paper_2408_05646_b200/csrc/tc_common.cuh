@@ -61,6 +61,23 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* statu
     }
   }
 }
+// One arrival that also announces `bytes` of asynchronous copies which will complete on the barrier.
+__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// TMA: one box of a 3-D tensor map (in global memory) at element coordinates (x, y, z) into shared memory;
+// the bytes of the whole box, zero fill included, complete on the barrier.  x * element size must be a
+// multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_3d(void* dst, const void* tmap, int x, int y, int z, void* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+      : "memory");
+}
+// Orders earlier writes of a tensor map through ordinary stores or copies before its use by TMA.
+__device__ __forceinline__ void tensormap_acquire(const void* tmap) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
+}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -152,6 +169,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return static_cast<uint64_t>((saddr >> 4) & 0x3FFFu) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16) |
          (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+// Same for the 128-byte swizzle (bits 61-63 = 2): rows of 128 bytes whose 16-byte chunks are permuted by
+// chunk ^= row % 8; tiles must start on a 1024-byte boundary.  K-major operands: SBO = stride between
+// 8-row groups, LBO unused.  MN-major operands: LBO = stride between 64-element atoms along MN, SBO =
+// stride between 8-row groups along K.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return smem_desc(saddr, lbo_bytes, sbo_bytes) | (2ull << 61);
+}
+// Byte offset of chunk c (16 bytes) of row `row` inside a 128-byte-swizzled atom column of dense rows.
+__device__ __forceinline__ uint32_t sw128_off(int row, int c) {
+  return static_cast<uint32_t>((row << 7) + ((c ^ (row & 7)) << 4));
 }
 // Instruction descriptor, kind::f16: f32 accumulator, bf16 A and B, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
