@@ -8,13 +8,15 @@
 //     stages by TMA (tensor maps of the cache slabs, 64 x 64 boxes in the 128-byte swizzled layout the
 //     MMA descriptors name; each tile is fetched once for both query tiles).  Elements past the rank
 //     and rows past the capacity arrive as zeros;
-//   * two threads feed the tensor pipe, one with the S products and one with the PV products; every
-//     group of MMAs is followed by a tcgen05.commit onto the mbarrier that its consumer waits on;
+//   * two threads feed the tensor pipe, one per query tile: PV of key tile j when the softmax group has
+//     written P(j), then S of tile j + 2 into the buffer that P(j) occupied; every group of MMAs is
+//     followed by a tcgen05.commit onto the mbarrier that its consumer waits on;
 //   * two softmax warpgroups (4 warps each, one thread per query row = one TMEM lane), one per query
-//     tile.  S is double-buffered in TMEM (2 x 64 columns per group) and P in shared memory, so the S
-//     product of key tile j + 1 runs while the group turns tile j into P; a 64-key row fits in
-//     registers, so a tile costs one TMEM round trip.
-// TMEM (512 columns): S_A[2], S_B[2] (64 columns each), O'_A, O'_B (up to 128 each).
+//     tile.  S is double-buffered in TMEM (2 x 64 columns per group), so the S product of key tile
+//     j + 1 runs while the group turns tile j into P; a 64-key row fits in registers, so a tile costs
+//     one TMEM round trip.  P (bf16) goes back into the first 32 columns of the S buffer it came from
+//     and is the A operand of the PV product straight from TMEM: it never touches shared memory.
+// TMEM (512 columns): S_A[2], S_B[2] (64 columns each, P aliased), O'_A, O'_B (up to 128 each).
 // Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -29,19 +31,18 @@ using namespace tc;
 constexpr int kKeys = 64;                     // key rows per tile
 constexpr int kAtomBytes = kKeys * 128;       // one swizzled atom column of a K'/V' tile: 64 rows x 64 elements
 constexpr int kSoftmaxWarps = 8;
-constexpr int kMmaWarp = 8;                   // issues the PV products (and the lift)
+constexpr int kMmaWarp = 8;                   // issues the MMAs of query tile A (and the lift)
 constexpr int kLoadWarp = 9;                  // lane 0 issues the TMA copies
-constexpr int kHelperWarp = 10;               // takes part in the epilogue only
-constexpr int kSIssueWarp = 11;               // issues the S products
-constexpr int kWsThreads = 12 * 32;            // 8 softmax warps, PV issuer, TMA producer, helper, S issuer
+constexpr int kMmaWarpB = 10;                 // issues the MMAs of query tile B
+constexpr int kWsThreads = 11 * 32;           // 8 softmax warps, two MMA issuers, TMA producer
 constexpr int kMaxStages = 8;
 
 struct __align__(16) WsHeader {
   unsigned long long kv_full[kMaxStages], kv_empty[kMaxStages];
   unsigned long long q_full;
-  unsigned long long s_full[2][2];            // [query tile][S buffer]: S product of a key tile complete
-  unsigned long long p_full[2][2];            // [query tile][P buffer]: P written and the S buffer consumed
-  unsigned long long o_done[2];               // [query tile]: PV product of a key tile complete
+  unsigned long long s_full[2][2];            // [query tile][buffer]: S product of a key tile complete
+  unsigned long long p_full[2][2];            // [query tile][buffer]: P written over S, O' rescaled if needed
+  unsigned long long o_done[2][2];            // [query tile][buffer]: PV product of a key tile complete (P consumed)
   unsigned long long lift_done;
   uint32_t tmem_base;
   int abort_flag;
@@ -61,6 +62,27 @@ __device__ __forceinline__ void load_q_tile_async(unsigned char* dst, const __nv
   }
 }
 
+// S = Q' K'^T for one query tile and one key tile: KS steps of 16 rank elements.  K' sits in atom columns of
+// 64 elements (8192 bytes each); a step advances 32 bytes along the swizzled rows.
+template <int KS>
+__device__ __forceinline__ void issue_s(uint32_t d_tmem, uint64_t dq, uint64_t dk, uint32_t idesc) {
+#pragma unroll
+  for (int s = 0; s < KS; ++s)
+    mma_ss(d_tmem, dq + 16 * s, dk + (s >> 2) * (kAtomBytes >> 4) + (s & 3) * 2, idesc, s > 0);
+}
+__device__ __forceinline__ void issue_s_steps(int ks, uint32_t d_tmem, uint64_t dq, uint64_t dk, uint32_t idesc) {
+  switch (ks) {
+    case 1: issue_s<1>(d_tmem, dq, dk, idesc); break;
+    case 2: issue_s<2>(d_tmem, dq, dk, idesc); break;
+    case 3: issue_s<3>(d_tmem, dq, dk, idesc); break;
+    case 4: issue_s<4>(d_tmem, dq, dk, idesc); break;
+    case 5: issue_s<5>(d_tmem, dq, dk, idesc); break;
+    case 6: issue_s<6>(d_tmem, dq, dk, idesc); break;
+    case 7: issue_s<7>(d_tmem, dq, dk, idesc); break;
+    default: issue_s<8>(d_tmem, dq, dk, idesc); break;
+  }
+}
+
 __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const PrefillParams p, int stages) {
   extern __shared__ __align__(1024) unsigned char smem[];
   WsHeader* hdr = reinterpret_cast<WsHeader*>(smem);
@@ -72,7 +94,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int t0 = qblk * 2 * kTile;
   const int rpk16 = (hd.rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
   const int nch_k = rpk16 >> 3, nch_v = rpv16 >> 3;
-  const int grp_k = nch_k << 7, grp_v = nch_v << 7, grp_p = (kKeys >> 3) << 7;
+  const int grp_k = nch_k << 7, grp_v = nch_v << 7;
   // K'/V' tiles: atom columns of 64 rank elements, each [64 keys][128 bytes] with the 128-byte swizzle
   const int q_bytes = kTile * rpk16 * 2, k_bytes = ((rpk16 + 63) >> 6) * kAtomBytes, v_bytes = ((rpv16 + 63) >> 6) * kAtomBytes;
   const int o_bytes = kTile * rpv16 * 2;                     // an O' tile of the epilogue
@@ -81,22 +103,30 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   unsigned char* tiles = smem + 1024;
   unsigned char* Qs = tiles;                                 // Q_A, Q_B
   unsigned char* ring = Qs + 2 * q_bytes;                    // stages x (K tile, V tile)
-  unsigned char* Ps = ring + stages * stage_bytes;           // P[query tile][buffer], 128 rows x 64 keys each
-  const int p_bytes = kTile * kKeys * 2;
+
+  // key tiles each query tile needs (tile B starts 128 rows later, so it needs two more in general)
+  int n_tiles[2];
+  for (int x = 0; x < 2; ++x) {
+    const int tx = t0 + x * kTile;
+    n_tiles[x] = tx < p.T ? (p.len0 + min(p.T, tx + kTile) + kKeys - 1) / kKeys : 0;
+  }
+  const int n_max_tiles = max(n_tiles[0], n_tiles[1]);
+  const int active_groups = (n_tiles[0] > 0) + (n_tiles[1] > 0);
+  const int total_rows = p.B * p.T;
 
   if (warp == 0) tmem_alloc(&hdr->tmem_base, 512);
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(&hdr->kv_full[s], 1);                        // the producer's arrival; the copies add their bytes
-      mbar_init(&hdr->kv_empty[s], 1);
+      mbar_init(&hdr->kv_empty[s], active_groups);           // one arrival per query tile that the CTA works on
     }
     mbar_init(&hdr->q_full, kSoftmaxWarps * 32);
     for (int x = 0; x < 2; ++x) {
       for (int bb = 0; bb < 2; ++bb) {
         mbar_init(&hdr->s_full[x][bb], 1);
         mbar_init(&hdr->p_full[x][bb], kTile);
+        mbar_init(&hdr->o_done[x][bb], 1);
       }
-      mbar_init(&hdr->o_done[x], 1);
     }
     mbar_init(&hdr->lift_done, 1);
     hdr->abort_flag = 0;
@@ -108,14 +138,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const uint32_t tmem = hdr->tmem_base;
   volatile int* abort_flag = &hdr->abort_flag;
 
-  // key tiles each query tile needs (tile B starts 128 rows later, so it needs two more in general)
-  int n_tiles[2];
-  for (int x = 0; x < 2; ++x) {
-    const int tx = t0 + x * kTile;
-    n_tiles[x] = tx < p.T ? (p.len0 + min(p.T, tx + kTile) + kKeys - 1) / kKeys : 0;
-  }
-  const int n_max_tiles = max(n_tiles[0], n_tiles[1]);
-  const int total_rows = p.B * p.T;
 
   if (warp == kLoadWarp) {
     // ------------------------------------------------------------------ TMA producer
@@ -152,67 +174,67 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         }
       }
     }
-  } else if (warp == kHelperWarp) {
-    // nothing to do in the main loop
-  } else if (warp == kMmaWarp || warp == kSIssueWarp) {
-    // ------------------------------------------------------------------ MMA issuers
-    // Two threads feed the tensor pipe so that their per-instruction latencies overlap.  The S thread runs up
-    // to two key tiles ahead of the softmax (one S buffer in use, one being filled); the PV thread follows
-    // the softmax.  Descriptors are built once and advanced by adding 16-byte units to their address field.
+  } else if (warp == kMmaWarp || warp == kMmaWarpB) {
+    // ------------------------------------------------------------------ MMA issuers, one per query tile
+    // Per key tile j: PV(j) once the group has written P(j); then, once PV(j) has read P out of its buffer,
+    // S(j + 2) into the same buffer.  S(0) and S(1) go out up front.  The two issuers share nothing but the
+    // tensor pipe and the ring, so neither query tile waits for the other.
     if (lane == 0) {
-      const bool pv_role = warp == kMmaWarp;
+      const int x = warp == kMmaWarpB ? 1 : 0;
+      const int nt = n_tiles[x];
       const uint32_t idesc_s = instr_desc(kKeys, false);
       const uint32_t idesc_o = instr_desc(rpv16, true);
-      const uint32_t qa = smem_u32(Qs), ra = smem_u32(ring), pa = smem_u32(Ps);
-      const uint64_t dq[2] = {smem_desc(qa, 128, grp_k), smem_desc(qa + q_bytes, 128, grp_k)};
-      const uint64_t dp0 = smem_desc(pa, 128, grp_p);                 // P buffer 0 of tile A (K-major A operand)
+      const uint32_t ra = smem_u32(ring);
+      const uint64_t dq = smem_desc(smem_u32(Qs) + x * q_bytes, 128, grp_k);
       const uint64_t dk0 = smem_desc_sw128(ra, 16, 1024);             // K tile of stage 0 (K-major B operand)
       const uint64_t dv0 = smem_desc_sw128(ra + k_bytes, kAtomBytes, 1024);   // V tile of stage 0 (MN-major B operand)
       const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
-      const uint64_t p_step = static_cast<uint64_t>(p_bytes >> 4);
       const uint64_t v_step = static_cast<uint64_t>(2048 >> 4);       // 16 keys = two 8-row groups of 1024 bytes
       const int ks_steps = rpk16 >> 4;
+      const uint32_t tSx = tmem + x * kTile, tOx = tmem + 256 + x * kTile;
       bool ok = true;
-      if (!pv_role) ok = mbar_wait(&hdr->q_full, 0, p.status);
+      if (nt > 0) ok = mbar_wait(&hdr->q_full, 0, p.status);
+      // ring position of the next S product's key tile
+      int s_stage = 0;
+      uint32_t s_parity = 0;
+      auto issue_s_tile = [&](int buf) {                     // S(tile at the ring position) into S buffer `buf`
+        ok = mbar_wait(&hdr->kv_full[s_stage], s_parity, p.status);
+        if (!ok) return;
+        tc_fence_after();
+        issue_s_steps(ks_steps, tSx + buf * kKeys, dq, dk0 + s_stage * stage_step, idesc_s);
+        mma_commit(&hdr->s_full[x][buf]);
+        if (++s_stage == stages) { s_stage = 0; s_parity ^= 1u; }
+      };
+      for (int j = 0; j < min(2, nt) && ok; ++j) issue_s_tile(j);
       int stage = 0;
-      uint32_t kv_parity = 0;                                // kv_full parity of the fill that holds tile j
-      for (int j = 0; j < n_max_tiles && ok; ++j) {
+      for (int j = 0; j < nt && ok; ++j) {
         const int buf = j & 1;
         const uint32_t buf_parity = (j >> 1) & 1u;           // phase of tile j on the barriers of its buffer
-        ok = mbar_wait(&hdr->kv_full[stage], kv_parity, p.status);   // (long complete for the PV thread)
+        ok = mbar_wait(&hdr->p_full[x][buf], buf_parity, p.status) && !*abort_flag;
         if (!ok) break;
-        for (int x = 0; x < 2 && ok; ++x) {
-          if (j >= n_tiles[x]) continue;
-          if (pv_role) {
-            ok = mbar_wait(&hdr->p_full[x][buf], buf_parity, p.status) && !*abort_flag;
-            if (!ok) break;
-            tc_fence_after();
-            uint64_t a = dp0 + (2 * x + buf) * p_step, bv = dv0 + stage * stage_step;
+        tc_fence_after();
+        const uint32_t tP = tSx + buf * kKeys;               // P: 64 bf16 per lane in 32 columns
+        const uint64_t bv = dv0 + stage * stage_step;
 #pragma unroll
-            for (int s = 0; s < kKeys / 16; ++s, a += 16, bv += v_step)   // O'_x += P_x V_j over the 64 keys
-              mma_ss(tmem + 256 + x * kTile, a, bv, idesc_o, j > 0 || s > 0);
-            mma_commit(&hdr->o_done[x]);
-          } else {
-            if (j >= 2) {                                    // the group has taken tile j - 2 out of this S buffer
-              ok = mbar_wait(&hdr->p_full[x][buf], buf_parity ^ 1u, p.status) && !*abort_flag;
-              if (!ok) break;
-            }
-            tc_fence_after();
-            uint64_t a = dq[x];
-            const uint64_t bk = dk0 + stage * stage_step;
-            for (int s = 0; s < ks_steps; ++s, a += 16)      // S_x = Q_x K_j^T over the rank, 16 elements a step:
-              mma_ss(tmem + x * kTile + buf * kKeys, a,      // atom column s / 4, 32 bytes along its rows per step
-                     bk + (s >> 2) * (kAtomBytes >> 4) + (s & 3) * 2, idesc_s, s > 0);
-            mma_commit(&hdr->s_full[x][buf]);
-          }
+        for (int s = 0; s < kKeys / 16; ++s)                 // O'_x += P_x V_j over the 64 keys
+          mma_ts(tOx, tP + 8 * s, bv + s * v_step, idesc_o, j > 0 || s > 0);
+        mma_commit(&hdr->o_done[x][buf]);
+        mma_commit(&hdr->kv_empty[stage]);                   // PV is this tile's last reader of the stage
+        if (++stage == stages) stage = 0;
+        if (j + 2 < nt) {
+          ok = mbar_wait(&hdr->o_done[x][buf], buf_parity, p.status) && !*abort_flag;
+          if (!ok) break;
+          issue_s_tile(buf);
         }
-        // the PV products are the last readers of a stage (its S products completed before the softmax ran)
-        if (ok && pv_role) mma_commit(&hdr->kv_empty[stage]);
-        if (++stage == stages) { stage = 0; kv_parity ^= 1u; }
       }
-      // the last commit's arrival must have landed before the CTA may leave
-      if (ok && pv_role)
-        ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
+      // Key tiles that only the other query tile reads still need this tile's arrival on their stage, one
+      // phase at a time: wait until the previous use of the stage is over, then arrive.
+      for (int j = nt; j < n_max_tiles && ok && nt > 0; ++j) {
+        if (j >= stages) ok = mbar_wait(&hdr->kv_empty[j % stages], ((j / stages) - 1) & 1u, p.status) && !*abort_flag;
+        if (ok) mbar_arrive(&hdr->kv_empty[j % stages]);
+      }
+      // the last commits' arrivals must have landed before the CTA may leave
+      if (ok && nt > 0) ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
       if (!ok) *abort_flag = 1;
     }
   } else {
@@ -264,31 +286,33 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         alpha = ex2(m_run - row_max);
         m_run = row_max;
       }
-      // exponentials, row sum, P as bf16 into this tile's P buffer (free: the PV product of tile j - 2 was
-      // seen complete during the previous iteration)
-      unsigned char* Px = Ps + (2 * x + buf) * p_bytes;
+      // exponentials, row sum, P as bf16 pairs over the first 32 columns of this S buffer
       float row_sum = 0.f;
       const float neg_m = -m_run;
 #pragma unroll
-      for (int g = 0; g < 8; ++g) {
-        // P is cut to bf16 by truncation with integer ops, and the row sum adds the truncated values, so
-        // numerator and denominator of the softmax use identical weights.
-        uint32_t pt[8];
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float e = ex2(fmaf(__uint_as_float(r[g * 8 + i]), p.scale_log2, neg_m));
-          if (diag && key0 + g * 8 + i > my_pos) e = 0.f;
-          pt[i] = __float_as_uint(e) & 0xffff0000u;
-          row_sum += __uint_as_float(pt[i]);
+        for (int g = 0; g < 4; ++g) {
+          // P is cut to bf16 by truncation with integer ops, and the row sum adds the truncated values, so
+          // numerator and denominator of the softmax use identical weights.
+          uint32_t pt[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int c = half * 32 + g * 8 + i;
+            float e = ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, neg_m));
+            if (diag && key0 + c > my_pos) e = 0.f;
+            pt[i] = __float_as_uint(e) & 0xffff0000u;
+            row_sum += __uint_as_float(pt[i]);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) pk[g * 4 + i] = __byte_perm(pt[2 * i], pt[2 * i + 1], 0x7632);
         }
-        uint4 w;
-        w.x = __byte_perm(pt[0], pt[1], 0x7632); w.y = __byte_perm(pt[2], pt[3], 0x7632);
-        w.z = __byte_perm(pt[4], pt[5], 0x7632); w.w = __byte_perm(pt[6], pt[7], 0x7632);
-        *reinterpret_cast<uint4*>(Px + chunk_off(row, g, grp_p)) = w;
+        tmem_st16(tS + buf * kKeys + half * 16, pk);
       }
       l_run = l_run * alpha + row_sum;
       if (j > 0) {                                           // O'_x may be touched once PV_x(j-1) is done
-        ok = mbar_wait(&hdr->o_done[x], (j - 1) & 1u, p.status);
+        ok = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);
         ok = __all_sync(0xffffffffu, ok && !*abort_flag);
         if (!ok) break;
         tc_fence_after();
@@ -308,15 +332,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
                 tmem_st16(tO + h0 + c0, *reinterpret_cast<const uint32_t(*)[16]>(&o[c0]));
               }
           }
-          tmem_wait_st();
         }
       }
-      fence_async_smem();
+      tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&hdr->p_full[x][buf]);
     }
     if (ok && n_tiles[x] > 0) {
-      ok = mbar_wait(&hdr->o_done[x], (n_tiles[x] - 1) & 1u, p.status);
+      ok = mbar_wait(&hdr->o_done[x][(n_tiles[x] - 1) & 1], ((n_tiles[x] - 1) >> 1) & 1u, p.status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
     }
@@ -434,10 +457,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
 
 }  // namespace
 
-// Stages of the K'/V' ring that fit beside the two Q tiles and the four P buffers (0 = does not fit).
+// Stages of the K'/V' ring that fit beside the two Q tiles (0 = does not fit).
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes) {
   const size_t k16 = (max_rp_k + 15) & ~15, v16 = (max_rp_v + 15) & ~15;
-  const size_t fixed = 1024 + 2 * kTile * k16 * 2 + 4 * kTile * kKeys * 2;
+  const size_t fixed = 1024 + 2 * kTile * k16 * 2;
   const size_t stage = (((k16 + 63) >> 6) + ((v16 + 63) >> 6)) * static_cast<size_t>(kAtomBytes);
   const size_t limit = 227 * 1024;
   int stages = 0;
