@@ -269,14 +269,20 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       uint32_t r[64];
       tmem_ld64(tS + buf * kKeys, r);                        // this row of the tile: one TMEM round trip
       tmem_wait_ld();
-      float row_max = -INFINITY;
+      float row_max;
       if (diag) {
+        row_max = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 64; ++i)
           if (key0 + i <= my_pos) row_max = fmaxf(row_max, __uint_as_float(r[i]));
       } else {
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains of three-input maxima
 #pragma unroll
-        for (int i = 0; i < 64; ++i) row_max = fmaxf(row_max, __uint_as_float(r[i]));
+        for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(r[i + 2 * c]), __uint_as_float(r[i + 2 * c + 1]));
+        }
+        row_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       }
       row_max *= p.scale_log2;                               // the scale is positive: max and scale commute
       // Lazy reference: the exponentials use m_run, which follows the true maximum only when that has grown
@@ -286,30 +292,29 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         alpha = ex2(m_run - row_max);
         m_run = row_max;
       }
-      // exponentials, row sum, P as bf16 pairs over the first 32 columns of this S buffer
-      float row_sum = 0.f;
+      // exponentials (two per fused multiply-add), row sum, P as bf16 pairs (round to nearest) over the first 32
+      // columns of this S buffer
+      float sum0 = 0.f, sum1 = 0.f;
       const float neg_m = -m_run;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t pk[16];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          // P is cut to bf16 by truncation with integer ops, and the row sum adds the truncated values, so
-          // numerator and denominator of the softmax use identical weights.
-          uint32_t pt[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int c = half * 32 + g * 8 + i;
-            float e = ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, neg_m));
-            if (diag && key0 + c > my_pos) e = 0.f;
-            pt[i] = __float_as_uint(e) & 0xffff0000u;
-            row_sum += __uint_as_float(pt[i]);
+        for (int i = 0; i < 16; ++i) {
+          const int c = half * 32 + 2 * i;
+          float y0, y1;
+          fma2(y0, y1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), p.scale_log2, neg_m);
+          float e0 = ex2(y0), e1 = ex2(y1);
+          if (diag) {
+            if (key0 + c > my_pos) e0 = 0.f;
+            if (key0 + c + 1 > my_pos) e1 = 0.f;
           }
-#pragma unroll
-          for (int i = 0; i < 4; ++i) pk[g * 4 + i] = __byte_perm(pt[2 * i], pt[2 * i + 1], 0x7632);
+          add2(sum0, sum1, e0, e1);
+          pk[i] = pack_bf16(e0, e1);
         }
         tmem_st16(tS + buf * kKeys + half * 16, pk);
       }
+      const float row_sum = sum0 + sum1;
       l_run = l_run * alpha + row_sum;
       if (j > 0) {                                           // O'_x may be touched once PV_x(j-1) is done
         ok = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);
