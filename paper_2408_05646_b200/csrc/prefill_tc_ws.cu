@@ -9,13 +9,15 @@
 //     MMA descriptors name; each tile is fetched once for both query tiles).  Elements past the rank
 //     and rows past the capacity arrive as zeros;
 //   * two threads feed the tensor pipe, one per query tile: PV of key tile j when the softmax group has
-//     written P(j), then S of tile j + 2 into the buffer that P(j) occupied; every group of MMAs is
+//     written P(j), then S of tile j + 3 into the buffer that P(j) occupied; every group of MMAs is
 //     followed by a tcgen05.commit onto the mbarrier that its consumer waits on;
 //   * two softmax warpgroups (4 warps each, one thread per query row = one TMEM lane), one per query
 //     tile.  S is double-buffered in TMEM (2 x 64 columns per group), so the S product of key tile
-//     j + 1 runs while the group turns tile j into P; a 64-key row fits in registers, so a tile costs
-//     one TMEM round trip.  P (bf16) goes back into the first 32 columns of the S buffer it came from
-//     and is the A operand of the PV product straight from TMEM: it never touches shared memory.
+//     j + 1 runs while the group turns tile j into P; a 64-key row fits in registers, and the row of
+//     tile j + 1 is fetched from TMEM while the exponentials of tile j run (the softmax warps take
+//     registers from the other warps for that).  P(j) (bf16) goes into the first 32 columns of the
+//     buffer that S(j + 1) has just left and is the A operand of the PV product straight from TMEM: it
+//     never touches shared memory.  A buffer thus cycles S(t) -> registers -> P(t-1) -> PV(t-1) -> S(t+2).
 // TMEM (512 columns): S_A[2], S_B[2] (64 columns each, P aliased), O'_A, O'_B (up to 128 each).
 // Every wait is bounded.
 #include <cuda_bf16.h>
@@ -34,7 +36,8 @@ constexpr int kSoftmaxWarps = 8;
 constexpr int kMmaWarp = 8;                   // issues the MMAs of query tile A (and the lift)
 constexpr int kLoadWarp = 9;                  // lane 0 issues the TMA copies
 constexpr int kMmaWarpB = 10;                 // issues the MMAs of query tile B
-constexpr int kWsThreads = 11 * 32;           // 8 softmax warps, two MMA issuers, TMA producer
+constexpr int kWsThreads = 12 * 32;           // 8 softmax warps, two MMA issuers, TMA producer, one spare warp
+constexpr int kRegsSoftmax = 224, kRegsOther = 56;   // registers per thread after the reallocation (launch: 168)
 constexpr int kMaxStages = 8;
 
 struct __align__(16) WsHeader {
@@ -60,6 +63,33 @@ __device__ __forceinline__ void load_q_tile_async(unsigned char* dst, const __nv
     const void* g = live ? static_cast<const void*>(src + static_cast<int64_t>(row) * rp + c * 8) : src;
     cp_async16(dst + chunk_off(row, c, group_stride), g, live ? 16u : 0u);
   }
+}
+
+// One row of a 64-key tile: exponentials relative to the reference `neg_m` (= -m, log2 domain), their sum,
+// and P as 32 bf16 pairs (round to nearest) in `pk`.  DIAG: keys past `my_pos` get weight zero.  TRACK: also
+// returns the row maximum of the raw scores (for the lazy reference check).
+template <bool DIAG, bool TRACK>
+__device__ __forceinline__ float exp_row(const uint32_t (&r)[64], float scale, float neg_m, int key0, int my_pos,
+                                         uint32_t (&pk)[32], float* raw_max) {
+  float sum0 = 0.f, sum1 = 0.f;
+  float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int c = 2 * i;
+    const float s0 = __uint_as_float(r[c]), s1 = __uint_as_float(r[c + 1]);
+    if (TRACK) mx[i & 3] = max3(mx[i & 3], s0, s1);
+    float y0, y1;
+    fma2(y0, y1, s0, s1, scale, neg_m);
+    float e0 = ex2(y0), e1 = ex2(y1);
+    if (DIAG) {
+      if (key0 + c > my_pos) e0 = 0.f;
+      if (key0 + c + 1 > my_pos) e1 = 0.f;
+    }
+    add2(sum0, sum1, e0, e1);
+    pk[i] = pack_bf16(e0, e1);
+  }
+  if (TRACK) *raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+  return sum0 + sum1;
 }
 
 // S = Q' K'^T for one query tile and one key tile: KS steps of 16 rank elements.  K' sits in atom columns of
@@ -139,6 +169,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   volatile int* abort_flag = &hdr->abort_flag;
 
 
+  if (warp >= kSoftmaxWarps) {
+  reg_dealloc<kRegsOther>();
   if (warp == kLoadWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -176,9 +208,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     }
   } else if (warp == kMmaWarp || warp == kMmaWarpB) {
     // ------------------------------------------------------------------ MMA issuers, one per query tile
-    // Per key tile j: PV(j) once the group has written P(j); then, once PV(j) has read P out of its buffer,
-    // S(j + 2) into the same buffer.  S(0) and S(1) go out up front.  The two issuers share nothing but the
-    // tensor pipe and the ring, so neither query tile waits for the other.
+    // Per key tile j: PV(j) once the group has written P(j) (into the buffer S(j + 1) came from); then, once
+    // PV(j) has read P out of that buffer, S(j + 3) into it.  S(0) and S(1) go out up front, S(2) when P(0)
+    // is there (the group then holds S(0) in registers).  The two issuers share nothing but the tensor pipe
+    // and the ring, so neither query tile waits for the other.
     if (lane == 0) {
       const int x = warp == kMmaWarpB ? 1 : 0;
       const int nt = n_tiles[x];
@@ -213,7 +246,11 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         ok = mbar_wait(&hdr->p_full[x][buf], buf_parity, p.status) && !*abort_flag;
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tP = tSx + buf * kKeys;               // P: 64 bf16 per lane in 32 columns
+        if (j == 0 && nt > 2) {
+          issue_s_tile(0);
+          if (!ok) break;
+        }
+        const uint32_t tP = tSx + (buf ^ 1) * kKeys;         // P: 64 bf16 per lane in 32 columns
         const uint64_t bv = dv0 + stage * stage_step;
 #pragma unroll
         for (int s = 0; s < kKeys / 16; ++s)                 // O'_x += P_x V_j over the 64 keys
@@ -221,10 +258,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         mma_commit(&hdr->o_done[x][buf]);
         mma_commit(&hdr->kv_empty[stage]);                   // PV is this tile's last reader of the stage
         if (++stage == stages) stage = 0;
-        if (j + 2 < nt) {
+        if (j + 3 < nt) {
           ok = mbar_wait(&hdr->o_done[x][buf], buf_parity, p.status) && !*abort_flag;
           if (!ok) break;
-          issue_s_tile(buf);
+          issue_s_tile(buf ^ 1);
         }
       }
       // Key tiles that only the other query tile reads still need this tile's arrival on their stage, one
@@ -237,7 +274,48 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       if (ok && nt > 0) ok = mbar_wait(&hdr->kv_empty[(n_max_tiles - 1) % stages], ((n_max_tiles - 1) / stages) & 1u, p.status);
       if (!ok) *abort_flag = 1;
     }
-  } else {
+  }
+
+  // ---- MMA and loader warps: epilogue
+  tc_fence_before();
+  __syncthreads();                                           // #1
+  const bool lowrank = (p.flags & 0x2u) != 0;
+  const bool run = !*abort_flag && !lowrank;
+  unsigned char* Uh = tiles + 4 * o_bytes;                   // lift image of U^V: [d_head][rpv16] hi, then lo
+  const int img16 = p.d_head * rpv16 * 2 / 16;               // 16-byte words per image
+  if (run) {
+    const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.uvl16_off);
+    for (int idx = tid - kMmaWarp * 32; idx < 2 * img16; idx += kWsThreads - kSoftmaxWarps * 32)
+      reinterpret_cast<uint4*>(Uh)[idx] = __ldg(Ug + idx);
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();                                           // #2
+  if (run && warp == kMmaWarp && lane == 0) {
+    tc_fence_after();
+    const uint32_t idesc_l = instr_desc(p.d_head, false);
+    const uint32_t uh = smem_u32(Uh), ul = uh + img16 * 16;
+    for (int x = 0; x < 2; ++x) {
+      if (n_tiles[x] == 0) continue;
+      const uint32_t oh = smem_u32(tiles + x * 2 * o_bytes), ol = oh + o_bytes;
+      bool acc = false;
+      for (int pass = 0; pass < 3; ++pass) {                 // hi*hi + lo*hi + hi*lo
+        const uint32_t a = pass == 1 ? ol : oh, bb = pass == 2 ? ul : uh;
+        for (int s = 0; s < rpv16 / 16; ++s) {
+          mma_ss(tmem + x * kTile, smem_desc(a + s * 256, 128, grp_v), smem_desc(bb + s * 256, 128, grp_v), idesc_l, acc);
+          acc = true;
+        }
+      }
+    }
+    mma_commit(&hdr->lift_done);
+  }
+  tc_fence_before();
+  __syncthreads();                                           // #3
+  return;
+  }
+
+  reg_alloc<kRegsSoftmax>();
+  {
     // ------------------------------------------------------------------ softmax warpgroups
     const int x = warp >> 2;                                 // 0 = tile A, 1 = tile B
     const int row = (warp & 3) * 32 + lane;
@@ -259,89 +337,94 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     }
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_tiles[x] && ok; ++j) {
+    const int nt = n_tiles[x];
+    // One key tile: `cur` holds this thread's row of S(j); the row of S(j + 1) is requested into `nxt` before
+    // the arithmetic starts and awaited before P(j) goes out over the buffer it came from.
+    auto tile = [&](const uint32_t (&cur)[64], uint32_t (&nxt)[64], int j) {
       const int key0 = j * kKeys, buf = j & 1;
-      ok = mbar_wait(&hdr->s_full[x][buf], (j >> 1) & 1u, p.status);
-      ok = __all_sync(0xffffffffu, ok && !*abort_flag);      // one decision for the whole warp
-      if (!ok) break;
-      tc_fence_after();
-      const bool diag = key0 + kKeys - 1 > p.len0 + tx;      // some (row, key) pair of the tile is masked
-      uint32_t r[64];
-      tmem_ld64(tS + buf * kKeys, r);                        // this row of the tile: one TMEM round trip
-      tmem_wait_ld();
-      float row_max;
-      if (diag) {
-        row_max = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (key0 + i <= my_pos) row_max = fmaxf(row_max, __uint_as_float(r[i]));
-      } else {
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains of three-input maxima
-#pragma unroll
-        for (int i = 0; i < 64; i += 8) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) mx[c] = max3(mx[c], __uint_as_float(r[i + 2 * c]), __uint_as_float(r[i + 2 * c + 1]));
-        }
-        row_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      const bool has_next = j + 1 < nt;
+      if (has_next) {
+        ok = mbar_wait(&hdr->s_full[x][buf ^ 1], ((j + 1) >> 1) & 1u, p.status);
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);    // one decision for the whole warp
+        if (!ok) return;
+        tc_fence_after();
+        tmem_ld64(tS + (buf ^ 1) * kKeys, nxt);
       }
-      row_max *= p.scale_log2;                               // the scale is positive: max and scale commute
+      const uint32_t tP = tS + (buf ^ 1) * kKeys;            // P(j) goes where S(j + 1) was
+      const bool diag = key0 + kKeys - 1 > p.len0 + tx;      // some (row, key) pair of the tile is masked
       // Lazy reference: the exponentials use m_run, which follows the true maximum only when that has grown
       // by more than 8 (a factor 256 that fp32 sums and bf16 P absorb); O' is rescaled only then.
-      float alpha = 1.f;
-      if (row_max > m_run + 8.f) {
-        alpha = ex2(m_run - row_max);
-        m_run = row_max;
-      }
-      // exponentials (two per fused multiply-add), row sum, P as bf16 pairs (round to nearest) over the first 32
-      // columns of this S buffer
-      float sum0 = 0.f, sum1 = 0.f;
-      const float neg_m = -m_run;
+      float alpha = 1.f, row_sum;
+      uint32_t pk[32];
+      if (j == 0 || diag) {                                  // maximum first, then the exponentials
+        float row_max = -INFINITY;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int c = half * 32 + 2 * i;
-          float y0, y1;
-          fma2(y0, y1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), p.scale_log2, neg_m);
-          float e0 = ex2(y0), e1 = ex2(y1);
-          if (diag) {
-            if (key0 + c > my_pos) e0 = 0.f;
-            if (key0 + c + 1 > my_pos) e1 = 0.f;
-          }
-          add2(sum0, sum1, e0, e1);
-          pk[i] = pack_bf16(e0, e1);
+        for (int i = 0; i < 64; ++i)
+          if (!diag || key0 + i <= my_pos) row_max = fmaxf(row_max, __uint_as_float(cur[i]));
+        row_max *= p.scale_log2;                             // the scale is positive: max and scale commute
+        if (row_max > m_run + 8.f) {
+          alpha = ex2(m_run - row_max);
+          m_run = row_max;
         }
-        tmem_st16(tS + buf * kKeys + half * 16, pk);
-      }
-      const float row_sum = sum0 + sum1;
-      l_run = l_run * alpha + row_sum;
-      if (j > 0) {                                           // O'_x may be touched once PV_x(j-1) is done
-        ok = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {         // rescale this row of O' (rare after the first tiles)
-#pragma unroll 1
-          for (int h0 = 0; h0 < rpv16; h0 += 64) {           // up to 64 columns per round trip
-            uint32_t o[64];
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 16)
-              if (h0 + c0 < rpv16) tmem_ld16(tO + h0 + c0, *reinterpret_cast<uint32_t(*)[16]>(&o[c0]));
-            tmem_wait_ld();
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 16)
-              if (h0 + c0 < rpv16) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) o[c0 + i] = __float_as_uint(__uint_as_float(o[c0 + i]) * alpha);
-                tmem_st16(tO + h0 + c0, *reinterpret_cast<const uint32_t(*)[16]>(&o[c0]));
-              }
+        row_sum = diag ? exp_row<true, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr)
+                       : exp_row<false, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr);
+      } else {                                               // exponentials against the old reference, maximum on the side
+        float raw_max;
+        row_sum = exp_row<false, true>(cur, p.scale_log2, -m_run, key0, my_pos, pk, &raw_max);
+        const float row_max = raw_max * p.scale_log2;
+        if (__any_sync(0xffffffffu, row_max > m_run + 8.f)) { // the reference moved for some row: once more
+          if (row_max > m_run + 8.f) {
+            alpha = ex2(m_run - row_max);
+            m_run = row_max;
           }
+          row_sum = exp_row<false, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr);
+        }
+      }
+      if (has_next) {
+        tmem_wait_ld();                                      // S(j + 1) is in registers: its buffer may take P(j)
+      } else if (j >= 2) {                                   // no S(j + 1) whose arrival implies it: PV_x(j-2) has read P(j-2)
+        ok = mbar_wait(&hdr->o_done[x][buf], ((j - 2) >> 1) & 1u, p.status);
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+      }
+      tmem_st16(tP, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+      tmem_st16(tP + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+      l_run = l_run * alpha + row_sum;
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale this row of O' (rare after the first tiles)
+        ok = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);   // PV_x(j-1) has added to O'
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+#pragma unroll 1
+        for (int h0 = 0; h0 < rpv16; h0 += 16) {
+          uint32_t o[16];
+          tmem_ld16(tO + h0, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+          tmem_st16(tO + h0, o);
         }
       }
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&hdr->p_full[x][buf]);
+    };
+    {
+      uint32_t ra[64], rb[64];
+      if (nt > 0) {
+        ok = mbar_wait(&hdr->s_full[x][0], 0, p.status);
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+        if (ok) {
+          tc_fence_after();
+          tmem_ld64(tS, ra);
+          tmem_wait_ld();
+        }
+      }
+      for (int j = 0; j < nt && ok; j += 2) {
+        tile(ra, rb, j);
+        if (ok && j + 1 < nt) tile(rb, ra, j + 1);
+      }
     }
     if (ok && n_tiles[x] > 0) {
       ok = mbar_wait(&hdr->o_done[x][(n_tiles[x] - 1) & 1], ((n_tiles[x] - 1) >> 1) & 1u, p.status);
@@ -420,44 +503,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     tc_fence_before();
     __syncthreads();                                         // #3
     if (warp == 0) tmem_dealloc(tmem, 512);
-    return;
   }
-
-  // ---- MMA and loader warps: epilogue
-  tc_fence_before();
-  __syncthreads();                                           // #1
-  const bool lowrank = (p.flags & 0x2u) != 0;
-  const bool run = !*abort_flag && !lowrank;
-  unsigned char* Uh = tiles + 4 * o_bytes;                   // lift image of U^V: [d_head][rpv16] hi, then lo
-  const int img16 = p.d_head * rpv16 * 2 / 16;               // 16-byte words per image
-  if (run) {
-    const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.uvl16_off);
-    for (int idx = tid - kMmaWarp * 32; idx < 2 * img16; idx += kWsThreads - kSoftmaxWarps * 32)
-      reinterpret_cast<uint4*>(Uh)[idx] = __ldg(Ug + idx);
-  }
-  fence_async_smem();
-  tc_fence_before();
-  __syncthreads();                                           // #2
-  if (run && warp == kMmaWarp && lane == 0) {
-    tc_fence_after();
-    const uint32_t idesc_l = instr_desc(p.d_head, false);
-    const uint32_t uh = smem_u32(Uh), ul = uh + img16 * 16;
-    for (int x = 0; x < 2; ++x) {
-      if (n_tiles[x] == 0) continue;
-      const uint32_t oh = smem_u32(tiles + x * 2 * o_bytes), ol = oh + o_bytes;
-      bool acc = false;
-      for (int pass = 0; pass < 3; ++pass) {                 // hi*hi + lo*hi + hi*lo
-        const uint32_t a = pass == 1 ? ol : oh, bb = pass == 2 ? ul : uh;
-        for (int s = 0; s < rpv16 / 16; ++s) {
-          mma_ss(tmem + x * kTile, smem_desc(a + s * 256, 128, grp_v), smem_desc(bb + s * 256, 128, grp_v), idesc_l, acc);
-          acc = true;
-        }
-      }
-    }
-    mma_commit(&hdr->lift_done);
-  }
-  tc_fence_before();
-  __syncthreads();                                           // #3
 }
 
 }  // namespace
@@ -469,7 +515,7 @@ int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_by
   const size_t stage = (((k16 + 63) >> 6) + ((v16 + 63) >> 6)) * static_cast<size_t>(kAtomBytes);
   const size_t limit = 227 * 1024;
   int stages = 0;
-  for (int s = kMaxStages; s >= 2; --s)
+  for (int s = kMaxStages; s >= 3; --s)   // the S products run three key tiles ahead of the PV products
     if (fixed + s * stage <= limit) { stages = s; break; }
   if (stages == 0) return 0;
   const size_t total = fixed + stages * stage;

@@ -55,6 +55,9 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* statu
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
+    // a wait that already gave up anywhere on this handle ends every other one: the launch drains in
+    // one bound, not in one bound per wait
+    if (*reinterpret_cast<volatile int*>(status) == kStatusTimeout) return false;
     if (global_ns() - t0 > kWaitBoundNs) {
       atomicExch(status, kStatusTimeout);
       return false;
@@ -151,6 +154,12 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Register reallocation between the warpgroups of a CTA: every warp of a warpgroup executes the same one.
+template <int N>
+__device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
