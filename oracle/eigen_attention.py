@@ -17,8 +17,10 @@ one head is handled.
 Parity pins (see tests): the functions here are pinned against an independent
 library routine for softmax attention applied to the d_h-wide low-rank inputs
 Q', K', V' of Eq. 6, brute-force Python loops on tiny inputs, closed-form
-special cases, and the numbers the paper prints for cache sizes.  Nothing in
-this file is "parity unpinned".
+special cases, and the numbers the paper prints for cache sizes.  The ALiBi
+bias is pinned by the same library routine given the bias as an additive
+mask, by the geometric-series closed form for a zero query, and by loops.
+Nothing in this file is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -57,21 +59,31 @@ def lift(Y: np.ndarray, U: np.ndarray) -> np.ndarray:
 # One head, stateless: the definition
 # --------------------------------------------------------------------------
 
+def alibi_bias(slope: float, pos: int, n: int) -> np.ndarray:
+    """Linear position bias of the MPT models (Section 5.1 names ALiBi as their position scheme; the
+    paper prints no formula, this is the published one): the score of the query at position `pos`
+    against key j gets -slope * (pos - j), j = 0..n-1.  The head's slope is an input."""
+    return -float(slope) * (float(pos) - np.arange(n, dtype=F64))
+
+
 def decode_head(q: np.ndarray, K: np.ndarray, V: np.ndarray,
-                U_K: np.ndarray, U_V: np.ndarray, lowrank_out: bool = False) -> np.ndarray:
+                U_K: np.ndarray, U_V: np.ndarray, lowrank_out: bool = False,
+                alibi_slope: float = 0.0) -> np.ndarray:
     """Generation-phase Eigen Attention for one head (Eq. 3 in the space of Eq. 7).
 
     q [d_h]; K, V [n, d_h] are the un-projected rows of the n cached tokens
     (the new token's row included: the cache is extended first, then attended,
     Section 2 "LLM Inference").  Returns [d_h] (or [r_V] with lowrank_out).
     The softmax scale is 1/sqrt(d_h) -- Eq. 7 keeps d_h although the vectors
-    are r wide.
+    are r wide.  With alibi_slope the query (position n-1) adds alibi_bias to the scores.
     """
     d_h = U_K.shape[0]
     qp = to_rank_space(q, U_K)                    # [r_K]
     Kp = to_rank_space(K, U_K)                    # [n, r_K]
     Vp = to_rank_space(V, U_V)                    # [n, r_V]
     s = (Kp @ qp) / math.sqrt(d_h)                # [n]
+    if alibi_slope:
+        s = s + alibi_bias(alibi_slope, Kp.shape[0] - 1, Kp.shape[0])
     p = softmax_rows(s[None, :])[0]
     o = p @ Vp                                    # [r_V]
     return o if lowrank_out else lift(o, U_V)
@@ -79,7 +91,7 @@ def decode_head(q: np.ndarray, K: np.ndarray, V: np.ndarray,
 
 def prefill_head(Q: np.ndarray, K: np.ndarray, V: np.ndarray,
                  U_K: np.ndarray, U_V: np.ndarray, len0: int = 0,
-                 lowrank_out: bool = False) -> np.ndarray:
+                 lowrank_out: bool = False, alibi_slope: float = 0.0) -> np.ndarray:
     """Causal Eigen Attention for one head over a prompt.
 
     Q [T, d_h] are the T new queries; K, V [len0+T, d_h] are all rows cached
@@ -96,6 +108,8 @@ def prefill_head(Q: np.ndarray, K: np.ndarray, V: np.ndarray,
     for t in range(T):
         n_t = len0 + t + 1
         s = (Kp[:n_t] @ Qp[t]) / math.sqrt(d_h)
+        if alibi_slope:
+            s = s + alibi_bias(alibi_slope, n_t - 1, n_t)
         p = softmax_rows(s[None, :])[0]
         O[t] = p @ Vp[:n_t]
     return O if lowrank_out else lift(O, U_V)
@@ -115,8 +129,11 @@ class LayerOracle:
 
     def __init__(self, batch: int, n_heads: int, d_head: int,
                  U_K: Sequence[np.ndarray], U_V: Sequence[np.ndarray],
-                 tracked: Optional[Sequence[Tuple[int, int]]] = None):
+                 tracked: Optional[Sequence[Tuple[int, int]]] = None,
+                 alibi_slopes: Optional[Sequence[float]] = None):
         assert len(U_K) == n_heads and len(U_V) == n_heads
+        self.alibi = [float(x) for x in alibi_slopes] if alibi_slopes is not None else [0.0] * n_heads
+        assert len(self.alibi) == n_heads
         self.B, self.H, self.d_h = batch, n_heads, d_head
         self.U_K = [np.asarray(u, dtype=F64) for u in U_K]
         self.U_V = [np.asarray(u, dtype=F64) for u in U_V]
@@ -173,6 +190,8 @@ class LayerOracle:
             qp = to_rank_space(q[b, h], self.U_K[h])
             self.projection_macs += self.d_h * qp.shape[0]
             s = (Kp @ qp) / math.sqrt(self.d_h)
+            if self.alibi[h]:
+                s = s + alibi_bias(self.alibi[h], self.len - 1, self.len)
             p = softmax_rows(s[None, :])[0]
             o = p @ Vp
             self.attention_macs += Kp.size + Vp.size
@@ -206,6 +225,8 @@ class LayerOracle:
             for t in range(T):
                 n_t = len0 + t + 1
                 s = (Kp[:n_t] @ Qp[t]) / math.sqrt(self.d_h)
+                if self.alibi[h]:
+                    s = s + alibi_bias(self.alibi[h], n_t - 1, n_t)
                 p = softmax_rows(s[None, :])[0]
                 O[t] = p @ Vp[:n_t]
             out[(b, h)] = lift(O, self.U_V[h])

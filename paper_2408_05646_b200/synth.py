@@ -141,6 +141,17 @@ def gaussian_query(batch: int, n_heads: int, d_head: int, scale: float, config: 
     return q.to(dtype).contiguous()
 
 
+def alibi_slopes(n_heads: int) -> List[float]:
+    """Per-head ALiBi slopes as published for a power-of-two head count: 2^(-8 (h+1) / H), h = 0..H-1;
+    other head counts take the slopes of the next power of two, the even ones first then the odd ones."""
+    def pow2(n):
+        return [2.0 ** (-8.0 * (i + 1) / n) for i in range(n)]
+    if n_heads & (n_heads - 1) == 0:
+        return pow2(n_heads)
+    lower = 1 << (n_heads.bit_length() - 1)
+    return pow2(lower) + pow2(2 * lower)[0::2][: n_heads - lower]
+
+
 def sample_units(batch: int, n_heads: int, ranks: Sequence[int], count: int, config: int):
     """Seeded subset of (b, h) units: always the two corners, every distinct rank and every batch index."""
     rng = np.random.default_rng(stream_seed(config, "subset"))
