@@ -130,8 +130,12 @@ class LayerOracle:
     def __init__(self, batch: int, n_heads: int, d_head: int,
                  U_K: Sequence[np.ndarray], U_V: Sequence[np.ndarray],
                  tracked: Optional[Sequence[Tuple[int, int]]] = None,
-                 alibi_slopes: Optional[Sequence[float]] = None):
+                 alibi_slopes: Optional[Sequence[float]] = None,
+                 storage=None):
+        """`storage`, if given, maps an array of freshly projected rows to what the cache keeps of them
+        (e.g. rounding to the 16-bit format of Section 2, p = 16); None keeps fp64."""
         assert len(U_K) == n_heads and len(U_V) == n_heads
+        self.storage = storage
         self.alibi = [float(x) for x in alibi_slopes] if alibi_slopes is not None else [0.0] * n_heads
         assert len(self.alibi) == n_heads
         self.B, self.H, self.d_h = batch, n_heads, d_head
@@ -158,6 +162,8 @@ class LayerOracle:
         for (b, h) in self.units:
             kp = to_rank_space(k[b, :, h, :], self.U_K[h])
             vp = to_rank_space(v[b, :, h, :], self.U_V[h])
+            if self.storage is not None:
+                kp, vp = self.storage(kp), self.storage(vp)
             self.Kp[(b, h)] = np.concatenate([self.Kp[(b, h)], kp], axis=0)
             self.Vp[(b, h)] = np.concatenate([self.Vp[(b, h)], vp], axis=0)
             self.cache_elements += kp.size + vp.size
@@ -170,6 +176,8 @@ class LayerOracle:
         b, h = unit
         kp = to_rank_space(k_rows, self.U_K[h])
         vp = to_rank_space(v_rows, self.U_V[h])
+        if self.storage is not None:
+            kp, vp = self.storage(kp), self.storage(vp)
         self.Kp[unit] = np.concatenate([self.Kp[unit], kp], axis=0)
         self.Vp[unit] = np.concatenate([self.Vp[unit], vp], axis=0)
         self.cache_elements += kp.size + vp.size

@@ -231,7 +231,10 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   float m = -INFINITY, l = 0.f;
 
   // score of one cached row against q', online-softmax update, weighted accumulation of its value row
-  auto process_row = [&](const unsigned char* kr, const unsigned char* vr, bool valid) {
+  // ALiBi: the query sits at position n_total - 1; row j gets slope * (j - (n_total - 1)) <= 0 (log2 domain)
+  const float slope2 = hd.alibi_slope2;
+  const int pos_q = p.n - 1 + (p.k_new != nullptr ? 1 : 0);
+  auto process_row = [&](const unsigned char* kr, const unsigned char* vr, bool valid, int j_abs) {
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
     for (int j = 0; j < NCH; ++j) {
@@ -245,6 +248,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     }
     float s = (a0 + a1) + (a2 + a3);
     s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s = fmaf(slope2, static_cast<float>(j_abs - pos_q), s);
     if (valid) {
       if (s > m) {                      // rare after the first rows: rescale the running state
         const float c = fast_exp2(m - s);
@@ -286,7 +290,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     for (int rbase = warp * 16; rbase < rows; rbase += kDecodeConsumerWarps * 16) {
       const bool valid = rbase + pair < rows;
       const int row = valid ? rbase + pair : rbase;
-      process_row(kt + row * rowb_k, vt + row * rowb_v, valid);
+      process_row(kt + row * rowb_k, vt + row * rowb_v, valid, i * p.tile_rows + row);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&fx->empty[stage]);
@@ -294,7 +298,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
 
   // the new token's row (already projected, in shared memory) is attended by one lane pair
   if (with_new_row && warp == 0 && !__any_sync(0xffffffffu, *abort_flag != 0))
-    process_row(fx->new_k, fx->new_v, pair == 0);
+    process_row(fx->new_k, fx->new_v, pair == 0, pos_q);
 
   // ---- merge the 128 lane pairs of the CTA into one partial
   float wm = m;
@@ -540,8 +544,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
               rg.filled &= ~(1u << s2);
             }
           if (!ok) { *abort_flag = 1; break; }
-          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb; rg.v_off = voff;
+          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb;
         }
+        rg.v_off = voff;                  // two heads can share the slot size and still split it differently
         const uint32_t rowb_k = hd.rp_k * sizeof(T), rowb_v = hd.rp_v * sizeof(T);
         const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i0) * p.tile_rows;
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
@@ -598,8 +603,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         int sb, voff, nst;
         ring_geometry<T>(p, hd, &sb, &voff, &nst);
         if (sb != rg.stage_bytes || nst != rg.stages) {      // same decision as the producer's
-          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb; rg.v_off = voff;
+          rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb;
         }
+        rg.v_off = voff;
       }
       const bool whole = i0 == 0 && i1 == p.nt;
       const bool with_new_row = p.k_new != nullptr && i1 == p.nt;

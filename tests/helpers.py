@@ -44,9 +44,19 @@ def make_case(B, H, d_head, ranks_k, ranks_v, n, dtype, seed_cfg=90, rho=16, sig
     return U_k, U_v, q, k, v
 
 
-def oracle_layer(B, H, d_head, U_k, U_v, tracked=None):
-    return orc.LayerOracle(B, H, d_head, U_k, U_v, tracked)
+def oracle_layer(B, H, d_head, U_k, U_v, tracked=None, alibi_slopes=None, storage=None):
+    return orc.LayerOracle(B, H, d_head, U_k, U_v, tracked, alibi_slopes=alibi_slopes, storage=storage)
 
 
 def to_np(x: torch.Tensor) -> np.ndarray:
     return x.detach().double().cpu().numpy()
+
+
+def storage_model(dtype: torch.dtype):
+    """The 16-bit KV cache the paper assumes (Section 2: p = 16) as a rounding of freshly projected rows, for
+    oracle layers in tests where few rows carry the softmax (a steep position bias): the rounding of those
+    rows is then not averaged out and exceeds the tolerance the long-context workloads state, although both
+    sides compute the same thing."""
+    if dtype == torch.float32:
+        return None
+    return lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dtype).double().numpy()

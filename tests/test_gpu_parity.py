@@ -366,3 +366,25 @@ def test_errors_leave_state_unchanged(B):
         B.EigenAttnLayer(B_, H, d, 8, BF16, bad, U_v, check_orthonormal=True)
     assert e.value.status == B.EA_ERR_NOT_ORTHONORMAL
     lay.poll_status()
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_peaked_attention_over_heads_that_share_a_slot_size(B, dtype):
+    """Heads whose K' and V' widths differ but add up to the same row size, streamed by the same CTA one after
+    the other, with sharply peaked weights: an error in a handful of rows (a stale tile layout, a ragged tail)
+    shows up here, whereas diffuse weights average it away."""
+    B_, H, d, n = 2, 6, 128, 1037
+    rk, rv = [48, 64, 80, 96, 64, 48], [96, 80, 64, 48, 80, 96]        # every head: 144 columns per row
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, dtype, seed_cfg=141, q_scale=6.0)
+    from helpers import storage_model
+    lay = B.EigenAttnLayer(B_, H, d, n, dtype, U_k, U_v)
+    lay.append_kv(k, v)
+    ref = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(dtype))
+    ref.append_kv(to_np(k), to_np(v))
+    expect = ref.decode_dense(to_np(q))
+    tol = dict(fp32_rel=2e-4) if dtype == FP32 else {}               # scores of a few tens: see the adversarial test
+    for ctas, fused in ((0, 1), (1, 1), (2, 0), (5, 1), (12, 1), (37, 0), (148, 1)):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        lay.set_option(B.EA_OPT_DECODE_FUSED, fused)
+        assert_close(lay.decode(q), expect, dtype, f"ctas={ctas} fused={fused}", **tol)
+    lay.poll_status()

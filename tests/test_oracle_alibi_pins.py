@@ -109,3 +109,25 @@ def test_published_slopes():
     assert abs(s32[0] - 2.0 ** -0.25) < 1e-15 and abs(s32[-1] - 2.0 ** -8) < 1e-15
     s12 = synth.alibi_slopes(12)
     assert len(s12) == 12 and s12[:8] == s8 and s12[8:] == [2.0 ** -0.5, 2.0 ** -1.5, 2.0 ** -2.5, 2.0 ** -3.5]
+
+
+def test_storage_hook_rounds_only_the_cached_rows():
+    B, H, d_h, T = 1, 2, 16, 6
+    rng = np.random.default_rng(9)
+    U = [synth.orthonormal_basis(d_h, 8, 40 + h) for h in range(H)]
+    k, v, q = (rng.standard_normal((B, T, H, d_h)) for _ in range(3))
+    to_bf16 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).double().numpy()
+    plain = orc.LayerOracle(B, H, d_h, U, U)
+    same = orc.LayerOracle(B, H, d_h, U, U, storage=lambda a: a)
+    rounded = orc.LayerOracle(B, H, d_h, U, U, storage=to_bf16)
+    for lay in (plain, same, rounded):
+        lay.append_kv(k, v)
+    assert np.array_equal(plain.decode_dense(q[:, -1:]), same.decode_dense(q[:, -1:]))
+    for u in rounded.units:
+        assert np.array_equal(rounded.Kp[u], to_bf16(plain.Kp[u])) and np.array_equal(rounded.Vp[u], to_bf16(plain.Vp[u]))
+    # attention over the rounded rows equals the per-head definition given rows that are exact in the basis
+    b, h = 0, 1
+    K_exact = rounded.Kp[(b, h)] @ U[h].T           # rows whose coordinates are the stored ones
+    V_exact = rounded.Vp[(b, h)] @ U[h].T
+    ref = orc.decode_head(q[b, -1, h], K_exact, V_exact, U[h], U[h])
+    assert np.abs(rounded.decode_dense(q[:, -1:])[b, 0, h] - ref).max() < 1e-12
