@@ -111,6 +111,13 @@ class ClockSampler:
 # the CPU oracle leg (also the --impl reference arm)
 # ----------------------------------------------------------------------------------------------
 
+VARIANT = {"alibi": False}   # --alibi: per-head ALiBi slopes on both sides (decode workloads)
+
+
+def variant_slopes(wl):
+    return synth.alibi_slopes(wl.n_heads) if VARIANT["alibi"] else None
+
+
 def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -125,7 +132,7 @@ def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, sample_heads, history=No
     `history` maps h -> (k_rows, v_rows) [n, d_head] float64; if None it is drawn on the CPU."""
     from oracle import eigen_attention as orc
     units = [(0, h) for h in sample_heads]
-    lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units)
+    lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units, alibi_slopes=variant_slopes(wl))
     if history is None:
         W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
         W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
@@ -238,6 +245,8 @@ def build_layer(wl, device, binding, keep_heads=(), rank=0):
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
     dt = synth.torch_dtype(wl.dtype)
     lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + 1, dt, U_k, U_v, device=device)
+    if VARIANT["alibi"]:
+        lay.set_alibi(variant_slopes(wl))
     W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K", device=device)
     W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V", device=device)
     hist = {h: ([], []) for h in keep_heads}
@@ -381,7 +390,7 @@ def run_ours(args, wl):
         "dtype": "bf16 storage, f32 accumulate" if wl.dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": wl.name, "batch_per_gpu": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
-                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1,
+                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "alibi": VARIANT["alibi"],
                    "cache_gb_per_gpu": bytes_step / 1e9, "parallelism": f"{world} independent batch shard(s)",
                    "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
         "frac_of_nominal_8TBs": value / world / 8000.0,
@@ -535,11 +544,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--alibi", action="store_true", help="decode workloads: add the per-head ALiBi position bias")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")
     args = ap.parse_args()
+    VARIANT["alibi"] = bool(args.alibi)
     if args.warmup < 3:
         args.warmup = 3
     wl = synth.WORKLOADS[args.workload]

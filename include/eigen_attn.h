@@ -144,6 +144,15 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                              int64_t out_stride_b, int64_t out_stride_t,
                              uint32_t flags, void* cuda_stream);
 
+/* Section 5.1 (MPT models use ALiBi; the paper prints no formula, this is the published bias): from the
+ * next call on, the score of the query at position pos against cached row j of head i gets
+ * -slopes[i] * (pos - j) before the softmax, pos = len - 1 in a decode call (after the new row is
+ * appended) and len0 + t for prompt token t.  slopes: HOST [H], each finite and >= 0; NULL or all
+ * zeros switches the bias off (the default).  Copies into the workspace and synchronises `cuda_stream`;
+ * calls still in flight on other streams must have finished.  With a bias the prefill runs on the
+ * single-tile tensor-core kernel (bf16) or the CUDA-core kernel, not the warp-specialised one. */
+ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream);
+
 /* Current number of cached rows; set_len truncates or rewinds (0 <= len <= n_max), e.g. to re-run
  * a step at a fixed context length.  Rows beyond the previous length hold whatever was last written. */
 ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len);

@@ -65,6 +65,7 @@ SYMBOLS = {
     "eigen_attn_cache_layout": (_i32, [_vp, _i32, ctypes.POINTER(_sz), ctypes.POINTER(_sz),
                                        ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "eigen_attn_set_option": (_i32, [_vp, _i32, _i64]),
+    "eigen_attn_set_alibi": (_i32, [_vp, ctypes.POINTER(ctypes.c_float), _vp]),
     "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
     "eigen_attn_version": (_i32, []),
@@ -294,6 +295,15 @@ class EigenAttnLayer:
 
     def poll_status(self, stream=None) -> None:
         self._check(lib.eigen_attn_poll_status(self.handle, _stream_ptr(stream)), "eigen_attn_poll_status")
+
+    def set_alibi(self, slopes, stream=None) -> None:
+        """Per-head ALiBi slopes (host floats, one per head); None switches the bias off."""
+        if slopes is None:
+            arr = None
+        else:
+            assert len(slopes) == self.H
+            arr = (ctypes.c_float * self.H)(*[float(x) for x in slopes])
+        self._check(lib.eigen_attn_set_alibi(self.handle, arr, _stream_ptr(stream)), "eigen_attn_set_alibi")
 
     def set_option(self, option: int, value: int) -> None:
         self._check(lib.eigen_attn_set_option(self.handle, option, int(value)), "eigen_attn_set_option")

@@ -158,6 +158,7 @@ struct eigen_attn {
   int32_t len = 0;
   int sm_count = 148;
   bool tmaps_ok = false;  // the workspace holds tensor maps of the cache slabs
+  bool alibi = false;     // some head has a non-zero ALiBi slope
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
@@ -608,7 +609,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   size_t ws_smem = 0;
   const int ws_stages = tc_attn && h->tmaps_ok ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
-  if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 2)
+  if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 2 && !h->alibi)
     e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, s, &h->launches);   // warp-specialised, 256 query rows per CTA
   else if (tc_attn && h->opt_prefill != 1)
     e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);  // single query tile per CTA (wide ranks)
@@ -673,6 +674,24 @@ ea_status eigen_attn_cache_layout(eigen_attn_t h, int32_t head, size_t* k_offset
   *v_offset = static_cast<size_t>(hi.v_off);
   *rp_k = hi.rp_k;
   *rp_v = hi.rp_v;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  const int H = h->desc.n_heads;
+  bool any = false;
+  for (int i = 0; i < H; ++i) {
+    const float sl = slopes ? slopes[i] : 0.f;
+    if (!(sl >= 0.f) || !isfinite(sl)) return fail(h, EA_ERR_INVALID_ARG, "set_alibi: slope[%d] = %g", i, sl);
+    h->L.heads[i].alibi_slope2 = static_cast<float>(static_cast<double>(sl) * 1.4426950408889634);
+    any = any || sl != 0.f;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_heads, h->L.heads.data(), sizeof(HeadInfo) * H, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "set_alibi");
+  h->alibi = any;
   return EA_OK;
 }
 

@@ -21,7 +21,8 @@ struct HeadInfo {
   int32_t ukt16_off;  // float offset of the tensor-core image of (U^K)^T: bf16 high part then low part, each
   int32_t uvt16_off;  //   [rp16][d_head] in the canonical core-matrix order (rp16 = rank padded to 16); same for U^V
   int32_t uvl16_off;  // float offset of the lift image of U^V: bf16 high then low part, each [d_head][rv16] canonical
-  int32_t pad_[2];
+  float alibi_slope2;  // ALiBi slope of the head times log2(e); 0 = no position bias
+  int32_t pad_;
 };
 
 constexpr int kDecodeConsumerWarps = 8;

@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(kThreads) prefill_simt_kernel(const PrefillPar
       float s = s0 + s1;
       s += __shfl_xor_sync(0xffffffffu, s, 1);
       s += __shfl_xor_sync(0xffffffffu, s, 2);
+      s = fmaf(hd.alibi_slope2, static_cast<float>(j0 + j - my_last), s);   // ALiBi: slope * (key - query position)
       if (live && j0 + j <= my_last) {
         if (s > m) {
           const float c0 = ex2(m - s);

@@ -68,6 +68,7 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
   load_tile(Qs, Qg, hd.rp_k, q_valid, nch_k, tid);
 
   const int my_pos = p.len0 + t0 + tid;                      // last key this thread's query sees
+  const float slope2 = hd.alibi_slope2;                      // ALiBi: slope * (key - query position), log2 domain
   const int n_keys = p.len0 + min(p.T, t0 + kTile);          // keys the block needs
   const int n_tiles = (n_keys + kTile - 1) / kTile;
   const uint32_t idesc_s = instr_desc(kTile, false);
@@ -105,7 +106,7 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
       tmem_wait_ld();
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float s = __uint_as_float(r[i]) * p.scale_log2;
+        float s = fmaf(__uint_as_float(r[i]), p.scale_log2, slope2 * static_cast<float>(key0 + c0 + i - my_pos));
         if (diag && key0 + c0 + i > my_pos) s = -INFINITY;
         row_max = fmaxf(row_max, s);
       }
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
       float pr[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        float s = __uint_as_float(r[i]) * p.scale_log2 - m_new;
+        float s = fmaf(__uint_as_float(r[i]), p.scale_log2, slope2 * static_cast<float>(key0 + c0 + i - my_pos)) - m_new;
         if (diag && key0 + c0 + i > my_pos) s = -INFINITY;
         pr[i] = ex2(s);
         row_sum += pr[i];
