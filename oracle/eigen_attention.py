@@ -20,6 +20,9 @@ Q', K', V' of Eq. 6, brute-force Python loops on tiny inputs, closed-form
 special cases, and the numbers the paper prints for cache sizes.  The ALiBi
 bias is pinned by the same library routine given the bias as an additive
 mask, by the geometric-series closed form for a zero query, and by loops.
+The RoPE variant (Section 4.3) is pinned by library attention on keys and
+queries rotated with complex arithmetic, by its relative-position invariance,
+by the zero-angle special case and by loops.
 Nothing in this file is "parity unpinned".
 """
 from __future__ import annotations
@@ -116,6 +119,54 @@ def prefill_head(Q: np.ndarray, K: np.ndarray, V: np.ndarray,
 
 
 # --------------------------------------------------------------------------
+# Section 4.3: Eigen Attention for models with rotary position embedding
+# --------------------------------------------------------------------------
+
+def rope_rotate(x: np.ndarray, pos, base: float = 10000.0, interleaved: bool = False) -> np.ndarray:
+    """x R for the row(s) x [..., d_h] at position(s) `pos` (Section 4.3, first equation): coordinate
+    pair i is turned by the angle pos * base^(-2i/d_h).  Pairs are (i, i + d_h/2) as in the Llama models the
+    paper evaluates, or (2i, 2i+1) with interleaved=True (the original RoPE layout).  Built as an explicit
+    block rotation: y_a = x_a cos - x_b sin, y_b = x_a sin + x_b cos."""
+    x = np.asarray(x, dtype=F64)
+    d = x.shape[-1]
+    half = d // 2
+    pos = np.asarray(pos, dtype=F64)
+    ang = pos[..., None] * (float(base) ** (-2.0 * np.arange(half, dtype=F64) / d))   # [..., half]
+    c, s_ = np.cos(ang), np.sin(ang)
+    if interleaved:
+        a, b = x[..., 0::2], x[..., 1::2]
+    else:
+        a, b = x[..., :half], x[..., half:]
+    ya, yb = a * c - b * s_, a * s_ + b * c
+    y = np.empty_like(x)
+    if interleaved:
+        y[..., 0::2], y[..., 1::2] = ya, yb
+    else:
+        y[..., :half], y[..., half:] = ya, yb
+    return y
+
+
+def decode_head_rope(q: np.ndarray, Kp: np.ndarray, Vp: np.ndarray, U_K: np.ndarray, U_V: np.ndarray,
+                     base: float = 10000.0, interleaved: bool = False, pos0: int = 0,
+                     lowrank_out: bool = False) -> np.ndarray:
+    """Generation-phase Eigen Attention with RoPE for one head (Section 4.3, second equation, Fig. 6b).
+
+    The query stays full rank.  The cache holds the low-dimensional keys Kp [n, r_K] (= K U^K of the
+    un-rotated keys); each is taken back to d_h dimensions through (U^K)^T, rotated by its own position, and
+    dotted with the rotated query.  Row j sits at position pos0 + j, the query at the last row's position.
+    The value side is Eq. 7 unchanged.  q [d_h]; Vp [n, r_V]."""
+    d_h = U_K.shape[0]
+    n = Kp.shape[0]
+    K_back = lift(Kp, U_K)                                         # [n, d_h]
+    K_pos = rope_rotate(K_back, pos0 + np.arange(n), base, interleaved)
+    q_pos = rope_rotate(np.asarray(q, dtype=F64), pos0 + n - 1, base, interleaved)
+    s = (K_pos @ q_pos) / math.sqrt(d_h)
+    p = softmax_rows(s[None, :])[0]
+    o = p @ np.asarray(Vp, dtype=F64)
+    return o if lowrank_out else lift(o, U_V)
+
+
+# --------------------------------------------------------------------------
 # One decoder layer with a rank-r KV cache (stateful, mirrors the library calls)
 # --------------------------------------------------------------------------
 
@@ -131,11 +182,12 @@ class LayerOracle:
                  U_K: Sequence[np.ndarray], U_V: Sequence[np.ndarray],
                  tracked: Optional[Sequence[Tuple[int, int]]] = None,
                  alibi_slopes: Optional[Sequence[float]] = None,
-                 storage=None):
+                 storage=None, rope: Optional[dict] = None):
         """`storage`, if given, maps an array of freshly projected rows to what the cache keeps of them
         (e.g. rounding to the 16-bit format of Section 2, p = 16); None keeps fp64."""
         assert len(U_K) == n_heads and len(U_V) == n_heads
         self.storage = storage
+        self.rope = rope          # None, or {"base": float, "interleaved": bool}: decode() follows Section 4.3
         self.alibi = [float(x) for x in alibi_slopes] if alibi_slopes is not None else [0.0] * n_heads
         assert len(self.alibi) == n_heads
         self.B, self.H, self.d_h = batch, n_heads, d_head
@@ -195,6 +247,14 @@ class LayerOracle:
         for (b, h) in self.units:
             Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]
             assert Kp.shape[0] == self.len and self.len > 0
+            if self.rope is not None:
+                assert not self.alibi[h]
+                o = decode_head_rope(q[b, h], Kp, Vp, self.U_K[h], self.U_V[h], self.rope["base"],
+                                     self.rope.get("interleaved", False), 0, lowrank_out)
+                self.projection_macs += self.d_h * (Kp.size + (0 if lowrank_out else o.shape[0]))
+                self.attention_macs += self.d_h * Kp.shape[0] + Vp.size
+                out[(b, h)] = o
+                continue
             qp = to_rank_space(q[b, h], self.U_K[h])
             self.projection_macs += self.d_h * qp.shape[0]
             s = (Kp @ qp) / math.sqrt(self.d_h)
@@ -222,6 +282,7 @@ class LayerOracle:
     def prefill(self, q: np.ndarray, k: np.ndarray, v: np.ndarray) -> dict:
         """q, k, v: [B, T, H, d_h].  Returns {(b,h): out[T, d_h]}."""
         q = np.asarray(q, dtype=F64)
+        assert self.rope is None, "the RoPE variant is built for the generation phase only"
         len0 = self.len
         self.append_kv(k, v)
         T = q.shape[1]
