@@ -153,6 +153,18 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
  * single-tile tensor-core kernel (bf16) or the CUDA-core kernel, not the warp-specialised one. */
 ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream);
 
+/* Section 4.3 + Fig. 6(b) (models with rotary position embedding): from the next call on, decode keeps the
+ * query full rank, takes every cached low-dimensional key back to d_head dimensions through (U^K)^T, rotates
+ * it by its position (row j of the cache = position j) and the query by position len - 1, and scores them
+ * with 1/sqrt(d_head); the value side is unchanged.  Pair i is turned by pos * base^(-2i/d_head); pairs are
+ * (i, i + d_head/2), or (2i, 2i+1) with interleaved != 0.  d_q must then be the un-rotated [B][1][H][d_head]
+ * query (EA_Q_PREPROJECTED is rejected) and the cache must hold projections of un-rotated keys, as
+ * eigen_attn_append_kv writes them.  The paper shares one U^K among the heads of a layer; here that is the
+ * special case of equal U_k[h].  base == 0 switches back.  bf16 layers with d_head % 16 == 0 only
+ * (EA_ERR_UNSUPPORTED otherwise); eigen_attn_prefill and eigen_attn_decode_static do not take part: they
+ * return EA_ERR_UNSUPPORTED while a rotary embedding is set.  Synchronises `cuda_stream`. */
+ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, void* cuda_stream);
+
 /* Current number of cached rows; set_len truncates or rewinds (0 <= len <= n_max), e.g. to re-run
  * a step at a fixed context length.  Rows beyond the previous length hold whatever was last written. */
 ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len);

@@ -66,6 +66,7 @@ SYMBOLS = {
                                        ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "eigen_attn_set_option": (_i32, [_vp, _i32, _i64]),
     "eigen_attn_set_alibi": (_i32, [_vp, ctypes.POINTER(ctypes.c_float), _vp]),
+    "eigen_attn_set_rope": (_i32, [_vp, ctypes.c_double, _i32, _vp]),
     "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
     "eigen_attn_version": (_i32, []),
@@ -304,6 +305,11 @@ class EigenAttnLayer:
             assert len(slopes) == self.H
             arr = (ctypes.c_float * self.H)(*[float(x) for x in slopes])
         self._check(lib.eigen_attn_set_alibi(self.handle, arr, _stream_ptr(stream)), "eigen_attn_set_alibi")
+
+    def set_rope(self, base: float, interleaved: bool = False, stream=None) -> None:
+        """Rotary position embedding for decode (Section 4.3); base 0 switches it off."""
+        self._check(lib.eigen_attn_set_rope(self.handle, float(base), int(bool(interleaved)), _stream_ptr(stream)),
+                    "eigen_attn_set_rope")
 
     def set_option(self, option: int, value: int) -> None:
         self._check(lib.eigen_attn_set_option(self.handle, option, int(value)), "eigen_attn_set_option")

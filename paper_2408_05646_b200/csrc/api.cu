@@ -42,7 +42,7 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0;
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -90,6 +90,7 @@ void make_layout(const ea_desc* d, Layout* L) {
       hi.ukt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_k + 15) & ~15) * dh;
       hi.uvt16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_v + 15) & ~15) * dh;
       hi.uvl16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_v + 15) & ~15) * dh;
+      hi.ukl16_off = static_cast<int32_t>(basis); basis += static_cast<size_t>((hi.rp_k + 15) & ~15) * dh;
     }
     hi.lr_k_off = lk; lk += hi.rp_k;
     hi.lr_v_off = lv; lv += hi.rp_v;
@@ -112,6 +113,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
   L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
+  L->off_rope = off;     off = align_up(off + 64 * sizeof(double));   // inverse frequencies of the rotary embedding
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->workspace_bytes = off;
 }
@@ -159,6 +161,8 @@ struct eigen_attn {
   int sm_count = 148;
   bool tmaps_ok = false;  // the workspace holds tensor maps of the cache slabs
   bool alibi = false;     // some head has a non-zero ALiBi slope
+  bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
+  int rope_interleaved = 0;
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
@@ -299,8 +303,51 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
   return EA_OK;
 }
 
+// Section 4.3: decode for a layer with rotary position embedding.  Row j of the cache sits at position j, the
+// query at position len - 1.
+ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
+                         uint32_t flags, cudaStream_t s) {
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
+  if (flags & ~EA_OUT_LOWRANK)
+    return fail(h, EA_ERR_INVALID_ARG, "decode with rotary embedding: flag 0x%x (the query must be full rank)", flags);
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
+  const Layout& L = h->L;
+  const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
+  const size_t smem = ea::decode_rope_smem_bytes(L.max_rp_k, L.max_rp_v, h->desc.d_head);
+  if (smem > static_cast<size_t>(kSmemLimit)) return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: tiles do not fit");
+  ea::RopeDecodeParams p{};
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
+  p.q = d_q; p.q_stride_b = stride_b;
+  p.out = d_out; p.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
+  p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
+  p.status = dev_status(h);
+  p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+  p.part_stride = L.part_stride;
+  p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
+  p.nt = (n + 127) / 128;
+  // CTAs per unit: fill the machine a few times over, within the partials the workspace holds
+  const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
+  const int64_t want = (h->opt_ctas > 0 ? h->opt_ctas : 3ll * h->sm_count * ctas_per_sm);
+  int64_t splits = (want + static_cast<int64_t>(B) * H - 1) / (static_cast<int64_t>(B) * H);
+  const int64_t cap = (static_cast<int64_t>(B) * H + kMaxDecodeCtas) / (static_cast<int64_t>(B) * H);
+  if (splits > cap) splits = cap;
+  if (splits > p.nt) splits = p.nt;
+  if (splits < 1) splits = 1;
+  if (splits > 65535) splits = 65535;
+  p.splits = static_cast<int32_t>(splits);
+  p.interleaved = h->rope_interleaved;
+  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  p.flags = flags;
+  if (h->ev_start) cudaEventRecord(h->ev_start, s);
+  const cudaError_t e = ea::launch_decode_rope(p, smem, s, &h->launches);
+  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode launch (rotary embedding)");
+  return EA_OK;
+}
+
 ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
                     uint32_t flags, cudaStream_t s) {
+  if (h->rope) return do_decode_rope(h, d_q, stride_b, d_out, stride_b_out, flags, s);
   DecodePlan plan;
   const ea_status st = plan_decode(h, "decode", d_q, stride_b, d_out, stride_b_out, flags,
                                    reinterpret_cast<float*>(h->ws + h->L.off_partials), nullptr, nullptr, 0,
@@ -314,7 +361,7 @@ ea_status do_decode(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_o
 // decomposition is over cached rows); otherwise, or with fusion switched off, append then decode.
 ea_status do_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q, const void* d_k, const void* d_v,
                   int64_t stride_b_kv, void* d_out, int64_t stride_b_out, uint32_t flags, cudaStream_t s) {
-  if (h->opt_fused && h->len >= 1) {
+  if (h->opt_fused && h->len >= 1 && !h->rope) {
     if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL k or v");
     if (h->len + 1 > h->desc.n_max)
       return fail(h, EA_ERR_CAPACITY, "decode_step: len %d + 1 exceeds n_max %d", h->len, h->desc.n_max);
@@ -404,14 +451,17 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
           }
       }
     }
-    if (dh % 16 == 0) {   // lift image of U^V: rows = d (the N index of the lift product), contraction over the rank
-      const int rv16 = (hi.rp_v + 15) & ~15;
-      uint16_t* img_hi = reinterpret_cast<uint16_t*>(basis.data() + hi.uvl16_off);
+    for (int pass = 0; pass < 2 && dh % 16 == 0; ++pass) {
+      // lift images of U^V (pass 0) and U^K (pass 1): rows = d (the N index of the lift product), contraction over the rank
+      const float* U = pass ? uk : uv;
+      const int r = pass ? hi.r_k : hi.r_v;
+      const int rv16 = ((pass ? hi.rp_k : hi.rp_v) + 15) & ~15;
+      uint16_t* img_hi = reinterpret_cast<uint16_t*>(basis.data() + (pass ? hi.ukl16_off : hi.uvl16_off));
       uint16_t* img_lo = img_hi + static_cast<size_t>(rv16) * dh;
       const int grp = (rv16 / 8) * 128;                       // bytes per group of 8 rows (d values)
       for (int d = 0; d < dh; ++d)
         for (int c = 0; c < rv16; ++c) {
-          const float x = c < hi.r_v ? uv[static_cast<size_t>(d) * hi.r_v + c] : 0.f;
+          const float x = c < r ? U[static_cast<size_t>(d) * r + c] : 0.f;
           const uint16_t xh = bf16_rne(x);
           const uint16_t xl = bf16_rne(x - bf16_to_float(xh));
           const size_t off = (static_cast<size_t>(d >> 3) * grp + (c >> 3) * 128 + (d & 7) * 16 + (c & 7) * 2) / 2;
@@ -528,6 +578,7 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
 ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                    int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "decode_static: not available with a rotary embedding");
   DecodePlan plan;
   ea_status st = plan_decode(h, "decode_static", d_q, stride_b_q, d_out, stride_b_out, flags, nullptr, nullptr,
                              nullptr, 0, &plan);
@@ -550,6 +601,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                              int64_t stride_b, int64_t stride_t, void* d_out, int64_t out_stride_b,
                              int64_t out_stride_t, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available with a rotary embedding");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
   if (flags & ~EA_OUT_LOWRANK) return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
   if (T < 1) return fail(h, EA_ERR_SHAPE, "prefill: T = %d", T);
@@ -679,6 +731,7 @@ ea_status eigen_attn_cache_layout(eigen_attn_t h, int32_t head, size_t* k_offset
 
 ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->rope && slopes) return fail(h, EA_ERR_INVALID_ARG, "set_alibi: the layer has a rotary embedding");
   const int H = h->desc.n_heads;
   bool any = false;
   for (int i = 0; i < H; ++i) {
@@ -692,6 +745,28 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return cuda_fail(h, e, "set_alibi");
   h->alibi = any;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (base == 0.0) {
+    h->rope = false;
+    return EA_OK;
+  }
+  if (!(base > 1.0) || !isfinite(base)) return fail(h, EA_ERR_INVALID_ARG, "set_rope: base %g", base);
+  if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16)
+    return fail(h, EA_ERR_UNSUPPORTED, "set_rope: needs a bf16 layer with d_head %% 16 == 0");
+  if (h->alibi) return fail(h, EA_ERR_INVALID_ARG, "set_rope: the layer has an ALiBi bias");
+  const int dh = h->desc.d_head;
+  double freq[64] = {};
+  for (int i = 0; i < dh / 2; ++i) freq[i] = pow(base, -2.0 * i / dh);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_rope, freq, sizeof(freq), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "set_rope");
+  h->rope = true;
+  h->rope_interleaved = interleaved ? 1 : 0;
   return EA_OK;
 }
 

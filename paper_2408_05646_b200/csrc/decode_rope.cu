@@ -1,0 +1,335 @@
+// Generation-phase Eigen Attention for models with rotary position embedding (Section 4.3, Fig. 6b).
+//
+// The query stays full rank.  Each cached low-dimensional key row k'_j is taken back to d_h dimensions
+// through (U^K)^T, rotated by its position j and dotted with the rotated query; the value side is the
+// rank-r path unchanged.  Per cached row that is a d_h x r product instead of an r-long dot product, so the
+// lift runs on the tensor cores: for a tile of 128 cached rows, X = K'_tile (U^K)^T is one tcgen05 product
+// (M = 128 rows, N = d_h, K = r; U^K as bf16 high + low parts, two products, so that the lift keeps
+// fp32-class accuracy) with X in TMEM, one row per thread.
+//
+// Rotation without a table per position: with complex pairs Q = q_a + i q_b, X = x_a + i x_b and the
+// pair's frequency phi, the rotated dot product of the pair is Re(Q e^{i p phi} conj(X e^{i j phi})) =
+// Re(Q e^{i (p - j) phi} conj(X)).  For row l of tile t, p - j = D_t - l with D_t = p - 128 t, so
+// e^{i (p-j) phi} = e^{i D_t phi} conj(e^{i l phi}): the first factor is applied to the query once per tile
+// (64 threads, angle reduced in fp64), the second is a per-thread constant held in registers.
+//
+// One CTA (128 threads) walks a contiguous range of the tiles of one (sequence, head) unit: K' tiles are
+// double-buffered (cp.async into the canonical core-matrix layout), V' tiles single-buffered and fetched
+// while the next tile's scores are computed.  Scores -> online softmax in base 2 -> o' += p V' on the CUDA
+// cores (thread c owns column c).  A unit split over several CTAs leaves partials (m, l, o') that
+// rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+#include "tc_common.cuh"
+
+namespace ea {
+namespace {
+
+using namespace tc;
+
+struct __align__(16) RopeSmemHeader {
+  unsigned long long mma_done;
+  uint32_t tmem_base;
+  int abort_flag;
+  float red[8];          // cross-warp reductions
+  float tile_max;
+  float pad_[3];
+};
+
+// Asynchronous copy of `rows_valid` rows of a row-major bf16 matrix (row pitch `rp` elements) into a canonical
+// no-swizzle tile of 128 rows x `nch` chunks (zeros elsewhere), 128 threads.
+__device__ __forceinline__ void load_canonical_async(unsigned char* dst, const __nv_bfloat16* src, int rp,
+                                                     int rows_valid, int nch, int tid) {
+  const int src_chunks = rp >> 3;
+  const int group_stride = nch << 7;
+  for (int idx = tid; idx < kTile * nch; idx += kThreads) {
+    const int c = ((idx / (2 * kTile)) << 1) + (idx & 1), row = (idx >> 1) & (kTile - 1);
+    const bool live = row < rows_valid && c < src_chunks;
+    const void* g = live ? static_cast<const void*>(src + static_cast<int64_t>(row) * rp + c * 8) : src;
+    cp_async16(dst + chunk_off(row, c, group_stride), g, live ? 16u : 0u);
+  }
+}
+// Same for a plain row-major tile (the V' rows as the CUDA cores read them).
+__device__ __forceinline__ void load_rows_async(unsigned char* dst, const __nv_bfloat16* src, int rp, int rows_valid,
+                                                int tid) {
+  const int chunks = rp >> 3;
+  for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
+    const int row = idx / chunks;
+    const bool live = row < rows_valid;
+    cp_async16(dst + idx * 16, live ? static_cast<const void*>(src + static_cast<int64_t>(idx) * 8) : src,
+               live ? 16u : 0u);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int unit = blockIdx.x, split = blockIdx.y;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const int rpk16 = (hd.rp_k + 15) & ~15;
+  const int nch_k = rpk16 >> 3, grp_k = nch_k << 7;
+  const int k_bytes = kTile * rpk16 * 2, v_bytes = kTile * hd.rp_v * 2;
+  const int u_bytes = p.d_head * rpk16 * 2;                  // one image (high or low part) of U^K
+  const int half = p.d_head >> 1;
+
+  float* q_tile = reinterpret_cast<float*>(smem + 256);      // [d_head]: (re, im) of the query pairs for this tile
+  float* p_row = q_tile + 128;                               // [128] softmax weights of the tile
+  unsigned char* tiles = smem + 2048;
+  unsigned char* Us = tiles;                                 // U^K image: high part, then low part
+  unsigned char* Ks = Us + 2 * u_bytes;                      // two K' tiles
+  unsigned char* Vs = Ks + 2 * k_bytes;                      // one V' tile
+
+  // tiles [t_lo, t_hi) of the unit
+  const int per = (p.nt + p.splits - 1) / p.splits;
+  const int t_lo = split * per, t_hi = min(p.nt, t_lo + per);
+  float* part = p.partials + (static_cast<size_t>(unit) * p.splits + split) * p.part_stride;
+  if (t_lo >= t_hi) {                                        // an empty piece: the neutral partial
+    if (tid == 0) { part[0] = -INFINITY; part[1] = 0.f; }
+    if (tid < hd.rp_v) part[4 + tid] = 0.f;
+    return;
+  }
+
+  if (warp == 0) tmem_alloc(&hdr->tmem_base, 128);
+  if (tid == 0) {
+    mbar_init(&hdr->mma_done, 1);
+    hdr->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+
+  const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.k_off) +
+                            static_cast<int64_t>(b) * p.n_max * hd.rp_k;
+  const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.v_off) +
+                            static_cast<int64_t>(b) * p.n_max * hd.rp_v;
+  // U^K image and the first K'/V' tiles
+  {
+    const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.ukl16_off);
+    for (int idx = tid; idx < 2 * u_bytes / 16; idx += kThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
+    const int rows0 = min(kTile, p.n - t_lo * kTile);
+    load_canonical_async(Ks, Kg + static_cast<int64_t>(t_lo) * kTile * hd.rp_k, hd.rp_k, rows0, nch_k, tid);
+    cp_async_commit();
+    load_rows_async(Vs, Vg + static_cast<int64_t>(t_lo) * kTile * hd.rp_v, hd.rp_v, rows0, tid);
+    cp_async_commit();
+  }
+
+  // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
+  float el_c[64], el_s[64];
+#pragma unroll
+  for (int i = 0; i < 64; ++i) {
+    float s_, c_;
+    sincosf(static_cast<float>(tid) * static_cast<float>(i < half ? p.inv_freq[i] : 0.0), &s_, &c_);
+    el_c[i] = c_;
+    el_s[i] = s_;
+  }
+  // the query of this unit, scaled by log2(e)/sqrt(d_h): thread i < half owns pair i
+  float q_re = 0.f, q_im = 0.f;
+  double my_freq = 0.0;
+  if (tid < half) {
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head;
+    const int ia = p.interleaved ? 2 * tid : tid, ib = p.interleaved ? 2 * tid + 1 : tid + half;
+    q_re = __bfloat162float(qg[ia]) * p.q_scale;
+    q_im = __bfloat162float(qg[ib]) * p.q_scale;
+    my_freq = p.inv_freq[tid];
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = hdr->tmem_base;
+  const uint32_t tX = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+  volatile int* abort_flag = &hdr->abort_flag;
+  const uint32_t idesc = instr_desc(p.d_head, false);
+  const int ks_steps = rpk16 >> 4;
+  const int pos_q = p.n - 1;
+
+  float m_run = -INFINITY, l_thr = 0.f, o_acc = 0.f;         // o_acc: column tid of o'
+  bool ok = true;
+  for (int t = t_lo; t < t_hi && ok; ++t) {
+    const int buf = (t - t_lo) & 1;
+    unsigned char* Kt = Ks + buf * k_bytes;
+    // ---- the query pairs turned by (pos_q - 128 t) phi, angle reduced in fp64
+    if (tid < half) {
+      const double ang = static_cast<double>(pos_q - t * kTile) * my_freq;
+      const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+      float s_, c_;
+      sincosf(static_cast<float>(red), &s_, &c_);
+      q_tile[2 * tid] = q_re * c_ - q_im * s_;
+      q_tile[2 * tid + 1] = q_re * s_ + q_im * c_;
+    }
+    // ---- K'(t) has landed (V'(t) may still be in flight); the next K' tile goes out
+    cp_async_wait<1>();
+    fence_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t ka = smem_u32(Kt), ua = smem_u32(Us);
+      for (int part_i = 0; part_i < 2; ++part_i)             // U^K high part, then low part
+        for (int s = 0; s < ks_steps; ++s)
+          mma_ss(tmem, smem_desc(ka + s * 256, 128, grp_k), smem_desc(ua + part_i * u_bytes + s * 256, 128, grp_k),
+                 idesc, part_i > 0 || s > 0);
+      mma_commit(&hdr->mma_done);
+    }
+    // (cp.async groups in flight here: V'(t), then K'(t+1))
+    if (t + 1 < t_hi) {
+      const int rows1 = min(kTile, p.n - (t + 1) * kTile);
+      load_canonical_async(Ks + (buf ^ 1) * k_bytes, Kg + static_cast<int64_t>(t + 1) * kTile * hd.rp_k, hd.rp_k, rows1,
+                           nch_k, tid);
+    }
+    cp_async_commit();
+    // ---- X = K' (U^K)^T is in TMEM: score of this thread's row
+    ok = mbar_wait(&hdr->mma_done, (t - t_lo) & 1u, p.status);
+    ok = !__syncthreads_or(!ok || *abort_flag);
+    if (!ok) break;
+    tc_fence_after();
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int c0 = 0; c0 < 64; c0 += 16) {
+      if (c0 < half) {
+        uint32_t xa[16], xb[16];
+        if (p.interleaved) {                                 // pairs (2i, 2i+1): columns 2 c0 .. 2 c0 + 31
+          tmem_ld16(tX + 2 * c0, xa);
+          tmem_ld16(tX + 2 * c0 + 16, xb);
+        } else {                                             // pairs (i, i + d_h/2)
+          tmem_ld16(tX + c0, xa);
+          tmem_ld16(tX + half + c0, xb);
+        }
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float x_re, x_im;
+          if (p.interleaved) {
+            const uint32_t* src = i < 8 ? xa : xb;
+            x_re = __uint_as_float(src[(2 * i) & 15]);
+            x_im = __uint_as_float(src[(2 * i + 1) & 15]);
+          } else {
+            x_re = __uint_as_float(xa[i]);
+            x_im = __uint_as_float(xb[i]);
+          }
+          const float2 qt = *reinterpret_cast<const float2*>(q_tile + 2 * (c0 + i));
+          // W = Q_t conj(E_l); pair term = Re(W conj(X)) = W_re x_re + W_im x_im
+          const float w_re = fmaf(qt.x, el_c[c0 + i], qt.y * el_s[c0 + i]);
+          const float w_im = fmaf(qt.y, el_c[c0 + i], -qt.x * el_s[c0 + i]);
+          s0 = fmaf(w_re, x_re, s0);
+          s1 = fmaf(w_im, x_im, s1);
+        }
+      }
+    }
+    const int j = t * kTile + tid;
+    const bool live = j < p.n;
+    float s = live ? s0 + s1 : -INFINITY;
+    // ---- online softmax over the tile: block maximum, weights, running sum per thread
+    float mx = s;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) hdr->red[warp] = mx;
+    cp_async_wait<1>();                                      // V'(t) has landed (K'(t+1) may be in flight)
+    __syncthreads();
+    const float m_new = fmaxf(m_run, fmaxf(fmaxf(hdr->red[0], hdr->red[1]), fmaxf(hdr->red[2], hdr->red[3])));
+    const float alpha = ex2(m_run - m_new);                  // 0 at the first tile
+    m_run = m_new;
+    const float pj = live ? ex2(s - m_new) : 0.f;
+    l_thr = fmaf(l_thr, alpha, pj);
+    p_row[tid] = pj;
+    __syncthreads();
+    // ---- o'[c] = alpha o'[c] + sum_j p_j V'[j][c], thread c = tid
+    if (tid < hd.rp_v) {
+      const __nv_bfloat16* vcol = reinterpret_cast<const __nv_bfloat16*>(Vs) + tid;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+      for (int r = 0; r < kTile; r += 4) {
+        const float4 pr = *reinterpret_cast<const float4*>(p_row + r);
+        a0 = fmaf(pr.x, __bfloat162float(vcol[(r + 0) * hd.rp_v]), a0);
+        a1 = fmaf(pr.y, __bfloat162float(vcol[(r + 1) * hd.rp_v]), a1);
+        a2 = fmaf(pr.z, __bfloat162float(vcol[(r + 2) * hd.rp_v]), a2);
+        a3 = fmaf(pr.w, __bfloat162float(vcol[(r + 3) * hd.rp_v]), a3);
+      }
+      o_acc = fmaf(o_acc, alpha, (a0 + a1) + (a2 + a3));
+    }
+    tc_fence_before();
+    __syncthreads();                                         // V' tile and TMEM rows are free again
+    if (t + 1 < t_hi) {
+      const int rows1 = min(kTile, p.n - (t + 1) * kTile);
+      load_rows_async(Vs, Vg + static_cast<int64_t>(t + 1) * kTile * hd.rp_v, hd.rp_v, rows1, tid);
+    }
+    cp_async_commit();
+    // (groups in flight: K'(t+1), then V'(t+1))
+  }
+  cp_async_wait<0>();
+  if (!ok) *abort_flag = 1;
+
+  // ---- the piece's partial: m, l (sum over the threads' rows), o'
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l_thr += __shfl_xor_sync(0xffffffffu, l_thr, o);
+  __syncthreads();
+  if (lane == 0) hdr->red[4 + warp] = l_thr;
+  __syncthreads();
+  if (tid == 0) {
+    part[0] = m_run;
+    part[1] = (hdr->red[4] + hdr->red[5]) + (hdr->red[6] + hdr->red[7]);
+  }
+  if (tid < hd.rp_v) part[4 + tid] = o_acc;
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 128);
+}
+
+// Merges the partials of a unit and lifts o'/l through (U^V)^T (or writes the rank-space row).
+__global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParams p) {
+  __shared__ float o_sm[128];
+  const int unit = blockIdx.x, t = threadIdx.x;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const float* base = p.partials + static_cast<size_t>(unit) * p.splits * p.part_stride;
+  float M = -INFINITY;
+  for (int c = 0; c < p.splits; ++c) M = fmaxf(M, base[static_cast<size_t>(c) * p.part_stride]);
+  float L = 0.f, acc = 0.f;
+  for (int c = 0; c < p.splits; ++c) {
+    const float* part = base + static_cast<size_t>(c) * p.part_stride;
+    const float f = ex2(part[0] - M);                        // 0 for an empty piece
+    L = fmaf(part[1], f, L);
+    if (t < hd.rp_v) acc = fmaf(part[4 + t], f, acc);
+  }
+  const float o = acc / L;
+  __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out);
+  if (p.flags & 0x2u) {
+    if (t < hd.rp_v) out[b * p.out_stride_b + hd.lr_v_off + t] = __float2bfloat16_rn(o);
+    return;
+  }
+  if (t < hd.rp_v) o_sm[t] = o;
+  __syncthreads();
+  if (t < p.d_head) {
+    const float* Ut = p.basis + hd.uvt_off;                  // (U^V)^T : rp_v x d_head
+    float y = 0.f;
+    for (int c = 0; c < hd.rp_v; ++c) y = fmaf(o_sm[c], __ldg(Ut + c * p.d_head + t), y);
+    out[b * p.out_stride_b + static_cast<int64_t>(h) * p.d_head + t] = __float2bfloat16_rn(y);
+  }
+}
+
+}  // namespace
+
+size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
+  const size_t k16 = (max_rp_k + 15) & ~15;
+  return 2048 + 2 * static_cast<size_t>(d_head) * k16 * 2 + 2 * kTile * k16 * 2 + static_cast<size_t>(kTile) * max_rp_v * 2;
+}
+
+cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
+  static size_t configured = 0;
+  if (smem > configured) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  dim3 grid(p.B * p.H, p.splits);
+  decode_rope_kernel<<<grid, kThreads, smem, s>>>(p);
+  ++*launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  rope_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace ea

@@ -22,7 +22,7 @@ struct HeadInfo {
   int32_t uvt16_off;  //   [rp16][d_head] in the canonical core-matrix order (rp16 = rank padded to 16); same for U^V
   int32_t uvl16_off;  // float offset of the lift image of U^V: bf16 high then low part, each [d_head][rv16] canonical
   float alibi_slope2;  // ALiBi slope of the head times log2(e); 0 = no position bias
-  int32_t pad_;
+  int32_t ukl16_off;   // float offset of the lift image of U^K (as uvl16_off, [d_head][rk16] canonical, high then low)
 };
 
 constexpr int kDecodeConsumerWarps = 8;
@@ -127,6 +127,27 @@ struct PrefillParams {
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head (warp-specialised kernel only)
 };
 
+struct RopeDecodeParams {    // decode for models with rotary position embedding (bf16 layers)
+  const HeadInfo* heads;
+  const float* basis;
+  const char* cache;
+  const void* q;            // [B][1][H][d_head], full rank, not rotated
+  int64_t q_stride_b;
+  void* out;                // [B][1][H][d_head] or packed [B][sum rp_v]
+  int64_t out_stride_b;
+  float* partials;          // [B*H][splits][part_stride]: m, l, pad, pad, o'[rp_v]
+  int* status;
+  const double* inv_freq;   // [d_head/2]: base^(-2i/d_head)
+  int32_t part_stride;
+  int32_t B, H, d_head;
+  int32_t n, n_max;
+  int32_t nt;               // tiles of 128 rows per unit
+  int32_t splits;           // CTAs per unit
+  int32_t interleaved;      // pairs (2i, 2i+1) instead of (i, i + d_head/2)
+  float q_scale;            // log2(e) / sqrt(d_head)
+  uint32_t flags;
+};
+
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.
 cudaError_t launch_project_append(const ProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t smem_bytes,
@@ -134,6 +155,8 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
+cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
 cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches);

@@ -1,0 +1,93 @@
+"""GPU parity of the RoPE variant of the generation phase (Section 4.3) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, make_case, oracle_layer, to_np
+from oracle import eigen_attention as orc
+
+pytestmark = pytest.mark.gpu
+BF16, FP32 = torch.bfloat16, torch.float32
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    return binding
+
+
+def rope_oracle(B_, H, d, U_k, U_v, base, interleaved):
+    return orc.LayerOracle(B_, H, d, U_k, U_v, rope={"base": base, "interleaved": interleaved})
+
+
+@pytest.mark.parametrize("H,d,rk,rv,n,base,interleaved", [
+    (2, 128, [80, 80], [80, 80], 128, 10000.0, False),              # exactly one tile
+    (2, 128, [80, 80], [80, 80], 1037, 10000.0, False),             # several tiles, ragged tail
+    (4, 128, [48, 64, 112, 128], [96, 80, 48, 128], 700, 10000.0, True),
+    (3, 64, [24, 64, 40], [56, 8, 64], 517, 500000.0, False),       # small d_head, ranks that are not multiples of 16
+    (1, 128, [80], [80], 17, 10000.0, True),                        # shorter than a tile
+    (2, 128, [64, 64], [64, 64], 9000, 10000.0, False),             # positions in the thousands
+])
+def test_rope_decode_matches_oracle(B, H, d, rk, rv, n, base, interleaved):
+    B_ = 2
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, BF16, seed_cfg=151)
+    lay = B.EigenAttnLayer(B_, H, d, n + 4, BF16, U_k, U_v)
+    lay.set_rope(base, interleaved)
+    lay.append_kv(k, v)
+    ref = rope_oracle(B_, H, d, U_k, U_v, base, interleaved)
+    ref.append_kv(to_np(k), to_np(v))
+    expect = ref.decode_dense(to_np(q))
+    assert_close(lay.decode(q), expect, BF16, "rope decode")
+    for ctas in (1, 7, 300, 1024):                                   # CTAs per unit must not matter
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode(q), expect, BF16, f"rope decode ctas={ctas}")
+    lay.poll_status()
+
+
+def test_rope_decode_steps_lowrank_output_and_switching_off(B):
+    B_, H, d, n, steps = 2, 2, 128, 300, 5
+    rk, rv = [80, 48], [64, 80]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + steps, BF16, seed_cfg=153, T_q=steps)
+    lay = B.EigenAttnLayer(B_, H, d, n + steps, BF16, U_k, U_v)
+    lay.set_rope(10000.0)
+    lay.append_kv(k[:, :n], v[:, :n])
+    ref = rope_oracle(B_, H, d, U_k, U_v, 10000.0, False)
+    ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
+    for s in range(steps):                                           # append + decode, positions advance by one
+        o = lay.decode_step(q[:, s:s + 1], k[:, n + s:n + s + 1], v[:, n + s:n + s + 1])
+        ref.append_kv(to_np(k[:, n + s:n + s + 1]), to_np(v[:, n + s:n + s + 1]))
+        assert_close(o, ref.decode_dense(to_np(q[:, s:s + 1])), BF16, f"rope step {s}")
+    low = lay.decode(q[:, :1], out_lowrank=True)
+    res = ref.decode(to_np(q[:, :1]), lowrank_out=True)
+    for b in range(B_):
+        for h in range(H):
+            assert_close(low[b, 0, lay.offs_v[h]:lay.offs_v[h] + rv[h]], res[(b, h)], BF16, "rope lowrank out")
+    lay.set_rope(0.0)                                                # back to the plain path
+    plain = oracle_layer(B_, H, d, U_k, U_v)
+    plain.append_kv(to_np(k), to_np(v))
+    assert_close(lay.decode(q[:, :1]), plain.decode_dense(to_np(q[:, :1])), BF16, "rope off")
+    lay.poll_status()
+
+
+def test_rope_rejections(B):
+    U_k, U_v, q, k, v = make_case(1, 2, 64, [16, 16], [16, 16], 8, FP32, seed_cfg=155)
+    lay32 = B.EigenAttnLayer(1, 2, 64, 8, FP32, U_k, U_v)
+    with pytest.raises(B.EigenAttnError):
+        lay32.set_rope(10000.0)                                      # bf16 layers only
+    U_k, U_v, q, k, v = make_case(1, 2, 64, [16, 16], [16, 16], 8, BF16, seed_cfg=155)
+    lay = B.EigenAttnLayer(1, 2, 64, 8, BF16, U_k, U_v, max_prefill_tokens=8)
+    with pytest.raises(B.EigenAttnError):
+        lay.set_rope(0.5)
+    lay.set_rope(10000.0)
+    with pytest.raises(B.EigenAttnError):
+        lay.prefill(q.expand(1, 8, 2, 64).contiguous(), k, v)
+    lay.append_kv(k, v)
+    with pytest.raises(B.EigenAttnError):
+        lay.decode_static(q)
+    with pytest.raises(B.EigenAttnError):
+        lay.set_alibi([0.5, 0.25])
+    qp = torch.zeros((1, 1, lay.offs_k[-1]), dtype=BF16, device="cuda")
+    with pytest.raises(B.EigenAttnError):
+        lay.decode(qp, q_preprojected=True)
