@@ -111,7 +111,8 @@ class ClockSampler:
 # the CPU oracle leg (also the --impl reference arm)
 # ----------------------------------------------------------------------------------------------
 
-VARIANT = {"alibi": False}   # --alibi: per-head ALiBi slopes on both sides (decode workloads)
+VARIANT = {"alibi": False, "rope": False}   # --alibi / --rope: position schemes on both sides (decode workloads)
+ROPE_BASE = 10000.0
 
 
 def variant_slopes(wl):
@@ -132,7 +133,8 @@ def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, sample_heads, history=No
     `history` maps h -> (k_rows, v_rows) [n, d_head] float64; if None it is drawn on the CPU."""
     from oracle import eigen_attention as orc
     units = [(0, h) for h in sample_heads]
-    lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units, alibi_slopes=variant_slopes(wl))
+    lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units, alibi_slopes=variant_slopes(wl),
+                          rope={"base": ROPE_BASE, "interleaved": False} if VARIANT["rope"] else None)
     if history is None:
         W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
         W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
@@ -247,6 +249,8 @@ def build_layer(wl, device, binding, keep_heads=(), rank=0):
     lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + 1, dt, U_k, U_v, device=device)
     if VARIANT["alibi"]:
         lay.set_alibi(variant_slopes(wl))
+    if VARIANT["rope"]:
+        lay.set_rope(ROPE_BASE)
     W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K", device=device)
     W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V", device=device)
     hist = {h: ([], []) for h in keep_heads}
@@ -390,11 +394,11 @@ def run_ours(args, wl):
         "dtype": "bf16 storage, f32 accumulate" if wl.dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": wl.name, "batch_per_gpu": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
-                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "alibi": VARIANT["alibi"],
+                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "alibi": VARIANT["alibi"], "rope": VARIANT["rope"],
                    "cache_gb_per_gpu": bytes_step / 1e9, "parallelism": f"{world} independent batch shard(s)",
                    "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
         "frac_of_nominal_8TBs": value / world / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "decode_splitkv_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_rope_kernel" if VARIANT["rope"] else "decode_splitkv_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "kernel_us": kern_avg_ms * 1e3, "algorithmic_bytes": bytes_step,
                      "traffic": (bytes_step * DECODE_TRAFFIC_RATIO
@@ -545,12 +549,14 @@ def main():
     ap.add_argument("--workload", default="llama2_7b_b16_n32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--alibi", action="store_true", help="decode workloads: add the per-head ALiBi position bias")
+    ap.add_argument("--rope", action="store_true", help="decode workloads: the RoPE variant (full-rank query, lifted rotated keys)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")
     args = ap.parse_args()
     VARIANT["alibi"] = bool(args.alibi)
+    VARIANT["rope"] = bool(args.rope)
     if args.warmup < 3:
         args.warmup = 3
     wl = synth.WORKLOADS[args.workload]

@@ -322,6 +322,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
   p.status = dev_status(h);
   p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+  p.tmaps = h->ws + L.off_tmaps;
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;
@@ -755,8 +756,8 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
     return EA_OK;
   }
   if (!(base > 1.0) || !isfinite(base)) return fail(h, EA_ERR_INVALID_ARG, "set_rope: base %g", base);
-  if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16)
-    return fail(h, EA_ERR_UNSUPPORTED, "set_rope: needs a bf16 layer with d_head %% 16 == 0");
+  if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
+    return fail(h, EA_ERR_UNSUPPORTED, "set_rope: needs a bf16 layer with d_head %% 16 == 0 (and the driver's tensor-map encoder)");
   if (h->alibi) return fail(h, EA_ERR_INVALID_ARG, "set_rope: the layer has an ALiBi bias");
   const int dh = h->desc.d_head;
   double freq[64] = {};

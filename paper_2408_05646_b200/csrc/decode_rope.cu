@@ -4,8 +4,8 @@
 // through (U^K)^T, rotated by its position j and dotted with the rotated query; the value side is the
 // rank-r path unchanged.  Per cached row that is a d_h x r product instead of an r-long dot product, so the
 // lift runs on the tensor cores: for a tile of 128 cached rows, X = K'_tile (U^K)^T is one tcgen05 product
-// (M = 128 rows, N = d_h, K = r; U^K as bf16 high + low parts, two products, so that the lift keeps
-// fp32-class accuracy) with X in TMEM, one row per thread.
+// (M = 128 rows, N = d_h, K = r; U^K rounded to bf16, the precision the cached rows already have) with X in
+// TMEM, one row per thread.
 //
 // Rotation without a table per position: with complex pairs Q = q_a + i q_b, X = x_a + i x_b and the
 // pair's frequency phi, the rotated dot product of the pair is Re(Q e^{i p phi} conj(X e^{i j phi})) =
@@ -13,10 +13,11 @@
 // e^{i (p-j) phi} = e^{i D_t phi} conj(e^{i l phi}): the first factor is applied to the query once per tile
 // (64 threads, angle reduced in fp64), the second is a per-thread constant held in registers.
 //
-// One CTA (128 threads) walks a contiguous range of the tiles of one (sequence, head) unit: K' tiles are
-// double-buffered (cp.async into the canonical core-matrix layout), V' tiles single-buffered and fetched
-// while the next tile's scores are computed.  Scores -> online softmax in base 2 -> o' += p V' on the CUDA
-// cores (thread c owns column c).  A unit split over several CTAs leaves partials (m, l, o') that
+// One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  One
+// thread fetches the K' and V' tiles by TMA (the tensor maps of the cache slabs, 64 x 64 boxes, 128-byte
+// swizzle): K'(t+1) as soon as the lift of tile t has read K'(t), V'(t+1) as soon as tile t's weighted sum
+// is done, so both land behind the arithmetic of the tile in between.  Scores -> online softmax in base 2 ->
+// o' += p V' on the CUDA cores (thread c owns column c and reads the swizzled tile).  A unit split over several CTAs leaves partials (m, l, o') that
 // rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -28,39 +29,16 @@ namespace {
 
 using namespace tc;
 
+constexpr int kAtom = kTile * 128;            // one swizzled atom column of a 128-row tile: 64 elements wide
+
 struct __align__(16) RopeSmemHeader {
-  unsigned long long mma_done;
+  unsigned long long mma_done, k_full, v_full;
   uint32_t tmem_base;
   int abort_flag;
   float red[8];          // cross-warp reductions
   float tile_max;
   float pad_[3];
 };
-
-// Asynchronous copy of `rows_valid` rows of a row-major bf16 matrix (row pitch `rp` elements) into a canonical
-// no-swizzle tile of 128 rows x `nch` chunks (zeros elsewhere), 128 threads.
-__device__ __forceinline__ void load_canonical_async(unsigned char* dst, const __nv_bfloat16* src, int rp,
-                                                     int rows_valid, int nch, int tid) {
-  const int src_chunks = rp >> 3;
-  const int group_stride = nch << 7;
-  for (int idx = tid; idx < kTile * nch; idx += kThreads) {
-    const int c = ((idx / (2 * kTile)) << 1) + (idx & 1), row = (idx >> 1) & (kTile - 1);
-    const bool live = row < rows_valid && c < src_chunks;
-    const void* g = live ? static_cast<const void*>(src + static_cast<int64_t>(row) * rp + c * 8) : src;
-    cp_async16(dst + chunk_off(row, c, group_stride), g, live ? 16u : 0u);
-  }
-}
-// Same for a plain row-major tile (the V' rows as the CUDA cores read them).
-__device__ __forceinline__ void load_rows_async(unsigned char* dst, const __nv_bfloat16* src, int rp, int rows_valid,
-                                                int tid) {
-  const int chunks = rp >> 3;
-  for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
-    const int row = idx / chunks;
-    const bool live = row < rows_valid;
-    cp_async16(dst + idx * 16, live ? static_cast<const void*>(src + static_cast<int64_t>(idx) * 8) : src,
-               live ? 16u : 0u);
-  }
-}
 
 __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -71,16 +49,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15;
   const int nch_k = rpk16 >> 3, grp_k = nch_k << 7;
-  const int k_bytes = kTile * rpk16 * 2, v_bytes = kTile * hd.rp_v * 2;
-  const int u_bytes = p.d_head * rpk16 * 2;                  // one image (high or low part) of U^K
+  const int atoms_k = (rpk16 + 63) >> 6, atoms_v = (hd.rp_v + 63) >> 6;
+  const int k_bytes = atoms_k * kAtom, v_bytes = atoms_v * kAtom;
+  const int u_bytes = p.d_head * rpk16 * 2;                  // bf16 image of U^K (the high part of the stored pair)
   const int half = p.d_head >> 1;
 
   float* q_tile = reinterpret_cast<float*>(smem + 256);      // [d_head]: (re, im) of the query pairs for this tile
   float* p_row = q_tile + 128;                               // [128] softmax weights of the tile
   unsigned char* tiles = smem + 2048;
-  unsigned char* Us = tiles;                                 // U^K image: high part, then low part
-  unsigned char* Ks = Us + 2 * u_bytes;                      // two K' tiles
-  unsigned char* Vs = Ks + 2 * k_bytes;                      // one V' tile
+  unsigned char* Ks = tiles;                                 // one K' tile, swizzled atom columns of 128 rows
+  unsigned char* Vs = Ks + k_bytes;                          // one V' tile, same layout
+  unsigned char* Us = Vs + v_bytes;                          // U^K image, canonical no-swizzle layout
 
   // tiles [t_lo, t_hi) of the unit
   const int per = (p.nt + p.splits - 1) / p.splits;
@@ -95,24 +74,33 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   if (warp == 0) tmem_alloc(&hdr->tmem_base, 128);
   if (tid == 0) {
     mbar_init(&hdr->mma_done, 1);
+    mbar_init(&hdr->k_full, 1);
+    mbar_init(&hdr->v_full, 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
 
-  const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.k_off) +
-                            static_cast<int64_t>(b) * p.n_max * hd.rp_k;
-  const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.v_off) +
-                            static_cast<int64_t>(b) * p.n_max * hd.rp_v;
-  // U^K image and the first K'/V' tiles
+  // U^K image (read through L2 by every CTA of the head)
   {
     const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.ukl16_off);
-    for (int idx = tid; idx < 2 * u_bytes / 16; idx += kThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
-    const int rows0 = min(kTile, p.n - t_lo * kTile);
-    load_canonical_async(Ks, Kg + static_cast<int64_t>(t_lo) * kTile * hd.rp_k, hd.rp_k, rows0, nch_k, tid);
-    cp_async_commit();
-    load_rows_async(Vs, Vg + static_cast<int64_t>(t_lo) * kTile * hd.rp_v, hd.rp_v, rows0, tid);
+    for (int idx = tid; idx < u_bytes / 16; idx += kThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
     cp_async_commit();
   }
+  const unsigned char* maps = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
+  // one tile = two boxes of 64 rows per atom column; rows past the current length hold earlier or zero data
+  // and get weight zero, rows past the capacity arrive as zeros
+  auto fetch_k = [&](int t) {
+    mbar_arrive_expect_tx(&hdr->k_full, static_cast<uint32_t>(k_bytes));
+    for (int a = 0; a < atoms_k; ++a)
+      for (int hf = 0; hf < 2; ++hf)
+        tma_load_3d(Ks + a * kAtom + hf * (kAtom / 2), maps, a * 64, t * kTile + hf * 64, b, &hdr->k_full);
+  };
+  auto fetch_v = [&](int t) {
+    mbar_arrive_expect_tx(&hdr->v_full, static_cast<uint32_t>(v_bytes));
+    for (int a = 0; a < atoms_v; ++a)
+      for (int hf = 0; hf < 2; ++hf)
+        tma_load_3d(Vs + a * kAtom + hf * (kAtom / 2), maps + 128, a * 64, t * kTile + hf * 64, b, &hdr->v_full);
+  };
 
   // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
   float el_c[64], el_s[64];
@@ -134,9 +122,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     my_freq = p.inv_freq[tid];
   }
 
+  cp_async_wait<0>();
+  fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (tid == 0) {
+    tensormap_acquire(maps);
+    tensormap_acquire(maps + 128);
+    fetch_k(t_lo);
+    fetch_v(t_lo);
+  }
   const uint32_t tmem = hdr->tmem_base;
   const uint32_t tX = tmem + (static_cast<uint32_t>(warp * 32) << 16);
   volatile int* abort_flag = &hdr->abort_flag;
@@ -147,8 +143,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   float m_run = -INFINITY, l_thr = 0.f, o_acc = 0.f;         // o_acc: column tid of o'
   bool ok = true;
   for (int t = t_lo; t < t_hi && ok; ++t) {
-    const int buf = (t - t_lo) & 1;
-    unsigned char* Kt = Ks + buf * k_bytes;
+    const uint32_t par = (t - t_lo) & 1u;
     // ---- the query pairs turned by (pos_q - 128 t) phi, angle reduced in fp64
     if (tid < half) {
       const double ang = static_cast<double>(pos_q - t * kTile) * my_freq;
@@ -158,30 +153,23 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
       q_tile[2 * tid] = q_re * c_ - q_im * s_;
       q_tile[2 * tid + 1] = q_re * s_ + q_im * c_;
     }
-    // ---- K'(t) has landed (V'(t) may still be in flight); the next K' tile goes out
-    cp_async_wait<1>();
-    fence_async_smem();
-    __syncthreads();
+    // ---- lift: X = K'(t) (U^K)^T; then K'(t+1) may replace K'(t)
     if (tid == 0) {
-      tc_fence_after();
-      const uint32_t ka = smem_u32(Kt), ua = smem_u32(Us);
-      for (int part_i = 0; part_i < 2; ++part_i)             // U^K high part, then low part
+      ok = mbar_wait(&hdr->k_full, par, p.status);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t ka = smem_u32(Ks), ua = smem_u32(Us);
         for (int s = 0; s < ks_steps; ++s)
-          mma_ss(tmem, smem_desc(ka + s * 256, 128, grp_k), smem_desc(ua + part_i * u_bytes + s * 256, 128, grp_k),
-                 idesc, part_i > 0 || s > 0);
-      mma_commit(&hdr->mma_done);
+          mma_ss(tmem, smem_desc_sw128(ka + (s >> 2) * kAtom + (s & 3) * 32, 16, 1024), smem_desc(ua + s * 256, 128, grp_k),
+                 idesc, s > 0);
+        mma_commit(&hdr->mma_done);
+        ok = mbar_wait(&hdr->mma_done, par, p.status);
+        if (ok && t + 1 < t_hi) fetch_k(t + 1);
+      }
+      if (!ok) *abort_flag = 1;
     }
-    // (cp.async groups in flight here: V'(t), then K'(t+1))
-    if (t + 1 < t_hi) {
-      const int rows1 = min(kTile, p.n - (t + 1) * kTile);
-      load_canonical_async(Ks + (buf ^ 1) * k_bytes, Kg + static_cast<int64_t>(t + 1) * kTile * hd.rp_k, hd.rp_k, rows1,
-                           nch_k, tid);
-    }
-    cp_async_commit();
-    // ---- X = K' (U^K)^T is in TMEM: score of this thread's row
-    ok = mbar_wait(&hdr->mma_done, (t - t_lo) & 1u, p.status);
-    ok = !__syncthreads_or(!ok || *abort_flag);
-    if (!ok) break;
+    __syncthreads();                                         // q_tile written, X complete (thread 0 waited for it)
+    if (*abort_flag) { ok = false; break; }
     tc_fence_after();
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
@@ -209,8 +197,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
           }
           const float2 qt = *reinterpret_cast<const float2*>(q_tile + 2 * (c0 + i));
           // W = Q_t conj(E_l); pair term = Re(W conj(X)) = W_re x_re + W_im x_im
-          const float w_re = fmaf(qt.x, el_c[c0 + i], qt.y * el_s[c0 + i]);
-          const float w_im = fmaf(qt.y, el_c[c0 + i], -qt.x * el_s[c0 + i]);
+          float w_re, w_im;
+          fma2(w_re, w_im, qt.x, qt.y, el_c[c0 + i], 0.f);                       // (Qr c, Qi c)
+          w_re = fmaf(qt.y, el_s[c0 + i], w_re);
+          w_im = fmaf(-qt.x, el_s[c0 + i], w_im);
           s0 = fmaf(w_re, x_re, s0);
           s1 = fmaf(w_im, x_im, s1);
         }
@@ -218,45 +208,44 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     }
     const int j = t * kTile + tid;
     const bool live = j < p.n;
-    float s = live ? s0 + s1 : -INFINITY;
+    const float s = live ? s0 + s1 : -INFINITY;
     // ---- online softmax over the tile: block maximum, weights, running sum per thread
     float mx = s;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (lane == 0) hdr->red[warp] = mx;
-    cp_async_wait<1>();                                      // V'(t) has landed (K'(t+1) may be in flight)
-    __syncthreads();
+    tc_fence_before();
+    __syncthreads();                                         // every thread has read its row of X
     const float m_new = fmaxf(m_run, fmaxf(fmaxf(hdr->red[0], hdr->red[1]), fmaxf(hdr->red[2], hdr->red[3])));
     const float alpha = ex2(m_run - m_new);                  // 0 at the first tile
     m_run = m_new;
     const float pj = live ? ex2(s - m_new) : 0.f;
     l_thr = fmaf(l_thr, alpha, pj);
     p_row[tid] = pj;
+    if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
     __syncthreads();
-    // ---- o'[c] = alpha o'[c] + sum_j p_j V'[j][c], thread c = tid
+    if (*abort_flag) { ok = false; break; }
+    // ---- o'[c] = alpha o'[c] + sum_j p_j V'[j][c], thread c = tid; element (j, c) of the swizzled tile sits in
+    //      atom column c / 64, row j, 16-byte chunk ((c % 64) / 8) ^ (j % 8)
     if (tid < hd.rp_v) {
-      const __nv_bfloat16* vcol = reinterpret_cast<const __nv_bfloat16*>(Vs) + tid;
+      const unsigned char* vbase = Vs + (tid >> 6) * kAtom + (tid & 7) * 2;
+      const int chunk = (tid & 63) >> 3;
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 4
-      for (int r = 0; r < kTile; r += 4) {
-        const float4 pr = *reinterpret_cast<const float4*>(p_row + r);
-        a0 = fmaf(pr.x, __bfloat162float(vcol[(r + 0) * hd.rp_v]), a0);
-        a1 = fmaf(pr.y, __bfloat162float(vcol[(r + 1) * hd.rp_v]), a1);
-        a2 = fmaf(pr.z, __bfloat162float(vcol[(r + 2) * hd.rp_v]), a2);
-        a3 = fmaf(pr.w, __bfloat162float(vcol[(r + 3) * hd.rp_v]), a3);
+#pragma unroll 2
+      for (int r = 0; r < kTile; r += 8) {
+        const float4 pa = *reinterpret_cast<const float4*>(p_row + r);
+        const float4 pb = *reinterpret_cast<const float4*>(p_row + r + 4);
+        const unsigned char* vr = vbase + r * 128;
+#define EA_V(jj) __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vr + (jj) * 128 + ((chunk ^ (jj)) << 4)))
+        a0 = fmaf(pa.x, EA_V(0), a0); a1 = fmaf(pa.y, EA_V(1), a1); a2 = fmaf(pa.z, EA_V(2), a2); a3 = fmaf(pa.w, EA_V(3), a3);
+        a0 = fmaf(pb.x, EA_V(4), a0); a1 = fmaf(pb.y, EA_V(5), a1); a2 = fmaf(pb.z, EA_V(6), a2); a3 = fmaf(pb.w, EA_V(7), a3);
+#undef EA_V
       }
       o_acc = fmaf(o_acc, alpha, (a0 + a1) + (a2 + a3));
     }
-    tc_fence_before();
-    __syncthreads();                                         // V' tile and TMEM rows are free again
-    if (t + 1 < t_hi) {
-      const int rows1 = min(kTile, p.n - (t + 1) * kTile);
-      load_rows_async(Vs, Vg + static_cast<int64_t>(t + 1) * kTile * hd.rp_v, hd.rp_v, rows1, tid);
-    }
-    cp_async_commit();
-    // (groups in flight: K'(t+1), then V'(t+1))
+    __syncthreads();                                         // the V' tile is free again
+    if (tid == 0 && t + 1 < t_hi) fetch_v(t + 1);
   }
-  cp_async_wait<0>();
   if (!ok) *abort_flag = 1;
 
   // ---- the piece's partial: m, l (sum over the threads' rows), o'
@@ -311,7 +300,7 @@ __global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParam
 
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
   const size_t k16 = (max_rp_k + 15) & ~15;
-  return 2048 + 2 * static_cast<size_t>(d_head) * k16 * 2 + 2 * kTile * k16 * 2 + static_cast<size_t>(kTile) * max_rp_v * 2;
+  return 2048 + static_cast<size_t>(d_head) * k16 * 2 + (((k16 + 63) >> 6) + ((max_rp_v + 63) >> 6)) * static_cast<size_t>(kAtom);
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
