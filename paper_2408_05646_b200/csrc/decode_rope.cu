@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     return;
   }
 
-  if (warp == 0) tmem_alloc(&hdr->tmem_base, 128);
+  if (warp == 0) tmem_alloc(&hdr->tmem_base, 256);           // two accumulators: X(t) is read while X(t+1) is computed
   if (tid == 0) {
     mbar_init(&hdr->mma_done, 1);
     mbar_init(&hdr->k_full, 1);
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     fetch_v(t_lo);
   }
   const uint32_t tmem = hdr->tmem_base;
-  const uint32_t tX = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+  const uint32_t tX0 = tmem + (static_cast<uint32_t>(warp * 32) << 16);
   volatile int* abort_flag = &hdr->abort_flag;
   const uint32_t idesc = instr_desc(p.d_head, false);
   const int ks_steps = rpk16 >> 4;
@@ -142,8 +142,23 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
 
   float m_run = -INFINITY, l_thr = 0.f, o_acc = 0.f;         // o_acc: column tid of o'
   bool ok = true;
+  // lift of one tile (thread 0): X = K' (U^K)^T into accumulator `acc`
+  auto issue_lift = [&](int acc) {
+    tc_fence_after();
+    const uint32_t ka = smem_u32(Ks), ua = smem_u32(Us);
+    for (int s = 0; s < ks_steps; ++s)
+      mma_ss(tmem + acc * kTile, smem_desc_sw128(ka + (s >> 2) * kAtom + (s & 3) * 32, 16, 1024),
+             smem_desc(ua + s * 256, 128, grp_k), idesc, s > 0);
+    mma_commit(&hdr->mma_done);
+  };
+  if (tid == 0) {
+    ok = mbar_wait(&hdr->k_full, 0, p.status);
+    if (ok) issue_lift(0);
+    else *abort_flag = 1;
+  }
   for (int t = t_lo; t < t_hi && ok; ++t) {
     const uint32_t par = (t - t_lo) & 1u;
+    const uint32_t tX = tX0 + par * kTile;
     // ---- the query pairs turned by (pos_q - 128 t) phi, angle reduced in fp64
     if (tid < half) {
       const double ang = static_cast<double>(pos_q - t * kTile) * my_freq;
@@ -153,22 +168,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
       q_tile[2 * tid] = q_re * c_ - q_im * s_;
       q_tile[2 * tid + 1] = q_re * s_ + q_im * c_;
     }
-    // ---- lift: X = K'(t) (U^K)^T; then K'(t+1) may replace K'(t)
-    if (tid == 0) {
-      ok = mbar_wait(&hdr->k_full, par, p.status);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t ka = smem_u32(Ks), ua = smem_u32(Us);
-        for (int s = 0; s < ks_steps; ++s)
-          mma_ss(tmem, smem_desc_sw128(ka + (s >> 2) * kAtom + (s & 3) * 32, 16, 1024), smem_desc(ua + s * 256, 128, grp_k),
-                 idesc, s > 0);
-        mma_commit(&hdr->mma_done);
-        ok = mbar_wait(&hdr->mma_done, par, p.status);
-        if (ok && t + 1 < t_hi) fetch_k(t + 1);
-      }
-      if (!ok) *abort_flag = 1;
-    }
-    __syncthreads();                                         // q_tile written, X complete (thread 0 waited for it)
+    // ---- X(t) is complete (its lift went out during the previous tile): K'(t+1) may replace K'(t)
+    if (!mbar_wait(&hdr->mma_done, par, p.status)) *abort_flag = 1;
+    if (tid == 0 && t + 1 < t_hi) fetch_k(t + 1);
+    __syncthreads();                                         // q_tile written
     if (*abort_flag) { ok = false; break; }
     tc_fence_after();
     float s0 = 0.f, s1 = 0.f;
@@ -205,6 +208,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
           s1 = fmaf(w_im, x_im, s1);
         }
       }
+    }
+    // ---- K'(t+1) has had the score phase to land: its lift runs during the softmax and the weighted sum
+    if (tid == 0 && t + 1 < t_hi) {
+      if (mbar_wait(&hdr->k_full, par ^ 1u, p.status)) issue_lift(static_cast<int>(par ^ 1u));
+      else *abort_flag = 1;
     }
     const int j = t * kTile + tid;
     const bool live = j < p.n;
@@ -261,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   if (tid < hd.rp_v) part[4 + tid] = o_acc;
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 128);
+  if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
 // Merges the partials of a unit and lifts o'/l through (U^V)^T (or writes the rank-space row).
