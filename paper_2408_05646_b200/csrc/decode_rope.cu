@@ -40,6 +40,7 @@ struct __align__(16) RopeSmemHeader {
   float pad_[3];
 };
 
+template <bool INTERLEAVED>
 __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
@@ -54,7 +55,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const int u_bytes = p.d_head * rpk16 * 2;                  // bf16 image of U^K (the high part of the stored pair)
   const int half = p.d_head >> 1;
 
-  float* q_tile = reinterpret_cast<float*>(smem + 256);      // [d_head]: (re, im) of the query pairs for this tile
+  float* q_tile = reinterpret_cast<float*>(smem + 256);      // the query pairs for this tile: re[64], then im[64]
   float* p_row = q_tile + 128;                               // [128] softmax weights of the tile
   unsigned char* tiles = smem + 2048;
   unsigned char* Ks = tiles;                                 // one K' tile, swizzled atom columns of 128 rows
@@ -103,20 +104,21 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   };
 
   // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
-  float el_c[64], el_s[64];
+  unsigned long long el_c[32], el_s[32];                     // pairs (2k, 2k+1) packed: (cos, cos), (sin, sin)
 #pragma unroll
-  for (int i = 0; i < 64; ++i) {
-    float s_, c_;
-    sincosf(static_cast<float>(tid) * static_cast<float>(i < half ? p.inv_freq[i] : 0.0), &s_, &c_);
-    el_c[i] = c_;
-    el_s[i] = s_;
+  for (int k = 0; k < 32; ++k) {
+    float s0_, c0_, s1_, c1_;
+    sincosf(static_cast<float>(tid) * static_cast<float>(2 * k < half ? p.inv_freq[2 * k] : 0.0), &s0_, &c0_);
+    sincosf(static_cast<float>(tid) * static_cast<float>(2 * k + 1 < half ? p.inv_freq[2 * k + 1] : 0.0), &s1_, &c1_);
+    el_c[k] = pack2(c0_, c1_);
+    el_s[k] = pack2(s0_, s1_);
   }
   // the query of this unit, scaled by log2(e)/sqrt(d_h): thread i < half owns pair i
   float q_re = 0.f, q_im = 0.f;
   double my_freq = 0.0;
   if (tid < half) {
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head;
-    const int ia = p.interleaved ? 2 * tid : tid, ib = p.interleaved ? 2 * tid + 1 : tid + half;
+    const int ia = INTERLEAVED ? 2 * tid : tid, ib = INTERLEAVED ? 2 * tid + 1 : tid + half;
     q_re = __bfloat162float(qg[ia]) * p.q_scale;
     q_im = __bfloat162float(qg[ib]) * p.q_scale;
     my_freq = p.inv_freq[tid];
@@ -165,8 +167,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
       const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
       float s_, c_;
       sincosf(static_cast<float>(red), &s_, &c_);
-      q_tile[2 * tid] = q_re * c_ - q_im * s_;
-      q_tile[2 * tid + 1] = q_re * s_ + q_im * c_;
+      q_tile[tid] = q_re * c_ - q_im * s_;
+      q_tile[64 + tid] = q_re * s_ + q_im * c_;
     }
     // ---- X(t) is complete (its lift went out during the previous tile): K'(t+1) may replace K'(t)
     if (!mbar_wait(&hdr->mma_done, par, p.status)) *abort_flag = 1;
@@ -174,12 +176,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     __syncthreads();                                         // q_tile written
     if (*abort_flag) { ok = false; break; }
     tc_fence_after();
-    float s0 = 0.f, s1 = 0.f;
+    // two pairs per packed instruction: W = Q_t conj(E_l), pair term = Re(W conj(X)) = W_re x_re + W_im x_im
+    unsigned long long acc_re = 0ull, acc_im = 0ull;         // (0.f, 0.f)
 #pragma unroll
     for (int c0 = 0; c0 < 64; c0 += 16) {
       if (c0 < half) {
         uint32_t xa[16], xb[16];
-        if (p.interleaved) {                                 // pairs (2i, 2i+1): columns 2 c0 .. 2 c0 + 31
+        if (INTERLEAVED) {                                   // pairs (2i, 2i+1): columns 2 c0 .. 2 c0 + 31
           tmem_ld16(tX + 2 * c0, xa);
           tmem_ld16(tX + 2 * c0 + 16, xb);
         } else {                                             // pairs (i, i + d_h/2)
@@ -188,27 +191,31 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
         }
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float x_re, x_im;
-          if (p.interleaved) {
+        for (int i = 0; i < 16; i += 2) {
+          unsigned long long x_re, x_im;
+          if (INTERLEAVED) {
             const uint32_t* src = i < 8 ? xa : xb;
-            x_re = __uint_as_float(src[(2 * i) & 15]);
-            x_im = __uint_as_float(src[(2 * i + 1) & 15]);
+            x_re = pack2(__uint_as_float(src[(2 * i) & 15]), __uint_as_float(src[(2 * i + 2) & 15]));
+            x_im = pack2(__uint_as_float(src[(2 * i + 1) & 15]), __uint_as_float(src[(2 * i + 3) & 15]));
           } else {
-            x_re = __uint_as_float(xa[i]);
-            x_im = __uint_as_float(xb[i]);
+            x_re = pack2(__uint_as_float(xa[i]), __uint_as_float(xa[i + 1]));
+            x_im = pack2(__uint_as_float(xb[i]), __uint_as_float(xb[i + 1]));
           }
-          const float2 qt = *reinterpret_cast<const float2*>(q_tile + 2 * (c0 + i));
-          // W = Q_t conj(E_l); pair term = Re(W conj(X)) = W_re x_re + W_im x_im
-          float w_re, w_im;
-          fma2(w_re, w_im, qt.x, qt.y, el_c[c0 + i], 0.f);                       // (Qr c, Qi c)
-          w_re = fmaf(qt.y, el_s[c0 + i], w_re);
-          w_im = fmaf(-qt.x, el_s[c0 + i], w_im);
-          s0 = fmaf(w_re, x_re, s0);
-          s1 = fmaf(w_im, x_im, s1);
+          const unsigned long long qr = *reinterpret_cast<const unsigned long long*>(q_tile + c0 + i);
+          const unsigned long long qi = *reinterpret_cast<const unsigned long long*>(q_tile + 64 + c0 + i);
+          const unsigned long long ec = el_c[(c0 + i) >> 1], es = el_s[(c0 + i) >> 1];
+          const unsigned long long w_re = fma2p(qi, es, mul2p(qr, ec));                  // Qr c + Qi s
+          const unsigned long long w_im = fma2p(qr ^ 0x8000000080000000ull, es, mul2p(qi, ec));   // Qi c - Qr s
+          acc_re = fma2p(w_re, x_re, acc_re);
+          acc_im = fma2p(w_im, x_im, acc_im);
         }
       }
     }
+    float s0, s1, s2, s3;
+    unpack2(acc_re, s0, s1);
+    unpack2(acc_im, s2, s3);
+    s0 += s2;
+    s1 += s3;
     // ---- K'(t+1) has had the score phase to land: its lift runs during the softmax and the weighted sum
     if (tid == 0 && t + 1 < t_hi) {
       if (mbar_wait(&hdr->k_full, par ^ 1u, p.status)) issue_lift(static_cast<int>(par ^ 1u));
@@ -314,13 +321,16 @@ size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
   static size_t configured = 0;
   if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
+    cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(decode_rope_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     configured = smem;
   }
   dim3 grid(p.B * p.H, p.splits);
-  decode_rope_kernel<<<grid, kThreads, smem, s>>>(p);
+  if (p.interleaved) decode_rope_kernel<true><<<grid, kThreads, smem, s>>>(p);
+  else decode_rope_kernel<false><<<grid, kThreads, smem, s>>>(p);
   ++*launches;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
