@@ -11,7 +11,8 @@
 // pair's frequency phi, the rotated dot product of the pair is Re(Q e^{i p phi} conj(X e^{i j phi})) =
 // Re(Q e^{i (p - j) phi} conj(X)).  For row l of tile t, p - j = D_t - l with D_t = p - 128 t, so
 // e^{i (p-j) phi} = e^{i D_t phi} conj(e^{i l phi}): the first factor is applied to the query once per tile
-// (64 threads, angle reduced in fp64), the second is a per-thread constant held in registers.
+// (64 threads; the first tile's angle is reduced in fp64, every further tile turns the query by the constant
+// e^{-i 128 phi}, one complex multiplication, renormalised), the second is a per-thread constant in registers.
 //
 // One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  One
 // thread fetches the K' and V' tiles by TMA (the tensor maps of the cache slabs, 64 x 64 boxes, 128-byte
@@ -114,14 +115,21 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     el_s[k] = pack2(s0_, s1_);
   }
   // the query of this unit, scaled by log2(e)/sqrt(d_h): thread i < half owns pair i
-  float q_re = 0.f, q_im = 0.f;
-  double my_freq = 0.0;
+  // turned to the first tile's offset here (fp64 once), then by (step_c, step_s) = e^{-i 128 phi} per tile
+  float q_re = 0.f, q_im = 0.f, step_c = 1.f, step_s = 0.f, q_norm2 = 0.f;
   if (tid < half) {
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head;
     const int ia = INTERLEAVED ? 2 * tid : tid, ib = INTERLEAVED ? 2 * tid + 1 : tid + half;
-    q_re = __bfloat162float(qg[ia]) * p.q_scale;
-    q_im = __bfloat162float(qg[ib]) * p.q_scale;
-    my_freq = p.inv_freq[tid];
+    const float a_re = __bfloat162float(qg[ia]) * p.q_scale, a_im = __bfloat162float(qg[ib]) * p.q_scale;
+    const double freq = p.inv_freq[tid];
+    double s_, c_;
+    sincos(static_cast<double>(p.n - 1 - t_lo * kTile) * freq, &s_, &c_);
+    q_re = static_cast<float>(a_re * c_ - a_im * s_);
+    q_im = static_cast<float>(a_re * s_ + a_im * c_);
+    q_norm2 = a_re * a_re + a_im * a_im;
+    sincos(-static_cast<double>(kTile) * freq, &s_, &c_);
+    step_c = static_cast<float>(c_);
+    step_s = static_cast<float>(s_);
   }
 
   cp_async_wait<0>();
@@ -142,7 +150,16 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const int ks_steps = rpk16 >> 4;
   const int pos_q = p.n - 1;
 
-  float m_run = -INFINITY, l_thr = 0.f, o_acc = 0.f;         // o_acc: column tid of o'
+  // weighted sum o' += p V': thread (g, c) owns the column pair (2c, 2c+1) over the rows of row group g of every
+  // tile; the groups are added up once, at the end
+  const int col_pairs = hd.rp_v >> 1;
+  const int row_groups = min(kThreads / col_pairs, 16);
+  const int rows_per_group = (kTile + row_groups - 1) / row_groups;
+  const int pv_g = tid / col_pairs, pv_c = tid - pv_g * col_pairs;
+  const int r_lo = min(kTile, pv_g * rows_per_group), r_hi = pv_g < row_groups ? min(kTile, r_lo + rows_per_group) : r_lo;
+  const unsigned char* v_col = Vs + ((2 * pv_c) >> 6) * kAtom + ((2 * pv_c) & 7) * 2;
+  const int v_chunk = ((2 * pv_c) & 63) >> 3;
+  float m_run = -INFINITY, l_thr = 0.f, o_acc0 = 0.f, o_acc1 = 0.f;
   bool ok = true;
   // lift of one tile (thread 0): X = K' (U^K)^T into accumulator `acc`
   auto issue_lift = [&](int acc) {
@@ -161,14 +178,16 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   for (int t = t_lo; t < t_hi && ok; ++t) {
     const uint32_t par = (t - t_lo) & 1u;
     const uint32_t tX = tX0 + par * kTile;
-    // ---- the query pairs turned by (pos_q - 128 t) phi, angle reduced in fp64
+    // ---- the query pairs turned by (pos_q - 128 t) phi
     if (tid < half) {
-      const double ang = static_cast<double>(pos_q - t * kTile) * my_freq;
-      const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
-      float s_, c_;
-      sincosf(static_cast<float>(red), &s_, &c_);
-      q_tile[tid] = q_re * c_ - q_im * s_;
-      q_tile[64 + tid] = q_re * s_ + q_im * c_;
+      q_tile[tid] = q_re;
+      q_tile[64 + tid] = q_im;
+      // the next tile's query: one more turn by -128 phi; the length is pulled back to |q| so that rounding
+      // does not drift over a thousand tiles
+      const float n_re = q_re * step_c - q_im * step_s, n_im = q_re * step_s + q_im * step_c;
+      const float fix = 1.5f - 0.5f * (n_re * n_re + n_im * n_im) / fmaxf(q_norm2, 1e-30f);   // ~ |q| / |n|
+      q_re = n_re * fix;
+      q_im = n_im * fix;
     }
     // ---- X(t) is complete (its lift went out during the previous tile): K'(t+1) may replace K'(t)
     if (!mbar_wait(&hdr->mma_done, par, p.status)) *abort_flag = 1;
@@ -240,23 +259,28 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
     __syncthreads();
     if (*abort_flag) { ok = false; break; }
-    // ---- o'[c] = alpha o'[c] + sum_j p_j V'[j][c], thread c = tid; element (j, c) of the swizzled tile sits in
-    //      atom column c / 64, row j, 16-byte chunk ((c % 64) / 8) ^ (j % 8)
-    if (tid < hd.rp_v) {
-      const unsigned char* vbase = Vs + (tid >> 6) * kAtom + (tid & 7) * 2;
-      const int chunk = (tid & 63) >> 3;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 2
-      for (int r = 0; r < kTile; r += 8) {
-        const float4 pa = *reinterpret_cast<const float4*>(p_row + r);
-        const float4 pb = *reinterpret_cast<const float4*>(p_row + r + 4);
-        const unsigned char* vr = vbase + r * 128;
-#define EA_V(jj) __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vr + (jj) * 128 + ((chunk ^ (jj)) << 4)))
-        a0 = fmaf(pa.x, EA_V(0), a0); a1 = fmaf(pa.y, EA_V(1), a1); a2 = fmaf(pa.z, EA_V(2), a2); a3 = fmaf(pa.w, EA_V(3), a3);
-        a0 = fmaf(pb.x, EA_V(4), a0); a1 = fmaf(pb.y, EA_V(5), a1); a2 = fmaf(pb.z, EA_V(6), a2); a3 = fmaf(pb.w, EA_V(7), a3);
-#undef EA_V
+    // ---- o' = alpha o' + sum_j p_j V'[j][2c..2c+1] over this thread's rows; element (j, c) of the swizzled tile
+    //      sits in atom column c / 64, row j, 16-byte chunk ((c % 64) / 8) ^ (j % 8)
+    {
+      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+      int r = r_lo;
+      for (; r + 1 < r_hi; r += 2) {
+        const uint32_t va = *reinterpret_cast<const uint32_t*>(v_col + r * 128 + ((v_chunk ^ (r & 7)) << 4));
+        const uint32_t vb = *reinterpret_cast<const uint32_t*>(v_col + (r + 1) * 128 + ((v_chunk ^ ((r + 1) & 7)) << 4));
+        const float pa = p_row[r], pb = p_row[r + 1];
+        a0 = fmaf(pa, __uint_as_float(va << 16), a0);
+        a1 = fmaf(pa, __uint_as_float(va & 0xffff0000u), a1);
+        b0 = fmaf(pb, __uint_as_float(vb << 16), b0);
+        b1 = fmaf(pb, __uint_as_float(vb & 0xffff0000u), b1);
       }
-      o_acc = fmaf(o_acc, alpha, (a0 + a1) + (a2 + a3));
+      if (r < r_hi) {
+        const uint32_t va = *reinterpret_cast<const uint32_t*>(v_col + r * 128 + ((v_chunk ^ (r & 7)) << 4));
+        const float pa = p_row[r];
+        a0 = fmaf(pa, __uint_as_float(va << 16), a0);
+        a1 = fmaf(pa, __uint_as_float(va & 0xffff0000u), a1);
+      }
+      o_acc0 = fmaf(o_acc0, alpha, a0 + b0);
+      o_acc1 = fmaf(o_acc1, alpha, a1 + b1);
     }
     __syncthreads();                                         // the V' tile is free again
     if (tid == 0 && t + 1 < t_hi) fetch_v(t + 1);
@@ -273,7 +297,18 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     part[0] = m_run;
     part[1] = (hdr->red[4] + hdr->red[5]) + (hdr->red[6] + hdr->red[7]);
   }
-  if (tid < hd.rp_v) part[4 + tid] = o_acc;
+  // add up the row groups (the V' tile's shared memory is free now)
+  float* o_red = reinterpret_cast<float*>(Vs);
+  if (pv_g < row_groups) {
+    o_red[pv_g * hd.rp_v + 2 * pv_c] = o_acc0;
+    o_red[pv_g * hd.rp_v + 2 * pv_c + 1] = o_acc1;
+  }
+  __syncthreads();
+  if (tid < hd.rp_v) {
+    float o = 0.f;
+    for (int g = 0; g < row_groups; ++g) o += o_red[g * hd.rp_v + tid];
+    part[4 + tid] = o;
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, 256);
