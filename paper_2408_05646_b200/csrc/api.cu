@@ -326,15 +326,27 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;
-  // CTAs per unit: fill the machine a few times over, within the partials the workspace holds
+  // CTAs per unit.  The CTAs run in waves of (SMs x CTAs per SM) and each one pays a start-up (trigonometric
+  // constants, the U^K image) worth about ten tiles: take the split count with the least waves x (tiles + start-up),
+  // within the partials the workspace holds.
   const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
-  const int64_t want = (h->opt_ctas > 0 ? h->opt_ctas : 3ll * h->sm_count * ctas_per_sm);
-  int64_t splits = (want + static_cast<int64_t>(B) * H - 1) / (static_cast<int64_t>(B) * H);
-  const int64_t cap = (static_cast<int64_t>(B) * H + kMaxDecodeCtas) / (static_cast<int64_t>(B) * H);
-  if (splits > cap) splits = cap;
-  if (splits > p.nt) splits = p.nt;
-  if (splits < 1) splits = 1;
-  if (splits > 65535) splits = 65535;
+  const int64_t units = static_cast<int64_t>(B) * H;
+  int64_t cap = (units + kMaxDecodeCtas) / units;
+  if (cap > p.nt) cap = p.nt;
+  if (cap > 65535) cap = 65535;
+  if (cap < 1) cap = 1;
+  int64_t splits = 1;
+  if (h->opt_ctas > 0) {
+    splits = (h->opt_ctas + units - 1) / units;
+    if (splits > cap) splits = cap;
+  } else {
+    const int64_t wave = static_cast<int64_t>(h->sm_count) * ctas_per_sm;
+    int64_t best = INT64_MAX;
+    for (int64_t s2 = 1; s2 <= cap && s2 <= 256; ++s2) {
+      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 10);
+      if (cost < best) { best = cost; splits = s2; }
+    }
+  }
   p.splits = static_cast<int32_t>(splits);
   p.interleaved = h->rope_interleaved;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));

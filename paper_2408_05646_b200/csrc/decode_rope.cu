@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   // tile; the groups are added up once, at the end
   const int col_pairs = hd.rp_v >> 1;
   const int row_groups = min(kThreads / col_pairs, 16);
-  const int rows_per_group = (kTile + row_groups - 1) / row_groups;
+  const int rows_per_group = (((kTile + row_groups - 1) / row_groups) + 7) & ~7;   // whole blocks of 8 rows
   const int pv_g = tid / col_pairs, pv_c = tid - pv_g * col_pairs;
   const int r_lo = min(kTile, pv_g * rows_per_group), r_hi = pv_g < row_groups ? min(kTile, r_lo + rows_per_group) : r_lo;
   const unsigned char* v_col = Vs + ((2 * pv_c) >> 6) * kAtom + ((2 * pv_c) & 7) * 2;
@@ -162,12 +162,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   float m_run = -INFINITY, l_thr = 0.f, o_acc0 = 0.f, o_acc1 = 0.f;
   bool ok = true;
   // lift of one tile (thread 0): X = K' (U^K)^T into accumulator `acc`
+  const uint64_t desc_k = smem_desc_sw128(smem_u32(Ks), 16, 1024), desc_u = smem_desc(smem_u32(Us), 128, grp_k);
   auto issue_lift = [&](int acc) {
     tc_fence_after();
-    const uint32_t ka = smem_u32(Ks), ua = smem_u32(Us);
-    for (int s = 0; s < ks_steps; ++s)
-      mma_ss(tmem + acc * kTile, smem_desc_sw128(ka + (s >> 2) * kAtom + (s & 3) * 32, 16, 1024),
-             smem_desc(ua + s * 256, 128, grp_k), idesc, s > 0);
+    for (int s = 0; s < ks_steps; ++s)                       // 16 rank elements a step: 32 bytes along the swizzled
+      mma_ss(tmem + acc * kTile, desc_k + (s >> 2) * (kAtom >> 4) + (s & 3) * 2, desc_u + s * 16, idesc, s > 0);   // rows
     mma_commit(&hdr->mma_done);
   };
   if (tid == 0) {
@@ -263,21 +262,21 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     //      sits in atom column c / 64, row j, 16-byte chunk ((c % 64) / 8) ^ (j % 8)
     {
       float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-      int r = r_lo;
-      for (; r + 1 < r_hi; r += 2) {
-        const uint32_t va = *reinterpret_cast<const uint32_t*>(v_col + r * 128 + ((v_chunk ^ (r & 7)) << 4));
-        const uint32_t vb = *reinterpret_cast<const uint32_t*>(v_col + (r + 1) * 128 + ((v_chunk ^ ((r + 1) & 7)) << 4));
-        const float pa = p_row[r], pb = p_row[r + 1];
-        a0 = fmaf(pa, __uint_as_float(va << 16), a0);
-        a1 = fmaf(pa, __uint_as_float(va & 0xffff0000u), a1);
-        b0 = fmaf(pb, __uint_as_float(vb << 16), b0);
-        b1 = fmaf(pb, __uint_as_float(vb & 0xffff0000u), b1);
-      }
-      if (r < r_hi) {
-        const uint32_t va = *reinterpret_cast<const uint32_t*>(v_col + r * 128 + ((v_chunk ^ (r & 7)) << 4));
-        const float pa = p_row[r];
-        a0 = fmaf(pa, __uint_as_float(va << 16), a0);
-        a1 = fmaf(pa, __uint_as_float(va & 0xffff0000u), a1);
+      for (int r = r_lo; r < r_hi; r += 8) {                 // r is a multiple of 8: row r + jj has chunk v_chunk ^ jj
+        const float4 pa = *reinterpret_cast<const float4*>(p_row + r);
+        const float4 pb = *reinterpret_cast<const float4*>(p_row + r + 4);
+        const unsigned char* vr = v_col + r * 128;
+        uint32_t v[8];
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) v[jj] = *reinterpret_cast<const uint32_t*>(vr + jj * 128 + ((v_chunk ^ jj) << 4));
+        a0 = fmaf(pa.x, __uint_as_float(v[0] << 16), a0); a1 = fmaf(pa.x, __uint_as_float(v[0] & 0xffff0000u), a1);
+        b0 = fmaf(pa.y, __uint_as_float(v[1] << 16), b0); b1 = fmaf(pa.y, __uint_as_float(v[1] & 0xffff0000u), b1);
+        a0 = fmaf(pa.z, __uint_as_float(v[2] << 16), a0); a1 = fmaf(pa.z, __uint_as_float(v[2] & 0xffff0000u), a1);
+        b0 = fmaf(pa.w, __uint_as_float(v[3] << 16), b0); b1 = fmaf(pa.w, __uint_as_float(v[3] & 0xffff0000u), b1);
+        a0 = fmaf(pb.x, __uint_as_float(v[4] << 16), a0); a1 = fmaf(pb.x, __uint_as_float(v[4] & 0xffff0000u), a1);
+        b0 = fmaf(pb.y, __uint_as_float(v[5] << 16), b0); b1 = fmaf(pb.y, __uint_as_float(v[5] & 0xffff0000u), b1);
+        a0 = fmaf(pb.z, __uint_as_float(v[6] << 16), a0); a1 = fmaf(pb.z, __uint_as_float(v[6] & 0xffff0000u), a1);
+        b0 = fmaf(pb.w, __uint_as_float(v[7] << 16), b0); b1 = fmaf(pb.w, __uint_as_float(v[7] & 0xffff0000u), b1);
       }
       o_acc0 = fmaf(o_acc0, alpha, a0 + b0);
       o_acc1 = fmaf(o_acc1, alpha, a1 + b1);
