@@ -20,6 +20,8 @@ Q', K', V' of Eq. 6, brute-force Python loops on tiny inputs, closed-form
 special cases, and the numbers the paper prints for cache sizes.  The ALiBi
 bias is pinned by the same library routine given the bias as an additive
 mask, by the geometric-series closed form for a zero query, and by loops.
+Grouped-query decode is pinned by the library routine's own grouped mode and
+by ordinary decode with the K/V heads repeated.
 The RoPE variant (Section 4.3) is pinned by library attention on keys and
 queries rotated with complex arithmetic, by its relative-position invariance,
 by the zero-angle special case and by loops.
@@ -268,6 +270,27 @@ class LayerOracle:
             else:
                 out[(b, h)] = lift(o, self.U_V[h])
                 self.projection_macs += self.d_h * o.shape[0]
+        return out
+
+    # -- grouped-query attention (Section 5.1: Llama-2-70b and Llama-3 share each K/V head among a group of
+    #    query heads): the cache, U^K and U^V belong to the K/V head, every query head of its group uses them
+    def decode_gqa(self, q: np.ndarray, group: int) -> np.ndarray:
+        """q: [B, 1, H*group, d_h], query head hq belongs to K/V head hq // group.  Returns [B, 1, H*group, d_h].
+        Each query head is Eq. 3 in the space of Eq. 7 against its K/V head's rank-r rows."""
+        q = np.asarray(q, dtype=F64).reshape(self.B, self.H * group, self.d_h)
+        assert self.rope is None
+        out = np.zeros((self.B, 1, self.H * group, self.d_h), dtype=F64)
+        for (b, h) in self.units:
+            Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]
+            assert Kp.shape[0] == self.len and self.len > 0
+            for i in range(group):
+                hq = h * group + i
+                qp = to_rank_space(q[b, hq], self.U_K[h])
+                s = (Kp @ qp) / math.sqrt(self.d_h)
+                if self.alibi[h]:
+                    s = s + alibi_bias(self.alibi[h], self.len - 1, self.len)
+                p = softmax_rows(s[None, :])[0]
+                out[b, 0, hq] = lift(p @ Vp, self.U_V[h])
         return out
 
     def decode_dense(self, q: np.ndarray) -> np.ndarray:
