@@ -153,6 +153,16 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
  * single-tile tensor-core kernel (bf16) or the CUDA-core kernel, not the warp-specialised one. */
 ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream);
 
+/* Grouped-query attention (the Llama-2-70b / Llama-3 models of Section 5.1): the layer's n_heads are the K/V
+ * heads; each has `group` query heads, query head hq = kv_head * group + i, which all attend over that K/V
+ * head's rank-r rows with its U^K and are lifted with its U^V (Eq. 7 per query head).  d_q and d_out:
+ * [B][1][n_heads * group][d_head], batch strides in elements.  One pass over the cache serves the whole
+ * group.  1 <= group <= 16; bf16 layers with d_head % 16 == 0 and no position scheme set
+ * (EA_ERR_UNSUPPORTED otherwise); the partials of batch x n_heads x group x splits must fit the workspace
+ * (EA_ERR_CAPACITY).  Attends over the rows the cache holds: append the new token's rows first. */
+ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
+                                int64_t stride_b_out, void* cuda_stream);
+
 /* Section 4.3 + Fig. 6(b) (models with rotary position embedding): from the next call on, decode keeps the
  * query full rank, takes every cached low-dimensional key back to d_head dimensions through (U^K)^T, rotates
  * it by its position (row j of the cache = position j) and the query by position len - 1, and scores them

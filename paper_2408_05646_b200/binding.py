@@ -67,6 +67,7 @@ SYMBOLS = {
     "eigen_attn_set_option": (_i32, [_vp, _i32, _i64]),
     "eigen_attn_set_alibi": (_i32, [_vp, ctypes.POINTER(ctypes.c_float), _vp]),
     "eigen_attn_set_rope": (_i32, [_vp, ctypes.c_double, _i32, _vp]),
+    "eigen_attn_decode_gqa": (_i32, [_vp, _vp, _i64, _i32, _vp, _i64, _vp]),
     "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
     "eigen_attn_version": (_i32, []),
@@ -305,6 +306,17 @@ class EigenAttnLayer:
             assert len(slopes) == self.H
             arr = (ctypes.c_float * self.H)(*[float(x) for x in slopes])
         self._check(lib.eigen_attn_set_alibi(self.handle, arr, _stream_ptr(stream)), "eigen_attn_set_alibi")
+
+    def decode_gqa(self, q: torch.Tensor, group: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """eigen_attn_decode_gqa: q [B][1][H * group][d_head]; the layer's heads are the K/V heads."""
+        assert q.shape == (self.B, 1, self.H * group, self.d_head) and q.dtype == self.torch_dtype
+        assert q.stride(3) == 1 and q.stride(2) == self.d_head
+        if out is None:
+            out = torch.empty((self.B, 1, self.H * group, self.d_head), dtype=self.torch_dtype, device=self.device)
+        assert out.stride(3) == 1 and out.stride(2) == self.d_head
+        self._check(lib.eigen_attn_decode_gqa(self.handle, q.data_ptr(), q.stride(0), int(group), out.data_ptr(),
+                                              out.stride(0), _stream_ptr(stream)), "eigen_attn_decode_gqa")
+        return out
 
     def set_rope(self, base: float, interleaved: bool = False, stream=None) -> None:
         """Rotary position embedding for decode (Section 4.3); base 0 switches it off."""

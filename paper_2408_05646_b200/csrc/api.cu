@@ -761,6 +761,59 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
   return EA_OK;
 }
 
+ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
+                                int64_t stride_b_out, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_gqa: NULL q or out");
+  if (group < 1 || group > 16) return fail(h, EA_ERR_SHAPE, "decode_gqa: group %d (1..16)", group);
+  if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
+  if (h->rope || h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a position scheme set");
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty");
+  const Layout& L = h->L;
+  const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
+  const size_t smem = ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
+  if (smem > static_cast<size_t>(kSmemLimit)) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: tiles do not fit");
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  ea::GqaDecodeParams p{};
+  p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
+  p.q = d_q; p.q_stride_b = stride_b_q; p.out = d_out; p.out_stride_b = stride_b_out;
+  p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
+  p.status = dev_status(h);
+  p.tmaps = h->ws + L.off_tmaps;
+  p.part_stride = L.part_stride;
+  p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
+  p.nt = (n + 127) / 128;
+  p.group = group;
+  // CTAs per unit: waves of (SMs x CTAs per SM), a start-up worth a few tiles per CTA, and room for
+  // units x splits x group partials in the workspace
+  const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
+  const int64_t units = static_cast<int64_t>(B) * H;
+  int64_t cap = (units + kMaxDecodeCtas) / (units * group);
+  if (cap < 1) return fail(h, EA_ERR_CAPACITY, "decode_gqa: batch x heads x group = %lld partials exceed the workspace",
+                           static_cast<long long>(units * group));
+  if (cap > p.nt) cap = p.nt;
+  int64_t splits = 1;
+  if (h->opt_ctas > 0) {
+    splits = (h->opt_ctas + units - 1) / units;
+    if (splits > cap) splits = cap;
+  } else {
+    const int64_t wave = static_cast<int64_t>(h->sm_count) * ctas_per_sm;
+    int64_t best = INT64_MAX;
+    for (int64_t s2 = 1; s2 <= cap && s2 <= 256; ++s2) {
+      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 4);
+      if (cost < best) { best = cost; splits = s2; }
+    }
+  }
+  p.splits = static_cast<int32_t>(splits);
+  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  if (h->ev_start) cudaEventRecord(h->ev_start, s);
+  const cudaError_t e = ea::launch_decode_gqa(p, smem, s, &h->launches);
+  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_gqa launch");
+  return EA_OK;
+}
+
 ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (base == 0.0) {

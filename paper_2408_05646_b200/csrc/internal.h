@@ -149,6 +149,27 @@ struct RopeDecodeParams {    // decode for models with rotary position embedding
   uint32_t flags;
 };
 
+struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` query heads per K/V head
+  const HeadInfo* heads;
+  const float* basis;
+  const char* cache;
+  const void* q;            // [B][1][H * group][d_head]
+  int64_t q_stride_b;
+  void* out;                // [B][1][H * group][d_head]
+  int64_t out_stride_b;
+  float* partials;          // [B*H][splits][group][part_stride]: m, l, pad, pad, o'[rp_v]
+  int* status;
+  const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every K/V head
+  int32_t part_stride;
+  int32_t B, H, d_head;
+  int32_t n, n_max;
+  int32_t nt;               // tiles of 128 rows per unit
+  int32_t splits;           // CTAs per unit
+  int32_t group;            // 1..16
+  float q_scale;            // log2(e) / sqrt(d_head)
+  uint32_t flags;
+};
+
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.
 cudaError_t launch_project_append(const ProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t smem_bytes,
@@ -156,6 +177,8 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
+cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
