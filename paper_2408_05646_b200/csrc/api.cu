@@ -21,6 +21,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxDecodeCtas = 1024;
+constexpr int kPartialSlack = 4;     // the partials area holds this many times (batch x heads + kMaxDecodeCtas) slots
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kInFlightBytes = 120 * 1024;   // target bytes of bulk copies in flight per SM (decode)
 
@@ -108,7 +109,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_heads = off;    off = align_up(off + sizeof(HeadInfo) * H);
   L->off_basis = off;    off = align_up(off + basis * sizeof(float));
   L->off_partials = off;
-  off = align_up(off + (static_cast<size_t>(d->batch) * H + kMaxDecodeCtas) * L->part_stride * sizeof(float));
+  off = align_up(off + (static_cast<size_t>(d->batch) * H + kMaxDecodeCtas) * kPartialSlack * L->part_stride * sizeof(float));
   L->off_counters = off; off = align_up(off + static_cast<size_t>(d->batch) * H * sizeof(int));
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
@@ -331,7 +332,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   // within the partials the workspace holds.
   const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
   const int64_t units = static_cast<int64_t>(B) * H;
-  int64_t cap = (units + kMaxDecodeCtas) / units;
+  int64_t cap = (units + kMaxDecodeCtas) * kPartialSlack / units;
   if (cap > p.nt) cap = p.nt;
   if (cap > 65535) cap = 65535;
   if (cap < 1) cap = 1;
@@ -789,7 +790,7 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   // units x splits x group partials in the workspace
   const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
   const int64_t units = static_cast<int64_t>(B) * H;
-  int64_t cap = (units + kMaxDecodeCtas) / (units * group);
+  int64_t cap = (units + kMaxDecodeCtas) * kPartialSlack / (units * group);
   if (cap < 1) return fail(h, EA_ERR_CAPACITY, "decode_gqa: batch x heads x group = %lld partials exceed the workspace",
                            static_cast<long long>(units * group));
   if (cap > p.nt) cap = p.nt;

@@ -8,10 +8,12 @@
 //                                                       by log2(e)/sqrt(d_h), as bf16 high + low parts (two products)
 //   softmax in base 2, one thread per cached row, g running maxima kept identical in every thread (lazy
 //   reference: a maximum moves only when it grew by more than 8), P rounded to bf16
-//   O' [16(128) x r_v] += P^T [128 x 128 rows] . V'_tile   P^T has the queries as rows; only g of its 128 rows are
-//                                                       ever non-zero
-// K' and V' tiles arrive by TMA (tensor maps of the cache slabs, 128-byte swizzle), one tile of each in flight
-// per CTA, two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that
+//   O' [16(128) x r_v] += P^T [16(128) x 128 rows] . V'_tile   P^T has the queries as rows.  The product has M = 128,
+//                                                       but only 16 rows of P^T exist in shared memory: the other
+//                                                       112 rows of the operand fall on whatever follows (Q', the
+//                                                       tiles: finite numbers) and fill rows of O' nobody reads
+// K' and V' tiles arrive by TMA (tensor maps of the cache slabs, 128-byte swizzle): K'(t+1) once the scores of tile
+// t are done, V'(t+1) (two buffers) once the weighted sum of tile t-1 is done; two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that
 // gqa_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -27,7 +29,7 @@ constexpr int kAtom = kTile * 128;            // one swizzled atom column of a 1
 constexpr int kMaxGroup = 16;                 // query heads per K/V head (N of the score product)
 
 struct __align__(16) GqaSmemHeader {
-  unsigned long long s_done, o_done, k_full, v_full;
+  unsigned long long s_done, o_done, k_full, v_full[2];
   uint32_t tmem_base;
   int abort_flag;
   float pad_[2];
@@ -47,13 +49,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
   const int atoms_k = (rpk16 + 63) >> 6, atoms_v = (hd.rp_v + 63) >> 6;
   const int k_bytes = atoms_k * kAtom, v_bytes = atoms_v * kAtom;
   const int q_bytes = kMaxGroup * rpk16 * 2;                 // one image (high or low part) of Q'
-  const int p_bytes = kTile * kTile * 2;
+  const int p_bytes = kMaxGroup * kTile * 2;                 // the 16 rows of P^T that exist
 
   unsigned char* tiles = smem + 1024;
-  unsigned char* Ks = tiles;                                 // K' tile, swizzled atom columns of 128 rows
-  unsigned char* Vs = Ks + k_bytes;                          // V' tile, same layout
-  unsigned char* Ps = Vs + v_bytes;                          // P^T [128 (queries, g used)][128 rows], canonical
+  unsigned char* Ps = tiles;                                 // P^T [16 queries][128 rows], canonical (two 8-row groups)
   unsigned char* Qs = Ps + p_bytes;                          // Q' images [16][rk16], canonical: high, then low
+  unsigned char* Ks = Qs + 2 * q_bytes;                      // K' tile, swizzled atom columns of 128 rows (1024-aligned)
+  unsigned char* Vs = Ks + k_bytes;                          // two V' tiles, same layout
 
   const int per = (p.nt + p.splits - 1) / p.splits;
   const int t_lo = split * per, t_hi = min(p.nt, t_lo + per);
@@ -71,7 +73,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     mbar_init(&hdr->s_done, 1);
     mbar_init(&hdr->o_done, 1);
     mbar_init(&hdr->k_full, 1);
-    mbar_init(&hdr->v_full, 1);
+    mbar_init(&hdr->v_full[0], 1);
+    mbar_init(&hdr->v_full[1], 1);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -103,11 +106,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
       for (int hf = 0; hf < 2; ++hf)
         tma_load_3d(Ks + a * kAtom + hf * (kAtom / 2), maps, a * 64, t * kTile + hf * 64, b, &hdr->k_full);
   };
-  auto fetch_v = [&](int t) {
-    mbar_arrive_expect_tx(&hdr->v_full, static_cast<uint32_t>(v_bytes));
+  auto fetch_v = [&](int t) {                                // into buffer (t - t_lo) % 2
+    const int vb = (t - t_lo) & 1;
+    mbar_arrive_expect_tx(&hdr->v_full[vb], static_cast<uint32_t>(v_bytes));
     for (int a = 0; a < atoms_v; ++a)
       for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(Vs + a * kAtom + hf * (kAtom / 2), maps + 128, a * 64, t * kTile + hf * 64, b, &hdr->v_full);
+        tma_load_3d(Vs + vb * v_bytes + a * kAtom + hf * (kAtom / 2), maps + 128, a * 64, t * kTile + hf * 64, b,
+                    &hdr->v_full[vb]);
   };
   fence_async_smem();
   tc_fence_before();
@@ -139,6 +144,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     tensormap_acquire(maps + 128);
     fetch_k(t_lo);
     fetch_v(t_lo);
+    if (t_lo + 1 < t_hi) fetch_v(t_lo + 1);
     ok = mbar_wait(&hdr->k_full, 0, p.status);
     if (ok) issue_s(0);
     else *abort_flag = 1;
@@ -154,7 +160,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     if (!mbar_wait(&hdr->s_done, par, p.status)) *abort_flag = 1;
     if (t > t_lo && !mbar_wait(&hdr->o_done, par ^ 1u, p.status)) *abort_flag = 1;
     if (tid == 0 && t + 1 < t_hi) fetch_k(t + 1);
-    if (tid == 0 && t > t_lo) fetch_v(t);                    // (V'(t_lo) went out before the loop)
+    if (tid == 0 && t > t_lo && t + 1 < t_hi) fetch_v(t + 1);   // its buffer was PV(t-1)'s; the first two went out earlier
     tc_fence_after();
     uint32_t sr[16];
     tmem_ld16(tmem + lane_base + 32 * par, sr);
@@ -214,14 +220,14 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     }
     fence_async_smem();
     tc_fence_before();
-    if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
+    if (!mbar_wait(&hdr->v_full[par], ((t - t_lo) >> 1) & 1u, p.status)) *abort_flag = 1;
     __syncthreads();
     if (*abort_flag) { ok = false; break; }
     // ---- O' += P^T V'(t); then S(t+1) as soon as K'(t+1) is there
     if (tid == 0) {
       tc_fence_after();
       for (int s = 0; s < kTile / 16; ++s)                   // 16 cached rows a step
-        mma_ss(tO, desc_p + s * 16, desc_v + s * (2048 >> 4), idesc_o, t > t_lo || s > 0);
+        mma_ss(tO, desc_p + s * 16, desc_v + par * (v_bytes >> 4) + s * (2048 >> 4), idesc_o, t > t_lo || s > 0);
       mma_commit(&hdr->o_done);
       if (t + 1 < t_hi) {
         if (mbar_wait(&hdr->k_full, par ^ 1u, p.status)) issue_s(static_cast<int>(par ^ 1u));
@@ -300,8 +306,10 @@ __global__ void __launch_bounds__(128) gqa_combine_kernel(const GqaDecodeParams 
 
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
   const size_t k16 = (max_rp_k + 15) & ~15;
-  return 1024 + (((k16 + 63) >> 6) + ((max_rp_v + 63) >> 6)) * static_cast<size_t>(kAtom) + kTile * kTile * 2 +
-         2 * kMaxGroup * k16 * 2;
+  // P^T (16 rows), Q' images, one K' tile, two V' tiles; the P^T operand of the weighted sum spans 32 KB from its
+  // start, which the tiles behind it cover
+  return 1024 + kMaxGroup * kTile * 2 + 2 * kMaxGroup * k16 * 2 +
+         (((k16 + 63) >> 6) + 2 * ((max_rp_v + 63) >> 6)) * static_cast<size_t>(kAtom);
 }
 
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {

@@ -67,7 +67,10 @@ WORKLOADS = {
     "opt_6p7b_hetero": Workload(3, "opt_6p7b_hetero", 4, 32, 128, (48, 64, 80, 96, 112), 8192, "bf16", 64, 0.1, 1.0),
     "mpt_7b_long": Workload(4, "mpt_7b_long", 1, 32, 128, (64,), 131072, "bf16", 64, 0.1, 1.0),
     "prefill_b4_t4096": Workload(5, "prefill_b4_t4096", 4, 32, 128, (80,), 4096, "bf16", 64, 0.1, 1.0),
+    # grouped-query layer of the 8B-class models: 8 K/V heads (n_heads), 4 query heads each
+    "llama3_8b_gqa_b16_n32k": Workload(6, "llama3_8b_gqa_b16_n32k", 16, 8, 128, (80,), 32768, "bf16", 64, 0.1, 1.0),
 }
+GQA_GROUP = {"llama3_8b_gqa_b16_n32k": 4}
 
 
 def torch_dtype(name: str) -> torch.dtype:
