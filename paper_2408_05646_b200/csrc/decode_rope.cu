@@ -14,11 +14,13 @@
 // (64 threads; the first tile's angle is reduced in fp64, every further tile turns the query by the constant
 // e^{-i 128 phi}, one complex multiplication, renormalised), the second is a per-thread constant in registers.
 //
-// One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  One
-// thread fetches the K' and V' tiles by TMA (the tensor maps of the cache slabs, 64 x 64 boxes, 128-byte
-// swizzle): K'(t+1) as soon as the lift of tile t has read K'(t), V'(t+1) as soon as tile t's weighted sum
-// is done, so both land behind the arithmetic of the tile in between.  Scores -> online softmax in base 2 ->
-// o' += p V' on the CUDA cores (thread c owns column c and reads the swizzled tile).  A unit split over several CTAs leaves partials (m, l, o') that
+// One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  A tile
+// of K' or V' rows is contiguous in the cache, so each arrives as one bulk copy (cp.async.bulk, the form that
+// reaches the HBM rate in the plain decode kernel; tiled TMA boxes of 128-byte rows were issue-bound at about
+// half of it).  K' lands row-major in a staging buffer, the threads move it into the core-matrix layout the
+// tensor core reads (16-byte chunks, 20 KB a tile), and the staging buffer takes the next tile at once, a whole
+// tile ahead of its use; V' is read row-major where it lands.  Scores -> online softmax in base 2 ->
+// o' += p V' on the CUDA cores (thread (g, c) owns a column pair over a row group).  A unit split over several CTAs leaves partials (m, l, o') that
 // rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -30,7 +32,6 @@ namespace {
 
 using namespace tc;
 
-constexpr int kAtom = kTile * 128;            // one swizzled atom column of a 128-row tile: 64 elements wide
 
 struct __align__(16) RopeSmemHeader {
   unsigned long long mma_done, k_full, v_full;
@@ -51,17 +52,18 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15;
   const int nch_k = rpk16 >> 3, grp_k = nch_k << 7;
-  const int atoms_k = (rpk16 + 63) >> 6, atoms_v = (hd.rp_v + 63) >> 6;
-  const int k_bytes = atoms_k * kAtom, v_bytes = atoms_v * kAtom;
+  const int rowb_k = hd.rp_k * 2, rowb_v = hd.rp_v * 2;      // bytes per cached row
+  const int kst_bytes = kTile * rowb_k, km_bytes = kTile * rpk16 * 2, v_bytes = kTile * rowb_v;
   const int u_bytes = p.d_head * rpk16 * 2;                  // bf16 image of U^K (the high part of the stored pair)
   const int half = p.d_head >> 1;
 
   float* q_tile = reinterpret_cast<float*>(smem + 256);      // the query pairs for this tile: re[64], then im[64]
   float* p_row = q_tile + 128;                               // [128] softmax weights of the tile
   unsigned char* tiles = smem + 2048;
-  unsigned char* Ks = tiles;                                 // one K' tile, swizzled atom columns of 128 rows
-  unsigned char* Vs = Ks + k_bytes;                          // one V' tile, same layout
-  unsigned char* Us = Vs + v_bytes;                          // U^K image, canonical no-swizzle layout
+  unsigned char* Kst = tiles;                                // K' tile as it lands: row-major
+  unsigned char* Km = Kst + kst_bytes;                       // K' tile in the canonical core-matrix layout
+  unsigned char* Vs = Km + km_bytes;                         // V' tile, row-major
+  unsigned char* Us = Vs + v_bytes;                          // U^K image, canonical layout
 
   // tiles [t_lo, t_hi) of the unit
   const int per = (p.nt + p.splits - 1) / p.splits;
@@ -88,20 +90,29 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     for (int idx = tid; idx < u_bytes / 16; idx += kThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
     cp_async_commit();
   }
-  const unsigned char* maps = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
-  // one tile = two boxes of 64 rows per atom column; rows past the current length hold earlier or zero data
-  // and get weight zero, rows past the capacity arrive as zeros
+  // rows that no copy has filled must hold finite numbers: they meet zero weights (a ragged last tile)
+  for (int idx = tid; idx < (kst_bytes + km_bytes + v_bytes) / 16; idx += kThreads)
+    reinterpret_cast<uint4*>(Kst)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  const uint64_t policy = policy_evict_first();
+  const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
+  const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
   auto fetch_k = [&](int t) {
-    mbar_arrive_expect_tx(&hdr->k_full, static_cast<uint32_t>(k_bytes));
-    for (int a = 0; a < atoms_k; ++a)
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(Ks + a * kAtom + hf * (kAtom / 2), maps, a * 64, t * kTile + hf * 64, b, &hdr->k_full);
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_k;
+    mbar_arrive_expect_tx(&hdr->k_full, bytes);
+    bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
   };
   auto fetch_v = [&](int t) {
-    mbar_arrive_expect_tx(&hdr->v_full, static_cast<uint32_t>(v_bytes));
-    for (int a = 0; a < atoms_v; ++a)
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(Vs + a * kAtom + hf * (kAtom / 2), maps + 128, a * 64, t * kTile + hf * 64, b, &hdr->v_full);
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_v;
+    mbar_arrive_expect_tx(&hdr->v_full, bytes);
+    bulk_load(Vs, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
+  };
+  // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * grp_k + c * 128 + (row % 8) * 16
+  auto relayout_k = [&]() {
+    const int chunks = hd.rp_k >> 3;
+    for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
+      const int c = idx >> 7, row = idx & (kTile - 1);
+      *reinterpret_cast<uint4*>(Km + chunk_off(row, c, grp_k)) = *reinterpret_cast<const uint4*>(Kst + row * rowb_k + (c << 4));
+    }
   };
 
   // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
@@ -138,8 +149,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   __syncthreads();
   tc_fence_after();
   if (tid == 0) {
-    tensormap_acquire(maps);
-    tensormap_acquire(maps + 128);
     fetch_k(t_lo);
     fetch_v(t_lo);
   }
@@ -157,22 +166,26 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const int rows_per_group = (((kTile + row_groups - 1) / row_groups) + 7) & ~7;   // whole blocks of 8 rows
   const int pv_g = tid / col_pairs, pv_c = tid - pv_g * col_pairs;
   const int r_lo = min(kTile, pv_g * rows_per_group), r_hi = pv_g < row_groups ? min(kTile, r_lo + rows_per_group) : r_lo;
-  const unsigned char* v_col = Vs + ((2 * pv_c) >> 6) * kAtom + ((2 * pv_c) & 7) * 2;
-  const int v_chunk = ((2 * pv_c) & 63) >> 3;
+  const unsigned char* v_col = Vs + 4 * pv_c;
   float m_run = -INFINITY, l_thr = 0.f, o_acc0 = 0.f, o_acc1 = 0.f;
   bool ok = true;
   // lift of one tile (thread 0): X = K' (U^K)^T into accumulator `acc`
-  const uint64_t desc_k = smem_desc_sw128(smem_u32(Ks), 16, 1024), desc_u = smem_desc(smem_u32(Us), 128, grp_k);
+  const uint64_t desc_k = smem_desc(smem_u32(Km), 128, grp_k), desc_u = smem_desc(smem_u32(Us), 128, grp_k);
   auto issue_lift = [&](int acc) {
     tc_fence_after();
-    for (int s = 0; s < ks_steps; ++s)                       // 16 rank elements a step: 32 bytes along the swizzled
-      mma_ss(tmem + acc * kTile, desc_k + (s >> 2) * (kAtom >> 4) + (s & 3) * 2, desc_u + s * 16, idesc, s > 0);   // rows
+    for (int s = 0; s < ks_steps; ++s)                       // 16 rank elements (two chunks) a step
+      mma_ss(tmem + acc * kTile, desc_k + s * 16, desc_u + s * 16, idesc, s > 0);
     mma_commit(&hdr->mma_done);
   };
-  if (tid == 0) {
-    ok = mbar_wait(&hdr->k_full, 0, p.status);
-    if (ok) issue_lift(0);
-    else *abort_flag = 1;
+  // the first tile: into the core-matrix layout, lift, and the staging buffer takes the second tile
+  if (!mbar_wait(&hdr->k_full, 0, p.status)) *abort_flag = 1;
+  relayout_k();
+  fence_async_smem();
+  __syncthreads();
+  if (*abort_flag) ok = false;
+  if (tid == 0 && ok) {
+    issue_lift(0);
+    if (t_lo + 1 < t_hi) fetch_k(t_lo + 1);
   }
   for (int t = t_lo; t < t_hi && ok; ++t) {
     const uint32_t par = (t - t_lo) & 1u;
@@ -188,9 +201,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
       q_re = n_re * fix;
       q_im = n_im * fix;
     }
-    // ---- X(t) is complete (its lift went out during the previous tile): K'(t+1) may replace K'(t)
+    // ---- X(t) is complete (its lift went out during the previous tile): the core-matrix buffer is free
     if (!mbar_wait(&hdr->mma_done, par, p.status)) *abort_flag = 1;
-    if (tid == 0 && t + 1 < t_hi) fetch_k(t + 1);
     __syncthreads();                                         // q_tile written
     if (*abort_flag) { ok = false; break; }
     tc_fence_after();
@@ -234,10 +246,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     unpack2(acc_im, s2, s3);
     s0 += s2;
     s1 += s3;
-    // ---- K'(t+1) has had the score phase to land: its lift runs during the softmax and the weighted sum
-    if (tid == 0 && t + 1 < t_hi) {
-      if (mbar_wait(&hdr->k_full, par ^ 1u, p.status)) issue_lift(static_cast<int>(par ^ 1u));
-      else *abort_flag = 1;
+    // ---- K'(t+1) landed a tile ago: into the core-matrix layout now, its lift goes out after the barrier below
+    if (t + 1 < t_hi) {
+      if (!mbar_wait(&hdr->k_full, par ^ 1u, p.status)) *abort_flag = 1;
+      relayout_k();
+      fence_async_smem();
     }
     const int j = t * kTile + tid;
     const bool live = j < p.n;
@@ -248,7 +261,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (lane == 0) hdr->red[warp] = mx;
     tc_fence_before();
-    __syncthreads();                                         // every thread has read its row of X
+    __syncthreads();                                         // every thread has read its row of X and moved its chunks
+    if (tid == 0 && t + 1 < t_hi && !*abort_flag) {          // lift of tile t+1 behind the softmax and the weighted sum;
+      issue_lift(static_cast<int>(par ^ 1u));                // the staging buffer takes tile t+2
+      if (t + 2 < t_hi) fetch_k(t + 2);
+    }
     const float m_new = fmaxf(m_run, fmaxf(fmaxf(hdr->red[0], hdr->red[1]), fmaxf(hdr->red[2], hdr->red[3])));
     const float alpha = ex2(m_run - m_new);                  // 0 at the first tile
     m_run = m_new;
@@ -258,17 +275,16 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
     __syncthreads();
     if (*abort_flag) { ok = false; break; }
-    // ---- o' = alpha o' + sum_j p_j V'[j][2c..2c+1] over this thread's rows; element (j, c) of the swizzled tile
-    //      sits in atom column c / 64, row j, 16-byte chunk ((c % 64) / 8) ^ (j % 8)
+    // ---- o' = alpha o' + sum_j p_j V'[j][2c..2c+1] over this thread's rows (row-major tile)
     {
       float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-      for (int r = r_lo; r < r_hi; r += 8) {                 // r is a multiple of 8: row r + jj has chunk v_chunk ^ jj
+      for (int r = r_lo; r < r_hi; r += 8) {
         const float4 pa = *reinterpret_cast<const float4*>(p_row + r);
         const float4 pb = *reinterpret_cast<const float4*>(p_row + r + 4);
-        const unsigned char* vr = v_col + r * 128;
+        const unsigned char* vr = v_col + r * rowb_v;
         uint32_t v[8];
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj) v[jj] = *reinterpret_cast<const uint32_t*>(vr + jj * 128 + ((v_chunk ^ jj) << 4));
+        for (int jj = 0; jj < 8; ++jj) v[jj] = *reinterpret_cast<const uint32_t*>(vr + jj * rowb_v);
         a0 = fmaf(pa.x, __uint_as_float(v[0] << 16), a0); a1 = fmaf(pa.x, __uint_as_float(v[0] & 0xffff0000u), a1);
         b0 = fmaf(pa.y, __uint_as_float(v[1] << 16), b0); b1 = fmaf(pa.y, __uint_as_float(v[1] & 0xffff0000u), b1);
         a0 = fmaf(pa.z, __uint_as_float(v[2] << 16), a0); a1 = fmaf(pa.z, __uint_as_float(v[2] & 0xffff0000u), a1);
@@ -349,7 +365,8 @@ __global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParam
 
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
   const size_t k16 = (max_rp_k + 15) & ~15;
-  return 2048 + static_cast<size_t>(d_head) * k16 * 2 + (((k16 + 63) >> 6) + ((max_rp_v + 63) >> 6)) * static_cast<size_t>(kAtom);
+  // header, U^K image, K' staging + core-matrix copy, V' tile
+  return 2048 + static_cast<size_t>(d_head) * k16 * 2 + kTile * static_cast<size_t>(max_rp_k + k16 + max_rp_v) * 2;
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
