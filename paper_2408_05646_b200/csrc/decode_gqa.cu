@@ -12,8 +12,12 @@
 //                                                       but only 16 rows of P^T exist in shared memory: the other
 //                                                       112 rows of the operand fall on whatever follows (Q', the
 //                                                       tiles: finite numbers) and fill rows of O' nobody reads
-// K' and V' tiles arrive by TMA (tensor maps of the cache slabs, 128-byte swizzle): K'(t+1) once the scores of tile
-// t are done, V'(t+1) (two buffers) once the weighted sum of tile t-1 is done; two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that
+// A tile of K' or V' rows is contiguous in the cache and arrives as one bulk copy (cp.async.bulk; tiled TMA boxes of
+// 128-byte rows were issue-bound at about half the HBM rate) into a row-major staging buffer; the threads move it
+// into the core-matrix layout the tensor core reads and the staging buffer takes the next tile at once.  The score
+// product of tile t+1 goes out at the top of tile t, so it runs under tile t's softmax.  A fifth warp issues the
+// MMAs and the copies: tcgen05.mma issue blocks while the tensor pipe is busy, and a worker thread that issued them
+// held all 128 workers at the next barrier.  Workers and the issuer meet on mbarriers only.  Two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that
 // gqa_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
@@ -25,18 +29,21 @@ namespace {
 
 using namespace tc;
 
-constexpr int kAtom = kTile * 128;            // one swizzled atom column of a 128-row tile: 64 elements wide
 constexpr int kMaxGroup = 16;                 // query heads per K/V head (N of the score product)
+constexpr int kGqaThreads = kThreads + 32;    // 128 workers (one per cached row of a tile) + the issuing warp
+
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
 struct __align__(16) GqaSmemHeader {
-  unsigned long long s_done, o_done, k_full, v_full[2];
+  unsigned long long s_done, o_done, k_full, v_full;
+  unsigned long long tiles_ready, p_ready;    // 128 arrivals each: tiles moved into place / P^T written
   uint32_t tmem_base;
   int abort_flag;
   float pad_[2];
-  float red[4][kMaxGroup];                    // per-warp maxima / sums per query
+  float red[2][4][kMaxGroup];                 // per-warp maxima / sums per query, alternating between tiles
 };
 
-__global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecodeParams p) {
+__global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   GqaSmemHeader* hdr = reinterpret_cast<GqaSmemHeader*>(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -45,17 +52,20 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
   const int G = p.group;
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
-  const int grp_k = (rpk16 >> 3) << 7, grp_p = (kTile >> 3) << 7;
-  const int atoms_k = (rpk16 + 63) >> 6, atoms_v = (hd.rp_v + 63) >> 6;
-  const int k_bytes = atoms_k * kAtom, v_bytes = atoms_v * kAtom;
+  const int grp_k = (rpk16 >> 3) << 7, grp_v = (rpv16 >> 3) << 7, grp_p = (kTile >> 3) << 7;
+  const int rowb_k = hd.rp_k * 2, rowb_v = hd.rp_v * 2;      // bytes per cached row
+  const int kst_bytes = kTile * rowb_k, vst_bytes = kTile * rowb_v;          // staging, row-major
+  const int km_bytes = kTile * rpk16 * 2, vm_bytes = kTile * rpv16 * 2;      // core-matrix layout
   const int q_bytes = kMaxGroup * rpk16 * 2;                 // one image (high or low part) of Q'
   const int p_bytes = kMaxGroup * kTile * 2;                 // the 16 rows of P^T that exist
 
   unsigned char* tiles = smem + 1024;
   unsigned char* Ps = tiles;                                 // P^T [16 queries][128 rows], canonical (two 8-row groups)
   unsigned char* Qs = Ps + p_bytes;                          // Q' images [16][rk16], canonical: high, then low
-  unsigned char* Ks = Qs + 2 * q_bytes;                      // K' tile, swizzled atom columns of 128 rows (1024-aligned)
-  unsigned char* Vs = Ks + k_bytes;                          // two V' tiles, same layout
+  unsigned char* Kst = Qs + 2 * q_bytes;                     // K' tile as it lands
+  unsigned char* Vst = Kst + kst_bytes;                      // V' tile as it lands
+  unsigned char* Km = Vst + vst_bytes;                       // K' tile, canonical core-matrix layout
+  unsigned char* Vm = Km + km_bytes;                         // V' tile, canonical core-matrix layout
 
   const int per = (p.nt + p.splits - 1) / p.splits;
   const int t_lo = split * per, t_hi = min(p.nt, t_lo + per);
@@ -73,13 +83,15 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     mbar_init(&hdr->s_done, 1);
     mbar_init(&hdr->o_done, 1);
     mbar_init(&hdr->k_full, 1);
-    mbar_init(&hdr->v_full[0], 1);
-    mbar_init(&hdr->v_full[1], 1);
+    mbar_init(&hdr->v_full, 1);
+    mbar_init(&hdr->tiles_ready, kThreads);
+    mbar_init(&hdr->p_ready, kThreads);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // P^T and the Q' images start as zeros
-  for (int idx = tid; idx < (p_bytes + 2 * q_bytes) / 16; idx += kThreads)
+  // P^T, the Q' images and the tiles start as zeros (rows that no copy fills meet zero weights and must be finite;
+  // padding chunks of the core-matrix tiles stay zero)
+  for (int idx = tid; idx < (p_bytes + 2 * q_bytes + kst_bytes + vst_bytes + km_bytes + vm_bytes) / 16; idx += kGqaThreads)
     reinterpret_cast<uint4*>(Ps)[idx] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   // Q' = q U^K for the g queries of the group, times log2(e)/sqrt(d_h), split into bf16 high + low parts
@@ -87,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b +
                               static_cast<int64_t>(h) * G * p.d_head;
     const float* U = p.basis + hd.uk_off;                    // d_head x rp_k, zero padded columns
-    for (int idx = tid; idx < G * hd.rp_k; idx += kThreads) {
+    for (int idx = tid; idx < G * hd.rp_k; idx += kGqaThreads) {
       const int qi = idx / hd.rp_k, c = idx - qi * hd.rp_k;
       float acc = 0.f;
       for (int d = 0; d < p.d_head; ++d) acc = fmaf(__bfloat162float(qg[qi * p.d_head + d]), __ldg(U + d * hd.rp_k + c), acc);
@@ -99,20 +111,26 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
       *reinterpret_cast<__nv_bfloat16*>(Qs + q_bytes + off) = lo;
     }
   }
-  const unsigned char* maps = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
+  const uint64_t policy = policy_evict_first();
+  const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
+  const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
   auto fetch_k = [&](int t) {
-    mbar_arrive_expect_tx(&hdr->k_full, static_cast<uint32_t>(k_bytes));
-    for (int a = 0; a < atoms_k; ++a)
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(Ks + a * kAtom + hf * (kAtom / 2), maps, a * 64, t * kTile + hf * 64, b, &hdr->k_full);
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_k;
+    mbar_arrive_expect_tx(&hdr->k_full, bytes);
+    bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
   };
-  auto fetch_v = [&](int t) {                                // into buffer (t - t_lo) % 2
-    const int vb = (t - t_lo) & 1;
-    mbar_arrive_expect_tx(&hdr->v_full[vb], static_cast<uint32_t>(v_bytes));
-    for (int a = 0; a < atoms_v; ++a)
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(Vs + vb * v_bytes + a * kAtom + hf * (kAtom / 2), maps + 128, a * 64, t * kTile + hf * 64, b,
-                    &hdr->v_full[vb]);
+  auto fetch_v = [&](int t) {
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_v;
+    mbar_arrive_expect_tx(&hdr->v_full, bytes);
+    bulk_load(Vst, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
+  };
+  // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * group + c * 128 + (row % 8) * 16
+  auto relayout = [&](unsigned char* dst, const unsigned char* src, int rowb, int grp) {
+    const int chunks = rowb >> 4;
+    for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
+      const int c = idx >> 7, row = idx & (kTile - 1);
+      *reinterpret_cast<uint4*>(dst + chunk_off(row, c, grp)) = *reinterpret_cast<const uint4*>(src + row * rowb + (c << 4));
+    }
   };
   fence_async_smem();
   tc_fence_before();
@@ -125,42 +143,81 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
   const uint32_t idesc_s = instr_desc(kMaxGroup, false);
   const uint32_t idesc_o = instr_desc(rpv16, true);
   const int ks_steps = rpk16 >> 4;
-  const uint64_t desc_k = smem_desc_sw128(smem_u32(Ks), 16, 1024);
+  const uint64_t desc_k = smem_desc(smem_u32(Km), 128, grp_k);
   const uint64_t desc_q = smem_desc(smem_u32(Qs), 128, grp_k);
   const uint64_t desc_p = smem_desc(smem_u32(Ps), 128, grp_p);
-  const uint64_t desc_v = smem_desc_sw128(smem_u32(Vs), kAtom, 1024);
+  const uint64_t desc_v = smem_desc(smem_u32(Vm), grp_v, 128);   // MN-major operand: 8-row groups along K, chunks along N
   // S(t) = K'(t) Q'^T into score buffer `buf` (columns 32 buf .. 32 buf + 15)
   auto issue_s = [&](int buf) {
     tc_fence_after();
     for (int part_i = 0; part_i < 2; ++part_i)               // Q' high part, then low part
       for (int s = 0; s < ks_steps; ++s)
-        mma_ss(tmem + 32 * buf, desc_k + (s >> 2) * (kAtom >> 4) + (s & 3) * 2, desc_q + part_i * (q_bytes >> 4) + s * 16,
-               idesc_s, part_i > 0 || s > 0);
+        mma_ss(tmem + 32 * buf, desc_k + s * 16, desc_q + part_i * (q_bytes >> 4) + s * 16, idesc_s, part_i > 0 || s > 0);
     mma_commit(&hdr->s_done);
   };
   bool ok = true;
-  if (tid == 0) {
-    tensormap_acquire(maps);
-    tensormap_acquire(maps + 128);
+  const bool issuer = warp == kThreads / 32;                 // warp 4
+  if (issuer && lane == 0) {
     fetch_k(t_lo);
     fetch_v(t_lo);
-    if (t_lo + 1 < t_hi) fetch_v(t_lo + 1);
-    ok = mbar_wait(&hdr->k_full, 0, p.status);
-    if (ok) issue_s(0);
-    else *abort_flag = 1;
+  }
+  // the first K' tile: into the core-matrix layout, its score product, and the staging buffer takes the second
+  if (!issuer) {
+    if (!mbar_wait(&hdr->k_full, 0, p.status)) *abort_flag = 1;
+    relayout(Km, Kst, rowb_k, grp_k);
+    fence_async_smem();
+  }
+  __syncthreads();
+  if (*abort_flag) ok = false;
+
+  if (issuer) {
+    // ------------------------------------------------------------------ the issuing warp
+    if (lane == 0 && ok) {
+      issue_s(0);
+      if (t_lo + 1 < t_hi) fetch_k(t_lo + 1);
+      for (int t = t_lo; t < t_hi && ok; ++t) {
+        const uint32_t par = (t - t_lo) & 1u;
+        ok = mbar_wait(&hdr->tiles_ready, par, p.status) && !*abort_flag;   // K'(t+1), V'(t) are in place
+        if (!ok) break;
+        if (t + 1 < t_hi) {
+          issue_s(static_cast<int>(par ^ 1u));
+          fetch_v(t + 1);
+          if (t + 2 < t_hi) fetch_k(t + 2);
+        }
+        ok = mbar_wait(&hdr->p_ready, par, p.status) && !*abort_flag;       // P^T(t) written, O' rescaled if needed
+        if (!ok) break;
+        tc_fence_after();
+        for (int s = 0; s < kTile / 16; ++s)                 // O' += P^T V'(t), 16 cached rows (two 8-row groups) a step
+          mma_ss(tO, desc_p + s * 16, desc_v + s * ((2 * grp_v) >> 4), idesc_o, t > t_lo || s > 0);
+        mma_commit(&hdr->o_done);
+      }
+      if (!ok) *abort_flag = 1;
+    }
+    __syncthreads();                                         // the workers' epilogue
+    __syncthreads();
+    return;
   }
 
+  // -------------------------------------------------------------------- the 128 workers
   float m_run[kMaxGroup], l_thr[kMaxGroup];
 #pragma unroll
   for (int qi = 0; qi < kMaxGroup; ++qi) { m_run[qi] = -INFINITY; l_thr[qi] = 0.f; }
 
   for (int t = t_lo; t < t_hi && ok; ++t) {
     const uint32_t par = (t - t_lo) & 1u;
-    // ---- S(t) is complete: K'(t+1) may replace K'(t); PV(t-1) is complete: P^T and the V' tile are free
+    // ---- S(t) is complete: the K' core-matrix tile is free; PV(t-1) is complete: P^T and the V' core-matrix tile
+    //      are free.  K'(t+1) and V'(t) have landed: move them and tell the issuer.
     if (!mbar_wait(&hdr->s_done, par, p.status)) *abort_flag = 1;
     if (t > t_lo && !mbar_wait(&hdr->o_done, par ^ 1u, p.status)) *abort_flag = 1;
-    if (tid == 0 && t + 1 < t_hi) fetch_k(t + 1);
-    if (tid == 0 && t > t_lo && t + 1 < t_hi) fetch_v(t + 1);   // its buffer was PV(t-1)'s; the first two went out earlier
+    if (t + 1 < t_hi) {
+      if (!mbar_wait(&hdr->k_full, par ^ 1u, p.status)) *abort_flag = 1;
+      relayout(Km, Kst, rowb_k, grp_k);
+    }
+    if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
+    relayout(Vm, Vst, rowb_v, grp_v);
+    fence_async_smem();
+    tc_fence_before();
+    mbar_arrive(&hdr->tiles_ready);
     tc_fence_after();
     uint32_t sr[16];
     tmem_ld16(tmem + lane_base + 32 * par, sr);
@@ -182,10 +239,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
       float mine = -INFINITY;
 #pragma unroll
       for (int qi = 0; qi < kMaxGroup; ++qi) mine = lane == qi ? mx[qi] : mine;
-      hdr->red[warp][lane] = mine;
+      hdr->red[par][warp][lane] = mine;
     }
-    tc_fence_before();
-    __syncthreads();
+    worker_sync();
     if (*abort_flag) { ok = false; break; }
     // lazy reference: m_run follows the maximum only when that grew by more than 8 (every thread decides alike)
     bool rescale = false;
@@ -193,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
 #pragma unroll
     for (int qi = 0; qi < kMaxGroup; ++qi) {
       if (qi < G) {
-        const float tm = fmaxf(fmaxf(hdr->red[0][qi], hdr->red[1][qi]), fmaxf(hdr->red[2][qi], hdr->red[3][qi]));
+        const float tm = fmaxf(fmaxf(hdr->red[par][0][qi], hdr->red[par][1][qi]), fmaxf(hdr->red[par][2][qi], hdr->red[par][3][qi]));
         float alpha = 1.f;
         if (tm > m_run[qi] + 8.f) {
           alpha = ex2(m_run[qi] - tm);
@@ -220,26 +276,14 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
     }
     fence_async_smem();
     tc_fence_before();
-    if (!mbar_wait(&hdr->v_full[par], ((t - t_lo) >> 1) & 1u, p.status)) *abort_flag = 1;
-    __syncthreads();
-    if (*abort_flag) { ok = false; break; }
-    // ---- O' += P^T V'(t); then S(t+1) as soon as K'(t+1) is there
-    if (tid == 0) {
-      tc_fence_after();
-      for (int s = 0; s < kTile / 16; ++s)                   // 16 cached rows a step
-        mma_ss(tO, desc_p + s * 16, desc_v + par * (v_bytes >> 4) + s * (2048 >> 4), idesc_o, t > t_lo || s > 0);
-      mma_commit(&hdr->o_done);
-      if (t + 1 < t_hi) {
-        if (mbar_wait(&hdr->k_full, par ^ 1u, p.status)) issue_s(static_cast<int>(par ^ 1u));
-        else *abort_flag = 1;
-      }
-    }
+    mbar_arrive(&hdr->p_ready);                              // the issuer sends the weighted sum of this tile off
   }
   if (ok) {
     if (!mbar_wait(&hdr->o_done, (t_hi - 1 - t_lo) & 1u, p.status)) ok = false;
   }
   if (!ok) *abort_flag = 1;
   tc_fence_after();
+  worker_sync();                                             // every worker is done with the last tile's maxima
 
   // ---- partials per query: m, l (summed over the threads' rows), o' (row `query` of O')
 #pragma unroll
@@ -248,7 +292,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
       float v = l_thr[qi];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) hdr->red[warp][qi] = v;
+      if (lane == 0) hdr->red[0][warp][qi] = v;
     }
   }
   __syncthreads();
@@ -257,7 +301,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_gqa_kernel(const GqaDecode
 #pragma unroll
     for (int qi = 0; qi < kMaxGroup; ++qi) mine_m = tid == qi ? m_run[qi] : mine_m;
     part[tid * p.part_stride] = mine_m;
-    part[tid * p.part_stride + 1] = (hdr->red[0][tid] + hdr->red[1][tid]) + (hdr->red[2][tid] + hdr->red[3][tid]);
+    part[tid * p.part_stride + 1] = (hdr->red[0][0][tid] + hdr->red[0][1][tid]) + (hdr->red[0][2][tid] + hdr->red[0][3][tid]);
   }
   if (warp == 0) {
     for (int c0 = 0; c0 < rpv16; c0 += 16) {
@@ -306,10 +350,12 @@ __global__ void __launch_bounds__(128) gqa_combine_kernel(const GqaDecodeParams 
 
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
   const size_t k16 = (max_rp_k + 15) & ~15;
-  // P^T (16 rows), Q' images, one K' tile, two V' tiles; the P^T operand of the weighted sum spans 32 KB from its
-  // start, which the tiles behind it cover
-  return 1024 + kMaxGroup * kTile * 2 + 2 * kMaxGroup * k16 * 2 +
-         (((k16 + 63) >> 6) + 2 * ((max_rp_v + 63) >> 6)) * static_cast<size_t>(kAtom);
+  // P^T (16 rows), Q' images, K' and V' tiles as they land and in the core-matrix layout; the P^T operand of the
+  // weighted sum spans 32 KB from its start, which the tiles behind it cover
+  const size_t v16 = (max_rp_v + 15) & ~15;
+  size_t total = 1024 + kMaxGroup * kTile * 2 + 2 * kMaxGroup * k16 * 2 + kTile * static_cast<size_t>(max_rp_k + max_rp_v + k16 + v16) * 2;
+  const size_t need = 1024 + static_cast<size_t>(kTile) * kTile * 2;
+  return total < need ? need : total;
 }
 
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
@@ -321,7 +367,7 @@ cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_
     configured = smem;
   }
   dim3 grid(p.B * p.H, p.splits);
-  decode_gqa_kernel<<<grid, kThreads, smem, s>>>(p);
+  decode_gqa_kernel<<<grid, kGqaThreads, smem, s>>>(p);
   ++*launches;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
