@@ -12,9 +12,9 @@
 //                                                       but only 16 rows of P^T exist in shared memory: the other
 //                                                       112 rows of the operand fall on whatever follows (Q', the
 //                                                       tiles: finite numbers) and fill rows of O' nobody reads
-// A tile of K' or V' rows is contiguous in the cache and arrives as one bulk copy (cp.async.bulk; tiled TMA boxes of
-// 128-byte rows were issue-bound at about half the HBM rate) into a row-major staging buffer; the threads move it
-// into the core-matrix layout the tensor core reads and the staging buffer takes the next tile at once.  The score
+// A tile of K' or V' rows is contiguous in the cache and arrives as one bulk copy (cp.async.bulk) into a row-major
+// staging buffer; the threads move it into the core-matrix layout the tensor core reads and the staging buffer takes
+// the next tile at once, a whole tile ahead of its use.  The score
 // product of tile t+1 goes out at the top of tile t, so it runs under tile t's softmax.  A fifth warp issues the
 // MMAs and the copies: tcgen05.mma issue blocks while the tensor pipe is busy, and a worker thread that issued them
 // held all 128 workers at the next barrier.  Workers and the issuer meet on mbarriers only.  Two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that

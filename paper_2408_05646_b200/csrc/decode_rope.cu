@@ -15,11 +15,12 @@
 // e^{-i 128 phi}, one complex multiplication, renormalised), the second is a per-thread constant in registers.
 //
 // One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  A tile
-// of K' or V' rows is contiguous in the cache, so each arrives as one bulk copy (cp.async.bulk, the form that
-// reaches the HBM rate in the plain decode kernel; tiled TMA boxes of 128-byte rows were issue-bound at about
-// half of it).  K' lands row-major in a staging buffer, the threads move it into the core-matrix layout the
-// tensor core reads (16-byte chunks, 20 KB a tile), and the staging buffer takes the next tile at once, a whole
-// tile ahead of its use; V' is read row-major where it lands.  Scores -> online softmax in base 2 ->
+// of K' or V' rows is contiguous in the cache, so each arrives as one bulk copy (cp.async.bulk).  K' lands
+// row-major in a staging buffer, the threads move it into the core-matrix layout the tensor core reads (16-byte
+// chunks, 20 KB a tile), and the staging buffer takes the next tile at once, a whole tile ahead of its use: with
+// a single tile in flight per CTA it is the distance between request and use that sets the pace, not the kind of
+// copy (tiled TMA boxes stream at the same rate when four tiles are in flight).  V' is read row-major where it
+// lands.  Scores -> online softmax in base 2 ->
 // o' += p V' on the CUDA cores (thread (g, c) owns a column pair over a row group).  A unit split over several CTAs leaves partials (m, l, o') that
 // rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
