@@ -549,7 +549,7 @@ def run_gqa(args, wl):
     from paper_2408_05646_b200 import build
     build.build_library()
     from paper_2408_05646_b200 import binding
-    g = synth.GQA_GROUP[wl.name]
+    g = synth.GQA_GROUP[wl.name.split("[")[0]]
     keep = [0, wl.n_heads - 1]
     lay, ranks, U_k, U_v, hist, _, k_new, v_new = build_layer(wl, device, binding, keep)
     dt = synth.torch_dtype(wl.dtype)
@@ -661,7 +661,7 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
-    if wl.name in synth.GQA_GROUP:
+    if args.workload in synth.GQA_GROUP:
         return run_gqa(args, wl)
     if wl.name.startswith("prefill"):
         run_prefill(args, wl)
