@@ -34,7 +34,7 @@ FILL_CHUNK = 1024          # tokens per append call while filling the cache
 # DRAM bytes moved per algorithmic byte by decode_splitkv_kernel, from the ncu capture summarised in
 # profiles/decode_splitkv_llama2_7b_b2_n32k_full.md (B = 2 case: 680.4 MB for 671.1 MB; traffic grows in
 # proportion to the number of units).  Set to None whenever that kernel changes after the capture.
-DECODE_TRAFFIC_RATIO = 680.44 / 671.11
+DECODE_TRAFFIC_RATIO = 681.43 / 671.11
 
 
 def measured_peaks():

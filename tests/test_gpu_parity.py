@@ -388,3 +388,22 @@ def test_peaked_attention_over_heads_that_share_a_slot_size(B, dtype):
         lay.set_option(B.EA_OPT_DECODE_FUSED, fused)
         assert_close(lay.decode(q), expect, dtype, f"ctas={ctas} fused={fused}", **tol)
     lay.poll_status()
+
+
+@pytest.mark.parametrize("impl", [2, 3, 1])
+def test_prefill_with_peaked_attention(B, impl):
+    """Queries scaled by 3: the weights of a prompt row sit on a few keys, so an error in a few rows (a stale tile, a
+    ragged tail, the diagonal mask) is not averaged away.  (Not more: the kernels keep Q' in bf16, and its rounding
+    grows with the scores, about |s| * 2^-9 per score.)  All three prefill kernels, two chunks."""
+    from helpers import storage_model
+    B_, H, d, T = 2, 4, 128, 700
+    rk, rv = [80, 48, 128, 64], [64, 112, 16, 80]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, BF16, seed_cfg=143, T_q=T, q_scale=3.0)
+    ref = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(BF16))
+    expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
+    lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, impl)
+    a = lay.prefill(q[:, :300], k[:, :300], v[:, :300])
+    c = lay.prefill(q[:, 300:], k[:, 300:], v[:, 300:])
+    lay.poll_status()
+    assert_close(torch.cat([a, c], dim=1), expect, BF16, f"peaked prefill impl {impl}")
