@@ -34,15 +34,36 @@ constexpr int kGqaThreads = kThreads + 32;    // 128 workers (one per cached row
 
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
+// Warp maximum of a float in one instruction: floats ordered as integers (sign-magnitude -> two's complement).
+__device__ __forceinline__ float warp_max(float v) {
+  int i = __float_as_int(v);
+  i ^= (i >> 31) & 0x7fffffff;
+  i = __reduce_max_sync(0xffffffffu, i);
+  i ^= (i >> 31) & 0x7fffffff;
+  return __int_as_float(i);
+}
+// S = K'_tile Q'^T, KS steps of 16 rank elements, Q' high part then low part; unrolled so that the issuing thread
+// spends its time in the MMAs and not in address arithmetic
+template <int KS>
+__device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint64_t dk, uint64_t dq, uint32_t q_lo, uint32_t idesc) {
+#pragma unroll
+  for (int s = 0; s < KS; ++s) mma_ss(d_tmem, dk + s * 16, dq + s * 16, idesc, s > 0);
+#pragma unroll
+  for (int s = 0; s < KS; ++s) mma_ss(d_tmem, dk + s * 16, dq + q_lo + s * 16, idesc, true);
+}
+
 struct __align__(16) GqaSmemHeader {
   unsigned long long s_done, o_done, k_full, v_full;
   unsigned long long tiles_ready, p_ready;    // 128 arrivals each: tiles moved into place / P^T written
   uint32_t tmem_base;
   int abort_flag;
   float pad_[2];
-  float red[2][4][kMaxGroup];                 // per-warp maxima / sums per query, alternating between tiles
+  float red[2][kMaxGroup][4];                 // per query: the four warps' maxima / sums, alternating between tiles
 };
 
+// GP: query slots the kernel carries (the group size rounded up to 4, 8 or 16); slots past the group score zero
+// queries and are never written out.
+template <int GP>
 __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   GqaSmemHeader* hdr = reinterpret_cast<GqaSmemHeader*>(smem);
@@ -125,11 +146,20 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     bulk_load(Vst, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
   };
   // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * group + c * 128 + (row % 8) * 16
+  // one thread per row: all loads first, then the stores (consecutive threads store consecutive 16-byte pieces)
   auto relayout = [&](unsigned char* dst, const unsigned char* src, int rowb, int grp) {
     const int chunks = rowb >> 4;
-    for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
-      const int c = idx >> 7, row = idx & (kTile - 1);
-      *reinterpret_cast<uint4*>(dst + chunk_off(row, c, grp)) = *reinterpret_cast<const uint4*>(src + row * rowb + (c << 4));
+    const unsigned char* s_row = src + tid * rowb;
+    unsigned char* d_row = dst + chunk_off(tid, 0, grp);
+#pragma unroll
+    for (int c0 = 0; c0 < 16; c0 += 8) {                     // eight chunks in flight at a time
+      uint4 tmp[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        if (c0 + c < chunks) tmp[c] = *reinterpret_cast<const uint4*>(s_row + ((c0 + c) << 4));
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        if (c0 + c < chunks) *reinterpret_cast<uint4*>(d_row + ((c0 + c) << 7)) = tmp[c];
     }
   };
   fence_async_smem();
@@ -150,9 +180,17 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
   // S(t) = K'(t) Q'^T into score buffer `buf` (columns 32 buf .. 32 buf + 15)
   auto issue_s = [&](int buf) {
     tc_fence_after();
-    for (int part_i = 0; part_i < 2; ++part_i)               // Q' high part, then low part
-      for (int s = 0; s < ks_steps; ++s)
-        mma_ss(tmem + 32 * buf, desc_k + s * 16, desc_q + part_i * (q_bytes >> 4) + s * 16, idesc_s, part_i > 0 || s > 0);
+    const uint32_t d = tmem + 32 * buf, q_lo = static_cast<uint32_t>(q_bytes >> 4);
+    switch (ks_steps) {
+      case 1: issue_scores<1>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 2: issue_scores<2>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 3: issue_scores<3>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 4: issue_scores<4>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 5: issue_scores<5>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 6: issue_scores<6>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      case 7: issue_scores<7>(d, desc_k, desc_q, q_lo, idesc_s); break;
+      default: issue_scores<8>(d, desc_k, desc_q, q_lo, idesc_s); break;
+    }
     mma_commit(&hdr->s_done);
   };
   bool ok = true;
@@ -199,9 +237,9 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
   }
 
   // -------------------------------------------------------------------- the 128 workers
-  float m_run[kMaxGroup], l_thr[kMaxGroup];
+  float m_run[GP], l_thr[GP];
 #pragma unroll
-  for (int qi = 0; qi < kMaxGroup; ++qi) { m_run[qi] = -INFINITY; l_thr[qi] = 0.f; }
+  for (int qi = 0; qi < GP; ++qi) { m_run[qi] = -INFINITY; l_thr[qi] = 0.f; }
 
   for (int t = t_lo; t < t_hi && ok; ++t) {
     const uint32_t par = (t - t_lo) & 1u;
@@ -223,23 +261,11 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     tmem_ld16(tmem + lane_base + 32 * par, sr);
     tmem_wait_ld();
     const bool live = t * kTile + tid < p.n;
-    // ---- per-query maximum over the tile
-    float mx[kMaxGroup];
+    // ---- per-query maximum over the tile: one reduction instruction per query and warp, lane q keeps query q's
 #pragma unroll
-    for (int qi = 0; qi < kMaxGroup; ++qi) {
-      mx[qi] = -INFINITY;
-      if (qi < G) {
-        float v = live ? __uint_as_float(sr[qi]) : -INFINITY;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-        mx[qi] = v;
-      }
-    }
-    if (lane < kMaxGroup) {
-      float mine = -INFINITY;
-#pragma unroll
-      for (int qi = 0; qi < kMaxGroup; ++qi) mine = lane == qi ? mx[qi] : mine;
-      hdr->red[par][warp][lane] = mine;
+    for (int qi = 0; qi < GP; ++qi) {
+      const float v = warp_max(live ? __uint_as_float(sr[qi]) : -INFINITY);
+      if (lane == qi) hdr->red[par][qi][warp] = v;
     }
     worker_sync();
     if (*abort_flag) { ok = false; break; }
@@ -247,20 +273,19 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     bool rescale = false;
     float alpha_mine = 1.f;                                  // for the O' row this thread owns (lane = query)
 #pragma unroll
-    for (int qi = 0; qi < kMaxGroup; ++qi) {
-      if (qi < G) {
-        const float tm = fmaxf(fmaxf(hdr->red[par][0][qi], hdr->red[par][1][qi]), fmaxf(hdr->red[par][2][qi], hdr->red[par][3][qi]));
-        float alpha = 1.f;
-        if (tm > m_run[qi] + 8.f) {
-          alpha = ex2(m_run[qi] - tm);
-          m_run[qi] = tm;
-          rescale = rescale || t > t_lo;
-        }
-        const float pj = live ? ex2(__uint_as_float(sr[qi]) - m_run[qi]) : 0.f;
-        l_thr[qi] = fmaf(l_thr[qi], alpha, pj);
-        if (tid == qi) alpha_mine = alpha;
-        *reinterpret_cast<__nv_bfloat16*>(Ps + chunk_off(qi, tid >> 3, grp_p) + (tid & 7) * 2) = __float2bfloat16_rn(pj);
+    for (int qi = 0; qi < GP; ++qi) {
+      const float4 r4 = *reinterpret_cast<const float4*>(&hdr->red[par][qi][0]);
+      const float tm = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
+      float alpha = 1.f;
+      if (tm > m_run[qi] + 8.f) {
+        alpha = ex2(m_run[qi] - tm);
+        m_run[qi] = tm;
+        rescale = rescale || t > t_lo;
       }
+      const float pj = live ? ex2(__uint_as_float(sr[qi]) - m_run[qi]) : 0.f;
+      l_thr[qi] = fmaf(l_thr[qi], alpha, pj);
+      if (tid == qi) alpha_mine = alpha;
+      *reinterpret_cast<__nv_bfloat16*>(Ps + chunk_off(qi, tid >> 3, grp_p) + (tid & 7) * 2) = __float2bfloat16_rn(pj);
     }
     if (rescale && warp == 0) {                              // O' rows (lanes 0..g-1 of warp 0) times their alpha
       tc_fence_after();
@@ -287,21 +312,19 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
 
   // ---- partials per query: m, l (summed over the threads' rows), o' (row `query` of O')
 #pragma unroll
-  for (int qi = 0; qi < kMaxGroup; ++qi) {
-    if (qi < G) {
-      float v = l_thr[qi];
+  for (int qi = 0; qi < GP; ++qi) {
+    float v = l_thr[qi];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) hdr->red[0][warp][qi] = v;
-    }
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) hdr->red[0][qi][warp] = v;
   }
   __syncthreads();
   if (tid < G) {
     float mine_m = -INFINITY;
 #pragma unroll
-    for (int qi = 0; qi < kMaxGroup; ++qi) mine_m = tid == qi ? m_run[qi] : mine_m;
+    for (int qi = 0; qi < GP; ++qi) mine_m = tid == qi ? m_run[qi] : mine_m;
     part[tid * p.part_stride] = mine_m;
-    part[tid * p.part_stride + 1] = (hdr->red[0][0][tid] + hdr->red[0][1][tid]) + (hdr->red[0][2][tid] + hdr->red[0][3][tid]);
+    part[tid * p.part_stride + 1] = (hdr->red[0][tid][0] + hdr->red[0][tid][1]) + (hdr->red[0][tid][2] + hdr->red[0][tid][3]);
   }
   if (warp == 0) {
     for (int c0 = 0; c0 < rpv16; c0 += 16) {
@@ -358,18 +381,24 @@ size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
   return total < need ? need : total;
 }
 
-cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
+template <int GP>
+cudaError_t launch_gqa_variant(const GqaDecodeParams& p, size_t smem, cudaStream_t s) {
   static size_t configured = 0;
   if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    const cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel<GP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     configured = smem;
   }
   dim3 grid(p.B * p.H, p.splits);
-  decode_gqa_kernel<<<grid, kGqaThreads, smem, s>>>(p);
+  decode_gqa_kernel<GP><<<grid, kGqaThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
+  cudaError_t e = p.group <= 4 ? launch_gqa_variant<4>(p, smem, s)
+                  : p.group <= 8 ? launch_gqa_variant<8>(p, smem, s) : launch_gqa_variant<16>(p, smem, s);
   ++*launches;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   gqa_combine_kernel<<<p.B * p.H * p.group, 128, 0, s>>>(p);
   ++*launches;
