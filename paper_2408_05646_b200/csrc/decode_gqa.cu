@@ -146,21 +146,8 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     bulk_load(Vst, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
   };
   // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * group + c * 128 + (row % 8) * 16
-  // one thread per row: all loads first, then the stores (consecutive threads store consecutive 16-byte pieces)
   auto relayout = [&](unsigned char* dst, const unsigned char* src, int rowb, int grp) {
-    const int chunks = rowb >> 4;
-    const unsigned char* s_row = src + tid * rowb;
-    unsigned char* d_row = dst + chunk_off(tid, 0, grp);
-#pragma unroll
-    for (int c0 = 0; c0 < 16; c0 += 8) {                     // eight chunks in flight at a time
-      uint4 tmp[8];
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        if (c0 + c < chunks) tmp[c] = *reinterpret_cast<const uint4*>(s_row + ((c0 + c) << 4));
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        if (c0 + c < chunks) *reinterpret_cast<uint4*>(d_row + ((c0 + c) << 7)) = tmp[c];
-    }
+    relayout_tile(dst, src, rowb, grp, warp, lane);
   };
   fence_async_smem();
   tc_fence_before();

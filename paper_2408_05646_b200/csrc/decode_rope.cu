@@ -108,13 +108,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     bulk_load(Vs, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
   };
   // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * grp_k + c * 128 + (row % 8) * 16
-  auto relayout_k = [&]() {
-    const int chunks = hd.rp_k >> 3;
-    for (int idx = tid; idx < kTile * chunks; idx += kThreads) {
-      const int c = idx >> 7, row = idx & (kTile - 1);
-      *reinterpret_cast<uint4*>(Km + chunk_off(row, c, grp_k)) = *reinterpret_cast<const uint4*>(Kst + row * rowb_k + (c << 4));
-    }
-  };
+  auto relayout_k = [&]() { relayout_tile(Km, Kst, rowb_k, grp_k, warp, lane); };
 
   // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
   unsigned long long el_c[32], el_s[32];                     // pairs (2k, 2k+1) packed: (cos, cos), (sin, sin)

@@ -271,6 +271,30 @@ __device__ __forceinline__ void load_tile(unsigned char* dst, const __nv_bfloat1
   }
 }
 
+// Moves a tile of 128 rows from row-major form (row pitch `rowb` bytes, a multiple of 16) into the canonical
+// core-matrix layout, by four warps.  A warp instruction takes a block of 8 rows x 4 chunks: lane = (row % 8) +
+// 8 * (chunk % 4).  For pitches of 32 bytes modulo 64 (ranks 48, 80, 112) both the reads and the writes then spread
+// evenly over the banks; lane = row would read with an 8-way conflict.
+__device__ __forceinline__ void relayout_tile(unsigned char* dst, const unsigned char* src, int rowb, int group_stride,
+                                              int warp, int lane) {
+  const int chunks = rowb >> 4;
+  const int blocks = 16 * ((chunks + 3) >> 2);               // 16 row groups x quads of chunks
+  const int r8 = lane & 7, cc = lane >> 3;
+  for (int b0 = warp; b0 < blocks; b0 += 16) {               // four blocks in flight per warp
+    uint4 tmp[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int b = b0 + 4 * u, c = ((b >> 4) << 2) + cc, row = ((b & 15) << 3) + r8;
+      if (b < blocks && c < chunks) tmp[u] = *reinterpret_cast<const uint4*>(src + row * rowb + (c << 4));
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int b = b0 + 4 * u, c = ((b >> 4) << 2) + cc, row = ((b & 15) << 3) + r8;
+      if (b < blocks && c < chunks) *reinterpret_cast<uint4*>(dst + chunk_off(row, c, group_stride)) = tmp[u];
+    }
+  }
+}
+
 struct __align__(16) TcSmemHeader {
   unsigned long long bar;
   uint32_t tmem_base;
