@@ -25,6 +25,7 @@ by ordinary decode with the K/V heads repeated.
 The RoPE variant (Section 4.3) is pinned by library attention on keys and
 queries rotated with complex arithmetic, by its relative-position invariance,
 by the zero-angle special case and by loops.
+decode_quant is ordinary decode over the rows returned by kv_quant.quantized_view, which has its own pins.
 Nothing in this file is "parity unpinned".
 """
 from __future__ import annotations
@@ -291,6 +292,24 @@ class LayerOracle:
                     s = s + alibi_bias(self.alibi[h], self.len - 1, self.len)
                 p = softmax_rows(s[None, :])[0]
                 out[b, 0, hq] = lift(p @ Vp, self.U_V[h])
+        return out
+
+    # -- Section 5.3: the same decode step over a cache whose complete groups of G rows are kept as b-bit codes
+    def decode_quant(self, q: np.ndarray, bits: int, group: int, lowrank_out: bool = False) -> dict:
+        """Eq. 3 in the space of Eq. 7 with K', V' replaced by what the quantised cache holds of them
+        (oracle/kv_quant.py: keys per channel, values per token, the newest n mod G rows as stored)."""
+        from .kv_quant import quantized_view
+        q = np.asarray(q, dtype=F64).reshape(self.B, self.H, self.d_h)
+        assert self.rope is None
+        out = {}
+        for (b, h) in self.units:
+            Kq, Vq = quantized_view(self.Kp[(b, h)], self.Vp[(b, h)], bits, group)
+            qp = to_rank_space(q[b, h], self.U_K[h])
+            s = (Kq @ qp) / math.sqrt(self.d_h)
+            if self.alibi[h]:
+                s = s + alibi_bias(self.alibi[h], self.len - 1, self.len)
+            o = softmax_rows(s[None, :])[0] @ Vq
+            out[(b, h)] = o if lowrank_out else lift(o, self.U_V[h])
         return out
 
     def decode_dense(self, q: np.ndarray) -> np.ndarray:
