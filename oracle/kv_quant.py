@@ -11,7 +11,7 @@ storage cost: every printed size equals elements * (b + 16/G) / 8 bytes, i.e. ON
 metadata per group.  The reading taken here: that number is a half-precision scale and there is no
 zero point, hence symmetric codes
 
-    s = fp16( max|x| / (2^(b-1) - 1) ),    c = clip( rint(x / s), -(2^(b-1)-1), 2^(b-1)-1 ),    x^ = c * s .
+    s = fp16( min(max|x| / (2^(b-1) - 1), 65504) ),    c = clip( rint(x / s), -(2^(b-1)-1), 2^(b-1)-1 ),    x^ = c * s .
 
 The code is an integer decided by floating point, so the precision of that decision is part of the
 definition: x is the stored (16-bit) cache value, the quotient max|x| / qmax and x / s are single
@@ -50,7 +50,8 @@ def quantize_groups(x: np.ndarray, bits: int, group: int, axis: int):
     for g in range(n_groups):
         seg = x32[..., g * group:(g + 1) * group]
         amax = np.max(np.abs(seg), axis=-1)
-        s16 = (amax / qmax).astype(np.float16)          # single-precision quotient, then round to half
+        # single-precision quotient (kept inside the half-precision range), then round to half
+        s16 = np.minimum(amax / qmax, np.float32(65504.0)).astype(np.float16)
         s32 = s16.astype(np.float32)[..., None]
         with np.errstate(divide="ignore", invalid="ignore"):
             c = np.where(s32 > 0, np.rint(seg / s32), np.float32(0))

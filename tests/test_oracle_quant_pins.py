@@ -123,6 +123,13 @@ def test_keys_are_grouped_per_channel_and_values_per_token():
     assert set(changed_v[:, 0]) == {20} and set(changed_v[:, 1]) <= set(range(0, 16))      # one token, its 16 channels
 
 
+def test_scale_saturates_at_the_largest_half_precision_number():
+    x = np.array([1e6, -3e5, 2e4, 0.0])
+    c, s = kq.quantize_groups(x, 4, 4, axis=0)
+    assert float(s[0]) == 65504.0 and np.all(np.isfinite(kq.dequantize_groups(c, s, 4, 0)))
+    assert list(c) == [7, -5, 0, 0]                      # 1e6 / 65504 = 15.3 clips to 7; -3e5 / 65504 = -4.58
+
+
 def test_view_keeps_the_incomplete_group_as_stored():
     rng = np.random.default_rng(5)
     K, V = rng.standard_normal((70, 24)), rng.standard_normal((70, 24))
