@@ -175,6 +175,40 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
  * return EA_ERR_UNSUPPORTED while a rotary embedding is set.  Synchronises `cuda_stream`. */
 ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, void* cuda_stream);
 
+/* Section 5.3 ("Eigen Attention with Quantization") and Table 8: a quantised copy of the rank-r cache.
+ * Integer codes of `bits` bits with one half-precision scale per group of `group` numbers (the storage cost
+ * behind every size printed in Table 8: bits + 16/group bits per element).  Keys are grouped per channel
+ * (a group = `group` consecutive tokens of one channel of one head), values per token (a group = `group`
+ * consecutive channels of one token's row; the last group of a row may be shorter).  Codes are symmetric:
+ *     s = half(min(max|x| / (2^(bits-1) - 1), 65504)),  c = clip(rint(x / s)),  x^ = c * s ,
+ * x being the stored 16-bit row, the two divisions IEEE single precision, rint to nearest even.  Rows that do
+ * not fill a block of `group` tokens yet stay in the 16-bit cache and are attended from there.
+ * Built: bits == 4, group in {16, 32, 64, 128}, bf16 layers (EA_ERR_UNSUPPORTED otherwise).
+ *
+ * quant_bytes:  size of the caller's quantised buffer for this layer (host arithmetic).
+ * quant_attach: hands the library that DEVICE buffer (256-byte aligned, >= quant_bytes; owned by the caller, as
+ *               the cache is) and writes the per-head table at its start; no row is quantised yet.  NULL
+ *               detaches.  Synchronises `cuda_stream`.
+ * quant_sync:   quantises every complete block of `group` rows of the 16-bit cache that is not quantised yet
+ *               (rows [quant_len, floor(len / group) * group)); asynchronous.  The 16-bit rows stay where they
+ *               are; a caller that wants the memory back keeps only a window of the 16-bit cache.
+ * decode_quant: eigen_attn_decode (same arguments, flags and ALiBi bias) over the codes of rows [0, quant_len)
+ *               and the 16-bit rows [quant_len, len).  Not available with a rotary embedding.
+ * quant_len:    rows currently held as codes.  eigen_attn_set_len below quant_len rounds it down to a whole block.
+ * quant_layout: where head `head` lives in the buffer: byte offset of its slab [B][n_max / group][block_bytes],
+ *               and inside a block the offsets of the key scales [rp_k] halves, the value codes and the value
+ *               scales [ceil(rp_v / group)][group] halves; key codes sit at offset 0.  Codes are 32-bit words
+ *               [rp / 8][group]: word j of row i holds channels 8j..8j+7, channel 8j+k in bits 4k..4k+3 as c + 8. */
+ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, size_t* bytes);
+ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
+                                  void* cuda_stream);
+ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream);
+ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                                  int64_t stride_b_out, uint32_t flags, void* cuda_stream);
+ea_status eigen_attn_quant_len(eigen_attn_t h, int32_t* qlen);
+ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_offset, size_t* block_bytes,
+                                  size_t* k_scale_offset, size_t* v_code_offset, size_t* v_scale_offset);
+
 /* Current number of cached rows; set_len truncates or rewinds (0 <= len <= n_max), e.g. to re-run
  * a step at a fixed context length.  Rows beyond the previous length hold whatever was last written. */
 ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len);

@@ -68,6 +68,12 @@ SYMBOLS = {
     "eigen_attn_set_alibi": (_i32, [_vp, ctypes.POINTER(ctypes.c_float), _vp]),
     "eigen_attn_set_rope": (_i32, [_vp, ctypes.c_double, _i32, _vp]),
     "eigen_attn_decode_gqa": (_i32, [_vp, _vp, _i64, _i32, _vp, _i64, _vp]),
+    "eigen_attn_quant_bytes": (_i32, [_vp, _i32, _i32, ctypes.POINTER(_sz)]),
+    "eigen_attn_quant_attach": (_i32, [_vp, _i32, _i32, _vp, _sz, _vp]),
+    "eigen_attn_quant_sync": (_i32, [_vp, _vp]),
+    "eigen_attn_decode_quant": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
+    "eigen_attn_quant_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
+    "eigen_attn_quant_layout": (_i32, [_vp, _i32] + [ctypes.POINTER(_sz)] * 5),
     "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
     "eigen_attn_version": (_i32, []),
@@ -207,7 +213,7 @@ class EigenAttnLayer:
                     "eigen_attn_append_kv")
 
     def decode(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, q_preprojected: bool = False,
-               out_lowrank: bool = False, stream=None) -> torch.Tensor:
+               out_lowrank: bool = False, stream=None, _fn=None, _name="eigen_attn_decode") -> torch.Tensor:
         flags = 0
         if q_preprojected:
             assert q.is_contiguous() and q.shape == (self.B, 1, self.offs_k[-1]) and q.dtype == self.torch_dtype
@@ -225,9 +231,51 @@ class EigenAttnLayer:
             if out is None:
                 out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
             _, _, sbo, _ = self._tok(out, 1)
-        self._check(lib.eigen_attn_decode(self.handle, pq, sbq, out.data_ptr(), sbo, flags, _stream_ptr(stream)),
-                    "eigen_attn_decode")
+        fn = _fn if _fn is not None else lib.eigen_attn_decode
+        self._check(fn(self.handle, pq, sbq, out.data_ptr(), sbo, flags, _stream_ptr(stream)), _name)
         return out
+
+    # -- quantised copy of the cache (4-bit codes, one half-precision scale per group)
+    def quant_bytes(self, bits: int, group: int) -> int:
+        n = _sz(0)
+        self._check(lib.eigen_attn_quant_bytes(self.handle, int(bits), int(group), ctypes.byref(n)), "eigen_attn_quant_bytes")
+        return n.value
+
+    def quant_attach(self, bits: int, group: int, stream=None) -> torch.Tensor:
+        """Allocates the quantised buffer (a torch byte tensor kept on the layer) and attaches it."""
+        nbytes = self.quant_bytes(bits, group)
+        self.qcache = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+        self.q_group = int(group)
+        self._check(lib.eigen_attn_quant_attach(self.handle, int(bits), int(group), self.qcache.data_ptr(), nbytes,
+                                                _stream_ptr(stream)), "eigen_attn_quant_attach")
+        return self.qcache
+
+    def quant_sync(self, stream=None) -> None:
+        self._check(lib.eigen_attn_quant_sync(self.handle, _stream_ptr(stream)), "eigen_attn_quant_sync")
+
+    @property
+    def quant_len(self) -> int:
+        n = ctypes.c_int32(0)
+        self._check(lib.eigen_attn_quant_len(self.handle, ctypes.byref(n)), "eigen_attn_quant_len")
+        return n.value
+
+    def decode_quant(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, q_preprojected: bool = False,
+                     out_lowrank: bool = False, stream=None) -> torch.Tensor:
+        return self.decode(q, out, q_preprojected, out_lowrank, stream, _fn=lib.eigen_attn_decode_quant,
+                           _name="eigen_attn_decode_quant")
+
+    def quant_layout(self, head: int):
+        """(slab offset, block bytes, key-scale offset, value-code offset, value-scale offset) of a head."""
+        v = [_sz(0) for _ in range(5)]
+        self._check(lib.eigen_attn_quant_layout(self.handle, int(head), *[ctypes.byref(x) for x in v]),
+                    "eigen_attn_quant_layout")
+        return tuple(x.value for x in v)
+
+    def quant_blocks(self, head: int) -> torch.Tensor:
+        """View of head `head`'s slab [B][n_max // group][block_bytes] of the quantised buffer (for inspection)."""
+        slab, bb, _, _, _ = self.quant_layout(head)
+        nb = self.n_max // self.q_group
+        return self.qcache[slab:slab + self.B * nb * bb].view(self.B, nb, bb)
 
     def decode_static(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
         """eigen_attn_decode_static: decode with the partials in the library's built-in scratch array

@@ -167,6 +167,12 @@ struct eigen_attn {
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  // quantised copy of the cache (Section 5.3), attached by the caller
+  char* qcache = nullptr;
+  int q_group = 0;
+  int32_t qlen = 0;       // rows held as codes (a multiple of q_group)
+  int q_max_stage_bytes = 0;
+  std::vector<ea::QuantHead> qheads;
   char err[256];
 };
 
@@ -183,6 +189,40 @@ ea_status fail(eigen_attn_t h, ea_status st, const char* fmt, ...) {
 }
 ea_status cuda_fail(eigen_attn_t h, cudaError_t e, const char* what) {
   return fail(h, EA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+// Layout of the quantised buffer for group size G: the per-head table, then one slab per head.
+size_t make_quant_layout(const eigen_attn* h, int G, std::vector<ea::QuantHead>* qheads, int* max_stage_bytes) {
+  const int H = h->desc.n_heads;
+  const int64_t blocks_max = h->desc.n_max / G;
+  qheads->resize(H);
+  size_t off = align_up(sizeof(ea::QuantHead) * H);
+  int widest = 0;
+  for (int i = 0; i < H; ++i) {
+    const HeadInfo& hi = h->L.heads[i];
+    ea::QuantHead& q = (*qheads)[i];
+    memset(&q, 0, sizeof(q));
+    q.nvg = (hi.rp_v + G - 1) / G;
+    q.ks_off = G * hi.rp_k / 2;
+    q.vc_off = q.ks_off + 2 * hi.rp_k;
+    q.vs_off = q.vc_off + G * hi.rp_v / 2;
+    q.block_bytes = q.vs_off + 2 * G * q.nvg;
+    q.slab_off = static_cast<int64_t>(off);
+    off = align_up(off + static_cast<size_t>(h->desc.batch) * blocks_max * q.block_bytes);
+    const int stage = (128 / G) * q.block_bytes;
+    if (stage > widest) widest = stage;
+  }
+  if (max_stage_bytes) *max_stage_bytes = widest;
+  return off;
+}
+
+ea_status check_quant_args(eigen_attn_t h, const char* who, int32_t bits, int32_t group) {
+  if (bits != 4) return fail(h, EA_ERR_UNSUPPORTED, "%s: %d-bit codes (4 is built)", who, bits);
+  if (group != 16 && group != 32 && group != 64 && group != 128)
+    return fail(h, EA_ERR_UNSUPPORTED, "%s: group %d (16, 32, 64 or 128)", who, group);
+  if (h->desc.dtype != EA_BF16) return fail(h, EA_ERR_UNSUPPORTED, "%s: needs a bf16 layer", who);
+  if (h->desc.n_max < group) return fail(h, EA_ERR_SHAPE, "%s: n_max %d holds no group of %d rows", who, h->desc.n_max, group);
+  return EA_OK;
 }
 
 const HeadInfo* dev_heads(eigen_attn_t h) { return reinterpret_cast<const HeadInfo*>(h->ws + h->L.off_heads); }
@@ -697,6 +737,7 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
   if (len < 0 || len > h->desc.n_max)
     return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %d]", len, h->desc.n_max);
   h->len = len;
+  if (h->q_group && h->qlen > len) h->qlen = len / h->q_group * h->q_group;   // rows past len are forgotten
   return EA_OK;
 }
 
@@ -834,6 +875,150 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
   if (e != cudaSuccess) return cuda_fail(h, e, "set_rope");
   h->rope = true;
   h->rope_interleaved = interleaved ? 1 : 0;
+  return EA_OK;
+}
+
+// ---- Section 5.3: quantised copy of the rank-r cache
+
+ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, size_t* bytes) {
+  if (!h || !bytes) return EA_ERR_INVALID_ARG;
+  const ea_status st = check_quant_args(h, "quant_bytes", bits, group);
+  if (st != EA_OK) return st;
+  std::vector<ea::QuantHead> qh;
+  *bytes = make_quant_layout(h, group, &qh, nullptr);
+  return EA_OK;
+}
+
+ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
+                                  void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!d_qcache) {             // detach
+    h->qcache = nullptr; h->q_group = 0; h->qlen = 0;
+    return EA_OK;
+  }
+  const ea_status st = check_quant_args(h, "quant_attach", bits, group);
+  if (st != EA_OK) return st;
+  if (reinterpret_cast<uintptr_t>(d_qcache) % kAlign) return fail(h, EA_ERR_INVALID_ARG, "quant_attach: buffer not 256-byte aligned");
+  std::vector<ea::QuantHead> qh;
+  int widest = 0;
+  const size_t need = make_quant_layout(h, group, &qh, &widest);
+  if (bytes < need) return fail(h, EA_ERR_CAPACITY, "quant_attach: %zu bytes given, %zu needed", bytes, need);
+  if (ea::decode_quant_smem_bytes(widest, h->L.max_rp_v) > static_cast<size_t>(kSmemLimit))
+    return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: a stage of 128 rows does not fit in shared memory");
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(d_qcache, qh.data(), sizeof(ea::QuantHead) * qh.size(), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "quant_attach");
+  h->qcache = static_cast<char*>(d_qcache);
+  h->q_group = group;
+  h->qlen = 0;
+  h->q_max_stage_bytes = widest;
+  h->qheads.swap(qh);
+  return EA_OK;
+}
+
+namespace {
+void fill_quant_params(eigen_attn_t h, ea::QuantParams* p) {
+  *p = ea::QuantParams{};
+  p->heads = dev_heads(h);
+  p->qheads = reinterpret_cast<const ea::QuantHead*>(h->qcache);
+  p->basis = dev_basis(h);
+  p->cache = h->cache; p->qcache = h->qcache;
+  p->status = dev_status(h);
+  p->part_stride = h->L.part_stride;
+  p->B = h->desc.batch; p->H = h->desc.n_heads; p->d_head = h->desc.d_head;
+  p->n = h->len; p->n_max = h->desc.n_max;
+  p->nq = h->qlen; p->group = h->q_group; p->blocks_max = h->desc.n_max / h->q_group;
+}
+}  // namespace
+
+ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "quant_sync: no quantised buffer attached");
+  const int G = h->q_group;
+  const int b0 = h->qlen / G, b1 = h->len / G;
+  if (b1 <= b0) return EA_OK;
+  ea::QuantParams p;
+  fill_quant_params(h, &p);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // the second grid dimension holds at most 65535 blocks
+  for (int lo = b0; lo < b1; lo += 65535) {
+    p.b0 = lo; p.b1 = lo + 65535 < b1 ? lo + 65535 : b1;
+    const cudaError_t e = ea::launch_quantize_blocks(p, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, "quant_sync launch");
+  }
+  h->qlen = b1 * G;
+  return EA_OK;
+}
+
+ea_status eigen_attn_quant_len(eigen_attn_t h, int32_t* qlen) {
+  if (!h || !qlen) return EA_ERR_INVALID_ARG;
+  *qlen = h->qlen;
+  return EA_OK;
+}
+
+ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_offset, size_t* block_bytes,
+                                  size_t* k_scale_offset, size_t* v_code_offset, size_t* v_scale_offset) {
+  if (!h || !slab_offset || !block_bytes || !k_scale_offset || !v_code_offset || !v_scale_offset) return EA_ERR_INVALID_ARG;
+  if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "quant_layout: no quantised buffer attached");
+  if (head < 0 || head >= h->desc.n_heads) return fail(h, EA_ERR_SHAPE, "quant_layout: head %d", head);
+  const ea::QuantHead& q = h->qheads[head];
+  *slab_offset = static_cast<size_t>(q.slab_off);
+  *block_bytes = static_cast<size_t>(q.block_bytes);
+  *k_scale_offset = static_cast<size_t>(q.ks_off);
+  *v_code_offset = static_cast<size_t>(q.vc_off);
+  *v_scale_offset = static_cast<size_t>(q.vs_off);
+  return EA_OK;
+}
+
+ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
+                                  int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: no quantised buffer attached");
+  if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: NULL q or out");
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK)) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: unknown flag 0x%x", flags);
+  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "decode_quant: not available with a rotary embedding");
+  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_quant: the cache is empty");
+  const Layout& L = h->L;
+  ea::QuantParams p;
+  fill_quant_params(h, &p);
+  p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
+  p.out = d_out; p.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
+  p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
+  p.nst = (p.nq + 127) / 128;
+  p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+  p.flags = flags;
+  const size_t smem = ea::decode_quant_smem_bytes(h->q_max_stage_bytes, L.max_rp_v);
+  const int max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
+  // CTAs per unit: waves of (SMs x resident CTAs), a start-up worth a few stages per CTA, and room for
+  // units x splits partials in the workspace
+  int ctas_per_sm = static_cast<int>(static_cast<size_t>(228 * 1024) / (smem + 1024));
+  const int reg_limit = max_rp <= 80 ? 3 : 2;
+  if (ctas_per_sm > reg_limit) ctas_per_sm = reg_limit;
+  if (ctas_per_sm < 1) ctas_per_sm = 1;
+  const int64_t units = static_cast<int64_t>(p.B) * p.H;
+  int64_t cap = (units + kMaxDecodeCtas) * kPartialSlack / units;
+  if (cap > p.nst) cap = p.nst;
+  if (cap > 65535) cap = 65535;
+  if (cap < 1) cap = 1;
+  int64_t splits = 1;
+  if (h->opt_ctas > 0) {
+    splits = (h->opt_ctas + units - 1) / units;
+    if (splits > cap) splits = cap;
+  } else {
+    const int64_t wave = static_cast<int64_t>(h->sm_count) * ctas_per_sm;
+    int64_t best = INT64_MAX;
+    for (int64_t s2 = 1; s2 <= cap && s2 <= 256; ++s2) {
+      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nst + s2 - 1) / s2 + 4);
+      if (cost < best) { best = cost; splits = s2; }
+    }
+  }
+  p.splits = static_cast<int32_t>(splits);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (h->ev_start) cudaEventRecord(h->ev_start, s);
+  const cudaError_t e = ea::launch_decode_quant(p, max_rp, smem, s, &h->launches);
+  if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  if (e != cudaSuccess) return cuda_fail(h, e, "decode_quant launch");
   return EA_OK;
 }
 

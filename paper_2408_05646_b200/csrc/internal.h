@@ -170,6 +170,44 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
   uint32_t flags;
 };
 
+// Quantised copy of the cache (Section 5.3 of the paper): per head a slab [B][blocks_max][block_bytes]; a block
+// holds G consecutive rows of one sequence as 4-bit codes (code + 8 in a nibble, eight channels per 32-bit word,
+// channel 8j+k in bits 4k..4k+3) and half-precision scales:
+//   K codes  [rp_k/8][G] words     K scales [rp_k] halves        (one scale per channel and block)
+//   V codes  [rp_v/8][G] words     V scales [nvg][G] halves      (one scale per row and G channels)
+struct QuantHead {
+  int64_t slab_off;        // byte offset of the head's slab in the quantised buffer
+  int32_t block_bytes;
+  int32_t ks_off, vc_off, vs_off;   // byte offsets of K scales, V codes, V scales inside a block
+  int32_t nvg;             // scale groups per value row = ceil(rp_v / G)
+  int32_t pad_;
+};
+
+struct QuantParams {
+  const HeadInfo* heads;
+  const QuantHead* qheads;
+  const float* basis;
+  const char* cache;        // the 16-bit cache: source of the quantiser, and rows [nq, n) of a decode
+  char* qcache;
+  const void* q;            // decode: [B][1][H][d_head] or packed rank-space [B][sum rp_k]
+  int64_t q_stride_b;
+  void* out;
+  int64_t out_stride_b;
+  float* partials;          // [B*H][splits][part_stride]: m, l, pad, pad, o'[rp_v]
+  int* status;
+  int32_t part_stride;
+  int32_t B, H, d_head;
+  int32_t n, n_max;
+  int32_t nq;               // rows held as codes (a multiple of group)
+  int32_t group;            // G: 16, 32, 64 or 128
+  int32_t blocks_max;       // blocks per sequence the buffer holds = n_max / G
+  int32_t nst;              // stages of 128 rows per unit = ceil(nq / 128)
+  int32_t splits;           // CTAs per unit
+  int32_t b0, b1;           // quantiser: blocks [b0, b1) of every sequence
+  float q_scale;            // log2(e) / sqrt(d_head)
+  uint32_t flags;
+};
+
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.
 cudaError_t launch_project_append(const ProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t smem_bytes,
@@ -186,6 +224,10 @@ cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem
 cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s,
                               uint64_t* launches);
+
+cudaError_t launch_quantize_blocks(const QuantParams& p, cudaStream_t s, uint64_t* launches);
+size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v);
+cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches);
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
 // library's own partials array on the current device.  Resolves the address on first use per device.

@@ -1,0 +1,419 @@
+// Quantised rank-r cache (Section 5.3 of the paper, "Eigen Attention with Quantization"; sizes in Table 8):
+// keys per channel, values per token, integer codes of 4 bits with one half-precision scale per group of G.
+//
+//   s = half( min(max|x| / 7, 65504) ),   c = clip( rint(x / s), -7, 7 ),   x^ = c * s      (c + 8 is stored)
+//
+// A key group is G consecutive tokens of one channel, a value group is G consecutive channels of one token.
+// Rows that do not fill a block of G tokens yet stay in the 16-bit cache and are attended from there.
+//
+// quantize_blocks_kernel: one CTA per (sequence, head, block); reads the block's G rows of K' and V' from the
+//   16-bit cache, takes the group maxima, writes codes and scales.  Divisions are IEEE single precision and the
+//   rounding is to nearest even, so the codes are a function of the stored rows alone.
+// decode_quant_kernel: split-KV decode over the codes.  A CTA owns a run of 128-row stages of one unit; one
+//   thread streams them into a shared-memory ring with bulk copies, every thread owns one row of a stage.  The
+//   key scales are folded into the query once per block (q'_c * s_c), the value scale into the softmax weight
+//   (p * s_g), so a cached element costs one mask, half a packed subtract and half a packed multiply-add.
+//   A nibble is turned into a float without a conversion instruction: masked in place and OR-ed with the
+//   exponent whose unit in the last place lines up with the nibble's lowest bit, (w & (15 << 4k)) | E_k is
+//   2^(23-4k) + nibble exactly; subtracting 2^(23-4k) + 8 leaves the signed code.
+// quant_combine_kernel: merges the splits of a unit, normalises and lifts through (U^V)^T.
+// Every wait is bounded.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "internal.h"
+#include "tc_common.cuh"
+
+namespace ea {
+namespace {
+
+using namespace tc;
+
+constexpr int kQThreads = 128;
+constexpr int kQStages = 4;           // ring slots of the decode kernel
+constexpr int kStageRows = 128;
+
+// ---------------------------------------------------------------- quantiser
+
+__device__ __forceinline__ uint32_t code_nibble(float x, float s) {
+  float c = s > 0.f ? rintf(x / s) : 0.f;
+  c = fminf(fmaxf(c, -7.f), 7.f);
+  return static_cast<uint32_t>(static_cast<int>(c) + 8);
+}
+
+__global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantParams p) {
+  __shared__ __align__(16) __nv_bfloat16 tile[128 * 128];   // G rows x rp (row-major), K' then V'
+  __shared__ float scale_sm[256];                         // K: [rp_k]; V: [nvg][G]
+  const int tid = threadIdx.x;
+  const int unit = blockIdx.x, blk = p.b0 + blockIdx.y;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const QuantHead qh = p.qheads[h];
+  const int G = p.group;
+  const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(blk) * G;
+  char* dst = p.qcache + qh.slab_off + (static_cast<int64_t>(b) * p.blocks_max + blk) * qh.block_bytes;
+
+  for (int pass = 0; pass < 2; ++pass) {
+    const int rp = pass ? hd.rp_v : hd.rp_k;
+    const uint4* src = reinterpret_cast<const uint4*>(p.cache + (pass ? hd.v_off : hd.k_off) + row0 * rp * 2);
+    const int chunks = G * rp / 8;
+    for (int i = tid; i < chunks; i += kQThreads) reinterpret_cast<uint4*>(tile)[i] = src[i];
+    __syncthreads();
+    if (pass == 0) {          // keys: one scale per channel over the block's G tokens
+      __half* ks = reinterpret_cast<__half*>(dst + qh.ks_off);
+      for (int c = tid; c < rp; c += kQThreads) {
+        float amax = 0.f;
+        for (int r = 0; r < G; ++r) amax = fmaxf(amax, fabsf(__bfloat162float(tile[r * rp + c])));
+        const __half s16 = __float2half_rn(fminf(amax / 7.f, 65504.f));
+        ks[c] = s16;
+        scale_sm[c] = __half2float(s16);
+      }
+    } else {                  // values: one scale per token and G channels
+      __half* vs = reinterpret_cast<__half*>(dst + qh.vs_off);
+      for (int i = tid; i < qh.nvg * G; i += kQThreads) {
+        const int g = i / G, r = i - g * G;
+        const int c1 = min(rp, (g + 1) * G);
+        float amax = 0.f;
+        for (int c = g * G; c < c1; ++c) amax = fmaxf(amax, fabsf(__bfloat162float(tile[r * rp + c])));
+        const __half s16 = __float2half_rn(fminf(amax / 7.f, 65504.f));
+        vs[i] = s16;
+        scale_sm[i] = __half2float(s16);
+      }
+    }
+    __syncthreads();
+    uint32_t* codes = reinterpret_cast<uint32_t*>(dst + (pass ? qh.vc_off : 0));
+    const int words = (rp / 8) * G;
+    for (int i = tid; i < words; i += kQThreads) {
+      const int j = i / G, r = i - j * G;
+      uint32_t w = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int c = 8 * j + k;
+        const float s = pass ? scale_sm[(c / G) * G + r] : scale_sm[c];
+        w |= code_nibble(__bfloat162float(tile[r * rp + c]), s) << (4 * k);
+      }
+      codes[i] = w;
+    }
+    __syncthreads();          // the tile and the scales are reused by the second pass
+  }
+}
+
+// ---------------------------------------------------------------- decode over the codes
+
+struct __align__(16) QuantSmemHeader {
+  unsigned long long full[kQStages];
+  float wmax[4], wsum[4];
+  float qraw[128];         // the unit's query as fp32
+  float qp[128];           // q' * log2(e)/sqrt(d_head)
+};
+constexpr int kQsOffset = 2048;                     // per warp: q'_c * s_c of (up to) two blocks, [2][128] floats
+constexpr int kRingOffset = kQsOffset + 4 * 2 * 128 * 4;
+static_assert(sizeof(QuantSmemHeader) <= kQsOffset, "header overlaps the scaled-query area");
+
+// Eight codes of a word as four packed float pairs (exact small integers in -7..7; a nibble 0 gives -8).
+struct Consts {
+  unsigned long long c01, c23, c45, c67;
+};
+__device__ __forceinline__ Consts make_consts() {
+  Consts c;
+  c.c01 = pack2(-8388616.f, -524296.f);             // -(2^23 + 8), -(2^19 + 8)
+  c.c23 = pack2(-32776.f, -2056.f);                 // -(2^15 + 8), -(2^11 + 8)
+  c.c45 = pack2(-136.f, -32776.f);                  // -(2^7 + 8), then nibbles 5..7 after a shift by 12
+  c.c67 = pack2(-2056.f, -136.f);
+  return c;
+}
+__device__ __forceinline__ void codes_to_floats(uint32_t w, const Consts& k, unsigned long long (&f)[4]) {
+  const uint32_t u = w >> 12;
+  const float x0 = __uint_as_float((w & 0x0000000Fu) | 0x4B000000u);
+  const float x1 = __uint_as_float((w & 0x000000F0u) | 0x49000000u);
+  const float x2 = __uint_as_float((w & 0x00000F00u) | 0x47000000u);
+  const float x3 = __uint_as_float((w & 0x0000F000u) | 0x45000000u);
+  const float x4 = __uint_as_float((w & 0x000F0000u) | 0x43000000u);
+  const float x5 = __uint_as_float((u & 0x00000F00u) | 0x47000000u);
+  const float x6 = __uint_as_float((u & 0x0000F000u) | 0x45000000u);
+  const float x7 = __uint_as_float((u & 0x000F0000u) | 0x43000000u);
+  f[0] = add2p(pack2(x0, x1), k.c01);
+  f[1] = add2p(pack2(x2, x3), k.c23);
+  f[2] = add2p(pack2(x4, x5), k.c45);
+  f[3] = add2p(pack2(x6, x7), k.c67);
+}
+__device__ __forceinline__ void bf16x8_to_floats(const uint4& x, unsigned long long (&f)[4]) {
+  f[0] = pack2(__uint_as_float(x.x << 16), __uint_as_float(x.x & 0xffff0000u));
+  f[1] = pack2(__uint_as_float(x.y << 16), __uint_as_float(x.y & 0xffff0000u));
+  f[2] = pack2(__uint_as_float(x.z << 16), __uint_as_float(x.z & 0xffff0000u));
+  f[3] = pack2(__uint_as_float(x.w << 16), __uint_as_float(x.w & 0xffff0000u));
+}
+
+template <int NW, int MINB>   // NW: 8-channel words a row can have (widest padded rank / 8)
+__global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const QuantParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  QuantSmemHeader* hdr = reinterpret_cast<QuantSmemHeader*>(smem);
+  float* qs_w = reinterpret_cast<float*>(smem + kQsOffset) + (threadIdx.x >> 5) * 256;
+  unsigned char* ring = smem + kRingOffset;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int unit = blockIdx.x, split = blockIdx.y;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const QuantHead qh = p.qheads[h];
+  const int G = p.group;
+  const int gshift = 31 - __clz(G);
+  const int bps = kStageRows >> gshift;                       // blocks per stage
+  const int nqb = p.nq >> gshift;                             // blocks held as codes
+  const int nwk = hd.rp_k >> 3, nwv = hd.rp_v >> 3;
+  const int stage_stride = (bps * qh.block_bytes + 127) & ~127;
+
+  const int per = (p.nst + p.splits - 1) / p.splits;
+  const int s_lo = min(p.nst, split * per), s_hi = min(p.nst, s_lo + per);
+  const char* slab = p.qcache + qh.slab_off + static_cast<int64_t>(b) * p.blocks_max * qh.block_bytes;
+
+  if (tid == 0) {
+    for (int s = 0; s < kQStages; ++s) mbar_init(&hdr->full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const uint64_t policy = policy_evict_first();
+  auto issue = [&](int s, int slot) {                         // thread 0
+    const int nblk = min(bps, nqb - s * bps);
+    const uint32_t bytes = static_cast<uint32_t>(nblk) * qh.block_bytes;
+    mbar_arrive_expect_tx(&hdr->full[slot], bytes);
+    bulk_load(ring + slot * stage_stride, slab + static_cast<int64_t>(s) * bps * qh.block_bytes, bytes,
+              &hdr->full[slot], policy);
+  };
+  if (tid == 0)
+    for (int i = 0; i < kQStages && s_lo + i < s_hi; ++i) issue(s_lo + i, i);
+
+  // q' = q U^K, scaled into the base-2 domain
+  const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(p.q);
+  if (p.flags & 0x1u) {
+    if (tid < hd.rp_k) hdr->qp[tid] = __bfloat162float(q[b * p.q_stride_b + hd.lr_k_off + tid]) * p.q_scale;
+  } else {
+    if (tid < p.d_head) hdr->qraw[tid] = __bfloat162float(q[b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head + tid]);
+    __syncthreads();
+    if (tid < hd.rp_k) {
+      const float* U = p.basis + hd.uk_off + tid;
+      float acc = 0.f;
+#pragma unroll 8
+      for (int d = 0; d < p.d_head; ++d) acc = fmaf(hdr->qraw[d], __ldg(U + d * hd.rp_k), acc);
+      hdr->qp[tid] = acc * p.q_scale;
+    }
+  }
+  __syncthreads();
+
+  const Consts kc = make_consts();
+  unsigned long long o[NW * 4];
+#pragma unroll
+  for (int i = 0; i < NW * 4; ++i) o[i] = 0ull;
+  float m = -INFINITY, l = 0.f;
+  const float slope2 = hd.alibi_slope2;
+  const int pos_q = p.n - 1;
+  // online softmax of one score: returns the weight of the row under the (possibly raised) running maximum
+  auto weight = [&](float s) {
+    if (s > m) {
+      const float c = ex2(m - s);
+      const unsigned long long cc = pack2(c, c);
+      l *= c;
+#pragma unroll
+      for (int i = 0; i < NW * 4; ++i) o[i] = mul2p(o[i], cc);
+      m = s;
+    }
+    const float pr = ex2(s - m);
+    l += pr;
+    return pr;
+  };
+
+  bool aborted = false;
+  for (int s = s_lo; s < s_hi; ++s) {
+    const int it = s - s_lo, slot = it % kQStages;
+    const bool ok = mbar_wait(&hdr->full[slot], (it / kQStages) & 1, p.status);
+    const unsigned char* st = ring + slot * stage_stride;
+    const int nblk = min(bps, nqb - s * bps);
+    {   // the warp's blocks: q'_c * s_c
+      const int wb0 = (warp * 32) >> gshift, nwb = G >= 32 ? 1 : 2;
+      for (int i = 0; i < nwb; ++i)
+        if (wb0 + i < nblk) {
+          const __half* ks = reinterpret_cast<const __half*>(st + (wb0 + i) * qh.block_bytes + qh.ks_off);
+          for (int c = lane; c < hd.rp_k; c += 32) qs_w[i * 128 + c] = hdr->qp[c] * __half2float(ks[c]);
+        }
+      __syncwarp();
+    }
+    const int blk = tid >> gshift, ri = tid & (G - 1);
+    if (blk < nblk) {
+      const unsigned char* bb = st + blk * qh.block_bytes;
+      const uint32_t* kw = reinterpret_cast<const uint32_t*>(bb) + ri;
+      const float* qsr = qs_w + (G >= 32 ? 0 : (lane >> 4) * 128);
+      unsigned long long a0 = 0ull, a1 = 0ull, a2 = 0ull, a3 = 0ull;
+#pragma unroll
+      for (int j = 0; j < NW; ++j)
+        if (j < nwk) {
+          unsigned long long f[4];
+          codes_to_floats(kw[j * G], kc, f);
+          const ulonglong2 q0 = *reinterpret_cast<const ulonglong2*>(qsr + 8 * j);
+          const ulonglong2 q1 = *reinterpret_cast<const ulonglong2*>(qsr + 8 * j + 4);
+          a0 = fma2p(f[0], q0.x, a0); a1 = fma2p(f[1], q0.y, a1);
+          a2 = fma2p(f[2], q1.x, a2); a3 = fma2p(f[3], q1.y, a3);
+        }
+      float s0, s1;
+      unpack2(add2p(add2p(a0, a1), add2p(a2, a3)), s0, s1);
+      const int j_abs = s * kStageRows + tid;
+      const float pr = weight(fmaf(slope2, static_cast<float>(j_abs - pos_q), s0 + s1));
+      const uint32_t* vw = reinterpret_cast<const uint32_t*>(bb + qh.vc_off) + ri;
+      const __half* vs = reinterpret_cast<const __half*>(bb + qh.vs_off) + ri;
+#pragma unroll
+      for (int j = 0; j < NW; ++j)
+        if (j < nwv) {
+          const float sv = pr * __half2float(vs[((8 * j) >> gshift) * G]);
+          const unsigned long long svp = pack2(sv, sv);
+          unsigned long long f[4];
+          codes_to_floats(vw[j * G], kc, f);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) o[4 * j + i] = fma2p(f[i], svp, o[4 * j + i]);
+        }
+    }
+    // everyone is done with the slot (and with this warp's scaled query); a failed wait ends the loop for all
+    const int all_ok = __syncthreads_and(ok ? 1 : 0);
+    if (tid == 0 && all_ok && s + kQStages < s_hi) issue(s + kQStages, slot);
+    if (!all_ok) { aborted = true; break; }
+  }
+
+  // rows that are not quantised yet, straight from the 16-bit cache (the last split takes them)
+  if (split == p.splits - 1 && !aborted) {
+    for (int j = p.nq + tid; j < p.n; j += kQThreads) {
+      const int64_t row = static_cast<int64_t>(b) * p.n_max + j;
+      const uint4* kr = reinterpret_cast<const uint4*>(p.cache + hd.k_off + row * hd.rp_k * 2);
+      const uint4* vr = reinterpret_cast<const uint4*>(p.cache + hd.v_off + row * hd.rp_v * 2);
+      unsigned long long a0 = 0ull, a1 = 0ull, a2 = 0ull, a3 = 0ull;
+#pragma unroll
+      for (int c = 0; c < NW; ++c)
+        if (c < nwk) {
+          unsigned long long f[4];
+          bf16x8_to_floats(__ldg(kr + c), f);
+          const ulonglong2 q0 = *reinterpret_cast<const ulonglong2*>(hdr->qp + 8 * c);
+          const ulonglong2 q1 = *reinterpret_cast<const ulonglong2*>(hdr->qp + 8 * c + 4);
+          a0 = fma2p(f[0], q0.x, a0); a1 = fma2p(f[1], q0.y, a1);
+          a2 = fma2p(f[2], q1.x, a2); a3 = fma2p(f[3], q1.y, a3);
+        }
+      float s0, s1;
+      unpack2(add2p(add2p(a0, a1), add2p(a2, a3)), s0, s1);
+      const float pr = weight(fmaf(slope2, static_cast<float>(j - pos_q), s0 + s1));
+      const unsigned long long prp = pack2(pr, pr);
+#pragma unroll
+      for (int c = 0; c < NW; ++c)
+        if (c < nwv) {
+          unsigned long long f[4];
+          bf16x8_to_floats(__ldg(vr + c), f);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) o[4 * c + i] = fma2p(f[i], prp, o[4 * c + i]);
+        }
+    }
+  }
+
+  // ---- merge the 128 threads into one partial (max, sum, o'[rp_v]); the ring doubles as the staging area
+  float wm = m;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, d));
+  if (lane == 0) hdr->wmax[warp] = wm;
+  __syncthreads();
+  const float M = fmaxf(fmaxf(hdr->wmax[0], hdr->wmax[1]), fmaxf(hdr->wmax[2], hdr->wmax[3]));
+  const float f = (m == -INFINITY) ? 0.f : ex2(m - M);
+  float ls = l * f;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, d);
+  if (lane == 0) hdr->wsum[warp] = ls;
+  float* red = reinterpret_cast<float*>(ring);               // [128][rp_v + 1]
+  const int rstride = hd.rp_v + 1;
+  if (!aborted) {
+#pragma unroll
+    for (int i = 0; i < NW * 4; ++i)
+      if (2 * i < hd.rp_v) {
+        float x0, x1;
+        unpack2(o[i], x0, x1);
+        red[tid * rstride + 2 * i] = x0 * f;
+        red[tid * rstride + 2 * i + 1] = x1 * f;
+      }
+  }
+  __syncthreads();
+  float* part = p.partials + (static_cast<size_t>(unit) * p.splits + split) * p.part_stride;
+  if (tid < hd.rp_v) {
+    float acc = 0.f;
+    if (!aborted)
+      for (int r = 0; r < kQThreads; ++r) acc += red[r * rstride + tid];
+    part[4 + tid] = acc;
+  }
+  if (tid == 0) {
+    part[0] = M;
+    part[1] = (hdr->wsum[0] + hdr->wsum[1]) + (hdr->wsum[2] + hdr->wsum[3]);
+  }
+}
+
+__global__ void __launch_bounds__(128) quant_combine_kernel(const QuantParams p) {
+  __shared__ float o_sm[128];
+  const int unit = blockIdx.x, t = threadIdx.x;
+  const int h = unit / p.B, b = unit - h * p.B;
+  const HeadInfo hd = p.heads[h];
+  const float* base = p.partials + static_cast<size_t>(unit) * p.splits * p.part_stride;
+  float M = -INFINITY;
+  for (int c = 0; c < p.splits; ++c) M = fmaxf(M, base[static_cast<size_t>(c) * p.part_stride]);
+  float L = 0.f, acc = 0.f;
+  for (int c = 0; c < p.splits; ++c) {
+    const float* part = base + static_cast<size_t>(c) * p.part_stride;
+    const float f = ex2(part[0] - M);                        // 0 for a piece without rows
+    L = fmaf(part[1], f, L);
+    if (t < hd.rp_v) acc = fmaf(part[4 + t], f, acc);
+  }
+  const float o = acc / L;
+  __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out);
+  if (p.flags & 0x2u) {
+    if (t < hd.rp_v) out[b * p.out_stride_b + hd.lr_v_off + t] = __float2bfloat16_rn(o);
+    return;
+  }
+  if (t < hd.rp_v) o_sm[t] = o;
+  __syncthreads();
+  if (t < p.d_head) {
+    const float* Ut = p.basis + hd.uvt_off;                  // (U^V)^T : rp_v x d_head
+    float y = 0.f;
+    for (int c = 0; c < hd.rp_v; ++c) y = fmaf(o_sm[c], __ldg(Ut + c * p.d_head + t), y);
+    out[b * p.out_stride_b + static_cast<int64_t>(h) * p.d_head + t] = __float2bfloat16_rn(y);
+  }
+}
+
+template <int NW, int MINB>
+cudaError_t launch_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
+  static size_t configured = 0;
+  if (smem > configured) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_quant_kernel<NW, MINB>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  decode_quant_kernel<NW, MINB><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_blocks(const QuantParams& p, cudaStream_t s, uint64_t* launches) {
+  if (p.b1 <= p.b0) return cudaSuccess;
+  quantize_blocks_kernel<<<dim3(p.B * p.H, p.b1 - p.b0), kQThreads, 0, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v) {
+  const size_t ring = static_cast<size_t>(kQStages) * ((max_stage_bytes + 127) & ~127);
+  const size_t red = static_cast<size_t>(kQThreads) * (max_rp_v + 1) * sizeof(float);
+  return kRingOffset + (ring > red ? ring : red);
+}
+
+cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches) {
+  cudaError_t e;
+  if (max_rp <= 64) e = launch_variant<8, 3>(p, smem, s);
+  else if (max_rp <= 80) e = launch_variant<10, 3>(p, smem, s);
+  else e = launch_variant<16, 2>(p, smem, s);
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  quant_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace ea

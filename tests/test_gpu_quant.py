@@ -1,0 +1,226 @@
+"""GPU parity of the quantised rank-r cache (Section 5.3, Table 8) against the oracle, through the C ABI.
+
+Codes and scales are integer / bit work and must match exactly: both sides start from the same 16-bit rows
+(rank-space rows handed to the library as they are, so no projection arithmetic precedes the quantiser) and
+take every rounding decision in single precision.  The decode over the codes is compared with the fp64 oracle
+over the de-quantised rows within the bf16 tolerances of the other decode tests."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, make_case, oracle_layer, to_np
+from oracle import kv_quant as kq
+from paper_2408_05646_b200 import synth
+
+pytestmark = pytest.mark.gpu
+BF16 = torch.bfloat16
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    return binding
+
+
+def rank_space_case(B_, H, d, rk, rv, n, seed, q_scale=1.0):
+    """Bases, a query, and the rank-space rows K' = K U^K, V' = V U^V rounded to bf16 on the host: the packed
+    tensors for the library and the per-unit float64 arrays (the same values) for the oracle."""
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, BF16, seed_cfg=seed, q_scale=q_scale)
+    offs_k = np.concatenate([[0], np.cumsum([(r + 7) // 8 * 8 for r in rk])])
+    offs_v = np.concatenate([[0], np.cumsum([(r + 7) // 8 * 8 for r in rv])])
+    kp = torch.zeros((B_, n, int(offs_k[-1])), dtype=BF16)
+    vp = torch.zeros((B_, n, int(offs_v[-1])), dtype=BF16)
+    kn, vn = to_np(k), to_np(v)
+    rows = {}
+    for h in range(H):
+        a = torch.from_numpy(kn[:, :, h, :] @ U_k[h].astype(np.float64)).to(BF16)
+        c = torch.from_numpy(vn[:, :, h, :] @ U_v[h].astype(np.float64)).to(BF16)
+        kp[:, :, offs_k[h]:offs_k[h] + rk[h]] = a
+        vp[:, :, offs_v[h]:offs_v[h] + rv[h]] = c
+        for b in range(B_):
+            rows[(b, h)] = (a[b].double().numpy(), c[b].double().numpy())
+    return U_k, U_v, q, kp.cuda(), vp.cuda(), rows
+
+
+def fill_both(B, B_, H, d, rk, rv, n, n_max, seed, group, alibi=None, q_scale=1.0):
+    U_k, U_v, q, kp, vp, rows = rank_space_case(B_, H, d, rk, rv, n, seed, q_scale)
+    lay = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v)
+    lay.append_kv(kp, vp, preprojected=True)
+    ref = oracle_layer(B_, H, d, U_k, U_v, alibi_slopes=alibi)
+    for u, (a, c) in rows.items():
+        ref.Kp[u], ref.Vp[u] = a, c
+    ref.set_len(n)
+    if alibi is not None:
+        lay.set_alibi(alibi)
+    lay.quant_attach(4, group)
+    return lay, ref, q, rows
+
+
+def unpack_codes(words: np.ndarray) -> np.ndarray:
+    """words [rp/8][G] uint32 -> codes [G][rp] (channel 8j+k in bits 4k..4k+3 of word j, stored as code + 8)."""
+    nw, G = words.shape
+    out = np.zeros((G, nw * 8), dtype=np.int64)
+    for k in range(8):
+        out[:, k::8] = ((words.T >> np.uint32(4 * k)) & np.uint32(15)).astype(np.int64) - 8
+    return out
+
+
+def read_block(lay, head, b, blk, G, rp_k, rp_v):
+    _, bb, ks_off, vc_off, vs_off = lay.quant_layout(head)
+    raw = lay.quant_blocks(head)[b, blk].cpu().numpy()
+    kc = unpack_codes(raw[:ks_off].view(np.uint32).reshape(rp_k // 8, G))
+    ks = raw[ks_off:vc_off].view(np.float16)
+    vc = unpack_codes(raw[vc_off:vs_off].view(np.uint32).reshape(rp_v // 8, G))
+    nvg = (rp_v + G - 1) // G
+    vs = raw[vs_off:vs_off + 2 * G * nvg].view(np.float16).reshape(nvg, G).T       # -> [G][nvg]
+    return kc, ks, vc, vs
+
+
+@pytest.mark.parametrize("G,H,d,rk,rv,n", [
+    (32, 2, 128, [80, 80], [80, 80], 200),            # the headline rank; 6 blocks and 8 rows left over
+    (16, 2, 128, [80, 48], [64, 80], 100),            # smallest group: five value groups per row
+    (64, 3, 64, [24, 64, 37], [56, 8, 64], 300),      # ranks that are not multiples of 8 (zero padding inside a word)
+    (128, 2, 128, [128, 80], [128, 96], 400),         # widest rank; one value group per row
+])
+def test_codes_and_scales_are_bit_exact(B, G, H, d, rk, rv, n):
+    B_ = 2
+    lay, ref, q, rows = fill_both(B, B_, H, d, rk, rv, n, n + 5, 171, G)
+    lay.quant_sync()
+    torch.cuda.synchronize()
+    assert lay.quant_len == n // G * G
+    for h in range(H):
+        rp_k, rp_v = (rk[h] + 7) // 8 * 8, (rv[h] + 7) // 8 * 8
+        for b in range(B_):
+            Kp, Vp = rows[(b, h)]
+            nq = n // G * G
+            kc_ref, ks_ref = kq.quantize_keys(Kp[:nq], 4, G)
+            vc_ref, vs_ref = kq.quantize_values(Vp[:nq], 4, G)
+            for blk in range(n // G):
+                kc, ks, vc, vs = read_block(lay, h, b, blk, G, rp_k, rp_v)
+                sl = slice(blk * G, (blk + 1) * G)
+                assert np.array_equal(kc[:, :rk[h]], kc_ref[sl]), (h, b, blk, "key codes")
+                assert np.array_equal(ks[:rk[h]], ks_ref[blk]), (h, b, blk, "key scales")
+                assert np.array_equal(vc[:, :rv[h]], vc_ref[sl]), (h, b, blk, "value codes")
+                assert np.array_equal(vs[:, :vs_ref.shape[1]], vs_ref[sl]), (h, b, blk, "value scales")
+                assert np.all(kc[:, rk[h]:] == 0) and np.all(vc[:, rv[h]:] == 0)      # padding columns hold zeros
+
+
+@pytest.mark.parametrize("G,H,d,rk,rv,n", [
+    (32, 2, 128, [80, 80], [80, 80], 128),            # exactly one stage, nothing left over
+    (32, 2, 128, [80, 80], [80, 80], 1037),           # several stages, a partial last stage, 13 rows left over
+    (16, 2, 128, [80, 48], [64, 80], 777),            # two blocks per warp
+    (64, 3, 64, [24, 64, 37], [56, 8, 64], 2500),     # per-head ranks, small d_head
+    (128, 2, 128, [128, 80], [128, 96], 1500),        # widest rank (the 16-word kernel)
+    (32, 1, 128, [80], [80], 20),                     # shorter than one group: all rows come from the 16-bit cache
+    (32, 4, 128, [80] * 4, [80] * 4, 9000),           # many stages per CTA, several splits
+])
+def test_decode_quant_matches_oracle(B, G, H, d, rk, rv, n):
+    B_ = 2
+    lay, ref, q, _ = fill_both(B, B_, H, d, rk, rv, n, n + 7 + G, 172, G)
+    lay.quant_sync()
+    out = lay.decode_quant(q)
+    lay.poll_status()
+    res = ref.decode_quant(to_np(q), 4, G)
+    want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out, want, BF16, f"decode_quant G={G} n={n}")
+    # the quantisation error itself is far above the tolerance: the test would notice codes that are ignored
+    plain = ref.decode_dense(to_np(q))
+    if n >= 4 * G:
+        assert np.abs(plain - want).max() > 1e-3
+
+
+def test_decode_quant_with_rows_that_are_not_synced_yet(B):
+    """quant_sync is the caller's to schedule: rows appended after it are read from the 16-bit cache."""
+    B_, H, d, G = 2, 2, 128, 32
+    n0, n1 = 300, 420
+    U_k, U_v, q, kp, vp, rows = rank_space_case(B_, H, d, [80, 64], [80, 72], n1, 173)
+    lay = B.EigenAttnLayer(B_, H, d, n1, BF16, U_k, U_v)
+    lay.quant_attach(4, G)
+    lay.append_kv(kp[:, :n0].contiguous(), vp[:, :n0].contiguous(), preprojected=True)
+    lay.quant_sync()
+    assert lay.quant_len == 288
+    lay.append_kv(kp[:, n0:].contiguous(), vp[:, n0:].contiguous(), preprojected=True)
+    out = lay.decode_quant(q)
+    lay.poll_status()
+    # the oracle's view with 288 quantised rows: quantise the first 288, keep the rest
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    for u, (a, c) in rows.items():
+        Kq, Vq = kq.quantized_view(a[:288], c[:288], 4, G)
+        ref.Kp[u], ref.Vp[u] = np.concatenate([Kq, a[288:]]), np.concatenate([Vq, c[288:]])
+    ref.set_len(n1)
+    assert_close(out, ref.decode_dense(to_np(q)), BF16, "unsynced tail")
+    # after the next sync the newer blocks are codes too
+    lay.quant_sync()
+    assert lay.quant_len == 416
+    out2 = lay.decode_quant(q)
+    ref2 = oracle_layer(B_, H, d, U_k, U_v)
+    for u, (a, c) in rows.items():
+        ref2.Kp[u], ref2.Vp[u] = a, c
+    ref2.set_len(n1)
+    res = ref2.decode_quant(to_np(q), 4, G)
+    want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out2, want, BF16, "after the second sync")
+    # rewinding below the quantised length forgets whole blocks
+    lay.set_len(100)
+    assert lay.quant_len == 96
+
+
+def test_decode_quant_with_peaked_attention_and_alibi(B):
+    """Few rows carry the softmax (scaled query, steep bias on one head): a wrong scale or code of a single row
+    is not averaged away."""
+    B_, H, d, G, n = 2, 4, 128, 32, 1500
+    slopes = [0.25, 0.0, 2.0 ** -4, 2.0 ** -8]
+    lay, ref, q, _ = fill_both(B, B_, H, d, [80] * H, [80] * H, n, n, 174, G, alibi=slopes, q_scale=3.0)
+    lay.quant_sync()
+    out = lay.decode_quant(q)
+    lay.poll_status()
+    res = ref.decode_quant(to_np(q), 4, G)
+    want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out, want, BF16, "peaked + alibi")
+
+
+def test_decode_quant_merged_weight_flags(B):
+    B_, H, d, G, n = 2, 2, 128, 32, 500
+    lay, ref, q, _ = fill_both(B, B_, H, d, [80, 56], [72, 80], n, n, 175, G)
+    lay.quant_sync()
+    low = lay.decode_quant(q, out_lowrank=True)
+    res = ref.decode_quant(to_np(q), 4, G, lowrank_out=True)
+    for b in range(B_):
+        for h in range(H):
+            r = res[(b, h)].shape[0]
+            assert_close(low[b, 0, lay.offs_v[h]:lay.offs_v[h] + r], res[(b, h)], BF16, "lowrank out")
+    # rank-space query: q U^K rounded to bf16 on the host; the oracle gets the same rounded q' lifted back
+    qn = to_np(q)
+    qp = torch.zeros((B_, 1, lay.offs_k[-1]), dtype=BF16)
+    q_back = np.zeros_like(qn)
+    for h in range(H):
+        U = ref.U_K[h]
+        y = torch.from_numpy(qn[:, 0, h, :] @ U).to(BF16)
+        qp[:, 0, lay.offs_k[h]:lay.offs_k[h] + U.shape[1]] = y
+        q_back[:, 0, h, :] = y.double().numpy() @ U.T          # U^T U = I: projecting this gives y again
+    out = lay.decode_quant(qp.cuda(), q_preprojected=True)
+    res2 = ref.decode_quant(q_back, 4, G)
+    want = np.stack([np.stack([res2[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out, want, BF16, "preprojected q")
+
+
+def test_quant_argument_checks(B):
+    U_k, U_v, q, k, v = make_case(1, 1, 64, [32], [32], 64, BF16, seed_cfg=176)
+    lay = B.EigenAttnLayer(1, 1, 64, 64, BF16, U_k, U_v)
+    with pytest.raises(B.EigenAttnError):
+        lay.decode_quant(q)                                   # nothing attached
+    with pytest.raises(B.EigenAttnError):
+        lay.quant_bytes(3, 32)                                # only 4-bit codes are built
+    with pytest.raises(B.EigenAttnError):
+        lay.quant_bytes(4, 48)                                # group must be 16, 32, 64 or 128
+    lay.quant_attach(4, 32)
+    with pytest.raises(B.EigenAttnError):
+        lay.decode_quant(q)                                   # empty cache
+    lay32 = B.EigenAttnLayer(1, 1, 64, 64, torch.float32, U_k, U_v)
+    with pytest.raises(B.EigenAttnError):
+        lay32.quant_bytes(4, 32)                              # 16-bit layers only
+    # storage per element of whole blocks: 4 + 16/G bits for keys (Table 8's accounting)
+    _, bb, ks_off, vc_off, _ = lay.quant_layout(0)
+    assert vc_off * 8 / (32 * 32) == 4 + 16 / 32
