@@ -631,6 +631,104 @@ def run_gqa(args, wl):
     }))
 
 
+def run_quant(args, wl):
+    """Decode step over the quantised rank-r cache (4-bit codes, group --quant): append the new token's 16-bit rows,
+    then one pass over the codes.  One JSON line: bytes of codes and scales read per second against the HBM
+    roofline, the 16-bit decode of the same cache beside it, and parity of sampled units against the oracle."""
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    G = args.quant
+    keep = [0, wl.n_heads - 1]
+    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep)
+    lay.quant_attach(4, G)
+    lay.quant_sync()
+    n0 = wl.context
+    nq = n0 // G * G
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream(device)
+    steps, warmup = min(args.steps, 100), max(3, min(args.warmup, 10))
+
+    def step():
+        lay.set_len(n0)
+        lay.append_kv(k_new, v_new)
+        lay.decode_quant(q, out=out)
+
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, c in ev:
+        a.record(stream); c.record(stream)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(device.index or 0)
+    sampler.start(); time.sleep(0.2)
+    l0 = lay.launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        lay.set_decode_events(ev[i][0], ev[i][1])
+        step()
+    t1.record(stream)
+    torch.cuda.synchronize(device)
+    lay.set_decode_events(None, None)
+    clocks = sampler.stop()
+    launches = lay.launch_count() - l0
+    lay.poll_status()
+    ms = t0.elapsed_time(t1) / steps
+    kern = sum(a.elapsed_time(c) for a, c in ev) / steps
+    # bytes one step must read: every block of codes and scales, plus the 16-bit rows not quantised yet
+    block_bytes = [lay.quant_layout(h)[1] for h in range(wl.n_heads)]
+    bytes_codes = wl.batch * (nq // G) * sum(block_bytes)
+    bytes_tail = wl.batch * (n0 + 1 - nq) * 2 * sum(ranks) * 2
+    bytes_step = bytes_codes + bytes_tail
+    bytes_16bit = algorithmic_bytes(wl, ranks, ranks, n0 + 1)
+    peak, peak_src = measured_peaks()
+    # the 16-bit decode of the same cache
+    for _ in range(3):
+        lay.decode(q, out=out)
+    torch.cuda.synchronize(device)
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    for _ in range(20):
+        lay.decode(q, out=out)
+    a1.record(stream)
+    torch.cuda.synchronize(device)
+    ms_16bit = a0.elapsed_time(a1) / 20
+    step()
+    torch.cuda.synchronize(device)
+    # parity of the sampled units: the oracle keeps 16-bit rows (Section 2, p = 16) and quantises those
+    from oracle import eigen_attention as orc
+    dt = synth.torch_dtype(wl.dtype)
+    storage = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dt).double().numpy()
+    ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=[(0, h) for h in keep], storage=storage)
+    for h in keep:
+        ref.append_unit_rows((0, h), hist[h][0], hist[h][1])
+    ref.set_len(n0)
+    ref.append_kv(k_new.double().cpu().numpy(), v_new.double().cpu().numpy())
+    exp = ref.decode_quant(q.double().cpu().numpy(), 4, G)
+    got = out.double().cpu().numpy()
+    errs = [float(np.abs(got[0, 0, h] - exp[(0, h)]).max()) for h in keep]
+    achieved = bytes_step / (kern * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "rank-r decode over the 4-bit cache, bytes of codes and scales read per second",
+        "value": bytes_step / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms, "us_per_step": ms * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "4-bit codes + f16 scales, f32 arithmetic", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head,
+                   "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "bits": 4, "group": G,
+                   "quantised_rows": nq, "cache_gb": bytes_step / 1e9, "cache_gb_16bit": bytes_16bit / 1e9,
+                   "l2": "inputs larger than L2: every step streams all codes"},
+        "roofline": {"bound": "hbm", "kernel": "decode_quant_kernel (+ combine)", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "kernel_us": kern * 1e3,
+                     "algorithmic_bytes": bytes_step, "traffic": None},
+        "decode_16bit_us": ms_16bit * 1e3, "speedup_over_16bit": ms_16bit / (kern if kern > 0 else ms),
+        "gpu_launches": launches, "clocks": clocks,
+        "parity_sampled_units": {"units": len(errs), "max_abs": max(errs), "tolerance": "max_abs <= 2e-2"},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -641,6 +739,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--alibi", action="store_true", help="decode workloads: add the per-head ALiBi position bias")
     ap.add_argument("--rope", action="store_true", help="decode workloads: the RoPE variant (full-rank query, lifted rotated keys)")
+    ap.add_argument("--quant", type=int, default=0, metavar="G",
+                    help="decode workloads: attend over the 4-bit quantised cache with group size G (16, 32, 64, 128)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
@@ -663,6 +763,8 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     if args.workload in synth.GQA_GROUP:
         return run_gqa(args, wl)
+    if args.quant:
+        return run_quant(args, wl)
     if wl.name.startswith("prefill"):
         run_prefill(args, wl)
     else:

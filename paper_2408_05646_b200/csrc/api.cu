@@ -1016,7 +1016,12 @@ ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t strid
   p.splits = static_cast<int32_t>(splits);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  const cudaError_t e = ea::launch_decode_quant(p, max_rp, smem, s, &h->launches);
+  int min_rp = max_rp;
+  for (const HeadInfo& hi : L.heads) {
+    if (hi.rp_k < min_rp) min_rp = hi.rp_k;
+    if (hi.rp_v < min_rp) min_rp = hi.rp_v;
+  }
+  const cudaError_t e = ea::launch_decode_quant(p, max_rp, min_rp, smem, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_quant launch");
   return EA_OK;

@@ -206,6 +206,7 @@ struct QuantParams {
   int32_t b0, b1;           // quantiser: blocks [b0, b1) of every sequence
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
+  uint32_t magic[5];        // float exponent patterns the decode kernel ORs nibbles into (set by its launcher)
 };
 
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.
@@ -227,7 +228,8 @@ cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v
 
 cudaError_t launch_quantize_blocks(const QuantParams& p, cudaStream_t s, uint64_t* launches);
 size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v);
-cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, int min_rp, size_t smem, cudaStream_t s,
+                                uint64_t* launches);   // min_rp: narrowest padded rank over heads and K/V
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
 // library's own partials array on the current device.  Resolves the address on first use per device.

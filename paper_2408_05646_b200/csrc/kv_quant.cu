@@ -110,41 +110,52 @@ constexpr int kQsOffset = 2048;                     // per warp: q'_c * s_c of (
 constexpr int kRingOffset = kQsOffset + 4 * 2 * 128 * 4;
 static_assert(sizeof(QuantSmemHeader) <= kQsOffset, "header overlaps the scaled-query area");
 
+// Two 32-bit patterns as one 64-bit register pair (low word first).  Written as integer arithmetic so that the
+// compiler assigns the halves in place; a move instruction per half would double the cost of a cached element.
+__device__ __forceinline__ unsigned long long pair_of(uint32_t lo, uint32_t hi) {
+  return static_cast<unsigned long long>(lo) | (static_cast<unsigned long long>(hi) << 32);
+}
+__device__ __forceinline__ unsigned long long pair_of(float lo, float hi) {
+  return pair_of(__float_as_uint(lo), __float_as_uint(hi));
+}
+__device__ __forceinline__ float low_plus_high(unsigned long long v) {
+  return __uint_as_float(static_cast<uint32_t>(v)) + __uint_as_float(static_cast<uint32_t>(v >> 32));
+}
+
 // Eight codes of a word as four packed float pairs (exact small integers in -7..7; a nibble 0 gives -8).
 struct Consts {
   unsigned long long c01, c23, c45, c67;
+  uint32_t e23, e19, e15, e11, e7;     // exponent patterns of 2^23, 2^19, 2^15, 2^11, 2^7
 };
-__device__ __forceinline__ Consts make_consts() {
+// The exponent patterns come in as kernel arguments, not as literals: (w & mask) | pattern is one logic
+// instruction when the pattern sits in a register; with two literals the compiler emits a second logic
+// instruction and a move per element (counted on the device: 327 logic + 160 moves per row instead of 160).
+__device__ __forceinline__ Consts make_consts(const QuantParams& p) {
   Consts c;
-  c.c01 = pack2(-8388616.f, -524296.f);             // -(2^23 + 8), -(2^19 + 8)
-  c.c23 = pack2(-32776.f, -2056.f);                 // -(2^15 + 8), -(2^11 + 8)
-  c.c45 = pack2(-136.f, -32776.f);                  // -(2^7 + 8), then nibbles 5..7 after a shift by 12
-  c.c67 = pack2(-2056.f, -136.f);
+  c.e23 = p.magic[0]; c.e19 = p.magic[1]; c.e15 = p.magic[2]; c.e11 = p.magic[3]; c.e7 = p.magic[4];
+  c.c01 = pair_of(-8388616.f, -524296.f);            // -(2^23 + 8), -(2^19 + 8)
+  c.c23 = pair_of(-32776.f, -2056.f);               // -(2^15 + 8), -(2^11 + 8)
+  c.c45 = pair_of(-136.f, -32776.f);                // -(2^7 + 8), then nibbles 5..7 after a shift by 12
+  c.c67 = pair_of(-2056.f, -136.f);
   return c;
 }
 __device__ __forceinline__ void codes_to_floats(uint32_t w, const Consts& k, unsigned long long (&f)[4]) {
   const uint32_t u = w >> 12;
-  const float x0 = __uint_as_float((w & 0x0000000Fu) | 0x4B000000u);
-  const float x1 = __uint_as_float((w & 0x000000F0u) | 0x49000000u);
-  const float x2 = __uint_as_float((w & 0x00000F00u) | 0x47000000u);
-  const float x3 = __uint_as_float((w & 0x0000F000u) | 0x45000000u);
-  const float x4 = __uint_as_float((w & 0x000F0000u) | 0x43000000u);
-  const float x5 = __uint_as_float((u & 0x00000F00u) | 0x47000000u);
-  const float x6 = __uint_as_float((u & 0x0000F000u) | 0x45000000u);
-  const float x7 = __uint_as_float((u & 0x000F0000u) | 0x43000000u);
-  f[0] = add2p(pack2(x0, x1), k.c01);
-  f[1] = add2p(pack2(x2, x3), k.c23);
-  f[2] = add2p(pack2(x4, x5), k.c45);
-  f[3] = add2p(pack2(x6, x7), k.c67);
+  f[0] = add2p(pair_of((w & 0x0000000Fu) | k.e23, (w & 0x000000F0u) | k.e19), k.c01);
+  f[1] = add2p(pair_of((w & 0x00000F00u) | k.e15, (w & 0x0000F000u) | k.e11), k.c23);
+  f[2] = add2p(pair_of((w & 0x000F0000u) | k.e7, (u & 0x00000F00u) | k.e15), k.c45);
+  f[3] = add2p(pair_of((u & 0x0000F000u) | k.e11, (u & 0x000F0000u) | k.e7), k.c67);
 }
 __device__ __forceinline__ void bf16x8_to_floats(const uint4& x, unsigned long long (&f)[4]) {
-  f[0] = pack2(__uint_as_float(x.x << 16), __uint_as_float(x.x & 0xffff0000u));
-  f[1] = pack2(__uint_as_float(x.y << 16), __uint_as_float(x.y & 0xffff0000u));
-  f[2] = pack2(__uint_as_float(x.z << 16), __uint_as_float(x.z & 0xffff0000u));
-  f[3] = pack2(__uint_as_float(x.w << 16), __uint_as_float(x.w & 0xffff0000u));
+  f[0] = pair_of(x.x << 16, x.x & 0xffff0000u);
+  f[1] = pair_of(x.y << 16, x.y & 0xffff0000u);
+  f[2] = pair_of(x.z << 16, x.z & 0xffff0000u);
+  f[3] = pair_of(x.w << 16, x.w & 0xffff0000u);
 }
 
-template <int NW, int MINB>   // NW: 8-channel words a row can have (widest padded rank / 8)
+// NW: 8-channel words a row can have (widest padded rank / 8); G: group size (row offsets inside a block become
+// immediates); FULL: every head has exactly NW words of keys and of values (no per-word guards).
+template <int NW, int MINB, int G, bool FULL>
 __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const QuantParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   QuantSmemHeader* hdr = reinterpret_cast<QuantSmemHeader*>(smem);
@@ -155,9 +166,8 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   const int h = unit / p.B, b = unit - h * p.B;
   const HeadInfo hd = p.heads[h];
   const QuantHead qh = p.qheads[h];
-  const int G = p.group;
-  const int gshift = 31 - __clz(G);
-  const int bps = kStageRows >> gshift;                       // blocks per stage
+  constexpr int gshift = G == 16 ? 4 : G == 32 ? 5 : G == 64 ? 6 : 7;
+  constexpr int bps = kStageRows >> gshift;                      // blocks per stage
   const int nqb = p.nq >> gshift;                             // blocks held as codes
   const int nwk = hd.rp_k >> 3, nwv = hd.rp_v >> 3;
   const int stage_stride = (bps * qh.block_bytes + 127) & ~127;
@@ -199,7 +209,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   }
   __syncthreads();
 
-  const Consts kc = make_consts();
+  const Consts kc = make_consts(p);
   unsigned long long o[NW * 4];
 #pragma unroll
   for (int i = 0; i < NW * 4; ++i) o[i] = 0ull;
@@ -207,10 +217,12 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   const float slope2 = hd.alibi_slope2;
   const int pos_q = p.n - 1;
   // online softmax of one score: returns the weight of the row under the (possibly raised) running maximum
+  // (the maximum is only raised when a score exceeds it by more than 8: weights stay below 2^8, and a warp
+  // leaves the common path only when one of its lanes meets such a score)
   auto weight = [&](float s) {
-    if (s > m) {
+    if (s > m + 8.f) {
       const float c = ex2(m - s);
-      const unsigned long long cc = pack2(c, c);
+      const unsigned long long cc = pair_of(c, c);
       l *= c;
 #pragma unroll
       for (int i = 0; i < NW * 4; ++i) o[i] = mul2p(o[i], cc);
@@ -244,7 +256,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
       unsigned long long a0 = 0ull, a1 = 0ull, a2 = 0ull, a3 = 0ull;
 #pragma unroll
       for (int j = 0; j < NW; ++j)
-        if (j < nwk) {
+        if (FULL || j < nwk) {
           unsigned long long f[4];
           codes_to_floats(kw[j * G], kc, f);
           const ulonglong2 q0 = *reinterpret_cast<const ulonglong2*>(qsr + 8 * j);
@@ -252,17 +264,16 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
           a0 = fma2p(f[0], q0.x, a0); a1 = fma2p(f[1], q0.y, a1);
           a2 = fma2p(f[2], q1.x, a2); a3 = fma2p(f[3], q1.y, a3);
         }
-      float s0, s1;
-      unpack2(add2p(add2p(a0, a1), add2p(a2, a3)), s0, s1);
       const int j_abs = s * kStageRows + tid;
-      const float pr = weight(fmaf(slope2, static_cast<float>(j_abs - pos_q), s0 + s1));
+      const float pr = weight(fmaf(slope2, static_cast<float>(j_abs - pos_q),
+                                   low_plus_high(add2p(add2p(a0, a1), add2p(a2, a3)))));
       const uint32_t* vw = reinterpret_cast<const uint32_t*>(bb + qh.vc_off) + ri;
       const __half* vs = reinterpret_cast<const __half*>(bb + qh.vs_off) + ri;
 #pragma unroll
       for (int j = 0; j < NW; ++j)
-        if (j < nwv) {
+        if (FULL || j < nwv) {
           const float sv = pr * __half2float(vs[((8 * j) >> gshift) * G]);
-          const unsigned long long svp = pack2(sv, sv);
+          const unsigned long long svp = pair_of(sv, sv);
           unsigned long long f[4];
           codes_to_floats(vw[j * G], kc, f);
 #pragma unroll
@@ -284,7 +295,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
       unsigned long long a0 = 0ull, a1 = 0ull, a2 = 0ull, a3 = 0ull;
 #pragma unroll
       for (int c = 0; c < NW; ++c)
-        if (c < nwk) {
+        if (FULL || c < nwk) {
           unsigned long long f[4];
           bf16x8_to_floats(__ldg(kr + c), f);
           const ulonglong2 q0 = *reinterpret_cast<const ulonglong2*>(hdr->qp + 8 * c);
@@ -292,13 +303,12 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
           a0 = fma2p(f[0], q0.x, a0); a1 = fma2p(f[1], q0.y, a1);
           a2 = fma2p(f[2], q1.x, a2); a3 = fma2p(f[3], q1.y, a3);
         }
-      float s0, s1;
-      unpack2(add2p(add2p(a0, a1), add2p(a2, a3)), s0, s1);
-      const float pr = weight(fmaf(slope2, static_cast<float>(j - pos_q), s0 + s1));
-      const unsigned long long prp = pack2(pr, pr);
+      const float pr = weight(fmaf(slope2, static_cast<float>(j - pos_q),
+                                   low_plus_high(add2p(add2p(a0, a1), add2p(a2, a3)))));
+      const unsigned long long prp = pair_of(pr, pr);
 #pragma unroll
       for (int c = 0; c < NW; ++c)
-        if (c < nwv) {
+        if (FULL || c < nwv) {
           unsigned long long f[4];
           bf16x8_to_floats(__ldg(vr + c), f);
 #pragma unroll
@@ -325,10 +335,8 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
 #pragma unroll
     for (int i = 0; i < NW * 4; ++i)
       if (2 * i < hd.rp_v) {
-        float x0, x1;
-        unpack2(o[i], x0, x1);
-        red[tid * rstride + 2 * i] = x0 * f;
-        red[tid * rstride + 2 * i + 1] = x1 * f;
+        red[tid * rstride + 2 * i] = __uint_as_float(static_cast<uint32_t>(o[i])) * f;
+        red[tid * rstride + 2 * i + 1] = __uint_as_float(static_cast<uint32_t>(o[i] >> 32)) * f;
       }
   }
   __syncthreads();
@@ -376,17 +384,30 @@ __global__ void __launch_bounds__(128) quant_combine_kernel(const QuantParams p)
   }
 }
 
-template <int NW, int MINB>
+template <int NW, int MINB, int G, bool FULL>
 cudaError_t launch_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
   static size_t configured = 0;
   if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_quant_kernel<NW, MINB>,
+    const cudaError_t e = cudaFuncSetAttribute(decode_quant_kernel<NW, MINB, G, FULL>,
                                                cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  decode_quant_kernel<NW, MINB><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
+  decode_quant_kernel<NW, MINB, G, FULL><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
   return cudaGetLastError();
+}
+template <int NW, int MINB, int G>
+cudaError_t launch_full_or_not(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
+  return full ? launch_variant<NW, MINB, G, true>(p, smem, s) : launch_variant<NW, MINB, G, false>(p, smem, s);
+}
+template <int NW, int MINB>
+cudaError_t launch_group(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
+  switch (p.group) {
+    case 16: return launch_full_or_not<NW, MINB, 16>(p, full, smem, s);
+    case 32: return launch_full_or_not<NW, MINB, 32>(p, full, smem, s);
+    case 64: return launch_full_or_not<NW, MINB, 64>(p, full, smem, s);
+    default: return launch_full_or_not<NW, MINB, 128>(p, full, smem, s);
+  }
 }
 
 }  // namespace
@@ -404,11 +425,15 @@ size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v) {
   return kRingOffset + (ring > red ? ring : red);
 }
 
-cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches) {
+cudaError_t launch_decode_quant(const QuantParams& p0, int max_rp, int min_rp, size_t smem, cudaStream_t s,
+                                uint64_t* launches) {
+  QuantParams p = p0;
+  p.magic[0] = 0x4B000000u; p.magic[1] = 0x49000000u; p.magic[2] = 0x47000000u; p.magic[3] = 0x45000000u;
+  p.magic[4] = 0x43000000u;
   cudaError_t e;
-  if (max_rp <= 64) e = launch_variant<8, 3>(p, smem, s);
-  else if (max_rp <= 80) e = launch_variant<10, 3>(p, smem, s);
-  else e = launch_variant<16, 2>(p, smem, s);
+  if (max_rp <= 64) e = launch_group<8, 3>(p, min_rp == 64, smem, s);
+  else if (max_rp <= 80) e = launch_group<10, 3>(p, min_rp == 80, smem, s);
+  else e = launch_group<16, 2>(p, min_rp == 128, smem, s);
   if (e != cudaSuccess) return e;
   ++*launches;
   quant_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
