@@ -20,6 +20,7 @@
 // Every wait is bounded.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <stddef.h>
 
 #include "internal.h"
 #include "tc_common.cuh"
@@ -102,10 +103,13 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
 
 struct __align__(16) QuantSmemHeader {
   unsigned long long full[kQStages];
+  int done[kQStages];      // running count of warps that have finished with a stage in the slot (4 per stage)
+  int abort_flag;
   float wmax[4], wsum[4];
-  float qraw[128];         // the unit's query as fp32
-  float qp[128];           // q' * log2(e)/sqrt(d_head)
+  __align__(16) float qraw[128];   // the unit's query as fp32
+  __align__(16) float qp[128];     // q' * log2(e)/sqrt(d_head); read 16 bytes at a time
 };
+static_assert(offsetof(QuantSmemHeader, qp) % 16 == 0, "q' is read with 16-byte loads");
 constexpr int kQsOffset = 2048;                     // per warp: q'_c * s_c of (up to) two blocks, [2][128] floats
 constexpr int kRingOffset = kQsOffset + 4 * 2 * 128 * 4;
 static_assert(sizeof(QuantSmemHeader) <= kQsOffset, "header overlaps the scaled-query area");
@@ -177,12 +181,16 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   const char* slab = p.qcache + qh.slab_off + static_cast<int64_t>(b) * p.blocks_max * qh.block_bytes;
 
   if (tid == 0) {
-    for (int s = 0; s < kQStages; ++s) mbar_init(&hdr->full[s], 1);
+    for (int s = 0; s < kQStages; ++s) {
+      mbar_init(&hdr->full[s], 1);
+      hdr->done[s] = 0;
+    }
+    hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   const uint64_t policy = policy_evict_first();
-  auto issue = [&](int s, int slot) {                         // thread 0
+  auto issue = [&](int s, int slot) {                         // one thread
     const int nblk = min(bps, nqb - s * bps);
     const uint32_t bytes = static_cast<uint32_t>(nblk) * qh.block_bytes;
     mbar_arrive_expect_tx(&hdr->full[slot], bytes);
@@ -201,10 +209,13 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
     __syncthreads();
     if (tid < hd.rp_k) {
       const float* U = p.basis + hd.uk_off + tid;
-      float acc = 0.f;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};       // d_head is a multiple of 8; four chains keep 32 loads in flight
 #pragma unroll 8
-      for (int d = 0; d < p.d_head; ++d) acc = fmaf(hdr->qraw[d], __ldg(U + d * hd.rp_k), acc);
-      hdr->qp[tid] = acc * p.q_scale;
+      for (int d = 0; d < p.d_head; d += 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] = fmaf(hdr->qraw[d + i], __ldg(U + (d + i) * hd.rp_k), acc[i]);
+      }
+      hdr->qp[tid] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) * p.q_scale;
     }
   }
   __syncthreads();
@@ -233,10 +244,14 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
     return pr;
   };
 
-  bool aborted = false;
+  // The four warps walk the stages independently (no CTA-wide barrier per stage): a warp waits for the slot's
+  // copy, works on its 32 rows and counts itself off; the warp that counts off last refills the slot.
   for (int s = s_lo; s < s_hi; ++s) {
     const int it = s - s_lo, slot = it % kQStages;
-    const bool ok = mbar_wait(&hdr->full[slot], (it / kQStages) & 1, p.status);
+    if (__any_sync(0xffffffffu, !mbar_wait(&hdr->full[slot], (it / kQStages) & 1, p.status))) {
+      hdr->abort_flag = 1;         // a wait gave up: the status word is set, the other warps' waits end early
+      break;
+    }
     const unsigned char* st = ring + slot * stage_stride;
     const int nblk = min(bps, nqb - s * bps);
     {   // the warp's blocks: q'_c * s_c
@@ -280,11 +295,15 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
           for (int i = 0; i < 4; ++i) o[4 * j + i] = fma2p(f[i], svp, o[4 * j + i]);
         }
     }
-    // everyone is done with the slot (and with this warp's scaled query); a failed wait ends the loop for all
-    const int all_ok = __syncthreads_and(ok ? 1 : 0);
-    if (tid == 0 && all_ok && s + kQStages < s_hi) issue(s + kQStages, slot);
-    if (!all_ok) { aborted = true; break; }
+    // this warp is done with the slot (and with its scaled query)
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence_block();       // the warp's reads of the slot come before the count that may trigger the refill
+      if ((atomicAdd(&hdr->done[slot], 1) & 3) == 3 && s + kQStages < s_hi) issue(s + kQStages, slot);
+    }
   }
+  __syncthreads();
+  const bool aborted = *reinterpret_cast<volatile int*>(&hdr->abort_flag) != 0;
 
   // rows that are not quantised yet, straight from the 16-bit cache (the last split takes them)
   if (split == p.splits - 1 && !aborted) {
