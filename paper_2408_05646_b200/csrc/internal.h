@@ -206,7 +206,7 @@ struct QuantParams {
   int32_t b0, b1;           // quantiser: blocks [b0, b1) of every sequence
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
-  uint32_t magic[5];        // float exponent patterns the decode kernel ORs nibbles into (set by its launcher)
+  uint32_t magic[4];        // float exponent patterns the decode kernel ORs nibbles into (set by its launcher)
 };
 
 // Launchers (each returns the CUDA error of its launch); `launches` is incremented per kernel.

@@ -127,28 +127,28 @@ __device__ __forceinline__ float low_plus_high(unsigned long long v) {
 }
 
 // Eight codes of a word as four packed float pairs (exact small integers in -7..7; a nibble 0 gives -8).
+// Nibbles 0..3 sit at bits 0, 4, 8, 12 and meet the exponents of 2^23, 2^19, 2^15, 2^11; nibbles 4..7 do the
+// same after a shift by 16, so two packed constants serve the whole word.
 struct Consts {
-  unsigned long long c01, c23, c45, c67;
-  uint32_t e23, e19, e15, e11, e7;     // exponent patterns of 2^23, 2^19, 2^15, 2^11, 2^7
+  unsigned long long c01, c23;
+  uint32_t e23, e19, e15, e11;         // exponent patterns of 2^23, 2^19, 2^15, 2^11
 };
 // The exponent patterns come in as kernel arguments, not as literals: (w & mask) | pattern is one logic
 // instruction when the pattern sits in a register; with two literals the compiler emits a second logic
 // instruction and a move per element (counted on the device: 327 logic + 160 moves per row instead of 160).
 __device__ __forceinline__ Consts make_consts(const QuantParams& p) {
   Consts c;
-  c.e23 = p.magic[0]; c.e19 = p.magic[1]; c.e15 = p.magic[2]; c.e11 = p.magic[3]; c.e7 = p.magic[4];
-  c.c01 = pair_of(-8388616.f, -524296.f);            // -(2^23 + 8), -(2^19 + 8)
-  c.c23 = pair_of(-32776.f, -2056.f);               // -(2^15 + 8), -(2^11 + 8)
-  c.c45 = pair_of(-136.f, -32776.f);                // -(2^7 + 8), then nibbles 5..7 after a shift by 12
-  c.c67 = pair_of(-2056.f, -136.f);
+  c.e23 = p.magic[0]; c.e19 = p.magic[1]; c.e15 = p.magic[2]; c.e11 = p.magic[3];
+  c.c01 = pair_of(-8388616.f, -524296.f);          // -(2^23 + 8), -(2^19 + 8)
+  c.c23 = pair_of(-32776.f, -2056.f);              // -(2^15 + 8), -(2^11 + 8)
   return c;
 }
 __device__ __forceinline__ void codes_to_floats(uint32_t w, const Consts& k, unsigned long long (&f)[4]) {
-  const uint32_t u = w >> 12;
-  f[0] = add2p(pair_of((w & 0x0000000Fu) | k.e23, (w & 0x000000F0u) | k.e19), k.c01);
-  f[1] = add2p(pair_of((w & 0x00000F00u) | k.e15, (w & 0x0000F000u) | k.e11), k.c23);
-  f[2] = add2p(pair_of((w & 0x000F0000u) | k.e7, (u & 0x00000F00u) | k.e15), k.c45);
-  f[3] = add2p(pair_of((u & 0x0000F000u) | k.e11, (u & 0x000F0000u) | k.e7), k.c67);
+  const uint32_t u = w >> 16;
+  f[0] = add2p(pair_of((w & 0x000Fu) | k.e23, (w & 0x00F0u) | k.e19), k.c01);
+  f[1] = add2p(pair_of((w & 0x0F00u) | k.e15, (w & 0xF000u) | k.e11), k.c23);
+  f[2] = add2p(pair_of((u & 0x000Fu) | k.e23, (u & 0x00F0u) | k.e19), k.c01);
+  f[3] = add2p(pair_of((u & 0x0F00u) | k.e15, (u & 0xF000u) | k.e11), k.c23);
 }
 __device__ __forceinline__ void bf16x8_to_floats(const uint4& x, unsigned long long (&f)[4]) {
   f[0] = pair_of(x.x << 16, x.x & 0xffff0000u);
@@ -448,7 +448,6 @@ cudaError_t launch_decode_quant(const QuantParams& p0, int max_rp, int min_rp, s
                                 uint64_t* launches) {
   QuantParams p = p0;
   p.magic[0] = 0x4B000000u; p.magic[1] = 0x49000000u; p.magic[2] = 0x47000000u; p.magic[3] = 0x45000000u;
-  p.magic[4] = 0x43000000u;
   cudaError_t e;
   if (max_rp <= 64) e = launch_group<8, 3>(p, min_rp == 64, smem, s);
   else if (max_rp <= 80) e = launch_group<10, 3>(p, min_rp == 80, smem, s);
