@@ -237,8 +237,12 @@ typedef enum {
   EA_OPT_PREFILL_IMPL = 4,    /* 0 = automatic, 1 = CUDA-core kernel, 2 = tcgen05 tensor-core kernels, 3 = the
                                  single-tile tcgen05 kernel (otherwise only used for ranks too wide for the
                                  warp-specialised one)                                                     */
-  EA_OPT_DECODE_FUSED = 5     /* 1 (default): a decode step is one launch (append row, attend, merge the
+  EA_OPT_DECODE_FUSED = 5,    /* 1 (default): a decode step is one launch (append row, attend, merge the
                                  splits, lift); 0: separate append / attention / merge launches           */
+  EA_OPT_PREFILL_PROJECT = 6  /* tensor-core projections of prefill: 0 = automatic (the persistent kernel that
+                                 streams token tiles by TMA when d_head % 64 == 0 and T >= 128), 1 = always
+                                 one CTA per tile of 128 tokens, n >= 2 = the persistent kernel with at most
+                                 n CTAs                                                                    */
 } ea_option;
 ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value);
 

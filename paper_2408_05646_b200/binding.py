@@ -23,6 +23,7 @@ EA_CHECK_ORTHONORMAL = 0x1
 EA_Q_PREPROJECTED, EA_OUT_LOWRANK, EA_KV_PREPROJECTED = 0x1, 0x2, 0x4
 EA_OPT_DECODE_CTAS, EA_OPT_DECODE_TILE_ROWS, EA_OPT_DECODE_STAGES, EA_OPT_PREFILL_IMPL = 1, 2, 3, 4
 EA_OPT_DECODE_FUSED = 5
+EA_OPT_PREFILL_PROJECT = 6
 
 STATUS_NAMES = {0: "EA_OK", -1: "EA_ERR_INVALID_ARG", -2: "EA_ERR_SHAPE", -3: "EA_ERR_CAPACITY",
                 -4: "EA_ERR_UNSUPPORTED", -5: "EA_ERR_CUDA", -6: "EA_ERR_TIMEOUT",

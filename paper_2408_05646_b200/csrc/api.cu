@@ -151,6 +151,35 @@ bool encode_tensor_maps(const ea_desc* d, const Layout& L, char* cache, std::vec
   return true;
 }
 
+// Tensor maps of the q, k, v tensors of one prefill call for the streaming projection kernel: a 3-D view
+// {n_heads * d_head (inner), T tokens, batch} of bf16, box = 64 elements x 128 tokens with the 128-byte
+// swizzle; tokens past T read as zero.  Encoded on the host per call (the pointers are the caller's).
+bool encode_input_maps(const void* const ptrs[3], int H, int d_head, int T, int B, int64_t stride_b, int64_t stride_t,
+                       CUtensorMap maps[3]) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return false;
+    encode = reinterpret_cast<EncodeFn>(fn);
+  }
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(H) * d_head, static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(B)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(stride_t) * 2, static_cast<cuuint64_t>(stride_b) * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  for (int i = 0; i < 3; ++i)
+    if (encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptrs[i]), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  return true;
+}
+
 }  // namespace
 
 struct eigen_attn {
@@ -164,7 +193,7 @@ struct eigen_attn {
   bool alibi = false;     // some head has a non-zero ALiBi slope
   bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
   int rope_interleaved = 0;
-  int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1;
+  int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1, opt_project = 0;
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   // quantised copy of the cache (Section 5.3), attached by the caller
@@ -685,7 +714,24 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     pp.cache = h->cache; pp.qp = h->ws + L.off_qp; pp.stride_b = stride_b; pp.stride_t = stride_t;
     pp.B = h->desc.batch; pp.T = T; pp.H = h->desc.n_heads; pp.d_head = h->desc.d_head;
     pp.n_max = h->desc.n_max; pp.row0 = len0; pp.status = dev_status(h);
-    e = ea::launch_project_tc(pp, L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v, s, &h->launches);
+    const int max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
+    // Whole tiles of 64-element atoms and at least one full tile of tokens: the persistent kernel that streams
+    // the token tiles by TMA and keeps the basis images in shared memory; otherwise one CTA per tile.
+    CUtensorMap in_maps[3];
+    const void* const in_ptrs[3] = {d_q, d_k, d_v};
+    int ps_stages = 0;
+    bool stream = h->opt_project != 1 && h->desc.d_head % 64 == 0 && T >= 128 && stride_t > 0 && stride_b > 0 &&
+                  stride_t >= static_cast<int64_t>(h->desc.n_heads) * h->desc.d_head;
+    if (stream) {
+      ea::project_tc_stream_smem(max_rp, h->desc.d_head, &ps_stages);
+      stream = ps_stages >= 2 && encode_input_maps(in_ptrs, h->desc.n_heads, h->desc.d_head, T, h->desc.batch,
+                                                   stride_b, stride_t, in_maps);
+    }
+    if (stream)
+      e = ea::launch_project_tc_stream(pp, in_maps, max_rp, h->opt_project >= 2 ? static_cast<int>(h->opt_project) : h->sm_count,
+                                       s, &h->launches);
+    else
+      e = ea::launch_project_tc(pp, max_rp, s, &h->launches);
     if (e != cudaSuccess) return cuda_fail(h, e, "prefill projection launch");
     h->len += T;
   } else {
@@ -1053,6 +1099,10 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
     case EA_OPT_DECODE_FUSED:
       if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "DECODE_FUSED %lld", static_cast<long long>(value));
       h->opt_fused = value;
+      return EA_OK;
+    case EA_OPT_PREFILL_PROJECT:
+      if (value < 0 || value > 65535) return fail(h, EA_ERR_INVALID_ARG, "PREFILL_PROJECT %lld", static_cast<long long>(value));
+      h->opt_project = value;
       return EA_OK;
     default:
       return fail(h, EA_ERR_INVALID_ARG, "unknown option %d", option);

@@ -407,3 +407,32 @@ def test_prefill_with_peaked_attention(B, impl):
     c = lay.prefill(q[:, 300:], k[:, 300:], v[:, 300:])
     lay.poll_status()
     assert_close(torch.cat([a, c], dim=1), expect, BF16, f"peaked prefill impl {impl}")
+
+
+@pytest.mark.parametrize("H,d,rk,rv,cuts", [
+    (3, 128, [80, 48, 128], [80, 112, 8], [0, 128]),             # exactly one tile
+    (2, 128, [80, 64], [64, 96], [0, 333, 1000]),                # ragged tiles, second chunk starts mid-cache
+    (5, 64, [24, 64, 40, 8, 56], [56, 8, 64, 32, 16], [0, 700]), # one atom per row, more (head, tensor) pairs than a CTA keeps
+])
+def test_streaming_projection_equals_per_tile_projection(B, H, d, rk, rv, cuts):
+    """Prefill's projections run either as a persistent kernel (token tiles by TMA, basis resident) or with
+    one CTA per tile: the same products in the same order, so the cache rows and the outputs are bit-identical.
+    Inputs are slices of a wider tensor (token stride larger than H * d_head) and of a longer one."""
+    B_, T = 3, cuts[-1]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + 5, BF16, seed_cfg=103, T_q=T + 5)
+    wide = lambda x: torch.cat([x, torch.zeros_like(x)], dim=2)[:, :T, :H]      # views with padded strides
+    q, k, v = wide(q), wide(k), wide(v)
+    got = {}
+    for mode in (0, 1, 2, 7):                        # 2 and 7 CTAs: every CTA walks through several bases
+        lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
+        lay.set_option(B.EA_OPT_PREFILL_PROJECT, mode)
+        outs = [lay.prefill(q[:, a:b_], k[:, a:b_], v[:, a:b_]) for a, b_ in zip(cuts[:-1], cuts[1:])]
+        lay.poll_status()
+        got[mode] = (torch.cat(outs, dim=1), [lay.cache_rows(h, w).clone() for h in range(H) for w in "kv"])
+    for mode in (0, 2, 7):
+        assert torch.equal(got[mode][0], got[1][0])
+        for a, b_ in zip(got[mode][1], got[1][1]):
+            assert torch.equal(a, b_)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
+    assert_close(got[0][0], expect, BF16, "prefill with streamed projections")
