@@ -214,6 +214,21 @@ ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_off
 ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len);
 ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
 
+/* A batch of unequal lengths (the serving case: the prompts of a batch differ in length; the paper's generation
+ * phase, Section 2 "LLM Inference", is stated per sequence, so each sequence attends its own n cached rows).
+ * lens: HOST array [batch], 0 <= lens[b] <= n_max; sequence b then holds rows [0, lens[b]) of its slabs, whatever
+ * was written there before (a prompt batch padded to a common T and prefilled keeps its first lens[b] rows).
+ * eigen_attn_get_len reports the longest sequence.  Afterwards eigen_attn_append_kv and eigen_attn_decode_step
+ * add rows behind each sequence's own end, eigen_attn_decode / _decode_step / _decode_static attend each
+ * sequence's own rows (ALiBi positions count from the sequence's own end); decode needs lens[b] >= 1 for every
+ * b (EA_ERR_SHAPE otherwise).  The split-KV work decomposition stays that of the longest sequence, so a step
+ * costs about as much as if every sequence had that length.  eigen_attn_set_len returns to equal lengths.
+ * Not available (EA_ERR_UNSUPPORTED) with a rotary embedding or a quantised cache attached; while lengths differ,
+ * prefill, decode_gqa and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
+ * (asynchronous; the array may be reused when the call returns). */
+ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);
+ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens);
+
 /* Synchronises the stream and returns the device status word (EA_OK or EA_ERR_TIMEOUT), then clears it. */
 ea_status eigen_attn_poll_status(eigen_attn_t h, void* cuda_stream);
 

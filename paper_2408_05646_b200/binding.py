@@ -60,6 +60,8 @@ SYMBOLS = {
     "eigen_attn_prefill": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i64, _vp, _i64, _i64, _u32, _vp]),
     "eigen_attn_get_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "eigen_attn_set_len": (_i32, [_vp, _i32]),
+    "eigen_attn_set_lens": (_i32, [_vp, ctypes.POINTER(_i32), _vp]),
+    "eigen_attn_get_lens": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "eigen_attn_poll_status": (_i32, [_vp, _vp]),
     "eigen_attn_last_error": (ctypes.c_char_p, [_vp]),
     "eigen_attn_head_offsets": (_i32, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
@@ -343,6 +345,16 @@ class EigenAttnLayer:
 
     def set_len(self, n: int) -> None:
         self._check(lib.eigen_attn_set_len(self.handle, int(n)), "eigen_attn_set_len")
+
+    def set_lens(self, lens, stream=None) -> None:
+        """Per-sequence lengths of a batch whose sequences differ in length (host integers, one per sequence)."""
+        arr = (ctypes.c_int32 * self.B)(*[int(x) for x in lens])
+        self._check(lib.eigen_attn_set_lens(self.handle, arr, _stream_ptr(stream)), "eigen_attn_set_lens")
+
+    def lens(self):
+        arr = (ctypes.c_int32 * self.B)()
+        self._check(lib.eigen_attn_get_lens(self.handle, arr), "eigen_attn_get_lens")
+        return list(arr)
 
     def poll_status(self, stream=None) -> None:
         self._check(lib.eigen_attn_poll_status(self.handle, _stream_ptr(stream)), "eigen_attn_poll_status")

@@ -43,7 +43,7 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0;
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -116,6 +116,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
   L->off_rope = off;     off = align_up(off + 64 * sizeof(double));   // inverse frequencies of the rotary embedding
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
+  L->off_deficit = off;  off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // unequal lengths
   L->workspace_bytes = off;
 }
 
@@ -187,7 +188,9 @@ struct eigen_attn {
   Layout L;
   char* cache = nullptr;
   char* ws = nullptr;
-  int32_t len = 0;
+  int32_t len = 0;        // cached rows of the longest sequence
+  std::vector<int32_t> deficit;   // [B]: sequence b holds len - deficit[b] rows (eigen_attn_set_lens)
+  int32_t max_deficit = 0;        // > 0: the batch has unequal lengths and the workspace holds `deficit`
   int sm_count = 148;
   bool tmaps_ok = false;  // the workspace holds tensor maps of the cache slabs
   bool alibi = false;     // some head has a non-zero ALiBi slope
@@ -257,6 +260,9 @@ ea_status check_quant_args(eigen_attn_t h, const char* who, int32_t bits, int32_
 const HeadInfo* dev_heads(eigen_attn_t h) { return reinterpret_cast<const HeadInfo*>(h->ws + h->L.off_heads); }
 const float* dev_basis(eigen_attn_t h) { return reinterpret_cast<const float*>(h->ws + h->L.off_basis); }
 int* dev_status(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_status); }
+const int32_t* dev_deficit(eigen_attn_t h) {
+  return h->max_deficit > 0 ? reinterpret_cast<const int32_t*>(h->ws + h->L.off_deficit) : nullptr;
+}
 int* dev_counters(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_counters); }
 
 ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T, int64_t stride_b,
@@ -270,7 +276,7 @@ ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
   p.heads = dev_heads(h); p.basis = dev_basis(h); p.k = d_k; p.v = d_v; p.cache = h->cache;
   p.stride_b = stride_b; p.stride_t = stride_t;
   p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head;
-  p.n_max = h->desc.n_max; p.row0 = h->len; p.flags = flags;
+  p.n_max = h->desc.n_max; p.row0 = h->len; p.deficit = dev_deficit(h); p.flags = flags;
   p.lr_k_width = h->L.sum_rp_k; p.lr_v_width = h->L.sum_rp_v;
   const cudaError_t e = ea::launch_project_append(p, h->desc.dtype, s, &h->launches);
   if (e != cudaSuccess) return cuda_fail(h, e, "append_kv launch");
@@ -295,6 +301,8 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
     return fail(h, EA_ERR_INVALID_ARG, "%s: unknown flag 0x%x", who, flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "%s: the cache is empty", who);
+  if (!k_new && h->len - h->max_deficit < 1)
+    return fail(h, EA_ERR_SHAPE, "%s: a sequence of the batch has no cached row", who);
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
@@ -342,6 +350,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.partials = partials;
   p.counters = h->opt_fused ? dev_counters(h) : nullptr;
   p.status = dev_status(h);
+  p.deficit = dev_deficit(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.tile_rows = tile_rows; p.nt = nt; p.ring_bytes = ring_bytes; p.inflight_bytes = kInFlightBytes;
@@ -381,6 +390,8 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   if (flags & ~EA_OUT_LOWRANK)
     return fail(h, EA_ERR_INVALID_ARG, "decode with rotary embedding: flag 0x%x (the query must be full rank)", flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
+  if (h->max_deficit > 0)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: not available for a batch of unequal lengths");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const size_t smem = ea::decode_rope_smem_bytes(L.max_rp_k, L.max_rp_v, h->desc.d_head);
@@ -684,6 +695,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                              int64_t stride_b, int64_t stride_t, void* d_out, int64_t out_stride_b,
                              int64_t out_stride_t, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available with a rotary embedding");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
   if (flags & ~EA_OUT_LOWRANK) return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
@@ -783,7 +795,44 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
   if (len < 0 || len > h->desc.n_max)
     return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %d]", len, h->desc.n_max);
   h->len = len;
+  h->max_deficit = 0;     // every sequence holds len rows again
   if (h->q_group && h->qlen > len) h->qlen = len / h->q_group * h->q_group;   // rows past len are forgotten
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream) {
+  if (!h || !lens) return EA_ERR_INVALID_ARG;
+  if (h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a quantised cache attached");
+  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a rotary embedding");
+  const int B = h->desc.batch;
+  int32_t longest = 0;
+  for (int b = 0; b < B; ++b) {
+    if (lens[b] < 0 || lens[b] > h->desc.n_max)
+      return fail(h, EA_ERR_CAPACITY, "set_lens: lens[%d] = %d outside [0, %d]", b, lens[b], h->desc.n_max);
+    if (lens[b] > longest) longest = lens[b];
+  }
+  std::vector<int32_t> deficit(B);
+  int32_t widest = 0;
+  for (int b = 0; b < B; ++b) {
+    deficit[b] = longest - lens[b];
+    if (deficit[b] > widest) widest = deficit[b];
+  }
+  if (widest > 0) {
+    // a pageable source is staged by the runtime before the call returns, so the vector may change afterwards
+    const cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_deficit, deficit.data(), sizeof(int32_t) * B,
+                                          cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(h, e, "set_lens: upload");
+  }
+  h->deficit.swap(deficit);
+  h->len = longest;
+  h->max_deficit = widest;
+  return EA_OK;
+}
+
+ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens) {
+  if (!h || !lens) return EA_ERR_INVALID_ARG;
+  for (int b = 0; b < h->desc.batch; ++b)
+    lens[b] = h->len - (h->max_deficit > 0 ? h->deficit[b] : 0);
   return EA_OK;
 }
 
@@ -852,6 +901,7 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
 ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
                                 int64_t stride_b_out, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_gqa: NULL q or out");
   if (group < 1 || group > 16) return fail(h, EA_ERR_SHAPE, "decode_gqa: group %d (1..16)", group);
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
@@ -938,6 +988,7 @@ ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, si
 ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
                                   void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!d_qcache) {             // detach
     h->qcache = nullptr; h->q_group = 0; h->qlen = 0;
     return EA_OK;
@@ -980,6 +1031,7 @@ void fill_quant_params(eigen_attn_t h, ea::QuantParams* p) {
 
 ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "quant_sync: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "quant_sync: no quantised buffer attached");
   const int G = h->q_group;
   const int b0 = h->qlen / G, b1 = h->len / G;
@@ -1020,6 +1072,7 @@ ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_off
 ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                   int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
+  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "decode_quant: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: no quantised buffer attached");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: NULL q or out");
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK)) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: unknown flag 0x%x", flags);

@@ -190,12 +190,18 @@ __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
   return per_head_tiles * h + idx;
 }
 
+// Cached rows of sequence b: p.n for a batch of equal lengths, else p.n minus the sequence's deficit.  The work
+// decomposition stays the one of the longest sequence; a shorter sequence simply has no rows in its last tiles.
+__device__ __forceinline__ int seq_rows(const DecodeParams& p, int b) {
+  return p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;
+}
+
 // ---------------------------------------------------------------- one (CTA, unit) piece
 
 template <typename T, int NCH>
 __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
                                             unsigned char* ring, const HeadInfo& hd, int i0, int i1,
-                                            Ring& ring_state, int warp, int lane, bool with_new_row) {
+                                            Ring& ring_state, int warp, int lane, bool with_new_row, int n_b) {
   constexpr int EPC = Elem<T>::kPerChunk;
   const int pair = lane >> 1, half = lane & 1;
   const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
@@ -233,7 +239,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   // score of one cached row against q', online-softmax update, weighted accumulation of its value row
   // ALiBi: the query sits at position n_total - 1; row j gets slope * (j - (n_total - 1)) <= 0 (log2 domain)
   const float slope2 = hd.alibi_slope2;
-  const int pos_q = p.n - 1 + (p.k_new != nullptr ? 1 : 0);
+  const int pos_q = n_b - 1 + (p.k_new != nullptr ? 1 : 0);
   auto process_row = [&](const unsigned char* kr, const unsigned char* vr, bool valid, int j_abs) {
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -284,7 +290,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     }
     const unsigned char* kt = ring + static_cast<size_t>(stage) * ring_state.stage_bytes;
     const unsigned char* vt = kt + ring_state.v_off;
-    const int rows = min(p.tile_rows, p.n - i * p.tile_rows);
+    const int rows = min(p.tile_rows, n_b - i * p.tile_rows);
     // The loop bound is the same for all lanes of a warp (the shuffle inside needs every lane);
     // lane pairs past the last row recompute the group's first row and drop the result.
     for (int rbase = warp * 16; rbase < rows; rbase += kDecodeConsumerWarps * 16) {
@@ -355,10 +361,11 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
 
 // Projections at the head of a piece (all consumer threads): q' = q U^K * log2(e)/sqrt(d_head) into
 // fx->qp, and, when the piece ends its unit and a new token is supplied, k' = k U^K and v' = v U^V,
-// rounded to the cache dtype, into fx->new_k / fx->new_v and into row p.n of the cache.
+// rounded to the cache dtype, into fx->new_k / fx->new_v and into row n_b (the sequence's length) of the cache.
 template <typename T>
 __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmemFixed* fx,
-                                               const HeadInfo& hd, int h, int b, int t, bool with_new_row) {
+                                               const HeadInfo& hd, int h, int b, int t, bool with_new_row,
+                                               int n_b) {
   constexpr int kThreads = kDecodeConsumerWarps * 32;
   const T* q = static_cast<const T*>(p.q);
   const int d_head = p.d_head;
@@ -386,7 +393,7 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
   const int per = (d_head + groups - 1) / groups;
   T* knew = reinterpret_cast<T*>(fx->new_k);
   T* vnew = reinterpret_cast<T*>(fx->new_v);
-  const int64_t crow = static_cast<int64_t>(b) * p.n_max + p.n;
+  const int64_t crow = static_cast<int64_t>(b) * p.n_max + n_b;
   auto finish = [&](int o, float acc) {
     if (o < nq) {
       fx->qp[o] = acc * p.q_scale;
@@ -532,6 +539,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + (f_hi - F)));
         const int h = unit / p.B, b = unit - h * p.B;
         const HeadInfo hd = p.heads[h];
+        const int n_b = seq_rows(p, b);
+        const int nt_b = (n_b + p.tile_rows - 1) / p.tile_rows;
+        const int i1e = min(i1, nt_b);    // tiles past the sequence's own length hold nothing
         int sb, voff, nst;
         ring_geometry<T>(p, hd, &sb, &voff, &nst);
         if (sb != rg.stage_bytes || nst != rg.stages) {
@@ -552,7 +562,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
         const char* src_v = p.cache + hd.v_off + row0 * rowb_v;
         const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
-        for (int i = i0; i < i1; ++i) {
+        for (int i = i0; i < i1e; ++i) {
           if (*abort_flag) { ok = false; break; }
           const int st = rg.stage;
           const uint32_t bit = 1u << st;
@@ -565,8 +575,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
             rg.empty_bits ^= bit;
           }
           uint32_t bytes_k = tile_k, bytes_v = tile_v;
-          if (i == p.nt - 1) {            // ragged last tile of the unit
-            const uint32_t rows = p.n - i * p.tile_rows;
+          if (i == nt_b - 1) {            // ragged last tile of the unit
+            const uint32_t rows = n_b - i * p.tile_rows;
             bytes_k = rows * rowb_k;
             bytes_v = rows * rowb_v;
           }
@@ -609,19 +619,21 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       }
       const bool whole = i0 == 0 && i1 == p.nt;
       const bool with_new_row = p.k_new != nullptr && i1 == p.nt;
-      project_inputs<T>(p, fx, hd, h, b, tid, with_new_row);
+      const int n_b = seq_rows(p, b);
+      const int i1e = min(i1, (n_b + p.tile_rows - 1) / p.tile_rows);   // as in the producer
+      project_inputs<T>(p, fx, hd, h, b, tid, with_new_row, n_b);
       const int mx = max(hd.rp_k, hd.rp_v);
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
       }
       finish_piece<T>(p, fx, hd, unit, h, b, cta, grid, whole, tid);
       F += i1 - i0;

@@ -44,9 +44,10 @@ struct DecodeParams {
   float* partials;          // [(B*H + grid)][part_stride]: m, l, pad, pad, o'[rp_v]
   int* counters;            // [B*H] arrivals per unit (all zero between calls); NULL = separate combine launch
   int* status;
+  const int32_t* deficit;   // [B]: sequence b holds n - deficit[b] rows (a batch of unequal lengths); NULL = all hold n
   int32_t part_stride;      // floats per partial slot (multiple of 4)
   int32_t B, H, d_head;
-  int32_t n;                // cached rows to stream (the new token's row, if any, comes on top)
+  int32_t n;                // cached rows of the longest sequence (the new token's row, if any, comes on top)
   int32_t n_max;
   int32_t tile_rows;        // rows per tile
   int32_t nt;               // tiles per unit = ceil(n / tile_rows)
@@ -82,6 +83,7 @@ struct ProjectParams {       // project rows with U and scatter them into the ca
   int32_t B, T, H, d_head;
   int32_t n_max;
   int32_t row0;             // first cache row to write (= len before the call)
+  const int32_t* deficit;   // [B]: sequence b starts at row0 - deficit[b] (unequal lengths); NULL = all at row0
   int32_t lr_k_width, lr_v_width;   // widths of the packed rank-space rows (sum of rp_k / rp_v)
   uint32_t flags;
 };

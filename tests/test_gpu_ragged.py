@@ -1,0 +1,130 @@
+"""GPU parity for a batch whose sequences differ in length (eigen_attn_set_lens): every sequence attends its own
+rows and grows at its own end.  The generation phase of Section 2 is stated per sequence, so the expected value
+of sequence b is the oracle run on that sequence alone with its own history."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, make_case, oracle_layer, storage_model, to_np
+from paper_2408_05646_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+BF16, FP32 = torch.bfloat16, torch.float32
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    return binding
+
+
+class PerSequenceOracle:
+    """One single-sequence oracle layer per sequence of the batch."""
+
+    def __init__(self, H, d, U_k, U_v, k, v, lens, alibi_slopes=None, storage=None):
+        self.H, self.d = H, d
+        self.refs = []
+        for b, n in enumerate(lens):
+            r = oracle_layer(1, H, d, U_k, U_v, alibi_slopes=alibi_slopes, storage=storage)
+            if n > 0:
+                r.append_kv(to_np(k[b:b + 1, :n]), to_np(v[b:b + 1, :n]))
+            self.refs.append(r)
+
+    def append(self, k, v):                       # k, v: [B, T, H, d]
+        for b, r in enumerate(self.refs):
+            r.append_kv(to_np(k[b:b + 1]), to_np(v[b:b + 1]))
+
+    def decode(self, q):                          # q: [B, 1, H, d] -> [B, 1, H, d]
+        return np.concatenate([r.decode_dense(to_np(q[b:b + 1])).reshape(1, 1, self.H, self.d)
+                               for b, r in enumerate(self.refs)], axis=0)
+
+
+@pytest.mark.parametrize("dtype,d,rk,rv,n,lens", [
+    (FP32, 64, [32, 20, 64], [16, 40, 8], 700, [700, 1, 77, 570]),
+    (BF16, 128, [80, 48, 128], [80, 112, 64], 3000, [3000, 129, 1, 2871]),      # units split over many CTAs
+    (BF16, 128, [80, 80, 80], [80, 80, 80], 2048, [5, 2048, 2047, 1024]),       # the first sequence is the short one
+])
+def test_decode_and_steps_with_unequal_lengths(B, dtype, d, rk, rv, n, lens):
+    B_, H = 4, 3
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + 8, dtype, seed_cfg=140, T_q=8)
+    lay = B.EigenAttnLayer(B_, H, d, n + 8, dtype, U_k, U_v)
+    lay.append_kv(k[:, :n], v[:, :n])             # every sequence holds n rows; each keeps its first lens[b]
+    lay.set_lens(lens)
+    assert lay.lens() == list(lens) and lay.len == max(lens)
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens)
+    expect = ref.decode(q[:, :1])
+    for ctas, fused in ((0, 1), (0, 0), (1, 1), (37, 0), (5, 1)):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        lay.set_option(B.EA_OPT_DECODE_FUSED, fused)
+        assert_close(lay.decode(q[:, :1]), expect, dtype, f"decode ctas={ctas} fused={fused}")
+    lay.set_option(B.EA_OPT_DECODE_CTAS, 0)
+    assert_close(lay.decode_static(q[:, :1]), expect, dtype, "decode_static")
+    # generation: each sequence's new row goes behind its own end (fresh rows, not the ones cut off above)
+    for step, fused in enumerate((1, 1, 0)):
+        lay.set_option(B.EA_OPT_DECODE_FUSED, fused)
+        kn, vn = k[:, n + step:n + step + 1], v[:, n + step:n + step + 1]
+        o = lay.decode_step(q[:, step + 1:step + 2], kn, vn)
+        ref.append(kn, vn)
+        assert_close(o, ref.decode(q[:, step + 1:step + 2]), dtype, f"decode_step {step} fused={fused}")
+    assert lay.lens() == [x + 3 for x in lens]
+    # several rows at once behind each end
+    lay.append_kv(k[:, n + 3:n + 8], v[:, n + 3:n + 8])
+    ref.append(k[:, n + 3:n + 8], v[:, n + 3:n + 8])
+    lay.set_option(B.EA_OPT_DECODE_FUSED, 1)
+    assert_close(lay.decode(q[:, 4:5]), ref.decode(q[:, 4:5]), dtype, "decode after append_kv")
+    lay.poll_status()
+
+
+def test_sequence_with_no_rows_and_return_to_equal_lengths(B):
+    B_, H, d, n = 3, 2, 64, 300
+    rk, rv = [32, 24], [16, 40]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + 1, FP32, seed_cfg=141, T_q=2)
+    lay = B.EigenAttnLayer(B_, H, d, n + 1, FP32, U_k, U_v, max_prefill_tokens=16)
+    lay.append_kv(k[:, :n], v[:, :n])
+    uniform = lay.decode(q[:, :1]).clone()
+    lens = [0, n, 150]
+    lay.set_lens(lens)
+    with pytest.raises(B.EigenAttnError) as e:    # a sequence without rows has nothing to attend
+        lay.decode(q[:, :1])
+    assert e.value.status == B.EA_ERR_SHAPE
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.prefill(q[:, :1].contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous())
+    assert e.value.status == B.EA_ERR_UNSUPPORTED and lay.lens() == lens
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.set_lens([0, n + 2, 1])
+    assert e.value.status == B.EA_ERR_CAPACITY and lay.lens() == lens
+    # with its new token the empty sequence attends exactly that token
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens)
+    o = lay.decode_step(q[:, 1:2], k[:, n:n + 1], v[:, n:n + 1])
+    ref.append(k[:, n:n + 1], v[:, n:n + 1])
+    assert_close(o, ref.decode(q[:, 1:2]), FP32, "decode_step with an empty sequence")
+    assert lay.lens() == [1, n + 1, 151]
+    lay.set_len(n)                                # equal lengths again: rows [0, n) of every sequence
+    assert lay.lens() == [n] * B_
+    # the step above overwrote row 0 of sequence 0 and row 150 of sequence 2; sequence 1 is as before
+    again = lay.decode(q[:, :1])
+    assert torch.equal(again[1], uniform[1])
+    lay.poll_status()
+
+
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_alibi_positions_count_from_each_sequences_own_end(B, dtype):
+    B_, H, d, n = 3, 4, 64, 900
+    rk, rv = [32, 48, 64, 16], [32, 16, 64, 48]
+    lens = [900, 333, 2]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + 1, dtype, seed_cfg=142, T_q=2)
+    slopes = synth.alibi_slopes(H)
+    lay = B.EigenAttnLayer(B_, H, d, n + 1, dtype, U_k, U_v)
+    lay.set_alibi(slopes)
+    lay.append_kv(k[:, :n], v[:, :n])
+    lay.set_lens(lens)
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens, alibi_slopes=slopes, storage=storage_model(dtype))
+    tol = dict(fp32_rel=2e-5) if dtype == FP32 else {}
+    assert_close(lay.decode(q[:, :1]), ref.decode(q[:, :1]), dtype, "decode", **tol)
+    o = lay.decode_step(q[:, 1:2], k[:, n:n + 1], v[:, n:n + 1])
+    ref.append(k[:, n:n + 1], v[:, n:n + 1])
+    assert_close(o, ref.decode(q[:, 1:2]), dtype, "decode_step", **tol)
+    lay.poll_status()
