@@ -540,6 +540,63 @@ def run_prefill(args, wl):
     }))
 
 
+def run_ragged(args, wl):
+    """Decode over a batch whose sequences differ in length (eigen_attn_set_lens): sequence b keeps
+    (b + 1) / B of the context.  One JSON line: KV bytes of the TRUE lengths per second against the HBM roofline,
+    and the same batch with every sequence at full length beside it."""
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    lay, ranks, U_k, U_v, _, q, k_new, v_new = build_layer(wl, device, binding)
+    n0, Bn = wl.context, wl.batch
+    lens = [max(1, n0 * (b + 1) // Bn) for b in range(Bn)]
+    stream = torch.cuda.current_stream(device)
+    out = torch.empty_like(q)
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    def timed(prepare):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            a.record(stream); b.record(stream)
+        prepare()
+        for _ in range(warmup):
+            lay.decode(q, out=out)
+        torch.cuda.synchronize(device)
+        for i in range(steps):
+            lay.set_decode_events(ev[i][0], ev[i][1])
+            lay.decode(q, out=out)
+        torch.cuda.synchronize(device)
+        lay.set_decode_events(None, None)
+        return sum(a.elapsed_time(b) for a, b in ev) / steps * 1e3      # us per decode kernel
+
+    sampler = ClockSampler(device.index or 0)
+    sampler.start(); time.sleep(0.2)
+    l0 = lay.launch_count()
+    us_ragged = timed(lambda: lay.set_lens(lens))
+    launches = lay.launch_count() - l0
+    us_full = timed(lambda: lay.set_len(n0))
+    clocks = sampler.stop()
+    lay.poll_status()
+    row_bytes = sum(2 * (rk + rv) for rk, rv in zip(ranks, ranks))          # bf16 K' + V' row of all heads
+    bytes_true = sum(lens) * row_bytes
+    peak, src = measured_peaks()
+    achieved = bytes_true / (us_ragged * 1e-6) / 1e9
+    print(json.dumps({
+        "metric": "rank-r decode attention KV GB/s, batch of unequal lengths", "value": achieved, "unit": "GB/s",
+        "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": us_ragged * 1e-3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
+        "config": {"workload": wl.name + " with lens[b] = context * (b + 1) / batch", "batch": Bn, "context": n0,
+                   "mean_len": sum(lens) / Bn, "l2": "inputs larger than L2"},
+        "roofline": {"bound": "hbm", "kernel": "decode_splitkv_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": src, "kernel_us": us_ragged, "algorithmic_bytes": bytes_true,
+                     "traffic": None},
+        "all_sequences_at_full_length": {"kernel_us": us_full, "GB/s": Bn * n0 * row_bytes / (us_full * 1e-6) / 1e9},
+        "gpu_launches": launches, "clocks": clocks,
+    }))
+
+
 def run_gqa(args, wl):
     """Grouped-query decode step: append the new token's K/V rows, then one pass over the rank-r cache of every K/V
     head serves its whole group of query heads.  One JSON line: KV GB/s of that pass against the HBM roofline, and
@@ -741,6 +798,7 @@ def main():
     ap.add_argument("--rope", action="store_true", help="decode workloads: the RoPE variant (full-rank query, lifted rotated keys)")
     ap.add_argument("--quant", type=int, default=0, metavar="G",
                     help="decode workloads: attend over the 4-bit quantised cache with group size G (16, 32, 64, 128)")
+    ap.add_argument("--ragged", action="store_true", help="decode workloads: sequence b keeps (b + 1) / batch of the context")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
@@ -765,6 +823,8 @@ def main():
         return run_gqa(args, wl)
     if args.quant:
         return run_quant(args, wl)
+    if args.ragged:
+        return run_ragged(args, wl)
     if wl.name.startswith("prefill"):
         run_prefill(args, wl)
     else:

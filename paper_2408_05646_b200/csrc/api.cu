@@ -335,7 +335,17 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   }
 
   const int nt = (n + tile_rows - 1) / tile_rows;
-  const int64_t w_total = static_cast<int64_t>(nt) * B * L.sum_w;
+  // Tiles of one head.  Unequal lengths: every sequence contributes its own tiles (at least one, so that some CTA
+  // attends the new token of a sequence without rows), hence the CTA ranges follow the true lengths.
+  int64_t nt_total = static_cast<int64_t>(nt) * B;
+  if (h->max_deficit > 0) {
+    nt_total = 0;
+    for (int b = 0; b < B; ++b) {
+      const int tiles = (n - h->deficit[b] + tile_rows - 1) / tile_rows;
+      nt_total += tiles > 0 ? tiles : 1;
+    }
+  }
+  const int64_t w_total = nt_total * L.sum_w;
   int grid = sms;
   const int64_t cap = w_total / L.max_w;          // every CTA must own at least one tile
   if (grid > cap) grid = static_cast<int>(cap);
@@ -355,6 +365,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.tile_rows = tile_rows; p.nt = nt; p.ring_bytes = ring_bytes; p.inflight_bytes = kInFlightBytes;
   p.fixed_stages = static_cast<int>(h->opt_stages);
+  p.nt_total = nt_total;
   p.w_total = w_total;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
@@ -366,6 +377,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   c.heads = p.heads; c.basis = p.basis; c.partials = partials; c.out = d_out;
   c.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
   c.part_stride = L.part_stride; c.B = B; c.H = H; c.d_head = h->desc.d_head; c.nt = nt; c.grid = grid;
+  c.deficit = p.deficit; c.n = n; c.tile_rows = tile_rows; c.nt_total = nt_total;
   c.w_total = w_total; c.flags = flags;
   return EA_OK;
 }
@@ -805,6 +817,8 @@ ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_st
   if (h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a quantised cache attached");
   if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a rotary embedding");
   const int B = h->desc.batch;
+  if (B > ea::kMaxRaggedBatch)
+    return fail(h, EA_ERR_UNSUPPORTED, "set_lens: batch %d exceeds %d", B, ea::kMaxRaggedBatch);
   int32_t longest = 0;
   for (int b = 0; b < B; ++b) {
     if (lens[b] < 0 || lens[b] > h->desc.n_max)

@@ -42,6 +42,7 @@ struct __align__(128) DecodeSmemFixed {
   float wsum[kDecodeConsumerWarps];
   float o_acc[128];                        // the piece's (later the unit's) o'
   float stage_o[kDecodeConsumerWarps][4][128];
+  int pre[kMaxRaggedBatch + 1];            // unequal lengths: tiles of the sequences before b (exclusive prefix)
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -176,7 +177,7 @@ struct Elem<float> {
 // First tile (in the flat order head-major, then sequence, then tile) whose start weight x
 // satisfies x * grid >= c * w_total.  Tiles of head h weigh (rp_k + rp_v).
 __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
-  const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
+  const long long per_head_tiles = p.nt_total;
   if (c >= grid) return per_head_tiles * p.H;
   const long long num = static_cast<long long>(c) * p.w_total;
   const long long target = (num + grid - 1) / grid;
@@ -190,10 +191,48 @@ __device__ long long first_tile_of_cta(const DecodeParams& p, int grid, int c) {
   return per_head_tiles * h + idx;
 }
 
-// Cached rows of sequence b: p.n for a batch of equal lengths, else p.n minus the sequence's deficit.  The work
-// decomposition stays the one of the longest sequence; a shorter sequence simply has no rows in its last tiles.
+// Cached rows of sequence b: p.n for a batch of equal lengths, else p.n minus the sequence's deficit.
 __device__ __forceinline__ int seq_rows(const DecodeParams& p, int b) {
   return p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;
+}
+// Tiles of a sequence of n_b rows; a sequence without rows still owns one (empty) tile, so that some CTA
+// attends its new token.
+__device__ __forceinline__ int seq_tiles(const DecodeParams& p, int n_b) {
+  const int t = (n_b + p.tile_rows - 1) / p.tile_rows;
+  return t > 0 ? t : 1;
+}
+
+// Where the flat tile index F falls: the unit (head h, sequence b), the tile i0 inside it, the unit's tile count
+// and the tiles of the head that precede the unit.  Equal lengths: plain division.  Unequal lengths: the flat
+// order holds each sequence's own tiles only, and `pre` (shared memory) is their exclusive prefix over b.
+struct Piece {
+  int unit, h, b, i0, nt_u;
+  long long t0;
+};
+__device__ __forceinline__ Piece locate(const DecodeParams& p, const int* pre, long long F) {
+  Piece u;
+  if (p.deficit == nullptr) {
+    u.unit = static_cast<int>(F / p.nt);
+    u.i0 = static_cast<int>(F - static_cast<long long>(u.unit) * p.nt);
+    u.h = u.unit / p.B;
+    u.b = u.unit - u.h * p.B;
+    u.nt_u = p.nt;
+    u.t0 = static_cast<long long>(u.b) * p.nt;
+  } else {
+    u.h = static_cast<int>(F / p.nt_total);
+    const int rem = static_cast<int>(F - static_cast<long long>(u.h) * p.nt_total);
+    int lo = 0, hi = p.B;                            // largest b with pre[b] <= rem
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (pre[mid] <= rem) lo = mid; else hi = mid;
+    }
+    u.b = lo;
+    u.i0 = rem - pre[lo];
+    u.nt_u = pre[lo + 1] - pre[lo];
+    u.t0 = pre[lo];
+    u.unit = u.h * p.B + lo;
+  }
+  return u;
 }
 
 // ---------------------------------------------------------------- one (CTA, unit) piece
@@ -445,7 +484,8 @@ __device__ __forceinline__ int owner_cta(long long x, int grid, long long w_tota
 // directly if the piece is the whole unit, else through the partial slots and the arrival counter.
 template <typename T>
 __device__ __forceinline__ void finish_piece(const DecodeParams& p, DecodeSmemFixed* fx, const HeadInfo& hd,
-                                             int unit, int h, int b, int cta, int grid, bool whole, int t) {
+                                             const Piece& pc, int cta, int grid, bool whole, int t) {
+  const int unit = pc.unit, h = pc.h, b = pc.b;
   bool finalize = whole && p.counters != nullptr;
   float inv_l = 1.f / fx->piece_l;
   if (!finalize) {
@@ -456,11 +496,10 @@ __device__ __forceinline__ void finish_piece(const DecodeParams& p, DecodeSmemFi
       consumer_sync();
       return;
     }
-    const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
     const long long w = hd.rp_k + hd.rp_v;
-    const long long x0 = per_head_tiles * hd.w_prefix + static_cast<long long>(b) * p.nt * w;
+    const long long x0 = p.nt_total * hd.w_prefix + pc.t0 * w;
     const int c0 = owner_cta(x0, grid, p.w_total);
-    const int c1 = owner_cta(x0 + static_cast<long long>(p.nt - 1) * w, grid, p.w_total);
+    const int c1 = owner_cta(x0 + static_cast<long long>(pc.nt_u - 1) * w, grid, p.w_total);
     __threadfence();                  // this thread's partial is visible before the arrival is counted
     consumer_sync();
     if (t == 0) {
@@ -511,6 +550,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int grid = gridDim.x, cta = blockIdx.x;
 
+  if (p.deficit != nullptr) {         // unequal lengths: tiles per sequence, then their exclusive prefix
+    for (int b = tid; b < p.B; b += kDecodeThreads) fx->pre[b + 1] = seq_tiles(p, seq_rows(p, b));
+    __syncthreads();
+    if (tid == 0) {
+      fx->pre[0] = 0;
+      for (int b = 0; b < p.B; ++b) fx->pre[b + 1] += fx->pre[b];
+    }
+  }
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(&fx->full[s], 1);
@@ -534,14 +581,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       long long F = f_lo;
       while (F < f_hi && ok) {
         // one (CTA, unit) piece: tiles [i0, i1) of `unit`; everything per tile below is incremental
-        const int unit = static_cast<int>(F / p.nt);
-        const int i0 = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
-        const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + (f_hi - F)));
-        const int h = unit / p.B, b = unit - h * p.B;
-        const HeadInfo hd = p.heads[h];
+        const Piece pc = locate(p, fx->pre, F);
+        const int i0 = pc.i0, b = pc.b;
+        const int i1 = static_cast<int>(min(static_cast<long long>(pc.nt_u), i0 + (f_hi - F)));
+        const HeadInfo hd = p.heads[pc.h];
         const int n_b = seq_rows(p, b);
-        const int nt_b = (n_b + p.tile_rows - 1) / p.tile_rows;
-        const int i1e = min(i1, nt_b);    // tiles past the sequence's own length hold nothing
         int sb, voff, nst;
         ring_geometry<T>(p, hd, &sb, &voff, &nst);
         if (sb != rg.stage_bytes || nst != rg.stages) {
@@ -562,7 +606,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
         const char* src_v = p.cache + hd.v_off + row0 * rowb_v;
         const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
-        for (int i = i0; i < i1e; ++i) {
+        for (int i = i0; i < i1; ++i) {
           if (*abort_flag) { ok = false; break; }
           const int st = rg.stage;
           const uint32_t bit = 1u << st;
@@ -575,7 +619,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
             rg.empty_bits ^= bit;
           }
           uint32_t bytes_k = tile_k, bytes_v = tile_v;
-          if (i == nt_b - 1) {            // ragged last tile of the unit
+          if (i == pc.nt_u - 1) {         // ragged last tile of the unit
             const uint32_t rows = n_b - i * p.tile_rows;
             bytes_k = rows * rowb_k;
             bytes_v = rows * rowb_v;
@@ -583,8 +627,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
           unsigned char* dst = ring + static_cast<size_t>(st) * rg.stage_bytes;
           void* bar = &fx->full[st];
           mbar_arrive_expect_tx(bar, bytes_k + bytes_v);
-          bulk_g2s_hint(dst, src_k, bytes_k, bar, policy);
-          bulk_g2s_hint(dst + rg.v_off, src_v, bytes_v, bar, policy);
+          if (bytes_k != 0) {             // a sequence without cached rows owns one empty tile
+            bulk_g2s_hint(dst, src_k, bytes_k, bar, policy);
+            bulk_g2s_hint(dst + rg.v_off, src_v, bytes_v, bar, policy);
+          }
           rg.filled |= bit;
           rg.full_bits ^= bit;            // bit now holds the parity of the slot's next fill
           src_k += tile_k;
@@ -603,11 +649,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
     Ring rg;
     long long F = f_lo;
     while (F < f_hi) {
-      const int unit = static_cast<int>(F / p.nt);
-      const int i0 = static_cast<int>(F - static_cast<long long>(unit) * p.nt);
+      const Piece pc = locate(p, fx->pre, F);
+      const int i0 = pc.i0, h = pc.h, b = pc.b;
       const long long left = f_hi - F;
-      const int i1 = static_cast<int>(min(static_cast<long long>(p.nt), i0 + left));
-      const int h = unit / p.B, b = unit - h * p.B;
+      const int i1 = static_cast<int>(min(static_cast<long long>(pc.nt_u), i0 + left));
       const HeadInfo hd = p.heads[h];
       {
         int sb, voff, nst;
@@ -617,25 +662,24 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         }
         rg.v_off = voff;
       }
-      const bool whole = i0 == 0 && i1 == p.nt;
-      const bool with_new_row = p.k_new != nullptr && i1 == p.nt;
+      const bool whole = i0 == 0 && i1 == pc.nt_u;
+      const bool with_new_row = p.k_new != nullptr && i1 == pc.nt_u;
       const int n_b = seq_rows(p, b);
-      const int i1e = min(i1, (n_b + p.tile_rows - 1) / p.tile_rows);   // as in the producer
       project_inputs<T>(p, fx, hd, h, b, tid, with_new_row, n_b);
       const int mx = max(hd.rp_k, hd.rp_v);
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1e, rg, warp, lane, with_new_row, n_b); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
       }
-      finish_piece<T>(p, fx, hd, unit, h, b, cta, grid, whole, tid);
+      finish_piece<T>(p, fx, hd, pc, cta, grid, whole, tid);
       F += i1 - i0;
     }
   }
@@ -650,10 +694,20 @@ __global__ void __launch_bounds__(128) combine_lift_kernel(const CombineParams p
   const int unit = blockIdx.x;
   const int h = unit / p.B, b = unit - h * p.B;
   const HeadInfo hd = p.heads[h];
-  const long long per_head_tiles = static_cast<long long>(p.B) * p.nt;
   const long long w = hd.rp_k + hd.rp_v;
-  const long long x0 = per_head_tiles * hd.w_prefix + static_cast<long long>(b) * p.nt * w;
-  const long long x1 = x0 + static_cast<long long>(p.nt - 1) * w;
+  long long t0 = static_cast<long long>(b) * p.nt;        // tiles of the head before this unit
+  int nt_u = p.nt;
+  if (p.deficit != nullptr) {                             // unequal lengths: each sequence has its own tile count
+    auto tiles_of = [&](int bb) {
+      const int t = (p.n - __ldg(p.deficit + bb) + p.tile_rows - 1) / p.tile_rows;
+      return t > 0 ? t : 1;
+    };
+    t0 = 0;
+    for (int bb = 0; bb < b; ++bb) t0 += tiles_of(bb);
+    nt_u = tiles_of(b);
+  }
+  const long long x0 = p.nt_total * hd.w_prefix + t0 * w;
+  const long long x1 = x0 + static_cast<long long>(nt_u - 1) * w;
   const int c0 = owner_cta(x0, p.grid, p.w_total);
   const int c1 = owner_cta(x1, p.grid, p.w_total);
   const int t = threadIdx.x;

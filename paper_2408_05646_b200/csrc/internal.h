@@ -29,6 +29,7 @@ constexpr int kDecodeConsumerWarps = 8;
 constexpr int kDecodeThreads = (kDecodeConsumerWarps + 1) * 32;   // + one producer warp
 constexpr int kMaxHeads = 256;
 constexpr int kStatusTimeout = -6;
+constexpr int kMaxRaggedBatch = 1024;   // largest batch that may hold sequences of unequal lengths
 
 struct DecodeParams {
   const HeadInfo* heads;
@@ -54,7 +55,8 @@ struct DecodeParams {
   int32_t ring_bytes;       // shared memory of the tile ring; slots are sized per head inside the kernel
   int32_t inflight_bytes;   // target bytes of copies in flight per SM (sets the slot count per head)
   int32_t fixed_stages;     // > 0: use this many slots (if they fit) instead of the in-flight target
-  int64_t w_total;          // nt * B * sum_h (rp_k + rp_v)
+  int64_t nt_total;         // tiles of one head: B * nt, or the sum of the sequences' own tile counts
+  int64_t w_total;          // nt_total * sum_h (rp_k + rp_v)
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
 };
@@ -69,6 +71,9 @@ struct CombineParams {
   int32_t B, H, d_head;
   int32_t nt;
   int32_t grid;             // CTAs of the split-KV kernel that produced the partials
+  const int32_t* deficit;   // as in DecodeParams (NULL: equal lengths)
+  int32_t n, tile_rows;
+  int64_t nt_total;
   int64_t w_total;
   uint32_t flags;
 };
