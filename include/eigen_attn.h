@@ -219,12 +219,12 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
  * lens: HOST array [batch], 0 <= lens[b] <= n_max; sequence b then holds rows [0, lens[b]) of its slabs, whatever
  * was written there before (a prompt batch padded to a common T and prefilled keeps its first lens[b] rows).
  * eigen_attn_get_len reports the longest sequence.  Afterwards eigen_attn_append_kv and eigen_attn_decode_step
- * add rows behind each sequence's own end, eigen_attn_decode / _decode_step / _decode_static attend each
+ * add rows behind each sequence's own end, eigen_attn_decode / _decode_step / _decode_static / _decode_gqa attend each
  * sequence's own rows (ALiBi positions count from the sequence's own end); decode needs lens[b] >= 1 for every
  * b (EA_ERR_SHAPE otherwise).  The split-KV work decomposition follows the true lengths, so a step costs what
  * the rows actually cached cost.  batch <= 1024.  eigen_attn_set_len returns to equal lengths.
  * Not available (EA_ERR_UNSUPPORTED) with a rotary embedding or a quantised cache attached; while lengths differ,
- * prefill, decode_gqa and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
+ * prefill and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
  * (asynchronous; the array may be reused when the call returns). */
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);
 ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens);

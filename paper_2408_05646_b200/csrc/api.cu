@@ -915,13 +915,12 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
 ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
                                 int64_t stride_b_out, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_gqa: NULL q or out");
   if (group < 1 || group > 16) return fail(h, EA_ERR_SHAPE, "decode_gqa: group %d (1..16)", group);
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
   if (h->rope || h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a position scheme set");
-  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty");
+  if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty (for some sequence)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const size_t smem = ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
@@ -933,6 +932,7 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
   p.status = dev_status(h);
   p.tmaps = h->ws + L.off_tmaps;
+  p.deficit = dev_deficit(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;

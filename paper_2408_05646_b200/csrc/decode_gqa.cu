@@ -88,8 +88,12 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
   unsigned char* Km = Vst + vst_bytes;                       // K' tile, canonical core-matrix layout
   unsigned char* Vm = Km + km_bytes;                         // V' tile, canonical core-matrix layout
 
-  const int per = (p.nt + p.splits - 1) / p.splits;
-  const int t_lo = split * per, t_hi = min(p.nt, t_lo + per);
+  // rows and tiles of this sequence (a batch of unequal lengths gives every sequence its own count; the splits
+  // of a unit divide the sequence's own tiles)
+  const int n_b = p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;
+  const int nt_b = (n_b + kTile - 1) / kTile;
+  const int per = (nt_b + p.splits - 1) / p.splits;
+  const int t_lo = split * per, t_hi = min(nt_b, t_lo + per);
   float* part = p.partials + (static_cast<size_t>(unit) * p.splits + split) * G * p.part_stride;
   if (t_lo >= t_hi) {                                        // an empty piece: neutral partials
     for (int qi = 0; qi < G; ++qi) {
@@ -136,12 +140,12 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
   const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
   const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
   auto fetch_k = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_k;
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_k;
     mbar_arrive_expect_tx(&hdr->k_full, bytes);
     bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
   };
   auto fetch_v = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_v;
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
     mbar_arrive_expect_tx(&hdr->v_full, bytes);
     bulk_load(Vst, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
   };
@@ -247,7 +251,7 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     uint32_t sr[16];
     tmem_ld16(tmem + lane_base + 32 * par, sr);
     tmem_wait_ld();
-    const bool live = t * kTile + tid < p.n;
+    const bool live = t * kTile + tid < n_b;
     // ---- per-query maximum over the tile: one reduction instruction per query and warp, lane q keeps query q's
 #pragma unroll
     for (int qi = 0; qi < GP; ++qi) {

@@ -167,10 +167,11 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
   float* partials;          // [B*H][splits][group][part_stride]: m, l, pad, pad, o'[rp_v]
   int* status;
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every K/V head
+  const int32_t* deficit;   // [B]: sequence b holds n - deficit[b] rows; NULL = all hold n
   int32_t part_stride;
   int32_t B, H, d_head;
   int32_t n, n_max;
-  int32_t nt;               // tiles of 128 rows per unit
+  int32_t nt;               // tiles of 128 rows per unit (of the longest sequence)
   int32_t splits;           // CTAs per unit
   int32_t group;            // 1..16
   float q_scale;            // log2(e) / sqrt(d_head)
