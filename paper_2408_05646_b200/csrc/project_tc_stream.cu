@@ -36,21 +36,30 @@ struct PsHeader {
   int abort_flag;
 };
 
+// Position in the flat order of work items (pair = head * 3 + which, then sequence, then tile of the sequence);
+// set up with divisions once per CTA and role, advanced by increments.
 struct PsItem {
-  int h, which, b, t0;
+  int h, which, b, tt;      // which: 0 = Q, 1 = K, 2 = V; tt: tile of the sequence
+  __device__ __forceinline__ void init(int64_t w, int tiles, int tps) {
+    const int pair = static_cast<int>(w / tiles);
+    const int tile = static_cast<int>(w - static_cast<int64_t>(pair) * tiles);
+    h = pair / 3;
+    which = pair - h * 3;
+    b = tile / tps;
+    tt = tile - b * tps;
+  }
+  __device__ __forceinline__ void next(int B, int tps) {
+    if (++tt == tps) {
+      tt = 0;
+      if (++b == B) {
+        b = 0;
+        if (++which == 3) { which = 0; ++h; }
+      }
+    }
+  }
 };
 
-__device__ __forceinline__ PsItem ps_item(int64_t w, int tiles, int tps) {
-  PsItem it;
-  const int pair = static_cast<int>(w / tiles);
-  const int tile = static_cast<int>(w - static_cast<int64_t>(pair) * tiles);
-  it.h = pair / 3;
-  it.which = pair - it.h * 3;
-  it.b = tile / tps;
-  it.t0 = (tile - it.b * tps) * kTile;
-  return it;
-}
-
+template <int KS>               // contraction steps of 16 elements: d_head / 16 (4 or 8)
 __global__ void __launch_bounds__(kPsThreads, 1)
 project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtensorMap map_q,
                          const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -101,8 +110,9 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
       int prev_stage = 0;
       uint32_t prev_parity = 0;                              // phase in which the previous tile's stage is released
       int cur_h = -1, cur_v = -1, u_loads = 0;
-      for (int i = 0; i < n_items; ++i) {
-        const PsItem it = ps_item(w_begin + i, tiles, tps);
+      PsItem it;
+      it.init(w_begin, tiles, tps);
+      for (int i = 0; i < n_items; ++i, it.next(p.B, tps)) {
         const int is_v = it.which == 2;
         if (it.h != cur_h || is_v != cur_v) {
           // the products of every earlier tile have read the old image once the newest tile's stage is released
@@ -127,7 +137,7 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
         unsigned char* st = Xring + stage * x_bytes;
         mbar_arrive_expect_tx(&hdr->x_full[stage], static_cast<uint32_t>(x_bytes));
         for (int a = 0; a < atoms; ++a)
-          tma_load_3d(st + a * kAtomBytesA, map, it.h * p.d_head + a * 64, it.t0, it.b, &hdr->x_full[stage]);
+          tma_load_3d(st + a * kAtomBytesA, map, it.h * p.d_head + a * 64, it.tt * kTile, it.b, &hdr->x_full[stage]);
         ++issued;
         prev_stage = stage;
         prev_parity = empty_parity ^ 1u;
@@ -151,17 +161,25 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
       bool ok = true;
       int stage = 0;
       uint32_t full_parity = 0, u_parity = 0;
-      int cur_h = -1, cur_v = -1, rp16 = 16;
-      const uint32_t xa0 = smem_u32(Xring), uh = smem_u32(Us);
-      for (int i = 0; i < n_items && ok; ++i) {
-        const PsItem it = ps_item(w_begin + i, tiles, tps);
+      int cur_h = -1, cur_v = -1;
+      // descriptors of stage 0 / the high image; a step, a stage or the low image only moves the start address
+      const uint64_t a0 = smem_desc_sw128(smem_u32(Xring), 16, 1024);
+      const uint64_t b0 = smem_desc(smem_u32(Us), 128, grp_d);
+      const uint64_t stage_step = static_cast<uint64_t>(x_bytes >> 4);
+      uint64_t lo_step = 0;                                  // from the high to the low image of the current basis
+      uint32_t idesc = 0;
+      PsItem it;
+      it.init(w_begin, tiles, tps);
+      for (int i = 0; i < n_items && ok; ++i, it.next(p.B, tps)) {
         const int is_v = it.which == 2;
         if (it.h != cur_h || is_v != cur_v) {
           ok = mbar_wait(&hdr->u_full, u_parity, p.status) && !*abort_flag;
           if (!ok) break;
           u_parity ^= 1u;
           const HeadInfo hd = p.heads[it.h];
-          rp16 = ((is_v ? hd.rp_v : hd.rp_k) + 15) & ~15;
+          const int rp16 = ((is_v ? hd.rp_v : hd.rp_k) + 15) & ~15;
+          idesc = instr_desc(rp16, false);
+          lo_step = static_cast<uint64_t>((rp16 * p.d_head * 2) >> 4);
           cur_h = it.h;
           cur_v = is_v;
         }
@@ -173,17 +191,14 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
         ok = mbar_wait(&hdr->x_full[stage], full_parity, p.status) && !*abort_flag;
         if (!ok) break;
         tc_fence_after();
-        const uint32_t idesc = instr_desc(rp16, false);
-        const uint32_t xa = xa0 + stage * x_bytes;
-        const uint32_t ul = uh + rp16 * p.d_head * 2;
+        const uint64_t a_st = a0 + stage * stage_step;
         const uint32_t d_tmem = tmem + acc * ncols;
-        bool accumulate = false;
-        for (int pass = 0; pass < 2; ++pass)
-          for (int s = 0; s < p.d_head / 16; ++s) {           // contraction over d_head, 16 elements per step
-            mma_ss(d_tmem, smem_desc_sw128(xa + (s >> 2) * kAtomBytesA + (s & 3) * 32, 16, 1024),
-                   smem_desc((pass ? ul : uh) + s * 256, 128, grp_d), idesc, accumulate);
-            accumulate = true;
-          }
+#pragma unroll
+        for (int s = 0; s < KS; ++s)                         // contraction over d_head, 16 elements per step
+          mma_ss(d_tmem, a_st + ((s >> 2) * (kAtomBytesA >> 4) + (s & 3) * 2), b0 + s * 16, idesc, s > 0);
+#pragma unroll
+        for (int s = 0; s < KS; ++s)                         // the low part of the basis on top
+          mma_ss(d_tmem, a_st + ((s >> 2) * (kAtomBytesA >> 4) + (s & 3) * 2), b0 + lo_step + s * 16, idesc, true);
         mma_commit(&hdr->x_empty[stage]);                    // the tile (and the image) have been read
         mma_commit(&hdr->acc_full[acc]);
         if (++stage == stages) { stage = 0; full_parity ^= 1u; }
@@ -197,8 +212,9 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     const int64_t total_rows = static_cast<int64_t>(p.B) * p.T;
     bool ok = true;
-    for (int i = 0; i < n_items; ++i) {
-      const PsItem it = ps_item(w_begin + i, tiles, tps);
+    PsItem it;
+    it.init(w_begin, tiles, tps);
+    for (int i = 0; i < n_items; ++i, it.next(p.B, tps)) {
       const HeadInfo hd = p.heads[it.h];
       const bool is_v = it.which == 2;
       const int rp = is_v ? hd.rp_v : hd.rp_k;
@@ -207,7 +223,7 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
       ok = mbar_wait(&hdr->acc_full[acc], (i >> 1) & 1u, p.status) && !*abort_flag;
       if (!ok) break;
       tc_fence_after();
-      const int t = it.t0 + row;
+      const int t = it.tt * kTile + row;
       __nv_bfloat16* dst = nullptr;
       if (t < p.T) {
         if (it.which == 0)
@@ -266,12 +282,13 @@ cudaError_t launch_project_tc_stream(const ProjectTcParams& p, const void* maps_
   int stages = 0;
   const size_t smem = project_tc_stream_smem(max_rp, p.d_head, &stages);
   if (stages < 2) return cudaErrorInvalidConfiguration;
-  static size_t configured = 0;     // largest dynamic shared-memory size opted into so far
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(project_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
+  auto kernel = p.d_head == 128 ? project_tc_stream_kernel<8> : project_tc_stream_kernel<4>;
+  static size_t configured[2] = {0, 0};   // largest dynamic shared-memory size opted into so far, per instance
+  size_t& conf = configured[p.d_head == 128 ? 1 : 0];
+  if (smem > conf) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    configured = smem;
+    conf = smem;
   }
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(maps_qkv);
   const int64_t total = 3ll * p.H * p.B * ((p.T + kTile - 1) / kTile);
@@ -279,7 +296,7 @@ cudaError_t launch_project_tc_stream(const ProjectTcParams& p, const void* maps_
   const int rp16 = (max_rp + 15) & ~15;
   uint32_t ncols = 32;                                       // TMEM columns per accumulator: a power of two
   while (static_cast<int>(ncols) < rp16) ncols <<= 1;
-  project_tc_stream_kernel<<<grid, kPsThreads, smem, s>>>(p, maps[0], maps[1], maps[2], stages, ncols);
+  kernel<<<grid, kPsThreads, smem, s>>>(p, maps[0], maps[1], maps[2], stages, ncols);
   ++*launches;
   return cudaGetLastError();
 }
