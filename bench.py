@@ -340,7 +340,9 @@ def run_ours(args, wl):
     achieved = bytes_step / (kern_avg_ms * 1e-3) / 1e9
 
     # ---- end to end: host tensors in, host tensor out, through the C ABI
-    hq, hk, hv = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+    # one pinned buffer holding q, k, v back to back: the library then sends them as a single copy
+    hqkv = torch.stack([q.cpu(), k_new.cpu(), v_new.cpu()]).pin_memory()
+    hq, hk, hv = hqkv[0], hqkv[1], hqkv[2]
     hout = torch.empty_like(hq).pin_memory()
     for _ in range(args.warmup):
         lay.set_len(n0)

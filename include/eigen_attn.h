@@ -131,7 +131,8 @@ ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride
                                  void* d_out, int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
 /* The same step for HOST tensors (contiguous [B][1][H][d_head], ideally pinned): copies q, k, v to a
- * staging area of the workspace, runs the step, copies the result back and synchronises the stream. */
+ * staging area of the workspace, runs the step, copies the result back and synchronises the stream.
+ * When h_k == h_q + bytes and h_v == h_k + bytes (bytes = size of one of the tensors) the three travel as one copy. */
 ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const void* h_k, const void* h_v,
                                       void* h_out, uint32_t flags, void* cuda_stream);
 

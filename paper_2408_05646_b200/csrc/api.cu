@@ -666,9 +666,17 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   char* sk = sq + L.staging_each;
   char* sv = sk + L.staging_each;
   char* so = sv + L.staging_each;
-  cudaError_t e = cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(sk, h_k, bytes, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(sv, h_v, bytes, cudaMemcpyHostToDevice, s);
+  cudaError_t e;
+  const char* hq = static_cast<const char*>(h_q);
+  if (static_cast<const char*>(h_k) == hq + bytes && static_cast<const char*>(h_v) == hq + 2 * bytes &&
+      L.staging_each == bytes) {
+    // q, k, v adjacent on the host (and in the staging area): one copy instead of three
+    e = cudaMemcpyAsync(sq, h_q, 3 * bytes, cudaMemcpyHostToDevice, s);
+  } else {
+    e = cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sk, h_k, bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sv, h_v, bytes, cudaMemcpyHostToDevice, s);
+  }
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_step_host H2D");
   const int64_t sb = static_cast<int64_t>(h->desc.n_heads) * h->desc.d_head;
   const ea_status st = do_step(h, sq, sb, sk, sv, sb, so, sb, 0, s);
