@@ -670,8 +670,15 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   const char* hq = static_cast<const char*>(h_q);
   if (static_cast<const char*>(h_k) == hq + bytes && static_cast<const char*>(h_v) == hq + 2 * bytes &&
       L.staging_each == bytes) {
-    // q, k, v adjacent on the host (and in the staging area): one copy instead of three
+    // q, k, v adjacent on the host (and in the staging area): one copy instead of three.  Adjacent addresses
+    // can still belong to separate pinned allocations, which one copy may not span: then three copies after all.
     e = cudaMemcpyAsync(sq, h_q, 3 * bytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaErrorInvalidValue) {
+      (void)cudaGetLastError();
+      e = cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess) e = cudaMemcpyAsync(sk, h_k, bytes, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess) e = cudaMemcpyAsync(sv, h_v, bytes, cudaMemcpyHostToDevice, s);
+    }
   } else {
     e = cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(sk, h_k, bytes, cudaMemcpyHostToDevice, s);

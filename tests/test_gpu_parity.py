@@ -341,7 +341,8 @@ def test_strided_inputs_and_host_step(B):
     ref.append_kv(to_np(k), to_np(v))
     assert_close(hout, ref.decode_dense(to_np(q)), BF16, "host step")
     assert lay.launch_count() == 2          # one append launch, one fused decode-step launch
-    # q, k, v adjacent in one pinned buffer (they travel as one copy): same result
+    # q, k, v adjacent in one pinned buffer (they travel as one copy): same result.  (The three separate pinned
+    # tensors above can come out adjacent too, from different allocations: the library must then fall back.)
     lay.set_len(n - 1)
     packed = torch.stack([hq, hk, hv]).pin_memory()
     hout2 = torch.empty_like(hq).pin_memory()
