@@ -157,3 +157,27 @@ def test_grouped_query_decode_with_unequal_lengths(B, H, g, d, rk, rv, n, lens):
         r.append_kv(to_np(k[b:b + 1, n:]), to_np(v[b:b + 1, n:]))
     assert_close(lay.decode_gqa(q, g), expect(), BF16, "gqa decode after append")
     lay.poll_status()
+
+
+def test_unequal_lengths_are_refused_where_they_are_not_built(B):
+    B_, H, d, n = 2, 2, 128, 64
+    U_k, U_v, q, k, v = make_case(B_, H, d, [64] * H, [64] * H, n, BF16, seed_cfg=144)
+    lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
+    lay.append_kv(k, v)
+    lay.set_rope(10000.0)
+    with pytest.raises(B.EigenAttnError) as e:    # rotary embedding: positions per sequence are not built
+        lay.set_lens([n, 5])
+    assert e.value.status == B.EA_ERR_UNSUPPORTED
+    lay.set_rope(0.0)
+    lay.set_lens([n, 5])
+    for call in (lambda: lay.quant_attach(4, 32), lambda: lay.set_lens([n, -1]), lambda: lay.set_lens([n + 1, 1])):
+        with pytest.raises(B.EigenAttnError):
+            call()
+    assert lay.lens() == [n, 5]
+    lay.set_lens([n, n])                          # equal again: everything is available
+    assert lay.lens() == [n, n]
+    lay.quant_attach(4, 32)
+    with pytest.raises(B.EigenAttnError) as e:    # and with a quantised cache attached, lengths stay equal
+        lay.set_lens([n, 5])
+    assert e.value.status == B.EA_ERR_UNSUPPORTED
+    lay.poll_status()
