@@ -9,7 +9,8 @@
 //     128-byte swizzled layout (tensor maps of q, k, v are kernel parameters, encoded by the host per call);
 //     rows past T arrive as zeros.  The basis images come as one bulk copy when the basis changes.
 //   warp 1, one thread: MMA issuer, accumulators double-buffered in TMEM.
-//   warps 2-5: epilogue, one thread per token row: TMEM -> bf16 -> cache row (K', V') or Q' scratch row.
+//   warps 2-5: epilogue, one thread per token row: TMEM -> bf16 -> an output tile in shared memory; the rows of a
+//     tile are adjacent in the cache slab (K', V') or the Q' scratch, so the tile leaves as one bulk store.
 // The loads of the next tiles, the products of this one and the stores of the previous one overlap.
 #include <cuda.h>   // CUtensorMap only
 #include <cuda_bf16.h>
@@ -25,6 +26,32 @@ using namespace tc;
 constexpr int kPsThreads = 192;
 constexpr int kPsMaxStages = 4;
 constexpr int kAtomBytesA = kTile * 128;        // one atom column of the token tile: 128 rows of 128 bytes
+
+// Shared -> global bulk copy (both 16-byte aligned, size a multiple of 16) in this thread's bulk group.
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>                                // at most N of this thread's groups still read their source
+__device__ __forceinline__ void bulk_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+// Barrier of the 128 epilogue threads that also tells each of them whether `ok` held for all.
+__device__ __forceinline__ bool epilogue_sync_all(bool ok) {
+  uint32_t all;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "barrier.red.and.pred q, 2, 128, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(all)
+      : "r"(ok ? 1u : 0u)
+      : "memory");
+  return all != 0;
+}
 
 struct PsHeader {
   unsigned long long x_full[kPsMaxStages];
@@ -63,7 +90,7 @@ template <int KS>               // contraction steps of 16 elements: d_head / 16
 __global__ void __launch_bounds__(kPsThreads, 1)
 project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtensorMap map_q,
                          const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                         int stages, uint32_t ncols) {
+                         int stages, uint32_t ncols, int u_bytes_max, int o_bytes_max) {
   extern __shared__ __align__(1024) unsigned char smem[];
   PsHeader* hdr = reinterpret_cast<PsHeader*>(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -211,6 +238,8 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
     const int row = quarter * 32 + lane;
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     const int64_t total_rows = static_cast<int64_t>(p.B) * p.T;
+    const bool issuer = warp == 2 && lane == 0;              // the thread that sends the finished tiles out
+    unsigned char* Obuf = Us + u_bytes_max;                  // two output tiles, [128 rows][rp] bf16 each
     bool ok = true;
     PsItem it;
     it.init(w_begin, tiles, tps);
@@ -221,40 +250,48 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
       const int rp16 = (rp + 15) & ~15;
       const int acc = i & 1;
       ok = mbar_wait(&hdr->acc_full[acc], (i >> 1) & 1u, p.status) && !*abort_flag;
+      // The rows of a tile are adjacent in the destination (rows t0.. of one sequence in a slab or in the Q'
+      // scratch), so the tile is put together in shared memory and leaves as one bulk store.  The buffer of
+      // tile i served tile i - 2: its store must have read the buffer before anyone writes there again.
+      unsigned char* ob = Obuf + acc * o_bytes_max;
+      if (issuer) bulk_store_wait_read<1>();
+      ok = epilogue_sync_all(ok);                            // one decision for the whole group: nobody is left at a barrier
       if (!ok) break;
       tc_fence_after();
-      const int t = it.tt * kTile + row;
-      __nv_bfloat16* dst = nullptr;
-      if (t < p.T) {
-        if (it.which == 0)
-          dst = reinterpret_cast<__nv_bfloat16*>(p.qp) + static_cast<int64_t>(hd.lr_k_off) * total_rows +
-                (static_cast<int64_t>(it.b) * p.T + t) * rp;
-        else
-          dst = reinterpret_cast<__nv_bfloat16*>(p.cache + (is_v ? hd.v_off : hd.k_off)) +
-                (static_cast<int64_t>(it.b) * p.n_max + p.row0 + t) * rp;
-      }
       const uint32_t src = tmem + acc * ncols + lane_base;
+      unsigned char* orow = ob + row * rp * 2;
       for (int c0 = 0; c0 < rp16; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(src + c0, v);
         tmem_wait_ld();
-        if (dst != nullptr) {
-          uint4 w0, w1;
-          w0.x = pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1]));
-          w0.y = pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3]));
-          w0.z = pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5]));
-          w0.w = pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7]));
-          w1.x = pack_bf16(__uint_as_float(v[8]), __uint_as_float(v[9]));
-          w1.y = pack_bf16(__uint_as_float(v[10]), __uint_as_float(v[11]));
-          w1.z = pack_bf16(__uint_as_float(v[12]), __uint_as_float(v[13]));
-          w1.w = pack_bf16(__uint_as_float(v[14]), __uint_as_float(v[15]));
-          *reinterpret_cast<uint4*>(dst + c0) = w0;
-          if (c0 + 8 < rp) *reinterpret_cast<uint4*>(dst + c0 + 8) = w1;
-        }
+        uint4 w0, w1;
+        w0.x = pack_bf16(__uint_as_float(v[0]), __uint_as_float(v[1]));
+        w0.y = pack_bf16(__uint_as_float(v[2]), __uint_as_float(v[3]));
+        w0.z = pack_bf16(__uint_as_float(v[4]), __uint_as_float(v[5]));
+        w0.w = pack_bf16(__uint_as_float(v[6]), __uint_as_float(v[7]));
+        w1.x = pack_bf16(__uint_as_float(v[8]), __uint_as_float(v[9]));
+        w1.y = pack_bf16(__uint_as_float(v[10]), __uint_as_float(v[11]));
+        w1.z = pack_bf16(__uint_as_float(v[12]), __uint_as_float(v[13]));
+        w1.w = pack_bf16(__uint_as_float(v[14]), __uint_as_float(v[15]));
+        *reinterpret_cast<uint4*>(orow + c0 * 2) = w0;
+        if (c0 + 8 < rp) *reinterpret_cast<uint4*>(orow + c0 * 2 + 16) = w1;
       }
       tc_fence_before();
       mbar_arrive(&hdr->acc_empty[acc]);
+      fence_async_smem();                                    // the rows above, before the bulk store reads them
+      epilogue_sync();
+      if (issuer) {
+        const int t0 = it.tt * kTile;
+        const int rows_valid = min(kTile, p.T - t0);
+        char* dst;
+        if (it.which == 0)
+          dst = p.qp + (static_cast<int64_t>(hd.lr_k_off) * total_rows + (static_cast<int64_t>(it.b) * p.T + t0) * rp) * 2;
+        else
+          dst = p.cache + (is_v ? hd.v_off : hd.k_off) + (static_cast<int64_t>(it.b) * p.n_max + p.row0 + t0) * rp * 2;
+        bulk_store(dst, ob, static_cast<uint32_t>(rows_valid * rp * 2));
+      }
     }
+    if (issuer) bulk_store_wait_all();                       // every store issued has completed before the CTA leaves
     if (!ok) *abort_flag = 1;
   }
   tc_fence_before();
@@ -268,13 +305,14 @@ project_tc_stream_kernel(const ProjectTcParams p, const __grid_constant__ CUtens
 // (0 when not even two stages fit).
 size_t project_tc_stream_smem(int max_rp, int d_head, int* stages) {
   const int rp16 = (max_rp + 15) & ~15;
-  const size_t u_bytes = 2ull * rp16 * d_head * 2;
+  const size_t u_bytes = 2ull * rp16 * d_head * 2;             // basis images
+  const size_t o_bytes = 2ull * kTile * rp16 * 2;              // two output tiles
   const size_t x_bytes = static_cast<size_t>(d_head >> 6) * kAtomBytesA;
   const size_t budget = 227 * 1024;
   int s = kPsMaxStages;
-  while (s >= 2 && 1024 + s * x_bytes + u_bytes > budget) --s;
+  while (s >= 2 && 1024 + s * x_bytes + u_bytes + o_bytes > budget) --s;
   *stages = s >= 2 ? s : 0;
-  return 1024 + s * x_bytes + u_bytes;
+  return 1024 + s * x_bytes + u_bytes + o_bytes;
 }
 
 cudaError_t launch_project_tc_stream(const ProjectTcParams& p, const void* maps_qkv, int max_rp, int sm_count,
@@ -296,7 +334,8 @@ cudaError_t launch_project_tc_stream(const ProjectTcParams& p, const void* maps_
   const int rp16 = (max_rp + 15) & ~15;
   uint32_t ncols = 32;                                       // TMEM columns per accumulator: a power of two
   while (static_cast<int>(ncols) < rp16) ncols <<= 1;
-  kernel<<<grid, kPsThreads, smem, s>>>(p, maps[0], maps[1], maps[2], stages, ncols);
+  kernel<<<grid, kPsThreads, smem, s>>>(p, maps[0], maps[1], maps[2], stages, ncols, 2 * rp16 * p.d_head * 2,
+                                        kTile * rp16 * 2);
   ++*launches;
   return cudaGetLastError();
 }
