@@ -224,7 +224,8 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
  * sequence's own rows (ALiBi positions count from the sequence's own end); decode needs lens[b] >= 1 for every
  * b (EA_ERR_SHAPE otherwise).  The split-KV work decomposition follows the true lengths, so a step costs what
  * the rows actually cached cost.  batch <= 1024.  eigen_attn_set_len returns to equal lengths.
- * Not available (EA_ERR_UNSUPPORTED) with a rotary embedding or a quantised cache attached; while lengths differ,
+ * With a rotary embedding each sequence's query sits at its own last position.  Not available
+ * (EA_ERR_UNSUPPORTED) with a quantised cache attached; while lengths differ,
  * prefill and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
  * (asynchronous; the array may be reused when the call returns). */
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);

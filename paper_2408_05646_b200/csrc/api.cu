@@ -402,8 +402,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   if (flags & ~EA_OUT_LOWRANK)
     return fail(h, EA_ERR_INVALID_ARG, "decode with rotary embedding: flag 0x%x (the query must be full rank)", flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
-  if (h->max_deficit > 0)
-    return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: not available for a batch of unequal lengths");
+  if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode: a sequence of the batch has no cached row");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const size_t smem = ea::decode_rope_smem_bytes(L.max_rp_k, L.max_rp_v, h->desc.d_head);
@@ -416,6 +415,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   p.status = dev_status(h);
   p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
   p.tmaps = h->ws + L.off_tmaps;
+  p.deficit = dev_deficit(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;
@@ -830,7 +830,6 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream) {
   if (!h || !lens) return EA_ERR_INVALID_ARG;
   if (h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a quantised cache attached");
-  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a rotary embedding");
   const int B = h->desc.batch;
   if (B > ea::kMaxRaggedBatch)
     return fail(h, EA_ERR_UNSUPPORTED, "set_lens: batch %d exceeds %d", B, ea::kMaxRaggedBatch);

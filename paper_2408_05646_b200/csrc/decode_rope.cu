@@ -67,8 +67,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   unsigned char* Us = Vs + v_bytes;                          // U^K image, canonical layout
 
   // tiles [t_lo, t_hi) of the unit
-  const int per = (p.nt + p.splits - 1) / p.splits;
-  const int t_lo = split * per, t_hi = min(p.nt, t_lo + per);
+  // rows and tiles of this sequence (a batch of unequal lengths gives every sequence its own count and its own
+  // query position; the splits of a unit divide the sequence's own tiles)
+  const int n_b = p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;
+  const int nt_b = (n_b + kTile - 1) / kTile;
+  const int per = (nt_b + p.splits - 1) / p.splits;
+  const int t_lo = split * per, t_hi = min(nt_b, t_lo + per);
   float* part = p.partials + (static_cast<size_t>(unit) * p.splits + split) * p.part_stride;
   if (t_lo >= t_hi) {                                        // an empty piece: the neutral partial
     if (tid == 0) { part[0] = -INFINITY; part[1] = 0.f; }
@@ -98,12 +102,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
   const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
   auto fetch_k = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_k;
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_k;
     mbar_arrive_expect_tx(&hdr->k_full, bytes);
     bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
   };
   auto fetch_v = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, p.n - t * kTile)) * rowb_v;
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
     mbar_arrive_expect_tx(&hdr->v_full, bytes);
     bulk_load(Vs, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
   };
@@ -129,7 +133,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     const float a_re = __bfloat162float(qg[ia]) * p.q_scale, a_im = __bfloat162float(qg[ib]) * p.q_scale;
     const double freq = p.inv_freq[tid];
     double s_, c_;
-    sincos(static_cast<double>(p.n - 1 - t_lo * kTile) * freq, &s_, &c_);
+    sincos(static_cast<double>(n_b - 1 - t_lo * kTile) * freq, &s_, &c_);
     q_re = static_cast<float>(a_re * c_ - a_im * s_);
     q_im = static_cast<float>(a_re * s_ + a_im * c_);
     q_norm2 = a_re * a_re + a_im * a_im;
@@ -152,7 +156,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   volatile int* abort_flag = &hdr->abort_flag;
   const uint32_t idesc = instr_desc(p.d_head, false);
   const int ks_steps = rpk16 >> 4;
-  const int pos_q = p.n - 1;
+  const int pos_q = n_b - 1;
 
   // weighted sum o' += p V': thread (g, c) owns the column pair (2c, 2c+1) over the rows of row group g of every
   // tile; the groups are added up once, at the end
@@ -248,7 +252,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
       fence_async_smem();
     }
     const int j = t * kTile + tid;
-    const bool live = j < p.n;
+    const bool live = j < n_b;
     const float s = live ? s0 + s1 : -INFINITY;
     // ---- online softmax over the tile: block maximum, weights, running sum per thread
     float mx = s;

@@ -145,6 +145,7 @@ struct RopeDecodeParams {    // decode for models with rotary position embedding
   float* partials;          // [B*H][splits][part_stride]: m, l, pad, pad, o'[rp_v]
   int* status;
   const double* inv_freq;   // [d_head/2]: base^(-2i/d_head)
+  const int32_t* deficit;   // [B]: sequence b holds n - deficit[b] rows; NULL = all hold n
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head
   int32_t part_stride;
   int32_t B, H, d_head;

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from helpers import assert_close, make_case, oracle_layer, storage_model, to_np
+from oracle import eigen_attention as orc
 from paper_2408_05646_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -159,16 +160,11 @@ def test_grouped_query_decode_with_unequal_lengths(B, H, g, d, rk, rv, n, lens):
     lay.poll_status()
 
 
-def test_unequal_lengths_are_refused_where_they_are_not_built(B):
+def test_unequal_lengths_are_refused_with_a_quantised_cache(B):
     B_, H, d, n = 2, 2, 128, 64
     U_k, U_v, q, k, v = make_case(B_, H, d, [64] * H, [64] * H, n, BF16, seed_cfg=144)
     lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
     lay.append_kv(k, v)
-    lay.set_rope(10000.0)
-    with pytest.raises(B.EigenAttnError) as e:    # rotary embedding: positions per sequence are not built
-        lay.set_lens([n, 5])
-    assert e.value.status == B.EA_ERR_UNSUPPORTED
-    lay.set_rope(0.0)
     lay.set_lens([n, 5])
     for call in (lambda: lay.quant_attach(4, 32), lambda: lay.set_lens([n, -1]), lambda: lay.set_lens([n + 1, 1])):
         with pytest.raises(B.EigenAttnError):
@@ -180,4 +176,34 @@ def test_unequal_lengths_are_refused_where_they_are_not_built(B):
     with pytest.raises(B.EigenAttnError) as e:    # and with a quantised cache attached, lengths stay equal
         lay.set_lens([n, 5])
     assert e.value.status == B.EA_ERR_UNSUPPORTED
+    lay.poll_status()
+
+
+@pytest.mark.parametrize("interleaved,lens", [(False, [1037, 1, 300]), (True, [129, 1037, 128])])
+def test_rope_decode_with_unequal_lengths(B, interleaved, lens):
+    """Section 4.3 per sequence: row j of a sequence sits at position j, its query at its own last position."""
+    B_, H, d, n = len(lens), 2, 128, 1037
+    rk, rv = [80, 48], [64, 80]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + 2, BF16, seed_cfg=145, T_q=3)
+    lay = B.EigenAttnLayer(B_, H, d, n + 2, BF16, U_k, U_v)
+    lay.set_rope(10000.0, interleaved)
+    lay.append_kv(k[:, :n], v[:, :n])
+    lay.set_lens(lens)
+    refs = []
+    for b, nb in enumerate(lens):
+        r = orc.LayerOracle(1, H, d, U_k, U_v, storage=storage_model(BF16),       # few rows: model the 16-bit cache
+                            rope={"base": 10000.0, "interleaved": interleaved})
+        r.append_kv(to_np(k[b:b + 1, :nb]), to_np(v[b:b + 1, :nb]))
+        refs.append(r)
+    expect = lambda qq: np.concatenate([r.decode_dense(to_np(qq[b:b + 1])).reshape(1, 1, H, d)
+                                        for b, r in enumerate(refs)], axis=0)
+    for ctas in (0, 1, 300):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode(q[:, :1]), expect(q[:, :1]), BF16, f"rope decode ctas={ctas}")
+    for s_ in range(2):                           # each sequence's new row at its own next position
+        kn, vn = k[:, n + s_:n + s_ + 1], v[:, n + s_:n + s_ + 1]
+        o = lay.decode_step(q[:, s_ + 1:s_ + 2], kn, vn)
+        for b, r in enumerate(refs):
+            r.append_kv(to_np(kn[b:b + 1]), to_np(vn[b:b + 1]))
+        assert_close(o, expect(q[:, s_ + 1:s_ + 2]), BF16, f"rope step {s_}")
     lay.poll_status()
