@@ -207,3 +207,31 @@ def test_rope_decode_with_unequal_lengths(B, interleaved, lens):
             r.append_kv(to_np(kn[b:b + 1]), to_np(vn[b:b + 1]))
         assert_close(o, expect(q[:, s_ + 1:s_ + 2]), BF16, f"rope step {s_}")
     lay.poll_status()
+
+
+def test_padded_prompt_batch_then_generation_at_the_true_lengths(B):
+    """The serving pattern: prompts of different lengths are padded to a common T and prefilled in one call (causality
+    keeps the padding out of every real token's result), then the layer is told the true lengths and generation
+    appends behind each prompt's own end, over the padding rows."""
+    B_, H, d, T = 3, 2, 128, 300
+    rk, rv = [80, 48], [64, 80]
+    lens = [300, 131, 7]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + 2, BF16, seed_cfg=146, T_q=T + 2)
+    lay = B.EigenAttnLayer(B_, H, d, T + 2, BF16, U_k, U_v, max_prefill_tokens=T)
+    out = lay.prefill(q[:, :T], k[:, :T], v[:, :T])
+    refs = []
+    for b, nb in enumerate(lens):
+        r = oracle_layer(1, H, d, U_k, U_v)
+        expect = r.prefill_dense(to_np(q[b:b + 1, :nb]), to_np(k[b:b + 1, :nb]), to_np(v[b:b + 1, :nb]))
+        assert_close(out[b:b + 1, :nb], expect, BF16, f"prompt of sequence {b}")
+        refs.append(r)
+    lay.set_lens(lens)
+    for s_ in range(2):
+        qn, kn, vn = (x[:, T + s_:T + s_ + 1] for x in (q, k, v))
+        o = lay.decode_step(qn, kn, vn)
+        for b, r in enumerate(refs):
+            r.append_kv(to_np(kn[b:b + 1]), to_np(vn[b:b + 1]))
+        expect = np.concatenate([r.decode_dense(to_np(qn[b:b + 1])).reshape(1, 1, H, d) for b, r in enumerate(refs)], axis=0)
+        assert_close(o, expect, BF16, f"generated token {s_}")
+    assert lay.lens() == [x + 2 for x in lens]
+    lay.poll_status()
