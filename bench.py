@@ -463,7 +463,14 @@ def prefill_measure(wl, device, steps, warmup, impl=0):
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peak = float(json.load(open(peaks_path))["bf16_tflops"]) if os.path.exists(peaks_path) else 1590.0
     tf = flop / (kern * 1e-3) / 1e12
+    # the projection kernel (HBM-bound): q, k, v in, cache rows and Q' out, against the measured copy bandwidth
+    es = 2 if wl.dtype == "bf16" else 4
+    proj_bytes = wl.batch * T * (3 * wl.n_heads * wl.d_head + sum(3 * r for r in ranks)) * es
+    proj_ms = ms - kern
+    hbm, _ = measured_peaks()
     return {"workload": wl.name, "ms_per_call": ms, "attention_kernel_ms": kern, "attention_tflops": tf,
+            "projection_ms": proj_ms, "projection_gbs": proj_bytes / (proj_ms * 1e-3) / 1e9,
+            "projection_frac_of_hbm": proj_bytes / (proj_ms * 1e-3) / 1e9 / hbm,
             "bound": "tensor", "peak_tflops": peak, "frac": tf / peak,
             "peak_source": "measured burst" if os.path.exists(peaks_path) else "fallback",
             "flop_counted": "causal Q'K'^T + PV' (projections and lift excluded)"}
