@@ -553,9 +553,21 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
   if (p.deficit != nullptr) {         // unequal lengths: tiles per sequence, then their exclusive prefix
     for (int b = tid; b < p.B; b += kDecodeThreads) fx->pre[b + 1] = seq_tiles(p, seq_rows(p, b));
     __syncthreads();
-    if (tid == 0) {
-      fx->pre[0] = 0;
-      for (int b = 0; b < p.B; ++b) fx->pre[b + 1] += fx->pre[b];
+    if (warp == 0) {                  // inclusive scan, 32 sequences per step
+      int carry = 0;
+      for (int base = 0; base < p.B; base += 32) {
+        const int b = base + lane;
+        int v = b < p.B ? fx->pre[b + 1] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, v, d);
+          if (lane >= d) v += up;
+        }
+        if (b < p.B) fx->pre[b + 1] = v + carry;
+        carry += __shfl_sync(0xffffffffu, v, 31);
+      }
+      if (lane == 0) fx->pre[0] = 0;
+      __syncwarp();                   // thread 0 reads the prefix right below
     }
   }
   if (tid == 0) {

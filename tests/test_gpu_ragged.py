@@ -235,3 +235,21 @@ def test_padded_prompt_batch_then_generation_at_the_true_lengths(B):
         assert_close(o, expect, BF16, f"generated token {s_}")
     assert lay.lens() == [x + 2 for x in lens]
     lay.poll_status()
+
+
+def test_many_sequences_of_unequal_lengths(B):
+    """More sequences than one step of the tile-count prefix handles (32): lengths 1 .. n in a fixed shuffle."""
+    B_, H, d, n = 70, 1, 64, 200
+    lens = [1 + (37 * b) % n for b in range(B_)]
+    U_k, U_v, q, k, v = make_case(B_, H, d, [32], [24], n + 1, FP32, seed_cfg=147, T_q=2)
+    lay = B.EigenAttnLayer(B_, H, d, n + 1, FP32, U_k, U_v)
+    lay.append_kv(k[:, :n], v[:, :n])
+    lay.set_lens(lens)
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens)
+    for ctas in (0, 3):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode(q[:, :1]), ref.decode(q[:, :1]), FP32, f"decode ctas={ctas}")
+    o = lay.decode_step(q[:, 1:2], k[:, n:], v[:, n:])
+    ref.append(k[:, n:], v[:, n:])
+    assert_close(o, ref.decode(q[:, 1:2]), FP32, "decode_step")
+    lay.poll_status()
