@@ -32,9 +32,9 @@ METRIC = "rank-r decode attention KV GB/s (B=16, n=32k, 7B layer; us/step alongs
 UNIT = "GB/s"
 FILL_CHUNK = 1024          # tokens per append call while filling the cache
 # DRAM bytes moved per algorithmic byte by decode_splitkv_kernel, from the ncu capture summarised in
-# profiles/decode_splitkv_llama2_7b_b2_n32k_full.md (B = 2 case: 680.4 MB for 671.1 MB; traffic grows in
+# profiles/decode_splitkv_llama2_7b_b2_n32k_full.md (B = 2 case: 680.8 MB for 671.1 MB; traffic grows in
 # proportion to the number of units).  Set to None whenever that kernel changes after the capture.
-DECODE_TRAFFIC_RATIO = 681.43 / 671.11
+DECODE_TRAFFIC_RATIO = 680.81 / 671.11
 
 
 def measured_peaks():
