@@ -227,7 +227,8 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
  * With a rotary embedding each sequence's query sits at its own last position.  Not available
  * (EA_ERR_UNSUPPORTED) with a quantised cache attached; while lengths differ,
  * prefill and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
- * (asynchronous; the array may be reused when the call returns). */
+ * (asynchronous; the array may be reused when the call returns), so the calls that follow must run on that
+ * stream or be ordered after it. */
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);
 ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens);
 
