@@ -31,10 +31,10 @@ from paper_2408_05646_b200 import synth
 METRIC = "rank-r decode attention KV GB/s (B=16, n=32k, 7B layer; us/step alongside)"
 UNIT = "GB/s"
 FILL_CHUNK = 1024          # tokens per append call while filling the cache
-# DRAM bytes moved per algorithmic byte by decode_splitkv_kernel, from the ncu capture summarised in
-# profiles/decode_splitkv_llama2_7b_b2_n32k_full.md (B = 2 case: 680.8 MB for 671.1 MB; traffic grows in
-# proportion to the number of units).  Set to None whenever that kernel changes after the capture.
-DECODE_TRAFFIC_RATIO = 680.81 / 671.11
+# DRAM bytes moved per algorithmic byte by decode_splitkv_kernel, from an ncu capture of the B = 2 case of the
+# headline workload (dram__bytes_read.sum + dram__bytes_write.sum = 680.8 MB for 671.1 MB of K'/V' rows; traffic
+# grows in proportion to the number of units).  None whenever that kernel has changed since the capture.
+DECODE_TRAFFIC_RATIO = None
 
 
 def measured_peaks():
@@ -42,7 +42,9 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, torch copy read+write)"
+        return float(d["hbm_gbs"]), ("measured (MEASURED_PEAKS.json hbm_gbs): the rate of a device copy counting read + write "
+                                     "bytes, not a read ceiling; a read-only stream can exceed it, so frac may read above 1. "
+                                     "The number to hold against the >= 70 % of 8 TB/s target is frac_of_nominal_8TBs")
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
@@ -828,6 +830,11 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        raise SystemExit(f"bench.py --gpus {args.gpus} must run as {args.gpus} rank(s), one per GPU, but WORLD_SIZE is "
+                         f"{world}: launch it with `python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} "
+                         f"--master-addr 127.0.0.1 --master-port <port> bench.py --gpus {args.gpus} ...`")
     if args.workload in synth.GQA_GROUP:
         return run_gqa(args, wl)
     if args.quant:

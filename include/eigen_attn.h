@@ -25,7 +25,8 @@
  *   - Every function returns an ea_status.  Argument, shape and capacity errors are found on the
  *     host before anything is launched and leave the handle unchanged.  Kernels never trap: a wait that
  *     exceeds its bound records EA_ERR_TIMEOUT in a device status word read by eigen_attn_poll_status.
- *   - A handle is not thread-safe.  All sequences of a handle share one length (`len`).
+ *   - A handle is not thread-safe.  The sequences of a handle share one length (`len`) unless
+ *     eigen_attn_set_lens is in effect; `len` is then the length of the longest sequence.
  */
 #ifndef EIGEN_ATTN_H_
 #define EIGEN_ATTN_H_
@@ -109,17 +110,22 @@ ea_status eigen_attn_decode(eigen_attn_t h, const void* d_q, int64_t stride_b_q,
  * It is meant for callers that must not obtain device memory while they run -- e.g. a plugin inside
  * an inference engine whose memory plan is frozen, a real-time loop where cudaMalloc's device-wide
  * synchronisation is unacceptable, or a process whose memory pool is already handed out in full --
- * and that therefore want the decode call itself to depend on no scratch they have to provide.
+ * and that therefore cannot size a partials area for a plan they do not know in advance.
+ *   - Only the partials move.  The call still reads the head table and the bases in the workspace given
+ *     at create and, with EA_OPT_DECODE_FUSED = 1 (the default), counts arrivals in that workspace's
+ *     per-unit counters and reports through its status word, exactly as eigen_attn_decode does.
  *   - Limit: (batch * n_heads + decode CTAs) * (4 + widest rp_v) <= 270336 floats (2048 slots of 132
  *     floats, 1.03 MiB, resident on every GPU that loads the library until the process exits).
  *     Larger layers get EA_ERR_CAPACITY and a message; use eigen_attn_decode for them.
- *   - The first call on each device looks up the array's device address (a CUDA runtime query, no
- *     allocation); make that first call outside any stream capture.  The call itself never calls
- *     cudaMalloc/cudaFree or any allocating routine.
+ *   - Every call asks the CUDA runtime for the array's device address on the current device (a lookup,
+ *     no allocation; correct again after a cudaDeviceReset).  The first call on a device also makes the
+ *     runtime load the library image there: make that first call outside any stream capture.  The call
+ *     itself never calls cudaMalloc/cudaFree or any allocating routine.
  *   - All handles and all calls on a device share the one array, and it keeps whatever the previous
  *     call left.  Nothing in it has to start at zero: every slot the combine step reads is written
  *     earlier in the same call.  Two calls that may overlap on the GPU (different streams, or several
- *     host threads) race on the array and give undefined results; serialise them. */
+ *     host threads) race on the array and give undefined results; serialise them.  A decode and a
+ *     decode_static of the SAME handle that overlap also race on the handle's arrival counters. */
 ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                    int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 
@@ -257,10 +263,16 @@ typedef enum {
                                  warp-specialised one)                                                     */
   EA_OPT_DECODE_FUSED = 5,    /* 1 (default): a decode step is one launch (append row, attend, merge the
                                  splits, lift); 0: separate append / attention / merge launches           */
-  EA_OPT_PREFILL_PROJECT = 6  /* tensor-core projections of prefill: 0 = automatic (the persistent kernel that
+  EA_OPT_PREFILL_PROJECT = 6, /* tensor-core projections of prefill: 0 = automatic (the persistent kernel that
                                  streams token tiles by TMA when d_head % 64 == 0 and T >= 128), 1 = always
                                  one CTA per tile of 128 tokens, n >= 2 = the persistent kernel with at most
                                  n CTAs                                                                    */
+  EA_OPT_TEST_WAIT_GIVES_UP = 7 /* failure-path test hook.  1 arms it for the NEXT eigen_attn_decode /
+                                 _decode_step / _decode_static launch only: one warp of one CTA treats its
+                                 first wait for a tile as having exceeded the bound.  The launch then ends the
+                                 way a real timeout ends it (the CTA stops computing, the producer waits for
+                                 its copies in flight, the kernel returns), the call's output is undefined and
+                                 eigen_attn_poll_status reports EA_ERR_TIMEOUT once.  Nothing hangs or faults. */
 } ea_option;
 ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value);
 

@@ -24,6 +24,7 @@ EA_Q_PREPROJECTED, EA_OUT_LOWRANK, EA_KV_PREPROJECTED = 0x1, 0x2, 0x4
 EA_OPT_DECODE_CTAS, EA_OPT_DECODE_TILE_ROWS, EA_OPT_DECODE_STAGES, EA_OPT_PREFILL_IMPL = 1, 2, 3, 4
 EA_OPT_DECODE_FUSED = 5
 EA_OPT_PREFILL_PROJECT = 6
+EA_OPT_TEST_WAIT_GIVES_UP = 7
 
 STATUS_NAMES = {0: "EA_OK", -1: "EA_ERR_INVALID_ARG", -2: "EA_ERR_SHAPE", -3: "EA_ERR_CAPACITY",
                 -4: "EA_ERR_UNSUPPORTED", -5: "EA_ERR_CUDA", -6: "EA_ERR_TIMEOUT",
@@ -98,6 +99,14 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
 lib = load_library()
 
 
+def device_alloc(nbytes: int, device: torch.device) -> torch.Tensor:
+    """Every device buffer this module hands to the library (cache, workspace, quantised buffer, outputs it
+    creates itself) comes from this function: a flat uint8 tensor whose address is a multiple of 256.  It is a
+    module attribute so that a caller can substitute its own allocator, e.g. one that surrounds each buffer with
+    guard regions."""
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
@@ -159,8 +168,8 @@ class EigenAttnLayer:
         if st != EA_OK:
             raise EigenAttnError(st, "eigen_attn_cache_bytes")
         with torch.cuda.device(self.device):
-            self.cache = torch.empty(cb.value, dtype=torch.uint8, device=self.device)
-            self.workspace = torch.empty(wb.value, dtype=torch.uint8, device=self.device)
+            self.cache = device_alloc(cb.value, self.device)
+            self.workspace = device_alloc(wb.value, self.device)
             handle = _vp(0)
             st = lib.eigen_attn_create(ctypes.byref(desc), self.cache.data_ptr(), cb.value,
                                        self.workspace.data_ptr(), wb.value, _stream_ptr(stream),
@@ -175,6 +184,13 @@ class EigenAttnLayer:
         self.offs_k, self.offs_v = list(offs_k), list(offs_v)
 
     # -- plumbing
+    def _new_out(self, *shape) -> torch.Tensor:
+        es = 2 if self.torch_dtype == torch.bfloat16 else 4
+        n = 1
+        for d in shape:
+            n *= int(d)
+        return device_alloc(n * es, self.device).view(self.torch_dtype).view(*shape)
+
     def _check(self, st: int, where: str) -> None:
         if st != EA_OK:
             raise EigenAttnError(st, where, lib.eigen_attn_last_error(self.handle).decode())
@@ -227,12 +243,12 @@ class EigenAttnLayer:
         if out_lowrank:
             flags |= EA_OUT_LOWRANK
             if out is None:
-                out = torch.empty((self.B, 1, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
+                out = self._new_out(self.B, 1, self.offs_v[-1])
             assert out.is_contiguous() and out.dtype == self.torch_dtype
             sbo = self.offs_v[-1]
         else:
             if out is None:
-                out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+                out = self._new_out(self.B, 1, self.H, self.d_head)
             _, _, sbo, _ = self._tok(out, 1)
         fn = _fn if _fn is not None else lib.eigen_attn_decode
         self._check(fn(self.handle, pq, sbq, out.data_ptr(), sbo, flags, _stream_ptr(stream)), _name)
@@ -247,7 +263,7 @@ class EigenAttnLayer:
     def quant_attach(self, bits: int, group: int, stream=None) -> torch.Tensor:
         """Allocates the quantised buffer (a torch byte tensor kept on the layer) and attaches it."""
         nbytes = self.quant_bytes(bits, group)
-        self.qcache = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+        self.qcache = device_alloc(nbytes, self.device).zero_()
         self.q_group = int(group)
         self._check(lib.eigen_attn_quant_attach(self.handle, int(bits), int(group), self.qcache.data_ptr(), nbytes,
                                                 _stream_ptr(stream)), "eigen_attn_quant_attach")
@@ -286,7 +302,7 @@ class EigenAttnLayer:
         GPU share that array and must be serialised."""
         pq, _, sbq, _ = self._tok(q, 1)
         if out is None:
-            out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+            out = self._new_out(self.B, 1, self.H, self.d_head)
         _, _, sbo, _ = self._tok(out, 1)
         self._check(lib.eigen_attn_decode_static(self.handle, pq, sbq, out.data_ptr(), sbo, 0,
                                                  _stream_ptr(stream)), "eigen_attn_decode_static")
@@ -301,7 +317,7 @@ class EigenAttnLayer:
             pk, _, sbk, _ = self._tok(k, 1)
             pv, _, sbv, _ = self._tok(v, 1)
         if out is None:
-            out = torch.empty((self.B, 1, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+            out = self._new_out(self.B, 1, self.H, self.d_head)
         po, _, sbo, _ = self._tok(out, 1)
         self._check(lib.eigen_attn_decode_step(self.handle, pq, sbq, pk, pv, sbk, po, sbo, 0, _stream_ptr(stream)),
                     "eigen_attn_decode_step")
@@ -326,12 +342,12 @@ class EigenAttnLayer:
         if out_lowrank:
             flags = EA_OUT_LOWRANK
             if out is None:
-                out = torch.empty((self.B, T, self.offs_v[-1]), dtype=self.torch_dtype, device=self.device)
+                out = self._new_out(self.B, T, self.offs_v[-1])
             assert out.is_contiguous()
             po, sbo, sto = out.data_ptr(), T * self.offs_v[-1], self.offs_v[-1]
         else:
             if out is None:
-                out = torch.empty((self.B, T, self.H, self.d_head), dtype=self.torch_dtype, device=self.device)
+                out = self._new_out(self.B, T, self.H, self.d_head)
             po, _, sbo, sto = self._tok(out, T)
         self._check(lib.eigen_attn_prefill(self.handle, pq, pk, pv, T, sb, stt, po, sbo, sto, flags, _stream_ptr(stream)),
                     "eigen_attn_prefill")
@@ -373,7 +389,7 @@ class EigenAttnLayer:
         assert q.shape == (self.B, 1, self.H * group, self.d_head) and q.dtype == self.torch_dtype
         assert q.stride(3) == 1 and q.stride(2) == self.d_head
         if out is None:
-            out = torch.empty((self.B, 1, self.H * group, self.d_head), dtype=self.torch_dtype, device=self.device)
+            out = self._new_out(self.B, 1, self.H * group, self.d_head)
         assert out.stride(3) == 1 and out.stride(2) == self.d_head
         self._check(lib.eigen_attn_decode_gqa(self.handle, q.data_ptr(), q.stride(0), int(group), out.data_ptr(),
                                               out.stride(0), _stream_ptr(stream)), "eigen_attn_decode_gqa")

@@ -197,6 +197,7 @@ struct eigen_attn {
   bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
   int rope_interleaved = 0;
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1, opt_project = 0;
+  int64_t opt_give_up = 0;   // EA_OPT_TEST_WAIT_GIVES_UP: armed for the next split-KV decode launch
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   // quantised copy of the cache (Section 5.3), attached by the caller
@@ -369,6 +370,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.w_total = w_total;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
+  p.give_up_once = h->opt_give_up ? 1 : 0;
   plan->grid = grid;
   plan->smem = static_cast<size_t>(fixed) + static_cast<size_t>(ring_bytes);
 
@@ -386,6 +388,7 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
   if (events && h->ev_start) cudaEventRecord(h->ev_start, s);
   cudaError_t e = ea::launch_decode(plan.p, h->desc.dtype, plan.grid, plan.smem, s, &h->launches);
   if (events && h->ev_stop) cudaEventRecord(h->ev_stop, s);
+  h->opt_give_up = 0;                 // one launch only
   if (e != cudaSuccess) return cuda_fail(h, e, who);
   if (plan.p.counters == nullptr) {   // the merge + lift as its own launch
     e = ea::launch_combine(plan.c, h->desc.dtype, s, &h->launches);
@@ -1184,6 +1187,10 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
     case EA_OPT_PREFILL_PROJECT:
       if (value < 0 || value > 65535) return fail(h, EA_ERR_INVALID_ARG, "PREFILL_PROJECT %lld", static_cast<long long>(value));
       h->opt_project = value;
+      return EA_OK;
+    case EA_OPT_TEST_WAIT_GIVES_UP:
+      if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "TEST_WAIT_GIVES_UP %lld", static_cast<long long>(value));
+      h->opt_give_up = value;
       return EA_OK;
     default:
       return fail(h, EA_ERR_INVALID_ARG, "unknown option %d", option);

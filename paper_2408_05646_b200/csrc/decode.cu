@@ -76,13 +76,17 @@ __device__ __forceinline__ uint64_t global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false (and the status word set) if the phase did not complete within the bound.
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* status) {
+// Bounded wait: false (and the status word set) if the phase did not complete within the bound.  With
+// `abort_flag` the wait also ends (false) once another role of the CTA has given up: after that nobody
+// may be left to complete the phase.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* status,
+                                          const volatile int* abort_flag = nullptr) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
+    if (abort_flag != nullptr && *abort_flag != 0) return false;
     if (global_ns() - t0 > kWaitBoundNs) {
       atomicExch(status, kStatusTimeout);
       return false;
@@ -323,7 +327,14 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     ring_state.advance();
     // warp-uniform decisions: the row code below shuffles across the whole warp
     if (__any_sync(0xffffffffu, *abort_flag != 0)) continue;
-    if (__any_sync(0xffffffffu, !mbar_wait(&fx->full[stage], parity, p.status))) {
+    bool landed = mbar_wait(&fx->full[stage], parity, p.status);
+    if (p.give_up_once != 0 && blockIdx.x == 0 && warp == 0) {
+      // test hook: behave exactly as if this wait had exceeded its bound (the copy itself still lands
+      // and the producer waits for it before the CTA exits)
+      if (lane == 0) atomicExch(p.status, kStatusTimeout);
+      landed = false;
+    }
+    if (__any_sync(0xffffffffu, !landed)) {
       *abort_flag = 1;
       continue;
     }
@@ -605,7 +616,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
           // ring must have been released before the first copy into the new layout.
           for (int s2 = 0; s2 < kMaxStages && ok; ++s2)
             if (rg.filled & (1u << s2)) {
-              ok = mbar_wait(&fx->empty[s2], (rg.empty_bits >> s2) & 1u, p.status);
+              ok = mbar_wait(&fx->empty[s2], (rg.empty_bits >> s2) & 1u, p.status, abort_flag);
               rg.empty_bits ^= 1u << s2;
               rg.filled &= ~(1u << s2);
             }
@@ -623,7 +634,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
           const int st = rg.stage;
           const uint32_t bit = 1u << st;
           if (rg.filled & bit) {          // the slot's previous tile must have been released
-            if (!mbar_wait(&fx->empty[st], (rg.empty_bits >> st) & 1u, p.status)) {
+            if (!mbar_wait(&fx->empty[st], (rg.empty_bits >> st) & 1u, p.status, abort_flag)) {
               *abort_flag = 1;
               ok = false;
               break;
@@ -758,23 +769,17 @@ __global__ void __launch_bounds__(128) combine_lift_kernel(const CombineParams p
 // for the device object; static_partials() asks the runtime for the real device address.
 static __device__ __align__(256) float g_static_partials[kStaticPartialFloats];
 
-constexpr int kMaxDevices = 64;
-float* g_static_partials_addr[kMaxDevices] = {};
-
 }  // namespace
 
+// The address is asked for on every call and never kept: the query is a host-side table lookup once the
+// library image is loaded on the device (the first call per device loads it, which is why that call belongs
+// outside stream capture), it allocates nothing, it needs no lock between host threads, and it stays right
+// after a cudaDeviceReset, which would leave a remembered address dangling.
 cudaError_t static_partials(float** ptr) {
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  float* p = nullptr;
+  const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials);   // current device
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (!g_static_partials_addr[dev]) {
-    float* p = nullptr;
-    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials);   // `dev` is current
-    if (e != cudaSuccess) return e;
-    g_static_partials_addr[dev] = p;
-  }
-  *ptr = g_static_partials_addr[dev];
+  *ptr = p;
   return cudaSuccess;
 }
 

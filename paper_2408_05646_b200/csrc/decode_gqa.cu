@@ -374,13 +374,9 @@ size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
 
 template <int GP>
 cudaError_t launch_gqa_variant(const GqaDecodeParams& p, size_t smem, cudaStream_t s) {
-  static size_t configured = 0;
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel<GP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[kMaxDevices] = {};
+  const cudaError_t ec = ensure_dynamic_smem(decode_gqa_kernel<GP>, smem, configured);
+  if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, p.splits);
   decode_gqa_kernel<GP><<<grid, kGqaThreads, smem, s>>>(p);
   return cudaGetLastError();

@@ -369,15 +369,10 @@ size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(decode_rope_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[2][kMaxDevices] = {};
+  const cudaError_t ec = p.interleaved ? ensure_dynamic_smem(decode_rope_kernel<true>, smem, configured[1])
+                                       : ensure_dynamic_smem(decode_rope_kernel<false>, smem, configured[0]);
+  if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, p.splits);
   if (p.interleaved) decode_rope_kernel<true><<<grid, kThreads, smem, s>>>(p);
   else decode_rope_kernel<false><<<grid, kThreads, smem, s>>>(p);

@@ -59,6 +59,7 @@ struct DecodeParams {
   int64_t w_total;          // nt_total * sum_h (rp_k + rp_v)
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
+  int32_t give_up_once;     // test hook: warp 0 of CTA 0 reports its first wait for a tile as run out
 };
 
 struct CombineParams {
@@ -245,9 +246,25 @@ cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, int min_rp, si
                                 uint64_t* launches);   // min_rp: narrowest padded rank over heads and K/V
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
-// library's own partials array on the current device.  Resolves the address on first use per device.
+// library's own partials array on the current device (queried from the runtime on every call).
 constexpr size_t kStaticPartialFloats = 2048 * 132;
 cudaError_t static_partials(float** ptr);
+
+// Opts `kernel` in to `smem` bytes of dynamic shared memory on the CURRENT device.  The attribute belongs to
+// the (kernel, device) pair, so every launcher keeps its own table `done` of the largest size set so far,
+// indexed by device ordinal; a process that drives several GPUs configures each of them once.
+constexpr int kMaxDevices = 64;
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t smem, size_t (&done)[kMaxDevices]) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < kMaxDevices;
+  if (tracked && smem <= done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e == cudaSuccess && tracked) done[dev] = smem;
+  return e;
+}
 
 size_t decode_fixed_smem_bytes();         // shared memory the decode kernel needs besides the ring
 cudaError_t decode_configure(int dtype);  // opt in to large dynamic shared memory (once per device)

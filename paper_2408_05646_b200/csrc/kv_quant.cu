@@ -405,13 +405,9 @@ __global__ void __launch_bounds__(128) quant_combine_kernel(const QuantParams p)
 
 template <int NW, int MINB, int G, bool FULL>
 cudaError_t launch_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
-  static size_t configured = 0;
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_quant_kernel<NW, MINB, G, FULL>,
-                                               cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[kMaxDevices] = {};
+  const cudaError_t ec = ensure_dynamic_smem(decode_quant_kernel<NW, MINB, G, FULL>, smem, configured);
+  if (ec != cudaSuccess) return ec;
   decode_quant_kernel<NW, MINB, G, FULL><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
   return cudaGetLastError();
 }

@@ -285,13 +285,9 @@ size_t prefill_tc_smem_bytes(int max_rp_k, int max_rp_v) {
 cudaError_t launch_prefill_tc(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s,
                               uint64_t* launches) {
   const size_t smem = prefill_tc_smem_bytes(max_rp_k, max_rp_v);
-  static size_t configured = 0;     // largest dynamic shared-memory size opted into so far
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[kMaxDevices] = {};
+  const cudaError_t ec = ensure_dynamic_smem(prefill_tc_kernel, smem, configured);
+  if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, (p.T + kTile - 1) / kTile);
   prefill_tc_kernel<<<grid, kThreads, smem, s>>>(p);
   ++*launches;

@@ -526,13 +526,9 @@ int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_by
 }
 
 cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, cudaStream_t s, uint64_t* launches) {
-  static size_t configured = 0;     // largest dynamic shared-memory size opted into so far
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(prefill_tc_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[kMaxDevices] = {};
+  const cudaError_t ec = ensure_dynamic_smem(prefill_tc_ws_kernel, smem, configured);
+  if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, (p.T + 2 * kTile - 1) / (2 * kTile));
   prefill_tc_ws_kernel<<<grid, kWsThreads, smem, s>>>(p, stages);
   ++*launches;

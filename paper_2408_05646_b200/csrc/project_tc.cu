@@ -118,13 +118,9 @@ __global__ void __launch_bounds__(kThreads) project_tc_kernel(const ProjectTcPar
 cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches) {
   const int rp16 = (max_rp + 15) & ~15;
   const size_t smem = 1024 + static_cast<size_t>(kTile) * p.d_head * 2 + 2ull * rp16 * p.d_head * 2;
-  static size_t configured = 0;     // largest dynamic shared-memory size opted into so far
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  static size_t configured[kMaxDevices] = {};
+  const cudaError_t ec = ensure_dynamic_smem(project_tc_kernel, smem, configured);
+  if (ec != cudaSuccess) return ec;
   dim3 grid((p.B * p.T + kTile - 1) / kTile, p.H, 3);
   project_tc_kernel<<<grid, kThreads, smem, s>>>(p);
   ++*launches;

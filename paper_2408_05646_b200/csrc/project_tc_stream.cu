@@ -321,13 +321,9 @@ cudaError_t launch_project_tc_stream(const ProjectTcParams& p, const void* maps_
   const size_t smem = project_tc_stream_smem(max_rp, p.d_head, &stages);
   if (stages < 2) return cudaErrorInvalidConfiguration;
   auto kernel = p.d_head == 128 ? project_tc_stream_kernel<8> : project_tc_stream_kernel<4>;
-  static size_t configured[2] = {0, 0};   // largest dynamic shared-memory size opted into so far, per instance
-  size_t& conf = configured[p.d_head == 128 ? 1 : 0];
-  if (smem > conf) {
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    conf = smem;
-  }
+  static size_t configured[2][kMaxDevices] = {};   // per kernel instance
+  const cudaError_t ec = ensure_dynamic_smem(kernel, smem, configured[p.d_head == 128 ? 1 : 0]);
+  if (ec != cudaSuccess) return ec;
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(maps_qkv);
   const int64_t total = 3ll * p.H * p.B * ((p.T + kTile - 1) / kTile);
   const int grid = static_cast<int>(total < sm_count ? total : sm_count);

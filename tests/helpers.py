@@ -14,13 +14,39 @@ BF16_MAX_ABS, BF16_MEAN_ABS = 2e-2, 2e-3
 FP32_REL = 1e-5
 
 
-def assert_close(got: torch.Tensor, ref: np.ndarray, dtype: torch.dtype, what: str = "", fp32_rel: float = FP32_REL):
+class Expect:
+    """Expected values from an OraclePair: `kept` from the oracle layer whose storage hook rounds the cached rows
+    to the 16-bit cache format, `plain` from the layer that keeps fp64 rows."""
+    def __init__(self, kept: np.ndarray, plain: np.ndarray):
+        self.kept, self.plain = kept, plain
+
+
+# (what, max-abs against the plain fp64 oracle, max-abs against the oracle with the storage hook): filled by
+# assert_close whenever a test uses the hook; tests/conftest.py attaches it to the test's report.
+PLAIN_LOG = []
+
+
+def assert_close(got: torch.Tensor, ref, dtype: torch.dtype, what: str = "", fp32_rel: float = FP32_REL,
+                 plain_within: bool = False):
+    """Tolerance check against the oracle.  `ref` is an array, or an Expect: then the check is against the layer
+    with the storage hook, the distance to the plain fp64 oracle is logged and shown in every failure message, and
+    with plain_within it must meet the same tolerance too."""
+    note = ""
+    if isinstance(ref, Expect):
+        gp = got.detach().double().cpu().numpy().reshape(ref.plain.shape)
+        e_plain = float(np.abs(gp - ref.plain).max())
+        e_kept = float(np.abs(gp - ref.kept).max())
+        PLAIN_LOG.append((what, e_plain, e_kept))
+        note = f" [max-abs against the plain fp64 oracle {e_plain:.3e}, with the storage hook {e_kept:.3e}]"
+        if plain_within:
+            assert_close(got, ref.plain, dtype, what + " (plain fp64 oracle)", fp32_rel)
+        ref = ref.kept
     g = got.detach().double().cpu().numpy().reshape(ref.shape)
     assert np.isfinite(g).all(), f"{what}: non-finite output"
     diff = np.abs(g - ref)
     if dtype == torch.bfloat16:
-        assert diff.max() <= BF16_MAX_ABS, f"{what}: max-abs {diff.max():.3e}"
-        assert diff.mean() <= BF16_MEAN_ABS, f"{what}: mean-abs {diff.mean():.3e}"
+        assert diff.max() <= BF16_MAX_ABS, f"{what}: max-abs {diff.max():.3e}{note}"
+        assert diff.mean() <= BF16_MEAN_ABS, f"{what}: mean-abs {diff.mean():.3e}{note}"
     else:
         scale = max(np.abs(ref).max(), 1e-30)
         assert diff.max() / scale <= fp32_rel, f"{what}: rel max {diff.max() / scale:.3e}"
@@ -46,6 +72,29 @@ def make_case(B, H, d_head, ranks_k, ranks_v, n, dtype, seed_cfg=90, rho=16, sig
 
 def oracle_layer(B, H, d_head, U_k, U_v, tracked=None, alibi_slopes=None, storage=None):
     return orc.LayerOracle(B, H, d_head, U_k, U_v, tracked, alibi_slopes=alibi_slopes, storage=storage)
+
+
+class OraclePair:
+    """Two oracle layers that receive the same calls: `kept` rounds freshly projected rows to the cache's 16-bit
+    format (the storage hook), `plain` keeps them in fp64.  Results come back as Expect, so that every comparison
+    that leans on the hook also states how far the GPU is from the plain definition."""
+    def __init__(self, B, H, d_head, U_k, U_v, dtype, tracked=None, alibi_slopes=None, rope=None):
+        self.kept = orc.LayerOracle(B, H, d_head, U_k, U_v, tracked, alibi_slopes=alibi_slopes,
+                                    storage=storage_model(dtype), rope=rope)
+        self.plain = orc.LayerOracle(B, H, d_head, U_k, U_v, tracked, alibi_slopes=alibi_slopes, rope=rope)
+
+    def append_kv(self, k, v):
+        self.kept.append_kv(k, v)
+        self.plain.append_kv(k, v)
+
+    def decode_dense(self, q):
+        return Expect(self.kept.decode_dense(q), self.plain.decode_dense(q))
+
+    def prefill_dense(self, q, k, v):
+        return Expect(self.kept.prefill_dense(q, k, v), self.plain.prefill_dense(q, k, v))
+
+    def decode_gqa(self, q, group):
+        return Expect(self.kept.decode_gqa(q, group), self.plain.decode_gqa(q, group))
 
 
 def to_np(x: torch.Tensor) -> np.ndarray:

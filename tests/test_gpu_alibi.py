@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import assert_close, make_case, oracle_layer, storage_model, to_np
+from helpers import OraclePair, assert_close, make_case, oracle_layer, storage_model, to_np
 from paper_2408_05646_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -31,7 +31,7 @@ def test_decode_with_alibi_matches_oracle(B, dtype, H, d, rk, rv, n):
     slopes = synth.alibi_slopes(H)
     lay = B.EigenAttnLayer(B_, H, d, n + 8, dtype, U_k, U_v)
     lay.set_alibi(slopes)
-    ref = oracle_layer(B_, H, d, U_k, U_v, alibi_slopes=slopes, storage=storage_model(dtype))   # steep slopes
+    ref = OraclePair(B_, H, d, U_k, U_v, dtype, alibi_slopes=slopes)   # steep slopes: few rows carry the softmax
     lay.append_kv(k[:, :n], v[:, :n])
     ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
     tol = dict(fp32_rel=2e-5) if dtype == FP32 else {}
@@ -48,7 +48,7 @@ def test_decode_with_alibi_matches_oracle(B, dtype, H, d, rk, rv, n):
         assert_close(lay.decode(q[:, :1]), expect, dtype, f"decode ctas={ctas} fused={fused}", **tol)
     assert_close(lay.decode_static(q[:, :1]), expect, dtype, "decode_static", **tol)
     lay.set_alibi(None)                                            # back to the plain path
-    plain = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(dtype))
+    plain = OraclePair(B_, H, d, U_k, U_v, dtype)
     plain.append_kv(to_np(k[:, :n + 3]), to_np(v[:, :n + 3]))
     assert_close(lay.decode(q[:, :1]), plain.decode_dense(to_np(q[:, :1])), dtype, "bias off", **tol)
     lay.poll_status()
@@ -63,7 +63,7 @@ def test_alibi_dominates_at_long_range(B):
     lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
     lay.set_alibi(slopes)
     lay.append_kv(k, v)
-    ref = oracle_layer(B_, H, d, U_k, U_v, alibi_slopes=slopes, storage=storage_model(BF16))
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16, alibi_slopes=slopes)
     ref.append_kv(to_np(k), to_np(v))
     assert_close(lay.decode(q), ref.decode_dense(to_np(q)), BF16, "long range")
 
@@ -76,7 +76,7 @@ def test_prefill_with_alibi_matches_oracle(B, dtype, H, d, rk, rv, T):
     B_ = 2
     U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, dtype, seed_cfg=137, T_q=T)
     slopes = synth.alibi_slopes(H)
-    ref = oracle_layer(B_, H, d, U_k, U_v, alibi_slopes=slopes, storage=storage_model(dtype))
+    ref = OraclePair(B_, H, d, U_k, U_v, dtype, alibi_slopes=slopes)
     expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
     for impl in ((0, 1) if dtype == FP32 else (0, 3, 1)):          # auto, single-tile tcgen05, CUDA cores
         lay = B.EigenAttnLayer(B_, H, d, T, dtype, U_k, U_v, max_prefill_tokens=T)

@@ -55,13 +55,13 @@ def test_gqa_decode_matches_oracle(B, H, g, d, rk, rv, n):
 def test_gqa_peaked_attention_and_steps(B):
     """Sharply peaked weights (queries scaled by 6) over several appended tokens: an error in a handful of rows
     or in one query of the group shows up here."""
-    from helpers import storage_model
+    from helpers import OraclePair
     B_, H, g, d, n, steps = 2, 2, 4, 128, 300, 3
     rk, rv = [80, 48], [64, 80]
     U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n + steps, BF16, seed_cfg=163)
     lay = B.EigenAttnLayer(B_, H, d, n + steps, BF16, U_k, U_v)
     lay.append_kv(k[:, :n], v[:, :n])
-    ref = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(BF16))
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16)
     ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
     for s in range(steps):
         q = (group_queries(B_, H, g, d, 170 + s).float() * 6.0).to(BF16)

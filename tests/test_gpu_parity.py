@@ -383,10 +383,10 @@ def test_peaked_attention_over_heads_that_share_a_slot_size(B, dtype):
     B_, H, d, n = 2, 6, 128, 1037
     rk, rv = [48, 64, 80, 96, 64, 48], [96, 80, 64, 48, 80, 96]        # every head: 144 columns per row
     U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, dtype, seed_cfg=141, q_scale=6.0)
-    from helpers import storage_model
+    from helpers import OraclePair
     lay = B.EigenAttnLayer(B_, H, d, n, dtype, U_k, U_v)
     lay.append_kv(k, v)
-    ref = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(dtype))
+    ref = OraclePair(B_, H, d, U_k, U_v, dtype)
     ref.append_kv(to_np(k), to_np(v))
     expect = ref.decode_dense(to_np(q))
     tol = dict(fp32_rel=2e-4) if dtype == FP32 else {}               # scores of a few tens: see the adversarial test
@@ -402,11 +402,11 @@ def test_prefill_with_peaked_attention(B, impl):
     """Queries scaled by 3: the weights of a prompt row sit on a few keys, so an error in a few rows (a stale tile, a
     ragged tail, the diagonal mask) is not averaged away.  (Not more: the kernels keep Q' in bf16, and its rounding
     grows with the scores, about |s| * 2^-9 per score.)  All three prefill kernels, two chunks."""
-    from helpers import storage_model
+    from helpers import OraclePair
     B_, H, d, T = 2, 4, 128, 700
     rk, rv = [80, 48, 128, 64], [64, 112, 16, 80]
     U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T, BF16, seed_cfg=143, T_q=T, q_scale=3.0)
-    ref = oracle_layer(B_, H, d, U_k, U_v, storage=storage_model(BF16))
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16)
     expect = ref.prefill_dense(to_np(q), to_np(k), to_np(v))
     lay = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
     lay.set_option(B.EA_OPT_PREFILL_IMPL, impl)

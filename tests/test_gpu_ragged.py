@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import assert_close, make_case, oracle_layer, storage_model, to_np
+from helpers import Expect, assert_close, make_case, oracle_layer, storage_model, to_np
 from oracle import eigen_attention as orc
 from paper_2408_05646_b200 import synth
 
@@ -25,22 +25,27 @@ def B():
 class PerSequenceOracle:
     """One single-sequence oracle layer per sequence of the batch."""
 
-    def __init__(self, H, d, U_k, U_v, k, v, lens, alibi_slopes=None, storage=None):
+    def __init__(self, H, d, U_k, U_v, k, v, lens, alibi_slopes=None, storage=None, rope=None):
+        """With `storage` (the 16-bit cache model) a second set of layers keeps fp64 rows, and decode() returns
+        an Expect carrying both results."""
         self.H, self.d = H, d
-        self.refs = []
+        self.refs, self.plain = [], []
         for b, n in enumerate(lens):
-            r = oracle_layer(1, H, d, U_k, U_v, alibi_slopes=alibi_slopes, storage=storage)
-            if n > 0:
-                r.append_kv(to_np(k[b:b + 1, :n]), to_np(v[b:b + 1, :n]))
-            self.refs.append(r)
+            for group, st in ((self.refs, storage),) + (((self.plain, None),) if storage is not None else ()):
+                r = orc.LayerOracle(1, H, d, U_k, U_v, alibi_slopes=alibi_slopes, storage=st, rope=rope)
+                if n > 0:
+                    r.append_kv(to_np(k[b:b + 1, :n]), to_np(v[b:b + 1, :n]))
+                group.append(r)
 
     def append(self, k, v):                       # k, v: [B, T, H, d]
-        for b, r in enumerate(self.refs):
-            r.append_kv(to_np(k[b:b + 1]), to_np(v[b:b + 1]))
+        for group in (self.refs, self.plain):
+            for b, r in enumerate(group):
+                r.append_kv(to_np(k[b:b + 1]), to_np(v[b:b + 1]))
 
     def decode(self, q):                          # q: [B, 1, H, d] -> [B, 1, H, d]
-        return np.concatenate([r.decode_dense(to_np(q[b:b + 1])).reshape(1, 1, self.H, self.d)
-                               for b, r in enumerate(self.refs)], axis=0)
+        one = lambda group: np.concatenate([r.decode_dense(to_np(q[b:b + 1])).reshape(1, 1, self.H, self.d)
+                                            for b, r in enumerate(group)], axis=0)
+        return Expect(one(self.refs), one(self.plain)) if self.plain else one(self.refs)
 
 
 @pytest.mark.parametrize("dtype,d,rk,rv,n,lens", [
@@ -189,22 +194,16 @@ def test_rope_decode_with_unequal_lengths(B, interleaved, lens):
     lay.set_rope(10000.0, interleaved)
     lay.append_kv(k[:, :n], v[:, :n])
     lay.set_lens(lens)
-    refs = []
-    for b, nb in enumerate(lens):
-        r = orc.LayerOracle(1, H, d, U_k, U_v, storage=storage_model(BF16),       # few rows: model the 16-bit cache
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens, storage=storage_model(BF16),    # few rows: model the 16-bit cache
                             rope={"base": 10000.0, "interleaved": interleaved})
-        r.append_kv(to_np(k[b:b + 1, :nb]), to_np(v[b:b + 1, :nb]))
-        refs.append(r)
-    expect = lambda qq: np.concatenate([r.decode_dense(to_np(qq[b:b + 1])).reshape(1, 1, H, d)
-                                        for b, r in enumerate(refs)], axis=0)
+    expect = ref.decode
     for ctas in (0, 1, 300):
         lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
         assert_close(lay.decode(q[:, :1]), expect(q[:, :1]), BF16, f"rope decode ctas={ctas}")
     for s_ in range(2):                           # each sequence's new row at its own next position
         kn, vn = k[:, n + s_:n + s_ + 1], v[:, n + s_:n + s_ + 1]
         o = lay.decode_step(q[:, s_ + 1:s_ + 2], kn, vn)
-        for b, r in enumerate(refs):
-            r.append_kv(to_np(kn[b:b + 1]), to_np(vn[b:b + 1]))
+        ref.append(kn, vn)
         assert_close(o, expect(q[:, s_ + 1:s_ + 2]), BF16, f"rope step {s_}")
     lay.poll_status()
 

@@ -46,6 +46,29 @@ def test_rope_decode_matches_oracle(B, H, d, rk, rv, n, base, interleaved):
     lay.poll_status()
 
 
+@pytest.mark.parametrize("interleaved", [False, True])
+def test_rope_decode_with_peaked_attention(B, interleaved):
+    """Queries scaled by 4: a handful of positions carry the softmax, so one wrongly rotated or wrongly lifted row
+    (a tile boundary, the ragged tail, a stale staging buffer) is not averaged away.  Heads of unequal widths are
+    streamed one after the other; any number of CTAs per unit must agree."""
+    from helpers import OraclePair
+    B_, H, d, n = 2, 4, 128, 1037
+    rk, rv = [48, 80, 64, 112], [96, 64, 80, 32]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, BF16, seed_cfg=157, q_scale=4.0)
+    lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
+    lay.set_rope(10000.0, interleaved)
+    lay.append_kv(k, v)
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16, rope={"base": 10000.0, "interleaved": interleaved})
+    ref.append_kv(to_np(k), to_np(v))
+    expect = ref.decode_dense(to_np(q))
+    weights_on_few_rows = np.abs(expect.plain).max() > 0.5          # a diffuse average of ~1000 rows stays far below
+    assert weights_on_few_rows
+    for ctas in (0, 1, 9, 300):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode(q), expect, BF16, f"peaked rope decode ctas={ctas}")
+    lay.poll_status()
+
+
 def test_rope_decode_steps_lowrank_output_and_switching_off(B):
     B_, H, d, n, steps = 2, 2, 128, 300, 5
     rk, rv = [80, 48], [64, 80]

@@ -45,17 +45,31 @@ def build_and_fill(B, wl, units, extra_rows=1):
     return lay, ranks, U_k, U_v, W_k, W_v, hist
 
 
-def check_units(out, q, hist, new_rows, units, U_k, U_v):
+# Beside the stated tolerance, a regression bound for these diffuse workloads: thousands of rows share the softmax,
+# so the rounding of the cached rows averages out and what remains is the rounding of the bf16 output itself (half
+# a unit in the last place, 2^-9 relative) plus a small absolute term.  Errors of a few rows that the stated
+# tolerance (2e-2) would hide do not pass this one.
+def regression_bound(ref_max: float) -> float:
+    return 2.0 ** -8 * ref_max + 2e-4
+
+
+def check_units(out, q, hist, new_rows, units, U_k, U_v, record=None):
     """out[b, 0, h] against the definition for every sampled unit (history + the new rows)."""
-    errs = []
+    errs, mags = [], []
     for (b, h) in units:
         K = np.concatenate([hist[(b, h)][0]] + [to_np(r[0][b, :, h, :]) for r in new_rows])
         V = np.concatenate([hist[(b, h)][1]] + [to_np(r[1][b, :, h, :]) for r in new_rows])
         ref = orc.decode_head(to_np(q[b, 0, h]), K, V, U_k[h], U_v[h])
         errs.append(np.abs(to_np(out[b, 0, h]) - ref))
+        mags.append(np.abs(ref).max())
     e = np.stack(errs)
     assert np.isfinite(to_np(out)).all()
+    if record is not None:
+        record("max_abs", f"{e.max():.3e}")
+        record("units", len(units))
+    print(f"[parity] {len(units)} units: max-abs {e.max():.3e}, mean-abs {e.mean():.3e}, max|ref| {max(mags):.3e}")
     assert e.max() <= BF16_MAX_ABS and e.mean() <= BF16_MEAN_ABS, (e.max(), e.mean())
+    assert e.max() <= regression_bound(max(mags)), (e.max(), max(mags))
 
 
 def test_llama2_7b_b16_n32k_full_size_sampled_units(B):
@@ -77,12 +91,18 @@ def test_llama2_7b_b16_n32k_full_size_sampled_units(B):
     assert float((out2.float() - out.float()).abs().max()) <= 1e-2
 
 
-@pytest.mark.parametrize("batch,context", [(1, 2048), (4, 8192), (16, 2048)])
-def test_opt_6p7b_hetero_ranks_sampled_units(B, batch, context):
+@pytest.mark.parametrize("context", [2048, 8192, 32768])
+@pytest.mark.parametrize("batch", [1, 4, 16, 64])
+def test_opt_6p7b_hetero_ranks_sampled_units(B, batch, context, record_property):
+    """All twelve points of the batch x context sweep.  Sampled units: every unit when the layer has at most 64,
+    else a seeded subset of at least 64 that holds both corners, every distinct rank and every batch index."""
     wl = dataclasses.replace(synth.WORKLOADS["opt_6p7b_hetero"], batch=batch, context=context)
     ranks0 = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
     assert len(set(ranks0)) == 5                            # every rank of the set occurs
-    units = synth.sample_units(wl.batch, wl.n_heads, ranks0, 24, wl.index)[:24]
+    units = synth.sample_units(wl.batch, wl.n_heads, ranks0, 64, wl.index)
+    assert len(units) >= min(64, batch * wl.n_heads)
+    assert (0, 0) in units and (batch - 1, wl.n_heads - 1) in units
+    assert {b for b, _ in units} == set(range(batch)) and {ranks0[h] for _, h in units} == set(ranks0)
     lay, ranks, U_k, U_v, W_k, W_v, hist = build_and_fill(B, wl, units)
     dt = torch.bfloat16
     k1 = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device="cuda:0")
@@ -90,7 +110,7 @@ def test_opt_6p7b_hetero_ranks_sampled_units(B, batch, context):
     q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt, device="cuda:0")
     out = lay.decode_step(q, k1, v1)
     lay.poll_status()
-    check_units(out, q, hist, [(k1, v1)], units, U_k, U_v)
+    check_units(out, q, hist, [(k1, v1)], units, U_k, U_v, record_property)
 
 
 @pytest.mark.parametrize("batch", [1, 2])

@@ -296,6 +296,45 @@ def test_tracked_subset_equals_full_state():
         assert np.array_equal(of[u], os_[u])
 
 
+def test_append_unit_rows_equals_append_kv_and_the_per_head_definition():
+    # The unit-by-unit hand-over used for large workloads: same state, counters and outputs as append_kv on the
+    # same rows, in chunks, with and without a storage rounding; and the outputs equal the stateless per-head
+    # definition on the raw rows (itself pinned by library attention above), so a wrong basis, a skipped
+    # storage hook or rows filed under another unit cannot pass.
+    B, H, d_h, n = 3, 4, 16, 11
+    rk, rv = [4, 9, 16, 7], [7, 3, 12, 5]          # every head its own ranks: a swapped basis changes shapes or values
+    rng = np.random.default_rng(12)
+    q = rng.standard_normal((B, 1, H, d_h))
+    k = rng.standard_normal((B, n, H, d_h))
+    v = rng.standard_normal((B, n, H, d_h))
+    tracked = [(0, 1), (2, 3), (1, 0)]
+    half = lambda a: a.astype(np.float16).astype(np.float64)      # a 16-bit storage format (Section 2, p = 16)
+    for storage in (None, half):
+        a, U_K, U_V = make_layer(5, B, H, d_h, rk, rv, tracked=tracked)
+        b, _, _ = make_layer(5, B, H, d_h, rk, rv, tracked=tracked)
+        a.storage = b.storage = storage
+        a.append_kv(k, v)
+        for (bb, hh) in tracked:                                   # two chunks per unit, units in another order
+            b.append_unit_rows((bb, hh), k[bb, :4, hh], v[bb, :4, hh])
+        for (bb, hh) in reversed(tracked):
+            b.append_unit_rows((bb, hh), k[bb, 4:, hh], v[bb, 4:, hh])
+        assert b.len == 0                                          # the caller advances the length
+        b.set_len(n)
+        assert a.cache_elements == b.cache_elements == sum(n * (rk[h] + rv[h]) for _, h in tracked)
+        assert a.projection_macs == b.projection_macs
+        oa, ob = a.decode(q), b.decode(q)
+        for u in tracked:
+            assert b.Kp[u].shape == (n, rk[u[1]]) and b.Vp[u].shape == (n, rv[u[1]])
+            assert np.abs(a.Kp[u] - b.Kp[u]).max() < 1e-14 and np.abs(a.Vp[u] - b.Vp[u]).max() < 1e-14
+            assert np.abs(oa[u] - ob[u]).max() < 1e-13
+            if storage is None:
+                ref = orc.decode_head(q[u[0], 0, u[1]], k[u[0], :, u[1]], v[u[0], :, u[1]], U_K[u[1]], U_V[u[1]])
+                assert np.abs(ob[u] - ref).max() < 1e-13
+            else:                                                  # the hook really rounded what the unit keeps
+                assert np.array_equal(b.Kp[u], half(b.Kp[u])) and np.array_equal(b.Vp[u], half(b.Vp[u]))
+                assert np.abs(b.Kp[u] - k[u[0], :, u[1]] @ U_K[u[1]]).max() > 1e-6
+
+
 # ---- P7: tiny brute force with explicit d_h x d_h projectors (Eq. 7, second line) ---------------
 
 @pytest.mark.parametrize("n", [1, 2, 5])

@@ -43,6 +43,27 @@ def test_static_scratch_decode_matches_workspace_decode_twice(B, dtype):
             assert_close(got, ref.decode_dense(to_np(qq)), dtype, "static decode vs oracle")
 
 
+def test_static_scratch_decode_with_peaked_attention(B):
+    """Queries scaled by 6: a few rows carry the softmax, so a partial read from the wrong slot of the built-in
+    array, or a slot left over from the previous call, would show.  Checked against the oracle, for several split
+    plans in a row (each leaves its partials behind for the next)."""
+    from helpers import OraclePair
+    dtype = torch.bfloat16
+    B_, H, d, n = 2, 6, 128, 1037
+    rk, rv = [48, 64, 80, 96, 64, 48], [96, 80, 64, 48, 80, 96]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n, dtype, seed_cfg=122, q_scale=6.0)
+    lay = B.EigenAttnLayer(B_, H, d, n, dtype, U_k, U_v)
+    lay.append_kv(k, v)
+    ref = OraclePair(B_, H, d, U_k, U_v, dtype)
+    ref.append_kv(to_np(k), to_np(v))
+    expect = ref.decode_dense(to_np(q))
+    for ctas, fused in ((0, 1), (5, 1), (37, 0), (148, 1), (2, 1)):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        lay.set_option(B.EA_OPT_DECODE_FUSED, fused)
+        assert_close(lay.decode_static(q), expect, dtype, f"peaked static decode ctas={ctas} fused={fused}")
+    lay.poll_status()
+
+
 def test_static_scratch_rejects_layers_beyond_its_limit(B):
     # (batch*heads + CTAs) * (4 + widest rp_v) must stay within 270336 floats
     B_, H, d, n = 64, 32, 128, 4
