@@ -113,12 +113,31 @@ class ClockSampler:
 # the CPU oracle leg (also the --impl reference arm)
 # ----------------------------------------------------------------------------------------------
 
+QUANT_LEGS = ((4, 32),)                     # (bits, group) of the quantised-cache entries of the workload table
 VARIANT = {"alibi": False, "rope": False}   # --alibi / --rope: position schemes on both sides (decode workloads)
 ROPE_BASE = 10000.0
 
 
 def variant_slopes(wl):
     return synth.alibi_slopes(wl.n_heads) if VARIANT["alibi"] else None
+
+
+def host_description() -> dict:
+    """CPU model and core counts of the machine the oracle is timed on."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for ln in f:
+                if ln.lower().startswith("model name"):
+                    model = ln.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except AttributeError:
+        usable = os.cpu_count() or 1
+    return {"cpu_model": model, "logical_cpus": os.cpu_count(), "usable_cpus": usable}
 
 
 def blas_threads() -> int:
@@ -130,11 +149,11 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, sample_heads, history=None):
-    """Oracle state for the units (0, h), h in sample_heads: projects their whole history once.
-    `history` maps h -> (k_rows, v_rows) [n, d_head] float64; if None it is drawn on the CPU."""
+def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, units, history=None):
+    """Oracle state for the sampled (sequence, head) units: projects their whole history once.
+    `history` maps (b, h) -> (k_rows, v_rows) [n, d_head] float64; if None it is drawn on the CPU (sequence 0 only)."""
     from oracle import eigen_attention as orc
-    units = [(0, h) for h in sample_heads]
+    units = list(units)
     lay = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=units, alibi_slopes=variant_slopes(wl),
                           rope={"base": ROPE_BASE, "interleaved": False} if VARIANT["rope"] else None)
     if history is None:
@@ -145,11 +164,12 @@ def oracle_sample_setup(wl, ranks_k, ranks_v, U_k, U_v, sample_heads, history=No
             t = min(FILL_CHUNK, wl.context - c)
             k = synth.lowrank_rows(W_k, 1, t, wl.sigma, wl.index, "K", chunk=ci, dtype=dt).double().numpy()
             v = synth.lowrank_rows(W_v, 1, t, wl.sigma, wl.index, "V", chunk=ci, dtype=dt).double().numpy()
-            for h in sample_heads:
+            for (b, h) in units:
+                assert b == 0
                 lay.append_unit_rows((0, h), k[0, :, h, :], v[0, :, h, :])
     else:
-        for h in sample_heads:
-            lay.append_unit_rows((0, h), history[h][0], history[h][1])
+        for u in units:
+            lay.append_unit_rows(u, history[u][0], history[u][1])
     lay.set_len(wl.context)
     return lay
 
@@ -179,7 +199,7 @@ def run_reference(args, wl):
     U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
     sample_heads = list(range(wl.n_heads))                  # all heads of sequence 0
-    lay = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, sample_heads)
+    lay = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, [(0, h) for h in sample_heads])
     dt = synth.torch_dtype(wl.dtype)
     W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K")
     W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V")
@@ -241,9 +261,9 @@ def rank_chunk_base(rank: int) -> int:
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------
 
-def build_layer(wl, device, binding, keep_heads=(), rank=0):
+def build_layer(wl, device, binding, keep_units=(), rank=0):
     """Creates the layer and fills `context` rows through eigen_attn_append_kv.  Returns the layer, the
-    bases, and for the units (0, h), h in keep_heads, the raw K/V history as float64 arrays."""
+    bases, and for the (sequence, head) units in keep_units the raw K/V history as float64 arrays."""
     ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
     U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
@@ -255,17 +275,17 @@ def build_layer(wl, device, binding, keep_heads=(), rank=0):
         lay.set_rope(ROPE_BASE)
     W_k = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_K", device=device)
     W_v = synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_V", device=device)
-    hist = {h: ([], []) for h in keep_heads}
+    hist = {u: ([], []) for u in keep_units}
     for ci, c in enumerate(range(0, wl.context, FILL_CHUNK)):
         t = min(FILL_CHUNK, wl.context - c)
         cid = ci + rank_chunk_base(rank)
         k = synth.lowrank_rows(W_k, wl.batch, t, wl.sigma, wl.index, "K", chunk=cid, dtype=dt, device=device)
         v = synth.lowrank_rows(W_v, wl.batch, t, wl.sigma, wl.index, "V", chunk=cid, dtype=dt, device=device)
         lay.append_kv(k, v)
-        for h in keep_heads:
-            hist[h][0].append(k[0, :, h, :].double().cpu().numpy())
-            hist[h][1].append(v[0, :, h, :].double().cpu().numpy())
-    hist = {h: (np.concatenate(a), np.concatenate(b)) for h, (a, b) in hist.items()}
+        for (b, h) in keep_units:
+            hist[(b, h)][0].append(k[b, :, h, :].double().cpu().numpy())
+            hist[(b, h)][1].append(v[b, :, h, :].double().cpu().numpy())
+    hist = {u: (np.concatenate(a), np.concatenate(b)) for u, (a, b) in hist.items()}
     k_new = synth.lowrank_rows(W_k, wl.batch, 1, wl.sigma, wl.index, "K", chunk=10**6, dtype=dt, device=device)
     v_new = synth.lowrank_rows(W_v, wl.batch, 1, wl.sigma, wl.index, "V", chunk=10**6, dtype=dt, device=device)
     q = synth.gaussian_query(wl.batch, wl.n_heads, wl.d_head, wl.q_scale, wl.index, dtype=dt, device=device)
@@ -289,8 +309,10 @@ def run_ours(args, wl):
     from paper_2408_05646_b200 import binding
 
     do_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
-    keep_heads = list(range(0, wl.n_heads, 2)) if do_cpu else []      # 16 sampled units of sequence 0
-    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep_heads, rank=rank)
+    # the oracle's sample: 64 seeded (sequence, head) units with both corners, every rank and every sequence
+    ranks0 = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
+    keep_units = synth.sample_units(wl.batch, wl.n_heads, ranks0, 64, wl.index)[:64] if do_cpu else []
+    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep_units, rank=rank)
     n0 = wl.context
     assert lay.len == n0
     stream = torch.cuda.current_stream(device)
@@ -374,19 +396,29 @@ def run_ours(args, wl):
     cpu = None
     parity = None
     if do_cpu:
-        ref = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, keep_heads, history=hist)
+        ref = oracle_sample_setup(wl, ranks, ranks, U_k, U_v, keep_units, history=hist)
+        del hist
         qn, kn, vn = q.double().cpu().numpy(), k_new.double().cpu().numpy(), v_new.double().cpu().numpy()
-        sec, res = oracle_timed_steps(ref, wl, qn, kn, vn, steps=20, warmup=2)
+        sec, res = oracle_timed_steps(ref, wl, qn, kn, vn, steps=8, warmup=1)
+        cores = blas_threads()
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            sec1, _ = oracle_timed_steps(ref, wl, qn, kn, vn, steps=2, warmup=1)
         es = 2 if wl.dtype == "bf16" else 4
-        sample_bytes = (n0 + 1) * sum(2 * ranks[h] for h in keep_heads) * es
-        cpu = {"value": sample_bytes / sec / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+        sample_bytes = (n0 + 1) * sum(2 * ranks[h] for _, h in keep_units) * es
+        scale = wl.batch * wl.n_heads / len(keep_units)
+        cpu = {"value": sample_bytes / sec / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
                "us_per_step_sample": sec * 1e6,
-               "us_per_step_scaled_to_all_units": sec * 1e6 * wl.batch * wl.n_heads / len(keep_heads),
-               "sample": f"{len(keep_heads)} of {wl.batch * wl.n_heads} (sequence, head) units (sequence 0, every "
-                         f"second head), full context, 20 timed steps; history projected beforehand"}
+               "us_per_step_scaled_to_all_units": sec * 1e6 * scale,
+               "one_thread": {"value": sample_bytes / sec1 / 1e9, "unit": UNIT, "cores": 1,
+                              "us_per_step_sample": sec1 * 1e6, "us_per_step_scaled_to_all_units": sec1 * 1e6 * scale},
+               "host": host_description(),
+               "sample": f"{len(keep_units)} of {wl.batch * wl.n_heads} (sequence, head) units (seeded subset: both corners, "
+                         f"every sequence), full context; a step = append the new row + attend; 8 timed steps with all "
+                         f"BLAS threads, 2 with one thread; history projected beforehand"}
         g = out.double().cpu().numpy()
-        errs = [np.abs(g[0, 0, h] - res[(0, h)]) for h in keep_heads]
-        parity = {"units": len(keep_heads), "max_abs": float(max(e.max() for e in errs)),
+        errs = [np.abs(g[b, 0, h] - res[(b, h)]) for (b, h) in keep_units]
+        parity = {"units": len(keep_units), "max_abs": float(max(e.max() for e in errs)),
                   "mean_abs": float(np.mean([e.mean() for e in errs])),
                   "tolerance": "max_abs <= 2e-2, mean_abs <= 2e-3 (bf16 storage)"}
 
@@ -414,6 +446,12 @@ def run_ours(args, wl):
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    if not args.no_workloads and world == 1 and wl.name == "llama2_7b_b16_n32k" and not (VARIANT["alibi"] or VARIANT["rope"]):
+        line["workloads"] = workload_table(device, binding, lay, wl, ranks, q, k_new, v_new)
+        del lay
+        torch.cuda.empty_cache()
+        line["workloads"].update(workload_table_own_layers(device, binding))
+        lay = None
     if not args.no_prefill and world == 1:
         del lay
         torch.cuda.empty_cache()
@@ -424,6 +462,141 @@ def run_ours(args, wl):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def timed_kernel(lay, device, call, steps, warmup):
+    """Runs `call()` warmup + steps times with the library's event pair around its attention kernel.
+    Returns (median kernel us, mean us per call on the stream)."""
+    stream = torch.cuda.current_stream(device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        a.record(stream); b.record(stream)
+    for _ in range(warmup):
+        call()
+    torch.cuda.synchronize(device)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        lay.set_decode_events(ev[i][0], ev[i][1])
+        call()
+    t1.record(stream)
+    torch.cuda.synchronize(device)
+    lay.set_decode_events(None, None)
+    lay.poll_status()
+    ks = sorted(a.elapsed_time(b) for a, b in ev)
+    return ks[len(ks) // 2] * 1e3, t0.elapsed_time(t1) / steps * 1e3
+
+
+def table_entry(kernel, kernel_us, step_us, nbytes, peak, **extra):
+    d = {"kernel": kernel, "kernel_us": round(kernel_us, 2), "step_us": round(step_us, 2), "algorithmic_bytes": int(nbytes),
+         "GB/s": round(nbytes / kernel_us / 1e3, 1), "frac": round(nbytes / kernel_us / 1e3 / peak, 4)}
+    d.update(extra)
+    return d
+
+
+def workload_table(device, binding, lay2, wl2, ranks2, q2, k2, v2, steps=30, warmup=3):
+    """The other workloads, each as one short timed region of the call a user makes: kernel time from the library's
+    event pair (median), step time on the stream, algorithmic bytes of the rows (or codes) the step must read, and
+    the fraction of the measured copy bandwidth.  `lay2` is the headline layer, already filled; the variants that
+    share its cache (unequal lengths, rotary embedding, quantised copy) reuse it."""
+    import dataclasses
+    peak, _ = measured_peaks()
+    table = {}
+    n2 = wl2.context
+    out2 = torch.empty_like(q2)
+
+    # ---- unequal lengths on the headline cache: sequence b keeps (b + 1) / B of the context
+    lens = [max(1, n2 * (b + 1) // wl2.batch) for b in range(wl2.batch)]
+    lay2.set_lens(lens)
+    k_us, s_us = timed_kernel(lay2, device, lambda: lay2.decode(q2, out=out2), steps, warmup)
+    row_bytes = sum(2 * 2 * r for r in ranks2)
+    table["ragged"] = table_entry("decode_splitkv_kernel", k_us, s_us, sum(lens) * row_bytes, peak,
+                                  workload=wl2.name + " with lens[b] = context * (b + 1) / batch")
+    lay2.set_len(n2)
+
+    # ---- ALiBi bias on the headline cache
+    lay2.set_alibi(synth.alibi_slopes(wl2.n_heads))
+    def step_alibi():
+        lay2.set_len(n2); lay2.decode_step(q2, k2, v2, out=out2)
+    k_us, s_us = timed_kernel(lay2, device, step_alibi, steps, warmup)
+    table["alibi"] = table_entry("decode_splitkv_kernel", k_us, s_us, algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1), peak,
+                                 workload=wl2.name + " with per-head ALiBi slopes")
+    lay2.set_alibi(None)
+    lay2.set_len(n2)
+
+    # ---- RoPE variant of decode on the headline cache (full-rank query, keys lifted and rotated)
+    lay2.set_rope(ROPE_BASE)
+    def step_rope():
+        lay2.set_len(n2); lay2.decode_step(q2, k2, v2, out=out2)
+    k_us, s_us = timed_kernel(lay2, device, step_rope, steps, warmup)
+    table["rope"] = table_entry("decode_rope_kernel", k_us, s_us, algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1), peak,
+                                workload=wl2.name + " with rotary position embedding")
+    lay2.set_rope(0.0)
+    lay2.set_len(n2)
+
+    # ---- quantised copies of the headline cache
+    for bits, G in QUANT_LEGS:
+        lay2.set_len(n2)
+        lay2.quant_attach(bits, G)
+        lay2.quant_sync()
+        def step_quant():
+            lay2.set_len(n2); lay2.append_kv(k2, v2); lay2.decode_quant(q2, out=out2)
+        k_us, s_us = timed_kernel(lay2, device, step_quant, steps, warmup)
+        nq = n2 // G * G
+        codes = wl2.batch * (nq // G) * sum(lay2.quant_layout(h)[1] for h in range(wl2.n_heads))
+        tail = wl2.batch * (n2 + 1 - nq) * row_bytes
+        table[f"quant_{bits}bit_g{G}"] = table_entry("decode_quant_kernel", k_us, s_us, codes + tail, peak,
+                                                     workload=wl2.name + f", {bits}-bit codes, group {G}",
+                                                     bytes_16bit=algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1))
+        lay2.quant_detach()
+    lay2.set_len(n2)
+    return table
+
+
+def workload_table_own_layers(device, binding, steps=30, warmup=3):
+    """Workloads that need a layer of their own: the long-context layer (B = 1, 2), the batch x context sweep of the
+    layer with per-head ranks, and the grouped-query layer."""
+    import dataclasses
+    peak, _ = measured_peaks()
+    table = {}
+    for b in (1, 2):
+        wl = dataclasses.replace(synth.WORKLOADS["mpt_7b_long"], batch=b)
+        lay, ranks, _, _, _, q, kn, vn = build_layer(wl, device, binding)
+        out = torch.empty_like(q)
+        def step():
+            lay.set_len(wl.context); lay.decode_step(q, kn, vn, out=out)
+        k_us, s_us = timed_kernel(lay, device, step, steps, warmup)
+        table[f"mpt_7b_long[batch={b}]"] = table_entry("decode_splitkv_kernel", k_us, s_us,
+                                                       algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak)
+        del lay
+        torch.cuda.empty_cache()
+    for b in (1, 4, 16, 64):
+        wl = dataclasses.replace(synth.WORKLOADS["opt_6p7b_hetero"], batch=b, context=32768)
+        lay, ranks, _, _, _, q, kn, vn = build_layer(wl, device, binding)
+        out = torch.empty_like(q)
+        for n in (2048, 8192, 32768):                       # the rows beyond n stay in the cache and are not read
+            def step():
+                lay.set_len(n); lay.decode_step(q, kn, vn, out=out)
+            k_us, s_us = timed_kernel(lay, device, step, steps, warmup)
+            wn = dataclasses.replace(wl, context=n)
+            table[f"opt_6p7b_hetero[batch={b},context={n}]"] = table_entry(
+                "decode_splitkv_kernel", k_us, s_us, algorithmic_bytes(wn, ranks, ranks, n + 1), peak,
+                l2="cache-resident" if algorithmic_bytes(wn, ranks, ranks, n + 1) < 126e6 else "larger than L2")
+        del lay
+        torch.cuda.empty_cache()
+    wl = synth.WORKLOADS["llama3_8b_gqa_b16_n32k"]
+    g = synth.GQA_GROUP[wl.name]
+    lay, ranks, _, _, _, _, kn, vn = build_layer(wl, device, binding)
+    q = synth.gaussian_query(wl.batch, wl.n_heads * g, wl.d_head, wl.q_scale, wl.index, dtype=synth.torch_dtype(wl.dtype), device=device)
+    out = torch.empty_like(q)
+    def step_gqa():
+        lay.set_len(wl.context); lay.append_kv(kn, vn); lay.decode_gqa(q, g, out=out)
+    k_us, s_us = timed_kernel(lay, device, step_gqa, steps, warmup)
+    table[wl.name] = table_entry("decode_gqa_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
+                                 group=g)
+    del lay
+    torch.cuda.empty_cache()
+    return table
 
 
 def prefill_measure(wl, device, steps, warmup, impl=0):
@@ -619,7 +792,7 @@ def run_gqa(args, wl):
     from paper_2408_05646_b200 import binding
     g = synth.GQA_GROUP[wl.name.split("[")[0]]
     keep = [0, wl.n_heads - 1]
-    lay, ranks, U_k, U_v, hist, _, k_new, v_new = build_layer(wl, device, binding, keep)
+    lay, ranks, U_k, U_v, hist, _, k_new, v_new = build_layer(wl, device, binding, [(0, h) for h in keep])
     dt = synth.torch_dtype(wl.dtype)
     q = synth.gaussian_query(wl.batch, wl.n_heads * g, wl.d_head, wl.q_scale, wl.index, dtype=dt, device=device)
     out = torch.empty_like(q)
@@ -675,7 +848,7 @@ def run_gqa(args, wl):
     from oracle import eigen_attention as orc
     ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=[(0, h) for h in keep])
     for h in keep:
-        ref.append_unit_rows((0, h), hist[h][0], hist[h][1])
+        ref.append_unit_rows((0, h), hist[(0, h)][0], hist[(0, h)][1])
     ref.set_len(n0)
     ref.append_kv(k_new.double().cpu().numpy(), v_new.double().cpu().numpy())
     exp = ref.decode_gqa(q.double().cpu().numpy(), g)
@@ -710,7 +883,7 @@ def run_quant(args, wl):
     from paper_2408_05646_b200 import binding
     G = args.quant
     keep = [0, wl.n_heads - 1]
-    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, keep)
+    lay, ranks, U_k, U_v, hist, q, k_new, v_new = build_layer(wl, device, binding, [(0, h) for h in keep])
     lay.quant_attach(4, G)
     lay.quant_sync()
     n0 = wl.context
@@ -772,7 +945,7 @@ def run_quant(args, wl):
     storage = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dt).double().numpy()
     ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=[(0, h) for h in keep], storage=storage)
     for h in keep:
-        ref.append_unit_rows((0, h), hist[h][0], hist[h][1])
+        ref.append_unit_rows((0, h), hist[(0, h)][0], hist[(0, h)][1])
     ref.set_len(n0)
     ref.append_kv(k_new.double().cpu().numpy(), v_new.double().cpu().numpy())
     exp = ref.decode_quant(q.double().cpu().numpy(), 4, G)
@@ -811,6 +984,7 @@ def main():
                     help="decode workloads: attend over the 4-bit quantised cache with group size G (16, 32, 64, 128)")
     ap.add_argument("--ragged", action="store_true", help="decode workloads: sequence b keeps (b + 1) / batch of the context")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the table of the other workloads in the headline line")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")

@@ -267,6 +267,9 @@ typedef enum {
                                  streams token tiles by TMA when d_head % 64 == 0 and T >= 128), 1 = always
                                  one CTA per tile of 128 tokens, n >= 2 = the persistent kernel with at most
                                  n CTAs                                                                    */
+  EA_OPT_DECODE_MIN_COPY_BYTES = 8, /* split-KV decode: heads whose K' or V' tile is smaller than this many bytes
+                                 put up to four consecutive tiles into one ring slot, i.e. one bulk copy;
+                                 -1 = the default (16 KiB), 0 = always one tile per slot                     */
   EA_OPT_TEST_WAIT_GIVES_UP = 7 /* failure-path test hook.  1 arms it for the NEXT eigen_attn_decode /
                                  _decode_step / _decode_static launch only: one warp of one CTA treats its
                                  first wait for a tile as having exceeded the bound.  The launch then ends the

@@ -25,6 +25,7 @@ EA_OPT_DECODE_CTAS, EA_OPT_DECODE_TILE_ROWS, EA_OPT_DECODE_STAGES, EA_OPT_PREFIL
 EA_OPT_DECODE_FUSED = 5
 EA_OPT_PREFILL_PROJECT = 6
 EA_OPT_TEST_WAIT_GIVES_UP = 7
+EA_OPT_DECODE_MIN_COPY_BYTES = 8
 
 STATUS_NAMES = {0: "EA_OK", -1: "EA_ERR_INVALID_ARG", -2: "EA_ERR_SHAPE", -3: "EA_ERR_CAPACITY",
                 -4: "EA_ERR_UNSUPPORTED", -5: "EA_ERR_CUDA", -6: "EA_ERR_TIMEOUT",
@@ -268,6 +269,11 @@ class EigenAttnLayer:
         self._check(lib.eigen_attn_quant_attach(self.handle, int(bits), int(group), self.qcache.data_ptr(), nbytes,
                                                 _stream_ptr(stream)), "eigen_attn_quant_attach")
         return self.qcache
+
+    def quant_detach(self, stream=None) -> None:
+        """Detaches the quantised buffer (eigen_attn_quant_attach with NULL) and drops the tensor."""
+        self._check(lib.eigen_attn_quant_attach(self.handle, 0, 0, None, 0, _stream_ptr(stream)), "eigen_attn_quant_attach")
+        self.qcache = None
 
     def quant_sync(self, stream=None) -> None:
         self._check(lib.eigen_attn_quant_sync(self.handle, _stream_ptr(stream)), "eigen_attn_quant_sync")

@@ -24,6 +24,7 @@ constexpr int kMaxDecodeCtas = 1024;
 constexpr int kPartialSlack = 4;     // the partials area holds this many times (batch x heads + kMaxDecodeCtas) slots
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kInFlightBytes = 120 * 1024;   // target bytes of bulk copies in flight per SM (decode)
+constexpr int kMinCopyBytes = 16 * 1024;     // a bulk copy should move at least about this much (decode; narrow heads)
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 uint16_t bf16_rne(float x) {          // round to nearest even; inputs are finite
@@ -197,6 +198,7 @@ struct eigen_attn {
   bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
   int rope_interleaved = 0;
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1, opt_project = 0;
+  int64_t opt_min_copy = -1;  // EA_OPT_DECODE_MIN_COPY_BYTES; < 0 = the built-in default
   int64_t opt_give_up = 0;   // EA_OPT_TEST_WAIT_GIVES_UP: armed for the next split-KV decode launch
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
@@ -309,6 +311,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
   const int sms = h->opt_ctas > 0 ? static_cast<int>(h->opt_ctas) : h->sm_count;
 
+  const int min_copy = h->opt_min_copy >= 0 ? static_cast<int>(h->opt_min_copy) : kMinCopyBytes;
   // rows per tile: 128 unless the context is short (keep a few tiles per CTA) or a stage would be too big
   int tile_rows = 128;
   if (h->opt_tile_rows > 0) {
@@ -326,6 +329,15 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
     const int avail = kSmemLimit - fixed;
     if (3 * widest <= avail || tile_rows <= 16) {
       int want = 3 * widest > kInFlightBytes + widest ? 3 * widest : kInFlightBytes + widest;
+      // narrow heads put several tiles into a slot (one copy of about min_copy bytes): room for three such slots
+      for (const HeadInfo& hi : L.heads) {
+        const int kb = tile_rows * hi.rp_k * L.es, vb = tile_rows * hi.rp_v * L.es;
+        const int narrow = kb < vb ? kb : vb;
+        int tps = (min_copy + narrow - 1) / narrow;
+        if (tps > 4) tps = 4;
+        const int slot = static_cast<int>(align_up(static_cast<size_t>(kb + vb) * tps, 128));
+        if (3 * slot > want) want = 3 * slot;
+      }
       if (h->opt_stages > 0) want = static_cast<int>(h->opt_stages) * widest;
       ring_bytes = want < avail ? want : avail;
       if (ring_bytes < widest)
@@ -366,6 +378,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.tile_rows = tile_rows; p.nt = nt; p.ring_bytes = ring_bytes; p.inflight_bytes = kInFlightBytes;
   p.fixed_stages = static_cast<int>(h->opt_stages);
+  p.min_copy_bytes = min_copy > 0 ? min_copy : 1;
   p.nt_total = nt_total;
   p.w_total = w_total;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
@@ -1187,6 +1200,10 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
     case EA_OPT_PREFILL_PROJECT:
       if (value < 0 || value > 65535) return fail(h, EA_ERR_INVALID_ARG, "PREFILL_PROJECT %lld", static_cast<long long>(value));
       h->opt_project = value;
+      return EA_OK;
+    case EA_OPT_DECODE_MIN_COPY_BYTES:
+      if (value < -1 || value > (1 << 20)) return fail(h, EA_ERR_INVALID_ARG, "DECODE_MIN_COPY_BYTES %lld", static_cast<long long>(value));
+      h->opt_min_copy = value;
       return EA_OK;
     case EA_OPT_TEST_WAIT_GIVES_UP:
       if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "TEST_WAIT_GIVES_UP %lld", static_cast<long long>(value));

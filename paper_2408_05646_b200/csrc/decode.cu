@@ -25,6 +25,11 @@ namespace {
 
 constexpr int kMaxStages = 12;
 constexpr uint64_t kWaitBoundNs = 2000000000ull;   // every device-side wait gives up after 2 s
+// Registers per thread after the reallocation.  The CTA is launched with 384 threads x 168 registers (three
+// warps per scheduler share its 16 384); the producer's warpgroup keeps 56 each, the two consumer warpgroups
+// take the rest: 128 x 56 + 256 x 224 = 384 x 168.
+constexpr int kRegsProducerGroup = 56, kRegsConsumers = 224;
+static_assert(128 * kRegsProducerGroup + 256 * kRegsConsumers <= kDecodeThreads * 168, "register split exceeds the launch");
 
 struct __align__(128) DecodeSmemFixed {
   unsigned long long full[kMaxStages];
@@ -109,8 +114,9 @@ __device__ __forceinline__ float fast_exp2(float x) {
 struct Ring {
   int stage = 0;            // next slot
   int stages = 0;           // slots of the current geometry
-  int stage_bytes = 0;      // bytes per slot: K tile, then V tile at v_off
+  int stage_bytes = 0;      // bytes per slot: K tiles, then V tiles at v_off
   int v_off = 0;
+  int tps = 1;              // tiles per slot (consecutive tiles of a unit are one contiguous range of rows)
   uint32_t full_bits = 0;   // bit s: parity of slot s's next "full" phase
   uint32_t empty_bits = 0;  // bit s: parity of slot s's next "empty" phase (producer only)
   uint32_t filled = 0;      // bit s: the slot holds a tile not yet known to be released (producer only)
@@ -118,11 +124,20 @@ struct Ring {
 };
 
 // Slot geometry for a head: about p.inflight_bytes of copies in flight, at least three slots if they fit.
+// A slot of a narrow head holds `tps` consecutive tiles (one bulk copy for their K' rows, one for their V'
+// rows), so that a copy moves about p.min_copy_bytes: small copies do not reach the memory system's rate.
 template <typename T>
 __device__ __forceinline__ void ring_geometry(const DecodeParams& p, const HeadInfo& hd, int* stage_bytes,
-                                              int* v_off, int* stages) {
-  const int kb = p.tile_rows * hd.rp_k * static_cast<int>(sizeof(T));
-  const int vb = p.tile_rows * hd.rp_v * static_cast<int>(sizeof(T));
+                                              int* v_off, int* stages, int* tiles_per_slot) {
+  int kb = p.tile_rows * hd.rp_k * static_cast<int>(sizeof(T));
+  int vb = p.tile_rows * hd.rp_v * static_cast<int>(sizeof(T));
+  const int narrow = kb < vb ? kb : vb;
+  int tps = (p.min_copy_bytes + narrow - 1) / narrow;
+  if (tps > 4) tps = 4;
+  while (tps > 1 && 3 * (((kb + vb) * tps + 127) & ~127) > p.ring_bytes) --tps;   // keep three slots
+  if (tps < 1) tps = 1;
+  kb *= tps;
+  vb *= tps;
   const int sb = (kb + vb + 127) & ~127;
   int fit = p.ring_bytes / sb;
   if (fit > kMaxStages) fit = kMaxStages;
@@ -131,6 +146,7 @@ __device__ __forceinline__ void ring_geometry(const DecodeParams& p, const HeadI
   *stage_bytes = sb;
   *v_off = kb;
   *stages = want < fit ? want : fit;
+  *tiles_per_slot = tps;
 }
 
 // L2 policy for data that is read once: evict it first.
@@ -320,7 +336,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     }
   };
 
-  for (int i = i0; i < i1; ++i) {
+  for (int i = i0; i < i1; i += ring_state.tps) {           // one slot: up to tps tiles, contiguous rows
     const int stage = ring_state.stage;
     const uint32_t parity = (ring_state.full_bits >> stage) & 1u;
     ring_state.full_bits ^= 1u << stage;
@@ -340,7 +356,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     }
     const unsigned char* kt = ring + static_cast<size_t>(stage) * ring_state.stage_bytes;
     const unsigned char* vt = kt + ring_state.v_off;
-    const int rows = min(p.tile_rows, n_b - i * p.tile_rows);
+    const int rows = min(min(ring_state.tps, i1 - i) * p.tile_rows, n_b - i * p.tile_rows);
     // The loop bound is the same for all lanes of a warp (the shuffle inside needs every lane);
     // lane pairs past the last row recompute the group's first row and drop the result.
     for (int rbase = warp * 16; rbase < rows; rbase += kDecodeConsumerWarps * 16) {
@@ -467,7 +483,7 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
     else if (o < nq + hd.rp_k) { x = fx->kraw; U = p.basis + hd.uk_off + (o - nq); rp = hd.rp_k; }
     else { x = fx->vraw; U = p.basis + hd.uv_off + (o - nq - hd.rp_k); rp = hd.rp_v; }
     float acc = 0.f;
-#pragma unroll 16
+#pragma unroll 32
     for (int d = d0; d < d1; ++d) acc = fmaf(x[d], __ldg(U + d * rp), acc);
     return acc;
   };
@@ -595,9 +611,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
   const long long f_lo = fx->range[0], f_hi = fx->range[1];
   volatile int* abort_flag = &fx->abort_flag;
 
-  if (warp == kDecodeConsumerWarps) {
-    // ------------------------------------------------------------ producer
-    if (lane == 0) {
+  if (warp >= kDecodeConsumerWarps) {
+    // ------------------------------------------------------------ producer (first thread of its warpgroup)
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducerGroup));
+    if (warp == kDecodeConsumerWarps && lane == 0) {
       const uint64_t policy = policy_evict_first();
       Ring rg;
       bool ok = true;
@@ -609,8 +626,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const int i1 = static_cast<int>(min(static_cast<long long>(pc.nt_u), i0 + (f_hi - F)));
         const HeadInfo hd = p.heads[pc.h];
         const int n_b = seq_rows(p, b);
-        int sb, voff, nst;
-        ring_geometry<T>(p, hd, &sb, &voff, &nst);
+        int sb, voff, nst, tps;
+        ring_geometry<T>(p, hd, &sb, &voff, &nst, &tps);
         if (sb != rg.stage_bytes || nst != rg.stages) {
           // New slot layout: the new slots overlap the old ones differently, so every tile still in the
           // ring must have been released before the first copy into the new layout.
@@ -624,12 +641,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
           rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb;
         }
         rg.v_off = voff;                  // two heads can share the slot size and still split it differently
+        rg.tps = tps;
         const uint32_t rowb_k = hd.rp_k * sizeof(T), rowb_v = hd.rp_v * sizeof(T);
         const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(i0) * p.tile_rows;
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
         const char* src_v = p.cache + hd.v_off + row0 * rowb_v;
         const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
-        for (int i = i0; i < i1; ++i) {
+        for (int i = i0; i < i1; i += tps) {
           if (*abort_flag) { ok = false; break; }
           const int st = rg.stage;
           const uint32_t bit = 1u << st;
@@ -641,8 +659,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
             }
             rg.empty_bits ^= bit;
           }
-          uint32_t bytes_k = tile_k, bytes_v = tile_v;
-          if (i == pc.nt_u - 1) {         // ragged last tile of the unit
+          const int span = min(tps, i1 - i);
+          uint32_t bytes_k = span * tile_k, bytes_v = span * tile_v;
+          if (i + span == pc.nt_u) {      // the slot ends with the unit's (ragged) last tile
             const uint32_t rows = n_b - i * p.tile_rows;
             bytes_k = rows * rowb_k;
             bytes_v = rows * rowb_v;
@@ -656,8 +675,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
           }
           rg.filled |= bit;
           rg.full_bits ^= bit;            // bit now holds the parity of the slot's next fill
-          src_k += tile_k;
-          src_v += tile_v;
+          src_k += span * tile_k;
+          src_v += span * tile_v;
           rg.advance();
         }
         F += i1 - i0;
@@ -669,6 +688,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
     }
   } else {
     // ------------------------------------------------------------ consumers
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumers));
     Ring rg;
     long long F = f_lo;
     while (F < f_hi) {
@@ -678,12 +698,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const int i1 = static_cast<int>(min(static_cast<long long>(pc.nt_u), i0 + left));
       const HeadInfo hd = p.heads[h];
       {
-        int sb, voff, nst;
-        ring_geometry<T>(p, hd, &sb, &voff, &nst);
+        int sb, voff, nst, tps;
+        ring_geometry<T>(p, hd, &sb, &voff, &nst, &tps);
         if (sb != rg.stage_bytes || nst != rg.stages) {      // same decision as the producer's
           rg.stage = 0; rg.stages = nst; rg.stage_bytes = sb;
         }
         rg.v_off = voff;
+        rg.tps = tps;
       }
       const bool whole = i0 == 0 && i1 == pc.nt_u;
       const bool with_new_row = p.k_new != nullptr && i1 == pc.nt_u;

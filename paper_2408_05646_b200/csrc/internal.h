@@ -26,7 +26,9 @@ struct HeadInfo {
 };
 
 constexpr int kDecodeConsumerWarps = 8;
-constexpr int kDecodeThreads = (kDecodeConsumerWarps + 1) * 32;   // + one producer warp
+// + one warpgroup whose first thread is the producer: register reallocation works on whole warpgroups, and the
+// producer's group hands most of its registers to the consumers
+constexpr int kDecodeThreads = (kDecodeConsumerWarps + 4) * 32;
 constexpr int kMaxHeads = 256;
 constexpr int kStatusTimeout = -6;
 constexpr int kMaxRaggedBatch = 1024;   // largest batch that may hold sequences of unequal lengths
@@ -54,6 +56,7 @@ struct DecodeParams {
   int32_t nt;               // tiles per unit = ceil(n / tile_rows)
   int32_t ring_bytes;       // shared memory of the tile ring; slots are sized per head inside the kernel
   int32_t inflight_bytes;   // target bytes of copies in flight per SM (sets the slot count per head)
+  int32_t min_copy_bytes;   // a slot of a narrow head holds several tiles, so that one bulk copy moves about this much
   int32_t fixed_stages;     // > 0: use this many slots (if they fit) instead of the in-flight target
   int64_t nt_total;         // tiles of one head: B * nt, or the sum of the sequences' own tile counts
   int64_t w_total;          // nt_total * sum_h (rp_k + rp_v)

@@ -397,6 +397,33 @@ def test_peaked_attention_over_heads_that_share_a_slot_size(B, dtype):
     lay.poll_status()
 
 
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+def test_peaked_attention_with_several_tiles_per_ring_slot(B, dtype):
+    """Narrow heads put up to four consecutive tiles into one ring slot (one bulk copy).  Pieces start and end at
+    any tile, so a slot can hold 1..4 tiles and end with the unit's ragged tail; peaked weights make a row that is
+    skipped, read twice or taken from the neighbouring tile visible.  Wide and narrow heads alternate, so the slot
+    layout changes from piece to piece."""
+    from helpers import OraclePair
+    B_, H, d, n = 2, 5, 128, 2077
+    rk, rv = [16, 112, 24, 48, 8], [24, 96, 16, 40, 128]
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + 1, dtype, seed_cfg=147, q_scale=6.0, T_q=2)
+    lay = B.EigenAttnLayer(B_, H, d, n + 1, dtype, U_k, U_v)
+    lay.append_kv(k[:, :n], v[:, :n])
+    ref = OraclePair(B_, H, d, U_k, U_v, dtype)
+    ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
+    expect = ref.decode_dense(to_np(q[:, :1]))
+    tol = dict(fp32_rel=2e-4) if dtype == FP32 else {}
+    for rows, min_copy, ctas in ((0, -1, 0), (16, 1 << 20, 3), (32, 1 << 20, 148), (128, 1 << 20, 7), (64, 0, 37), (16, 6000, 1)):
+        lay.set_option(B.EA_OPT_DECODE_TILE_ROWS, rows)
+        lay.set_option(B.EA_OPT_DECODE_MIN_COPY_BYTES, min_copy)
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode(q[:, :1]), expect, dtype, f"tile_rows={rows} min_copy={min_copy} ctas={ctas}", **tol)
+    o = lay.decode_step(q[:, 1:], k[:, n:], v[:, n:])               # the fused step over multi-tile slots
+    ref.append_kv(to_np(k[:, n:]), to_np(v[:, n:]))
+    assert_close(o, ref.decode_dense(to_np(q[:, 1:])), dtype, "decode_step", **tol)
+    lay.poll_status()
+
+
 @pytest.mark.parametrize("impl", [2, 3, 1])
 def test_prefill_with_peaked_attention(B, impl):
     """Queries scaled by 3: the weights of a prompt row sit on a few keys, so an error in a few rows (a stale tile, a
