@@ -494,6 +494,73 @@ def table_entry(kernel, kernel_us, step_us, nbytes, peak, **extra):
     return d
 
 
+def merged_inputs(lay, wl, device, step=0):
+    """Packed rank-space q', k', v' of one new token, as a layer with merged weights would produce them: seeded
+    N(0,1) draws in the IO dtype with zero padding lanes."""
+    dt = synth.torch_dtype(wl.dtype)
+    outs = []
+    for tag, offs, ranks in (("Q", lay.offs_k, lay.r_k), ("K", lay.offs_k, lay.r_k), ("V", lay.offs_v, lay.r_v)):
+        g = torch.Generator(device=device).manual_seed(synth.stream_seed(wl.index, "z_" + tag, extra=7000000 + step))
+        x = torch.randn((wl.batch, 1, offs[-1]), generator=g, dtype=torch.float32, device=device)
+        mask = torch.zeros(offs[-1], dtype=torch.bool, device=device)
+        for h, r in enumerate(ranks):
+            mask[offs[h]:offs[h] + r] = True
+        outs.append((x * mask).to(dt).contiguous())
+    return outs
+
+
+def run_merged(args, wl):
+    """The decode step as a layer with merged weights (Eq. 8) calls it: rank-space q', k', v' in, rank-space o' out.
+    One JSON line: KV bytes per second against the HBM roofline, and parity of sampled units against the oracle,
+    which receives the d_head-wide vectors whose projections are exactly those rank-space rows (x' U^T)."""
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    from paper_2408_05646_b200 import build
+    build.build_library()
+    from paper_2408_05646_b200 import binding
+    keep = [(0, 0), (wl.batch - 1, wl.n_heads - 1)]
+    lay, ranks, U_k, U_v, hist, _, _, _ = build_layer(wl, device, binding, keep)
+    n0 = wl.context
+    qp, kp, vp = merged_inputs(lay, wl, device)
+    outp = torch.empty((wl.batch, 1, lay.offs_v[-1]), dtype=qp.dtype, device=device)
+    def step():
+        lay.set_len(n0)
+        lay.decode_step(qp, kp, vp, out=outp, q_preprojected=True, kv_preprojected=True, out_lowrank=True)
+    steps, warmup = min(args.steps, 100), max(3, min(args.warmup, 10))
+    sampler = ClockSampler(device.index or 0)
+    sampler.start(); time.sleep(0.2)
+    l0 = lay.launch_count()
+    k_us, s_us = timed_kernel(lay, device, step, steps, warmup)
+    launches = lay.launch_count() - l0
+    clocks = sampler.stop()
+    bytes_step = algorithmic_bytes(wl, ranks, ranks, n0 + 1)
+    peak, peak_src = measured_peaks()
+    from oracle import eigen_attention as orc
+    ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=keep)
+    errs = []
+    for (b, h) in keep:
+        back = lambda x, offs, U: x[b, 0, offs[h]:offs[h] + U[h].shape[1]].double().cpu().numpy() @ U[h].astype(np.float64).T
+        K = np.concatenate([hist[(b, h)][0], back(kp, lay.offs_k, U_k)[None]])
+        V = np.concatenate([hist[(b, h)][1], back(vp, lay.offs_v, U_v)[None]])
+        exp = orc.decode_head(back(qp, lay.offs_k, U_k), K, V, U_k[h], U_v[h], lowrank_out=True)
+        got = outp[b, 0, lay.offs_v[h]:lay.offs_v[h] + ranks[h]].double().cpu().numpy()
+        errs.append(float(np.abs(got - exp).max()))
+    achieved = bytes_step / k_us / 1e3
+    print(json.dumps({
+        "metric": "rank-r decode attention KV GB/s, merged-weight call (rank-space q', k', v' in, o' out)",
+        "value": bytes_step / s_us / 1e3, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warmup,
+        "ms_per_step": s_us * 1e-3, "us_per_step": s_us, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "rank": sorted(set(ranks)), "context": n0,
+                   "flags": "EA_Q_PREPROJECTED | EA_KV_PREPROJECTED | EA_OUT_LOWRANK", "l2": "inputs larger than L2"},
+        "roofline": {"bound": "hbm", "kernel": "decode_splitkv_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src, "kernel_us": k_us, "algorithmic_bytes": bytes_step,
+                     "traffic": None},
+        "gpu_launches": launches, "clocks": clocks,
+        "parity_sampled_units": {"units": len(errs), "max_abs": max(errs), "tolerance": "max_abs <= 2e-2"},
+    }))
+
+
 def workload_table(device, binding, lay2, wl2, ranks2, q2, k2, v2, steps=30, warmup=3):
     """The other workloads, each as one short timed region of the call a user makes: kernel time from the library's
     event pair (median), step time on the stream, algorithmic bytes of the rows (or codes) the step must read, and
@@ -532,6 +599,17 @@ def workload_table(device, binding, lay2, wl2, ranks2, q2, k2, v2, steps=30, war
     table["rope"] = table_entry("decode_rope_kernel", k_us, s_us, algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1), peak,
                                 workload=wl2.name + " with rotary position embedding")
     lay2.set_rope(0.0)
+    lay2.set_len(n2)
+
+    # ---- merged weights (Eq. 8): rank-space q', k', v' in, rank-space o' out; no multiplication by U in the step
+    qp, kp, vp = merged_inputs(lay2, wl2, device)
+    outp = torch.empty((wl2.batch, 1, lay2.offs_v[-1]), dtype=q2.dtype, device=device)
+    def step_merged():
+        lay2.set_len(n2)
+        lay2.decode_step(qp, kp, vp, out=outp, q_preprojected=True, kv_preprojected=True, out_lowrank=True)
+    k_us, s_us = timed_kernel(lay2, device, step_merged, steps, warmup)
+    table["merged_weights"] = table_entry("decode_splitkv_kernel", k_us, s_us, algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1), peak,
+                                          workload=wl2.name + ", rank-space q', k', v' in and o' out")
     lay2.set_len(n2)
 
     # ---- quantised copies of the headline cache
@@ -982,6 +1060,7 @@ def main():
     ap.add_argument("--rope", action="store_true", help="decode workloads: the RoPE variant (full-rank query, lifted rotated keys)")
     ap.add_argument("--quant", type=int, default=0, metavar="G",
                     help="decode workloads: attend over the 4-bit quantised cache with group size G (16, 32, 64, 128)")
+    ap.add_argument("--merged", action="store_true", help="decode workloads: the step as a layer with merged weights calls it")
     ap.add_argument("--ragged", action="store_true", help="decode workloads: sequence b keeps (b + 1) / batch of the context")
     ap.add_argument("--no-prefill", action="store_true", help="skip the short prefill measurement in the decode line")
     ap.add_argument("--no-workloads", action="store_true", help="skip the table of the other workloads in the headline line")
@@ -1015,6 +1094,8 @@ def main():
         return run_quant(args, wl)
     if args.ragged:
         return run_ragged(args, wl)
+    if args.merged:
+        return run_merged(args, wl)
     if wl.name.startswith("prefill"):
         run_prefill(args, wl)
     else:

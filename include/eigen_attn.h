@@ -131,7 +131,10 @@ ea_status eigen_attn_decode_static(eigen_attn_t h, const void* d_q, int64_t stri
 
 /* eigen_attn_append_kv with T = 1 followed by eigen_attn_decode (one generated token), fused into a
  * single launch when the cache already holds at least one row.
- * d_k and d_v share the batch stride `stride_b_kv`. */
+ * d_k and d_v share the batch stride `stride_b_kv`.  flags: EA_Q_PREPROJECTED, EA_KV_PREPROJECTED (d_k, d_v are the
+ * packed rank-space rows [B][1][sum rp_k] and [B][1][sum rp_v]; their stride argument is ignored), EA_OUT_LOWRANK.
+ * With all three the call is the attention core of a layer whose weights carry the bases (Eq. 8): no
+ * multiplication by U remains in it. */
 ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q,
                                  const void* d_k, const void* d_v, int64_t stride_b_kv,
                                  void* d_out, int64_t stride_b_out, uint32_t flags, void* cuda_stream);
@@ -145,7 +148,10 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
 /* Section 2 (prefill phase) with Eq. 7 and a causal mask: append T rows (as eigen_attn_append_kv) and
  * compute the attention output of the T queries, query t over rows [0, len0 + t] where len0 is the
  * length before the call.  T <= max_prefill_tokens.  d_q, d_k, d_v: [B][T][H][d_head] sharing
- * (stride_b, stride_t); d_out: [B][T][H][d_head] with its own strides.  flags: EA_OUT_LOWRANK. */
+ * (stride_b, stride_t); d_out: [B][T][H][d_head] with its own strides.  flags: EA_OUT_LOWRANK; EA_Q_PREPROJECTED
+ * (d_q is the packed [B][T][sum rp_k]); EA_KV_PREPROJECTED (d_k, d_v are the packed [B][T][sum rp_k], [B][T][sum rp_v]).
+ * With either input flag the rows are copied, not multiplied (Eq. 8: the weights carry the bases); a tensor left
+ * d_head-wide in such a call is projected on the CUDA cores. */
 ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, const void* d_v,
                              int32_t T, int64_t stride_b, int64_t stride_t, void* d_out,
                              int64_t out_stride_b, int64_t out_stride_t,

@@ -314,18 +314,38 @@ class EigenAttnLayer:
                                                  _stream_ptr(stream)), "eigen_attn_decode_static")
         return out
 
-    def decode_step(self, q, k, v, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-        pq, _, sbq, _ = self._tok(q, 1)
-        pk, _, sbk, _ = self._tok(k, 1)
-        pv, _, sbv, _ = self._tok(v, 1)
-        if sbk != sbv:
-            k, v = k.contiguous(), v.contiguous()
+    def _packed(self, x: torch.Tensor, T: int, width: int) -> int:
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.torch_dtype and x.shape == (self.B, T, width)
+        return x.data_ptr()
+
+    def decode_step(self, q, k, v, out: Optional[torch.Tensor] = None, q_preprojected: bool = False,
+                    kv_preprojected: bool = False, out_lowrank: bool = False, stream=None) -> torch.Tensor:
+        flags = 0
+        if q_preprojected:
+            flags |= EA_Q_PREPROJECTED
+            pq, sbq = self._packed(q, 1, self.offs_k[-1]), self.offs_k[-1]
+        else:
+            pq, _, sbq, _ = self._tok(q, 1)
+        if kv_preprojected:
+            flags |= EA_KV_PREPROJECTED
+            pk, pv, sbk = self._packed(k, 1, self.offs_k[-1]), self._packed(v, 1, self.offs_v[-1]), 0
+        else:
             pk, _, sbk, _ = self._tok(k, 1)
             pv, _, sbv, _ = self._tok(v, 1)
-        if out is None:
-            out = self._new_out(self.B, 1, self.H, self.d_head)
-        po, _, sbo, _ = self._tok(out, 1)
-        self._check(lib.eigen_attn_decode_step(self.handle, pq, sbq, pk, pv, sbk, po, sbo, 0, _stream_ptr(stream)),
+            if sbk != sbv:
+                k, v = k.contiguous(), v.contiguous()
+                pk, _, sbk, _ = self._tok(k, 1)
+                pv, _, sbv, _ = self._tok(v, 1)
+        if out_lowrank:
+            flags |= EA_OUT_LOWRANK
+            if out is None:
+                out = self._new_out(self.B, 1, self.offs_v[-1])
+            po, sbo = self._packed(out, 1, self.offs_v[-1]), self.offs_v[-1]
+        else:
+            if out is None:
+                out = self._new_out(self.B, 1, self.H, self.d_head)
+            po, _, sbo, _ = self._tok(out, 1)
+        self._check(lib.eigen_attn_decode_step(self.handle, pq, sbq, pk, pv, sbk, po, sbo, flags, _stream_ptr(stream)),
                     "eigen_attn_decode_step")
         return out
 
@@ -339,14 +359,28 @@ class EigenAttnLayer:
                     "eigen_attn_decode_step_host")
         return h_out
 
-    def prefill(self, q, k, v, out: Optional[torch.Tensor] = None, out_lowrank: bool = False, stream=None):
-        pq, T, sb, stt = self._tok(q)
-        pk, _, sbk, stk = self._tok(k, T)
-        pv, _, sbv, stv = self._tok(v, T)
-        assert (sb, stt) == (sbk, stk) == (sbv, stv)
+    def prefill(self, q, k, v, out: Optional[torch.Tensor] = None, out_lowrank: bool = False,
+                q_preprojected: bool = False, kv_preprojected: bool = False, stream=None):
+        T = q.shape[1]
         flags = 0
+        strides = []
+        if q_preprojected:
+            flags |= EA_Q_PREPROJECTED
+            pq = self._packed(q, T, self.offs_k[-1])
+        else:
+            pq, _, sb, stt = self._tok(q, T)
+            strides.append((sb, stt))
+        if kv_preprojected:
+            flags |= EA_KV_PREPROJECTED
+            pk, pv = self._packed(k, T, self.offs_k[-1]), self._packed(v, T, self.offs_v[-1])
+        else:
+            pk, _, sbk, stk = self._tok(k, T)
+            pv, _, sbv, stv = self._tok(v, T)
+            strides += [(sbk, stk), (sbv, stv)]
+        assert len(set(strides)) <= 1                    # the d_head-wide tensors share their strides
+        sb, stt = strides[0] if strides else (0, 0)
         if out_lowrank:
-            flags = EA_OUT_LOWRANK
+            flags |= EA_OUT_LOWRANK
             if out is None:
                 out = self._new_out(self.B, T, self.offs_v[-1])
             assert out.is_contiguous()

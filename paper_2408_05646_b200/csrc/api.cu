@@ -301,7 +301,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
                       int64_t stride_b_out, uint32_t flags, float* partials, const void* k_new,
                       const void* v_new, int64_t kv_stride_b, DecodePlan* plan) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "%s: NULL q or out", who);
-  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK | (k_new ? EA_KV_PREPROJECTED : 0u)))
     return fail(h, EA_ERR_INVALID_ARG, "%s: unknown flag 0x%x", who, flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "%s: the cache is empty", who);
   if (!k_new && h->len - h->max_deficit < 1)
@@ -368,7 +368,9 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p = ea::DecodeParams{};
   p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache;
   p.q = d_q; p.q_stride_b = (flags & EA_Q_PREPROJECTED) ? L.sum_rp_k : stride_b_q;
-  p.k_new = k_new; p.v_new = v_new; p.kv_stride_b = kv_stride_b;
+  p.k_new = k_new; p.v_new = v_new;
+  p.kv_stride_b = (flags & EA_KV_PREPROJECTED) ? L.sum_rp_k : kv_stride_b;
+  p.v_stride_b = (flags & EA_KV_PREPROJECTED) ? L.sum_rp_v : kv_stride_b;
   p.out = d_out; p.out_stride_b = (flags & EA_OUT_LOWRANK) ? L.sum_rp_v : stride_b_out;
   p.partials = partials;
   p.counters = h->opt_fused ? dev_counters(h) : nullptr;
@@ -496,9 +498,9 @@ ea_status do_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q, const voi
     if (sl == EA_OK) h->len += 1;
     return sl;
   }
-  const ea_status st = do_append(h, d_k, d_v, 1, stride_b_kv, stride_b_kv, 0, s);
+  const ea_status st = do_append(h, d_k, d_v, 1, stride_b_kv, stride_b_kv, flags & EA_KV_PREPROJECTED, s);
   if (st != EA_OK) return st;
-  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags, s);
+  return do_decode(h, d_q, stride_b_q, d_out, stride_b_out, flags & ~EA_KV_PREPROJECTED, s);
 }
 
 }  // namespace
@@ -663,7 +665,7 @@ ea_status eigen_attn_decode_step(eigen_attn_t h, const void* d_q, int64_t stride
                                  uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL q or out");
-  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK))
+  if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK | EA_KV_PREPROJECTED))
     return fail(h, EA_ERR_INVALID_ARG, "decode_step: unknown flag 0x%x", flags);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   return do_step(h, d_q, stride_b_q, d_k, d_v, stride_b_kv, d_out, stride_b_out, flags, s);
@@ -741,7 +743,9 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available with a rotary embedding");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
-  if (flags & ~EA_OUT_LOWRANK) return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
+  if (flags & ~(EA_OUT_LOWRANK | EA_Q_PREPROJECTED | EA_KV_PREPROJECTED))
+    return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
+  const bool merged_in = (flags & (EA_Q_PREPROJECTED | EA_KV_PREPROJECTED)) != 0;
   if (T < 1) return fail(h, EA_ERR_SHAPE, "prefill: T = %d", T);
   if (T > h->desc.max_prefill_tokens)
     return fail(h, EA_ERR_CAPACITY, "prefill: T %d exceeds max_prefill_tokens %d", T, h->desc.max_prefill_tokens);
@@ -758,7 +762,20 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   if (h->opt_prefill == 2 && !tc_attn)
     return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
   cudaError_t e;
-  if (tc_shape && in_aligned && h->opt_prefill != 1) {
+  if (merged_in) {
+    // Rank-space rows from merged weights (Eq. 8): nothing to multiply.  K', V' rows are copied into the cache, Q'
+    // rows into the per-head layout the attention kernels read; a tensor the caller left d_head-wide is projected
+    // on the CUDA cores.
+    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
+    if (st != EA_OK) return st;
+    ea::QProjectParams qp{};
+    qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
+    qp.stride_b = stride_b; qp.stride_t = stride_t;
+    qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
+    e = (flags & EA_Q_PREPROJECTED) ? ea::launch_q_scatter(qp, L.sum_rp_k, h->desc.dtype, s, &h->launches)
+                                    : ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill q launch");
+  } else if (tc_shape && in_aligned && h->opt_prefill != 1) {
     // Q', K', V' in one tensor-core launch.  Its rows equal eigen_attn_append_kv's except where the two
     // fp32 summation orders round to different bf16 values (one unit in the last place).
     if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
@@ -811,7 +828,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   p.len0 = len0;
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
-  p.flags = flags; p.status = dev_status(h);
+  p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
   p.tmaps = h->ws + L.off_tmaps;
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   size_t ws_smem = 0;

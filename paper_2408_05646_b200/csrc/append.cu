@@ -118,6 +118,18 @@ __global__ void __launch_bounds__(256) copy_lowrank_rows_kernel(const ProjectPar
   }
 }
 
+// Query rows already in the rank-r space (merged W^Q'): packed [B][T][width] into the per-head Q' scratch.
+template <typename T>
+__global__ void __launch_bounds__(128) scatter_q_lowrank_kernel(const QProjectParams p, int width) {
+  const int h = blockIdx.y;
+  const HeadInfo hd = p.heads[h];
+  const int row = blockIdx.x;                      // flattened (b, t)
+  const int64_t total_rows = static_cast<int64_t>(p.B) * p.T;
+  const T* src = static_cast<const T*>(p.q) + static_cast<int64_t>(row) * width + hd.lr_k_off;
+  T* dst = reinterpret_cast<T*>(p.qp) + static_cast<int64_t>(hd.lr_k_off) * total_rows + static_cast<int64_t>(row) * hd.rp_k;
+  for (int c = threadIdx.x; c < hd.rp_k; c += blockDim.x) dst[c] = c < hd.r_k ? src[c] : from_f<T>(0.f);
+}
+
 int pick_rows_per_cta(int total_rows, int H) {
   // enough CTAs to cover the chip when few rows arrive (decode), larger tiles otherwise
   int rows = 32;
@@ -143,6 +155,14 @@ cudaError_t launch_project_append(const ProjectParams& p, int dtype, cudaStream_
     project_rows_kernel<__nv_bfloat16, false><<<grid, kProjThreads, smem, s>>>(p, nullptr, rows);
   else
     project_rows_kernel<float, false><<<grid, kProjThreads, smem, s>>>(p, nullptr, rows);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_q_scatter(const QProjectParams& q, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches) {
+  dim3 grid(q.B * q.T, q.H);
+  if (dtype == 0) scatter_q_lowrank_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(q, lr_k_width);
+  else scatter_q_lowrank_kernel<float><<<grid, 128, 0, s>>>(q, lr_k_width);
   ++*launches;
   return cudaGetLastError();
 }

@@ -441,10 +441,25 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
   } else if (t < d_head) {
     fx->qraw[t] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + t]);
   }
+  const bool kv_lowrank = (p.flags & 0x4u) != 0;  // rank-space k', v' supplied by the caller (merged W^K', W^V')
+  if (with_new_row && kv_lowrank) {
+    // nothing to project: the packed rows go into the cache (padding columns zero) and into shared memory
+    const int64_t crow = static_cast<int64_t>(b) * p.n_max + n_b;
+    if (t < hd.rp_k) {
+      const T val = t < hd.r_k ? static_cast<const T*>(p.k_new)[b * p.kv_stride_b + hd.lr_k_off + t] : Elem<T>::from_float(0.f);
+      reinterpret_cast<T*>(fx->new_k)[t] = val;
+      reinterpret_cast<T*>(p.cache + hd.k_off)[crow * hd.rp_k + t] = val;
+    }
+    if (t < hd.rp_v) {
+      const T val = t < hd.r_v ? static_cast<const T*>(p.v_new)[b * p.v_stride_b + hd.lr_v_off + t] : Elem<T>::from_float(0.f);
+      reinterpret_cast<T*>(fx->new_v)[t] = val;
+      reinterpret_cast<T*>(p.cache + hd.v_off)[crow * hd.rp_v + t] = val;
+    }
+    with_new_row = false;                         // for the projection below
+  }
   if (with_new_row && t < d_head) {
-    const int64_t src = b * p.kv_stride_b + static_cast<int64_t>(h) * d_head + t;
-    fx->kraw[t] = Elem<T>::to_float(static_cast<const T*>(p.k_new)[src]);
-    fx->vraw[t] = Elem<T>::to_float(static_cast<const T*>(p.v_new)[src]);
+    fx->kraw[t] = Elem<T>::to_float(static_cast<const T*>(p.k_new)[b * p.kv_stride_b + static_cast<int64_t>(h) * d_head + t]);
+    fx->vraw[t] = Elem<T>::to_float(static_cast<const T*>(p.v_new)[b * p.v_stride_b + static_cast<int64_t>(h) * d_head + t]);
   }
   consumer_sync();
   // outputs: [0, nq) = q' columns, [nq, nq + rp_k) = k' columns, then rp_v v' columns

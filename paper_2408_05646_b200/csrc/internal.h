@@ -39,9 +39,10 @@ struct DecodeParams {
   char* cache;
   const void* q;            // [B][1][H][d_head] or packed rank-space [B][sum rp_k]
   int64_t q_stride_b;       // elements
-  const void* k_new;        // [B][1][H][d_head] new token to project, store at row n and attend; or NULL
-  const void* v_new;
-  int64_t kv_stride_b;
+  const void* k_new;        // [B][1][H][d_head] new token to project, store at row n and attend; or NULL.
+  const void* v_new;        //   With flag 0x4 the rows are already rank-space: packed [B][sum rp_k] and [B][sum rp_v]
+  int64_t kv_stride_b;      // batch stride of k_new (and of v_new unless the rows are packed)
+  int64_t v_stride_b;       // batch stride of v_new
   void* out;                // [B][1][H][d_head] or packed [B][sum rp_v]
   int64_t out_stride_b;
   float* partials;          // [(B*H + grid)][part_stride]: m, l, pad, pad, o'[rp_v]
@@ -228,6 +229,8 @@ cudaError_t launch_decode(const DecodeParams& p, int dtype, int grid, size_t sme
                           cudaStream_t s, uint64_t* launches);
 cudaError_t launch_combine(const CombineParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+// Q' rows that are already rank-space (packed [B][T][sum rp_k]) into the per-head layout of the Q' scratch.
+cudaError_t launch_q_scatter(const QProjectParams& p, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);

@@ -248,6 +248,94 @@ def test_merged_weight_flags(B):
             assert_close(got, res[(b, h)], FP32, "lowrank out")
 
 
+def rank_space_inputs(lay, U_k, U_v, q, k, v, dtype):
+    """What a layer with merged weights (Eq. 8) hands over: the packed rank-space tensors q U^K, k U^K, v U^V computed
+    on the host and rounded to the IO dtype, and the d_head-wide tensors whose projections are exactly those rounded
+    rows (x' U^T: since U^T U = I, projecting it returns x'), which is what the oracle receives."""
+    def one(x, U, offs):
+        xn = to_np(x)
+        packed = torch.zeros((x.shape[0], x.shape[1], offs[-1]), dtype=dtype)
+        back = np.zeros_like(xn)
+        for h in range(len(U)):
+            Uh = U[h].astype(np.float64)
+            y = torch.from_numpy(xn[:, :, h, :] @ Uh).to(dtype)
+            packed[:, :, offs[h]:offs[h] + Uh.shape[1]] = y
+            back[:, :, h, :] = y.double().numpy() @ Uh.T
+        return packed.cuda(), back
+    (qp, q_b), (kp, k_b), (vp, v_b) = one(q, U_k, lay.offs_k), one(k, U_k, lay.offs_k), one(v, U_v, lay.offs_v)
+    return qp, kp, vp, q_b, k_b, v_b
+
+
+@pytest.mark.parametrize("dtype,H,d,rk,rv,T", [
+    (FP32, 3, 64, [16, 24, 30], [8, 40, 21], 75),
+    (BF16, 4, 128, [80, 48, 128, 64], [80, 112, 8, 64], 300),
+])
+def test_merged_weight_mode_end_to_end(B, dtype, H, d, rk, rv, T):
+    """Eq. 8: a model whose W^Q, W^K, W^V, W^O carry the bases calls prefill and the decode step with rank-space
+    q', k', v' and takes o' back in rank space.  Prompt (two chunks), then three generated tokens, all three flags;
+    then each input flag alone."""
+    B_, steps = 2, 3
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + steps, dtype, seed_cfg=98, T_q=T + steps)
+    lay = B.EigenAttnLayer(B_, H, d, T + steps, dtype, U_k, U_v, max_prefill_tokens=T)
+    qp, kp, vp, q_b, k_b, v_b = rank_space_inputs(lay, U_k, U_v, q, k, v, dtype)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    want = ref.prefill(q_b[:, :T], k_b[:, :T], v_b[:, :T])
+    cut = T // 2 + 1
+    tol = dict(fp32_rel=2e-5) if dtype == FP32 else {}
+
+    def check_lowrank(got, res, t_axis, what):
+        for b in range(B_):
+            for h in range(H):
+                o = to_np(got[b, :, lay.offs_v[h]:lay.offs_v[h] + rv[h]])
+                exp = res[(b, h)]                                   # [T, d_h] (prefill) or [d_h] (decode): back to rank space
+                exp = (exp if t_axis else exp[None]) @ U_v[h].astype(np.float64)
+                assert_close(torch.from_numpy(o), exp, dtype, f"{what} unit ({b},{h})", **tol)
+                pad = got[b, :, lay.offs_v[h] + rv[h]:lay.offs_v[h + 1]]          # padding lanes of the packed output
+                assert pad.numel() == 0 or float(pad.float().abs().max()) == 0.0
+
+    a = lay.prefill(qp[:, :cut].contiguous(), kp[:, :cut].contiguous(), vp[:, :cut].contiguous(), out_lowrank=True,
+                    q_preprojected=True, kv_preprojected=True)
+    c = lay.prefill(qp[:, cut:T].contiguous(), kp[:, cut:T].contiguous(), vp[:, cut:T].contiguous(), out_lowrank=True,
+                    q_preprojected=True, kv_preprojected=True)
+    lay.poll_status()
+    check_lowrank(torch.cat([a, c], dim=1), want, True, "merged prefill")
+    for s in range(steps):
+        t = T + s
+        o = lay.decode_step(qp[:, t:t + 1].contiguous(), kp[:, t:t + 1].contiguous(), vp[:, t:t + 1].contiguous(),
+                            q_preprojected=True, kv_preprojected=True, out_lowrank=True)
+        ref.append_kv(k_b[:, t:t + 1], v_b[:, t:t + 1])
+        check_lowrank(o, ref.decode(q_b[:, t:t + 1]), False, f"merged decode step {s}")
+    assert lay.len == T + steps
+    # the rows the merged calls stored are the packed rows themselves
+    for h in (0, H - 1):
+        assert torch.equal(lay.cache_rows(h, "k")[:, :T + steps, :rk[h]], kp[:, :, lay.offs_k[h]:lay.offs_k[h] + rk[h]])
+        assert torch.equal(lay.cache_rows(h, "v")[:, :T + steps, :rv[h]], vp[:, :, lay.offs_v[h]:lay.offs_v[h] + rv[h]])
+    # one input flag at a time, d_head-wide output
+    for qf, kvf in ((True, False), (False, True)):
+        lay2 = B.EigenAttnLayer(B_, H, d, T + 1, dtype, U_k, U_v, max_prefill_tokens=T)
+        r2 = oracle_layer(B_, H, d, U_k, U_v)
+        q_in = qp[:, :T].contiguous() if qf else torch.from_numpy(q_b[:, :T]).to(dtype).cuda()
+        k_in = kp[:, :T].contiguous() if kvf else torch.from_numpy(k_b[:, :T]).to(dtype).cuda()
+        v_in = vp[:, :T].contiguous() if kvf else torch.from_numpy(v_b[:, :T]).to(dtype).cuda()
+        q_ref = q_b[:, :T] if qf else to_np(q_in)
+        k_ref = k_b[:, :T] if kvf else to_np(k_in)
+        v_ref = v_b[:, :T] if kvf else to_np(v_in)
+        got = lay2.prefill(q_in, k_in, v_in, q_preprojected=qf, kv_preprojected=kvf)
+        assert_close(got, r2.prefill_dense(q_ref, k_ref, v_ref), dtype, f"prefill q'={qf} kv'={kvf}", **tol)
+        t = T
+        q1 = qp[:, t:t + 1].contiguous() if qf else torch.from_numpy(q_b[:, t:t + 1]).to(dtype).cuda()
+        k1 = kp[:, t:t + 1].contiguous() if kvf else torch.from_numpy(k_b[:, t:t + 1]).to(dtype).cuda()
+        v1 = vp[:, t:t + 1].contiguous() if kvf else torch.from_numpy(v_b[:, t:t + 1]).to(dtype).cuda()
+        o1 = lay2.decode_step(q1, k1, v1, q_preprojected=qf, kv_preprojected=kvf)
+        r2.append_kv(k_b[:, t:t + 1] if kvf else to_np(k1), v_b[:, t:t + 1] if kvf else to_np(v1))
+        assert_close(o1, r2.decode_dense(q_b[:, t:t + 1] if qf else to_np(q1)), dtype, f"step q'={qf} kv'={kvf}", **tol)
+        lay2.set_option(B.EA_OPT_DECODE_FUSED, 0)                   # the separate-launch form of the same step
+        lay2.set_len(T)
+        o2 = lay2.decode_step(q1, k1, v1, q_preprojected=qf, kv_preprojected=kvf)
+        assert_close(o2, r2.decode_dense(q_b[:, t:t + 1] if qf else to_np(q1)), dtype, f"unfused step q'={qf} kv'={kvf}", **tol)
+        lay2.poll_status()
+
+
 @pytest.mark.parametrize("dtype,H,d,rk,rv,T", [
     (FP32, 2, 64, [32, 20], [16, 40], 75),
     (BF16, 4, 128, [80, 48, 128, 64], [80, 112, 8, 64], 200),
