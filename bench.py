@@ -113,7 +113,7 @@ class ClockSampler:
 # the CPU oracle leg (also the --impl reference arm)
 # ----------------------------------------------------------------------------------------------
 
-QUANT_LEGS = ((4, 32),)                     # (bits, group) of the quantised-cache entries of the workload table
+QUANT_LEGS = ((4, 32), (3, 32))                   # (bits, group) of the quantised-cache entries of the workload table
 VARIANT = {"alibi": False, "rope": False}   # --alibi / --rope: position schemes on both sides (decode workloads)
 ROPE_BASE = 10000.0
 

@@ -196,7 +196,8 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
  *     s = half(min(max|x| / (2^(bits-1) - 1), 65504)),  c = clip(rint(x / s)),  x^ = c * s ,
  * x being the stored 16-bit row, the two divisions IEEE single precision, rint to nearest even.  Rows that do
  * not fill a block of `group` tokens yet stay in the 16-bit cache and are attended from there.
- * Built: bits == 4, group in {16, 32, 64, 128}, bf16 layers (EA_ERR_UNSUPPORTED otherwise).
+ * Built: bits in {3, 4} (every Eigen Attention row of Table 8), group in {16, 32, 64, 128}, bf16 layers
+ * (EA_ERR_UNSUPPORTED otherwise).
  *
  * quant_bytes:  size of the caller's quantised buffer for this layer (host arithmetic).
  * quant_attach: hands the library that DEVICE buffer (256-byte aligned, >= quant_bytes; owned by the caller, as
@@ -207,11 +208,20 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
  *               are; a caller that wants the memory back keeps only a window of the 16-bit cache.
  * decode_quant: eigen_attn_decode (same arguments, flags and ALiBi bias) over the codes of rows [0, quant_len)
  *               and the 16-bit rows [quant_len, len).  Not available with a rotary embedding.
- * quant_len:    rows currently held as codes.  eigen_attn_set_len below quant_len rounds it down to a whole block.
+ * quant_len:    rows currently held as codes (of the sequence that holds most, while lengths differ).
+ *               eigen_attn_set_len below quant_len rounds it down to a whole block.
+ * quant_lens:   the same per sequence: HOST array [batch].  While lengths differ (eigen_attn_set_lens) every sequence
+ *               keeps its own count: set_lens keeps a sequence's codes of the complete blocks below its new length,
+ *               quant_sync quantises each sequence's own complete blocks, decode_quant attends each sequence's own
+ *               codes and 16-bit tail.
  * quant_layout: where head `head` lives in the buffer: byte offset of its slab [B][n_max / group][block_bytes],
  *               and inside a block the offsets of the key scales [rp_k] halves, the value codes and the value
- *               scales [ceil(rp_v / group)][group] halves; key codes sit at offset 0.  Codes are 32-bit words
- *               [rp / 8][group]: word j of row i holds channels 8j..8j+7, channel 8j+k in bits 4k..4k+3 as c + 8. */
+ *               scales [ceil(rp_v / group)][group] halves; key codes sit at offset 0.  A code area is [rp / 8][group]
+ *               units, unit j of row i holding channels 8j..8j+7.  4-bit: a unit is a 32-bit word, channel 8j+k in
+ *               bits 4k..4k+3 as c + 8.  3-bit: a unit is 24 bits, channel 8j+k in bits 3k..3k+2 as c + 4, kept as
+ *               two planes: the low 16 bits of all units ([rp / 8][group] halfwords), then their high 8 bits
+ *               ([rp / 8][group] bytes).  Keys therefore cost exactly bits + 16/group bits per (padded) element,
+ *               the accounting behind Table 8; a value row pays one scale per started group of its rp_v channels. */
 ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, size_t* bytes);
 ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
                                   void* cuda_stream);
@@ -219,6 +229,7 @@ ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream);
 ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                   int64_t stride_b_out, uint32_t flags, void* cuda_stream);
 ea_status eigen_attn_quant_len(eigen_attn_t h, int32_t* qlen);
+ea_status eigen_attn_quant_lens(eigen_attn_t h, int32_t* qlens);
 ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_offset, size_t* block_bytes,
                                   size_t* k_scale_offset, size_t* v_code_offset, size_t* v_scale_offset);
 
@@ -236,9 +247,9 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
  * sequence's own rows (ALiBi positions count from the sequence's own end); decode needs lens[b] >= 1 for every
  * b (EA_ERR_SHAPE otherwise).  The split-KV work decomposition follows the true lengths, so a step costs what
  * the rows actually cached cost.  batch <= 1024.  eigen_attn_set_len returns to equal lengths.
- * With a rotary embedding each sequence's query sits at its own last position.  Not available
- * (EA_ERR_UNSUPPORTED) with a quantised cache attached; while lengths differ,
- * prefill and the quantised calls return EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
+ * With a rotary embedding each sequence's query sits at its own last position.  With a quantised cache attached
+ * every sequence keeps its own count of rows held as codes (eigen_attn_quant_lens).  While lengths differ,
+ * prefill returns EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
  * (asynchronous; the array may be reused when the call returns), so the calls that follow must run on that
  * stream or be ordered after it. */
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);

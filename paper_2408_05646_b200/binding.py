@@ -78,6 +78,7 @@ SYMBOLS = {
     "eigen_attn_quant_sync": (_i32, [_vp, _vp]),
     "eigen_attn_decode_quant": (_i32, [_vp, _vp, _i64, _vp, _i64, _u32, _vp]),
     "eigen_attn_quant_len": (_i32, [_vp, ctypes.POINTER(_i32)]),
+    "eigen_attn_quant_lens": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "eigen_attn_quant_layout": (_i32, [_vp, _i32] + [ctypes.POINTER(_sz)] * 5),
     "eigen_attn_launch_count": (_i32, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "eigen_attn_set_decode_events": (_i32, [_vp, _vp, _vp]),
@@ -283,6 +284,11 @@ class EigenAttnLayer:
         n = ctypes.c_int32(0)
         self._check(lib.eigen_attn_quant_len(self.handle, ctypes.byref(n)), "eigen_attn_quant_len")
         return n.value
+
+    def quant_lens(self):
+        arr = (ctypes.c_int32 * self.B)()
+        self._check(lib.eigen_attn_quant_lens(self.handle, arr), "eigen_attn_quant_lens")
+        return list(arr)
 
     def decode_quant(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, q_preprojected: bool = False,
                      out_lowrank: bool = False, stream=None) -> torch.Tensor:

@@ -44,7 +44,7 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0, off_qlens = 0;
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -118,6 +118,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_rope = off;     off = align_up(off + 64 * sizeof(double));   // inverse frequencies of the rotary embedding
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->off_deficit = off;  off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // unequal lengths
+  L->off_qlens = off;    off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // ... of the quantised copy
   L->workspace_bytes = off;
 }
 
@@ -205,7 +206,9 @@ struct eigen_attn {
   // quantised copy of the cache (Section 5.3), attached by the caller
   char* qcache = nullptr;
   int q_group = 0;
-  int32_t qlen = 0;       // rows held as codes (a multiple of q_group)
+  int q_bits = 0;
+  int32_t qlen = 0;       // rows held as codes (a multiple of q_group); with unequal lengths the largest of `qlens`
+  std::vector<int32_t> qlens;   // [B]: rows of each sequence held as codes, kept (and uploaded) while lengths differ
   int q_max_stage_bytes = 0;
   std::vector<ea::QuantHead> qheads;
   char err[256];
@@ -227,7 +230,7 @@ ea_status cuda_fail(eigen_attn_t h, cudaError_t e, const char* what) {
 }
 
 // Layout of the quantised buffer for group size G: the per-head table, then one slab per head.
-size_t make_quant_layout(const eigen_attn* h, int G, std::vector<ea::QuantHead>* qheads, int* max_stage_bytes) {
+size_t make_quant_layout(const eigen_attn* h, int bits, int G, std::vector<ea::QuantHead>* qheads, int* max_stage_bytes) {
   const int H = h->desc.n_heads;
   const int64_t blocks_max = h->desc.n_max / G;
   qheads->resize(H);
@@ -238,9 +241,9 @@ size_t make_quant_layout(const eigen_attn* h, int G, std::vector<ea::QuantHead>*
     ea::QuantHead& q = (*qheads)[i];
     memset(&q, 0, sizeof(q));
     q.nvg = (hi.rp_v + G - 1) / G;
-    q.ks_off = G * hi.rp_k / 2;
+    q.ks_off = G * hi.rp_k * bits / 8;           // a multiple of 16: G % 16 == 0, rp % 8 == 0
     q.vc_off = q.ks_off + 2 * hi.rp_k;
-    q.vs_off = q.vc_off + G * hi.rp_v / 2;
+    q.vs_off = q.vc_off + G * hi.rp_v * bits / 8;
     q.block_bytes = q.vs_off + 2 * G * q.nvg;
     q.slab_off = static_cast<int64_t>(off);
     off = align_up(off + static_cast<size_t>(h->desc.batch) * blocks_max * q.block_bytes);
@@ -252,7 +255,7 @@ size_t make_quant_layout(const eigen_attn* h, int G, std::vector<ea::QuantHead>*
 }
 
 ea_status check_quant_args(eigen_attn_t h, const char* who, int32_t bits, int32_t group) {
-  if (bits != 4) return fail(h, EA_ERR_UNSUPPORTED, "%s: %d-bit codes (4 is built)", who, bits);
+  if (bits != 3 && bits != 4) return fail(h, EA_ERR_UNSUPPORTED, "%s: %d-bit codes (3 and 4 are built)", who, bits);
   if (group != 16 && group != 32 && group != 64 && group != 128)
     return fail(h, EA_ERR_UNSUPPORTED, "%s: group %d (16, 32, 64 or 128)", who, group);
   if (h->desc.dtype != EA_BF16) return fail(h, EA_ERR_UNSUPPORTED, "%s: needs a bf16 layer", who);
@@ -854,6 +857,9 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (len < 0 || len > h->desc.n_max)
     return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %d]", len, h->desc.n_max);
+  if (h->q_group && h->max_deficit > 0)      // leaving unequal lengths: rows every sequence holds as codes
+    for (int b = 0; b < h->desc.batch; ++b)
+      if (h->qlens[b] < h->qlen) h->qlen = h->qlens[b];
   h->len = len;
   h->max_deficit = 0;     // every sequence holds len rows again
   if (h->q_group && h->qlen > len) h->qlen = len / h->q_group * h->q_group;   // rows past len are forgotten
@@ -862,7 +868,6 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
 
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream) {
   if (!h || !lens) return EA_ERR_INVALID_ARG;
-  if (h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_lens: not available with a quantised cache attached");
   const int B = h->desc.batch;
   if (B > ea::kMaxRaggedBatch)
     return fail(h, EA_ERR_UNSUPPORTED, "set_lens: batch %d exceeds %d", B, ea::kMaxRaggedBatch);
@@ -883,6 +888,27 @@ ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_st
     const cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_deficit, deficit.data(), sizeof(int32_t) * B,
                                           cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(h, e, "set_lens: upload");
+  }
+  if (h->q_group) {
+    // a sequence keeps the codes of its complete blocks below its new length
+    std::vector<int32_t> q(B);
+    int32_t qmax = 0, qmin = INT32_MAX;
+    for (int b = 0; b < B; ++b) {
+      const int32_t had = h->max_deficit > 0 ? h->qlens[b] : h->qlen;
+      const int32_t cap = lens[b] / h->q_group * h->q_group;
+      q[b] = had < cap ? had : cap;
+      if (q[b] > qmax) qmax = q[b];
+      if (q[b] < qmin) qmin = q[b];
+    }
+    if (widest > 0) {
+      const cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_qlens, q.data(), sizeof(int32_t) * B, cudaMemcpyHostToDevice,
+                                            static_cast<cudaStream_t>(cuda_stream));
+      if (e != cudaSuccess) return cuda_fail(h, e, "set_lens: upload");
+      h->qlens.swap(q);
+      h->qlen = qmax;
+    } else {
+      h->qlen = qmin;
+    }
   }
   h->deficit.swap(deficit);
   h->len = longest;
@@ -1042,16 +1068,15 @@ ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, si
   const ea_status st = check_quant_args(h, "quant_bytes", bits, group);
   if (st != EA_OK) return st;
   std::vector<ea::QuantHead> qh;
-  *bytes = make_quant_layout(h, group, &qh, nullptr);
+  *bytes = make_quant_layout(h, bits, group, &qh, nullptr);
   return EA_OK;
 }
 
 ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
                                   void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!d_qcache) {             // detach
-    h->qcache = nullptr; h->q_group = 0; h->qlen = 0;
+    h->qcache = nullptr; h->q_group = 0; h->q_bits = 0; h->qlen = 0;
     return EA_OK;
   }
   const ea_status st = check_quant_args(h, "quant_attach", bits, group);
@@ -1059,7 +1084,7 @@ ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, v
   if (reinterpret_cast<uintptr_t>(d_qcache) % kAlign) return fail(h, EA_ERR_INVALID_ARG, "quant_attach: buffer not 256-byte aligned");
   std::vector<ea::QuantHead> qh;
   int widest = 0;
-  const size_t need = make_quant_layout(h, group, &qh, &widest);
+  const size_t need = make_quant_layout(h, bits, group, &qh, &widest);
   if (bytes < need) return fail(h, EA_ERR_CAPACITY, "quant_attach: %zu bytes given, %zu needed", bytes, need);
   if (ea::decode_quant_smem_bytes(widest, h->L.max_rp_v) > static_cast<size_t>(kSmemLimit))
     return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: a stage of 128 rows does not fit in shared memory");
@@ -1069,7 +1094,13 @@ ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, v
   if (e != cudaSuccess) return cuda_fail(h, e, "quant_attach");
   h->qcache = static_cast<char*>(d_qcache);
   h->q_group = group;
+  h->q_bits = bits;
   h->qlen = 0;
+  if (h->max_deficit > 0) {    // attached to a batch of unequal lengths: no sequence has codes yet
+    h->qlens.assign(h->desc.batch, 0);
+    e = cudaMemsetAsync(h->ws + h->L.off_qlens, 0, sizeof(int32_t) * h->desc.batch, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "quant_attach");
+  }
   h->q_max_stage_bytes = widest;
   h->qheads.swap(qh);
   return EA_OK;
@@ -1086,16 +1117,32 @@ void fill_quant_params(eigen_attn_t h, ea::QuantParams* p) {
   p->part_stride = h->L.part_stride;
   p->B = h->desc.batch; p->H = h->desc.n_heads; p->d_head = h->desc.d_head;
   p->n = h->len; p->n_max = h->desc.n_max;
-  p->nq = h->qlen; p->group = h->q_group; p->blocks_max = h->desc.n_max / h->q_group;
+  p->nq = h->qlen; p->group = h->q_group; p->bits = h->q_bits; p->blocks_max = h->desc.n_max / h->q_group;
+  p->deficit = dev_deficit(h);
+  p->qlens = h->max_deficit > 0 ? reinterpret_cast<const int32_t*>(h->ws + h->L.off_qlens) : nullptr;
 }
 }  // namespace
 
 ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "quant_sync: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "quant_sync: no quantised buffer attached");
   const int G = h->q_group;
-  const int b0 = h->qlen / G, b1 = h->len / G;
+  int b0 = h->qlen / G, b1 = h->len / G;
+  const bool ragged = h->max_deficit > 0;
+  std::vector<int32_t> q_new;
+  if (ragged) {
+    // every sequence's own complete blocks: the launch spans the union of the ranges, the kernel skips by sequence
+    q_new.resize(h->desc.batch);
+    b0 = INT32_MAX; b1 = 0;
+    for (int b = 0; b < h->desc.batch; ++b) {
+      const int lo = h->qlens[b] / G, hi = (h->len - h->deficit[b]) / G;
+      q_new[b] = (hi > lo ? hi : lo) * G;
+      if (hi > lo) {
+        if (lo < b0) b0 = lo;
+        if (hi > b1) b1 = hi;
+      }
+    }
+  }
   if (b1 <= b0) return EA_OK;
   ea::QuantParams p;
   fill_quant_params(h, &p);
@@ -1106,7 +1153,24 @@ ea_status eigen_attn_quant_sync(eigen_attn_t h, void* cuda_stream) {
     const cudaError_t e = ea::launch_quantize_blocks(p, s, &h->launches);
     if (e != cudaSuccess) return cuda_fail(h, e, "quant_sync launch");
   }
-  h->qlen = b1 * G;
+  if (ragged) {
+    // the kernel read the old per-sequence counts; the new ones follow it on the stream
+    const cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_qlens, q_new.data(), sizeof(int32_t) * q_new.size(),
+                                          cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "quant_sync: upload");
+    h->qlens.swap(q_new);
+    h->qlen = 0;
+    for (int32_t q : h->qlens) if (q > h->qlen) h->qlen = q;
+  } else {
+    h->qlen = b1 * G;
+  }
+  return EA_OK;
+}
+
+ea_status eigen_attn_quant_lens(eigen_attn_t h, int32_t* qlens) {
+  if (!h || !qlens) return EA_ERR_INVALID_ARG;
+  if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "quant_lens: no quantised buffer attached");
+  for (int b = 0; b < h->desc.batch; ++b) qlens[b] = h->max_deficit > 0 ? h->qlens[b] : h->qlen;
   return EA_OK;
 }
 
@@ -1133,12 +1197,11 @@ ea_status eigen_attn_quant_layout(eigen_attn_t h, int32_t head, size_t* slab_off
 ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t stride_b_q, void* d_out,
                                   int64_t stride_b_out, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "decode_quant: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!h->qcache) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: no quantised buffer attached");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: NULL q or out");
   if (flags & ~(EA_Q_PREPROJECTED | EA_OUT_LOWRANK)) return fail(h, EA_ERR_INVALID_ARG, "decode_quant: unknown flag 0x%x", flags);
   if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "decode_quant: not available with a rotary embedding");
-  if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode_quant: the cache is empty");
+  if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_quant: the cache is empty (for some sequence)");
   const Layout& L = h->L;
   ea::QuantParams p;
   fill_quant_params(h, &p);

@@ -185,10 +185,13 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
 };
 
 // Quantised copy of the cache (Section 5.3 of the paper): per head a slab [B][blocks_max][block_bytes]; a block
-// holds G consecutive rows of one sequence as 4-bit codes (code + 8 in a nibble, eight channels per 32-bit word,
-// channel 8j+k in bits 4k..4k+3) and half-precision scales:
-//   K codes  [rp_k/8][G] words     K scales [rp_k] halves        (one scale per channel and block)
-//   V codes  [rp_v/8][G] words     V scales [nvg][G] halves      (one scale per row and G channels)
+// holds G consecutive rows of one sequence as integer codes and half-precision scales:
+//   K codes  [rp_k/8][G] units     K scales [rp_k] halves        (one scale per channel and block)
+//   V codes  [rp_v/8][G] units     V scales [nvg][G] halves      (one scale per row and G channels)
+// A unit holds the eight channels 8j..8j+7 of one row.  4-bit codes: a 32-bit word, channel 8j+k in bits 4k..4k+3
+// as code + 8.  3-bit codes: 24 bits, channel 8j+k in bits 3k..3k+2 as code + 4, stored as two planes, the low 16
+// bits of every unit ([rp/8][G] halfwords) followed by the high 8 bits of every unit ([rp/8][G] bytes): exactly
+// 3 bits per element, and a warp's loads of either plane are consecutive.
 struct QuantHead {
   int64_t slab_off;        // byte offset of the head's slab in the quantised buffer
   int32_t block_bytes;
@@ -209,11 +212,14 @@ struct QuantParams {
   int64_t out_stride_b;
   float* partials;          // [B*H][splits][part_stride]: m, l, pad, pad, o'[rp_v]
   int* status;
+  const int32_t* deficit;   // [B]: sequence b holds n - deficit[b] rows (unequal lengths); NULL = all hold n
+  const int32_t* qlens;     // [B]: rows of sequence b held as codes (unequal lengths); NULL = all hold nq
   int32_t part_stride;
   int32_t B, H, d_head;
   int32_t n, n_max;
-  int32_t nq;               // rows held as codes (a multiple of group)
+  int32_t nq;               // rows held as codes (a multiple of group); the longest sequence's with unequal lengths
   int32_t group;            // G: 16, 32, 64 or 128
+  int32_t bits;             // 3 or 4
   int32_t blocks_max;       // blocks per sequence the buffer holds = n_max / G
   int32_t nst;              // stages of 128 rows per unit = ceil(nq / 128)
   int32_t splits;           // CTAs per unit

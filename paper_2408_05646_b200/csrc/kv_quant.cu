@@ -1,7 +1,8 @@
 // Quantised rank-r cache (Section 5.3 of the paper, "Eigen Attention with Quantization"; sizes in Table 8):
-// keys per channel, values per token, integer codes of 4 bits with one half-precision scale per group of G.
+// keys per channel, values per token, integer codes of 3 or 4 bits with one half-precision scale per group of G.
 //
-//   s = half( min(max|x| / 7, 65504) ),   c = clip( rint(x / s), -7, 7 ),   x^ = c * s      (c + 8 is stored)
+//   qmax = 2^(bits-1) - 1,  s = half( min(max|x| / qmax, 65504) ),  c = clip( rint(x / s), -qmax, qmax ),  x^ = c * s
+//   (c + qmax + 1 is stored)
 //
 // A key group is G consecutive tokens of one channel, a value group is G consecutive channels of one token.
 // Rows that do not fill a block of G tokens yet stay in the 16-bit cache and are attended from there.
@@ -36,10 +37,11 @@ constexpr int kStageRows = 128;
 
 // ---------------------------------------------------------------- quantiser
 
-__device__ __forceinline__ uint32_t code_nibble(float x, float s) {
+// clip(rint(x / s), -qmax, qmax) + qmax + 1: the stored (unsigned) code
+__device__ __forceinline__ uint32_t stored_code(float x, float s, float qmax) {
   float c = s > 0.f ? rintf(x / s) : 0.f;
-  c = fminf(fmaxf(c, -7.f), 7.f);
-  return static_cast<uint32_t>(static_cast<int>(c) + 8);
+  c = fminf(fmaxf(c, -qmax), qmax);
+  return static_cast<uint32_t>(static_cast<int>(c + qmax) + 1);
 }
 
 __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantParams p) {
@@ -51,6 +53,11 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
   const HeadInfo hd = p.heads[h];
   const QuantHead qh = p.qheads[h];
   const int G = p.group;
+  if (p.qlens != nullptr) {   // unequal lengths: this sequence's own range of complete blocks not quantised yet
+    const int n_b = p.n - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);
+    if (blk < __ldg(p.qlens + b) / G || blk >= n_b / G) return;
+  }
+  const float qmax = p.bits == 3 ? 3.f : 7.f;
   const int64_t row0 = static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(blk) * G;
   char* dst = p.qcache + qh.slab_off + (static_cast<int64_t>(b) * p.blocks_max + blk) * qh.block_bytes;
 
@@ -65,7 +72,7 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
       for (int c = tid; c < rp; c += kQThreads) {
         float amax = 0.f;
         for (int r = 0; r < G; ++r) amax = fmaxf(amax, fabsf(__bfloat162float(tile[r * rp + c])));
-        const __half s16 = __float2half_rn(fminf(amax / 7.f, 65504.f));
+        const __half s16 = __float2half_rn(fminf(amax / qmax, 65504.f));
         ks[c] = s16;
         scale_sm[c] = __half2float(s16);
       }
@@ -76,13 +83,13 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
         const int c1 = min(rp, (g + 1) * G);
         float amax = 0.f;
         for (int c = g * G; c < c1; ++c) amax = fmaxf(amax, fabsf(__bfloat162float(tile[r * rp + c])));
-        const __half s16 = __float2half_rn(fminf(amax / 7.f, 65504.f));
+        const __half s16 = __float2half_rn(fminf(amax / qmax, 65504.f));
         vs[i] = s16;
         scale_sm[i] = __half2float(s16);
       }
     }
     __syncthreads();
-    uint32_t* codes = reinterpret_cast<uint32_t*>(dst + (pass ? qh.vc_off : 0));
+    char* code_base = dst + (pass ? qh.vc_off : 0);
     const int words = (rp / 8) * G;
     for (int i = tid; i < words; i += kQThreads) {
       const int j = i / G, r = i - j * G;
@@ -91,9 +98,14 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
       for (int k = 0; k < 8; ++k) {
         const int c = 8 * j + k;
         const float s = pass ? scale_sm[(c / G) * G + r] : scale_sm[c];
-        w |= code_nibble(__bfloat162float(tile[r * rp + c]), s) << (4 * k);
+        w |= stored_code(__bfloat162float(tile[r * rp + c]), s, qmax) << (p.bits * k);
       }
-      codes[i] = w;
+      if (p.bits == 4) {
+        reinterpret_cast<uint32_t*>(code_base)[i] = w;
+      } else {                // two planes: low 16 bits of every unit, then the high 8 bits
+        reinterpret_cast<uint16_t*>(code_base)[i] = static_cast<uint16_t>(w);
+        reinterpret_cast<uint8_t*>(code_base + 2 * words)[i] = static_cast<uint8_t>(w >> 16);
+      }
     }
     __syncthreads();          // the tile and the scales are reused by the second pass
   }
@@ -128,27 +140,52 @@ __device__ __forceinline__ float low_plus_high(unsigned long long v) {
 
 // Eight codes of a word as four packed float pairs (exact small integers in -7..7; a nibble 0 gives -8).
 // Nibbles 0..3 sit at bits 0, 4, 8, 12 and meet the exponents of 2^23, 2^19, 2^15, 2^11; nibbles 4..7 do the
-// same after a shift by 16, so two packed constants serve the whole word.
+// same after a shift by 16, so two packed constants serve the whole word.  3-bit codes: fields at bits 0, 3, 6, 9
+// meet 2^23, 2^20, 2^17, 2^14, fields 4..7 after a shift by 12; the stored code is c + 4.
 struct Consts {
   unsigned long long c01, c23;
-  uint32_t e23, e19, e15, e11;         // exponent patterns of 2^23, 2^19, 2^15, 2^11
+  uint32_t e23, e19, e15, e11;         // exponent patterns of 2^23, 2^19, 2^15, 2^11 (3-bit: 2^23, 2^20, 2^17, 2^14)
 };
 // The exponent patterns come in as kernel arguments, not as literals: (w & mask) | pattern is one logic
 // instruction when the pattern sits in a register; with two literals the compiler emits a second logic
 // instruction and a move per element (counted on the device: 327 logic + 160 moves per row instead of 160).
+template <int BITS>
 __device__ __forceinline__ Consts make_consts(const QuantParams& p) {
   Consts c;
   c.e23 = p.magic[0]; c.e19 = p.magic[1]; c.e15 = p.magic[2]; c.e11 = p.magic[3];
-  c.c01 = pair_of(-8388616.f, -524296.f);          // -(2^23 + 8), -(2^19 + 8)
-  c.c23 = pair_of(-32776.f, -2056.f);              // -(2^15 + 8), -(2^11 + 8)
+  if (BITS == 4) {
+    c.c01 = pair_of(-8388616.f, -524296.f);          // -(2^23 + 8), -(2^19 + 8)
+    c.c23 = pair_of(-32776.f, -2056.f);              // -(2^15 + 8), -(2^11 + 8)
+  } else {
+    c.c01 = pair_of(-8388612.f, -1048580.f);         // -(2^23 + 4), -(2^20 + 4)
+    c.c23 = pair_of(-131076.f, -16388.f);            // -(2^17 + 4), -(2^14 + 4)
+  }
   return c;
 }
+template <int BITS>
 __device__ __forceinline__ void codes_to_floats(uint32_t w, const Consts& k, unsigned long long (&f)[4]) {
-  const uint32_t u = w >> 16;
-  f[0] = add2p(pair_of((w & 0x000Fu) | k.e23, (w & 0x00F0u) | k.e19), k.c01);
-  f[1] = add2p(pair_of((w & 0x0F00u) | k.e15, (w & 0xF000u) | k.e11), k.c23);
-  f[2] = add2p(pair_of((u & 0x000Fu) | k.e23, (u & 0x00F0u) | k.e19), k.c01);
-  f[3] = add2p(pair_of((u & 0x0F00u) | k.e15, (u & 0xF000u) | k.e11), k.c23);
+  if (BITS == 4) {
+    const uint32_t u = w >> 16;
+    f[0] = add2p(pair_of((w & 0x000Fu) | k.e23, (w & 0x00F0u) | k.e19), k.c01);
+    f[1] = add2p(pair_of((w & 0x0F00u) | k.e15, (w & 0xF000u) | k.e11), k.c23);
+    f[2] = add2p(pair_of((u & 0x000Fu) | k.e23, (u & 0x00F0u) | k.e19), k.c01);
+    f[3] = add2p(pair_of((u & 0x0F00u) | k.e15, (u & 0xF000u) | k.e11), k.c23);
+  } else {
+    const uint32_t u = w >> 12;
+    f[0] = add2p(pair_of((w & 0x007u) | k.e23, (w & 0x038u) | k.e19), k.c01);
+    f[1] = add2p(pair_of((w & 0x1C0u) | k.e15, (w & 0xE00u) | k.e11), k.c23);
+    f[2] = add2p(pair_of((u & 0x007u) | k.e23, (u & 0x038u) | k.e19), k.c01);
+    f[3] = add2p(pair_of((u & 0x1C0u) | k.e15, (u & 0xE00u) | k.e11), k.c23);
+  }
+}
+// The unit (eight channels 8j..8j+7) of row `ri` of a block's code area: a word, or the two planes of 3-bit codes
+// (`units` = units of the whole area = (rp / 8) * G).
+template <int BITS, int G>
+__device__ __forceinline__ uint32_t load_unit(const unsigned char* area, int units, int j, int ri) {
+  if (BITS == 4) return reinterpret_cast<const uint32_t*>(area)[j * G + ri];
+  const uint32_t lo = reinterpret_cast<const uint16_t*>(area)[j * G + ri];
+  const uint32_t hi = area[2 * units + j * G + ri];
+  return lo | (hi << 16);
 }
 __device__ __forceinline__ void bf16x8_to_floats(const uint4& x, unsigned long long (&f)[4]) {
   f[0] = pair_of(x.x << 16, x.x & 0xffff0000u);
@@ -159,7 +196,7 @@ __device__ __forceinline__ void bf16x8_to_floats(const uint4& x, unsigned long l
 
 // NW: 8-channel words a row can have (widest padded rank / 8); G: group size (row offsets inside a block become
 // immediates); FULL: every head has exactly NW words of keys and of values (no per-word guards).
-template <int NW, int MINB, int G, bool FULL>
+template <int NW, int MINB, int G, bool FULL, int BITS>
 __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const QuantParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   QuantSmemHeader* hdr = reinterpret_cast<QuantSmemHeader*>(smem);
@@ -172,12 +209,15 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   const QuantHead qh = p.qheads[h];
   constexpr int gshift = G == 16 ? 4 : G == 32 ? 5 : G == 64 ? 6 : 7;
   constexpr int bps = kStageRows >> gshift;                      // blocks per stage
-  const int nqb = p.nq >> gshift;                             // blocks held as codes
+  const int n_b = p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;      // this sequence's rows
+  const int nq_b = p.qlens != nullptr ? __ldg(p.qlens + b) : p.nq;              // ... of which held as codes
+  const int nqb = nq_b >> gshift;                             // blocks held as codes
   const int nwk = hd.rp_k >> 3, nwv = hd.rp_v >> 3;
   const int stage_stride = (bps * qh.block_bytes + 127) & ~127;
 
-  const int per = (p.nst + p.splits - 1) / p.splits;
-  const int s_lo = min(p.nst, split * per), s_hi = min(p.nst, s_lo + per);
+  const int nst_b = (nq_b + kStageRows - 1) / kStageRows;     // the splits divide the sequence's own stages
+  const int per = (nst_b + p.splits - 1) / p.splits;
+  const int s_lo = min(nst_b, split * per), s_hi = min(nst_b, s_lo + per);
   const char* slab = p.qcache + qh.slab_off + static_cast<int64_t>(b) * p.blocks_max * qh.block_bytes;
 
   if (tid == 0) {
@@ -220,13 +260,13 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
   }
   __syncthreads();
 
-  const Consts kc = make_consts(p);
+  const Consts kc = make_consts<BITS>(p);
   unsigned long long o[NW * 4];
 #pragma unroll
   for (int i = 0; i < NW * 4; ++i) o[i] = 0ull;
   float m = -INFINITY, l = 0.f;
   const float slope2 = hd.alibi_slope2;
-  const int pos_q = p.n - 1;
+  const int pos_q = n_b - 1;
   // online softmax of one score: returns the weight of the row under the (possibly raised) running maximum
   // (the maximum is only raised when a score exceeds it by more than 8: weights stay below 2^8, and a warp
   // leaves the common path only when one of its lanes meets such a score)
@@ -266,14 +306,13 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
     const int blk = tid >> gshift, ri = tid & (G - 1);
     if (blk < nblk) {
       const unsigned char* bb = st + blk * qh.block_bytes;
-      const uint32_t* kw = reinterpret_cast<const uint32_t*>(bb) + ri;
       const float* qsr = qs_w + (G >= 32 ? 0 : (lane >> 4) * 128);
       unsigned long long a0 = 0ull, a1 = 0ull, a2 = 0ull, a3 = 0ull;
 #pragma unroll
       for (int j = 0; j < NW; ++j)
         if (FULL || j < nwk) {
           unsigned long long f[4];
-          codes_to_floats(kw[j * G], kc, f);
+          codes_to_floats<BITS>(load_unit<BITS, G>(bb, nwk * G, j, ri), kc, f);
           const ulonglong2 q0 = *reinterpret_cast<const ulonglong2*>(qsr + 8 * j);
           const ulonglong2 q1 = *reinterpret_cast<const ulonglong2*>(qsr + 8 * j + 4);
           a0 = fma2p(f[0], q0.x, a0); a1 = fma2p(f[1], q0.y, a1);
@@ -282,7 +321,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
       const int j_abs = s * kStageRows + tid;
       const float pr = weight(fmaf(slope2, static_cast<float>(j_abs - pos_q),
                                    low_plus_high(add2p(add2p(a0, a1), add2p(a2, a3)))));
-      const uint32_t* vw = reinterpret_cast<const uint32_t*>(bb + qh.vc_off) + ri;
+      const unsigned char* varea = bb + qh.vc_off;
       const __half* vs = reinterpret_cast<const __half*>(bb + qh.vs_off) + ri;
 #pragma unroll
       for (int j = 0; j < NW; ++j)
@@ -290,7 +329,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
           const float sv = pr * __half2float(vs[((8 * j) >> gshift) * G]);
           const unsigned long long svp = pair_of(sv, sv);
           unsigned long long f[4];
-          codes_to_floats(vw[j * G], kc, f);
+          codes_to_floats<BITS>(load_unit<BITS, G>(varea, nwv * G, j, ri), kc, f);
 #pragma unroll
           for (int i = 0; i < 4; ++i) o[4 * j + i] = fma2p(f[i], svp, o[4 * j + i]);
         }
@@ -307,7 +346,7 @@ __global__ void __launch_bounds__(kQThreads, MINB) decode_quant_kernel(const Qua
 
   // rows that are not quantised yet, straight from the 16-bit cache (the last split takes them)
   if (split == p.splits - 1 && !aborted) {
-    for (int j = p.nq + tid; j < p.n; j += kQThreads) {
+    for (int j = nq_b + tid; j < n_b; j += kQThreads) {
       const int64_t row = static_cast<int64_t>(b) * p.n_max + j;
       const uint4* kr = reinterpret_cast<const uint4*>(p.cache + hd.k_off + row * hd.rp_k * 2);
       const uint4* vr = reinterpret_cast<const uint4*>(p.cache + hd.v_off + row * hd.rp_v * 2);
@@ -403,17 +442,19 @@ __global__ void __launch_bounds__(128) quant_combine_kernel(const QuantParams p)
   }
 }
 
-template <int NW, int MINB, int G, bool FULL>
+template <int NW, int MINB, int G, bool FULL, int BITS>
 cudaError_t launch_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
   static size_t configured[kMaxDevices] = {};
-  const cudaError_t ec = ensure_dynamic_smem(decode_quant_kernel<NW, MINB, G, FULL>, smem, configured);
+  const cudaError_t ec = ensure_dynamic_smem(decode_quant_kernel<NW, MINB, G, FULL, BITS>, smem, configured);
   if (ec != cudaSuccess) return ec;
-  decode_quant_kernel<NW, MINB, G, FULL><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
+  decode_quant_kernel<NW, MINB, G, FULL, BITS><<<dim3(p.B * p.H, p.splits), kQThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 template <int NW, int MINB, int G>
 cudaError_t launch_full_or_not(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
-  return full ? launch_variant<NW, MINB, G, true>(p, smem, s) : launch_variant<NW, MINB, G, false>(p, smem, s);
+  if (p.bits == 3)
+    return full ? launch_variant<NW, MINB, G, true, 3>(p, smem, s) : launch_variant<NW, MINB, G, false, 3>(p, smem, s);
+  return full ? launch_variant<NW, MINB, G, true, 4>(p, smem, s) : launch_variant<NW, MINB, G, false, 4>(p, smem, s);
 }
 template <int NW, int MINB>
 cudaError_t launch_group(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
@@ -443,7 +484,11 @@ size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v) {
 cudaError_t launch_decode_quant(const QuantParams& p0, int max_rp, int min_rp, size_t smem, cudaStream_t s,
                                 uint64_t* launches) {
   QuantParams p = p0;
-  p.magic[0] = 0x4B000000u; p.magic[1] = 0x49000000u; p.magic[2] = 0x47000000u; p.magic[3] = 0x45000000u;
+  if (p.bits == 3) {   // 2^23, 2^20, 2^17, 2^14
+    p.magic[0] = 0x4B000000u; p.magic[1] = 0x49800000u; p.magic[2] = 0x48000000u; p.magic[3] = 0x46800000u;
+  } else {             // 2^23, 2^19, 2^15, 2^11
+    p.magic[0] = 0x4B000000u; p.magic[1] = 0x49000000u; p.magic[2] = 0x47000000u; p.magic[3] = 0x45000000u;
+  }
   cudaError_t e;
   if (max_rp <= 64) e = launch_group<8, 3>(p, min_rp == 64, smem, s);
   else if (max_rp <= 80) e = launch_group<10, 3>(p, min_rp == 80, smem, s);

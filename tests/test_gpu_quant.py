@@ -44,7 +44,7 @@ def rank_space_case(B_, H, d, rk, rv, n, seed, q_scale=1.0):
     return U_k, U_v, q, kp.cuda(), vp.cuda(), rows
 
 
-def fill_both(B, B_, H, d, rk, rv, n, n_max, seed, group, alibi=None, q_scale=1.0):
+def fill_both(B, B_, H, d, rk, rv, n, n_max, seed, group, alibi=None, q_scale=1.0, bits=4):
     U_k, U_v, q, kp, vp, rows = rank_space_case(B_, H, d, rk, rv, n, seed, q_scale)
     lay = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v)
     lay.append_kv(kp, vp, preprojected=True)
@@ -54,39 +54,49 @@ def fill_both(B, B_, H, d, rk, rv, n, n_max, seed, group, alibi=None, q_scale=1.
     ref.set_len(n)
     if alibi is not None:
         lay.set_alibi(alibi)
-    lay.quant_attach(4, group)
+    lay.quant_attach(bits, group)
     return lay, ref, q, rows
 
 
-def unpack_codes(words: np.ndarray) -> np.ndarray:
-    """words [rp/8][G] uint32 -> codes [G][rp] (channel 8j+k in bits 4k..4k+3 of word j, stored as code + 8)."""
-    nw, G = words.shape
-    out = np.zeros((G, nw * 8), dtype=np.int64)
+def unpack_codes(area: np.ndarray, rp: int, G: int, bits: int) -> np.ndarray:
+    """A block's code area (bytes) -> codes [G][rp].  Unit j of row i holds channels 8j..8j+7, channel 8j+k in bits
+    bits*k.. as code + 2^(bits-1).  4-bit: units are 32-bit words [rp/8][G].  3-bit: the low 16 bits of all units
+    ([rp/8][G] halfwords), then their high 8 bits ([rp/8][G] bytes)."""
+    nw = rp // 8
+    if bits == 4:
+        units = area.view(np.uint32).reshape(nw, G).astype(np.int64)
+    else:
+        lo = area[:2 * nw * G].view(np.uint16).reshape(nw, G).astype(np.int64)
+        hi = area[2 * nw * G:3 * nw * G].reshape(nw, G).astype(np.int64)
+        units = lo | (hi << 16)
+    out = np.zeros((G, rp), dtype=np.int64)
     for k in range(8):
-        out[:, k::8] = ((words.T >> np.uint32(4 * k)) & np.uint32(15)).astype(np.int64) - 8
+        out[:, k::8] = ((units.T >> (bits * k)) & ((1 << bits) - 1)) - (1 << (bits - 1))
     return out
 
 
-def read_block(lay, head, b, blk, G, rp_k, rp_v):
+def read_block(lay, head, b, blk, G, rp_k, rp_v, bits=4):
     _, bb, ks_off, vc_off, vs_off = lay.quant_layout(head)
     raw = lay.quant_blocks(head)[b, blk].cpu().numpy()
-    kc = unpack_codes(raw[:ks_off].view(np.uint32).reshape(rp_k // 8, G))
+    assert ks_off == G * rp_k * bits // 8 and vs_off - vc_off == G * rp_v * bits // 8      # exactly `bits` per element
+    kc = unpack_codes(raw[:ks_off], rp_k, G, bits)
     ks = raw[ks_off:vc_off].view(np.float16)
-    vc = unpack_codes(raw[vc_off:vs_off].view(np.uint32).reshape(rp_v // 8, G))
+    vc = unpack_codes(raw[vc_off:vs_off], rp_v, G, bits)
     nvg = (rp_v + G - 1) // G
     vs = raw[vs_off:vs_off + 2 * G * nvg].view(np.float16).reshape(nvg, G).T       # -> [G][nvg]
     return kc, ks, vc, vs
 
 
+@pytest.mark.parametrize("bits", [4, 3])
 @pytest.mark.parametrize("G,H,d,rk,rv,n", [
     (32, 2, 128, [80, 80], [80, 80], 200),            # the headline rank; 6 blocks and 8 rows left over
     (16, 2, 128, [80, 48], [64, 80], 100),            # smallest group: five value groups per row
     (64, 3, 64, [24, 64, 37], [56, 8, 64], 300),      # ranks that are not multiples of 8 (zero padding inside a word)
     (128, 2, 128, [128, 80], [128, 96], 400),         # widest rank; one value group per row
 ])
-def test_codes_and_scales_are_bit_exact(B, G, H, d, rk, rv, n):
+def test_codes_and_scales_are_bit_exact(B, G, H, d, rk, rv, n, bits):
     B_ = 2
-    lay, ref, q, rows = fill_both(B, B_, H, d, rk, rv, n, n + 5, 171, G)
+    lay, ref, q, rows = fill_both(B, B_, H, d, rk, rv, n, n + 5, 171, G, bits=bits)
     lay.quant_sync()
     torch.cuda.synchronize()
     assert lay.quant_len == n // G * G
@@ -95,10 +105,10 @@ def test_codes_and_scales_are_bit_exact(B, G, H, d, rk, rv, n):
         for b in range(B_):
             Kp, Vp = rows[(b, h)]
             nq = n // G * G
-            kc_ref, ks_ref = kq.quantize_keys(Kp[:nq], 4, G)
-            vc_ref, vs_ref = kq.quantize_values(Vp[:nq], 4, G)
+            kc_ref, ks_ref = kq.quantize_keys(Kp[:nq], bits, G)
+            vc_ref, vs_ref = kq.quantize_values(Vp[:nq], bits, G)
             for blk in range(n // G):
-                kc, ks, vc, vs = read_block(lay, h, b, blk, G, rp_k, rp_v)
+                kc, ks, vc, vs = read_block(lay, h, b, blk, G, rp_k, rp_v, bits)
                 sl = slice(blk * G, (blk + 1) * G)
                 assert np.array_equal(kc[:, :rk[h]], kc_ref[sl]), (h, b, blk, "key codes")
                 assert np.array_equal(ks[:rk[h]], ks_ref[blk]), (h, b, blk, "key scales")
@@ -116,13 +126,14 @@ def test_codes_and_scales_are_bit_exact(B, G, H, d, rk, rv, n):
     (32, 1, 128, [80], [80], 20),                     # shorter than one group: all rows come from the 16-bit cache
     (32, 4, 128, [80] * 4, [80] * 4, 9000),           # many stages per CTA, several splits
 ])
-def test_decode_quant_matches_oracle(B, G, H, d, rk, rv, n):
+@pytest.mark.parametrize("bits", [4, 3])
+def test_decode_quant_matches_oracle(B, G, H, d, rk, rv, n, bits):
     B_ = 2
-    lay, ref, q, _ = fill_both(B, B_, H, d, rk, rv, n, n + 7 + G, 172, G)
+    lay, ref, q, _ = fill_both(B, B_, H, d, rk, rv, n, n + 7 + G, 172, G, bits=bits)
     lay.quant_sync()
     out = lay.decode_quant(q)
     lay.poll_status()
-    res = ref.decode_quant(to_np(q), 4, G)
+    res = ref.decode_quant(to_np(q), bits, G)
     want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
     assert_close(out, want, BF16, f"decode_quant G={G} n={n}")
     # the quantisation error itself is far above the tolerance: the test would notice codes that are ignored
@@ -167,16 +178,17 @@ def test_decode_quant_with_rows_that_are_not_synced_yet(B):
     assert lay.quant_len == 96
 
 
-def test_decode_quant_with_peaked_attention_and_alibi(B):
+@pytest.mark.parametrize("bits", [4, 3])
+def test_decode_quant_with_peaked_attention_and_alibi(B, bits):
     """Few rows carry the softmax (scaled query, steep bias on one head): a wrong scale or code of a single row
     is not averaged away."""
     B_, H, d, G, n = 2, 4, 128, 32, 1500
     slopes = [0.25, 0.0, 2.0 ** -4, 2.0 ** -8]
-    lay, ref, q, _ = fill_both(B, B_, H, d, [80] * H, [80] * H, n, n, 174, G, alibi=slopes, q_scale=3.0)
+    lay, ref, q, _ = fill_both(B, B_, H, d, [80] * H, [80] * H, n, n, 174, G, alibi=slopes, q_scale=3.0, bits=bits)
     lay.quant_sync()
     out = lay.decode_quant(q)
     lay.poll_status()
-    res = ref.decode_quant(to_np(q), 4, G)
+    res = ref.decode_quant(to_np(q), bits, G)
     want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
     assert_close(out, want, BF16, "peaked + alibi")
 
@@ -212,7 +224,7 @@ def test_quant_argument_checks(B):
     with pytest.raises(B.EigenAttnError):
         lay.decode_quant(q)                                   # nothing attached
     with pytest.raises(B.EigenAttnError):
-        lay.quant_bytes(3, 32)                                # only 4-bit codes are built
+        lay.quant_bytes(2, 32)                                # 3- and 4-bit codes are built
     with pytest.raises(B.EigenAttnError):
         lay.quant_bytes(4, 48)                                # group must be 16, 32, 64 or 128
     lay.quant_attach(4, 32)
@@ -221,6 +233,15 @@ def test_quant_argument_checks(B):
     lay32 = B.EigenAttnLayer(1, 1, 64, 64, torch.float32, U_k, U_v)
     with pytest.raises(B.EigenAttnError):
         lay32.quant_bytes(4, 32)                              # 16-bit layers only
-    # storage per element of whole blocks: 4 + 16/G bits for keys (Table 8's accounting)
+    # storage per element of whole blocks: bits + 16/G bits for keys (Table 8's accounting), both precisions
     _, bb, ks_off, vc_off, _ = lay.quant_layout(0)
     assert vc_off * 8 / (32 * 32) == 4 + 16 / 32
+    for bits, G in ((3, 128), (3, 32), (3, 64), (4, 16), (4, 128), (4, 32)):       # the Eigen Attention rows of Table 8
+        U_k, U_v, *_ = make_case(1, 2, 128, [80, 80], [80, 80], 256, BF16, seed_cfg=176)
+        lay2 = B.EigenAttnLayer(1, 2, 128, 256, BF16, U_k, U_v)
+        lay2.quant_attach(bits, G)
+        _, bb, ks_off, vc_off, vs_off = lay2.quant_layout(0)
+        assert vc_off == kq.quant_cache_bytes(G * 80, bits, G)                        # keys: bits + 16/G per element
+        assert (bb - vc_off) * 8 == G * 80 * bits + 16 * G * -(-80 // G)               # values: one scale per started group
+        table, blocks = 256, 256 // G                                                   # per-head table (padded), blocks per sequence
+        assert lay2.quant_bytes(bits, G) == table + 2 * ((blocks * bb + 255) // 256 * 256)

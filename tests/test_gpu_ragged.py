@@ -165,22 +165,80 @@ def test_grouped_query_decode_with_unequal_lengths(B, H, g, d, rk, rv, n, lens):
     lay.poll_status()
 
 
-def test_unequal_lengths_are_refused_with_a_quantised_cache(B):
+def test_set_lens_argument_checks(B):
     B_, H, d, n = 2, 2, 128, 64
     U_k, U_v, q, k, v = make_case(B_, H, d, [64] * H, [64] * H, n, BF16, seed_cfg=144)
     lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
     lay.append_kv(k, v)
     lay.set_lens([n, 5])
-    for call in (lambda: lay.quant_attach(4, 32), lambda: lay.set_lens([n, -1]), lambda: lay.set_lens([n + 1, 1])):
+    for call in (lambda: lay.set_lens([n, -1]), lambda: lay.set_lens([n + 1, 1])):
         with pytest.raises(B.EigenAttnError):
             call()
     assert lay.lens() == [n, 5]
-    lay.set_lens([n, n])                          # equal again: everything is available
+    lay.set_lens([n, n])                          # equal again
     assert lay.lens() == [n, n]
-    lay.quant_attach(4, 32)
-    with pytest.raises(B.EigenAttnError) as e:    # and with a quantised cache attached, lengths stay equal
-        lay.set_lens([n, 5])
-    assert e.value.status == B.EA_ERR_UNSUPPORTED
+    lay.poll_status()
+
+
+@pytest.mark.parametrize("bits,G", [(4, 32), (3, 16), (4, 128)])
+def test_quantised_cache_with_unequal_lengths(B, bits, G):
+    """Section 5.3 per sequence: every sequence keeps the codes of its own complete blocks and attends them plus
+    its own 16-bit tail.  The expected value is the oracle's quantised decode of each sequence alone.  Order of
+    events: uniform fill and sync, then the true lengths (codes below each length are kept), decode; more rows
+    behind every sequence's own end, sync with lengths in force, decode; a buffer attached while lengths differ;
+    back to equal lengths."""
+    from oracle import kv_quant as kq
+    H, d, n = 3, 128, 1500
+    rk, rv = [80, 48, 128], [80, 112, 64]
+    lens = [1500, 700, 37, 1]                      # 37 < G for G = 128: that sequence has no codes at all
+    B_ = len(lens)
+    extra = 40
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + extra, BF16, seed_cfg=146, T_q=3)
+    lay = B.EigenAttnLayer(B_, H, d, n + extra, BF16, U_k, U_v)
+    lay.append_kv(k[:, :n], v[:, :n])
+    lay.quant_attach(bits, G)
+    lay.quant_sync()
+    assert lay.quant_len == n // G * G
+    lay.set_lens(lens)
+    assert lay.quant_lens() == [x // G * G for x in lens] and lay.quant_len == lens[0] // G * G
+
+    store = storage_model(BF16)                    # the oracle quantises the 16-bit rows the cache holds
+    def expect(qq, cur_lens, rows_of):
+        outs = []
+        for b, nb in enumerate(cur_lens):
+            r = orc.LayerOracle(1, H, d, U_k, U_v, storage=store)
+            kk, vv = rows_of(b, nb)
+            r.append_kv(kk, vv)
+            res = r.decode_quant(to_np(qq[b:b + 1]), bits, G)
+            outs.append(np.stack([res[(0, h)] for h in range(H)])[None, None])
+        return np.concatenate(outs, axis=0)
+
+    first = lambda b, nb: (to_np(k[b:b + 1, :nb]), to_np(v[b:b + 1, :nb]))
+    for ctas in (0, 1, 400):
+        lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        assert_close(lay.decode_quant(q[:, :1]), expect(q[:, :1], lens, first), BF16, f"ragged quant decode ctas={ctas}")
+    lay.set_option(B.EA_OPT_DECODE_CTAS, 0)
+    # `extra` more rows behind each sequence's own end; some sequences complete new blocks, which the sync quantises
+    lay.append_kv(k[:, n:], v[:, n:])
+    lens2 = [x + extra for x in lens]
+    grown = lambda b, nb: (np.concatenate([to_np(k[b:b + 1, :lens[b]]), to_np(k[b:b + 1, n:])], axis=1),
+                           np.concatenate([to_np(v[b:b + 1, :lens[b]]), to_np(v[b:b + 1, n:])], axis=1))
+    before = lay.quant_lens()
+    out_unsynced = lay.decode_quant(q[:, 1:2])     # new rows still 16-bit: codes below the old counts only
+    lay.quant_sync()
+    assert lay.quant_lens() == [x // G * G for x in lens2] and lay.quant_lens() != before
+    assert_close(lay.decode_quant(q[:, 1:2]), expect(q[:, 1:2], lens2, grown), BF16, "after a sync with lengths in force")
+    assert float((out_unsynced.float() - lay.decode_quant(q[:, 1:2]).float()).abs().max()) < 0.25   # same rows, other precision
+    # a fresh buffer attached while lengths differ starts without codes: the decode reads 16-bit rows only
+    lay.quant_attach(bits, G)
+    assert lay.quant_lens() == [0] * B_
+    plain = lay.decode(q[:, 1:2])
+    assert torch.equal(lay.decode_quant(q[:, 1:2]), plain) or float((lay.decode_quant(q[:, 1:2]).float() - plain.float()).abs().max()) < 2e-2
+    lay.quant_sync()
+    assert_close(lay.decode_quant(q[:, 1:2]), expect(q[:, 1:2], lens2, grown), BF16, "buffer attached while lengths differ")
+    # back to equal lengths: the codes every sequence holds stay
+    lay.set_len(min(lens2))
+    assert lay.quant_len == min(lens2) // G * G
     lay.poll_status()
 
 
