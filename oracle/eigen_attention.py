@@ -26,6 +26,8 @@ The RoPE variant (Section 4.3) is pinned by library attention on keys and
 queries rotated with complex arithmetic, by its relative-position invariance,
 by the zero-angle special case and by loops.
 decode_quant is ordinary decode over the rows returned by kv_quant.quantized_view, which has its own pins.
+paged_gather / paged_scatter (address arithmetic of a paged cache) are pinned by the identity "paged == contiguous"
+for random page tables, by the identity table, and by a hand-written two-page example.
 Nothing in this file is "parity unpinned".
 """
 from __future__ import annotations
@@ -350,6 +352,33 @@ class LayerOracle:
         for (b, h), o in res.items():
             out[b, :, h, :] = o
         return out
+
+
+# --------------------------------------------------------------------------
+# A paged cache: where a sequence's rows live, nothing else
+# --------------------------------------------------------------------------
+
+def paged_gather(pool: np.ndarray, table_row: Sequence[int], page_rows: int, n: int) -> np.ndarray:
+    """Rows 0..n-1 of one sequence out of a pool of pages.  `pool` is [pages * page_rows, width] (physical page p =
+    rows p*page_rows .. (p+1)*page_rows - 1); logical row r lives in physical page table_row[r // page_rows] at
+    offset r % page_rows.  Paging changes addresses only: the paper's generation phase (Section 2) is stated on
+    the rows K, V of a sequence, wherever they are kept, so attention over the gathered rows IS the paged result."""
+    pool = np.asarray(pool)
+    out = np.empty((n, pool.shape[1]), dtype=pool.dtype)
+    for r in range(n):
+        page = int(table_row[r // page_rows])
+        assert page >= 0, "row in an unmapped page"
+        out[r] = pool[page * page_rows + r % page_rows]
+    return out
+
+
+def paged_scatter(pool: np.ndarray, table_row: Sequence[int], page_rows: int, row0: int, rows: np.ndarray) -> None:
+    """Writes `rows` at logical rows row0.. of one sequence into the pool (the append of Section 2, paged)."""
+    for i in range(rows.shape[0]):
+        r = row0 + i
+        page = int(table_row[r // page_rows])
+        assert page >= 0, "row in an unmapped page"
+        pool[page * page_rows + r % page_rows] = rows[i]
 
 
 # --------------------------------------------------------------------------

@@ -335,6 +335,44 @@ def test_append_unit_rows_equals_append_kv_and_the_per_head_definition():
                 assert np.abs(b.Kp[u] - k[u[0], :, u[1]] @ U_K[u[1]]).max() > 1e-6
 
 
+def test_paged_rows_equal_contiguous_rows():
+    # Paging moves rows, nothing else: scatter through any page table then gather returns the rows, attention over the
+    # gathered rows equals attention over the contiguous ones, pages of different sequences never mix, and a
+    # two-page example written out by hand fixes the index arithmetic (page = r // page_rows, offset = r % page_rows).
+    rng = np.random.default_rng(21)
+    page_rows, pages, width, B = 4, 9, 3, 3
+    pool = np.full((pages * page_rows, width), np.nan)
+    perm = rng.permutation(pages)
+    table = [list(perm[0:4]), list(perm[4:6]) + [-1, -1], list(perm[6:9]) + [-1]]
+    lens = [14, 7, 9]
+    rows = [rng.standard_normal((n, width)) for n in lens]
+    for b in range(B):                                   # appended in chunks that straddle page boundaries
+        cut = lens[b] // 2 + 1
+        orc.paged_scatter(pool, table[b], page_rows, 0, rows[b][:cut])
+        orc.paged_scatter(pool, table[b], page_rows, cut, rows[b][cut:])
+    for b in range(B):
+        assert np.array_equal(orc.paged_gather(pool, table[b], page_rows, lens[b]), rows[b])
+    written = int(np.isfinite(pool[:, 0]).sum())
+    assert written == sum(lens)                          # no row written twice, none outside the sequences' pages
+    ident = list(range(pages))
+    flat = rng.standard_normal((pages * page_rows, width))
+    assert np.array_equal(orc.paged_gather(flat, ident, page_rows, 30), flat[:30])       # identity table = contiguous
+    hand = np.arange(16, dtype=np.float64).reshape(8, 2)                                  # 2 pages of 4 rows
+    got = orc.paged_gather(hand, [1, 0], 4, 6)                                            # logical rows 0..3 in page 1, 4..5 in page 0
+    assert np.array_equal(got, hand[[4, 5, 6, 7, 0, 1]])
+    with pytest.raises(AssertionError):
+        orc.paged_gather(pool, table[1], page_rows, 9)                                    # row 8 is in an unmapped page
+    # attention over rows kept in pages = attention over the same rows kept contiguously
+    d_h, r = 8, 5
+    U_K, U_V = synth.orthonormal_basis(d_h, r, 31), synth.orthonormal_basis(d_h, r, 32)
+    K, V, q = rng.standard_normal((11, d_h)), rng.standard_normal((11, d_h)), rng.standard_normal(d_h)
+    poolK, poolV = np.zeros((3 * 4, d_h)), np.zeros((3 * 4, d_h))
+    orc.paged_scatter(poolK, [2, 0, 1], 4, 0, K)
+    orc.paged_scatter(poolV, [2, 0, 1], 4, 0, V)
+    a = orc.decode_head(q, orc.paged_gather(poolK, [2, 0, 1], 4, 11), orc.paged_gather(poolV, [2, 0, 1], 4, 11), U_K, U_V)
+    assert np.array_equal(a, orc.decode_head(q, K, V, U_K, U_V))
+
+
 # ---- P7: tiny brute force with explicit d_h x d_h projectors (Eq. 7, second line) ---------------
 
 @pytest.mark.parametrize("n", [1, 2, 5])
