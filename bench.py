@@ -261,14 +261,26 @@ def rank_chunk_base(rank: int) -> int:
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------
 
-def build_layer(wl, device, binding, keep_units=(), rank=0):
+def shuffled_page_table(batch, n_max, page_rows, seed):
+    """Every sequence gets n_max / page_rows pages drawn without replacement from the whole pool."""
+    per = n_max // page_rows
+    perm = np.random.default_rng(seed).permutation(batch * per)
+    return [[int(x) for x in perm[b * per:(b + 1) * per]] for b in range(batch)]
+
+
+def build_layer(wl, device, binding, keep_units=(), rank=0, page_rows=0):
     """Creates the layer and fills `context` rows through eigen_attn_append_kv.  Returns the layer, the
     bases, and for the (sequence, head) units in keep_units the raw K/V history as float64 arrays."""
     ranks = synth.draw_ranks(wl.n_heads, wl.ranks, wl.index)
     U_k = synth.make_bases(wl.d_head, ranks, wl.index, "U_K")
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
     dt = synth.torch_dtype(wl.dtype)
-    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, wl.context + 1, dt, U_k, U_v, device=device)
+    n_max = wl.context + 1
+    if page_rows:
+        n_max = (n_max + page_rows - 1) // page_rows * page_rows
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, n_max, dt, U_k, U_v, device=device)
+    if page_rows:                                       # pages shuffled across the pool before the first row is written
+        lay.set_page_table(shuffled_page_table(wl.batch, n_max, page_rows, synth.stream_seed(wl.index, "subset", 99)), page_rows)
     if VARIANT["alibi"]:
         lay.set_alibi(variant_slopes(wl))
     if VARIANT["rope"]:
@@ -637,6 +649,16 @@ def workload_table_own_layers(device, binding, steps=30, warmup=3):
     import dataclasses
     peak, _ = measured_peaks()
     table = {}
+    wl = synth.WORKLOADS["llama2_7b_b16_n32k"]             # the headline layer on a paged cache, pages of 128 rows
+    lay, ranks, _, _, _, q, kn, vn = build_layer(wl, device, binding, page_rows=128)
+    out = torch.empty_like(q)
+    def step_paged():
+        lay.set_len(wl.context); lay.decode_step(q, kn, vn, out=out)
+    k_us, s_us = timed_kernel(lay, device, step_paged, steps, warmup)
+    table["paged_cache"] = table_entry("decode_splitkv_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
+                                       workload=wl.name + ", page table with pages of 128 rows shuffled over the pool")
+    del lay
+    torch.cuda.empty_cache()
     for b in (1, 2):
         wl = dataclasses.replace(synth.WORKLOADS["mpt_7b_long"], batch=b)
         lay, ranks, _, _, _, q, kn, vn = build_layer(wl, device, binding)

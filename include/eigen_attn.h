@@ -255,6 +255,26 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);
 ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens);
 
+/* A paged cache (the paper's introduction lists paging among the systems-level ways to fit long contexts, and its
+ * outlook names the serving frameworks built on it; the generation phase of Section 2 is stated on a sequence's
+ * rows K, V wherever they are kept, so paging changes addresses and nothing else).
+ * Each head's K' (and V') slab is viewed as one array of batch * n_max rows cut into physical pages of `page_rows`
+ * rows (a power of two, at least 128: a page holds whole tiles, so a tile is still one bulk copy); page p is rows
+ * [p * page_rows, (p + 1) * page_rows).  h_table: HOST array [batch][pages_per_seq]; logical row r of sequence b
+ * lives in physical page h_table[b][r / page_rows] at offset r % page_rows, in every head's slabs.  -1 = not mapped;
+ * mapped entries of a sequence come first, no physical page may appear twice (EA_ERR_INVALID_ARG).  A sequence can
+ * then hold as many rows as its mapped pages, which may exceed n_max when others map fewer: calls that add rows
+ * return EA_ERR_CAPACITY when a sequence's next row has no page.  Rows are not moved: after the call a sequence's
+ * rows are whatever its pages hold (the identity table h_table[b][i] = b * (n_max / page_rows) + i keeps a
+ * contiguous cache as it is, when page_rows divides n_max).  NULL returns to the contiguous layout.
+ * Available for eigen_attn_append_kv, _decode, _decode_step(_host), _decode_static, _set_len(s), and
+ * eigen_attn_prefill (which then runs on the CUDA cores); not (EA_ERR_UNSUPPORTED) with a rotary embedding, a
+ * quantised cache or eigen_attn_decode_gqa.  batch * pages_per_seq entries must fit the table area of the workspace
+ * (batch * batch * n_max / 128 entries, at most 4 Mi).  Uploaded on the stream (asynchronous; the array may be reused
+ * when the call returns): later calls must run on that stream or be ordered after it. */
+ea_status eigen_attn_set_page_table(eigen_attn_t h, const int32_t* h_table, int32_t pages_per_seq, int32_t page_rows,
+                                    void* cuda_stream);
+
 /* Synchronises the stream and returns the device status word (EA_OK or EA_ERR_TIMEOUT), then clears it. */
 ea_status eigen_attn_poll_status(eigen_attn_t h, void* cuda_stream);
 

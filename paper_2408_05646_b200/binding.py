@@ -64,6 +64,7 @@ SYMBOLS = {
     "eigen_attn_set_len": (_i32, [_vp, _i32]),
     "eigen_attn_set_lens": (_i32, [_vp, ctypes.POINTER(_i32), _vp]),
     "eigen_attn_get_lens": (_i32, [_vp, ctypes.POINTER(_i32)]),
+    "eigen_attn_set_page_table": (_i32, [_vp, ctypes.POINTER(_i32), _i32, _i32, _vp]),
     "eigen_attn_poll_status": (_i32, [_vp, _vp]),
     "eigen_attn_last_error": (ctypes.c_char_p, [_vp]),
     "eigen_attn_head_offsets": (_i32, [_vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
@@ -417,6 +418,17 @@ class EigenAttnLayer:
         arr = (ctypes.c_int32 * self.B)()
         self._check(lib.eigen_attn_get_lens(self.handle, arr), "eigen_attn_get_lens")
         return list(arr)
+
+    def set_page_table(self, table, page_rows: int = 128, stream=None) -> None:
+        """table: [batch][pages_per_seq] physical page of every logical page (-1 = not mapped); None = contiguous."""
+        if table is None:
+            self._check(lib.eigen_attn_set_page_table(self.handle, None, 0, 0, _stream_ptr(stream)), "eigen_attn_set_page_table")
+            return
+        width = len(table[0])
+        assert len(table) == self.B and all(len(r) == width for r in table)
+        arr = (ctypes.c_int32 * (self.B * width))(*[int(x) for r in table for x in r])
+        self._check(lib.eigen_attn_set_page_table(self.handle, arr, width, int(page_rows), _stream_ptr(stream)),
+                    "eigen_attn_set_page_table")
 
     def poll_status(self, stream=None) -> None:
         self._check(lib.eigen_attn_poll_status(self.handle, _stream_ptr(stream)), "eigen_attn_poll_status")

@@ -44,7 +44,8 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0, off_qlens = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0, off_qlens = 0, off_pages = 0;
+  size_t page_entries = 0;   // capacity of the page-table area, in entries
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
   int part_stride = 0;
@@ -119,6 +120,12 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->off_deficit = off;  off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // unequal lengths
   L->off_qlens = off;    off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // ... of the quantised copy
+  // page table [batch][pages per sequence]: room for every sequence to map the whole pool of 128-row pages,
+  // at most 4 Mi entries
+  const size_t pool_pages = static_cast<size_t>(d->batch) * d->n_max / 128;
+  L->page_entries = static_cast<size_t>(d->batch) * pool_pages;
+  if (L->page_entries > (1u << 22)) L->page_entries = 1u << 22;
+  L->off_pages = off;    off = align_up(off + L->page_entries * sizeof(int32_t));
   L->workspace_bytes = off;
 }
 
@@ -199,6 +206,10 @@ struct eigen_attn {
   bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
   int rope_interleaved = 0;
   int64_t opt_ctas = 0, opt_tile_rows = 0, opt_stages = 0, opt_prefill = 0, opt_fused = 1, opt_project = 0;
+  // paged cache (eigen_attn_set_page_table)
+  bool paged = false;
+  int page_shift = 0, page_width = 0;
+  std::vector<int32_t> page_cap;      // [B]: rows sequence b can hold = leading mapped pages * page_rows
   int64_t opt_min_copy = -1;  // EA_OPT_DECODE_MIN_COPY_BYTES; < 0 = the built-in default
   int64_t opt_give_up = 0;   // EA_OPT_TEST_WAIT_GIVES_UP: armed for the next split-KV decode launch
   uint64_t launches = 0;
@@ -266,6 +277,25 @@ ea_status check_quant_args(eigen_attn_t h, const char* who, int32_t bits, int32_
 const HeadInfo* dev_heads(eigen_attn_t h) { return reinterpret_cast<const HeadInfo*>(h->ws + h->L.off_heads); }
 const float* dev_basis(eigen_attn_t h) { return reinterpret_cast<const float*>(h->ws + h->L.off_basis); }
 int* dev_status(eigen_attn_t h) { return reinterpret_cast<int*>(h->ws + h->L.off_status); }
+ea::PageMap dev_pages(eigen_attn_t h) {
+  ea::PageMap pm{};
+  if (h->paged) {
+    pm.table = reinterpret_cast<const int32_t*>(h->ws + h->L.off_pages);
+    pm.width = h->page_width;
+    pm.shift = h->page_shift;
+  }
+  return pm;
+}
+// Rows sequence b can hold: n_max, or what its page table maps.
+int64_t capacity_of(const eigen_attn* h, int b) { return h->paged ? h->page_cap[b] : h->desc.n_max; }
+// True if every sequence has room for T more rows; *bad = a sequence that has not.
+bool room_for(const eigen_attn* h, int64_t T, int* bad) {
+  for (int b = 0; b < h->desc.batch; ++b) {
+    const int64_t have = h->len - (h->max_deficit > 0 ? h->deficit[b] : 0);
+    if (have + T > capacity_of(h, b)) { *bad = b; return false; }
+  }
+  return true;
+}
 const int32_t* dev_deficit(eigen_attn_t h) {
   return h->max_deficit > 0 ? reinterpret_cast<const int32_t*>(h->ws + h->L.off_deficit) : nullptr;
 }
@@ -276,14 +306,17 @@ ea_status do_append(eigen_attn_t h, const void* d_k, const void* d_v, int32_t T,
   if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "append_kv: NULL k or v");
   if (flags & ~EA_KV_PREPROJECTED) return fail(h, EA_ERR_INVALID_ARG, "append_kv: unknown flag 0x%x", flags);
   if (T < 1) return fail(h, EA_ERR_SHAPE, "append_kv: T = %d", T);
-  if (static_cast<int64_t>(h->len) + T > h->desc.n_max)
-    return fail(h, EA_ERR_CAPACITY, "append_kv: len %d + T %d exceeds n_max %d", h->len, T, h->desc.n_max);
+  int bad = 0;
+  if (!room_for(h, T, &bad))
+    return fail(h, EA_ERR_CAPACITY, "append_kv: T %d more rows exceed the capacity of sequence %d (%lld rows)", T, bad,
+                static_cast<long long>(capacity_of(h, bad)));
   ea::ProjectParams p{};
   p.heads = dev_heads(h); p.basis = dev_basis(h); p.k = d_k; p.v = d_v; p.cache = h->cache;
   p.stride_b = stride_b; p.stride_t = stride_t;
   p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head;
   p.n_max = h->desc.n_max; p.row0 = h->len; p.deficit = dev_deficit(h); p.flags = flags;
   p.lr_k_width = h->L.sum_rp_k; p.lr_v_width = h->L.sum_rp_v;
+  p.pages = dev_pages(h);
   const cudaError_t e = ea::launch_project_append(p, h->desc.dtype, s, &h->launches);
   if (e != cudaSuccess) return cuda_fail(h, e, "append_kv launch");
   h->len += T;
@@ -314,7 +347,10 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   const int fixed = static_cast<int>(ea::decode_fixed_smem_bytes());
   const int sms = h->opt_ctas > 0 ? static_cast<int>(h->opt_ctas) : h->sm_count;
 
-  const int min_copy = h->opt_min_copy >= 0 ? static_cast<int>(h->opt_min_copy) : kMinCopyBytes;
+  // paged cache: one tile per ring slot (consecutive tiles need not be neighbours in memory)
+  const int min_copy = h->paged ? 0 : h->opt_min_copy >= 0 ? static_cast<int>(h->opt_min_copy) : kMinCopyBytes;
+  if (h->paged && (h->opt_tile_rows & (h->opt_tile_rows - 1)) != 0)
+    return fail(h, EA_ERR_UNSUPPORTED, "%s: with a page table DECODE_TILE_ROWS must be a power of two", who);
   // rows per tile: 128 unless the context is short (keep a few tiles per CTA) or a stage would be too big
   int tile_rows = 128;
   if (h->opt_tile_rows > 0) {
@@ -389,6 +425,7 @@ ea_status plan_decode(eigen_attn_t h, const char* who, const void* d_q, int64_t 
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
   p.give_up_once = h->opt_give_up ? 1 : 0;
+  p.pages = dev_pages(h);
   plan->grid = grid;
   plan->smem = static_cast<size_t>(fixed) + static_cast<size_t>(ring_bytes);
 
@@ -420,6 +457,7 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
 ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
                          uint32_t flags, cudaStream_t s) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
+  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: not available with a page table");
   if (flags & ~EA_OUT_LOWRANK)
     return fail(h, EA_ERR_INVALID_ARG, "decode with rotary embedding: flag 0x%x (the query must be full rank)", flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
@@ -490,8 +528,10 @@ ea_status do_step(eigen_attn_t h, const void* d_q, int64_t stride_b_q, const voi
                   int64_t stride_b_kv, void* d_out, int64_t stride_b_out, uint32_t flags, cudaStream_t s) {
   if (h->opt_fused && h->len >= 1 && !h->rope) {
     if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "decode_step: NULL k or v");
-    if (h->len + 1 > h->desc.n_max)
-      return fail(h, EA_ERR_CAPACITY, "decode_step: len %d + 1 exceeds n_max %d", h->len, h->desc.n_max);
+    int bad = 0;
+    if (!room_for(h, 1, &bad))
+      return fail(h, EA_ERR_CAPACITY, "decode_step: one more row exceeds the capacity of sequence %d (%lld rows)", bad,
+                  static_cast<long long>(capacity_of(h, bad)));
     DecodePlan plan;
     const ea_status st = plan_decode(h, "decode_step", d_q, stride_b_q, d_out, stride_b_out, flags,
                                      reinterpret_cast<float*>(h->ws + h->L.off_partials), d_k, d_v, stride_b_kv,
@@ -679,7 +719,8 @@ ea_status eigen_attn_decode_step_host(eigen_attn_t h, const void* h_q, const voi
   if (!h) return EA_ERR_INVALID_ARG;
   if (!h_q || !h_k || !h_v || !h_out) return fail(h, EA_ERR_INVALID_ARG, "decode_step_host: NULL buffer");
   if (flags) return fail(h, EA_ERR_INVALID_ARG, "decode_step_host: flags must be 0");
-  if (h->len + 1 > h->desc.n_max) return fail(h, EA_ERR_CAPACITY, "decode_step_host: cache full");
+  int bad = 0;
+  if (!room_for(h, 1, &bad)) return fail(h, EA_ERR_CAPACITY, "decode_step_host: cache full (sequence %d)", bad);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const Layout& L = h->L;
   const size_t bytes = static_cast<size_t>(h->desc.batch) * h->desc.n_heads * h->desc.d_head * L.es;
@@ -761,7 +802,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                           reinterpret_cast<uintptr_t>(d_v) % 16 == 0 && stride_b % 8 == 0 && stride_t % 8 == 0;
   const bool out_aligned = (flags & EA_OUT_LOWRANK) || (reinterpret_cast<uintptr_t>(d_out) % 16 == 0 &&
                                                         out_stride_b % 8 == 0 && out_stride_t % 8 == 0);
-  const bool tc_attn = tc_shape && out_aligned;
+  const bool tc_attn = tc_shape && out_aligned && !h->paged;    // the tensor-core kernels address contiguous slabs
   if (h->opt_prefill == 2 && !tc_attn)
     return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
   cudaError_t e;
@@ -778,7 +819,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     e = (flags & EA_Q_PREPROJECTED) ? ea::launch_q_scatter(qp, L.sum_rp_k, h->desc.dtype, s, &h->launches)
                                     : ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
     if (e != cudaSuccess) return cuda_fail(h, e, "prefill q launch");
-  } else if (tc_shape && in_aligned && h->opt_prefill != 1) {
+  } else if (tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged) {
     // Q', K', V' in one tensor-core launch.  Its rows equal eigen_attn_append_kv's except where the two
     // fp32 summation orders round to different bf16 values (one unit in the last place).
     if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
@@ -833,6 +874,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
   p.tmaps = h->ws + L.off_tmaps;
+  p.pages = dev_pages(h);
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   size_t ws_smem = 0;
   const int ws_stages = tc_attn && h->tmaps_ok ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
@@ -855,8 +897,13 @@ ea_status eigen_attn_get_len(eigen_attn_t h, int32_t* len) {
 
 ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (len < 0 || len > h->desc.n_max)
-    return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %d]", len, h->desc.n_max);
+  int64_t cap = h->desc.n_max;
+  if (h->paged) {
+    cap = INT32_MAX;
+    for (int b = 0; b < h->desc.batch; ++b) cap = capacity_of(h, b) < cap ? capacity_of(h, b) : cap;
+  }
+  if (len < 0 || len > cap)
+    return fail(h, EA_ERR_CAPACITY, "set_len: %d outside [0, %lld]", len, static_cast<long long>(cap));
   if (h->q_group && h->max_deficit > 0)      // leaving unequal lengths: rows every sequence holds as codes
     for (int b = 0; b < h->desc.batch; ++b)
       if (h->qlens[b] < h->qlen) h->qlen = h->qlens[b];
@@ -873,8 +920,9 @@ ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_st
     return fail(h, EA_ERR_UNSUPPORTED, "set_lens: batch %d exceeds %d", B, ea::kMaxRaggedBatch);
   int32_t longest = 0;
   for (int b = 0; b < B; ++b) {
-    if (lens[b] < 0 || lens[b] > h->desc.n_max)
-      return fail(h, EA_ERR_CAPACITY, "set_lens: lens[%d] = %d outside [0, %d]", b, lens[b], h->desc.n_max);
+    if (lens[b] < 0 || lens[b] > capacity_of(h, b))
+      return fail(h, EA_ERR_CAPACITY, "set_lens: lens[%d] = %d outside [0, %lld]", b, lens[b],
+                  static_cast<long long>(capacity_of(h, b)));
     if (lens[b] > longest) longest = lens[b];
   }
   std::vector<int32_t> deficit(B);
@@ -913,6 +961,52 @@ ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_st
   h->deficit.swap(deficit);
   h->len = longest;
   h->max_deficit = widest;
+  return EA_OK;
+}
+
+ea_status eigen_attn_set_page_table(eigen_attn_t h, const int32_t* h_table, int32_t pages_per_seq, int32_t page_rows,
+                                    void* cuda_stream) {
+  if (!h) return EA_ERR_INVALID_ARG;
+  const int B = h->desc.batch;
+  if (!h_table) {                       // back to the contiguous layout
+    int64_t longest = h->len;
+    if (longest > h->desc.n_max) return fail(h, EA_ERR_CAPACITY, "set_page_table: len %d exceeds n_max %d", h->len, h->desc.n_max);
+    h->paged = false;
+    return EA_OK;
+  }
+  if (h->rope || h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_page_table: not available with a rotary embedding or a quantised cache");
+  if (page_rows < 128 || (page_rows & (page_rows - 1)) != 0)
+    return fail(h, EA_ERR_SHAPE, "set_page_table: page_rows %d (a power of two, at least 128)", page_rows);
+  const int64_t pool = static_cast<int64_t>(B) * h->desc.n_max / page_rows;      // physical pages of a head's slab
+  if (pool < 1) return fail(h, EA_ERR_SHAPE, "set_page_table: the cache holds no page of %d rows", page_rows);
+  if (pages_per_seq < 1 || static_cast<int64_t>(pages_per_seq) * page_rows > INT32_MAX)
+    return fail(h, EA_ERR_SHAPE, "set_page_table: pages_per_seq %d", pages_per_seq);
+  if (static_cast<size_t>(B) * pages_per_seq > h->L.page_entries)
+    return fail(h, EA_ERR_CAPACITY, "set_page_table: %d x %d entries exceed the table area (%zu)", B, pages_per_seq, h->L.page_entries);
+  std::vector<bool> used(static_cast<size_t>(pool), false);
+  std::vector<int32_t> cap(B, 0);
+  for (int b = 0; b < B; ++b) {
+    bool gap = false;
+    for (int i = 0; i < pages_per_seq; ++i) {
+      const int32_t pg = h_table[static_cast<size_t>(b) * pages_per_seq + i];
+      if (pg == -1) { gap = true; continue; }
+      if (pg < 0 || pg >= pool) return fail(h, EA_ERR_INVALID_ARG, "set_page_table: table[%d][%d] = %d outside [0, %lld)", b, i, pg, static_cast<long long>(pool));
+      if (gap) return fail(h, EA_ERR_INVALID_ARG, "set_page_table: sequence %d maps page %d behind an unmapped one", b, i);
+      if (used[pg]) return fail(h, EA_ERR_INVALID_ARG, "set_page_table: physical page %d is mapped twice", pg);
+      used[pg] = true;
+      cap[b] = (i + 1) * page_rows;
+    }
+    const int64_t have = h->len - (h->max_deficit > 0 ? h->deficit[b] : 0);
+    if (have > cap[b]) return fail(h, EA_ERR_CAPACITY, "set_page_table: sequence %d holds %lld rows, the table maps %d", b, static_cast<long long>(have), cap[b]);
+  }
+  const cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_pages, h_table, sizeof(int32_t) * B * pages_per_seq,
+                                        cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(h, e, "set_page_table: upload");
+  h->paged = true;
+  h->page_width = pages_per_seq;
+  h->page_shift = 0;
+  while ((1 << h->page_shift) < page_rows) ++h->page_shift;
+  h->page_cap.swap(cap);
   return EA_OK;
 }
 
@@ -993,6 +1087,7 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
   if (h->rope || h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a position scheme set");
+  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table");
   if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty (for some sequence)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
@@ -1049,6 +1144,7 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "set_rope: needs a bf16 layer with d_head %% 16 == 0 (and the driver's tensor-map encoder)");
   if (h->alibi) return fail(h, EA_ERR_INVALID_ARG, "set_rope: the layer has an ALiBi bias");
+  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "set_rope: not available with a page table");
   const int dh = h->desc.d_head;
   double freq[64] = {};
   for (int i = 0; i < dh / 2; ++i) freq[i] = pow(base, -2.0 * i / dh);
@@ -1081,6 +1177,7 @@ ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, v
   }
   const ea_status st = check_quant_args(h, "quant_attach", bits, group);
   if (st != EA_OK) return st;
+  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: not available with a page table");
   if (reinterpret_cast<uintptr_t>(d_qcache) % kAlign) return fail(h, EA_ERR_INVALID_ARG, "quant_attach: buffer not 256-byte aligned");
   std::vector<ea::QuantHead> qh;
   int widest = 0;

@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kProjThreads) project_rows_kernel(const Projec
                      static_cast<int64_t>(row) * rp + col;
             *dst = from_f<T>(acc[i]);
           } else {
-            const int64_t crow = static_cast<int64_t>(b) * p.n_max + p.row0 - (p.deficit ? p.deficit[b] : 0) + t;
+            const int64_t crow = physical_row(p.pages, b, p.n_max, p.row0 - (p.deficit ? p.deficit[b] : 0) + t);
             T* dst = reinterpret_cast<T*>(p.cache + (is_k ? hd.k_off : hd.v_off)) + crow * rp + col;
             *dst = from_f<T>(acc[i]);
           }
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(256) copy_lowrank_rows_kernel(const ProjectPar
   const int b = row / p.T, t = row - b * p.T;
   const T* k = static_cast<const T*>(p.k);
   const T* v = static_cast<const T*>(p.v);
-  const int64_t crow = static_cast<int64_t>(b) * p.n_max + p.row0 - (p.deficit ? p.deficit[b] : 0) + t;
+  const int64_t crow = physical_row(p.pages, b, p.n_max, p.row0 - (p.deficit ? p.deficit[b] : 0) + t);
   for (int c = threadIdx.x; c < hd.rp_k + hd.rp_v; c += blockDim.x) {
     const bool is_k = c < hd.rp_k;
     const int col = is_k ? c : c - hd.rp_k;

@@ -444,7 +444,7 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
   const bool kv_lowrank = (p.flags & 0x4u) != 0;  // rank-space k', v' supplied by the caller (merged W^K', W^V')
   if (with_new_row && kv_lowrank) {
     // nothing to project: the packed rows go into the cache (padding columns zero) and into shared memory
-    const int64_t crow = static_cast<int64_t>(b) * p.n_max + n_b;
+    const int64_t crow = physical_row(p.pages, b, p.n_max, n_b);
     if (t < hd.rp_k) {
       const T val = t < hd.r_k ? static_cast<const T*>(p.k_new)[b * p.kv_stride_b + hd.lr_k_off + t] : Elem<T>::from_float(0.f);
       reinterpret_cast<T*>(fx->new_k)[t] = val;
@@ -474,7 +474,7 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
   const int per = (d_head + groups - 1) / groups;
   T* knew = reinterpret_cast<T*>(fx->new_k);
   T* vnew = reinterpret_cast<T*>(fx->new_v);
-  const int64_t crow = static_cast<int64_t>(b) * p.n_max + n_b;
+  const int64_t crow = physical_row(p.pages, b, p.n_max, n_b);
   auto finish = [&](int o, float acc) {
     if (o < nq) {
       fx->qp[o] = acc * p.q_scale;
@@ -662,8 +662,17 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
         const char* src_k = p.cache + hd.k_off + row0 * rowb_k;
         const char* src_v = p.cache + hd.v_off + row0 * rowb_v;
         const uint32_t tile_k = p.tile_rows * rowb_k, tile_v = p.tile_rows * rowb_v;
+        // paged cache: a tile lies inside one page (tps == 1); its page is looked up one tile ahead, so that the
+        // table read has a whole tile's time to come back
+        const bool paged = p.pages.table != nullptr;
+        int64_t next_phys = paged && i0 < i1 ? physical_row(p.pages, b, p.n_max, i0 * p.tile_rows) : 0;
         for (int i = i0; i < i1; i += tps) {
           if (*abort_flag) { ok = false; break; }
+          if (paged) {
+            src_k = p.cache + hd.k_off + next_phys * rowb_k;
+            src_v = p.cache + hd.v_off + next_phys * rowb_v;
+            if (i + 1 < i1) next_phys = physical_row(p.pages, b, p.n_max, (i + 1) * p.tile_rows);
+          }
           const int st = rg.stage;
           const uint32_t bit = 1u << st;
           if (rg.filled & bit) {          // the slot's previous tile must have been released

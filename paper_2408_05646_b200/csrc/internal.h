@@ -25,6 +25,22 @@ struct HeadInfo {
   int32_t ukl16_off;   // float offset of the lift image of U^K (as uvl16_off, [d_head][rk16] canonical, high then low)
 };
 
+// Paged cache: where logical row `row` of sequence `b` lives in a head's slab, viewed as one array of
+// batch * n_max rows cut into pages of `page_rows` rows (a power of two, at least 128).  table == NULL: the
+// contiguous layout, sequence b at rows [b * n_max, (b + 1) * n_max).
+struct PageMap {
+  const int32_t* table;     // [B][width]: physical page of every logical page of a sequence (-1 = not mapped)
+  int32_t width;            // logical pages per sequence
+  int32_t shift;            // log2(page_rows)
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ int64_t physical_row(const PageMap& pm, int b, int n_max, int row) {
+  if (pm.table == nullptr) return static_cast<int64_t>(b) * n_max + row;
+  const int page = __ldg(pm.table + static_cast<int64_t>(b) * pm.width + (row >> pm.shift));
+  return (static_cast<int64_t>(page) << pm.shift) + (row & ((1 << pm.shift) - 1));
+}
+#endif
+
 constexpr int kDecodeConsumerWarps = 8;
 // + one warpgroup whose first thread is the producer: register reallocation works on whole warpgroups, and the
 // producer's group hands most of its registers to the consumers
@@ -64,6 +80,7 @@ struct DecodeParams {
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
   int32_t give_up_once;     // test hook: warp 0 of CTA 0 reports its first wait for a tile as run out
+  PageMap pages;            // paged cache (tile_rows divides the page size, one tile per ring slot)
 };
 
 struct CombineParams {
@@ -96,6 +113,7 @@ struct ProjectParams {       // project rows with U and scatter them into the ca
   const int32_t* deficit;   // [B]: sequence b starts at row0 - deficit[b] (unequal lengths); NULL = all at row0
   int32_t lr_k_width, lr_v_width;   // widths of the packed rank-space rows (sum of rp_k / rp_v)
   uint32_t flags;
+  PageMap pages;
 };
 
 struct QProjectParams {      // prefill: Q' = Q U^K into a scratch buffer (IO dtype)
@@ -137,6 +155,7 @@ struct PrefillParams {
   uint32_t flags;
   int* status;
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head (warp-specialised kernel only)
+  PageMap pages;            // paged cache (CUDA-core kernel only)
 };
 
 struct RopeDecodeParams {    // decode for models with rotary position embedding (bf16 layers)

@@ -60,14 +60,15 @@ __global__ void __launch_bounds__(kThreads) prefill_simt_kernel(const PrefillPar
   float m = -INFINITY, l = 0.f;
   const int my_last = p.len0 + t;                                      // last key this query sees
   const int blk_last = p.len0 + min(p.T - 1, qblk * kQRows + kQRows - 1);
-  const T* Kc = reinterpret_cast<const T*>(p.cache + hd.k_off) + static_cast<int64_t>(b) * p.n_max * rpk;
-  const T* Vc = reinterpret_cast<const T*>(p.cache + hd.v_off) + static_cast<int64_t>(b) * p.n_max * rpv;
+  const T* Kslab = reinterpret_cast<const T*>(p.cache + hd.k_off);
+  const T* Vslab = reinterpret_cast<const T*>(p.cache + hd.v_off);
 
   for (int j0 = 0; j0 <= blk_last; j0 += kKeyTile) {
     const int nk = min(kKeyTile, blk_last + 1 - j0);
     __syncthreads();
-    for (int idx = tid; idx < nk * rpk; idx += kThreads) Ks[idx] = to_f<T>(Kc[static_cast<int64_t>(j0) * rpk + idx]);
-    for (int idx = tid; idx < nk * rpv; idx += kThreads) Vs[idx] = to_f<T>(Vc[static_cast<int64_t>(j0) * rpv + idx]);
+    const int64_t prow = physical_row(p.pages, b, p.n_max, j0);     // a key tile of 32 rows lies inside one page
+    for (int idx = tid; idx < nk * rpk; idx += kThreads) Ks[idx] = to_f<T>(Kslab[prow * rpk + idx]);
+    for (int idx = tid; idx < nk * rpv; idx += kThreads) Vs[idx] = to_f<T>(Vslab[prow * rpv + idx]);
     __syncthreads();
     for (int j = 0; j < nk; ++j) {
       const float* kr = Ks + j * rpk + sub * cwk;
