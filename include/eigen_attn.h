@@ -162,8 +162,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
  * -slopes[i] * (pos - j) before the softmax, pos = len - 1 in a decode call (after the new row is
  * appended) and len0 + t for prompt token t.  slopes: HOST [H], each finite and >= 0; NULL or all
  * zeros switches the bias off (the default).  Copies into the workspace and synchronises `cuda_stream`;
- * calls still in flight on other streams must have finished.  With a bias the prefill runs on the
- * single-tile tensor-core kernel (bf16) or the CUDA-core kernel, not the warp-specialised one. */
+ * calls still in flight on other streams must have finished.  Every decode and prefill kernel carries the bias. */
 ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_stream);
 
 /* Grouped-query attention (the Llama-2-70b / Llama-3 models of Section 5.1): the layer's n_heads are the K/V

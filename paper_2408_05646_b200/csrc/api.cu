@@ -878,8 +878,8 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   size_t ws_smem = 0;
   const int ws_stages = tc_attn && h->tmaps_ok ? ea::prefill_tc_ws_stages(L.max_rp_k, L.max_rp_v, h->desc.d_head, &ws_smem) : 0;
-  if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 2 && !h->alibi)
-    e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, s, &h->launches);   // warp-specialised, 256 query rows per CTA
+  if (tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 && ws_stages >= 3)
+    e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, h->alibi, s, &h->launches);   // warp-specialised, 256 query rows per CTA
   else if (tc_attn && h->opt_prefill != 1)
     e = ea::launch_prefill_tc(p, L.max_rp_k, L.max_rp_v, s, &h->launches);  // single query tile per CTA (wide ranks)
   else

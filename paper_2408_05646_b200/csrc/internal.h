@@ -262,7 +262,8 @@ cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
-cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, bool alibi, cudaStream_t s,
+                                 uint64_t* launches);
 cudaError_t launch_project_tc(const ProjectTcParams& p, int max_rp, cudaStream_t s, uint64_t* launches);
 // Persistent variant: maps_qkv = CUtensorMap[3] (host) of the q, k, v tensors; needs d_head % 64 == 0.
 size_t project_tc_stream_smem(int max_rp, int d_head, int* stages);

@@ -8,16 +8,20 @@
 //     stages by TMA (tensor maps of the cache slabs, 64 x 64 boxes in the 128-byte swizzled layout the
 //     MMA descriptors name; each tile is fetched once for both query tiles).  Elements past the rank
 //     and rows past the capacity arrive as zeros;
-//   * two threads feed the tensor pipe, one per query tile: PV of key tile j when the softmax group has
-//     written P(j), then S of tile j + 3 into the buffer that P(j) occupied; every group of MMAs is
-//     followed by a tcgen05.commit onto the mbarrier that its consumer waits on;
-//   * two softmax warpgroups (4 warps each, one thread per query row = one TMEM lane), one per query
-//     tile.  S is double-buffered in TMEM (2 x 64 columns per group), so the S product of key tile
-//     j + 1 runs while the group turns tile j into P; a 64-key row fits in registers, and the row of
-//     tile j + 1 is fetched from TMEM while the exponentials of tile j run (the softmax warps take
-//     registers from the other warps for that).  P(j) (bf16) goes into the first 32 columns of the
-//     buffer that S(j + 1) has just left and is the A operand of the PV product straight from TMEM: it
-//     never touches shared memory.  A buffer thus cycles S(t) -> registers -> P(t-1) -> PV(t-1) -> S(t+2).
+//   * two threads feed the tensor pipe, one per query tile.  S is double-buffered in TMEM (2 x 64
+//     columns per query tile): S(j + 1) is computed while the softmax works on S(j).  Per key tile j the
+//     issuer waits for P(j), issues O' += P(j) V'(j), and once that product has read P(j) issues S(j + 2)
+//     into the buffer P(j) occupied; every group of MMAs is followed by a tcgen05.commit onto the
+//     mbarrier its consumer waits on;
+//   * sixteen softmax warps, four per scheduler, so that the fixed latencies of one warp's instruction
+//     stream are covered by the others.  A query tile has two warpgroups: a thread owns one query row
+//     (= one TMEM lane) and one half of the tile's 64 keys.  Per key tile it loads its 32 scores, takes
+//     their maximum, agrees with the other half of its row on the softmax reference through one
+//     reducing barrier (the reference moves only when some row's maximum grew by more than 8 in the
+//     log2 domain; only then do the halves exchange maxima through shared memory and rescale O'),
+//     computes 32 exponentials and writes P (bf16) IN PLACE over the first 32 columns of the S buffer,
+//     from where it is the A operand of the PV product: P never touches shared memory.
+//     The ALiBi bias (per-head slope) is added to the scaled scores in a second instantiation.
 // TMEM (512 columns): S_A[2], S_B[2] (64 columns each, P aliased), O'_A, O'_B (up to 128 each).
 // Every wait is bounded.
 #include <cuda_bf16.h>
@@ -31,13 +35,17 @@ namespace {
 using namespace tc;
 
 constexpr int kKeys = 64;                     // key rows per tile
+constexpr int kHalfKeys = kKeys / 2;          // keys per softmax thread and tile
 constexpr int kAtomBytes = kKeys * 128;       // one swizzled atom column of a K'/V' tile: 64 rows x 64 elements
-constexpr int kSoftmaxWarps = 8;
-constexpr int kMmaWarp = 8;                   // issues the MMAs of query tile A (and the lift)
-constexpr int kLoadWarp = 9;                  // lane 0 issues the TMA copies
-constexpr int kMmaWarpB = 10;                 // issues the MMAs of query tile B
-constexpr int kWsThreads = 12 * 32;           // 8 softmax warps, two MMA issuers, TMA producer, one spare warp
-constexpr int kRegsSoftmax = 224, kRegsOther = 56;   // registers per thread after the reallocation (launch: 168)
+constexpr int kSoftmaxWarps = 16;             // warpgroups 0,1: query tile A (keys 0..31, 32..63); 2,3: tile B
+constexpr int kMmaWarp = 16;                  // issues the MMAs of query tile A (and the lift)
+constexpr int kLoadWarp = 17;                 // lane 0 issues the TMA copies
+constexpr int kMmaWarpB = 18;                 // issues the MMAs of query tile B
+constexpr int kWsThreads = 20 * 32;           // 16 softmax warps, two MMA issuers, TMA producer, one spare warp
+// Registers per thread after the reallocation: the CTA is launched with 640 x 96; the last warpgroup keeps 40,
+// the softmax warpgroups take 104: 128 x 40 + 512 x 104 = 58 368 <= 61 440.
+constexpr int kRegsSoftmax = 104, kRegsOther = 40;
+static_assert(128 * kRegsOther + 512 * kRegsSoftmax <= kWsThreads * 96, "register split exceeds the launch");
 constexpr int kMaxStages = 8;
 
 struct __align__(16) WsHeader {
@@ -49,15 +57,18 @@ struct __align__(16) WsHeader {
   unsigned long long lift_done;
   uint32_t tmem_base;
   int abort_flag;
+  float exch[2][2][kTile];                    // [query tile][half][row]: row maxima (main loop), row sums (epilogue)
 };
+static_assert(sizeof(WsHeader) <= 3072, "header outgrew its area");
+constexpr int kHeaderBytes = 3072;            // tiles start here (1024-byte aligned for the swizzled layout)
 
-// One thread's share of a canonical (no swizzle) Q' tile of 128 rows, loaded by the 128 threads of a softmax
-// group: 16-byte chunks (row, c); two neighbouring lanes fetch the two halves of a 32-byte piece of a row.
+// One thread's share of a canonical (no swizzle) Q' tile of 128 rows, loaded by the 256 threads of a query tile:
+// 16-byte chunks (row, c); two neighbouring lanes fetch the two halves of a 32-byte piece of a row.
 __device__ __forceinline__ void load_q_tile_async(unsigned char* dst, const __nv_bfloat16* src, int rp, int rows_valid,
                                                   int nch, int t) {
   const int src_chunks = rp >> 3;
   const int group_stride = nch << 7;
-  for (int idx = t; idx < kTile * nch; idx += kTile) {
+  for (int idx = t; idx < kTile * nch; idx += 2 * kTile) {
     const int c = ((idx / (2 * kTile)) << 1) + (idx & 1), row = (idx >> 1) & (kTile - 1);
     const bool live = row < rows_valid && c < src_chunks;
     const void* g = live ? static_cast<const void*>(src + static_cast<int64_t>(row) * rp + c * 8) : src;
@@ -65,32 +76,20 @@ __device__ __forceinline__ void load_q_tile_async(unsigned char* dst, const __nv
   }
 }
 
-// One row of a 64-key tile: exponentials relative to the reference `neg_m` (= -m, log2 domain), their sum,
-// and P as 32 bf16 pairs (round to nearest) in `pk`.  DIAG: keys past `my_pos` get weight zero.  TRACK: also
-// returns the row maximum of the raw scores (for the lazy reference check).
-template <bool DIAG, bool TRACK>
-__device__ __forceinline__ float exp_row(const uint32_t (&r)[64], float scale, float neg_m, int key0, int my_pos,
-                                         uint32_t (&pk)[32], float* raw_max) {
-  float sum0 = 0.f, sum1 = 0.f;
-  float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const int c = 2 * i;
-    const float s0 = __uint_as_float(r[c]), s1 = __uint_as_float(r[c + 1]);
-    if (TRACK) mx[i & 3] = max3(mx[i & 3], s0, s1);
-    float y0, y1;
-    fma2(y0, y1, s0, s1, scale, neg_m);
-    float e0 = ex2(y0), e1 = ex2(y1);
-    if (DIAG) {
-      if (key0 + c > my_pos) e0 = 0.f;
-      if (key0 + c + 1 > my_pos) e1 = 0.f;
-    }
-    add2(sum0, sum1, e0, e1);
-    pk[i] = pack_bf16(e0, e1);
-  }
-  if (TRACK) *raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-  return sum0 + sum1;
+// Barrier of the 256 softmax threads of one query tile that also ORs a predicate over them.
+__device__ __forceinline__ bool tile_barrier_or(int id, bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, %2, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"(pred ? 1u : 0u), "r"(id)
+      : "memory");
+  return out != 0;
 }
+__device__ __forceinline__ void tile_barrier(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
 
 // S = Q' K'^T for one query tile and one key tile: KS steps of 16 rank elements.  K' sits in atom columns of
 // 64 elements (8192 bytes each); a step advances 32 bytes along the swizzled rows.
@@ -113,6 +112,7 @@ __device__ __forceinline__ void issue_s_steps(int ks, uint32_t d_tmem, uint64_t 
   }
 }
 
+template <bool ALIBI>
 __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const PrefillParams p, int stages) {
   extern __shared__ __align__(1024) unsigned char smem[];
   WsHeader* hdr = reinterpret_cast<WsHeader*>(smem);
@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int o_bytes = kTile * rpv16 * 2;                     // an O' tile of the epilogue
   const int stage_bytes = k_bytes + v_bytes;
 
-  unsigned char* tiles = smem + 1024;
+  unsigned char* tiles = smem + kHeaderBytes;
   unsigned char* Qs = tiles;                                 // Q_A, Q_B
   unsigned char* ring = Qs + 2 * q_bytes;                    // stages x (K tile, V tile)
 
@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     for (int x = 0; x < 2; ++x) {
       for (int bb = 0; bb < 2; ++bb) {
         mbar_init(&hdr->s_full[x][bb], 1);
-        mbar_init(&hdr->p_full[x][bb], kTile);
+        mbar_init(&hdr->p_full[x][bb], 2 * kTile);           // both halves of every row
         mbar_init(&hdr->o_done[x][bb], 1);
       }
     }
@@ -167,7 +167,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   tc_fence_after();
   const uint32_t tmem = hdr->tmem_base;
   volatile int* abort_flag = &hdr->abort_flag;
-
 
   if (warp >= kSoftmaxWarps) {
   reg_dealloc<kRegsOther>();
@@ -208,10 +207,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     }
   } else if (warp == kMmaWarp || warp == kMmaWarpB) {
     // ------------------------------------------------------------------ MMA issuers, one per query tile
-    // Per key tile j: PV(j) once the group has written P(j) (into the buffer S(j + 1) came from); then, once
-    // PV(j) has read P out of that buffer, S(j + 3) into it.  S(0) and S(1) go out up front, S(2) when P(0)
-    // is there (the group then holds S(0) in registers).  The two issuers share nothing but the tensor pipe
-    // and the ring, so neither query tile waits for the other.
+    // S(0) and S(1) go out up front.  Per key tile j: O' += P(j) V'(j) once both halves of every row have
+    // written P(j) over S(j); then, once that product has read P(j), S(j + 2) into the same buffer.  The two
+    // issuers share nothing but the tensor pipe and the ring, so neither query tile waits for the other.
     if (lane == 0) {
       const int x = warp == kMmaWarpB ? 1 : 0;
       const int nt = n_tiles[x];
@@ -246,11 +244,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         ok = mbar_wait(&hdr->p_full[x][buf], buf_parity, p.status) && !*abort_flag;
         if (!ok) break;
         tc_fence_after();
-        if (j == 0 && nt > 2) {
-          issue_s_tile(0);
-          if (!ok) break;
-        }
-        const uint32_t tP = tSx + (buf ^ 1) * kKeys;         // P: 64 bf16 per lane in 32 columns
+        const uint32_t tP = tSx + buf * kKeys;               // P(j): 64 bf16 per lane in the first 32 columns of S(j)
         const uint64_t bv = dv0 + stage * stage_step;
 #pragma unroll
         for (int s = 0; s < kKeys / 16; ++s)                 // O'_x += P_x V_j over the 64 keys
@@ -258,10 +252,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
         mma_commit(&hdr->o_done[x][buf]);
         mma_commit(&hdr->kv_empty[stage]);                   // PV is this tile's last reader of the stage
         if (++stage == stages) stage = 0;
-        if (j + 3 < nt) {
+        if (j + 2 < nt) {
           ok = mbar_wait(&hdr->o_done[x][buf], buf_parity, p.status) && !*abort_flag;
           if (!ok) break;
-          issue_s_tile(buf ^ 1);
+          issue_s_tile(buf);
         }
       }
       // Key tiles that only the other query tile reads still need this tile's arrival on their stage, one
@@ -285,7 +279,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int img16 = p.d_head * rpv16 * 2 / 16;               // 16-byte words per image
   if (run) {
     const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.uvl16_off);
-    for (int idx = tid - kMmaWarp * 32; idx < 2 * img16; idx += kWsThreads - kSoftmaxWarps * 32)
+    for (int idx = tid - kSoftmaxWarps * 32; idx < 2 * img16; idx += kWsThreads - kSoftmaxWarps * 32)
       reinterpret_cast<uint4*>(Uh)[idx] = __ldg(Ug + idx);
   }
   fence_async_smem();
@@ -317,127 +311,148 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   reg_alloc<kRegsSoftmax>();
   {
     // ------------------------------------------------------------------ softmax warpgroups
-    const int x = warp >> 2;                                 // 0 = tile A, 1 = tile B
+    const int x = warp >> 3;                                 // 0 = tile A, 1 = tile B
+    const int hf = (warp >> 2) & 1;                          // which half of a tile's 64 keys
     const int row = (warp & 3) * 32 + lane;
+    const int bar_id = 1 + x;                                // named barrier of this query tile's 256 threads
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + x * kTile;        // S buffers at +0 and +64
     const uint32_t tO = tmem + lane_base + 256 + x * kTile;
     const int tx = t0 + x * kTile;
     const int my_pos = p.len0 + tx + row;                    // last key this thread's query sees
-    {                                                        // this group's Q' tile (zeros past the prompt's end)
+    {                                                        // this tile's Q' (zeros past the prompt's end)
       const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.qp) +
                                 static_cast<int64_t>(hd.lr_k_off) * total_rows + static_cast<int64_t>(b) * p.T * hd.rp_k;
       const int q_rows = max(0, min(kTile, p.T - tx));
       load_q_tile_async(Qs + x * q_bytes, q_rows > 0 ? Qg + static_cast<int64_t>(tx) * hd.rp_k : Qg, hd.rp_k, q_rows,
-                        nch_k, row);
+                        nch_k, hf * kTile + row);
       cp_async_commit();
       cp_async_wait<0>();
       fence_async_smem();
       mbar_arrive(&hdr->q_full);
     }
+    // columns of O' (and of the lifted output) each half of a row looks after in the rescale and the epilogue
+    const int o_split = ((rpv16 >> 4) + 1) / 2 * 16;
+    const int o_lo = hf ? o_split : 0, o_hi = hf ? rpv16 : o_split;
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
     const int nt = n_tiles[x];
-    // One key tile: `cur` holds this thread's row of S(j); the row of S(j + 1) is requested into `nxt` before
-    // the arithmetic starts and awaited before P(j) goes out over the buffer it came from.
-    auto tile = [&](const uint32_t (&cur)[64], uint32_t (&nxt)[64], int j) {
-      const int key0 = j * kKeys, buf = j & 1;
-      const bool has_next = j + 1 < nt;
-      if (has_next) {
-        ok = mbar_wait(&hdr->s_full[x][buf ^ 1], ((j + 1) >> 1) & 1u, p.status);
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);    // one decision for the whole warp
-        if (!ok) return;
+    const float slope2 = ALIBI ? hd.alibi_slope2 : 0.f;
+
+    // The 256 threads of a query tile meet at named barriers, which have no time limit: every decision to leave
+    // the loop is therefore taken through a reducing barrier, so that all of them leave after the same tile.
+    for (int j = 0; j < nt; ++j) {
+      const int buf = j & 1;
+      const int key0 = j * kKeys + hf * kHalfKeys;           // first key of this thread's half
+      const uint32_t tSb = tS + buf * kKeys;
+      const bool waited = mbar_wait(&hdr->s_full[x][buf], (j >> 1) & 1u, p.status);
+      const bool diag = j * kKeys + kKeys - 1 > p.len0 + tx; // some (row, key) pair of the tile is masked
+      uint32_t r[kHalfKeys];
+      float cand = -INFINITY;                                // this half-row's largest score, scaled (log2 domain)
+      if (waited) {
         tc_fence_after();
-        tmem_ld64(tS + (buf ^ 1) * kKeys, nxt);
-      }
-      const uint32_t tP = tS + (buf ^ 1) * kKeys;            // P(j) goes where S(j + 1) was
-      const bool diag = key0 + kKeys - 1 > p.len0 + tx;      // some (row, key) pair of the tile is masked
-      // Lazy reference: the exponentials use m_run, which follows the true maximum only when that has grown
-      // by more than 8 (a factor 256 that fp32 sums and bf16 P absorb); O' is rescaled only then.
-      float alpha = 1.f, row_sum;
-      uint32_t pk[32];
-      if (j == 0 || diag) {                                  // maximum first, then the exponentials
-        float row_max = -INFINITY;
+        tmem_ld16(tSb + hf * kHalfKeys, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
+        tmem_ld16(tSb + hf * kHalfKeys + 16, *reinterpret_cast<uint32_t(*)[16]>(&r[16]));
+        tmem_wait_ld();
+        if (ALIBI) {
+          // scaled score plus the bias slope * (key - position), kept in place of the raw score
+          float off = slope2 * static_cast<float>(key0 - my_pos);
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (!diag || key0 + i <= my_pos) row_max = fmaxf(row_max, __uint_as_float(cur[i]));
-        row_max *= p.scale_log2;                             // the scale is positive: max and scale commute
+          for (int c = 0; c < kHalfKeys; ++c) {
+            r[c] = __float_as_uint(fmaf(__uint_as_float(r[c]), p.scale_log2, off));
+            off += slope2;
+          }
+        }
+        if (diag) {
+#pragma unroll
+          for (int c = 0; c < kHalfKeys; ++c)
+            if (key0 + c <= my_pos) cand = fmaxf(cand, __uint_as_float(r[c]));
+        } else {
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < kHalfKeys; c += 4) {
+            mx0 = max3(mx0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+          }
+          cand = fmaxf(mx0, mx1);
+        }
+        if (!ALIBI) cand *= p.scale_log2;                    // the scale is positive: max and scale commute
+      }
+      // Lazy reference: it follows the row maximum only when that has grown by more than 8 (a factor 256 that
+      // fp32 sums and bf16 P absorb).  One reducing barrier tells whether any row of the tile needs it; it also
+      // orders the other half's loads of S before this half's stores of P into the same columns.
+      float alpha = 1.f;
+      if (tile_barrier_or(bar_id, !waited || cand > m_run + 8.f || *abort_flag != 0)) {
+        hdr->exch[x][hf][row] = cand;
+        if (tile_barrier_or(bar_id, !waited || *abort_flag != 0)) {   // a wait gave up somewhere: all 256 leave here
+          ok = false;
+          break;
+        }
+        const float row_max = fmaxf(cand, hdr->exch[x][hf ^ 1][row]);  // both halves take the same decision
         if (row_max > m_run + 8.f) {
           alpha = ex2(m_run - row_max);
           m_run = row_max;
         }
-        row_sum = diag ? exp_row<true, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr)
-                       : exp_row<false, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr);
-      } else {                                               // exponentials against the old reference, maximum on the side
-        float raw_max;
-        row_sum = exp_row<false, true>(cur, p.scale_log2, -m_run, key0, my_pos, pk, &raw_max);
-        const float row_max = raw_max * p.scale_log2;
-        if (__any_sync(0xffffffffu, row_max > m_run + 8.f)) { // the reference moved for some row: once more
-          if (row_max > m_run + 8.f) {
-            alpha = ex2(m_run - row_max);
-            m_run = row_max;
-          }
-          row_sum = exp_row<false, false>(cur, p.scale_log2, -m_run, key0, my_pos, pk, nullptr);
-        }
-      }
-      if (has_next) {
-        tmem_wait_ld();                                      // S(j + 1) is in registers: its buffer may take P(j)
-      } else if (j >= 2) {                                   // no S(j + 1) whose arrival implies it: PV_x(j-2) has read P(j-2)
-        ok = mbar_wait(&hdr->o_done[x][buf], ((j - 2) >> 1) & 1u, p.status);
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
-        if (!ok) return;
-        tc_fence_after();
-      }
-      tmem_st16(tP, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
-      tmem_st16(tP + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
-      l_run = l_run * alpha + row_sum;
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rescale this row of O' (rare after the first tiles)
-        ok = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);   // PV_x(j-1) has added to O'
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
-        if (!ok) return;
-        tc_fence_after();
+        l_run *= alpha;
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {          // rescale this half's columns of the row of O'
+          const bool got = mbar_wait(&hdr->o_done[x][buf ^ 1], ((j - 1) >> 1) & 1u, p.status);   // PV(j-1) has added to O'
+          if (__all_sync(0xffffffffu, got)) {
+            tc_fence_after();
 #pragma unroll 1
-        for (int h0 = 0; h0 < rpv16; h0 += 16) {
-          uint32_t o[16];
-          tmem_ld16(tO + h0, o);
-          tmem_wait_ld();
+            for (int h0 = o_lo; h0 < o_hi; h0 += 16) {
+              uint32_t o[16];
+              tmem_ld16(tO + h0, o);
+              tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-          tmem_st16(tO + h0, o);
+              for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st16(tO + h0, o);
+            }
+          } else {
+            *abort_flag = 1;                                 // seen by every thread of the tile at the next barrier
+          }
         }
       }
+      // exponentials against the reference, their sum, P as bf16 pairs
+      uint32_t pk[kHalfKeys / 2];
+      float sum0 = 0.f, sum1 = 0.f;
+      const float neg_m = -m_run;
+#pragma unroll
+      for (int i = 0; i < kHalfKeys / 2; ++i) {
+        const int c = 2 * i;
+        float y0, y1;
+        if (ALIBI) {
+          y0 = __uint_as_float(r[c]) + neg_m;
+          y1 = __uint_as_float(r[c + 1]) + neg_m;
+        } else {
+          fma2(y0, y1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), p.scale_log2, neg_m);
+        }
+        float e0 = ex2(y0), e1 = ex2(y1);
+        if (diag) {
+          if (key0 + c > my_pos) e0 = 0.f;
+          if (key0 + c + 1 > my_pos) e1 = 0.f;
+        }
+        add2(sum0, sum1, e0, e1);
+        pk[i] = pack_bf16(e0, e1);
+      }
+      l_run += sum0 + sum1;
+      tmem_st16(tSb + hf * (kHalfKeys / 2), pk);             // in place: P(j) takes the first 32 columns of S(j)
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&hdr->p_full[x][buf]);
-    };
-    {
-      uint32_t ra[64], rb[64];
-      if (nt > 0) {
-        ok = mbar_wait(&hdr->s_full[x][0], 0, p.status);
-        ok = __all_sync(0xffffffffu, ok && !*abort_flag);
-        if (ok) {
-          tc_fence_after();
-          tmem_ld64(tS, ra);
-          tmem_wait_ld();
-        }
-      }
-      for (int j = 0; j < nt && ok; j += 2) {
-        tile(ra, rb, j);
-        if (ok && j + 1 < nt) tile(rb, ra, j + 1);
-      }
     }
-    if (ok && n_tiles[x] > 0) {
-      ok = mbar_wait(&hdr->o_done[x][(n_tiles[x] - 1) & 1], ((n_tiles[x] - 1) >> 1) & 1u, p.status);
+    if (ok && nt > 0) {
+      ok = mbar_wait(&hdr->o_done[x][(nt - 1) & 1], ((nt - 1) >> 1) & 1u, p.status);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
     }
     if (!ok) *abort_flag = 1;
+    hdr->exch[x][hf][row] = l_run;                           // the two halves' sums share the reference
 
     // ---- epilogue part 1 (after every role is done with the main loop)
     tc_fence_before();
     __syncthreads();                                         // #1
     const bool run = !*abort_flag && n_tiles[x] > 0;
-    const float inv_l = 1.f / l_run;
+    const float inv_l = 1.f / (hdr->exch[x][0][row] + hdr->exch[x][1][row]);
     const bool lowrank = (p.flags & 0x2u) != 0;
     const int q_valid = min(kTile, p.T - tx);
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out);
@@ -446,7 +461,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     if (run) {
       tc_fence_after();
       __nv_bfloat16* dst_lr = out + b * p.out_stride_b + static_cast<int64_t>(tx + row) * p.out_stride_t + hd.lr_v_off;
-      for (int c0 = 0; c0 < rpv16; c0 += 16) {
+      for (int c0 = o_lo; c0 < o_hi; c0 += 16) {             // this half's columns of the row
         uint32_t r[16];
         tmem_ld16(tO + c0, r);
         tmem_wait_ld();
@@ -480,7 +495,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       if (ok2) {
         __nv_bfloat16* dst = out + b * p.out_stride_b + static_cast<int64_t>(tx + row) * p.out_stride_t +
                              static_cast<int64_t>(h) * p.d_head;
-        for (int c0 = 0; c0 < p.d_head; c0 += 16) {
+        const int d_split = ((p.d_head >> 4) + 1) / 2 * 16;  // this half's share of the d_head output columns
+        const int d_lo = hf ? d_split : 0, d_hi = hf ? p.d_head : d_split;
+        for (int c0 = d_lo; c0 < d_hi; c0 += 16) {
           uint32_t r[16];
           tmem_ld16(tS + c0, r);
           tmem_wait_ld();
@@ -511,26 +528,29 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
 // Stages of the K'/V' ring that fit beside the two Q tiles (0 = does not fit).
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes) {
   const size_t k16 = (max_rp_k + 15) & ~15, v16 = (max_rp_v + 15) & ~15;
-  const size_t fixed = 1024 + 2 * kTile * k16 * 2;
+  const size_t fixed = kHeaderBytes + 2 * kTile * k16 * 2;
   const size_t stage = (((k16 + 63) >> 6) + ((v16 + 63) >> 6)) * static_cast<size_t>(kAtomBytes);
   const size_t limit = 227 * 1024;
   int stages = 0;
-  for (int s = kMaxStages; s >= 3; --s)   // the S products run three key tiles ahead of the PV products
+  for (int s = kMaxStages; s >= 3; --s)   // the S products run two key tiles ahead of the PV products
     if (fixed + s * stage <= limit) { stages = s; break; }
   if (stages == 0) return 0;
   const size_t total = fixed + stages * stage;
-  const size_t epilogue = 1024 + 4 * kTile * v16 * 2 + 2 * static_cast<size_t>(d_head) * v16 * 2;
+  const size_t epilogue = kHeaderBytes + 4 * kTile * v16 * 2 + 2 * static_cast<size_t>(d_head) * v16 * 2;
   if (epilogue > total) return 0;
   *smem_bytes = total;
   return stages;
 }
 
-cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, cudaStream_t s, uint64_t* launches) {
-  static size_t configured[kMaxDevices] = {};
-  const cudaError_t ec = ensure_dynamic_smem(prefill_tc_ws_kernel, smem, configured);
+cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, bool alibi, cudaStream_t s,
+                                 uint64_t* launches) {
+  static size_t configured[2][kMaxDevices] = {};
+  const cudaError_t ec = alibi ? ensure_dynamic_smem(prefill_tc_ws_kernel<true>, smem, configured[1])
+                               : ensure_dynamic_smem(prefill_tc_ws_kernel<false>, smem, configured[0]);
   if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, (p.T + 2 * kTile - 1) / (2 * kTile));
-  prefill_tc_ws_kernel<<<grid, kWsThreads, smem, s>>>(p, stages);
+  if (alibi) prefill_tc_ws_kernel<true><<<grid, kWsThreads, smem, s>>>(p, stages);
+  else prefill_tc_ws_kernel<false><<<grid, kWsThreads, smem, s>>>(p, stages);
   ++*launches;
   return cudaGetLastError();
 }
