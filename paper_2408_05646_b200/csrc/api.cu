@@ -1121,14 +1121,14 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
     const int64_t wave = static_cast<int64_t>(h->sm_count) * ctas_per_sm;
     int64_t best = INT64_MAX;
     for (int64_t s2 = 1; s2 <= cap && s2 <= 256; ++s2) {
-      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 4);
+      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 6);
       if (cost < best) { best = cost; splits = s2; }
     }
   }
   p.splits = static_cast<int32_t>(splits);
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  const cudaError_t e = ea::launch_decode_gqa(p, smem, s, &h->launches);
+  const cudaError_t e = ea::launch_decode_gqa(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_gqa launch");
   return EA_OK;

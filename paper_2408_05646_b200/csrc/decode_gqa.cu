@@ -4,21 +4,22 @@
 // tensor cores worthwhile for a decode step.
 //
 // Per tile of 128 cached rows (tcgen05, accumulators in TMEM):
-//   S  [128 rows x 16]   = K'_tile [128 x r_k] . Q'^T   Q' = q U^K of the g queries (rows past g are zero), scaled
-//                                                       by log2(e)/sqrt(d_h), as bf16 high + low parts (two products)
+//   S    [128 rows x 16]  = K'_tile [128 x r_k] . Q'^T    Q' = q U^K of the g queries (rows past g are zero), scaled by
+//                                                         log2(e)/sqrt(d_h) and rounded to bf16
 //   softmax in base 2, one thread per cached row, g running maxima kept identical in every thread (lazy
-//   reference: a maximum moves only when it grew by more than 8), P rounded to bf16
-//   O' [16(128) x r_v] += P^T [16(128) x 128 rows] . V'_tile   P^T has the queries as rows.  The product has M = 128,
-//                                                       but only 16 rows of P^T exist in shared memory: the other
-//                                                       112 rows of the operand fall on whatever follows (Q', the
-//                                                       tiles: finite numbers) and fill rows of O' nobody reads
-// A tile of K' or V' rows is contiguous in the cache and arrives as one bulk copy (cp.async.bulk) into a row-major
-// staging buffer; the threads move it into the core-matrix layout the tensor core reads and the staging buffer takes
-// the next tile at once, a whole tile ahead of its use.  The score
-// product of tile t+1 goes out at the top of tile t, so it runs under tile t's softmax.  A fifth warp issues the
-// MMAs and the copies: tcgen05.mma issue blocks while the tensor pipe is busy, and a worker thread that issued them
-// held all 128 workers at the next barrier.  Workers and the issuer meet on mbarriers only.  Two CTAs per SM.  A unit split over several CTAs leaves partials (m, l, o') per query that
-// gqa_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
+//   reference: a maximum moves only when it grew by more than 8), P rounded to bf16 into P^T [16 x 128 rows]
+//   O'^T [r_v x 16]       += V'_tile^T [r_v x 128 rows] . P^T^T   the rank runs over the TMEM lanes, the queries over
+//                                                         16 columns: both operands exist in full (the V' tile is
+//                                                         128 elements wide with zeros past the rank, P^T has its 16 rows)
+// One CTA per SM with three roles that meet on mbarriers only:
+//   * one thread streams the K'/V' tiles by TMA (tensor maps of the cache slabs, 64 x 64 boxes, 128-byte swizzle:
+//     the layout the MMA descriptors name, so no thread ever moves a tile) into a ring of three or more stages,
+//     about 120 KB in flight;
+//   * one thread issues the MMAs: S(t + 1) goes out before the weighted sum of tile t, so it runs under tile t's
+//     softmax (S is double-buffered in TMEM, P^T in shared memory);
+//   * 128 workers (one per cached row of a tile = one TMEM lane of S; one per rank element = one lane of O'^T).
+// A unit split over several CTAs leaves partials (m, l, o') per query that gqa_combine_kernel merges and lifts
+// through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -29,10 +30,27 @@ namespace {
 
 using namespace tc;
 
-constexpr int kMaxGroup = 16;                 // query heads per K/V head (N of the score product)
-constexpr int kGqaThreads = kThreads + 32;    // 128 workers (one per cached row of a tile) + the issuing warp
+constexpr int kMaxGroup = 16;                 // query heads per K/V head (N of both products)
+constexpr int kGqaThreads = kThreads + 64;    // 128 workers + the MMA-issuing warp + the TMA warp
+constexpr int kGqaAtom = kTile * 128;         // one swizzled atom column of a tile: 128 rows x 64 elements
+constexpr int kGqaMaxStages = 6;
+constexpr int kGqaHeader = 1024;
 
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+// The same barrier, returning the OR of a predicate over the 128 workers: the barrier has no time limit, so the
+// decision to leave the tile loop is taken through it and every worker leaves after the same tile.
+__device__ __forceinline__ bool worker_sync_or(bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"(pred ? 1u : 0u), "n"(kThreads)
+      : "memory");
+  return out != 0;
+}
 
 // Warp maximum of a float in one instruction: floats ordered as integers (sign-magnitude -> two's complement).
 __device__ __forceinline__ float warp_max(float v) {
@@ -42,29 +60,24 @@ __device__ __forceinline__ float warp_max(float v) {
   i ^= (i >> 31) & 0x7fffffff;
   return __int_as_float(i);
 }
-// S = K'_tile Q'^T, KS steps of 16 rank elements, Q' high part then low part; unrolled so that the issuing thread
-// spends its time in the MMAs and not in address arithmetic
-template <int KS>
-__device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint64_t dk, uint64_t dq, uint32_t q_lo, uint32_t idesc) {
-#pragma unroll
-  for (int s = 0; s < KS; ++s) mma_ss(d_tmem, dk + s * 16, dq + s * 16, idesc, s > 0);
-#pragma unroll
-  for (int s = 0; s < KS; ++s) mma_ss(d_tmem, dk + s * 16, dq + q_lo + s * 16, idesc, true);
-}
 
 struct __align__(16) GqaSmemHeader {
-  unsigned long long s_done, o_done, k_full, v_full;
-  unsigned long long tiles_ready, p_ready;    // 128 arrivals each: tiles moved into place / P^T written
+  unsigned long long kv_full[kGqaMaxStages], kv_empty[kGqaMaxStages];
+  unsigned long long s_done[2], p_ready[2], o_done[2];   // per S / P^T buffer
+  unsigned long long q_ready;
   uint32_t tmem_base;
   int abort_flag;
-  float pad_[2];
   float red[2][kMaxGroup][4];                 // per query: the four warps' maxima / sums, alternating between tiles
 };
+static_assert(sizeof(GqaSmemHeader) <= kGqaHeader, "header outgrew its area");
+
+// Instruction descriptor with the A operand MN-major (bit 15) and B K-major: O'^T = V'^T P.
+__host__ __device__ constexpr uint32_t instr_desc_a_mn(int n) { return instr_desc(n, false) | (1u << 15); }
 
 // GP: query slots the kernel carries (the group size rounded up to 4, 8 or 16); slots past the group score zero
 // queries and are never written out.
 template <int GP>
-__global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDecodeParams p) {
+__global__ void __launch_bounds__(kGqaThreads, 1) decode_gqa_kernel(const GqaDecodeParams p, int stages) {
   extern __shared__ __align__(1024) unsigned char smem[];
   GqaSmemHeader* hdr = reinterpret_cast<GqaSmemHeader*>(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -73,20 +86,15 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
   const int G = p.group;
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
-  const int grp_k = (rpk16 >> 3) << 7, grp_v = (rpv16 >> 3) << 7, grp_p = (kTile >> 3) << 7;
-  const int rowb_k = hd.rp_k * 2, rowb_v = hd.rp_v * 2;      // bytes per cached row
-  const int kst_bytes = kTile * rowb_k, vst_bytes = kTile * rowb_v;          // staging, row-major
-  const int km_bytes = kTile * rpk16 * 2, vm_bytes = kTile * rpv16 * 2;      // core-matrix layout
-  const int q_bytes = kMaxGroup * rpk16 * 2;                 // one image (high or low part) of Q'
-  const int p_bytes = kMaxGroup * kTile * 2;                 // the 16 rows of P^T that exist
+  const int grp_k = (rpk16 >> 3) << 7, grp_p = (kTile >> 3) << 7;
+  const int ak = (rpk16 + 63) >> 6, av = (rpv16 + 63) >> 6;  // atom columns (64 elements) the copies fill
+  const int k_bytes = ak * kGqaAtom;
+  const int stage_bytes = k_bytes + 2 * kGqaAtom;            // the V' part always spans two atom columns (M = 128 of O'^T)
+  const int p_bytes = kMaxGroup * kTile * 2;                 // one P^T buffer
 
-  unsigned char* tiles = smem + 1024;
-  unsigned char* Ps = tiles;                                 // P^T [16 queries][128 rows], canonical (two 8-row groups)
-  unsigned char* Qs = Ps + p_bytes;                          // Q' images [16][rk16], canonical: high, then low
-  unsigned char* Kst = Qs + 2 * q_bytes;                     // K' tile as it lands
-  unsigned char* Vst = Kst + kst_bytes;                      // V' tile as it lands
-  unsigned char* Km = Vst + vst_bytes;                       // K' tile, canonical core-matrix layout
-  unsigned char* Vm = Km + km_bytes;                         // V' tile, canonical core-matrix layout
+  unsigned char* Qs = smem + kGqaHeader;                     // Q' image [16][rk16], canonical (4 KB reserved)
+  unsigned char* Ps = Qs + 4096;                             // P^T [2][16 queries][128 rows], canonical
+  unsigned char* ring = Ps + 2 * p_bytes;                    // stages x (K' atoms, V' atoms), 128-byte swizzle
 
   // rows and tiles of this sequence (a batch of unequal lengths gives every sequence its own count; the splits
   // of a unit divide the sequence's own tiles)
@@ -102,206 +110,229 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     }
     return;
   }
+  const int nt = t_hi - t_lo;
 
-  if (warp == 0) tmem_alloc(&hdr->tmem_base, 256);
+  if (warp == 0) tmem_alloc(&hdr->tmem_base, 128);
   if (tid == 0) {
-    mbar_init(&hdr->s_done, 1);
-    mbar_init(&hdr->o_done, 1);
-    mbar_init(&hdr->k_full, 1);
-    mbar_init(&hdr->v_full, 1);
-    mbar_init(&hdr->tiles_ready, kThreads);
-    mbar_init(&hdr->p_ready, kThreads);
+    for (int s = 0; s < kGqaMaxStages; ++s) {
+      mbar_init(&hdr->kv_full[s], 1);
+      mbar_init(&hdr->kv_empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&hdr->s_done[i], 1);
+      mbar_init(&hdr->p_ready[i], kThreads);
+      mbar_init(&hdr->o_done[i], 1);
+    }
+    mbar_init(&hdr->q_ready, kThreads);
     hdr->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // P^T, the Q' images and the tiles start as zeros (rows that no copy fills meet zero weights and must be finite;
-  // padding chunks of the core-matrix tiles stay zero)
-  for (int idx = tid; idx < (p_bytes + 2 * q_bytes + kst_bytes + vst_bytes + km_bytes + vm_bytes) / 16; idx += kGqaThreads)
-    reinterpret_cast<uint4*>(Ps)[idx] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  // Q' = q U^K for the g queries of the group, times log2(e)/sqrt(d_h), split into bf16 high + low parts
-  {
-    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b +
-                              static_cast<int64_t>(h) * G * p.d_head;
-    const float* U = p.basis + hd.uk_off;                    // d_head x rp_k, zero padded columns
-    for (int idx = tid; idx < G * hd.rp_k; idx += kGqaThreads) {
-      const int qi = idx / hd.rp_k, c = idx - qi * hd.rp_k;
-      float acc = 0.f;
-      for (int d = 0; d < p.d_head; ++d) acc = fmaf(__bfloat162float(qg[qi * p.d_head + d]), __ldg(U + d * hd.rp_k + c), acc);
-      acc *= p.q_scale;
-      const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-      const __nv_bfloat16 lo = __float2bfloat16_rn(acc - __bfloat162float(hi));
-      const uint32_t off = chunk_off(qi, c >> 3, grp_k) + (c & 7) * 2;
-      *reinterpret_cast<__nv_bfloat16*>(Qs + off) = hi;
-      *reinterpret_cast<__nv_bfloat16*>(Qs + q_bytes + off) = lo;
-    }
-  }
-  const uint64_t policy = policy_evict_first();
-  const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
-  const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
-  auto fetch_k = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_k;
-    mbar_arrive_expect_tx(&hdr->k_full, bytes);
-    bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
-  };
-  auto fetch_v = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
-    mbar_arrive_expect_tx(&hdr->v_full, bytes);
-    bulk_load(Vst, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
-  };
-  // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * group + c * 128 + (row % 8) * 16
-  auto relayout = [&](unsigned char* dst, const unsigned char* src, int rowb, int grp) {
-    relayout_tile(dst, src, rowb, grp, warp, lane);
-  };
+  // Q' and P^T start as zeros (padding rows and columns); a V' atom column that no copy fills must hold zeros too
+  for (int idx = tid; idx < (4096 + 2 * p_bytes) / 16; idx += kGqaThreads) reinterpret_cast<uint4*>(Qs)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  if (av < 2)
+    for (int st = 0; st < stages; ++st)
+      for (int idx = tid; idx < kGqaAtom / 16; idx += kGqaThreads)
+        reinterpret_cast<uint4*>(ring + st * stage_bytes + k_bytes + kGqaAtom)[idx] = make_uint4(0u, 0u, 0u, 0u);
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = hdr->tmem_base;
-  const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-  const uint32_t tO = tmem + 64;                             // O': lanes = queries, columns = rank of V
+  const uint32_t tO = tmem + 64;                             // O'^T: lanes = rank of V, columns = queries
   volatile int* abort_flag = &hdr->abort_flag;
-  const uint32_t idesc_s = instr_desc(kMaxGroup, false);
-  const uint32_t idesc_o = instr_desc(rpv16, true);
   const int ks_steps = rpk16 >> 4;
-  const uint64_t desc_k = smem_desc(smem_u32(Km), 128, grp_k);
-  const uint64_t desc_q = smem_desc(smem_u32(Qs), 128, grp_k);
-  const uint64_t desc_p = smem_desc(smem_u32(Ps), 128, grp_p);
-  const uint64_t desc_v = smem_desc(smem_u32(Vm), grp_v, 128);   // MN-major operand: 8-row groups along K, chunks along N
-  // S(t) = K'(t) Q'^T into score buffer `buf` (columns 32 buf .. 32 buf + 15)
-  auto issue_s = [&](int buf) {
-    tc_fence_after();
-    const uint32_t d = tmem + 32 * buf, q_lo = static_cast<uint32_t>(q_bytes >> 4);
-    switch (ks_steps) {
-      case 1: issue_scores<1>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 2: issue_scores<2>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 3: issue_scores<3>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 4: issue_scores<4>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 5: issue_scores<5>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 6: issue_scores<6>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      case 7: issue_scores<7>(d, desc_k, desc_q, q_lo, idesc_s); break;
-      default: issue_scores<8>(d, desc_k, desc_q, q_lo, idesc_s); break;
-    }
-    mma_commit(&hdr->s_done);
-  };
-  bool ok = true;
-  const bool issuer = warp == kThreads / 32;                 // warp 4
-  if (issuer && lane == 0) {
-    fetch_k(t_lo);
-    fetch_v(t_lo);
-  }
-  // the first K' tile: into the core-matrix layout, its score product, and the staging buffer takes the second
-  if (!issuer) {
-    if (!mbar_wait(&hdr->k_full, 0, p.status)) *abort_flag = 1;
-    relayout(Km, Kst, rowb_k, grp_k);
-    fence_async_smem();
-  }
-  __syncthreads();
-  if (*abort_flag) ok = false;
 
-  if (issuer) {
-    // ------------------------------------------------------------------ the issuing warp
-    if (lane == 0 && ok) {
-      issue_s(0);
-      if (t_lo + 1 < t_hi) fetch_k(t_lo + 1);
-      for (int t = t_lo; t < t_hi && ok; ++t) {
-        const uint32_t par = (t - t_lo) & 1u;
-        ok = mbar_wait(&hdr->tiles_ready, par, p.status) && !*abort_flag;   // K'(t+1), V'(t) are in place
-        if (!ok) break;
-        if (t + 1 < t_hi) {
-          issue_s(static_cast<int>(par ^ 1u));
-          fetch_v(t + 1);
-          if (t + 2 < t_hi) fetch_k(t + 2);
+  if (warp == 5) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const unsigned char* maps = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
+      const void* map_k = maps;
+      const void* map_v = maps + 128;
+      tensormap_acquire(map_k);
+      tensormap_acquire(map_v);
+      const uint32_t tx_bytes = static_cast<uint32_t>((ak + av) * kGqaAtom);   // what the copies of a stage deliver
+      bool ok = true;
+      int stage = 0, issued = 0;
+      uint32_t empty_parity = 1;
+      for (int i = 0; i < nt; ++i) {
+        if (i >= stages) {
+          ok = mbar_wait(&hdr->kv_empty[stage], empty_parity, p.status) && !*abort_flag;
+          if (!ok) { *abort_flag = 1; break; }
         }
-        ok = mbar_wait(&hdr->p_ready, par, p.status) && !*abort_flag;       // P^T(t) written, O' rescaled if needed
+        unsigned char* st = ring + stage * stage_bytes;
+        const int row0 = (t_lo + i) * kTile;
+        mbar_arrive_expect_tx(&hdr->kv_full[stage], tx_bytes);
+        for (int a = 0; a < ak; ++a)
+          for (int hh = 0; hh < 2; ++hh)                     // two boxes of 64 rows fill one atom column of 128 rows
+            tma_load_3d(st + a * kGqaAtom + hh * (kGqaAtom / 2), map_k, a * 64, row0 + hh * 64, b, &hdr->kv_full[stage]);
+        for (int a = 0; a < av; ++a)
+          for (int hh = 0; hh < 2; ++hh)
+            tma_load_3d(st + k_bytes + a * kGqaAtom + hh * (kGqaAtom / 2), map_v, a * 64, row0 + hh * 64, b, &hdr->kv_full[stage]);
+        ++issued;
+        if (++stage == stages) { stage = 0; empty_parity ^= 1u; }
+      }
+      // if the CTA gives up, its copies in flight must land before it leaves
+      if (!ok || *abort_flag) {
+        for (int s2 = 0; s2 < stages; ++s2) {
+          int last = -1;
+          for (int jj = s2; jj < issued; jj += stages) last = jj;
+          if (last >= 0) mbar_wait(&hdr->kv_full[s2], (last / stages) & 1u, p.status);
+        }
+      }
+    }
+  } else if (warp == 4) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = instr_desc(kMaxGroup, false);
+      const uint32_t idesc_o = instr_desc_a_mn(kMaxGroup);
+      const uint32_t ra = smem_u32(ring);
+      const uint64_t dk0 = smem_desc_sw128(ra, 16, 1024);                      // K' tile of stage 0: A, K-major
+      const uint64_t dv0 = smem_desc_sw128(ra + k_bytes, kGqaAtom, 1024);      // V' tile of stage 0: A, MN-major
+      const uint64_t dq = smem_desc(smem_u32(Qs), 128, grp_k);                 // Q': B, K-major, 16 rows
+      const uint64_t dp0 = smem_desc(smem_u32(Ps), 128, grp_p);                // P^T: B, K-major, 16 rows
+      const uint64_t stage_step = static_cast<uint64_t>(stage_bytes >> 4);
+      bool ok = mbar_wait(&hdr->q_ready, 0, p.status);
+      int s_stage = 0;
+      uint32_t s_parity = 0;
+      auto issue_s = [&](int buf) {                          // S(next tile in the ring) into score buffer `buf`
+        ok = mbar_wait(&hdr->kv_full[s_stage], s_parity, p.status);
+        if (!ok) return;
+        tc_fence_after();
+        const uint64_t dk = dk0 + s_stage * stage_step;
+        for (int s = 0; s < ks_steps; ++s)
+          mma_ss(tmem + 32 * buf, dk + (s >> 2) * (kGqaAtom >> 4) + (s & 3) * 2, dq + s * 16, idesc_s, s > 0);
+        mma_commit(&hdr->s_done[buf]);
+        if (++s_stage == stages) { s_stage = 0; s_parity ^= 1u; }
+      };
+      if (ok) issue_s(0);
+      int stage = 0;
+      for (int i = 0; i < nt && ok; ++i) {
+        const int buf = i & 1;
+        const uint32_t par = (i >> 1) & 1u;
+        if (i + 1 < nt) {                                    // S(i + 1) runs under the softmax of tile i
+          issue_s(buf ^ 1);
+          if (!ok) break;
+        }
+        ok = mbar_wait(&hdr->p_ready[buf], par, p.status) && !*abort_flag;     // P^T(i) written, O'^T rescaled if needed
         if (!ok) break;
         tc_fence_after();
-        for (int s = 0; s < kTile / 16; ++s)                 // O' += P^T V'(t), 16 cached rows (two 8-row groups) a step
-          mma_ss(tO, desc_p + s * 16, desc_v + s * ((2 * grp_v) >> 4), idesc_o, t > t_lo || s > 0);
-        mma_commit(&hdr->o_done);
+        const uint64_t dv = dv0 + stage * stage_step, dp = dp0 + static_cast<uint64_t>(buf) * (p_bytes >> 4);
+#pragma unroll
+        for (int s = 0; s < kTile / 16; ++s)                 // O'^T += V'(i)^T P(i), 16 cached rows a step
+          mma_ss(tO, dv + s * (2048 >> 4), dp + s * 16, idesc_o, i > 0 || s > 0);
+        mma_commit(&hdr->o_done[buf]);
+        mma_commit(&hdr->kv_empty[stage]);                   // the weighted sum is the stage's last reader
+        if (++stage == stages) stage = 0;
       }
+      // the last commits' arrivals must have landed before the CTA may leave
+      if (ok) ok = mbar_wait(&hdr->kv_empty[(nt - 1) % stages], ((nt - 1) / stages) & 1u, p.status);
       if (!ok) *abort_flag = 1;
     }
+  }
+  if (warp >= 4) {
     __syncthreads();                                         // the workers' epilogue
     __syncthreads();
     return;
   }
 
   // -------------------------------------------------------------------- the 128 workers
+  // Q' = q U^K for the g queries of the group, times log2(e)/sqrt(d_h), rounded to bf16
+  {
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b +
+                              static_cast<int64_t>(h) * G * p.d_head;
+    const float* U = p.basis + hd.uk_off;                    // d_head x rp_k, zero padded columns
+    // The queries go through shared memory as fp32 (the P^T buffers are idle until the first tile), a thread owns
+    // column c of U^K for all queries of the group, 32 loads of U in flight: the projection costs a few
+    // microseconds per CTA, and every CTA pays it before its first product.
+    float* qs = reinterpret_cast<float*>(Ps);                // [G][d_head]
+    for (int idx = tid; idx < G * p.d_head; idx += kThreads) qs[idx] = __bfloat162float(qg[idx]);
+    worker_sync();
+    for (int c = tid; c < hd.rp_k; c += kThreads) {
+      float acc[GP];
+#pragma unroll
+      for (int qi = 0; qi < GP; ++qi) acc[qi] = 0.f;
+#pragma unroll 32
+      for (int d = 0; d < p.d_head; ++d) {
+        const float u = __ldg(U + d * hd.rp_k + c);
+#pragma unroll
+        for (int qi = 0; qi < GP; ++qi)
+          if (qi < G) acc[qi] = fmaf(qs[qi * p.d_head + d], u, acc[qi]);
+      }
+#pragma unroll
+      for (int qi = 0; qi < GP; ++qi)
+        if (qi < G)
+          *reinterpret_cast<__nv_bfloat16*>(Qs + chunk_off(qi, c >> 3, grp_k) + (c & 7) * 2) = __float2bfloat16_rn(acc[qi] * p.q_scale);
+    }
+    worker_sync();                                           // every thread is done reading the staged queries
+    for (int idx = tid; idx < (2 * p_bytes) / 16; idx += kThreads) reinterpret_cast<uint4*>(Ps)[idx] = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+    mbar_arrive(&hdr->q_ready);
+  }
+  const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
   float m_run[GP], l_thr[GP];
 #pragma unroll
   for (int qi = 0; qi < GP; ++qi) { m_run[qi] = -INFINITY; l_thr[qi] = 0.f; }
+  bool ok = true;
 
-  for (int t = t_lo; t < t_hi && ok; ++t) {
-    const uint32_t par = (t - t_lo) & 1u;
-    // ---- S(t) is complete: the K' core-matrix tile is free; PV(t-1) is complete: P^T and the V' core-matrix tile
-    //      are free.  K'(t+1) and V'(t) have landed: move them and tell the issuer.
-    if (!mbar_wait(&hdr->s_done, par, p.status)) *abort_flag = 1;
-    if (t > t_lo && !mbar_wait(&hdr->o_done, par ^ 1u, p.status)) *abort_flag = 1;
-    if (t + 1 < t_hi) {
-      if (!mbar_wait(&hdr->k_full, par ^ 1u, p.status)) *abort_flag = 1;
-      relayout(Km, Kst, rowb_k, grp_k);
-    }
-    if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
-    relayout(Vm, Vst, rowb_v, grp_v);
-    fence_async_smem();
-    tc_fence_before();
-    mbar_arrive(&hdr->tiles_ready);
+  for (int i = 0; i < nt; ++i) {
+    const int t = t_lo + i, buf = i & 1;
+    const uint32_t par = (i >> 1) & 1u;
+    if (!mbar_wait(&hdr->s_done[buf], par, p.status)) *abort_flag = 1;
     tc_fence_after();
     uint32_t sr[16];
-    tmem_ld16(tmem + lane_base + 32 * par, sr);
+    tmem_ld16(tmem + lane_base + 32 * buf, sr);
     tmem_wait_ld();
     const bool live = t * kTile + tid < n_b;
     // ---- per-query maximum over the tile: one reduction instruction per query and warp, lane q keeps query q's
 #pragma unroll
     for (int qi = 0; qi < GP; ++qi) {
       const float v = warp_max(live ? __uint_as_float(sr[qi]) : -INFINITY);
-      if (lane == qi) hdr->red[par][qi][warp] = v;
+      if (lane == qi) hdr->red[buf][qi][warp] = v;
     }
-    worker_sync();
-    if (*abort_flag) { ok = false; break; }
+    // the P^T buffer of this tile was read by the weighted sum of tile i - 2
+    if (i >= 2 && !mbar_wait(&hdr->o_done[buf], par ^ 1u, p.status)) *abort_flag = 1;
+    if (worker_sync_or(*abort_flag != 0)) { ok = false; break; }   // some role gave up: all workers leave here
     // lazy reference: m_run follows the maximum only when that grew by more than 8 (every thread decides alike)
+    unsigned char* Pb = Ps + buf * p_bytes;
+    float alpha[GP];
     bool rescale = false;
-    float alpha_mine = 1.f;                                  // for the O' row this thread owns (lane = query)
 #pragma unroll
     for (int qi = 0; qi < GP; ++qi) {
-      const float4 r4 = *reinterpret_cast<const float4*>(&hdr->red[par][qi][0]);
+      const float4 r4 = *reinterpret_cast<const float4*>(&hdr->red[buf][qi][0]);
       const float tm = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
-      float alpha = 1.f;
+      alpha[qi] = 1.f;
       if (tm > m_run[qi] + 8.f) {
-        alpha = ex2(m_run[qi] - tm);
+        alpha[qi] = ex2(m_run[qi] - tm);
         m_run[qi] = tm;
-        rescale = rescale || t > t_lo;
+        rescale = rescale || i > 0;
       }
       const float pj = live ? ex2(__uint_as_float(sr[qi]) - m_run[qi]) : 0.f;
-      l_thr[qi] = fmaf(l_thr[qi], alpha, pj);
-      if (tid == qi) alpha_mine = alpha;
-      *reinterpret_cast<__nv_bfloat16*>(Ps + chunk_off(qi, tid >> 3, grp_p) + (tid & 7) * 2) = __float2bfloat16_rn(pj);
+      l_thr[qi] = fmaf(l_thr[qi], alpha[qi], pj);
+      *reinterpret_cast<__nv_bfloat16*>(Pb + chunk_off(qi, tid >> 3, grp_p) + (tid & 7) * 2) = __float2bfloat16_rn(pj);
     }
-    if (rescale && warp == 0) {                              // O' rows (lanes 0..g-1 of warp 0) times their alpha
+    if (rescale) {                                           // uniform over the workers; this thread's lane of O'^T
+      if (!mbar_wait(&hdr->o_done[buf ^ 1], ((i - 1) >> 1) & 1u, p.status)) *abort_flag = 1;   // the sum of tile i - 1 is in
       tc_fence_after();
-      for (int c0 = 0; c0 < rpv16; c0 += 16) {
-        uint32_t o[16];
-        tmem_ld16(tO + c0, o);
-        tmem_wait_ld();
+      uint32_t o[16];
+      tmem_ld16(tO + lane_base, o);
+      tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha_mine);
-        tmem_st16(tO + c0, o);
-      }
+      for (int qi = 0; qi < GP; ++qi) o[qi] = __float_as_uint(__uint_as_float(o[qi]) * alpha[qi]);
+      tmem_st16(tO + lane_base, o);
       tmem_wait_st();
     }
     fence_async_smem();
     tc_fence_before();
-    mbar_arrive(&hdr->p_ready);                              // the issuer sends the weighted sum of this tile off
+    mbar_arrive(&hdr->p_ready[buf]);                         // the issuer sends the weighted sum of this tile off
   }
   if (ok) {
-    if (!mbar_wait(&hdr->o_done, (t_hi - 1 - t_lo) & 1u, p.status)) ok = false;
+    if (!mbar_wait(&hdr->o_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1u, p.status)) ok = false;
   }
   if (!ok) *abort_flag = 1;
   tc_fence_after();
   worker_sync();                                             // every worker is done with the last tile's maxima
 
-  // ---- partials per query: m, l (summed over the threads' rows), o' (row `query` of O')
+  // ---- partials per query: m, l (summed over the threads' rows), o' (column `query` of O'^T)
 #pragma unroll
   for (int qi = 0; qi < GP; ++qi) {
     float v = l_thr[qi];
@@ -317,19 +348,16 @@ __global__ void __launch_bounds__(kGqaThreads, 2) decode_gqa_kernel(const GqaDec
     part[tid * p.part_stride] = mine_m;
     part[tid * p.part_stride + 1] = (hdr->red[0][tid][0] + hdr->red[0][tid][1]) + (hdr->red[0][tid][2] + hdr->red[0][tid][3]);
   }
-  if (warp == 0) {
-    for (int c0 = 0; c0 < rpv16; c0 += 16) {
-      uint32_t o[16];
-      tmem_ld16(tO + c0, o);
-      tmem_wait_ld();
-      if (lane < G)
-        for (int i = 0; i < 16; ++i)
-          if (c0 + i < hd.rp_v) part[lane * p.part_stride + 4 + c0 + i] = __uint_as_float(o[i]);
-    }
+  {
+    uint32_t o[16];
+    tmem_ld16(tO + lane_base, o);
+    tmem_wait_ld();
+    if (tid < hd.rp_v)
+      for (int qi = 0; qi < G; ++qi) part[qi * p.part_stride + 4 + tid] = __uint_as_float(o[qi]);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 256);
+  if (warp == 0) tmem_dealloc(tmem, 128);
 }
 
 // Merges the partials of one query head and lifts o'/l through (U^V)^T of its K/V head.
@@ -362,29 +390,44 @@ __global__ void __launch_bounds__(128) gqa_combine_kernel(const GqaDecodeParams 
 
 }  // namespace
 
-size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
+// Stages of the K'/V' ring: about 120 KB of copies in flight, at least two, as far as shared memory reaches.
+static int gqa_stages(int max_rp_k, int max_rp_v, size_t* stage_bytes) {
   const size_t k16 = (max_rp_k + 15) & ~15;
-  // P^T (16 rows), Q' images, K' and V' tiles as they land and in the core-matrix layout; the P^T operand of the
-  // weighted sum spans 32 KB from its start, which the tiles behind it cover
-  const size_t v16 = (max_rp_v + 15) & ~15;
-  size_t total = 1024 + kMaxGroup * kTile * 2 + 2 * kMaxGroup * k16 * 2 + kTile * static_cast<size_t>(max_rp_k + max_rp_v + k16 + v16) * 2;
-  const size_t need = 1024 + static_cast<size_t>(kTile) * kTile * 2;
-  return total < need ? need : total;
+  (void)max_rp_v;
+  const size_t stage = (((k16 + 63) >> 6) + 2) * static_cast<size_t>(kGqaAtom);
+  const size_t avail = 227 * 1024 - (kGqaHeader + 4096 + 2 * kMaxGroup * kTile * 2);
+  size_t st = (150 * 1024 + stage - 1) / stage;              // the tiles are padded to 64-element atoms: 120 KB of rows
+  if (st < 3) st = 3;
+  if (st > static_cast<size_t>(kGqaMaxStages)) st = kGqaMaxStages;
+  while (st > 1 && st * stage > avail) --st;
+  *stage_bytes = stage;
+  return static_cast<int>(st);
+}
+
+size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v) {
+  size_t stage = 0;
+  const int st = gqa_stages(max_rp_k, max_rp_v, &stage);
+  if (st < 2) return 1 << 30;                                // does not fit: the caller refuses
+  return kGqaHeader + 4096 + 2 * kMaxGroup * kTile * 2 + st * stage;
 }
 
 template <int GP>
-cudaError_t launch_gqa_variant(const GqaDecodeParams& p, size_t smem, cudaStream_t s) {
+cudaError_t launch_gqa_variant(const GqaDecodeParams& p, size_t smem, int stages, cudaStream_t s) {
   static size_t configured[kMaxDevices] = {};
   const cudaError_t ec = ensure_dynamic_smem(decode_gqa_kernel<GP>, smem, configured);
   if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, p.splits);
-  decode_gqa_kernel<GP><<<grid, kGqaThreads, smem, s>>>(p);
+  decode_gqa_kernel<GP><<<grid, kGqaThreads, smem, s>>>(p, stages);
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
-  cudaError_t e = p.group <= 4 ? launch_gqa_variant<4>(p, smem, s)
-                  : p.group <= 8 ? launch_gqa_variant<8>(p, smem, s) : launch_gqa_variant<16>(p, smem, s);
+cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches) {
+  size_t stage_bytes = 0;
+  const int stages = gqa_stages(max_rp_k, max_rp_v, &stage_bytes);
+  if (stages < 2) return cudaErrorInvalidConfiguration;
+  const size_t smem = decode_gqa_smem_bytes(max_rp_k, max_rp_v);
+  cudaError_t e = p.group <= 4 ? launch_gqa_variant<4>(p, smem, stages, s)
+                  : p.group <= 8 ? launch_gqa_variant<8>(p, smem, stages, s) : launch_gqa_variant<16>(p, smem, stages, s);
   ++*launches;
   if (e != cudaSuccess) return e;
   gqa_combine_kernel<<<p.B * p.H * p.group, 128, 0, s>>>(p);

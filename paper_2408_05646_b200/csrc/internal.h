@@ -258,7 +258,7 @@ cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s,
 cudaError_t launch_q_scatter(const QProjectParams& p, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
-cudaError_t launch_decode_gqa(const GqaDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
