@@ -24,7 +24,9 @@ Grouped-query decode is pinned by the library routine's own grouped mode and
 by ordinary decode with the K/V heads repeated.
 The RoPE variant (Section 4.3) is pinned by library attention on keys and
 queries rotated with complex arithmetic, by its relative-position invariance,
-by the zero-angle special case and by loops.
+by the zero-angle special case and by loops; its prompt form (prefill_head_rope)
+by causal library attention on the same rotated tensors and by the generation
+form row by row.
 decode_quant is ordinary decode over the rows returned by kv_quant.quantized_view, which has its own pins.
 paged_gather / paged_scatter (address arithmetic of a paged cache) are pinned by the identity "paged == contiguous"
 for random page tables, by the identity table, and by a hand-written two-page example.
@@ -169,6 +171,30 @@ def decode_head_rope(q: np.ndarray, Kp: np.ndarray, Vp: np.ndarray, U_K: np.ndar
     p = softmax_rows(s[None, :])[0]
     o = p @ np.asarray(Vp, dtype=F64)
     return o if lowrank_out else lift(o, U_V)
+
+
+def prefill_head_rope(Q: np.ndarray, Kp: np.ndarray, Vp: np.ndarray, U_K: np.ndarray, U_V: np.ndarray,
+                      base: float = 10000.0, interleaved: bool = False, len0: int = 0,
+                      lowrank_out: bool = False) -> np.ndarray:
+    """Causal prompt attention of the RoPE variant for one head (Section 4.3 applied to the prefill phase of
+    Section 2): Q [T, d_h] are the T new full-rank queries, Kp [len0+T, r_K], Vp [len0+T, r_V] the
+    low-dimensional rows cached after the call.  Row j of the cache sits at position j, query t at position
+    len0 + t and sees rows 0..len0+t.  Every cached key is lifted through (U^K)^T and rotated by its position,
+    every query is rotated by its own; the value side is Eq. 7 unchanged."""
+    d_h = U_K.shape[0]
+    Q = np.asarray(Q, dtype=F64)
+    T, n = Q.shape[0], Kp.shape[0]
+    assert n == len0 + T
+    K_pos = rope_rotate(lift(Kp, U_K), np.arange(n), base, interleaved)        # [n, d_h]
+    Q_pos = rope_rotate(Q, len0 + np.arange(T), base, interleaved)             # [T, d_h]
+    Vp = np.asarray(Vp, dtype=F64)
+    O = np.zeros((T, Vp.shape[1]), dtype=F64)
+    for t in range(T):
+        n_t = len0 + t + 1
+        s = (K_pos[:n_t] @ Q_pos[t]) / math.sqrt(d_h)
+        p = softmax_rows(s[None, :])[0]
+        O[t] = p @ Vp[:n_t]
+    return O if lowrank_out else lift(O, U_V)
 
 
 # --------------------------------------------------------------------------
@@ -326,11 +352,16 @@ class LayerOracle:
     def prefill(self, q: np.ndarray, k: np.ndarray, v: np.ndarray) -> dict:
         """q, k, v: [B, T, H, d_h].  Returns {(b,h): out[T, d_h]}."""
         q = np.asarray(q, dtype=F64)
-        assert self.rope is None, "the RoPE variant is built for the generation phase only"
         len0 = self.len
         self.append_kv(k, v)
         T = q.shape[1]
         out = {}
+        if self.rope is not None:
+            for (b, h) in self.units:
+                assert not self.alibi[h]
+                out[(b, h)] = prefill_head_rope(q[b, :, h, :], self.Kp[(b, h)], self.Vp[(b, h)], self.U_K[h], self.U_V[h],
+                                                self.rope["base"], self.rope.get("interleaved", False), len0)
+            return out
         for (b, h) in self.units:
             Qp = to_rank_space(q[b, :, h, :], self.U_K[h])
             Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]

@@ -131,5 +131,58 @@ def test_layer_decode_follows_the_per_head_function():
         for h in range(H):
             ref = orc.decode_head_rope(q[b, 0, h], k[b, :, h] @ U_K[h], v[b, :, h] @ U_V[h], U_K[h], U_V[h], 10000.0, True)
             assert np.abs(out[b, 0, h] - ref).max() < 1e-12
-    with pytest.raises(AssertionError):
-        lay.prefill(q, q, q)
+
+
+@pytest.mark.parametrize("interleaved", [False, True])
+@pytest.mark.parametrize("d_h,r_k,r_v,T,len0,base", [(16, 16, 16, 9, 0, 10000.0), (64, 20, 32, 17, 6, 500000.0), (128, 80, 48, 12, 30, 10000.0)])
+def test_rope_prompt_form_equals_causal_library_attention_and_the_generation_form(d_h, r_k, r_v, T, len0, base, interleaved):
+    # The prompt form of Section 4.3: causal library attention on lifted keys and queries rotated through complex
+    # multiplication (another route to the rotation, another implementation of the softmax and of the mask), with
+    # the queries aligned to the END of the key axis (query t sits at position len0 + t); and row t equals the
+    # generation form over the first len0 + t + 1 rows.
+    rng = np.random.default_rng(d_h + T)
+    U_K, U_V = synth.orthonormal_basis(d_h, r_k, 13), synth.orthonormal_basis(d_h, r_v, 14)
+    n = len0 + T
+    Q, K, V = rng.standard_normal((T, d_h)), rng.standard_normal((n, d_h)), rng.standard_normal((n, d_h))
+    Kp, Vp = K @ U_K, V @ U_V
+    got = orc.prefill_head_rope(Q, Kp, Vp, U_K, U_V, base, interleaved, len0)
+    k_rot = rotate_complex(Kp @ U_K.T, np.arange(n), base, interleaved)
+    q_rot = rotate_complex(Q, len0 + np.arange(T), base, interleaved)
+    mask = torch.from_numpy(np.arange(n)[None, :] <= (len0 + np.arange(T))[:, None])
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q_rot)[None, None], torch.from_numpy(k_rot)[None, None],
+        torch.from_numpy(Vp @ U_V.T)[None, None], attn_mask=mask)[0, 0].numpy()
+    assert np.abs(got - ref).max() < 1e-12
+    for t in (0, T // 2, T - 1):
+        n_t = len0 + t + 1
+        row = orc.decode_head_rope(Q[t], Kp[:n_t], Vp[:n_t], U_K, U_V, base, interleaved, 0)
+        assert np.abs(got[t] - row).max() < 1e-12
+    low = orc.prefill_head_rope(Q, Kp, Vp, U_K, U_V, base, interleaved, len0, lowrank_out=True)
+    assert np.abs(low @ U_V.T - got).max() < 1e-12
+    # a mask off by one (query t seeing row len0 + t + 1) or positions that ignore len0 do not pass
+    if len0:
+        wrong = orc.prefill_head_rope(Q, Kp[len0:], Vp[len0:], U_K, U_V, base, interleaved, 0)
+        assert np.abs(wrong - got).max() > 1e-6
+
+
+def test_layer_prefill_with_rope_follows_the_per_head_function_in_chunks():
+    B, H, d_h, T = 2, 3, 16, 11
+    rng = np.random.default_rng(14)
+    rk, rv = [4, 16, 7], [8, 5, 16]
+    U_K = [synth.orthonormal_basis(d_h, r, 70 + h) for h, r in enumerate(rk)]
+    U_V = [synth.orthonormal_basis(d_h, r, 80 + h) for h, r in enumerate(rv)]
+    q, k, v = rng.standard_normal((3, B, T, H, d_h))
+    rope = {"base": 10000.0, "interleaved": False}
+    one = orc.LayerOracle(B, H, d_h, U_K, U_V, rope=rope).prefill_dense(q, k, v)
+    lay = orc.LayerOracle(B, H, d_h, U_K, U_V, rope=rope)
+    two = np.concatenate([lay.prefill_dense(q[:, :4], k[:, :4], v[:, :4]), lay.prefill_dense(q[:, 4:], k[:, 4:], v[:, 4:])], axis=1)
+    assert np.abs(one - two).max() < 1e-12                              # chunked prompt = one prompt
+    for b in range(B):
+        for h in range(H):
+            ref = orc.prefill_head_rope(q[b, :, h], k[b, :, h] @ U_K[h], v[b, :, h] @ U_V[h], U_K[h], U_V[h], 10000.0, False)
+            assert np.abs(one[b, :, h] - ref).max() < 1e-12
+    nxt = rng.standard_normal((3, B, 1, H, d_h))                        # the prompt's cache serves the generation phase
+    lay.append_kv(nxt[1], nxt[2])
+    full = orc.LayerOracle(B, H, d_h, U_K, U_V, rope=rope)
+    last = full.prefill_dense(np.concatenate([q, nxt[0]], axis=1), np.concatenate([k, nxt[1]], axis=1), np.concatenate([v, nxt[2]], axis=1))
+    assert np.abs(lay.decode_dense(nxt[0]) - last[:, -1:]).max() < 1e-12
