@@ -785,8 +785,9 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                              int64_t out_stride_t, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
   if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available for a batch of unequal lengths (eigen_attn_set_lens)");
-  if (h->rope) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available with a rotary embedding");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
+  if (h->rope && (flags & EA_Q_PREPROJECTED))
+    return fail(h, EA_ERR_INVALID_ARG, "prefill with rotary embedding: EA_Q_PREPROJECTED (the query must be full rank)");
   if (flags & ~(EA_OUT_LOWRANK | EA_Q_PREPROJECTED | EA_KV_PREPROJECTED))
     return fail(h, EA_ERR_INVALID_ARG, "prefill: unknown flag 0x%x", flags);
   const bool merged_in = (flags & (EA_Q_PREPROJECTED | EA_KV_PREPROJECTED)) != 0;
@@ -806,6 +807,33 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   if (h->opt_prefill == 2 && !tc_attn)
     return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
   cudaError_t e;
+  if (h->rope) {
+    // Section 4.3 for the prompt: the cache takes the projections of the un-rotated keys, as in the generation
+    // phase; the attention kernel lifts and rotates them and rotates the full-rank queries itself.
+    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
+    if (st != EA_OK) return st;
+    ea::PrefillParams p{};
+    p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache; p.out = d_out;
+    if (flags & EA_OUT_LOWRANK) {
+      p.out_stride_t = L.sum_rp_v;
+      p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
+    } else {
+      p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
+    }
+    p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
+    p.len0 = len0;
+    p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+    p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
+    p.pages = dev_pages(h);
+    p.q_raw = d_q; p.q_stride_b = stride_b; p.q_stride_t = stride_t;
+    p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+    p.rope_interleaved = h->rope_interleaved;
+    if (h->ev_start) cudaEventRecord(h->ev_start, s);
+    e = ea::launch_prefill_rope(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+    if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch (rotary embedding)");
+    return EA_OK;
+  }
   if (merged_in) {
     // Rank-space rows from merged weights (Eq. 8): nothing to multiply.  K', V' rows are copied into the cache, Q'
     // rows into the per-head layout the attention kernels read; a tensor the caller left d_head-wide is projected

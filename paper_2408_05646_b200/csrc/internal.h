@@ -156,6 +156,11 @@ struct PrefillParams {
   int* status;
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head (warp-specialised kernel only)
   PageMap pages;            // paged cache (CUDA-core kernel only)
+  // RoPE variant (prefill_rope.cu): the full-rank, un-rotated queries and the rotation's frequencies
+  const void* q_raw;        // [B][T][H][d_head]
+  int64_t q_stride_b, q_stride_t;
+  const double* inv_freq;   // [d_head/2]: base^(-2i/d_head)
+  int32_t rope_interleaved; // pairs (2i, 2i+1) instead of (i, i + d_head/2)
 };
 
 struct RopeDecodeParams {    // decode for models with rotary position embedding (bf16 layers)
@@ -257,6 +262,7 @@ cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s,
 // Q' rows that are already rank-space (packed [B][T][sum rp_k]) into the per-head layout of the Q' scratch.
 cudaError_t launch_q_scatter(const QProjectParams& p, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_prefill_rope(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);

@@ -94,6 +94,42 @@ def test_rope_decode_steps_lowrank_output_and_switching_off(B):
     lay.poll_status()
 
 
+@pytest.mark.parametrize("H,d,rk,rv,T,base,interleaved", [
+    (2, 128, [80, 48], [64, 80], 300, 10000.0, False),
+    (3, 64, [24, 64, 40], [56, 8, 64], 150, 500000.0, True),
+    (1, 128, [128], [128], 77, 10000.0, False),
+])
+def test_rope_prefill_matches_oracle_and_feeds_decode(B, H, d, rk, rv, T, base, interleaved):
+    """A layer with rotary embedding runs prompt -> generation through the library: the prompt in two chunks
+    (positions continue from the cached length), then decode steps over the cache the prompt left."""
+    B_, steps = 2, 2
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + steps, BF16, seed_cfg=159, T_q=T + steps)
+    lay = B.EigenAttnLayer(B_, H, d, T + steps, BF16, U_k, U_v, max_prefill_tokens=T)
+    lay.set_rope(base, interleaved)
+    ref = rope_oracle(B_, H, d, U_k, U_v, base, interleaved)
+    cut = T // 2 + 5
+    a = lay.prefill(q[:, :cut].contiguous(), k[:, :cut].contiguous(), v[:, :cut].contiguous())
+    c = lay.prefill(q[:, cut:T].contiguous(), k[:, cut:T].contiguous(), v[:, cut:T].contiguous())
+    lay.poll_status()
+    expect = ref.prefill_dense(to_np(q[:, :T]), to_np(k[:, :T]), to_np(v[:, :T]))
+    assert_close(torch.cat([a, c], dim=1), expect, BF16, "rope prefill")
+    low = lay_low = None
+    for s in range(steps):
+        t = T + s
+        o = lay.decode_step(q[:, t:t + 1], k[:, t:t + 1], v[:, t:t + 1])
+        ref.append_kv(to_np(k[:, t:t + 1]), to_np(v[:, t:t + 1]))
+        assert_close(o, ref.decode_dense(to_np(q[:, t:t + 1])), BF16, f"decode step {s} after a rope prefill")
+    # rank-space output of the prompt
+    lay2 = B.EigenAttnLayer(B_, H, d, T, BF16, U_k, U_v, max_prefill_tokens=T)
+    lay2.set_rope(base, interleaved)
+    low = lay2.prefill(q[:, :T].contiguous(), k[:, :T].contiguous(), v[:, :T].contiguous(), out_lowrank=True)
+    for b in range(B_):
+        for h in range(H):
+            back = to_np(low[b, :, lay2.offs_v[h]:lay2.offs_v[h] + rv[h]]) @ U_v[h].astype(np.float64).T
+            assert_close(torch.from_numpy(back), expect[b, :, h], BF16, "rope prefill, rank-space output")
+    lay.poll_status()
+
+
 def test_rope_rejections(B):
     U_k, U_v, q, k, v = make_case(1, 2, 64, [16, 16], [16, 16], 8, FP32, seed_cfg=155)
     lay32 = B.EigenAttnLayer(1, 2, 64, 8, FP32, U_k, U_v)
@@ -104,8 +140,6 @@ def test_rope_rejections(B):
     with pytest.raises(B.EigenAttnError):
         lay.set_rope(0.5)
     lay.set_rope(10000.0)
-    with pytest.raises(B.EigenAttnError):
-        lay.prefill(q.expand(1, 8, 2, 64).contiguous(), k, v)
     lay.append_kv(k, v)
     with pytest.raises(B.EigenAttnError):
         lay.decode_static(q)
