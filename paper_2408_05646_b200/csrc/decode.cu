@@ -26,9 +26,10 @@ namespace {
 constexpr int kMaxStages = 12;
 constexpr uint64_t kWaitBoundNs = 2000000000ull;   // every device-side wait gives up after 2 s
 // Registers per thread after the reallocation.  The CTA is launched with 384 threads x 168 registers (three
-// warps per scheduler share its 16 384); the producer's warpgroup keeps 56 each, the two consumer warpgroups
-// take the rest: 128 x 56 + 256 x 224 = 384 x 168.
-constexpr int kRegsProducerGroup = 56, kRegsConsumers = 224;
+// warps per scheduler share its 16 384); the warpgroup of the producer and the helper warps keeps 96 each, the
+// two consumer warpgroups take 200: 128 x 96 + 256 x 200 <= 384 x 168.
+constexpr int kRegsProducerGroup = 96, kRegsConsumers = 200;
+constexpr int kHelperThreads = 96;                 // warps 9..11: the projections of the next piece
 static_assert(128 * kRegsProducerGroup + 256 * kRegsConsumers <= kDecodeThreads * 168, "register split exceeds the launch");
 
 struct __align__(128) DecodeSmemFixed {
@@ -38,11 +39,13 @@ struct __align__(128) DecodeSmemFixed {
   int abort_flag;
   int is_last;
   float piece_m, piece_l;
-  float qraw[128], kraw[128], vraw[128];   // the unit's q (and new k, v) as fp32
+  unsigned long long proj_full[2];         // the helper warps have written q' (and the new row) of a piece
+  unsigned long long proj_empty[2];        // the consumers are done with them
+  float raw[2][3][128];                    // a unit's q, new k, new v as fp32: [0] for the consumers, [1] for the helpers
   float proj_part[256];                    // partial sums of the projections
-  float qp[128];                           // q' * log2(e)/sqrt(d_head)
-  __align__(16) unsigned char new_k[512];  // the new token's k', v' in cache format (one row each)
-  __align__(16) unsigned char new_v[512];
+  float qp[2][128];                        // q' * log2(e)/sqrt(d_head), for this piece and the next
+  __align__(16) unsigned char new_k[2][512];  // the new token's k', v' in cache format (one row each)
+  __align__(16) unsigned char new_v[2][512];
   float wmax[kDecodeConsumerWarps];
   float wsum[kDecodeConsumerWarps];
   float o_acc[128];                        // the piece's (later the unit's) o'
@@ -101,6 +104,7 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* statu
 __device__ __forceinline__ void consumer_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumerWarps * 32) : "memory");
 }
+__device__ __forceinline__ void helper_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kHelperThreads) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -260,7 +264,7 @@ __device__ __forceinline__ Piece locate(const DecodeParams& p, const int* pre, l
 template <typename T, int NCH>
 __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFixed* fx,
                                             unsigned char* ring, const HeadInfo& hd, int i0, int i1,
-                                            Ring& ring_state, int warp, int lane, bool with_new_row, int n_b) {
+                                            Ring& ring_state, int warp, int lane, bool with_new_row, int n_b, int buf) {
   constexpr int EPC = Elem<T>::kPerChunk;
   const int pair = lane >> 1, half = lane & 1;
   const int rowb_k = hd.rp_k * static_cast<int>(sizeof(T));
@@ -287,7 +291,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
     off_v[j] = cv < nch_v ? (cv << 4) : 0;
 #pragma unroll
     for (int e = 0; e < EPC; ++e) {
-      q[j][e] = vk ? fx->qp[ck * EPC + e] : 0.f;
+      q[j][e] = vk ? fx->qp[buf][ck * EPC + e] : 0.f;
       o[j][e] = 0.f;
     }
   }
@@ -370,7 +374,7 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
 
   // the new token's row (already projected, in shared memory) is attended by one lane pair
   if (with_new_row && warp == 0 && !__any_sync(0xffffffffu, *abort_flag != 0))
-    process_row(fx->new_k, fx->new_v, pair == 0, pos_q);
+    process_row(fx->new_k[buf], fx->new_v[buf], pair == 0, pos_q);
 
   // ---- merge the 128 lane pairs of the CTA into one partial
   float wm = m;
@@ -425,59 +429,61 @@ __device__ __forceinline__ void run_segment(const DecodeParams& p, DecodeSmemFix
   consumer_sync();
 }
 
-// Projections at the head of a piece (all consumer threads): q' = q U^K * log2(e)/sqrt(d_head) into
-// fx->qp, and, when the piece ends its unit and a new token is supplied, k' = k U^K and v' = v U^V,
-// rounded to the cache dtype, into fx->new_k / fx->new_v and into row n_b (the sequence's length) of the cache.
-template <typename T>
-__device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmemFixed* fx,
+// Projections of a piece: q' = q U^K * log2(e)/sqrt(d_head) into fx->qp[buf], and, when the piece ends its unit and
+// a new token is supplied, k' = k U^K and v' = v U^V, rounded to the cache dtype, into fx->new_k / fx->new_v [buf]
+// and into row n_b (the sequence's length) of the cache.  A CTA's first piece is projected by its 256 consumer
+// threads (NT = 256), every later one by the 96 threads of the helper warps (NT = 96) while the consumers stream
+// the piece before it.  t = 0 .. NT - 1.
+template <typename T, int NT>
+__device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmemFixed* fx, int buf,
                                                const HeadInfo& hd, int h, int b, int t, bool with_new_row,
                                                int n_b) {
-  constexpr int kThreads = kDecodeConsumerWarps * 32;
+  constexpr bool kHelpers = NT == kHelperThreads;
+  float* qraw = fx->raw[kHelpers ? 1 : 0][0];
+  float* kraw = fx->raw[kHelpers ? 1 : 0][1];
+  float* vraw = fx->raw[kHelpers ? 1 : 0][2];
+  auto group_sync = [] { if (kHelpers) helper_sync(); else consumer_sync(); };
   const T* q = static_cast<const T*>(p.q);
   const int d_head = p.d_head;
   const bool q_lowrank = (p.flags & 0x1u) != 0;   // rank-space query supplied by the caller (merged W^Q')
+  float* qp = fx->qp[buf];
+  T* knew = reinterpret_cast<T*>(fx->new_k[buf]);
+  T* vnew = reinterpret_cast<T*>(fx->new_v[buf]);
   if (q_lowrank) {
-    if (t < hd.rp_k) fx->qp[t] = Elem<T>::to_float(q[b * p.q_stride_b + hd.lr_k_off + t]) * p.q_scale;
-  } else if (t < d_head) {
-    fx->qraw[t] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + t]);
+    for (int c = t; c < hd.rp_k; c += NT) qp[c] = Elem<T>::to_float(q[b * p.q_stride_b + hd.lr_k_off + c]) * p.q_scale;
+  } else {
+    for (int d = t; d < d_head; d += NT) qraw[d] = Elem<T>::to_float(q[b * p.q_stride_b + static_cast<int64_t>(h) * d_head + d]);
   }
   const bool kv_lowrank = (p.flags & 0x4u) != 0;  // rank-space k', v' supplied by the caller (merged W^K', W^V')
+  const int64_t crow = physical_row(p.pages, b, p.n_max, n_b);
   if (with_new_row && kv_lowrank) {
     // nothing to project: the packed rows go into the cache (padding columns zero) and into shared memory
-    const int64_t crow = physical_row(p.pages, b, p.n_max, n_b);
-    if (t < hd.rp_k) {
-      const T val = t < hd.r_k ? static_cast<const T*>(p.k_new)[b * p.kv_stride_b + hd.lr_k_off + t] : Elem<T>::from_float(0.f);
-      reinterpret_cast<T*>(fx->new_k)[t] = val;
-      reinterpret_cast<T*>(p.cache + hd.k_off)[crow * hd.rp_k + t] = val;
+    for (int c = t; c < hd.rp_k; c += NT) {
+      const T val = c < hd.r_k ? static_cast<const T*>(p.k_new)[b * p.kv_stride_b + hd.lr_k_off + c] : Elem<T>::from_float(0.f);
+      knew[c] = val;
+      reinterpret_cast<T*>(p.cache + hd.k_off)[crow * hd.rp_k + c] = val;
     }
-    if (t < hd.rp_v) {
-      const T val = t < hd.r_v ? static_cast<const T*>(p.v_new)[b * p.v_stride_b + hd.lr_v_off + t] : Elem<T>::from_float(0.f);
-      reinterpret_cast<T*>(fx->new_v)[t] = val;
-      reinterpret_cast<T*>(p.cache + hd.v_off)[crow * hd.rp_v + t] = val;
+    for (int c = t; c < hd.rp_v; c += NT) {
+      const T val = c < hd.r_v ? static_cast<const T*>(p.v_new)[b * p.v_stride_b + hd.lr_v_off + c] : Elem<T>::from_float(0.f);
+      vnew[c] = val;
+      reinterpret_cast<T*>(p.cache + hd.v_off)[crow * hd.rp_v + c] = val;
     }
     with_new_row = false;                         // for the projection below
   }
-  if (with_new_row && t < d_head) {
-    fx->kraw[t] = Elem<T>::to_float(static_cast<const T*>(p.k_new)[b * p.kv_stride_b + static_cast<int64_t>(h) * d_head + t]);
-    fx->vraw[t] = Elem<T>::to_float(static_cast<const T*>(p.v_new)[b * p.v_stride_b + static_cast<int64_t>(h) * d_head + t]);
-  }
-  consumer_sync();
+  if (with_new_row)
+    for (int d = t; d < d_head; d += NT) {
+      kraw[d] = Elem<T>::to_float(static_cast<const T*>(p.k_new)[b * p.kv_stride_b + static_cast<int64_t>(h) * d_head + d]);
+      vraw[d] = Elem<T>::to_float(static_cast<const T*>(p.v_new)[b * p.v_stride_b + static_cast<int64_t>(h) * d_head + d]);
+    }
+  group_sync();
   // outputs: [0, nq) = q' columns, [nq, nq + rp_k) = k' columns, then rp_v v' columns
   const int nq = q_lowrank ? 0 : hd.rp_k;
   const int total = nq + (with_new_row ? hd.rp_k + hd.rp_v : 0);
-  if (total == 0) return;
-  int groups = kThreads / total;                  // split the d_head sum when few outputs are needed
-  if (groups > 4) groups = 4;
   // k' and v' are summed over d_head in one fixed order (the append kernel's), so that a row stored by
   // this kernel is bit-identical to the same row stored by eigen_attn_append_kv
-  if (groups < 1 || with_new_row) groups = 1;
-  const int per = (d_head + groups - 1) / groups;
-  T* knew = reinterpret_cast<T*>(fx->new_k);
-  T* vnew = reinterpret_cast<T*>(fx->new_v);
-  const int64_t crow = physical_row(p.pages, b, p.n_max, n_b);
   auto finish = [&](int o, float acc) {
     if (o < nq) {
-      fx->qp[o] = acc * p.q_scale;
+      qp[o] = acc * p.q_scale;
     } else if (o < nq + hd.rp_k) {
       const int c = o - nq;
       const T val = Elem<T>::from_float(acc);
@@ -490,31 +496,19 @@ __device__ __forceinline__ void project_inputs(const DecodeParams& p, DecodeSmem
       reinterpret_cast<T*>(p.cache + hd.v_off)[crow * hd.rp_v + c] = val;
     }
   };
-  auto dot = [&](int o, int d0, int d1) {
+  for (int o = t; o < total; o += NT) {
     const float* x;
     const float* U;
     int rp;
-    if (o < nq) { x = fx->qraw; U = p.basis + hd.uk_off + o; rp = hd.rp_k; }
-    else if (o < nq + hd.rp_k) { x = fx->kraw; U = p.basis + hd.uk_off + (o - nq); rp = hd.rp_k; }
-    else { x = fx->vraw; U = p.basis + hd.uv_off + (o - nq - hd.rp_k); rp = hd.rp_v; }
+    if (o < nq) { x = qraw; U = p.basis + hd.uk_off + o; rp = hd.rp_k; }
+    else if (o < nq + hd.rp_k) { x = kraw; U = p.basis + hd.uk_off + (o - nq); rp = hd.rp_k; }
+    else { x = vraw; U = p.basis + hd.uv_off + (o - nq - hd.rp_k); rp = hd.rp_v; }
     float acc = 0.f;
 #pragma unroll 32
-    for (int d = d0; d < d1; ++d) acc = fmaf(x[d], __ldg(U + d * rp), acc);
-    return acc;
-  };
-  if (groups == 1) {
-    for (int o = t; o < total; o += kThreads) finish(o, dot(o, 0, d_head));
-  } else {
-    const int g = t / total, o = t - g * total;
-    if (g < groups) fx->proj_part[g * total + o] = dot(o, g * per, min(d_head, (g + 1) * per));
-    consumer_sync();
-    if (t < total) {
-      float acc = 0.f;
-      for (int gg = 0; gg < groups; ++gg) acc += fx->proj_part[gg * total + t];
-      finish(t, acc);
-    }
+    for (int d = 0; d < d_head; ++d) acc = fmaf(x[d], __ldg(U + d * rp), acc);
+    finish(o, acc);
   }
-  consumer_sync();
+  group_sync();                                   // the raw vectors are reused by the next piece
 }
 
 // CTA that owns the tile with start weight x: floor(x * grid / w_total).
@@ -617,6 +611,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       mbar_init(&fx->full[s], 1);
       mbar_init(&fx->empty[s], kDecodeConsumerWarps);
     }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&fx->proj_full[i], kHelperThreads);
+      mbar_init(&fx->proj_empty[i], kDecodeConsumerWarps * 32);
+    }
     fx->abort_flag = 0;
     fx->range[0] = first_tile_of_cta(p, grid, cta);
     fx->range[1] = first_tile_of_cta(p, grid, cta + 1);
@@ -709,12 +707,32 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       // every slot in use (its phase parity is the opposite of the slot's next one).
       for (int s2 = 0; s2 < kMaxStages; ++s2)
         if (rg.filled & (1u << s2)) mbar_wait(&fx->full[s2], ((rg.full_bits >> s2) & 1u) ^ 1u, p.status);
+    } else if (warp > kDecodeConsumerWarps) {
+      // -------------------------------------------------------- helper warps: the projections of every piece
+      // but a CTA's first, one piece ahead of the consumers (two buffers).  They never leave their loop early: a wait that gave up
+      // sets the abort flag and the piece's buffers hold garbage, which the consumers then ignore.
+      const int ht = tid - (kDecodeConsumerWarps + 1) * 32;
+      long long F = f_lo;
+      for (int k = 0; F < f_hi; ++k) {
+        const Piece pc = locate(p, fx->pre, F);
+        const int i1 = static_cast<int>(min(static_cast<long long>(pc.nt_u), pc.i0 + (f_hi - F)));
+        if (k >= 1) {                     // the first piece is the consumers' own
+          const HeadInfo hd = p.heads[pc.h];
+          const int bufk = k & 1;
+          if (k >= 2 && !mbar_wait(&fx->proj_empty[bufk], ((k >> 1) - 1) & 1u, p.status, abort_flag)) *abort_flag = 1;
+          project_inputs<T, kHelperThreads>(p, fx, bufk, hd, pc.h, pc.b, ht, p.k_new != nullptr && i1 == pc.nt_u,
+                                            seq_rows(p, pc.b));
+          mbar_arrive(&fx->proj_full[bufk]);
+        }
+        F += i1 - pc.i0;
+      }
     }
   } else {
     // ------------------------------------------------------------ consumers
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumers));
     Ring rg;
     long long F = f_lo;
+    int piece_no = 0;
     while (F < f_hi) {
       const Piece pc = locate(p, fx->pre, F);
       const int i0 = pc.i0, h = pc.h, b = pc.b;
@@ -733,22 +751,28 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_splitkv_kernel(const
       const bool whole = i0 == 0 && i1 == pc.nt_u;
       const bool with_new_row = p.k_new != nullptr && i1 == pc.nt_u;
       const int n_b = seq_rows(p, b);
-      project_inputs<T>(p, fx, hd, h, b, tid, with_new_row, n_b);
+      const int bufk = piece_no & 1;
+      if (piece_no == 0)
+        project_inputs<T, kDecodeConsumerWarps * 32>(p, fx, 0, hd, h, b, tid, with_new_row, n_b);
+      else if (!mbar_wait(&fx->proj_full[bufk], ((piece_no - 1) >> 1) & 1u, p.status, abort_flag))
+        *abort_flag = 1;
       const int mx = max(hd.rp_k, hd.rp_v);
       const int cls = (mx + 15) >> 4;               // a lane pair covers 16 columns per step
       constexpr int MUL = 8 / Elem<T>::kPerChunk;   // 16-byte chunks per 8 columns: 1 (bf16) or 2 (fp32)
       switch (cls) {
-        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
-        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b); break;
+        case 1: run_segment<T, 1 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 2: run_segment<T, 2 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 3: run_segment<T, 3 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 4: run_segment<T, 4 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 5: run_segment<T, 5 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 6: run_segment<T, 6 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        case 7: run_segment<T, 7 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
+        default: run_segment<T, 8 * MUL>(p, fx, ring, hd, i0, i1, rg, warp, lane, with_new_row, n_b, bufk); break;
       }
+      mbar_arrive(&fx->proj_empty[bufk]);           // q' is in registers, the new row has been attended
       finish_piece<T>(p, fx, hd, pc, cta, grid, whole, tid);
       F += i1 - i0;
+      ++piece_no;
     }
   }
   __syncthreads();
