@@ -116,7 +116,7 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
   L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
-  L->off_rope = off;     off = align_up(off + 64 * sizeof(double));   // inverse frequencies of the rotary embedding
+  L->off_rope = off;     off = align_up(off + ea::kRopeConstBytes);   // constants of the rotary embedding
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->off_deficit = off;  off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // unequal lengths
   L->off_qlens = off;    off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // ... of the quantised copy
@@ -473,14 +473,16 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   p.partials = reinterpret_cast<float*>(h->ws + L.off_partials);
   p.status = dev_status(h);
   p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+  p.tile_step = reinterpret_cast<const float2*>(h->ws + L.off_rope + ea::kRopeStepOffset);
+  p.el_table = reinterpret_cast<const float4*>(h->ws + L.off_rope + ea::kRopeTableOffset);
   p.tmaps = h->ws + L.off_tmaps;
   p.deficit = dev_deficit(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;
-  // CTAs per unit.  The CTAs run in waves of (SMs x CTAs per SM) and each one pays a start-up (trigonometric
-  // constants, the U^K image) worth about ten tiles: take the split count with the least waves x (tiles + start-up),
-  // within the partials the workspace holds.
+  // CTAs per unit.  The CTAs run in waves of (SMs x CTAs per SM) and each one pays a start-up (the U^K image, the
+  // rotation constants, the first tiles' way from memory) worth a few tiles: take the split count with the least
+  // waves x (tiles + start-up), within the partials the workspace holds.
   const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
   const int64_t units = static_cast<int64_t>(B) * H;
   int64_t cap = (units + kMaxDecodeCtas) * kPartialSlack / units;
@@ -495,7 +497,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
     const int64_t wave = static_cast<int64_t>(h->sm_count) * ctas_per_sm;
     int64_t best = INT64_MAX;
     for (int64_t s2 = 1; s2 <= cap && s2 <= 256; ++s2) {
-      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 10);
+      const int64_t cost = ((units * s2 + wave - 1) / wave) * ((p.nt + s2 - 1) / s2 + 6);
       if (cost < best) { best = cost; splits = s2; }
     }
   }
@@ -1174,10 +1176,27 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
   if (h->alibi) return fail(h, EA_ERR_INVALID_ARG, "set_rope: the layer has an ALiBi bias");
   if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "set_rope: not available with a page table");
   const int dh = h->desc.d_head;
-  double freq[64] = {};
+  // the constants the kernels read: the inverse frequencies phi_i, e^{-i 128 phi_i} (one tile of cached rows back)
+  // and e^{i l phi_i} for the 128 row offsets of a tile, worked out here in double precision
+  std::vector<unsigned char> host(ea::kRopeConstBytes, 0);
+  double* freq = reinterpret_cast<double*>(host.data());
+  float* step = reinterpret_cast<float*>(host.data() + ea::kRopeStepOffset);
+  float* table = reinterpret_cast<float*>(host.data() + ea::kRopeTableOffset);
   for (int i = 0; i < dh / 2; ++i) freq[i] = pow(base, -2.0 * i / dh);
+  for (int i = 0; i < 64; ++i) {
+    step[2 * i] = static_cast<float>(cos(-128.0 * freq[i]));
+    step[2 * i + 1] = static_cast<float>(sin(-128.0 * freq[i]));
+  }
+  for (int k = 0; k < 32; ++k)
+    for (int l = 0; l < 128; ++l) {
+      float* e = table + (static_cast<size_t>(k) * 128 + l) * 4;
+      e[0] = static_cast<float>(cos(l * freq[2 * k]));
+      e[1] = static_cast<float>(cos(l * freq[2 * k + 1]));
+      e[2] = static_cast<float>(sin(l * freq[2 * k]));
+      e[3] = static_cast<float>(sin(l * freq[2 * k + 1]));
+    }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_rope, freq, sizeof(freq), cudaMemcpyHostToDevice, s);
+  cudaError_t e = cudaMemcpyAsync(h->ws + h->L.off_rope, host.data(), host.size(), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return cuda_fail(h, e, "set_rope");
   h->rope = true;

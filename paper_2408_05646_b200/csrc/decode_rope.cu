@@ -5,7 +5,7 @@
 // rank-r path unchanged.  Per cached row that is a d_h x r product instead of an r-long dot product, so the
 // lift runs on the tensor cores: for a tile of 128 cached rows, X = K'_tile (U^K)^T is one tcgen05 product
 // (M = 128 rows, N = d_h, K = r; U^K rounded to bf16, the precision the cached rows already have) with X in
-// TMEM, one row per thread.
+// TMEM, one row per lane.
 //
 // Rotation without a table per position: with complex pairs Q = q_a + i q_b, X = x_a + i x_b and the
 // pair's frequency phi, the rotated dot product of the pair is Re(Q e^{i p phi} conj(X e^{i j phi})) =
@@ -14,15 +14,20 @@
 // (64 threads; the first tile's angle is reduced in fp64, every further tile turns the query by the constant
 // e^{-i 128 phi}, one complex multiplication, renormalised), the second is a per-thread constant in registers.
 //
-// One CTA (128 threads, two per SM) walks a contiguous range of the tiles of one (sequence, head) unit.  A tile
-// of K' or V' rows is contiguous in the cache, so each arrives as one bulk copy (cp.async.bulk).  K' lands
-// row-major in a staging buffer, the threads move it into the core-matrix layout the tensor core reads (16-byte
-// chunks, 20 KB a tile), and the staging buffer takes the next tile at once, a whole tile ahead of its use: with
-// a single tile in flight per CTA it is the distance between request and use that sets the pace, not the kind of
-// copy (tiled TMA boxes stream at the same rate when four tiles are in flight).  V' is read row-major where it
-// lands.  Scores -> online softmax in base 2 ->
-// o' += p V' on the CUDA cores (thread (g, c) owns a column pair over a row group).  A unit split over several CTAs leaves partials (m, l, o') that
-// rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
+// One CTA (nine warps, two CTAs per SM) walks a contiguous range of the tiles of one (sequence, head) unit.
+//   * Warp 8 (its first lane) requests and issues: a K' tile arrives by TMA straight in the swizzled layout the
+//     lift's A operand names (two buffers, no thread moves it), a V' tile as one bulk copy (contiguous in the
+//     cache, read row-major where it lands), and the lift of tile i + 1 goes out while the other warps work on
+//     X(i) (two accumulators in TMEM).  mbarriers carry every hand-over: rows landed, X complete (which also
+//     frees the K' buffer), X read, V' landed, V' read.
+//   * Warps 0-7 do the arithmetic.  A TMEM lane (= cached row) is shared by two threads, warp w and warp w + 4,
+//     each taking every other chunk of eight pairs, so a thread keeps only half of its row's rotation constants
+//     in registers.  The two partial scores meet in shared memory; every thread adds up its lane's four rows, so
+//     the tile maximum is one warp reduction with no further barrier.  Online softmax in base 2, then
+//     o' += p V' on the CUDA cores (thread (g, c) owns a column pair over a row group).
+// The rotation constants (e^{i l phi} per row offset, e^{-i 128 phi} per tile) are built on the host in double
+// precision when the embedding is set; a CTA only loads them.  A unit split over several CTAs leaves partials
+// (m, l, o') that rope_combine_kernel merges and lifts through (U^V)^T.  Every wait is bounded.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -34,17 +39,31 @@ namespace {
 using namespace tc;
 
 
+constexpr int kRopeAtom = kTile * 128;        // one swizzled atom column of a K' tile: 128 rows x 64 elements
+constexpr int kRopeThreads = 256;             // eight warps: two threads per cached row of the tile
+constexpr int kRopeRequester = 192;           // first lane of warp 6: requests the K' and V' tiles
+constexpr int kRopeLifter = 224;              // first lane of warp 7: issues the lifts
+constexpr int kRopeSumThreads = 192;          // warps 0-5 do the weighted sum while those two lanes issue
+constexpr int kRopeHeaderBytes = 4096;        // barriers, the tile's query, weights and partial scores
+constexpr float kRopeLazy = 8.f;              // the softmax reference moves when a score passes it by this much (base 2)
+constexpr double kTwoPi = 6.283185307179586476925286766559;
+
+// Barrier of the CTA with a predicate ORed over its threads: every thread gets the same answer, so what follows it
+// (leaving the tile loop when a wait gave up) is decided alike by all and the next barrier is met by all.
+__device__ __forceinline__ bool cta_sync_or(bool pred) { return __syncthreads_or(pred ? 1 : 0) != 0; }
+
 struct __align__(16) RopeSmemHeader {
-  unsigned long long mma_done, k_full, v_full;
+  unsigned long long x_full[2], k_full[2], v_full, v_free;
   uint32_t tmem_base;
-  int abort_flag;
-  float red[8];          // cross-warp reductions
-  float tile_max;
-  float pad_[3];
+  int pad_;
+  float red[4];          // the row sums of warps 0-3
 };
 
+// parts of the shared memory image are multiples of 1 KB (the swizzled tiles need that alignment)
+__host__ __device__ constexpr int rope_kb(int bytes) { return (bytes + 1023) & ~1023; }
+
 template <bool INTERLEAVED>
-__global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
+__global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -53,22 +72,21 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15;
   const int nch_k = rpk16 >> 3, grp_k = nch_k << 7;
-  const int rowb_k = hd.rp_k * 2, rowb_v = hd.rp_v * 2;      // bytes per cached row
-  const int kst_bytes = kTile * rowb_k, km_bytes = kTile * rpk16 * 2, v_bytes = kTile * rowb_v;
+  const int rowb_v = hd.rp_v * 2;                            // bytes per cached value row
+  const int ak = (rpk16 + 63) >> 6;                          // atom columns (64 elements) of a K' tile
+  const int kt_bytes = ak * kRopeAtom, v_bytes = kTile * rowb_v;
   const int u_bytes = p.d_head * rpk16 * 2;                  // bf16 image of U^K (the high part of the stored pair)
   const int half = p.d_head >> 1;
 
-  float* q_tile = reinterpret_cast<float*>(smem + 256);      // the query pairs for this tile: re[64], then im[64]
-  float* p_row = q_tile + 128;                               // [128] softmax weights of the tile
-  unsigned char* tiles = smem + 2048;
-  unsigned char* Kst = tiles;                                // K' tile as it lands: row-major
-  unsigned char* Km = Kst + kst_bytes;                       // K' tile in the canonical core-matrix layout
-  unsigned char* Vs = Km + km_bytes;                         // V' tile, row-major
-  unsigned char* Us = Vs + v_bytes;                          // U^K image, canonical layout
+  float* q_tile = reinterpret_cast<float*>(smem + 256);      // [2][192] the query pairs of a tile: re[64], im[64], -re[64]
+  float* p_row = q_tile + 384;                               // [128] softmax weights of the tile
+  float* sc = p_row + 128;                                   // [2][128] the two partial scores of every row
+  unsigned char* Us = smem + kRopeHeaderBytes;               // U^K image, canonical layout
+  unsigned char* Kt = Us + rope_kb(u_bytes);                 // K' tiles [2], as TMA writes them: 128-byte swizzle
+  unsigned char* Vs = Kt + 2 * kt_bytes;                     // V' tile, row-major
 
-  // tiles [t_lo, t_hi) of the unit
   // rows and tiles of this sequence (a batch of unequal lengths gives every sequence its own count and its own
-  // query position; the splits of a unit divide the sequence's own tiles)
+  // query position; the splits of a unit divide the sequence's own tiles): this CTA takes tiles [t_lo, t_hi)
   const int n_b = p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;
   const int nt_b = (n_b + kTile - 1) / kTile;
   const int per = (nt_b + p.splits - 1) / p.splits;
@@ -79,67 +97,60 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
     if (tid < hd.rp_v) part[4 + tid] = 0.f;
     return;
   }
+  const int nt_cta = t_hi - t_lo;
 
-  if (warp == 0) tmem_alloc(&hdr->tmem_base, 256);           // two accumulators: X(t) is read while X(t+1) is computed
+  if (warp == 0) tmem_alloc(&hdr->tmem_base, 256);           // two accumulators: X(i) is read while X(i+1), X(i+2) are computed
   if (tid == 0) {
-    mbar_init(&hdr->mma_done, 1);
-    mbar_init(&hdr->k_full, 1);
+    mbar_init(&hdr->x_full[0], 1);
+    mbar_init(&hdr->x_full[1], 1);
+    mbar_init(&hdr->k_full[0], 1);
+    mbar_init(&hdr->k_full[1], 1);
     mbar_init(&hdr->v_full, 1);
-    hdr->abort_flag = 0;
+    mbar_init(&hdr->v_free, kRopeSumThreads / 32);           // one arrival per warp
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-
   // U^K image (read through L2 by every CTA of the head)
   {
     const uint4* Ug = reinterpret_cast<const uint4*>(p.basis + hd.ukl16_off);
-    for (int idx = tid; idx < u_bytes / 16; idx += kThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
+    for (int idx = tid; idx < u_bytes / 16; idx += kRopeThreads) cp_async16(Us + idx * 16, Ug + idx, 16u);
     cp_async_commit();
   }
   // rows that no copy has filled must hold finite numbers: they meet zero weights (a ragged last tile)
-  for (int idx = tid; idx < (kst_bytes + km_bytes + v_bytes) / 16; idx += kThreads)
-    reinterpret_cast<uint4*>(Kst)[idx] = make_uint4(0u, 0u, 0u, 0u);
-  const uint64_t policy = policy_evict_first();
-  const char* k_src = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * rowb_k;
-  const char* v_src = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * rowb_v;
-  auto fetch_k = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_k;
-    mbar_arrive_expect_tx(&hdr->k_full, bytes);
-    bulk_load(Kst, k_src + static_cast<int64_t>(t) * kTile * rowb_k, bytes, &hdr->k_full, policy);
-  };
-  auto fetch_v = [&](int t) {
-    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
-    mbar_arrive_expect_tx(&hdr->v_full, bytes);
-    bulk_load(Vs, v_src + static_cast<int64_t>(t) * kTile * rowb_v, bytes, &hdr->v_full, policy);
-  };
-  // staging -> core-matrix layout: chunk (row, c) of 16 bytes goes to (row / 8) * grp_k + c * 128 + (row % 8) * 16
-  auto relayout_k = [&]() { relayout_tile(Km, Kst, rowb_k, grp_k, warp, lane); };
+  for (int idx = tid; idx < v_bytes / 16; idx += kRopeThreads) reinterpret_cast<uint4*>(Vs)[idx] = make_uint4(0u, 0u, 0u, 0u);
 
-  // this thread's constants: e^{i l phi_i} for its row l = tid and every pair i
-  unsigned long long el_c[32], el_s[32];                     // pairs (2k, 2k+1) packed: (cos, cos), (sin, sin)
+  // Thread (row, hf): row = 32 (warp & 3) + lane is its TMEM lane, hf = warp >> 2 picks the chunks of eight pairs
+  // 2m + hf (m = 0..3).  Its constants e^{i row phi} for those pairs come from the table the layer keeps:
+  // entry [k][row] = cos, cos, sin, sin of pairs 2k, 2k + 1.
+  const int row = (warp & 3) * 32 + lane, hf = warp >> 2;
+  unsigned long long el_c[16], el_s[16];
 #pragma unroll
-  for (int k = 0; k < 32; ++k) {
-    float s0_, c0_, s1_, c1_;
-    sincosf(static_cast<float>(tid) * static_cast<float>(2 * k < half ? p.inv_freq[2 * k] : 0.0), &s0_, &c0_);
-    sincosf(static_cast<float>(tid) * static_cast<float>(2 * k + 1 < half ? p.inv_freq[2 * k + 1] : 0.0), &s1_, &c1_);
-    el_c[k] = pack2(c0_, c1_);
-    el_s[k] = pack2(s0_, s1_);
-  }
-  // the query of this unit, scaled by log2(e)/sqrt(d_h): thread i < half owns pair i
-  // turned to the first tile's offset here (fp64 once), then by (step_c, step_s) = e^{-i 128 phi} per tile
+  for (int m = 0; m < 4; ++m)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float4 c = __ldg(p.el_table + ((2 * m + hf) * 4 + e) * kTile + row);
+      el_c[4 * m + e] = pack2(c.x, c.y);
+      el_s[4 * m + e] = pack2(c.z, c.w);
+    }
+  // the query of this unit, scaled by log2(e)/sqrt(d_h): thread i < half owns pair i, turned to the first tile's
+  // offset here (the angle reduced in fp64), then by e^{-i 128 phi} per tile
   float q_re = 0.f, q_im = 0.f, step_c = 1.f, step_s = 0.f, q_norm2 = 0.f;
   if (tid < half) {
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head;
     const int ia = INTERLEAVED ? 2 * tid : tid, ib = INTERLEAVED ? 2 * tid + 1 : tid + half;
     const float a_re = __bfloat162float(qg[ia]) * p.q_scale, a_im = __bfloat162float(qg[ib]) * p.q_scale;
-    const double freq = p.inv_freq[tid];
-    double s_, c_;
-    sincos(static_cast<double>(n_b - 1 - t_lo * kTile) * freq, &s_, &c_);
-    q_re = static_cast<float>(a_re * c_ - a_im * s_);
-    q_im = static_cast<float>(a_re * s_ + a_im * c_);
+    double ang = static_cast<double>(n_b - 1 - t_lo * kTile) * p.inv_freq[tid];
+    ang -= kTwoPi * rint(ang / kTwoPi);
+    float s_, c_;
+    sincosf(static_cast<float>(ang), &s_, &c_);
+    q_re = a_re * c_ - a_im * s_;
+    q_im = a_re * s_ + a_im * c_;
     q_norm2 = a_re * a_re + a_im * a_im;
-    sincos(-static_cast<double>(kTile) * freq, &s_, &c_);
-    step_c = static_cast<float>(c_);
-    step_s = static_cast<float>(s_);
+    const float2 st = __ldg(p.tile_step + tid);
+    step_c = st.x;
+    step_s = st.y;
+    q_tile[tid] = q_re;                                      // the first tile's query
+    q_tile[64 + tid] = q_im;
+    q_tile[128 + tid] = -q_re;
   }
 
   cp_async_wait<0>();
@@ -147,180 +158,232 @@ __global__ void __launch_bounds__(kThreads, 2) decode_rope_kernel(const RopeDeco
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (tid == 0) {
-    fetch_k(t_lo);
-    fetch_v(t_lo);
-  }
   const uint32_t tmem = hdr->tmem_base;
-  const uint32_t tX0 = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-  volatile int* abort_flag = &hdr->abort_flag;
-  const uint32_t idesc = instr_desc(p.d_head, false);
-  const int ks_steps = rpk16 >> 4;
-  const int pos_q = n_b - 1;
 
-  // weighted sum o' += p V': thread (g, c) owns the column pair (2c, 2c+1) over the rows of row group g of every
-  // tile; the groups are added up once, at the end
-  const int col_pairs = hd.rp_v >> 1;
-  const int row_groups = min(kThreads / col_pairs, 16);
-  const int rows_per_group = (((kTile + row_groups - 1) / row_groups) + 7) & ~7;   // whole blocks of 8 rows
-  const int pv_g = tid / col_pairs, pv_c = tid - pv_g * col_pairs;
-  const int r_lo = min(kTile, pv_g * rows_per_group), r_hi = pv_g < row_groups ? min(kTile, r_lo + rows_per_group) : r_lo;
-  const unsigned char* v_col = Vs + 4 * pv_c;
-  float m_run = -INFINITY, l_thr = 0.f, o_acc0 = 0.f, o_acc1 = 0.f;
-  bool ok = true;
-  // lift of one tile (thread 0): X = K' (U^K)^T into accumulator `acc`
-  const uint64_t desc_k = smem_desc(smem_u32(Km), 128, grp_k), desc_u = smem_desc(smem_u32(Us), 128, grp_k);
-  auto issue_lift = [&](int acc) {
-    tc_fence_after();
-    for (int s = 0; s < ks_steps; ++s)                       // 16 rank elements (two chunks) a step
-      mma_ss(tmem + acc * kTile, desc_k + s * 16, desc_u + s * 16, idesc, s > 0);
-    mma_commit(&hdr->mma_done);
+  // ---- what the two issuing threads do (tile i of this CTA is tile t_lo + i of the unit)
+  const uint64_t policy = policy_evict_first();
+  const void* map_k = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
+  // K' tile i into buffer i & 1: two boxes of 64 rows per atom column, in the layout the lift's A operand names (no
+  // thread moves the tile); elements past the rank and rows past the capacity arrive as zeros, rows between the
+  // sequence's length and the capacity are finite (the cache starts as zeros) and meet zero weights
+  auto fetch_k = [&](int i) {
+    const int buf = i & 1, t = t_lo + i;
+    mbar_arrive_expect_tx(&hdr->k_full[buf], static_cast<uint32_t>(kt_bytes));
+    for (int a = 0; a < ak; ++a)
+      for (int hh = 0; hh < 2; ++hh)
+        tma_load_3d(Kt + buf * kt_bytes + a * kRopeAtom + hh * (kRopeAtom / 2), map_k, a * 64, t * kTile + hh * 64, b,
+                    &hdr->k_full[buf]);
   };
-  // the first tile: into the core-matrix layout, lift, and the staging buffer takes the second tile
-  if (!mbar_wait(&hdr->k_full, 0, p.status)) *abort_flag = 1;
-  relayout_k();
-  fence_async_smem();
-  __syncthreads();
-  if (*abort_flag) ok = false;
-  if (tid == 0 && ok) {
-    issue_lift(0);
-    if (t_lo + 1 < t_hi) fetch_k(t_lo + 1);
+  auto fetch_v = [&](int i) {
+    const int t = t_lo + i;
+    const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
+    mbar_arrive_expect_tx(&hdr->v_full, bytes);
+    bulk_load(Vs, p.cache + hd.v_off + (static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(t) * kTile) * rowb_v, bytes,
+              &hdr->v_full, policy);
+  };
+  // X(i) = K'(i) (U^K)^T into accumulator i & 1, once the tile's rows have landed; false if that wait gave up
+  auto issue_lift = [&](int i) -> bool {
+    if (!mbar_wait(&hdr->k_full[i & 1], (i >> 1) & 1u, p.status)) return false;
+    tc_fence_after();
+    const uint32_t idesc = instr_desc(p.d_head, false);
+    const uint64_t dk = smem_desc_sw128(smem_u32(Kt + (i & 1) * kt_bytes), 16, 1024), du = smem_desc(smem_u32(Us), 128, grp_k);
+    for (int s = 0; s < (rpk16 >> 4); ++s)                   // 16 rank elements a step: 32 bytes along the swizzled rows
+      mma_ss(tmem + (i & 1) * kTile, dk + (s >> 2) * (kRopeAtom >> 4) + (s & 3) * 2, du + s * 16, idesc, s > 0);
+    mma_commit(&hdr->x_full[i & 1]);
+    return true;
+  };
+  // ---- before the first tile: two K' tiles and the V' tile requested, X(0) and X(1) under way, then K'(2) behind X(0)
+  bool live = true;                                          // an issuing thread: none of its waits has given up
+  if (tid == kRopeRequester) {
+    tensormap_acquire(map_k);
+    fetch_k(0);
+    if (nt_cta > 1) fetch_k(1);
+    fetch_v(0);
+    if (nt_cta > 2) {
+      live = mbar_wait(&hdr->x_full[0], 0u, p.status);
+      if (live) fetch_k(2);
+    }
+  } else if (tid == kRopeLifter) {
+    live = issue_lift(0);
+    if (live && nt_cta > 1) live = issue_lift(1);
   }
-  for (int t = t_lo; t < t_hi && ok; ++t) {
-    const uint32_t par = (t - t_lo) & 1u;
-    const uint32_t tX = tX0 + par * kTile;
-    // ---- the query pairs turned by (pos_q - 128 t) phi
+  __syncwarp();
+
+  const uint32_t tX = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  // weighted sum o' += p V' (warps 0-5): thread (vg, vc) owns the eight columns of 16-byte chunk vc over the rows of
+  // row group vg of every tile; the row groups are added up once, at the end
+  const int chunks = hd.rp_v >> 3;
+  const int row_groups = min(kRopeSumThreads / chunks, 64);
+  const int rows_per_group = (kTile + row_groups - 1) / row_groups;
+  const int pv_g = tid / chunks, pv_c = tid - pv_g * chunks;
+  const bool pv_on = tid < kRopeSumThreads && pv_g < row_groups;
+  const int r_lo = min(kTile, pv_g * rows_per_group), r_hi = pv_on ? min(kTile, r_lo + rows_per_group) : r_lo;
+  unsigned long long o_acc[4] = {0ull, 0ull, 0ull, 0ull};   // columns (0,1), (2,3), (4,5), (6,7) of the chunk
+  // online softmax in base 2 against a reference m_ref that every thread of the CTA holds alike; it moves only when
+  // a score of the tile passes it by more than kRopeLazy (the first tile always does)
+  float m_ref = -INFINITY, l_thr = 0.f;
+  bool ok = true;
+  for (int i = 0; i < nt_cta; ++i) {
+    const int t = t_lo + i;
+    const uint32_t par = i & 1u;
+    const float* qt = q_tile + par * 192;                    // this tile's query pairs (written a tile ago)
+    // the V' tile is free once the weighted sum of tile i - 1 is over: request this tile's rows
+    if (tid == kRopeRequester && i >= 1 && live) {
+      live = mbar_wait(&hdr->v_free, (i - 1) & 1u, p.status);
+      if (live) fetch_v(i);
+    }
+    __syncwarp();
+    const bool have_x = mbar_wait(&hdr->x_full[par], (i >> 1) & 1u, p.status);
+    tc_fence_after();
+    // ---- this thread's half of the row's score.  Two pairs per packed instruction:
+    // W = Q_t conj(E_l), pair term = Re(W conj(X)) = W_re x_re + W_im x_im.
+    unsigned long long acc_re = 0ull, acc_im = 0ull;         // (0.f, 0.f)
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const int c = 2 * m + hf;
+      uint32_t xc[16];                                       // re[8], im[8] (pairs (i, i + d_h/2)) or re, im alternating
+      if (have_x && 8 * c < half) {
+        if (INTERLEAVED) {
+          tmem_ld16(tX + par * kTile + 16 * c, xc);
+        } else {
+          tmem_ld8(tX + par * kTile + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(&xc[0]));
+          tmem_ld8(tX + par * kTile + half + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(&xc[8]));
+        }
+      }
+      tmem_wait_ld();
+      if (8 * c < half) {
+        const float* qc = qt + 8 * c;
+#pragma unroll
+        for (int e = 0; e < 8; e += 4) {                     // four pairs a step
+          const float4 qr4 = *reinterpret_cast<const float4*>(qc + e);
+          const float4 qi4 = *reinterpret_cast<const float4*>(qc + 64 + e);
+          const float4 qn4 = *reinterpret_cast<const float4*>(qc + 128 + e);
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            const int ee = e + 2 * k;
+            unsigned long long x_re, x_im;
+            if (INTERLEAVED) {
+              x_re = pack2(__uint_as_float(xc[2 * ee]), __uint_as_float(xc[2 * ee + 2]));
+              x_im = pack2(__uint_as_float(xc[2 * ee + 1]), __uint_as_float(xc[2 * ee + 3]));
+            } else {
+              x_re = pack2(__uint_as_float(xc[ee]), __uint_as_float(xc[ee + 1]));
+              x_im = pack2(__uint_as_float(xc[8 + ee]), __uint_as_float(xc[8 + ee + 1]));
+            }
+            const unsigned long long qr = k == 0 ? pack2(qr4.x, qr4.y) : pack2(qr4.z, qr4.w);
+            const unsigned long long qi = k == 0 ? pack2(qi4.x, qi4.y) : pack2(qi4.z, qi4.w);
+            const unsigned long long qn = k == 0 ? pack2(qn4.x, qn4.y) : pack2(qn4.z, qn4.w);
+            const unsigned long long ec = el_c[4 * m + (ee >> 1)], es = el_s[4 * m + (ee >> 1)];
+            const unsigned long long w_re = fma2p(qi, es, mul2p(qr, ec));                  // Qr c + Qi s
+            const unsigned long long w_im = fma2p(qn, es, mul2p(qi, ec));                  // Qi c - Qr s
+            acc_re = fma2p(w_re, x_re, acc_re);
+            acc_im = fma2p(w_im, x_im, acc_im);
+          }
+        }
+      }
+    }
+    {
+      float s0, s1, s2, s3;
+      unpack2(acc_re, s0, s1);
+      unpack2(acc_im, s2, s3);
+      sc[hf * kTile + row] = (s0 + s2) + (s1 + s3);
+    }
+    tc_fence_before();
+    // both halves of every row's score are in shared memory and X(i) is read; a wait that gave up anywhere ends the loop
+    if (cta_sync_or(!have_x || !live)) { ok = false; break; }
+    // ---- the next tile's query: one more turn by -128 phi into the other buffer (read after the next barrier);
+    // the length is pulled back to |q| so that rounding does not drift over a thousand tiles
     if (tid < half) {
-      q_tile[tid] = q_re;
-      q_tile[64 + tid] = q_im;
-      // the next tile's query: one more turn by -128 phi; the length is pulled back to |q| so that rounding
-      // does not drift over a thousand tiles
       const float n_re = q_re * step_c - q_im * step_s, n_im = q_re * step_s + q_im * step_c;
       const float fix = 1.5f - 0.5f * (n_re * n_re + n_im * n_im) / fmaxf(q_norm2, 1e-30f);   // ~ |q| / |n|
       q_re = n_re * fix;
       q_im = n_im * fix;
+      float* qn = q_tile + (par ^ 1u) * 192;
+      qn[tid] = q_re;
+      qn[64 + tid] = q_im;
+      qn[128 + tid] = -q_re;
     }
-    // ---- X(t) is complete (its lift went out during the previous tile): the core-matrix buffer is free
-    if (!mbar_wait(&hdr->mma_done, par, p.status)) *abort_flag = 1;
-    __syncthreads();                                         // q_tile written
-    if (*abort_flag) { ok = false; break; }
-    tc_fence_after();
-    // two pairs per packed instruction: W = Q_t conj(E_l), pair term = Re(W conj(X)) = W_re x_re + W_im x_im
-    unsigned long long acc_re = 0ull, acc_im = 0ull;         // (0.f, 0.f)
+    // ---- the row's weight against the reference as it stands (warps 0-3: one thread per row)
+    float s = -INFINITY, pj = 0.f;
+    if (hf == 0) {
+      if (t * kTile + row < n_b) s = sc[row] + sc[kTile + row];
+      pj = ex2(s - m_ref);                                   // redone below if the reference moves
+      p_row[row] = pj;
+    }
+    const bool have_v = tid >= kRopeSumThreads || mbar_wait(&hdr->v_full, par, p.status);
+    // the weights are written, the V' tile has landed; the reference must move if a score passed it by kRopeLazy
+    if (cta_sync_or(s > m_ref + kRopeLazy || !have_v)) {
+      if (cta_sync_or(!have_v)) { ok = false; break; }       // (also: every thread has read the weights' flag state)
+      // every thread adds up the four rows lane, lane + 32, ...: the tile maximum is one warp reduction
+      float mx = -INFINITY;
 #pragma unroll
-    for (int c0 = 0; c0 < 64; c0 += 16) {
-      if (c0 < half) {
-        uint32_t xa[16], xb[16];
-        if (INTERLEAVED) {                                   // pairs (2i, 2i+1): columns 2 c0 .. 2 c0 + 31
-          tmem_ld16(tX + 2 * c0, xa);
-          tmem_ld16(tX + 2 * c0 + 16, xb);
-        } else {                                             // pairs (i, i + d_h/2)
-          tmem_ld16(tX + c0, xa);
-          tmem_ld16(tX + half + c0, xb);
-        }
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-          unsigned long long x_re, x_im;
-          if (INTERLEAVED) {
-            const uint32_t* src = i < 8 ? xa : xb;
-            x_re = pack2(__uint_as_float(src[(2 * i) & 15]), __uint_as_float(src[(2 * i + 2) & 15]));
-            x_im = pack2(__uint_as_float(src[(2 * i + 1) & 15]), __uint_as_float(src[(2 * i + 3) & 15]));
-          } else {
-            x_re = pack2(__uint_as_float(xa[i]), __uint_as_float(xa[i + 1]));
-            x_im = pack2(__uint_as_float(xb[i]), __uint_as_float(xb[i + 1]));
-          }
-          const unsigned long long qr = *reinterpret_cast<const unsigned long long*>(q_tile + c0 + i);
-          const unsigned long long qi = *reinterpret_cast<const unsigned long long*>(q_tile + 64 + c0 + i);
-          const unsigned long long ec = el_c[(c0 + i) >> 1], es = el_s[(c0 + i) >> 1];
-          const unsigned long long w_re = fma2p(qi, es, mul2p(qr, ec));                  // Qr c + Qi s
-          const unsigned long long w_im = fma2p(qr ^ 0x8000000080000000ull, es, mul2p(qi, ec));   // Qi c - Qr s
-          acc_re = fma2p(w_re, x_re, acc_re);
-          acc_im = fma2p(w_im, x_im, acc_im);
-        }
+      for (int k = 0; k < 4; ++k) {
+        const int r = k * 32 + lane;
+        if (t * kTile + r < n_b) mx = fmaxf(mx, sc[r] + sc[kTile + r]);
       }
-    }
-    float s0, s1, s2, s3;
-    unpack2(acc_re, s0, s1);
-    unpack2(acc_im, s2, s3);
-    s0 += s2;
-    s1 += s3;
-    // ---- K'(t+1) landed a tile ago: into the core-matrix layout now, its lift goes out after the barrier below
-    if (t + 1 < t_hi) {
-      if (!mbar_wait(&hdr->k_full, par ^ 1u, p.status)) *abort_flag = 1;
-      relayout_k();
-      fence_async_smem();
-    }
-    const int j = t * kTile + tid;
-    const bool live = j < n_b;
-    const float s = live ? s0 + s1 : -INFINITY;
-    // ---- online softmax over the tile: block maximum, weights, running sum per thread
-    float mx = s;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) hdr->red[warp] = mx;
-    tc_fence_before();
-    __syncthreads();                                         // every thread has read its row of X and moved its chunks
-    if (tid == 0 && t + 1 < t_hi && !*abort_flag) {          // lift of tile t+1 behind the softmax and the weighted sum;
-      issue_lift(static_cast<int>(par ^ 1u));                // the staging buffer takes tile t+2
-      if (t + 2 < t_hi) fetch_k(t + 2);
-    }
-    const float m_new = fmaxf(m_run, fmaxf(fmaxf(hdr->red[0], hdr->red[1]), fmaxf(hdr->red[2], hdr->red[3])));
-    const float alpha = ex2(m_run - m_new);                  // 0 at the first tile
-    m_run = m_new;
-    const float pj = live ? ex2(s - m_new) : 0.f;
-    l_thr = fmaf(l_thr, alpha, pj);
-    p_row[tid] = pj;
-    if (!mbar_wait(&hdr->v_full, par, p.status)) *abort_flag = 1;
-    __syncthreads();
-    if (*abort_flag) { ok = false; break; }
-    // ---- o' = alpha o' + sum_j p_j V'[j][2c..2c+1] over this thread's rows (row-major tile)
-    {
-      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-      for (int r = r_lo; r < r_hi; r += 8) {
-        const float4 pa = *reinterpret_cast<const float4*>(p_row + r);
-        const float4 pb = *reinterpret_cast<const float4*>(p_row + r + 4);
-        const unsigned char* vr = v_col + r * rowb_v;
-        uint32_t v[8];
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_new = fmaxf(m_ref, mx);
+      const float alpha = ex2(m_ref - m_new);                // 0 at the first tile
+      const unsigned long long alpha2 = pack2(alpha, alpha);
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj) v[jj] = *reinterpret_cast<const uint32_t*>(vr + jj * rowb_v);
-        a0 = fmaf(pa.x, __uint_as_float(v[0] << 16), a0); a1 = fmaf(pa.x, __uint_as_float(v[0] & 0xffff0000u), a1);
-        b0 = fmaf(pa.y, __uint_as_float(v[1] << 16), b0); b1 = fmaf(pa.y, __uint_as_float(v[1] & 0xffff0000u), b1);
-        a0 = fmaf(pa.z, __uint_as_float(v[2] << 16), a0); a1 = fmaf(pa.z, __uint_as_float(v[2] & 0xffff0000u), a1);
-        b0 = fmaf(pa.w, __uint_as_float(v[3] << 16), b0); b1 = fmaf(pa.w, __uint_as_float(v[3] & 0xffff0000u), b1);
-        a0 = fmaf(pb.x, __uint_as_float(v[4] << 16), a0); a1 = fmaf(pb.x, __uint_as_float(v[4] & 0xffff0000u), a1);
-        b0 = fmaf(pb.y, __uint_as_float(v[5] << 16), b0); b1 = fmaf(pb.y, __uint_as_float(v[5] & 0xffff0000u), b1);
-        a0 = fmaf(pb.z, __uint_as_float(v[6] << 16), a0); a1 = fmaf(pb.z, __uint_as_float(v[6] & 0xffff0000u), a1);
-        b0 = fmaf(pb.w, __uint_as_float(v[7] << 16), b0); b1 = fmaf(pb.w, __uint_as_float(v[7] & 0xffff0000u), b1);
+      for (int k = 0; k < 4; ++k) o_acc[k] = mul2p(o_acc[k], alpha2);
+      l_thr *= alpha;
+      m_ref = m_new;
+      if (hf == 0) {
+        pj = ex2(s - m_ref);                                 // 0 for a row past the sequence's length
+        p_row[row] = pj;
       }
-      o_acc0 = fmaf(o_acc0, alpha, a0 + b0);
-      o_acc1 = fmaf(o_acc1, alpha, a1 + b1);
+      __syncthreads();                                       // the weights are rewritten
     }
-    __syncthreads();                                         // the V' tile is free again
-    if (tid == 0 && t + 1 < t_hi) fetch_v(t + 1);
+    l_thr += pj;
+    if (tid < kRopeSumThreads) {
+      // ---- o' += sum_j p_j V'[j][8 vc .. 8 vc + 7] over this thread's rows (row-major tile, 16 bytes a row)
+      const unsigned char* v_chunk = Vs + 16 * pv_c;
+#pragma unroll 2
+      for (int r = r_lo; r < r_hi; ++r) {
+        const uint4 v = *reinterpret_cast<const uint4*>(v_chunk + r * rowb_v);
+        const float pr = p_row[r];
+        const unsigned long long p2 = pack2(pr, pr);
+        o_acc[0] = fma2p(p2, pack2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u)), o_acc[0]);
+        o_acc[1] = fma2p(p2, pack2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u)), o_acc[1]);
+        o_acc[2] = fma2p(p2, pack2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u)), o_acc[2]);
+        o_acc[3] = fma2p(p2, pack2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u)), o_acc[3]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&hdr->v_free);              // this warp has read its rows of the V' tile
+    } else {
+      // ---- meanwhile the two issuing threads: K'(i + 3) into the buffer X(i + 1) was lifted from (that lift went out
+      // a tile ago), and X(i + 2) into the accumulator every thread has just read (its rows were requested a tile ago)
+      if (tid == kRopeRequester && live && i + 3 < nt_cta) {
+        live = mbar_wait(&hdr->x_full[(i + 1) & 1], ((i + 1) >> 1) & 1u, p.status);
+        if (live) fetch_k(i + 3);
+      }
+      if (tid == kRopeLifter && live && i + 2 < nt_cta) live = issue_lift(i + 2);
+      __syncwarp();
+    }
   }
-  if (!ok) *abort_flag = 1;
 
-  // ---- the piece's partial: m, l (sum over the threads' rows), o'
+  // ---- the piece's partial: m, l (sum over the rows), o'
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) l_thr += __shfl_xor_sync(0xffffffffu, l_thr, o);
-  __syncthreads();
-  if (lane == 0) hdr->red[4 + warp] = l_thr;
+  __syncthreads();                                           // every thread is through with the V' tile
+  if (lane == 0 && hf == 0) hdr->red[warp] = l_thr;
+  // add up the row groups (the V' tile's shared memory is free: its last copy was waited for, or the launch gave up)
+  float* o_red = reinterpret_cast<float*>(Vs);
+  if (ok && pv_on) {
+    float* dst = o_red + pv_g * hd.rp_v + 8 * pv_c;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) unpack2(o_acc[k], dst[2 * k], dst[2 * k + 1]);
+  }
   __syncthreads();
   if (tid == 0) {
-    part[0] = m_run;
-    part[1] = (hdr->red[4] + hdr->red[5]) + (hdr->red[6] + hdr->red[7]);
+    part[0] = m_ref;
+    part[1] = (hdr->red[0] + hdr->red[1]) + (hdr->red[2] + hdr->red[3]);
   }
-  // add up the row groups (the V' tile's shared memory is free now)
-  float* o_red = reinterpret_cast<float*>(Vs);
-  if (pv_g < row_groups) {
-    o_red[pv_g * hd.rp_v + 2 * pv_c] = o_acc0;
-    o_red[pv_g * hd.rp_v + 2 * pv_c + 1] = o_acc1;
-  }
-  __syncthreads();
   if (tid < hd.rp_v) {
     float o = 0.f;
-    for (int g = 0; g < row_groups; ++g) o += o_red[g * hd.rp_v + tid];
+    if (ok)
+      for (int k = 0; k < row_groups; ++k) o += o_red[k * hd.rp_v + tid];
     part[4 + tid] = o;
   }
   tc_fence_before();
@@ -363,9 +426,10 @@ __global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParam
 }  // namespace
 
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
-  const size_t k16 = (max_rp_k + 15) & ~15;
-  // header, U^K image, K' staging + core-matrix copy, V' tile
-  return 2048 + static_cast<size_t>(d_head) * k16 * 2 + kTile * static_cast<size_t>(max_rp_k + k16 + max_rp_v) * 2;
+  const int k16 = (max_rp_k + 15) & ~15;
+  // header, U^K image, two K' tiles in swizzled atom columns of 64 elements, V' tile
+  return kRopeHeaderBytes + rope_kb(d_head * k16 * 2) + 2 * static_cast<size_t>((k16 + 63) >> 6) * kRopeAtom +
+         rope_kb(kTile * max_rp_v * 2);
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
@@ -374,8 +438,8 @@ cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStrea
                                        : ensure_dynamic_smem(decode_rope_kernel<false>, smem, configured[0]);
   if (ec != cudaSuccess) return ec;
   dim3 grid(p.B * p.H, p.splits);
-  if (p.interleaved) decode_rope_kernel<true><<<grid, kThreads, smem, s>>>(p);
-  else decode_rope_kernel<false><<<grid, kThreads, smem, s>>>(p);
+  if (p.interleaved) decode_rope_kernel<true><<<grid, kRopeThreads, smem, s>>>(p);
+  else decode_rope_kernel<false><<<grid, kRopeThreads, smem, s>>>(p);
   ++*launches;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -174,6 +174,8 @@ struct RopeDecodeParams {    // decode for models with rotary position embedding
   float* partials;          // [B*H][splits][part_stride]: m, l, pad, pad, o'[rp_v]
   int* status;
   const double* inv_freq;   // [d_head/2]: base^(-2i/d_head)
+  const float2* tile_step;  // [64]: cos, sin of -128 phi_i (one tile back along the cache)
+  const float4* el_table;   // [32][128]: cos, cos, sin, sin of l phi for pairs 2k, 2k + 1 and row offset l
   const int32_t* deficit;   // [B]: sequence b holds n - deficit[b] rows; NULL = all hold n
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head
   int32_t part_stride;
@@ -266,6 +268,11 @@ cudaError_t launch_prefill_rope(const PrefillParams& p, int max_rp_k, int max_rp
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
+// bytes of the rotary constants a layer keeps: inverse frequencies (64 doubles), per-tile steps (64 float2),
+// the row-offset table (32 x 128 float4)
+constexpr size_t kRopeStepOffset = 64 * sizeof(double);
+constexpr size_t kRopeTableOffset = kRopeStepOffset + 64 * 2 * sizeof(float);
+constexpr size_t kRopeConstBytes = kRopeTableOffset + 32 * 128 * 4 * sizeof(float);
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches);
 int prefill_tc_ws_stages(int max_rp_k, int max_rp_v, int d_head, size_t* smem_bytes);   // 0 = does not fit
 cudaError_t launch_prefill_tc_ws(const PrefillParams& p, int stages, size_t smem, bool alibi, cudaStream_t s,
