@@ -62,7 +62,9 @@ struct __align__(16) RopeSmemHeader {
 // parts of the shared memory image are multiples of 1 KB (the swizzled tiles need that alignment)
 __host__ __device__ constexpr int rope_kb(int bytes) { return (bytes + 1023) & ~1023; }
 
-template <bool INTERLEAVED>
+// HALF = d_head / 2 known at compile time (64: the usual head of 128 dimensions; no chunk of pairs is ever empty
+// and the TMEM columns are constants), or 0: taken from the launch parameters.
+template <bool INTERLEAVED, int HALF>
 __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
@@ -76,7 +78,7 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
   const int ak = (rpk16 + 63) >> 6;                          // atom columns (64 elements) of a K' tile
   const int kt_bytes = ak * kRopeAtom, v_bytes = kTile * rowb_v;
   const int u_bytes = p.d_head * rpk16 * 2;                  // bf16 image of U^K (the high part of the stored pair)
-  const int half = p.d_head >> 1;
+  const int half = HALF ? HALF : p.d_head >> 1;
 
   float* q_tile = reinterpret_cast<float*>(smem + 256);      // [2][192] the query pairs of a tile: re[64], im[64], -re[64]
   float* p_row = q_tile + 384;                               // [128] softmax weights of the tile
@@ -242,7 +244,7 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
     for (int m = 0; m < 4; ++m) {
       const int c = 2 * m + hf;
       uint32_t xc[16];                                       // re[8], im[8] (pairs (i, i + d_h/2)) or re, im alternating
-      if (have_x && 8 * c < half) {
+      if (have_x && (HALF == 64 || 8 * c < half)) {
         if (INTERLEAVED) {
           tmem_ld16(tX + par * kTile + 16 * c, xc);
         } else {
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
         }
       }
       tmem_wait_ld();
-      if (8 * c < half) {
+      if (HALF == 64 || 8 * c < half) {
         const float* qc = qt + 8 * c;
 #pragma unroll
         for (int e = 0; e < 8; e += 4) {                     // four pairs a step
@@ -433,15 +435,17 @@ size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
-  static size_t configured[2][kMaxDevices] = {};
-  const cudaError_t ec = p.interleaved ? ensure_dynamic_smem(decode_rope_kernel<true>, smem, configured[1])
-                                       : ensure_dynamic_smem(decode_rope_kernel<false>, smem, configured[0]);
-  if (ec != cudaSuccess) return ec;
-  dim3 grid(p.B * p.H, p.splits);
-  if (p.interleaved) decode_rope_kernel<true><<<grid, kRopeThreads, smem, s>>>(p);
-  else decode_rope_kernel<false><<<grid, kRopeThreads, smem, s>>>(p);
+  static size_t configured[4][kMaxDevices] = {};
+  auto run = [&](auto kernel, size_t (&done)[kMaxDevices]) -> cudaError_t {
+    const cudaError_t ec = ensure_dynamic_smem(kernel, smem, done);
+    if (ec != cudaSuccess) return ec;
+    kernel<<<dim3(p.B * p.H, p.splits), kRopeThreads, smem, s>>>(p);
+    return cudaGetLastError();
+  };
+  cudaError_t e;
+  if (p.d_head == 128) e = p.interleaved ? run(decode_rope_kernel<true, 64>, configured[3]) : run(decode_rope_kernel<false, 64>, configured[2]);
+  else e = p.interleaved ? run(decode_rope_kernel<true, 0>, configured[1]) : run(decode_rope_kernel<false, 0>, configured[0]);
   ++*launches;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   rope_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
   ++*launches;
