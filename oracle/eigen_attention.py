@@ -305,15 +305,20 @@ class LayerOracle:
     #    query heads): the cache, U^K and U^V belong to the K/V head, every query head of its group uses them
     def decode_gqa(self, q: np.ndarray, group: int) -> np.ndarray:
         """q: [B, 1, H*group, d_h], query head hq belongs to K/V head hq // group.  Returns [B, 1, H*group, d_h].
-        Each query head is Eq. 3 in the space of Eq. 7 against its K/V head's rank-r rows."""
+        Each query head is Eq. 3 in the space of Eq. 7 against its K/V head's rank-r rows; with a rotary embedding
+        each query head is the Section 4.3 form against its K/V head's rows and bases."""
         q = np.asarray(q, dtype=F64).reshape(self.B, self.H * group, self.d_h)
-        assert self.rope is None
         out = np.zeros((self.B, 1, self.H * group, self.d_h), dtype=F64)
         for (b, h) in self.units:
             Kp, Vp = self.Kp[(b, h)], self.Vp[(b, h)]
             assert Kp.shape[0] == self.len and self.len > 0
             for i in range(group):
                 hq = h * group + i
+                if self.rope is not None:
+                    assert not self.alibi[h]
+                    out[b, 0, hq] = decode_head_rope(q[b, hq], Kp, Vp, self.U_K[h], self.U_V[h], self.rope["base"],
+                                                     self.rope.get("interleaved", False), 0)
+                    continue
                 qp = to_rank_space(q[b, hq], self.U_K[h])
                 s = (Kp @ qp) / math.sqrt(self.d_h)
                 if self.alibi[h]:

@@ -455,7 +455,7 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
 // Section 4.3: decode for a layer with rotary position embedding.  Row j of the cache sits at position j, the
 // query at position len - 1.
 ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
-                         uint32_t flags, cudaStream_t s) {
+                         uint32_t flags, cudaStream_t s, int group = 1) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
   if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: not available with a page table");
   if (flags & ~EA_OUT_LOWRANK)
@@ -484,11 +484,12 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   // rotation constants, the first tiles' way from memory) worth a few tiles: take the split count with the least
   // waves x (tiles + start-up), within the partials the workspace holds.
   const int ctas_per_sm = smem * 2 + 4096 <= static_cast<size_t>(228 * 1024) ? 2 : 1;
-  const int64_t units = static_cast<int64_t>(B) * H;
-  int64_t cap = (units + kMaxDecodeCtas) * kPartialSlack / units;
+  const int64_t units = static_cast<int64_t>(B) * H * group;    // (sequence, query head) pairs
+  int64_t cap = (static_cast<int64_t>(B) * H + kMaxDecodeCtas) * kPartialSlack / units;
+  if (cap < 1) return fail(h, EA_ERR_CAPACITY, "decode with rotary embedding: batch x heads x group = %lld partials exceed the workspace",
+                           static_cast<long long>(units));
   if (cap > p.nt) cap = p.nt;
   if (cap > 65535) cap = 65535;
-  if (cap < 1) cap = 1;
   int64_t splits = 1;
   if (h->opt_ctas > 0) {
     splits = (h->opt_ctas + units - 1) / units;
@@ -503,6 +504,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   }
   p.splits = static_cast<int32_t>(splits);
   p.interleaved = h->rope_interleaved;
+  p.group = group;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
@@ -1116,9 +1118,12 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   if (group < 1 || group > 16) return fail(h, EA_ERR_SHAPE, "decode_gqa: group %d (1..16)", group);
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
-  if (h->rope || h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a position scheme set");
+  if (h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with an ALiBi bias set");
   if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table");
   if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty (for some sequence)");
+  // Section 4.3 for a group: every query head of the group is a unit of the rotary kernel over its K/V head's rows
+  if (h->rope)
+    return do_decode_rope(h, d_q, stride_b_q, d_out, stride_b_out, 0u, static_cast<cudaStream_t>(cuda_stream), group);
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const size_t smem = ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);

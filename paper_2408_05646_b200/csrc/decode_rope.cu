@@ -69,8 +69,11 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
   extern __shared__ __align__(1024) unsigned char smem[];
   RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // a unit is a (sequence, query head) pair; with grouped queries `group` query heads read the rows of one K/V head
+  // (its units are B apart, so they run at the same time and all but the first find the tiles in L2)
   const int unit = blockIdx.x, split = blockIdx.y;
-  const int h = unit / p.B, b = unit - h * p.B;
+  const int hq = unit / p.B, b = unit - hq * p.B;
+  const int h = hq / p.group;
   const HeadInfo hd = p.heads[h];
   const int rpk16 = (hd.rp_k + 15) & ~15;
   const int nch_k = rpk16 >> 3, grp_k = nch_k << 7;
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
   // offset here (the angle reduced in fp64), then by e^{-i 128 phi} per tile
   float q_re = 0.f, q_im = 0.f, step_c = 1.f, step_s = 0.f, q_norm2 = 0.f;
   if (tid < half) {
-    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(h) * p.d_head;
+    const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q) + b * p.q_stride_b + static_cast<int64_t>(hq) * p.d_head;
     const int ia = INTERLEAVED ? 2 * tid : tid, ib = INTERLEAVED ? 2 * tid + 1 : tid + half;
     const float a_re = __bfloat162float(qg[ia]) * p.q_scale, a_im = __bfloat162float(qg[ib]) * p.q_scale;
     double ang = static_cast<double>(n_b - 1 - t_lo * kTile) * p.inv_freq[tid];
@@ -397,7 +400,8 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
 __global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParams p) {
   __shared__ float o_sm[128];
   const int unit = blockIdx.x, t = threadIdx.x;
-  const int h = unit / p.B, b = unit - h * p.B;
+  const int hq = unit / p.B, b = unit - hq * p.B;
+  const int h = hq / p.group;
   const HeadInfo hd = p.heads[h];
   const float* base = p.partials + static_cast<size_t>(unit) * p.splits * p.part_stride;
   float M = -INFINITY;
@@ -421,7 +425,7 @@ __global__ void __launch_bounds__(128) rope_combine_kernel(const RopeDecodeParam
     const float* Ut = p.basis + hd.uvt_off;                  // (U^V)^T : rp_v x d_head
     float y = 0.f;
     for (int c = 0; c < hd.rp_v; ++c) y = fmaf(o_sm[c], __ldg(Ut + c * p.d_head + t), y);
-    out[b * p.out_stride_b + static_cast<int64_t>(h) * p.d_head + t] = __float2bfloat16_rn(y);
+    out[b * p.out_stride_b + static_cast<int64_t>(hq) * p.d_head + t] = __float2bfloat16_rn(y);
   }
 }
 
@@ -439,7 +443,7 @@ cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStrea
   auto run = [&](auto kernel, size_t (&done)[kMaxDevices]) -> cudaError_t {
     const cudaError_t ec = ensure_dynamic_smem(kernel, smem, done);
     if (ec != cudaSuccess) return ec;
-    kernel<<<dim3(p.B * p.H, p.splits), kRopeThreads, smem, s>>>(p);
+    kernel<<<dim3(p.B * p.H * p.group, p.splits), kRopeThreads, smem, s>>>(p);
     return cudaGetLastError();
   };
   cudaError_t e;
@@ -447,7 +451,7 @@ cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStrea
   else e = p.interleaved ? run(decode_rope_kernel<true, 0>, configured[1]) : run(decode_rope_kernel<false, 0>, configured[0]);
   ++*launches;
   if (e != cudaSuccess) return e;
-  rope_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
+  rope_combine_kernel<<<p.B * p.H * p.group, 128, 0, s>>>(p);
   ++*launches;
   return cudaGetLastError();
 }

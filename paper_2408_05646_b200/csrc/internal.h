@@ -184,6 +184,7 @@ struct RopeDecodeParams {    // decode for models with rotary position embedding
   int32_t nt;               // tiles of 128 rows per unit
   int32_t splits;           // CTAs per unit
   int32_t interleaved;      // pairs (2i, 2i+1) instead of (i, i + d_head/2)
+  int32_t group;            // query heads per K/V head (1: every head has its own rows); q and out have H * group heads
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
 };

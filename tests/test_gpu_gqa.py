@@ -88,3 +88,35 @@ def test_gqa_rejections(B):
     lay.set_alibi([0.5, 0.25])
     with pytest.raises(B.EigenAttnError):
         lay.decode_gqa(q, 1)
+
+
+@pytest.mark.parametrize("H,g,d,rk,rv,n,base,interleaved", [
+    (2, 4, 128, [80, 80], [80, 80], 1037, 10000.0, False),          # the 8B-class shape: several tiles, ragged tail
+    (3, 2, 64, [24, 64, 40], [56, 8, 64], 517, 500000.0, True),     # small d_head, per-head ranks, interleaved pairs
+    (1, 16, 128, [80], [80], 17, 10000.0, False),                   # largest group, shorter than a tile
+    (2, 5, 128, [64, 112], [96, 48], 3000, 10000.0, True),          # a group that is not a power of two
+])
+def test_gqa_decode_with_rotary_embedding_matches_oracle(B, H, g, d, rk, rv, n, base, interleaved):
+    """Section 4.3 for grouped queries (the Llama models that share K/V heads also rotate their keys): every query
+    head against its K/V head's lifted, rotated keys."""
+    from helpers import OraclePair
+    B_ = 2
+    U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n + 1, BF16, seed_cfg=167)
+    lay = B.EigenAttnLayer(B_, H, d, n + 4, BF16, U_k, U_v)
+    lay.set_rope(base, interleaved)
+    lay.append_kv(k[:, :n], v[:, :n])
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16, rope={"base": base, "interleaved": interleaved})
+    ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
+    for step, scale in enumerate((1.0, 4.0)):                        # the second step with peaked weights
+        if step:
+            lay.append_kv(k[:, n:n + 1], v[:, n:n + 1])
+            ref.append_kv(to_np(k[:, n:n + 1]), to_np(v[:, n:n + 1]))
+        q = (group_queries(B_, H, g, d, 180 + step).float() * scale).to(BF16)
+        expect = ref.decode_gqa(to_np(q), g)
+        for ctas in (0, 1, 7, 300):                                  # CTAs per unit must not matter
+            lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+            assert_close(lay.decode_gqa(q, g), expect, BF16, f"gqa rope decode step {step} ctas={ctas}")
+    lay.set_option(B.EA_OPT_DECODE_CTAS, 0)                          # one query head per K/V head: the multi-head call
+    q1 = q[:, :, ::g].contiguous()
+    assert torch.equal(lay.decode_gqa(q1, 1), lay.decode(q1))
+    lay.poll_status()
