@@ -251,8 +251,9 @@ ea_status eigen_attn_set_len(eigen_attn_t h, int32_t len);
  * b (EA_ERR_SHAPE otherwise).  The split-KV work decomposition follows the true lengths, so a step costs what
  * the rows actually cached cost.  batch <= 1024.  eigen_attn_set_len returns to equal lengths.
  * With a rotary embedding each sequence's query sits at its own last position.  With a quantised cache attached
- * every sequence keeps its own count of rows held as codes (eigen_attn_quant_lens).  While lengths differ,
- * prefill returns EA_ERR_UNSUPPORTED.  The lengths are uploaded on the stream
+ * every sequence keeps its own count of rows held as codes (eigen_attn_quant_lens).  eigen_attn_prefill places
+ * the T new tokens of sequence b behind that sequence's own rows (token t at position lens[b] + t, attending over
+ * the sequence's rows only; the projections then run on the CUDA cores).  The lengths are uploaded on the stream
  * (asynchronous; the array may be reused when the call returns), so the calls that follow must run on that
  * stream or be ordered after it. */
 ea_status eigen_attn_set_lens(eigen_attn_t h, const int32_t* lens, void* cuda_stream);

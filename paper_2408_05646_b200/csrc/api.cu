@@ -788,7 +788,6 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
                              int64_t stride_b, int64_t stride_t, void* d_out, int64_t out_stride_b,
                              int64_t out_stride_t, uint32_t flags, void* cuda_stream) {
   if (!h) return EA_ERR_INVALID_ARG;
-  if (h->max_deficit > 0) return fail(h, EA_ERR_UNSUPPORTED, "prefill: not available for a batch of unequal lengths (eigen_attn_set_lens)");
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL q or out");
   if (h->rope && (flags & EA_Q_PREPROJECTED))
     return fail(h, EA_ERR_INVALID_ARG, "prefill with rotary embedding: EA_Q_PREPROJECTED (the query must be full rank)");
@@ -825,7 +824,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
       p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
     }
     p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
-    p.len0 = len0;
+    p.len0 = len0; p.deficit = dev_deficit(h);
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
     p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
     p.pages = dev_pages(h);
@@ -851,7 +850,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     e = (flags & EA_Q_PREPROJECTED) ? ea::launch_q_scatter(qp, L.sum_rp_k, h->desc.dtype, s, &h->launches)
                                     : ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
     if (e != cudaSuccess) return cuda_fail(h, e, "prefill q launch");
-  } else if (tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged) {
+  } else if (tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged && h->max_deficit == 0) {
     // Q', K', V' in one tensor-core launch.  Its rows equal eigen_attn_append_kv's except where the two
     // fp32 summation orders round to different bf16 values (one unit in the last place).
     if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
@@ -901,7 +900,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
   }
   p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
-  p.len0 = len0;
+  p.len0 = len0; p.deficit = dev_deficit(h);   // unequal lengths: every sequence's T tokens follow its own rows
   p.max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
   p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);

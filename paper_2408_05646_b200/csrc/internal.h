@@ -149,7 +149,8 @@ struct PrefillParams {
   int64_t out_stride_b, out_stride_t;
   int32_t B, T, H, d_head;
   int32_t n_max;
-  int32_t len0;
+  int32_t len0;             // rows cached before the call (of the longest sequence)
+  const int32_t* deficit;   // [B]: sequence b held len0 - deficit[b] rows before the call; NULL = all held len0
   int32_t max_rp;           // widest padded rank over heads and over K/V
   float scale_log2;         // log2(e) / sqrt(d_head)
   uint32_t flags;

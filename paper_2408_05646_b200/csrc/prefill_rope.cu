@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kThreads) prefill_rope_kernel(const PrefillPar
   extern __shared__ __align__(16) float sm[];
   const int unit = blockIdx.x;
   const int h = unit / p.B, b = unit - h * p.B;
+  const int len0 = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);   // rows this sequence held before the call
   const HeadInfo hd = p.heads[h];
   const int rpk = hd.rp_k, rpv = hd.rp_v, dh = p.d_head, half = dh >> 1, dq = dh >> 2;
   const int cwv = rpv >> 2;
@@ -73,7 +74,7 @@ __global__ void __launch_bounds__(kThreads) prefill_rope_kernel(const PrefillPar
   if (live) {
     const __nv_bfloat16* qg = static_cast<const __nv_bfloat16*>(p.q_raw) + b * p.q_stride_b + t * p.q_stride_t +
                               static_cast<int64_t>(h) * dh;
-    const double pos = static_cast<double>(p.len0 + t);
+    const double pos = static_cast<double>(len0 + t);
 #pragma unroll
     for (int c = 0; c < 32; ++c)
       if (c < dq) {
@@ -88,8 +89,8 @@ __global__ void __launch_bounds__(kThreads) prefill_rope_kernel(const PrefillPar
       }
   }
   float m = -INFINITY, l = 0.f;
-  const int my_last = p.len0 + t;                                      // last key this query sees
-  const int blk_last = p.len0 + min(p.T - 1, qblk * kQRows + kQRows - 1);
+  const int my_last = len0 + t;                                      // last key this query sees
+  const int blk_last = len0 + min(p.T - 1, qblk * kQRows + kQRows - 1);
   const __nv_bfloat16* Kslab = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.k_off);
   const __nv_bfloat16* Vslab = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.v_off);
   const float* U = p.basis + hd.uk_off;                                // U^K: d_head x rp_k, row d = coordinates of e_d

@@ -34,6 +34,7 @@ __global__ void __launch_bounds__(kThreads) prefill_simt_kernel(const PrefillPar
   extern __shared__ __align__(16) float sm[];
   const int unit = blockIdx.x;
   const int h = unit / p.B, b = unit - h * p.B;
+  const int len0 = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);   // rows this sequence held before the call
   const HeadInfo hd = p.heads[h];
   const int rpk = hd.rp_k, rpv = hd.rp_v;
   const int cwk = rpk >> 2, cwv = rpv >> 2;           // rp is a multiple of 8 -> quarters are even
@@ -58,8 +59,8 @@ __global__ void __launch_bounds__(kThreads) prefill_simt_kernel(const PrefillPar
       if (c < cwk) q[c] = to_f<T>(qp[c]) * p.scale_log2;
   }
   float m = -INFINITY, l = 0.f;
-  const int my_last = p.len0 + t;                                      // last key this query sees
-  const int blk_last = p.len0 + min(p.T - 1, qblk * kQRows + kQRows - 1);
+  const int my_last = len0 + t;                                      // last key this query sees
+  const int blk_last = len0 + min(p.T - 1, qblk * kQRows + kQRows - 1);
   const T* Kslab = reinterpret_cast<const T*>(p.cache + hd.k_off);
   const T* Vslab = reinterpret_cast<const T*>(p.cache + hd.v_off);
 

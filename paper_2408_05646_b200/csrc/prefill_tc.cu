@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
   const int tid = threadIdx.x, warp = tid >> 5;
   const int unit = blockIdx.x;
   const int h = unit / p.B, b = unit - h * p.B;
+  const int len0 = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);   // rows this sequence held before the call
   const HeadInfo hd = p.heads[h];
   const int qblk = gridDim.y - 1 - blockIdx.y;              // late (long) query blocks first
   const int t0 = qblk * kTile;
@@ -67,9 +68,9 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
                             static_cast<int64_t>(b) * p.n_max * hd.rp_v;
   load_tile(Qs, Qg, hd.rp_k, q_valid, nch_k, tid);
 
-  const int my_pos = p.len0 + t0 + tid;                      // last key this thread's query sees
+  const int my_pos = len0 + t0 + tid;                      // last key this thread's query sees
   const float slope2 = hd.alibi_slope2;                      // ALiBi: slope * (key - query position), log2 domain
-  const int n_keys = p.len0 + min(p.T, t0 + kTile);          // keys the block needs
+  const int n_keys = len0 + min(p.T, t0 + kTile);          // keys the block needs
   const int n_tiles = (n_keys + kTile - 1) / kTile;
   const uint32_t idesc_s = instr_desc(kTile, false);
   const uint32_t idesc_o = instr_desc(rpv16, true);
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(kThreads) prefill_tc_kernel(const PrefillParam
     if (__syncthreads_or(!ok)) { ok = false; break; }
 
     // ---- softmax of this thread's row: pass 1 = max, pass 2 = exponentials, sum and P
-    const bool diag = key0 + kTile - 1 > p.len0 + t0;        // some (row, key) pair of the tile is masked
+    const bool diag = key0 + kTile - 1 > len0 + t0;        // some (row, key) pair of the tile is masked
     float row_max = -INFINITY;
 #pragma unroll 1
     for (int c0 = 0; c0 < kTile; c0 += 16) {

@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int h = unit / p.B, b = unit - h * p.B;
   const HeadInfo hd = p.heads[h];
   const int qblk = gridDim.y - 1 - blockIdx.y;              // late (long) query blocks first
+  const int len0 = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);   // rows this sequence held before the call
   const int t0 = qblk * 2 * kTile;
   const int rpk16 = (hd.rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
   const int nch_k = rpk16 >> 3, nch_v = rpv16 >> 3;
@@ -138,7 +139,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   int n_tiles[2];
   for (int x = 0; x < 2; ++x) {
     const int tx = t0 + x * kTile;
-    n_tiles[x] = tx < p.T ? (p.len0 + min(p.T, tx + kTile) + kKeys - 1) / kKeys : 0;
+    n_tiles[x] = tx < p.T ? (len0 + min(p.T, tx + kTile) + kKeys - 1) / kKeys : 0;
   }
   const int n_max_tiles = max(n_tiles[0], n_tiles[1]);
   const int active_groups = (n_tiles[0] > 0) + (n_tiles[1] > 0);
@@ -319,7 +320,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     const uint32_t tS = tmem + lane_base + x * kTile;        // S buffers at +0 and +64
     const uint32_t tO = tmem + lane_base + 256 + x * kTile;
     const int tx = t0 + x * kTile;
-    const int my_pos = p.len0 + tx + row;                    // last key this thread's query sees
+    const int my_pos = len0 + tx + row;                    // last key this thread's query sees
     {                                                        // this tile's Q' (zeros past the prompt's end)
       const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.qp) +
                                 static_cast<int64_t>(hd.lr_k_off) * total_rows + static_cast<int64_t>(b) * p.T * hd.rp_k;
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
       const int key0 = j * kKeys + hf * kHalfKeys;           // first key of this thread's half
       const uint32_t tSb = tS + buf * kKeys;
       const bool waited = mbar_wait(&hdr->s_full[x][buf], (j >> 1) & 1u, p.status);
-      const bool diag = j * kKeys + kKeys - 1 > p.len0 + tx; // some (row, key) pair of the tile is masked
+      const bool diag = j * kKeys + kKeys - 1 > len0 + tx; // some (row, key) pair of the tile is masked
       uint32_t r[kHalfKeys];
       float cand = -INFINITY;                                // this half-row's largest score, scaled (log2 domain)
       if (waited) {

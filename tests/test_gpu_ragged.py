@@ -42,6 +42,11 @@ class PerSequenceOracle:
             for b, r in enumerate(group):
                 r.append_kv(to_np(k[b:b + 1]), to_np(v[b:b + 1]))
 
+    def prefill(self, q, k, v):                   # q, k, v: [B, T, H, d] -> [B, T, H, d]; the rows are appended
+        one = lambda group: np.concatenate([r.prefill_dense(to_np(q[b:b + 1]), to_np(k[b:b + 1]), to_np(v[b:b + 1]))
+                                            for b, r in enumerate(group)], axis=0)
+        return Expect(one(self.refs), one(self.plain)) if self.plain else one(self.refs)
+
     def decode(self, q):                          # q: [B, 1, H, d] -> [B, 1, H, d]
         one = lambda group: np.concatenate([r.decode_dense(to_np(q[b:b + 1])).reshape(1, 1, self.H, self.d)
                                             for b, r in enumerate(group)], axis=0)
@@ -96,9 +101,6 @@ def test_sequence_with_no_rows_and_return_to_equal_lengths(B):
     with pytest.raises(B.EigenAttnError) as e:    # a sequence without rows has nothing to attend
         lay.decode(q[:, :1])
     assert e.value.status == B.EA_ERR_SHAPE
-    with pytest.raises(B.EigenAttnError) as e:
-        lay.prefill(q[:, :1].contiguous(), k[:, :1].contiguous(), v[:, :1].contiguous())
-    assert e.value.status == B.EA_ERR_UNSUPPORTED and lay.lens() == lens
     with pytest.raises(B.EigenAttnError) as e:
         lay.set_lens([0, n + 2, 1])
     assert e.value.status == B.EA_ERR_CAPACITY and lay.lens() == lens
@@ -309,4 +311,43 @@ def test_many_sequences_of_unequal_lengths(B):
     o = lay.decode_step(q[:, 1:2], k[:, n:], v[:, n:])
     ref.append(k[:, n:], v[:, n:])
     assert_close(o, ref.decode(q[:, 1:2]), FP32, "decode_step")
+    lay.poll_status()
+
+
+@pytest.mark.parametrize("dtype,d,rk,rv,n,lens,T,variant", [
+    (BF16, 128, [80, 48, 128], [80, 112, 64], 600, [600, 129, 0, 471], 300, "plain"),     # warp-specialised tcgen05 kernel
+    (BF16, 128, [80, 80, 80], [80, 80, 80], 300, [5, 300, 299, 64], 130, "alibi"),
+    (BF16, 128, [80, 64, 48], [64, 80, 96], 260, [260, 1, 77, 130], 70, "rope"),          # Section 4.3 prompt form
+    (FP32, 64, [32, 20, 64], [16, 40, 8], 200, [200, 1, 77, 0], 50, "plain"),             # CUDA-core kernel
+    (BF16, 128, [80, 48, 128], [80, 112, 64], 400, [400, 129, 3, 271], 200, "single-tile"),
+])
+def test_prompt_chunk_behind_sequences_of_unequal_lengths(B, dtype, d, rk, rv, n, lens, T, variant):
+    """A chunk of T prompt tokens for every sequence of a batch whose sequences hold different numbers of rows
+    (continuous batching: chunked prompts of some sequences beside others further along): token t of sequence b
+    sits at position lens[b] + t and sees that sequence's own rows only.  Then a generated token on top."""
+    B_, H = 4, 3
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + T + 1, dtype, seed_cfg=148, T_q=n + T + 1)
+    if dtype == BF16:
+        q = (q.float() * 0.25).to(dtype)                              # Q' is kept in 16 bits by the prompt kernels
+    lay = B.EigenAttnLayer(B_, H, d, n + T + 1, dtype, U_k, U_v, max_prefill_tokens=T)
+    slopes = [0.5, 0.0625, 0.25] if variant == "alibi" else None
+    rope = {"base": 10000.0, "interleaved": False} if variant == "rope" else None
+    if slopes:
+        lay.set_alibi(slopes)
+    if rope:
+        lay.set_rope(rope["base"], rope["interleaved"])
+    if variant == "single-tile":
+        lay.set_option(B.EA_OPT_PREFILL_IMPL, 3)
+    lay.append_kv(k[:, :n], v[:, :n])              # every sequence holds n rows; each keeps its first lens[b]
+    lay.set_lens(lens)
+    ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens, alibi_slopes=slopes, storage=storage_model(dtype), rope=rope)
+    # the chunk of sequence b: rows n .. n + T - 1 of the drawn tensors (any rows would do)
+    qc, kc, vc = (x[:, n:n + T].contiguous() for x in (q, k, v))
+    out = lay.prefill(qc, kc, vc)
+    assert_close(out, ref.prefill(qc, kc, vc), dtype, f"prompt chunk ({variant})")
+    assert lay.lens() == [x + T for x in lens]
+    qn, kn, vn = (x[:, n + T:n + T + 1] for x in (q, k, v))
+    o = lay.decode_step(qn, kn, vn)
+    ref.append(kn, vn)
+    assert_close(o, ref.decode(qn), dtype, f"generated token after the chunk ({variant})")
     lay.poll_status()
