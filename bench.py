@@ -657,6 +657,10 @@ def workload_table_own_layers(device, binding, steps=30, warmup=3):
     k_us, s_us = timed_kernel(lay, device, step_paged, steps, warmup)
     table["paged_cache"] = table_entry("decode_splitkv_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
                                        workload=wl.name + ", page table with pages of 128 rows shuffled over the pool")
+    lay.set_rope(10000.0)                                  # the same paged layer as a layer with rotary embedding
+    k_us, s_us = timed_kernel(lay, device, step_paged, steps, warmup)
+    table["paged_cache[rope]"] = table_entry("decode_rope_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1),
+                                             peak, workload=wl.name + ", rotary embedding, pages of 128 rows shuffled over the pool")
     del lay
     torch.cuda.empty_cache()
     for b in (1, 2):

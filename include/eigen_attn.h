@@ -272,8 +272,10 @@ ea_status eigen_attn_get_lens(eigen_attn_t h, int32_t* lens);
  * rows are whatever its pages hold (the identity table h_table[b][i] = b * (n_max / page_rows) + i keeps a
  * contiguous cache as it is, when page_rows divides n_max).  NULL returns to the contiguous layout.
  * Available for eigen_attn_append_kv, _decode, _decode_step(_host), _decode_static, _set_len(s), and
- * eigen_attn_prefill (which then runs on the CUDA cores); not (EA_ERR_UNSUPPORTED) with a rotary embedding, a
- * quantised cache or eigen_attn_decode_gqa.  batch * pages_per_seq entries must fit the table area of the workspace
+ * eigen_attn_prefill (which then runs on the CUDA cores), and with a rotary embedding for all of these and for
+ * eigen_attn_decode_gqa when page_rows divides n_max (a page then lies inside one sequence's slab, which the tiled
+ * copies of the rotary decode kernel need); not (EA_ERR_UNSUPPORTED) with a quantised cache, nor
+ * eigen_attn_decode_gqa without a rotary embedding.  batch * pages_per_seq entries must fit the table area of the workspace
  * (batch * batch * n_max / 128 entries, at most 4 Mi).  Uploaded on the stream (asynchronous; the array may be reused
  * when the call returns): later calls must run on that stream or be ordered after it. */
 ea_status eigen_attn_set_page_table(eigen_attn_t h, const int32_t* h_table, int32_t pages_per_seq, int32_t page_rows,

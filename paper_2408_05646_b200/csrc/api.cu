@@ -457,7 +457,9 @@ ea_status launch_plan(eigen_attn_t h, const char* who, const DecodePlan& plan, b
 ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void* d_out, int64_t stride_b_out,
                          uint32_t flags, cudaStream_t s, int group = 1) {
   if (!d_q || !d_out) return fail(h, EA_ERR_INVALID_ARG, "decode: NULL q or out");
-  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding: not available with a page table");
+  if (h->paged && h->desc.n_max % (1 << h->page_shift) != 0)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode with rotary embedding and a page table: page_rows %d must divide n_max %d",
+                1 << h->page_shift, h->desc.n_max);
   if (flags & ~EA_OUT_LOWRANK)
     return fail(h, EA_ERR_INVALID_ARG, "decode with rotary embedding: flag 0x%x (the query must be full rank)", flags);
   if (h->len < 1) return fail(h, EA_ERR_SHAPE, "decode: the cache is empty");
@@ -507,6 +509,7 @@ ea_status do_decode_rope(eigen_attn_t h, const void* d_q, int64_t stride_b, void
   p.group = group;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
+  p.pages = dev_pages(h);
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
   const cudaError_t e = ea::launch_decode_rope(p, smem, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
@@ -1005,7 +1008,7 @@ ea_status eigen_attn_set_page_table(eigen_attn_t h, const int32_t* h_table, int3
     h->paged = false;
     return EA_OK;
   }
-  if (h->rope || h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_page_table: not available with a rotary embedding or a quantised cache");
+  if (h->q_group) return fail(h, EA_ERR_UNSUPPORTED, "set_page_table: not available with a quantised cache");
   if (page_rows < 128 || (page_rows & (page_rows - 1)) != 0)
     return fail(h, EA_ERR_SHAPE, "set_page_table: page_rows %d (a power of two, at least 128)", page_rows);
   const int64_t pool = static_cast<int64_t>(B) * h->desc.n_max / page_rows;      // physical pages of a head's slab
@@ -1118,11 +1121,11 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
   if (h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with an ALiBi bias set");
-  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table");
   if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty (for some sequence)");
   // Section 4.3 for a group: every query head of the group is a unit of the rotary kernel over its K/V head's rows
   if (h->rope)
     return do_decode_rope(h, d_q, stride_b_q, d_out, stride_b_out, 0u, static_cast<cudaStream_t>(cuda_stream), group);
+  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table (without a rotary embedding)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   const size_t smem = ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
@@ -1178,7 +1181,6 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
   if (h->desc.dtype != EA_BF16 || h->desc.d_head % 16 || !h->tmaps_ok)
     return fail(h, EA_ERR_UNSUPPORTED, "set_rope: needs a bf16 layer with d_head %% 16 == 0 (and the driver's tensor-map encoder)");
   if (h->alibi) return fail(h, EA_ERR_INVALID_ARG, "set_rope: the layer has an ALiBi bias");
-  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "set_rope: not available with a page table");
   const int dh = h->desc.d_head;
   // the constants the kernels read: the inverse frequencies phi_i, e^{-i 128 phi_i} (one tile of cached rows back)
   // and e^{i l phi_i} for the 128 row offsets of a tile, worked out here in double precision

@@ -64,7 +64,8 @@ __host__ __device__ constexpr int rope_kb(int bytes) { return (bytes + 1023) & ~
 
 // HALF = d_head / 2 known at compile time (64: the usual head of 128 dimensions; no chunk of pairs is ever empty
 // and the TMEM columns are constants), or 0: taken from the launch parameters.
-template <bool INTERLEAVED, int HALF>
+// PAGED: the tiles' addresses come through a page table.
+template <bool INTERLEAVED, int HALF, bool PAGED>
 __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const RopeDecodeParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   RopeSmemHeader* hdr = reinterpret_cast<RopeSmemHeader*>(smem);
@@ -171,20 +172,28 @@ __global__ void __launch_bounds__(kRopeThreads, 2) decode_rope_kernel(const Rope
   // K' tile i into buffer i & 1: two boxes of 64 rows per atom column, in the layout the lift's A operand names (no
   // thread moves the tile); elements past the rank and rows past the capacity arrive as zeros, rows between the
   // sequence's length and the capacity are finite (the cache starts as zeros) and meet zero weights
+  // With a page table the tile's rows are where the table says: a page holds whole tiles and lies inside one
+  // sequence's slab, so the tile is still two boxes of the slab's tensor map and one contiguous run of V' rows.
   auto fetch_k = [&](int i) {
     const int buf = i & 1, t = t_lo + i;
+    int row0 = t * kTile, slab = b;
+    if (PAGED) {
+      const int64_t prow = physical_row(p.pages, b, p.n_max, row0);
+      slab = static_cast<int>(prow / p.n_max);
+      row0 = static_cast<int>(prow - static_cast<int64_t>(slab) * p.n_max);
+    }
     mbar_arrive_expect_tx(&hdr->k_full[buf], static_cast<uint32_t>(kt_bytes));
     for (int a = 0; a < ak; ++a)
       for (int hh = 0; hh < 2; ++hh)
-        tma_load_3d(Kt + buf * kt_bytes + a * kRopeAtom + hh * (kRopeAtom / 2), map_k, a * 64, t * kTile + hh * 64, b,
+        tma_load_3d(Kt + buf * kt_bytes + a * kRopeAtom + hh * (kRopeAtom / 2), map_k, a * 64, row0 + hh * 64, slab,
                     &hdr->k_full[buf]);
   };
   auto fetch_v = [&](int i) {
     const int t = t_lo + i;
     const uint32_t bytes = static_cast<uint32_t>(min(kTile, n_b - t * kTile)) * rowb_v;
     mbar_arrive_expect_tx(&hdr->v_full, bytes);
-    bulk_load(Vs, p.cache + hd.v_off + (static_cast<int64_t>(b) * p.n_max + static_cast<int64_t>(t) * kTile) * rowb_v, bytes,
-              &hdr->v_full, policy);
+    const int64_t prow = PAGED ? physical_row(p.pages, b, p.n_max, t * kTile) : static_cast<int64_t>(b) * p.n_max + t * kTile;
+    bulk_load(Vs, p.cache + hd.v_off + prow * rowb_v, bytes, &hdr->v_full, policy);
   };
   // X(i) = K'(i) (U^K)^T into accumulator i & 1, once the tile's rows have landed; false if that wait gave up
   auto issue_lift = [&](int i) -> bool {
@@ -439,16 +448,26 @@ size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head) {
 }
 
 cudaError_t launch_decode_rope(const RopeDecodeParams& p, size_t smem, cudaStream_t s, uint64_t* launches) {
-  static size_t configured[4][kMaxDevices] = {};
+  static size_t configured[8][kMaxDevices] = {};
   auto run = [&](auto kernel, size_t (&done)[kMaxDevices]) -> cudaError_t {
     const cudaError_t ec = ensure_dynamic_smem(kernel, smem, done);
     if (ec != cudaSuccess) return ec;
     kernel<<<dim3(p.B * p.H * p.group, p.splits), kRopeThreads, smem, s>>>(p);
     return cudaGetLastError();
   };
+  const bool paged = p.pages.table != nullptr, wide = p.d_head == 128, inter = p.interleaved != 0;
+  const int which = (paged ? 4 : 0) + (wide ? 2 : 0) + (inter ? 1 : 0);
   cudaError_t e;
-  if (p.d_head == 128) e = p.interleaved ? run(decode_rope_kernel<true, 64>, configured[3]) : run(decode_rope_kernel<false, 64>, configured[2]);
-  else e = p.interleaved ? run(decode_rope_kernel<true, 0>, configured[1]) : run(decode_rope_kernel<false, 0>, configured[0]);
+  switch (which) {
+    case 0: e = run(decode_rope_kernel<false, 0, false>, configured[0]); break;
+    case 1: e = run(decode_rope_kernel<true, 0, false>, configured[1]); break;
+    case 2: e = run(decode_rope_kernel<false, 64, false>, configured[2]); break;
+    case 3: e = run(decode_rope_kernel<true, 64, false>, configured[3]); break;
+    case 4: e = run(decode_rope_kernel<false, 0, true>, configured[4]); break;
+    case 5: e = run(decode_rope_kernel<true, 0, true>, configured[5]); break;
+    case 6: e = run(decode_rope_kernel<false, 64, true>, configured[6]); break;
+    default: e = run(decode_rope_kernel<true, 64, true>, configured[7]); break;
+  }
   ++*launches;
   if (e != cudaSuccess) return e;
   rope_combine_kernel<<<p.B * p.H * p.group, 128, 0, s>>>(p);

@@ -188,6 +188,7 @@ struct RopeDecodeParams {    // decode for models with rotary position embedding
   int32_t group;            // query heads per K/V head (1: every head has its own rows); q and out have H * group heads
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
+  PageMap pages;            // paged cache: a tile of 128 rows lies inside one page; pages lie inside one sequence's slab
 };
 
 struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` query heads per K/V head

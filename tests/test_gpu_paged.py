@@ -7,6 +7,7 @@ import torch
 
 from helpers import OraclePair, assert_close, make_case, oracle_layer, to_np
 from oracle import eigen_attention as orc
+from paper_2408_05646_b200 import synth
 
 pytestmark = pytest.mark.gpu
 BF16, FP32 = torch.bfloat16, torch.float32
@@ -129,9 +130,6 @@ def test_page_table_argument_checks(B):
     lay.set_page_table([[2, 3], [0, 1]], 128)
     lay.append_kv(k, v)
     with pytest.raises(B.EigenAttnError) as e:
-        lay.set_rope(10000.0)
-    assert e.value.status == B.EA_ERR_UNSUPPORTED
-    with pytest.raises(B.EigenAttnError) as e:
         lay.quant_attach(4, 32)
     assert e.value.status == B.EA_ERR_UNSUPPORTED
     with pytest.raises(B.EigenAttnError) as e:
@@ -142,3 +140,56 @@ def test_page_table_argument_checks(B):
     assert e.value.status == B.EA_ERR_CAPACITY
     lay.set_page_table(None)                           # contiguous again
     lay.poll_status()
+
+
+@pytest.mark.parametrize("interleaved", [False, True])
+def test_paged_layer_with_rotary_embedding_equals_contiguous_layer(B, interleaved):
+    """Section 4.3 over a paged cache: prompt, generation steps and grouped queries of a paged layer equal those of
+    the contiguous layer bit for bit (same kernels, same tiles, other addresses) and both agree with the oracle."""
+    B_, H, d, n_max, page_rows = 3, 3, 128, 1024, 256
+    rk, rv = [80, 48, 112], [64, 96, 80]
+    n, steps, g = 700, 2, 2
+    U_k, U_v, qq, k, v = make_case(B_, H, d, rk, rv, n + steps, BF16, seed_cfg=187, T_q=200 + steps + 1)
+    q_prompt, q = (qq[:, :200].float() / 4.0).to(BF16), qq[:, 200:]
+    rope = {"base": 10000.0, "interleaved": interleaved}
+    flat = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v, max_prefill_tokens=200)
+    paged = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v, max_prefill_tokens=200)
+    per_seq = n_max // page_rows
+    perm = np.random.default_rng(7).permutation(B_ * per_seq)
+    paged.set_page_table([[int(x) for x in perm[b * per_seq:(b + 1) * per_seq]] for b in range(B_)], page_rows)
+    ref = OraclePair(B_, H, d, U_k, U_v, BF16, rope=rope)
+    outs = []
+    for lay in (flat, paged):
+        lay.set_rope(rope["base"], interleaved)
+        outs.append(lay.prefill(q_prompt, k[:, :200].contiguous(), v[:, :200].contiguous()))
+        lay.append_kv(k[:, 200:n], v[:, 200:n])
+    assert torch.equal(outs[0], outs[1])
+    assert_close(outs[1], ref.prefill_dense(to_np(q_prompt), to_np(k[:, :200]), to_np(v[:, :200])), BF16, "rope prefill, paged")
+    ref.append_kv(to_np(k[:, 200:n]), to_np(v[:, 200:n]))
+    for ctas in (0, 1, 5):
+        for lay in (flat, paged):
+            lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        want = flat.decode(q[:, :1])
+        assert torch.equal(paged.decode(q[:, :1]), want), f"paged rope decode differs, ctas={ctas}"
+        assert_close(want, ref.decode_dense(to_np(q[:, :1])), BF16, f"rope decode ctas={ctas}")
+    W_q = synth.mixing_matrices(H * g, 16, d, 188, "W_Q")
+    qg = synth.lowrank_rows(W_q, B_, 1, 0.1, 188, "Q", dtype=BF16, device="cuda:0")
+    want = flat.decode_gqa(qg, g)
+    assert torch.equal(paged.decode_gqa(qg, g), want)
+    assert_close(want, ref.decode_gqa(to_np(qg), g), BF16, "grouped queries, rope, paged")
+    for s in range(steps):
+        t = n + s
+        o_f = flat.decode_step(q[:, s + 1:s + 2], k[:, t:t + 1], v[:, t:t + 1])
+        o_p = paged.decode_step(q[:, s + 1:s + 2], k[:, t:t + 1], v[:, t:t + 1])
+        ref.append_kv(to_np(k[:, t:t + 1]), to_np(v[:, t:t + 1]))
+        assert torch.equal(o_p, o_f), f"paged rope decode_step {s} differs"
+        assert_close(o_p, ref.decode_dense(to_np(q[:, s + 1:s + 2])), BF16, f"paged rope decode_step {s}")
+    paged.poll_status(); flat.poll_status()
+    # pages that straddle two sequences' slabs cannot be addressed by the rotary kernel's tiled copies
+    odd = B.EigenAttnLayer(2, 1, 128, 384, BF16, [U_k[0]], [U_v[0]])
+    odd.set_page_table([[0, 2], [1, -1]], 256)
+    odd.set_rope(10000.0)
+    odd.append_kv(k[:2, :8, :1].contiguous(), v[:2, :8, :1].contiguous())
+    with pytest.raises(B.EigenAttnError) as e:
+        odd.decode(q[:2, :1, :1].contiguous())
+    assert e.value.status == B.EA_ERR_UNSUPPORTED
