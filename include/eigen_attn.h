@@ -55,6 +55,10 @@ typedef enum { EA_BF16 = 0, EA_FP32 = 1 } ea_dtype;   /* cache + IO dtype; accum
 
 /* ea_desc.flags */
 #define EA_CHECK_ORTHONORMAL 0x1u   /* verify U^T U = I on the host at create (Section 4.2 assumes it) */
+#define EA_ROPE_PROMPT_SCRATCH 0x2u /* the workspace also holds the prompt's rotated full-rank queries and lifted,
+                                       rotated keys (2 * batch * max_prefill_tokens * n_heads * d_head 16-bit values):
+                                       eigen_attn_prefill of a layer with rotary embedding then runs on the tensor
+                                       cores while the rows cached after the call fit max_prefill_tokens */
 
 /* per-call flags */
 #define EA_Q_PREPROJECTED  0x1u  /* d_q already holds q U^K (merged W^Q', Eq. 8): [B][T][sum_h rp_k[h]]      */

@@ -20,6 +20,7 @@ EA_ERR_INVALID_ARG, EA_ERR_SHAPE, EA_ERR_CAPACITY, EA_ERR_UNSUPPORTED = -1, -2, 
 EA_ERR_CUDA, EA_ERR_TIMEOUT, EA_ERR_NOT_ORTHONORMAL = -5, -6, -7
 EA_BF16, EA_FP32 = 0, 1
 EA_CHECK_ORTHONORMAL = 0x1
+EA_ROPE_PROMPT_SCRATCH = 0x2
 EA_Q_PREPROJECTED, EA_OUT_LOWRANK, EA_KV_PREPROJECTED = 0x1, 0x2, 0x4
 EA_OPT_DECODE_CTAS, EA_OPT_DECODE_TILE_ROWS, EA_OPT_DECODE_STAGES, EA_OPT_PREFILL_IMPL = 1, 2, 3, 4
 EA_OPT_DECODE_FUSED = 5
@@ -153,7 +154,7 @@ class EigenAttnLayer:
     def __init__(self, batch: int, n_heads: int, d_head: int, n_max: int, dtype: torch.dtype,
                  U_k: Sequence[np.ndarray], U_v: Sequence[np.ndarray], max_prefill_tokens: int = 0,
                  device: str | torch.device = "cuda:0", check_orthonormal: bool = False,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, rope_prompt_scratch: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("EigenAttnLayer needs a CUDA device; there is no CPU fallback")
         self.B, self.H, self.d_head, self.n_max = batch, n_heads, d_head, n_max
@@ -165,7 +166,8 @@ class EigenAttnLayer:
         for u in list(U_k) + list(U_v):
             assert u.shape[0] == d_head
         desc, keep = _make_desc(batch, n_heads, d_head, n_max, self.ea_dtype, self.r_k, self.r_v, U_k, U_v,
-                                max_prefill_tokens, EA_CHECK_ORTHONORMAL if check_orthonormal else 0)
+                                max_prefill_tokens, (EA_CHECK_ORTHONORMAL if check_orthonormal else 0) |
+                                (EA_ROPE_PROMPT_SCRATCH if rope_prompt_scratch else 0))
         cb, wb = _sz(0), _sz(0)
         st = lib.eigen_attn_cache_bytes(ctypes.byref(desc), ctypes.byref(cb), ctypes.byref(wb))
         if st != EA_OK:

@@ -44,7 +44,8 @@ struct Layout {
   std::vector<HeadInfo> heads;
   size_t cache_bytes = 0;
   // workspace
-  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0, off_qlens = 0, off_pages = 0;
+  size_t off_status = 0, off_heads = 0, off_basis = 0, off_partials = 0, off_counters = 0, off_staging = 0, off_qp = 0, off_tmaps = 0, off_rope = 0, off_deficit = 0, off_qlens = 0, off_pages = 0, off_krot = 0, off_tmaps_krot = 0;
+  bool rope_scratch = false;   // the workspace holds the rotated queries and lifted keys of a prompt (EA_ROPE_PROMPT_SCRATCH)
   size_t page_entries = 0;   // capacity of the page-table area, in entries
   size_t basis_floats = 0, staging_each = 0, workspace_bytes = 0;
   int sum_rp_k = 0, sum_rp_v = 0, max_rp_k = 0, max_rp_v = 0, max_w = 0;
@@ -115,7 +116,16 @@ void make_layout(const ea_desc* d, Layout* L) {
   L->off_counters = off; off = align_up(off + static_cast<size_t>(d->batch) * H * sizeof(int));
   L->staging_each = align_up(static_cast<size_t>(d->batch) * H * dh * L->es);
   L->off_staging = off;  off += 4 * L->staging_each;
-  L->off_qp = off;       off = align_up(off + static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es);
+  // Q' of a prompt call; with EA_ROPE_PROMPT_SCRATCH at least the rotated full-rank queries, and behind them the
+  // lifted, rotated keys of up to max_prefill_tokens rows per sequence ([H][B][max_prefill_tokens][d_head], 16-bit)
+  const bool rope_scratch = (d->flags & EA_ROPE_PROMPT_SCRATCH) != 0 && d->dtype == EA_BF16 && dh % 16 == 0;
+  size_t qp_bytes = static_cast<size_t>(d->batch) * d->max_prefill_tokens * lk * L->es;
+  const size_t rot_bytes = static_cast<size_t>(d->batch) * d->max_prefill_tokens * H * dh * 2;
+  if (rope_scratch && rot_bytes > qp_bytes) qp_bytes = rot_bytes;
+  L->off_qp = off;       off = align_up(off + qp_bytes);
+  L->off_krot = off;     off = align_up(off + (rope_scratch ? rot_bytes : 0));
+  L->off_tmaps_krot = off; off = align_up(off + (rope_scratch ? static_cast<size_t>(H) * sizeof(CUtensorMap) : 0));
+  L->rope_scratch = rope_scratch && d->max_prefill_tokens >= 1;
   L->off_rope = off;     off = align_up(off + ea::kRopeConstBytes);   // constants of the rotary embedding
   L->off_tmaps = off;    off = align_up(off + 2 * static_cast<size_t>(H) * sizeof(CUtensorMap));   // K', V' per head
   L->off_deficit = off;  off = align_up(off + static_cast<size_t>(d->batch) * sizeof(int32_t));   // unequal lengths
@@ -161,6 +171,33 @@ bool encode_tensor_maps(const ea_desc* d, const Layout& L, char* cache, std::vec
   return true;
 }
 
+// Tensor maps of the lifted, rotated keys a prompt call of a layer with rotary embedding keeps in the workspace:
+// per head a 3-D view {d_head (inner), max_prefill_tokens rows, batch} of bf16, boxes as for the cache slabs.
+bool encode_krot_maps(const ea_desc* d, char* base, std::vector<CUtensorMap>* maps) {
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return false;
+  const EncodeFn encode = reinterpret_cast<EncodeFn>(fn);
+  const cuuint64_t dh = d->d_head, R = d->max_prefill_tokens, B = d->batch;
+  maps->resize(d->n_heads);
+  for (int h = 0; h < d->n_heads; ++h) {
+    const cuuint64_t dims[3] = {dh, R, B};
+    const cuuint64_t strides[2] = {dh * 2, R * dh * 2};
+    const cuuint32_t box[3] = {64, 64, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (encode(&(*maps)[h], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base + static_cast<size_t>(h) * B * R * dh * 2, dims, strides,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  return true;
+}
+
 // Tensor maps of the q, k, v tensors of one prefill call for the streaming projection kernel: a 3-D view
 // {n_heads * d_head (inner), T tokens, batch} of bf16, box = 64 elements x 128 tokens with the 128-byte
 // swizzle; tokens past T read as zero.  Encoded on the host per call (the pointers are the caller's).
@@ -202,6 +239,7 @@ struct eigen_attn {
   int32_t max_deficit = 0;        // > 0: the batch has unequal lengths and the workspace holds `deficit`
   int sm_count = 148;
   bool tmaps_ok = false;  // the workspace holds tensor maps of the cache slabs
+  bool krot_ok = false;   // ... and the scratch + tensor maps of a rotary layer's prompt on the tensor cores
   bool alibi = false;     // some head has a non-zero ALiBi slope
   bool rope = false;      // decode follows Section 4.3 (rotary position embedding)
   int rope_interleaved = 0;
@@ -680,6 +718,13 @@ ea_status eigen_attn_create(const ea_desc* desc, void* d_cache, size_t cache_byt
       encode_tensor_maps(desc, L, h->cache, &tmaps)) {
     e = cudaMemcpyAsync(h->ws + L.off_tmaps, tmaps.data(), tmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s);
     h->tmaps_ok = true;
+    std::vector<CUtensorMap> kmaps;
+    if (e == cudaSuccess && L.rope_scratch && encode_krot_maps(desc, h->ws + L.off_krot, &kmaps)) {
+      e = cudaMemcpyAsync(h->ws + L.off_tmaps_krot, kmaps.data(), kmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s);
+      // rows the first prompt does not write are read by whole key tiles and must be finite
+      if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + L.off_krot, 0, L.off_tmaps_krot - L.off_krot, s);
+      h->krot_ok = true;
+    }
   }
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   int dev = 0;
@@ -812,51 +857,11 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
   const bool tc_attn = tc_shape && out_aligned && !h->paged;    // the tensor-core kernels address contiguous slabs
   if (h->opt_prefill == 2 && !tc_attn)
     return fail(h, EA_ERR_UNSUPPORTED, "prefill: the tcgen05 kernel needs bf16, d_head %% 16 == 0 and 16-byte aligned output rows");
-  cudaError_t e;
-  if (h->rope) {
-    // Section 4.3 for the prompt: the cache takes the projections of the un-rotated keys, as in the generation
-    // phase; the attention kernel lifts and rotates them and rotates the full-rank queries itself.
-    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
-    if (st != EA_OK) return st;
-    ea::PrefillParams p{};
-    p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache; p.out = d_out;
-    if (flags & EA_OUT_LOWRANK) {
-      p.out_stride_t = L.sum_rp_v;
-      p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
-    } else {
-      p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
-    }
-    p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
-    p.len0 = len0; p.deficit = dev_deficit(h);
-    p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
-    p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
-    p.pages = dev_pages(h);
-    p.q_raw = d_q; p.q_stride_b = stride_b; p.q_stride_t = stride_t;
-    p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
-    p.rope_interleaved = h->rope_interleaved;
-    if (h->ev_start) cudaEventRecord(h->ev_start, s);
-    e = ea::launch_prefill_rope(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
-    if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
-    if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch (rotary embedding)");
-    return EA_OK;
-  }
-  if (merged_in) {
-    // Rank-space rows from merged weights (Eq. 8): nothing to multiply.  K', V' rows are copied into the cache, Q'
-    // rows into the per-head layout the attention kernels read; a tensor the caller left d_head-wide is projected
-    // on the CUDA cores.
-    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
-    if (st != EA_OK) return st;
-    ea::QProjectParams qp{};
-    qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
-    qp.stride_b = stride_b; qp.stride_t = stride_t;
-    qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
-    e = (flags & EA_Q_PREPROJECTED) ? ea::launch_q_scatter(qp, L.sum_rp_k, h->desc.dtype, s, &h->launches)
-                                    : ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
-    if (e != cudaSuccess) return cuda_fail(h, e, "prefill q launch");
-  } else if (tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged && h->max_deficit == 0) {
-    // Q', K', V' in one tensor-core launch.  Its rows equal eigen_attn_append_kv's except where the two
-    // fp32 summation orders round to different bf16 values (one unit in the last place).
-    if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
+  // Q', K', V' of the call's tokens in one tensor-core launch (K', V' into the cache, Q' into the workspace).  Its
+  // rows equal eigen_attn_append_kv's except where the two fp32 summation orders round to different bf16 values
+  // (one unit in the last place).
+  const bool tc_project = tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged && h->max_deficit == 0 && d_k && d_v;
+  auto project_on_tensor_cores = [&]() -> ea_status {
     if (static_cast<int64_t>(len0) + T > h->desc.n_max)
       return fail(h, EA_ERR_CAPACITY, "prefill: len %d + T %d exceeds n_max %d", len0, T, h->desc.n_max);
     ea::ProjectTcParams pp{};
@@ -877,13 +882,88 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
       stream = ps_stages >= 2 && encode_input_maps(in_ptrs, h->desc.n_heads, h->desc.d_head, T, h->desc.batch,
                                                    stride_b, stride_t, in_maps);
     }
-    if (stream)
-      e = ea::launch_project_tc_stream(pp, in_maps, max_rp, h->opt_project >= 2 ? static_cast<int>(h->opt_project) : h->sm_count,
-                                       s, &h->launches);
-    else
-      e = ea::launch_project_tc(pp, max_rp, s, &h->launches);
-    if (e != cudaSuccess) return cuda_fail(h, e, "prefill projection launch");
+    const cudaError_t ep =
+        stream ? ea::launch_project_tc_stream(pp, in_maps, max_rp, h->opt_project >= 2 ? static_cast<int>(h->opt_project) : h->sm_count,
+                                              s, &h->launches)
+               : ea::launch_project_tc(pp, max_rp, s, &h->launches);
+    if (ep != cudaSuccess) return cuda_fail(h, ep, "prefill projection launch");
     h->len += T;
+    return EA_OK;
+  };
+  cudaError_t e;
+  if (h->rope) {
+    // Section 4.3 for the prompt: the cache takes the projections of the un-rotated keys, as in the generation
+    // phase; the attention kernel lifts and rotates them and rotates the full-rank queries itself.
+    // On the tensor cores when the layer was created with the scratch for it and the rows cached after the call fit
+    // it: the rotated queries and the lifted, rotated keys are written out once, then the warp-specialised kernel
+    // runs an ordinary causal product over d_head-wide rows with the rank-r values of the cache.
+    size_t ws_smem = 0;
+    const int dh = h->desc.d_head;
+    const int ws_stages = h->krot_ok && tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 &&
+                                  static_cast<int64_t>(len0) + T <= h->desc.max_prefill_tokens
+                              ? ea::prefill_tc_ws_stages(dh, L.max_rp_v, dh, &ws_smem) : 0;
+    if (h->opt_prefill == 2 && ws_stages < 3)
+      return fail(h, EA_ERR_UNSUPPORTED, "prefill with rotary embedding: the tcgen05 kernel needs EA_ROPE_PROMPT_SCRATCH at create, "
+                                         "16-byte aligned output rows, no page table and len + T <= max_prefill_tokens");
+    // the tokens' rows: on the tensor cores when the attention runs there too (the Q' that launch also writes is
+    // not used: the rotated full-rank queries take its place in the workspace)
+    const ea_status st = ws_stages >= 3 && tc_project && !(flags & EA_KV_PREPROJECTED)
+                             ? project_on_tensor_cores()
+                             : do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
+    if (st != EA_OK) return st;
+    ea::PrefillParams p{};
+    p.heads = dev_heads(h); p.basis = dev_basis(h); p.cache = h->cache; p.out = d_out;
+    if (flags & EA_OUT_LOWRANK) {
+      p.out_stride_t = L.sum_rp_v;
+      p.out_stride_b = static_cast<int64_t>(T) * L.sum_rp_v;
+    } else {
+      p.out_stride_b = out_stride_b; p.out_stride_t = out_stride_t;
+    }
+    p.B = h->desc.batch; p.T = T; p.H = h->desc.n_heads; p.d_head = h->desc.d_head; p.n_max = h->desc.n_max;
+    p.len0 = len0; p.deficit = dev_deficit(h);
+    p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
+    p.flags = flags & EA_OUT_LOWRANK; p.status = dev_status(h);
+    p.pages = dev_pages(h);
+    p.q_raw = d_q; p.q_stride_b = stride_b; p.q_stride_t = stride_t;
+    p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+    p.rope_interleaved = h->rope_interleaved;
+    if (ws_stages >= 3) {
+      p.qp = h->ws + L.off_qp;
+      p.krot = h->ws + L.off_krot; p.krot_rows = h->desc.max_prefill_tokens;
+      p.el_table = reinterpret_cast<const float4*>(h->ws + L.off_rope + ea::kRopeTableOffset);
+      p.tmaps = h->ws + L.off_tmaps; p.tmaps_k = h->ws + L.off_tmaps_krot; p.k_width = dh;
+      p.max_rp = dh;
+      e = ea::launch_rope_prompt_prepare(p, L.max_rp_k, s, &h->launches);
+      if (e != cudaSuccess) return cuda_fail(h, e, "prefill preparation launch (rotary embedding)");
+      if (h->ev_start) cudaEventRecord(h->ev_start, s);
+      e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, false, s, &h->launches);
+      if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+      if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch (rotary embedding, tensor cores)");
+      return EA_OK;
+    }
+    if (h->ev_start) cudaEventRecord(h->ev_start, s);
+    e = ea::launch_prefill_rope(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+    if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill attention launch (rotary embedding)");
+    return EA_OK;
+  }
+  if (merged_in) {
+    // Rank-space rows from merged weights (Eq. 8): nothing to multiply.  K', V' rows are copied into the cache, Q'
+    // rows into the per-head layout the attention kernels read; a tensor the caller left d_head-wide is projected
+    // on the CUDA cores.
+    const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, flags & EA_KV_PREPROJECTED, s);
+    if (st != EA_OK) return st;
+    ea::QProjectParams qp{};
+    qp.heads = dev_heads(h); qp.basis = dev_basis(h); qp.q = d_q; qp.qp = h->ws + L.off_qp;
+    qp.stride_b = stride_b; qp.stride_t = stride_t;
+    qp.B = h->desc.batch; qp.T = T; qp.H = h->desc.n_heads; qp.d_head = h->desc.d_head;
+    e = (flags & EA_Q_PREPROJECTED) ? ea::launch_q_scatter(qp, L.sum_rp_k, h->desc.dtype, s, &h->launches)
+                                    : ea::launch_q_project(qp, h->desc.dtype, s, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill q launch");
+  } else if (tc_shape && in_aligned && h->opt_prefill != 1 && !h->paged && h->max_deficit == 0) {
+    if (!d_k || !d_v) return fail(h, EA_ERR_INVALID_ARG, "prefill: NULL k or v");
+    const ea_status st = project_on_tensor_cores();
+    if (st != EA_OK) return st;
   } else {
     const ea_status st = do_append(h, d_k, d_v, T, stride_b, stride_t, 0, s);
     if (st != EA_OK) return st;

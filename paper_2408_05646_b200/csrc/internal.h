@@ -156,12 +156,20 @@ struct PrefillParams {
   uint32_t flags;
   int* status;
   const void* tmaps;        // CUtensorMap[2 * H]: K' and V' slab of every head (warp-specialised kernel only)
+  // Key side taken from elsewhere than the cache (the rotary prompt path: full-rank rotated queries against lifted,
+  // rotated keys): every head's query and key rows are k_width wide, the queries sit at qp + h * k_width * B * T
+  // elements, the key tiles come through tmaps_k (CUtensorMap[H]).  0 / NULL: the rank-r rows of the cache.
+  int32_t k_width;
+  const void* tmaps_k;
   PageMap pages;            // paged cache (CUDA-core kernel only)
   // RoPE variant (prefill_rope.cu): the full-rank, un-rotated queries and the rotation's frequencies
   const void* q_raw;        // [B][T][H][d_head]
   int64_t q_stride_b, q_stride_t;
   const double* inv_freq;   // [d_head/2]: base^(-2i/d_head)
   int32_t rope_interleaved; // pairs (2i, 2i+1) instead of (i, i + d_head/2)
+  const float4* el_table;   // [32][128]: cos, cos, sin, sin of l phi for pairs 2k, 2k + 1 and row offset l
+  void* krot;               // lifted, rotated keys [H][B][krot_rows][d_head] (16-bit), written by the preparing kernels
+  int32_t krot_rows;
 };
 
 struct RopeDecodeParams {    // decode for models with rotary position embedding (bf16 layers)
@@ -267,6 +275,8 @@ cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s,
 // Q' rows that are already rank-space (packed [B][T][sum rp_k]) into the per-head layout of the Q' scratch.
 cudaError_t launch_q_scatter(const QProjectParams& p, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
+// the rotary prompt path on the tensor cores: rotated queries into p.qp, lifted rotated keys into p.krot
+cudaError_t launch_rope_prompt_prepare(const PrefillParams& p, int max_rp_k, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_rope(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);

@@ -123,7 +123,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
   const int qblk = gridDim.y - 1 - blockIdx.y;              // late (long) query blocks first
   const int len0 = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0);   // rows this sequence held before the call
   const int t0 = qblk * 2 * kTile;
-  const int rpk16 = (hd.rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
+  // width and place of this head's query and key rows: the rank-r rows, or the override of the rotary prompt path
+  const int rp_k = p.k_width ? p.k_width : hd.rp_k;
+  const int q_off = p.k_width ? h * p.k_width : hd.lr_k_off;
+  const int rpk16 = (rp_k + 15) & ~15, rpv16 = (hd.rp_v + 15) & ~15;
   const int nch_k = rpk16 >> 3, nch_v = rpv16 >> 3;
   const int grp_k = nch_k << 7, grp_v = nch_v << 7;
   // K'/V' tiles: atom columns of 64 rank elements, each [64 keys][128 bytes] with the 128-byte swizzle
@@ -175,7 +178,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const unsigned char* maps = static_cast<const unsigned char*>(p.tmaps) + static_cast<size_t>(h) * 256;
-      const void* map_k = maps;
+      const void* map_k = p.tmaps_k ? static_cast<const void*>(static_cast<const unsigned char*>(p.tmaps_k) + static_cast<size_t>(h) * 128)
+                                    : static_cast<const void*>(maps);
       const void* map_v = maps + 128;
       tensormap_acquire(map_k);
       tensormap_acquire(map_v);
@@ -323,9 +327,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) prefill_tc_ws_kernel(const Pref
     const int my_pos = len0 + tx + row;                    // last key this thread's query sees
     {                                                        // this tile's Q' (zeros past the prompt's end)
       const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.qp) +
-                                static_cast<int64_t>(hd.lr_k_off) * total_rows + static_cast<int64_t>(b) * p.T * hd.rp_k;
+                                static_cast<int64_t>(q_off) * total_rows + static_cast<int64_t>(b) * p.T * rp_k;
       const int q_rows = max(0, min(kTile, p.T - tx));
-      load_q_tile_async(Qs + x * q_bytes, q_rows > 0 ? Qg + static_cast<int64_t>(tx) * hd.rp_k : Qg, hd.rp_k, q_rows,
+      load_q_tile_async(Qs + x * q_bytes, q_rows > 0 ? Qg + static_cast<int64_t>(tx) * rp_k : Qg, rp_k, q_rows,
                         nch_k, hf * kTile + row);
       cp_async_commit();
       cp_async_wait<0>();

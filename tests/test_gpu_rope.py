@@ -130,6 +130,55 @@ def test_rope_prefill_matches_oracle_and_feeds_decode(B, H, d, rk, rv, T, base, 
     lay.poll_status()
 
 
+@pytest.mark.parametrize("H,d,rk,rv,T,base,interleaved", [
+    (2, 128, [80, 48], [64, 80], 700, 10000.0, False),              # several query blocks and key tiles
+    (3, 64, [24, 64, 40], [56, 8, 64], 150, 500000.0, True),
+    (1, 128, [128], [128], 77, 10000.0, False),
+    (2, 80, [40, 80], [80, 16], 333, 10000.0, True),                # d_head that is not a multiple of 64
+])
+def test_rope_prefill_on_the_tensor_cores(B, H, d, rk, rv, T, base, interleaved):
+    """The same prompt path with the scratch for rotated queries and lifted, rotated keys (a descriptor flag): the
+    warp-specialised tensor-core kernel, forced by option so that a silent fall back cannot pass.  Two chunks
+    (positions and keys continue from the cached rows), batches of unequal lengths, then generation; and the
+    CUDA-core kernel of a layer without the scratch must agree within the 16-bit roundings of the two."""
+    B_, steps = 2, 2
+    U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, T + steps, BF16, seed_cfg=191, T_q=T + steps)
+    q = (q.float() * 0.5).to(BF16)
+    lay = B.EigenAttnLayer(B_, H, d, T + steps, BF16, U_k, U_v, max_prefill_tokens=T, rope_prompt_scratch=True)
+    lay.set_rope(base, interleaved)
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, 2)
+    ref = rope_oracle(B_, H, d, U_k, U_v, base, interleaved)
+    cut = T // 2 + 5
+    a = lay.prefill(q[:, :cut].contiguous(), k[:, :cut].contiguous(), v[:, :cut].contiguous())
+    c = lay.prefill(q[:, cut:T].contiguous(), k[:, cut:T].contiguous(), v[:, cut:T].contiguous())
+    lay.poll_status()
+    expect = ref.prefill_dense(to_np(q[:, :T]), to_np(k[:, :T]), to_np(v[:, :T]))
+    got = torch.cat([a, c], dim=1)
+    assert_close(got, expect, BF16, "rope prefill on the tensor cores")
+    slow = B.EigenAttnLayer(B_, H, d, T + steps, BF16, U_k, U_v, max_prefill_tokens=T)
+    slow.set_rope(base, interleaved)
+    other = slow.prefill(q[:, :T].contiguous(), k[:, :T].contiguous(), v[:, :T].contiguous())
+    assert float((other.float() - got.float()).abs().max()) < 2e-2
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, 0)
+    for s in range(steps):
+        t = T + s
+        o = lay.decode_step(q[:, t:t + 1], k[:, t:t + 1], v[:, t:t + 1])
+        ref.append_kv(to_np(k[:, t:t + 1]), to_np(v[:, t:t + 1]))
+        assert_close(o, ref.decode_dense(to_np(q[:, t:t + 1])), BF16, f"decode step {s} after the prompt")
+    # a prompt that does not fit the scratch any more falls back (automatic) or is refused (forced)
+    lay.set_len(T)
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, 2)
+    with pytest.raises(B.EigenAttnError) as e:
+        lay.prefill(q[:, :2].contiguous(), k[:, :2].contiguous(), v[:, :2].contiguous())
+    assert e.value.status == B.EA_ERR_UNSUPPORTED and lay.len == T
+    lay.set_option(B.EA_OPT_PREFILL_IMPL, 0)
+    tail = lay.prefill(q[:, T:T + 2].contiguous(), k[:, T:T + 2].contiguous(), v[:, T:T + 2].contiguous())
+    full = rope_oracle(B_, H, d, U_k, U_v, base, interleaved)
+    assert_close(tail, full.prefill_dense(to_np(q[:, :T + 2]), to_np(k[:, :T + 2]), to_np(v[:, :T + 2]))[:, T:], BF16,
+                 "chunk past the scratch (CUDA-core kernel)")
+    lay.poll_status()
+
+
 def test_rope_rejections(B):
     U_k, U_v, q, k, v = make_case(1, 2, 64, [16, 16], [16, 16], 8, FP32, seed_cfg=155)
     lay32 = B.EigenAttnLayer(1, 2, 64, 8, FP32, U_k, U_v)
