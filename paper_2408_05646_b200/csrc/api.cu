@@ -900,7 +900,8 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
     size_t ws_smem = 0;
     const int dh = h->desc.d_head;
     const int ws_stages = h->krot_ok && tc_attn && h->opt_prefill != 1 && h->opt_prefill != 3 &&
-                                  static_cast<int64_t>(len0) + T <= h->desc.max_prefill_tokens
+                                  static_cast<int64_t>(len0) + T <= h->desc.max_prefill_tokens &&
+                                  ea::rope_lift_tc_smem_bytes(L.max_rp_k, dh) <= static_cast<size_t>(kSmemLimit)
                               ? ea::prefill_tc_ws_stages(dh, L.max_rp_v, dh, &ws_smem) : 0;
     if (h->opt_prefill == 2 && ws_stages < 3)
       return fail(h, EA_ERR_UNSUPPORTED, "prefill with rotary embedding: the tcgen05 kernel needs EA_ROPE_PROMPT_SCRATCH at create, "
@@ -933,7 +934,7 @@ ea_status eigen_attn_prefill(eigen_attn_t h, const void* d_q, const void* d_k, c
       p.el_table = reinterpret_cast<const float4*>(h->ws + L.off_rope + ea::kRopeTableOffset);
       p.tmaps = h->ws + L.off_tmaps; p.tmaps_k = h->ws + L.off_tmaps_krot; p.k_width = dh;
       p.max_rp = dh;
-      e = ea::launch_rope_prompt_prepare(p, L.max_rp_k, s, &h->launches);
+      e = ea::launch_rope_prompt_prepare(p, L.max_rp_k, h->sm_count, s, &h->launches);
       if (e != cudaSuccess) return cuda_fail(h, e, "prefill preparation launch (rotary embedding)");
       if (h->ev_start) cudaEventRecord(h->ev_start, s);
       e = ea::launch_prefill_tc_ws(p, ws_stages, ws_smem, false, s, &h->launches);

@@ -276,7 +276,9 @@ cudaError_t launch_q_project(const QProjectParams& p, int dtype, cudaStream_t s,
 cudaError_t launch_q_scatter(const QProjectParams& p, int lr_k_width, int dtype, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_prefill_simt(const PrefillParams& p, int dtype, cudaStream_t s, uint64_t* launches);
 // the rotary prompt path on the tensor cores: rotated queries into p.qp, lifted rotated keys into p.krot
-cudaError_t launch_rope_prompt_prepare(const PrefillParams& p, int max_rp_k, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_rope_prompt_prepare(const PrefillParams& p, int max_rp_k, int sm_count, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_rope_lift_tc(const PrefillParams& p, int max_rp_k, int sm_count, cudaStream_t s, uint64_t* launches);
+size_t rope_lift_tc_smem_bytes(int max_rp_k, int d_head);
 cudaError_t launch_prefill_rope(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);

@@ -196,78 +196,8 @@ __global__ void __launch_bounds__(kThreads) prefill_rope_kernel(const PrefillPar
 // With the full-rank rotated queries Qr_t = RoPE_{len0+t}(q_t) and the lifted, rotated keys Kr_j = RoPE_j(k'_j (U^K)^T)
 // written out (16-bit, d_head wide), score(t, j) = Qr_t . Kr_j / sqrt(d_h) is an ordinary causal attention product
 // over d_head-wide rows with rank-r values: the warp-specialised tensor-core kernel runs it unchanged, its key
-// operand coming from these rows instead of the cache.
-
-constexpr int kLiftRows = 32;
-
-// Kr of rows [32 blockIdx.x, +32) of one (sequence, head) unit: rows up to the end of the 64-row key tile that holds
-// the sequence's last row (the attention kernel reads whole tiles; rows past the length meet masked scores).
-__global__ void __launch_bounds__(128) rope_lift_rotate_kernel(const PrefillParams p) {
-  extern __shared__ __align__(16) float sm[];
-  const int unit = blockIdx.y;
-  const int h = unit / p.B, b = unit - h * p.B;
-  const HeadInfo hd = p.heads[h];
-  const int rpk = hd.rp_k, dh = p.d_head, half = dh >> 1;
-  const int len_b = p.len0 - (p.deficit != nullptr ? __ldg(p.deficit + b) : 0) + p.T;   // rows cached after the call
-  const int rows_b = min(min(p.krot_rows, p.n_max), (len_b + 63) & ~63);
-  const int j0 = blockIdx.x * kLiftRows;
-  if (j0 >= rows_b) return;
-  const int nk = min(kLiftRows, rows_b - j0);
-  float* Kraw = sm;                                   // [rpk][32]: rank element major, so that four rows are one 16-byte read
-  float* Ks = Kraw + kLiftRows * rpk;                 // [32][dh]  lifted, then rotated in place
-  float* base_cs = Ks + kLiftRows * dh;               // [half][2] cos, sin of (tile start) * freq
-  const int tid = threadIdx.x;
-  const bool inter = p.rope_interleaved != 0;
-  const __nv_bfloat16* Kslab = reinterpret_cast<const __nv_bfloat16*>(p.cache + hd.k_off) +
-                               (static_cast<int64_t>(b) * p.n_max + j0) * rpk;
-  for (int idx = tid; idx < kLiftRows * rpk; idx += 128) {
-    const int r = idx / rpk, c = idx - r * rpk;
-    Kraw[c * kLiftRows + r] = idx < nk * rpk ? __bfloat162float(Kslab[idx]) : 0.f;
-  }
-  if (tid < half) cos_sin_of(static_cast<double>(j0), p.inv_freq[tid], &base_cs[2 * tid], &base_cs[2 * tid + 1]);
-  __syncthreads();
-  if (tid < dh) {                                     // coordinate tid of k'_row (U^K)^T for the 32 rows
-    float acc[kLiftRows];
-#pragma unroll
-    for (int r = 0; r < kLiftRows; ++r) acc[r] = 0.f;
-    const float* Ud = p.basis + hd.uk_off + static_cast<size_t>(tid) * rpk;
-    for (int c = 0; c < rpk; ++c) {
-      const float u = __ldg(Ud + c);
-      const float4* kc = reinterpret_cast<const float4*>(Kraw + c * kLiftRows);
-#pragma unroll
-      for (int r4 = 0; r4 < kLiftRows / 4; ++r4) {
-        const float4 kv = kc[r4];
-        acc[4 * r4 + 0] = fmaf(kv.x, u, acc[4 * r4 + 0]);
-        acc[4 * r4 + 1] = fmaf(kv.y, u, acc[4 * r4 + 1]);
-        acc[4 * r4 + 2] = fmaf(kv.z, u, acc[4 * r4 + 2]);
-        acc[4 * r4 + 3] = fmaf(kv.w, u, acc[4 * r4 + 3]);
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < kLiftRows; ++r) Ks[r * dh + tid] = acc[r];
-  }
-  __syncthreads();
-  // pair i of row r turned by (j0 + r) * freq_i: the tile's base angle (reduced in double precision) plus the row
-  // offset from the layer's table, combined by the angle-addition formulas
-  for (int idx = tid; idx < nk * half; idx += 128) {
-    const int r = idx / half, i = idx - r * half;
-    const int da = inter ? 2 * i : i, db = inter ? 2 * i + 1 : i + half;
-    const float4 e = __ldg(p.el_table + (i >> 1) * 128 + r);
-    const float cl = (i & 1) ? e.y : e.x, sl = (i & 1) ? e.w : e.z;
-    const float c0 = base_cs[2 * i], s0 = base_cs[2 * i + 1];
-    const float cs = c0 * cl - s0 * sl, sn = s0 * cl + c0 * sl;
-    const float a = Ks[r * dh + da], bb = Ks[r * dh + db];
-    Ks[r * dh + da] = a * cs - bb * sn;
-    Ks[r * dh + db] = a * sn + bb * cs;
-  }
-  __syncthreads();
-  __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.krot) +
-                       ((static_cast<int64_t>(h) * p.B + b) * p.krot_rows + j0) * dh;
-  for (int idx = tid; idx < nk * dh / 2; idx += 128) {
-    const float2 v = *reinterpret_cast<const float2*>(Ks + 2 * idx);
-    reinterpret_cast<__nv_bfloat162*>(dst)[idx] = __floats2bfloat162_rn(v.x, v.y);
-  }
-}
+// operand coming from these rows instead of the cache.  The keys are prepared by the tensor-core kernel of
+// rope_lift_tc.cu, the queries here.
 
 // Qr of one prompt token of one sequence, all heads: [h][b * T + t][d_head] (the layout the attention kernel reads)
 __global__ void __launch_bounds__(256) rope_rotate_queries_kernel(const PrefillParams p) {
@@ -295,15 +225,8 @@ __global__ void __launch_bounds__(256) rope_rotate_queries_kernel(const PrefillP
 
 }  // namespace
 
-cudaError_t launch_rope_prompt_prepare(const PrefillParams& p, int max_rp_k, cudaStream_t s, uint64_t* launches) {
-  const int rows = min(min(p.krot_rows, p.n_max), (p.len0 + p.T + 63) & ~63);   // of the longest sequence
-  const size_t smem = (static_cast<size_t>(kLiftRows) * (max_rp_k + p.d_head) + p.d_head) * sizeof(float);
-  static size_t configured[kMaxDevices] = {};
-  const cudaError_t ec = ensure_dynamic_smem(rope_lift_rotate_kernel, smem, configured);
-  if (ec != cudaSuccess) return ec;
-  rope_lift_rotate_kernel<<<dim3((rows + kLiftRows - 1) / kLiftRows, p.B * p.H), 128, smem, s>>>(p);
-  ++*launches;
-  cudaError_t e = cudaGetLastError();
+cudaError_t launch_rope_prompt_prepare(const PrefillParams& p, int max_rp_k, int sm_count, cudaStream_t s, uint64_t* launches) {
+  const cudaError_t e = launch_rope_lift_tc(p, max_rp_k, sm_count, s, launches);   // Kr of every row held after the call
   if (e != cudaSuccess) return e;
   rope_rotate_queries_kernel<<<p.B * p.T, 256, 0, s>>>(p);
   ++*launches;
