@@ -468,6 +468,10 @@ def run_ours(args, wl):
         del lay
         torch.cuda.empty_cache()
         line["prefill"] = prefill_measure(synth.WORKLOADS["prefill_b4_t4096"], device, steps=10, warmup=3)
+        r = prefill_measure(synth.WORKLOADS["prefill_b4_t4096"], device, steps=10, warmup=3, rope=True)
+        line["prefill_rope"] = {k: r[k] for k in ("workload", "ms_per_call", "attention_kernel_ms", "attention_tflops", "frac")}
+        line["prefill_rope"]["what"] = ("the same prompt through a layer with rotary embedding: token rows projected, keys lifted "
+                                        "and rotated, queries rotated, causal attention over d_head-wide rows; ms_per_call is all of it")
     if cpu is not None:
         line["cpu_baseline"] = cpu
         line["parity_full_size"] = parity
@@ -709,7 +713,7 @@ def workload_table_own_layers(device, binding, steps=30, warmup=3):
     return table
 
 
-def prefill_measure(wl, device, steps, warmup, impl=0):
+def prefill_measure(wl, device, steps, warmup, impl=0, rope=False):
     """Times eigen_attn_prefill on the prompt workload; returns a small dict (call time, attention-kernel time,
     TFLOP/s of the causal contractions, fraction of the measured bf16 peak)."""
     from paper_2408_05646_b200 import binding
@@ -718,7 +722,10 @@ def prefill_measure(wl, device, steps, warmup, impl=0):
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
     dt = synth.torch_dtype(wl.dtype)
     T = wl.context
-    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device)
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device,
+                                 rope_prompt_scratch=rope)
+    if rope:                                       # Section 4.3: full-rank rotated queries against lifted, rotated keys
+        lay.set_rope(10000.0)
     if impl:
         lay.set_option(binding.EA_OPT_PREFILL_IMPL, impl)
     W = {t: synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_" + t, device=device) for t in "KVQ"}
@@ -744,7 +751,8 @@ def prefill_measure(wl, device, steps, warmup, impl=0):
     lay.poll_status()
     ms = t0.elapsed_time(t1) / steps
     kern = sum(a.elapsed_time(b) for a, b in ev) / steps
-    flop = 2 * (wl.batch * T * (T + 1) // 2) * sum(2 * r for r in ranks)
+    # causal contractions: Q'K'^T over r_k (d_head wide with the rotary embedding) and PV' over r_v
+    flop = 2 * (wl.batch * T * (T + 1) // 2) * sum((wl.d_head if rope else r) + r for r in ranks)
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peak = float(json.load(open(peaks_path))["bf16_tflops"]) if os.path.exists(peaks_path) else 1590.0
     tf = flop / (kern * 1e-3) / 1e12

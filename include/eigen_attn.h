@@ -190,9 +190,12 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
  * eigen_attn_append_kv writes them.  The paper shares one U^K among the heads of a layer; here that is the
  * special case of equal U_k[h].  base == 0 switches back.  bf16 layers with d_head % 16 == 0 only
  * (EA_ERR_UNSUPPORTED otherwise).  eigen_attn_prefill follows the same reading for a prompt (query t at position
- * len0 + t, the cache filled with projections of the un-rotated keys) on a CUDA-core kernel: the functional prompt
- * path of such a layer, not a tensor-core one.  eigen_attn_decode_static returns EA_ERR_UNSUPPORTED while a rotary
- * embedding is set.  Synchronises `cuda_stream`. */
+ * len0 + t, the cache filled with projections of the un-rotated keys).  A layer created with EA_ROPE_PROMPT_SCRATCH
+ * runs it on the tensor cores while the rows cached after the call fit max_prefill_tokens (the rotated queries and
+ * the lifted, rotated keys of those rows are written to the workspace once per call, then the prompt's causal
+ * product runs over d_head-wide rows); otherwise, and for later chunks of a longer prompt, a CUDA-core kernel does
+ * the same arithmetic tile by tile (two orders of magnitude slower).  eigen_attn_decode_static returns
+ * EA_ERR_UNSUPPORTED while a rotary embedding is set.  Synchronises `cuda_stream`. */
 ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, void* cuda_stream);
 
 /* Section 5.3 ("Eigen Attention with Quantization") and Table 8: a quantised copy of the rank-r cache.
