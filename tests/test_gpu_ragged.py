@@ -318,6 +318,7 @@ def test_many_sequences_of_unequal_lengths(B):
     (BF16, 128, [80, 48, 128], [80, 112, 64], 600, [600, 129, 0, 471], 300, "plain"),     # warp-specialised tcgen05 kernel
     (BF16, 128, [80, 80, 80], [80, 80, 80], 300, [5, 300, 299, 64], 130, "alibi"),
     (BF16, 128, [80, 64, 48], [64, 80, 96], 260, [260, 1, 77, 130], 70, "rope"),          # Section 4.3 prompt form
+    (BF16, 128, [80, 64, 48], [64, 80, 96], 260, [260, 1, 77, 130], 70, "rope-tc"),       # ... on the tensor cores
     (FP32, 64, [32, 20, 64], [16, 40, 8], 200, [200, 1, 77, 0], 50, "plain"),             # CUDA-core kernel
     (BF16, 128, [80, 48, 128], [80, 112, 64], 400, [400, 129, 3, 271], 200, "single-tile"),
 ])
@@ -329,15 +330,19 @@ def test_prompt_chunk_behind_sequences_of_unequal_lengths(B, dtype, d, rk, rv, n
     U_k, U_v, q, k, v = make_case(B_, H, d, rk, rv, n + T + 1, dtype, seed_cfg=148, T_q=n + T + 1)
     if dtype == BF16:
         q = (q.float() * 0.25).to(dtype)                              # Q' is kept in 16 bits by the prompt kernels
-    lay = B.EigenAttnLayer(B_, H, d, n + T + 1, dtype, U_k, U_v, max_prefill_tokens=T)
+    tc_rope = variant == "rope-tc"                 # the scratch must hold every row a sequence has after the call
+    lay = B.EigenAttnLayer(B_, H, d, n + T + 1, dtype, U_k, U_v, max_prefill_tokens=n + T if tc_rope else T,
+                           rope_prompt_scratch=tc_rope)
     slopes = [0.5, 0.0625, 0.25] if variant == "alibi" else None
-    rope = {"base": 10000.0, "interleaved": False} if variant == "rope" else None
+    rope = {"base": 10000.0, "interleaved": False} if variant.startswith("rope") else None
     if slopes:
         lay.set_alibi(slopes)
     if rope:
         lay.set_rope(rope["base"], rope["interleaved"])
     if variant == "single-tile":
         lay.set_option(B.EA_OPT_PREFILL_IMPL, 3)
+    if tc_rope:
+        lay.set_option(B.EA_OPT_PREFILL_IMPL, 2)   # refuse rather than fall back to the CUDA-core kernel
     lay.append_kv(k[:, :n], v[:, :n])              # every sequence holds n rows; each keeps its first lens[b]
     lay.set_lens(lens)
     ref = PerSequenceOracle(H, d, U_k, U_v, k, v, lens, alibi_slopes=slopes, storage=storage_model(dtype), rope=rope)
