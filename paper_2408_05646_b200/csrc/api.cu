@@ -1203,13 +1203,16 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
     return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: needs a bf16 layer with d_head %% 16 == 0");
   if (h->alibi) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with an ALiBi bias set");
   if (h->len - h->max_deficit < 1) return fail(h, EA_ERR_SHAPE, "decode_gqa: the cache is empty (for some sequence)");
-  // Section 4.3 for a group: every query head of the group is a unit of the rotary kernel over its K/V head's rows
-  if (h->rope)
+  // Section 4.3 for a group.  On the tensor cores where the tiles fit (decode_gqa_rope_kernel: the keys of a tile are
+  // lifted and turned once for the whole group); otherwise (wide ranks, a page table) every query head of the group
+  // is a unit of the multi-head rotary kernel over its K/V head's rows.
+  const bool rope_tc = h->rope && !h->paged && group > 1 && ea::decode_gqa_rope_smem_bytes(h->L.max_rp_k, h->desc.d_head) != 0;
+  if (h->rope && !rope_tc)
     return do_decode_rope(h, d_q, stride_b_q, d_out, stride_b_out, 0u, static_cast<cudaStream_t>(cuda_stream), group);
   if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table (without a rotary embedding)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
-  const size_t smem = ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
+  const size_t smem = rope_tc ? ea::decode_gqa_rope_smem_bytes(L.max_rp_k, h->desc.d_head) : ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
   if (smem > static_cast<size_t>(kSmemLimit)) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: tiles do not fit");
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   ea::GqaDecodeParams p{};
@@ -1246,7 +1249,14 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   p.splits = static_cast<int32_t>(splits);
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   if (h->ev_start) cudaEventRecord(h->ev_start, s);
-  const cudaError_t e = ea::launch_decode_gqa(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+  if (rope_tc) {
+    p.inv_freq = reinterpret_cast<const double*>(h->ws + L.off_rope);
+    p.tile_step = reinterpret_cast<const float2*>(h->ws + L.off_rope + ea::kRopeStepOffset);
+    p.el_table = reinterpret_cast<const float4*>(h->ws + L.off_rope + ea::kRopeTableOffset);
+    p.interleaved = h->rope_interleaved;
+  }
+  const cudaError_t e = rope_tc ? ea::launch_decode_gqa_rope(p, L.max_rp_k, s, &h->launches)
+                                : ea::launch_decode_gqa(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_gqa launch");
   return EA_OK;

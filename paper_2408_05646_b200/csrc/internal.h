@@ -219,6 +219,11 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
   int32_t group;            // 1..16
   float q_scale;            // log2(e) / sqrt(d_head)
   uint32_t flags;
+  // with a rotary embedding (decode_gqa_rope_kernel): the constants of eigen_attn_set_rope
+  const double* inv_freq;   // [d_head/2]
+  const float2* tile_step;  // [64]: cos, sin of -128 phi_i
+  const float4* el_table;   // [32][128]: cos, cos, sin, sin of l phi for pairs 2k, 2k + 1 and row offset l
+  int32_t interleaved;
 };
 
 // Quantised copy of the cache (Section 5.3 of the paper): per head a slab [B][blocks_max][block_bytes]; a block
@@ -281,6 +286,9 @@ cudaError_t launch_rope_lift_tc(const PrefillParams& p, int max_rp_k, int sm_cou
 size_t rope_lift_tc_smem_bytes(int max_rp_k, int d_head);
 cudaError_t launch_prefill_rope(const PrefillParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
+// grouped queries with a rotary embedding on the tensor cores; 0 bytes = the tiles do not fit
+size_t decode_gqa_rope_smem_bytes(int max_rp_k, int d_head);
+cudaError_t launch_decode_gqa_rope(const GqaDecodeParams& p, int max_rp_k, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
 // bytes of the rotary constants a layer keeps: inverse frequencies (64 doubles), per-tile steps (64 float2),

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 #include "internal.h"
@@ -232,6 +233,10 @@ __device__ __forceinline__ unsigned long long mul2p(unsigned long long a, unsign
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  const __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -260,6 +265,12 @@ __device__ __forceinline__ uint32_t sw128_off(int row, int c) {
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(kTile >> 4) << 24);
+}
+
+// The same with fp16 A and B (format fields 0): for operands a kernel writes itself and wants three more mantissa
+// bits in than bf16 gives (both operands of one product always have the same type).
+__host__ __device__ constexpr uint32_t instr_desc_f16(int n) {
+  return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTile >> 4) << 24);
 }
 
 // Canonical tile: chunk (row, c) of 16 bytes lives at (row/8) * group_stride + c * 128 + (row%8) * 16,
