@@ -702,11 +702,10 @@ def workload_table_own_layers(device, binding, steps=30, warmup=3):
     k_us, s_us = timed_kernel(lay, device, step_gqa, steps, warmup)
     table[wl.name] = table_entry("decode_gqa_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
                                  group=g)
-    # the same layer with the rotary embedding these models use: every query head is a unit of the rotary decode
-    # kernel over its K/V head's rows (the bytes counted are still the rows of the cache, read once)
+    # the same layer with the rotary embedding these models use (the bytes counted are the rows of the cache, read once)
     lay.set_rope(10000.0)
     k_us, s_us = timed_kernel(lay, device, step_gqa, steps, warmup)
-    table[wl.name + "[rope]"] = table_entry("decode_rope_kernel", k_us, s_us,
+    table[wl.name + "[rope]"] = table_entry("decode_gqa_rope_kernel", k_us, s_us,
                                             algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak, group=g, rope=True)
     del lay
     torch.cuda.empty_cache()

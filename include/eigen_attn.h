@@ -174,9 +174,10 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
  * head's rank-r rows with its U^K and are lifted with its U^V (Eq. 7 per query head).  d_q and d_out:
  * [B][1][n_heads * group][d_head], batch strides in elements.  One pass over the cache serves the whole
  * group.  1 <= group <= 16; bf16 layers with d_head % 16 == 0 and no ALiBi bias set (EA_ERR_UNSUPPORTED
- * otherwise).  With a rotary embedding set (the Llama models: Section 4.3 per query head) every query head of a
- * group is served as its own unit of the rotary decode kernel; its group's rows then come from the cache once and
- * from L2 for the other heads of the group.  The partials of batch x n_heads x group x splits must fit the workspace
+ * otherwise).  With a rotary embedding set (the Llama models: Section 4.3 per query head) the keys of a tile are
+ * lifted and turned once for the whole group and scored on the tensor cores (fp16 operand tiles: turned keys and
+ * scaled queries must stay below 65504); where the tiles do not fit shared memory (r_k above 96 at d_head 128) or a
+ * page table is set, every query head is served as its own unit of the multi-head rotary kernel.  The partials of batch x n_heads x group x splits must fit the workspace
  * (EA_ERR_CAPACITY).  Attends over the rows the cache holds: append the new token's rows first. */
 ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
                                 int64_t stride_b_out, void* cuda_stream);

@@ -138,22 +138,27 @@ def test_alibi_positions_count_from_each_sequences_own_end(B, dtype):
     lay.poll_status()
 
 
+@pytest.mark.parametrize("rope", [None, {"base": 10000.0, "interleaved": False}])
 @pytest.mark.parametrize("H,g,d,rk,rv,n,lens", [
     (2, 4, 128, [80, 80], [80, 80], 1037, [1037, 1, 500]),
     (3, 8, 128, [48, 64, 128], [96, 80, 128], 700, [129, 700, 128]),
 ])
-def test_grouped_query_decode_with_unequal_lengths(B, H, g, d, rk, rv, n, lens):
-    """Every query head of a group attends the own rows of its sequence's K/V head."""
+def test_grouped_query_decode_with_unequal_lengths(B, H, g, d, rk, rv, n, lens, rope):
+    """Every query head of a group attends the own rows of its sequence's K/V head; with a rotary embedding the
+    queries of a sequence sit at that sequence's own last position (first case: the grouped rotary kernel on the
+    tensor cores; second: a rank of 128 does not fit it, every query head is a unit of the multi-head kernel)."""
     B_ = len(lens)
     U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n + 1, BF16, seed_cfg=143)
     W_q = synth.mixing_matrices(H * g, 16, d, 143, "W_Q")
     q = synth.lowrank_rows(W_q, B_, 1, 0.1, 143, "Q", dtype=BF16, device="cuda:0")        # [B][1][H*g][d]
     lay = B.EigenAttnLayer(B_, H, d, n + 1, BF16, U_k, U_v)
+    if rope:
+        lay.set_rope(rope["base"], rope["interleaved"])
     lay.append_kv(k[:, :n], v[:, :n])
     lay.set_lens(lens)
     refs = []
     for b, nb in enumerate(lens):
-        r = oracle_layer(1, H, d, U_k, U_v)
+        r = orc.LayerOracle(1, H, d, U_k, U_v, rope=rope)
         r.append_kv(to_np(k[b:b + 1, :nb]), to_np(v[b:b + 1, :nb]))
         refs.append(r)
     expect = lambda: np.concatenate([r.decode_gqa(to_np(q[b:b + 1]), g) for b, r in enumerate(refs)], axis=0)
