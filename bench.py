@@ -781,7 +781,10 @@ def run_prefill(args, wl):
     U_v = synth.make_bases(wl.d_head, ranks, wl.index, "U_V")
     dt = synth.torch_dtype(wl.dtype)
     T = wl.context
-    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device)
+    lay = binding.EigenAttnLayer(wl.batch, wl.n_heads, wl.d_head, T + 1, dt, U_k, U_v, max_prefill_tokens=T, device=device,
+                                 rope_prompt_scratch=args.rope)
+    if args.rope:                                  # Section 4.3: rotated full-rank queries against lifted, rotated keys
+        lay.set_rope(10000.0)
     if args.prefill_impl:
         lay.set_option(binding.EA_OPT_PREFILL_IMPL, args.prefill_impl)
     W = {t: synth.mixing_matrices(wl.n_heads, wl.rho, wl.d_head, wl.index, "W_" + t, device=device) for t in "KVQ"}
@@ -813,7 +816,8 @@ def run_prefill(args, wl):
     ms = t0.elapsed_time(t1) / steps
     kern = sum(a.elapsed_time(b) for a, b in ev) / steps
     pairs = wl.batch * T * (T + 1) // 2                       # causal (query, key) pairs per head, summed over the batch
-    flop = 2 * pairs * sum(2 * r for r in ranks)             # Q'K'^T and PV' over the lower triangle
+    # Q'K'^T and PV' over the lower triangle (with the rotary embedding the score product is d_head wide)
+    flop = 2 * pairs * sum((wl.d_head if args.rope else r) + r for r in ranks)
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peak, src = 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
     if os.path.exists(peaks_path):
@@ -825,11 +829,17 @@ def run_prefill(args, wl):
         rows = [0, 1, 127, 128, 1000, T - 1]
         kk, vv = k[b, :, h].double().cpu().numpy(), v[b, :, h].double().cpu().numpy()
         for t in rows:
-            ref = orc.decode_head(q[b, t, h].double().cpu().numpy(), kk[:t + 1], vv[:t + 1], U_k[h], U_v[h])
+            qt = q[b, t, h].double().cpu().numpy()
+            if args.rope:                          # row t of the prompt form = the generation form over rows 0..t
+                ref = orc.decode_head_rope(qt, kk[:t + 1] @ U_k[h].astype(np.float64), vv[:t + 1] @ U_v[h].astype(np.float64),
+                                           U_k[h], U_v[h], 10000.0, False)
+            else:
+                ref = orc.decode_head(qt, kk[:t + 1], vv[:t + 1], U_k[h], U_v[h])
             errs.append(float(np.abs(out[b, t, h].double().cpu().numpy() - ref).max()))
     achieved = flop / (kern * 1e-3) / 1e12
     print(json.dumps({
-        "metric": "causal rank-r prefill attention TFLOP/s (B=4, T=4096, 7B layer)", "value": flop / (ms * 1e-3) / 1e12,
+        "metric": "causal rank-r prefill attention TFLOP/s (B=4, T=4096, 7B layer)" + (", rotary embedding" if args.rope else ""),
+        "value": flop / (ms * 1e-3) / 1e12,
         "unit": "TFLOP/s", "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "n_heads": wl.n_heads, "d_head": wl.d_head, "rank": sorted(set(ranks)),
@@ -916,6 +926,9 @@ def run_gqa(args, wl):
     n0 = wl.context
     stream = torch.cuda.current_stream(device)
     steps, warmup = min(args.steps, 100), max(3, min(args.warmup, 10))
+    rope = {"base": 10000.0, "interleaved": False} if args.rope else None
+    if rope:                                       # Section 4.3 for the group: the form the Llama-3 models run
+        lay.set_rope(rope["base"])
 
     def step():
         lay.set_len(n0)
@@ -963,7 +976,7 @@ def run_gqa(args, wl):
     ms_one_by_one = a0.elapsed_time(a1) / 10
     # parity of the sampled units against the oracle
     from oracle import eigen_attention as orc
-    ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=[(0, h) for h in keep])
+    ref = orc.LayerOracle(wl.batch, wl.n_heads, wl.d_head, U_k, U_v, tracked=[(0, h) for h in keep], rope=rope)
     for h in keep:
         ref.append_unit_rows((0, h), hist[(0, h)][0], hist[(0, h)][1])
     ref.set_len(n0)
@@ -973,14 +986,14 @@ def run_gqa(args, wl):
     errs = [float(np.abs(got[0, 0, h * g + i] - exp[0, 0, h * g + i]).max()) for h in keep for i in range(g)]
     achieved = bytes_step / (kern * 1e-3) / 1e9
     print(json.dumps({
-        "metric": "grouped-query rank-r decode KV GB/s (B=16, n=32k, 8 K/V heads x 4 query heads)",
+        "metric": "grouped-query rank-r decode KV GB/s (B=16, n=32k, 8 K/V heads x 4 query heads)" + (", rotary embedding" if rope else ""),
         "value": bytes_step / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warmup,
         "ms_per_step": ms, "us_per_step": ms * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 storage and operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "kv_heads": wl.n_heads, "group": g, "d_head": wl.d_head,
                    "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "cache_gb": bytes_step / 1e9,
                    "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
-        "roofline": {"bound": "hbm", "kernel": "decode_gqa_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "decode_gqa_rope_kernel" if rope else "decode_gqa_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "kernel_us": kern * 1e3,
                      "algorithmic_bytes": bytes_step, "traffic": None},
         "one_query_head_at_a_time_us": ms_one_by_one * 1e3,
