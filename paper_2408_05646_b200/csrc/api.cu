@@ -1327,7 +1327,9 @@ ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, v
   int widest = 0;
   const size_t need = make_quant_layout(h, bits, group, &qh, &widest);
   if (bytes < need) return fail(h, EA_ERR_CAPACITY, "quant_attach: %zu bytes given, %zu needed", bytes, need);
-  if (ea::decode_quant_smem_bytes(widest, h->L.max_rp_v) > static_cast<size_t>(kSmemLimit))
+  const int widest_rp = h->L.max_rp_k > h->L.max_rp_v ? h->L.max_rp_k : h->L.max_rp_v;
+  if ((bits == 4 ? ea::decode_quant_mma_smem_bytes(widest, widest_rp, group)
+                 : ea::decode_quant_smem_bytes(widest, h->L.max_rp_v)) > static_cast<size_t>(kSmemLimit))
     return fail(h, EA_ERR_UNSUPPORTED, "quant_attach: a stage of 128 rows does not fit in shared memory");
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = cudaMemcpyAsync(d_qcache, qh.data(), sizeof(ea::QuantHead) * qh.size(), cudaMemcpyHostToDevice, s);
@@ -1452,12 +1454,14 @@ ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t strid
   p.nst = (p.nq + 127) / 128;
   p.q_scale = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(h->desc.d_head)));
   p.flags = flags;
-  const size_t smem = ea::decode_quant_smem_bytes(h->q_max_stage_bytes, L.max_rp_v);
   const int max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
+  const bool mma = p.bits == 4;          // 4-bit codes run on the integer tensor-core kernel
+  const size_t smem = mma ? ea::decode_quant_mma_smem_bytes(h->q_max_stage_bytes, max_rp, p.group)
+                          : ea::decode_quant_smem_bytes(h->q_max_stage_bytes, L.max_rp_v);
   // CTAs per unit: waves of (SMs x resident CTAs), a start-up worth a few stages per CTA, and room for
   // units x splits partials in the workspace
   int ctas_per_sm = static_cast<int>(static_cast<size_t>(228 * 1024) / (smem + 1024));
-  const int reg_limit = max_rp <= 80 ? 3 : 2;
+  const int reg_limit = mma ? 4 : max_rp <= 80 ? 3 : 2;
   if (ctas_per_sm > reg_limit) ctas_per_sm = reg_limit;
   if (ctas_per_sm < 1) ctas_per_sm = 1;
   const int64_t units = static_cast<int64_t>(p.B) * p.H;
@@ -1485,7 +1489,8 @@ ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t strid
     if (hi.rp_k < min_rp) min_rp = hi.rp_k;
     if (hi.rp_v < min_rp) min_rp = hi.rp_v;
   }
-  const cudaError_t e = ea::launch_decode_quant(p, max_rp, min_rp, smem, s, &h->launches);
+  const cudaError_t e = mma ? ea::launch_decode_quant_mma(p, max_rp, smem, s, &h->launches)
+                            : ea::launch_decode_quant(p, max_rp, min_rp, smem, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_quant launch");
   return EA_OK;

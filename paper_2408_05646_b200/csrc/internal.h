@@ -230,10 +230,13 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
 // holds G consecutive rows of one sequence as integer codes and half-precision scales:
 //   K codes  [rp_k/8][G] units     K scales [rp_k] halves        (one scale per channel and block)
 //   V codes  [rp_v/8][G] units     V scales [nvg][G] halves      (one scale per row and G channels)
-// A unit holds the eight channels 8j..8j+7 of one row.  4-bit codes: a 32-bit word, channel 8j+k in bits 4k..4k+3
-// as code + 8.  3-bit codes: 24 bits, channel 8j+k in bits 3k..3k+2 as code + 4, stored as two planes, the low 16
-// bits of every unit ([rp/8][G] halfwords) followed by the high 8 bits of every unit ([rp/8][G] bytes): exactly
-// 3 bits per element, and a warp's loads of either plane are consecutive.
+// 3-bit codes: a unit holds the eight channels 8j..8j+7 of one row in 24 bits, channel 8j+k in bits 3k..3k+2 as
+// code + 4, stored as two planes, the low 16 bits of every unit ([rp/8][G] halfwords) followed by the high 8 bits of
+// every unit ([rp/8][G] bytes): exactly 3 bits per element, and a warp's loads of either plane are consecutive.
+// 4-bit codes: a unit is a 32-bit word of eight nibbles, each code + 8, laid out for the operand fragments of the
+// integer tensor-core products.  Keys: word j of row i holds channels 8j..8j+7 (channel 8j+k in bits 4k..4k+3) and
+// sits at j G + ((i + 8 (j mod 4)) mod G).  Values: chunks of min(G, 32) rows, a chunk [rp_v][rows/8] words, word
+// (c, o) holding rows 8o..8o+7 of channel c (row 8o+k in bits 4k..4k+3).
 struct QuantHead {
   int64_t slab_off;        // byte offset of the head's slab in the quantised buffer
   int32_t block_bytes;
@@ -312,6 +315,10 @@ cudaError_t launch_quantize_blocks(const QuantParams& p, cudaStream_t s, uint64_
 size_t decode_quant_smem_bytes(int max_stage_bytes, int max_rp_v);
 cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, int min_rp, size_t smem, cudaStream_t s,
                                 uint64_t* launches);   // min_rp: narrowest padded rank over heads and K/V
+// 4-bit codes: the integer tensor-core kernel
+size_t decode_quant_mma_smem_bytes(int max_stage_bytes, int max_rp, int group);
+cudaError_t launch_decode_quant_mma(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_quant_combine(const QuantParams& p, cudaStream_t s, uint64_t* launches);
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
 // library's own partials array on the current device (queried from the runtime on every call).

@@ -91,20 +91,36 @@ __global__ void __launch_bounds__(kQThreads) quantize_blocks_kernel(const QuantP
     __syncthreads();
     char* code_base = dst + (pass ? qh.vc_off : 0);
     const int words = (rp / 8) * G;
-    for (int i = tid; i < words; i += kQThreads) {
-      const int j = i / G, r = i - j * G;
-      uint32_t w = 0;
+    if (p.bits == 4 && pass == 1) {
+      // 4-bit values: chunks of min(G, 32) rows, a chunk [rp][rows / 8] words, a word = eight rows of one channel
+      const int opc = (G < 32 ? G : 32) / 8;
+      for (int i = tid; i < words; i += kQThreads) {
+        const int qc = i / (rp * opc), rem = i - qc * rp * opc;
+        const int c = rem / opc, o = rem - c * opc;
+        uint32_t w = 0;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int c = 8 * j + k;
-        const float s = pass ? scale_sm[(c / G) * G + r] : scale_sm[c];
-        w |= stored_code(__bfloat162float(tile[r * rp + c]), s, qmax) << (p.bits * k);
-      }
-      if (p.bits == 4) {
+        for (int k = 0; k < 8; ++k) {
+          const int r = qc * 32 + o * 8 + k;
+          w |= stored_code(__bfloat162float(tile[r * rp + c]), scale_sm[(c / G) * G + r], qmax) << (4 * k);
+        }
         reinterpret_cast<uint32_t*>(code_base)[i] = w;
-      } else {                // two planes: low 16 bits of every unit, then the high 8 bits
-        reinterpret_cast<uint16_t*>(code_base)[i] = static_cast<uint16_t>(w);
-        reinterpret_cast<uint8_t*>(code_base + 2 * words)[i] = static_cast<uint8_t>(w >> 16);
+      }
+    } else {
+      for (int i = tid; i < words; i += kQThreads) {
+        const int j = i / G, r = i - j * G;
+        uint32_t w = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int c = 8 * j + k;
+          const float s = pass ? scale_sm[(c / G) * G + r] : scale_sm[c];
+          w |= stored_code(__bfloat162float(tile[r * rp + c]), s, qmax) << (p.bits * k);
+        }
+        if (p.bits == 4) {      // keys: the word of row r sits 8 (j mod 4) rows further on (modulo G)
+          reinterpret_cast<uint32_t*>(code_base)[j * G + ((r + 8 * (j & 3)) & (G - 1))] = w;
+        } else {                // two planes: low 16 bits of every unit, then the high 8 bits
+          reinterpret_cast<uint16_t*>(code_base)[i] = static_cast<uint16_t>(w);
+          reinterpret_cast<uint8_t*>(code_base + 2 * words)[i] = static_cast<uint8_t>(w >> 16);
+        }
       }
     }
     __syncthreads();          // the tile and the scales are reused by the second pass
@@ -452,9 +468,7 @@ cudaError_t launch_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
 }
 template <int NW, int MINB, int G>
 cudaError_t launch_full_or_not(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
-  if (p.bits == 3)
-    return full ? launch_variant<NW, MINB, G, true, 3>(p, smem, s) : launch_variant<NW, MINB, G, false, 3>(p, smem, s);
-  return full ? launch_variant<NW, MINB, G, true, 4>(p, smem, s) : launch_variant<NW, MINB, G, false, 4>(p, smem, s);
+  return full ? launch_variant<NW, MINB, G, true, 3>(p, smem, s) : launch_variant<NW, MINB, G, false, 3>(p, smem, s);
 }
 template <int NW, int MINB>
 cudaError_t launch_group(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
@@ -495,6 +509,10 @@ cudaError_t launch_decode_quant(const QuantParams& p0, int max_rp, int min_rp, s
   else e = launch_group<16, 2>(p, min_rp == 128, smem, s);
   if (e != cudaSuccess) return e;
   ++*launches;
+  return launch_quant_combine(p, s, launches);
+}
+
+cudaError_t launch_quant_combine(const QuantParams& p, cudaStream_t s, uint64_t* launches) {
   quant_combine_kernel<<<p.B * p.H, 128, 0, s>>>(p);
   ++*launches;
   return cudaGetLastError();

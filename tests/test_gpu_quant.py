@@ -58,18 +58,32 @@ def fill_both(B, B_, H, d, rk, rv, n, n_max, seed, group, alibi=None, q_scale=1.
     return lay, ref, q, rows
 
 
-def unpack_codes(area: np.ndarray, rp: int, G: int, bits: int) -> np.ndarray:
-    """A block's code area (bytes) -> codes [G][rp].  Unit j of row i holds channels 8j..8j+7, channel 8j+k in bits
-    bits*k.. as code + 2^(bits-1).  4-bit: units are 32-bit words [rp/8][G].  3-bit: the low 16 bits of all units
-    ([rp/8][G] halfwords), then their high 8 bits ([rp/8][G] bytes)."""
+def unpack_codes(area: np.ndarray, rp: int, G: int, bits: int, values: bool = False) -> np.ndarray:
+    """A block's code area (bytes) -> codes [G][rp], each stored as code + 2^(bits-1).
+    3-bit: unit j of row i holds channels 8j..8j+7 (channel 8j+k in bits 3k..); the low 16 bits of all units
+    ([rp/8][G] halfwords), then their high 8 bits ([rp/8][G] bytes).
+    4-bit keys: word j of row i (channel 8j+k in bits 4k..) sits at j G + ((i + 8 (j mod 4)) mod G).
+    4-bit values: chunks of min(G, 32) rows, a chunk [rp][rows/8] words, word (c, o) = rows 8o..8o+7 of channel c."""
     nw = rp // 8
+    out = np.zeros((G, rp), dtype=np.int64)
+    if bits == 4 and values:
+        rows = min(G, 32)
+        words = area.view(np.uint32).reshape(G // rows, rp, rows // 8).astype(np.int64)
+        for k in range(8):
+            nib = ((words >> (4 * k)) & 15) - 8                     # [chunk][c][o] -> row 32 chunk + 8 o + k
+            for qc in range(G // rows):
+                for o in range(rows // 8):
+                    out[qc * rows + 8 * o + k, :] = nib[qc, :, o]
+        return out
     if bits == 4:
-        units = area.view(np.uint32).reshape(nw, G).astype(np.int64)
+        stored = area.view(np.uint32).reshape(nw, G).astype(np.int64)
+        units = np.zeros_like(stored)
+        for j in range(nw):
+            units[j, :] = stored[j, (np.arange(G) + 8 * (j % 4)) % G]
     else:
         lo = area[:2 * nw * G].view(np.uint16).reshape(nw, G).astype(np.int64)
         hi = area[2 * nw * G:3 * nw * G].reshape(nw, G).astype(np.int64)
         units = lo | (hi << 16)
-    out = np.zeros((G, rp), dtype=np.int64)
     for k in range(8):
         out[:, k::8] = ((units.T >> (bits * k)) & ((1 << bits) - 1)) - (1 << (bits - 1))
     return out
@@ -81,7 +95,7 @@ def read_block(lay, head, b, blk, G, rp_k, rp_v, bits=4):
     assert ks_off == G * rp_k * bits // 8 and vs_off - vc_off == G * rp_v * bits // 8      # exactly `bits` per element
     kc = unpack_codes(raw[:ks_off], rp_k, G, bits)
     ks = raw[ks_off:vc_off].view(np.float16)
-    vc = unpack_codes(raw[vc_off:vs_off], rp_v, G, bits)
+    vc = unpack_codes(raw[vc_off:vs_off], rp_v, G, bits, values=True)
     nvg = (rp_v + G - 1) // G
     vs = raw[vs_off:vs_off + 2 * G * nvg].view(np.float16).reshape(nvg, G).T       # -> [G][nvg]
     return kc, ks, vc, vs
