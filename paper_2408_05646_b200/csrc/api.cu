@@ -1489,7 +1489,7 @@ ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t strid
     if (hi.rp_k < min_rp) min_rp = hi.rp_k;
     if (hi.rp_v < min_rp) min_rp = hi.rp_v;
   }
-  const cudaError_t e = mma ? ea::launch_decode_quant_mma(p, max_rp, smem, s, &h->launches)
+  const cudaError_t e = mma ? ea::launch_decode_quant_mma(p, max_rp, min_rp, smem, s, &h->launches)
                             : ea::launch_decode_quant(p, max_rp, min_rp, smem, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_quant launch");

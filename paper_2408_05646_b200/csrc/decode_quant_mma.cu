@@ -54,8 +54,11 @@ struct __align__(16) MmaSmemHeader {
 constexpr int kMHeaderBytes = 1152;
 static_assert(sizeof(MmaSmemHeader) <= kMHeaderBytes, "header overlaps the warps' areas");
 
-// per warp: digits of q' s [NB][3][128] bytes, digits of the weights [NVG][4][32] bytes, o' in fp32 [128]
-__host__ __device__ constexpr int warp_area_bytes(int nb, int nvg) { return nb * 384 + nvg * 128 + 512; }
+// per warp: digits of q' s [NB][3][kDigitStride] bytes, digits of the weights [NVG][4][32] bytes, o' in fp32 [128]
+constexpr int kDigitStride = 144;        // 128 channels + 16: the three digit rows of a block start 4 banks apart
+constexpr int kQdBytes = 3 * kDigitStride;
+__host__ __device__ constexpr int warp_area_bytes(int nb, int nvg) { return nb * kQdBytes + nvg * 128 + 512; }
+__host__ __device__ constexpr int ring_offset(int nb, int nvg) { return (kMHeaderBytes + 4 * warp_area_bytes(nb, nvg) + 127) & ~127; }
 
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
@@ -80,8 +83,9 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-// NKS: 32-channel steps of the widest key row; NMT: 16-channel tiles of the widest value row; G: group size.
-template <int NKS, int NMT, int G>
+// NKS: 32-channel steps of the widest key row; NMT: 16-channel tiles of the widest value row; G: group size;
+// FULL: every head's padded key and value ranks are 16 NMT (no per-word, per-tile or per-group guards).
+template <int NKS, int NMT, int G, bool FULL>
 __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const QuantParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int gshift = G == 16 ? 4 : G == 32 ? 5 : G == 64 ? 6 : 7;
@@ -93,9 +97,9 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gid = lane >> 2, tig = lane & 3;
   unsigned char* qd = smem + kMHeaderBytes + warp * kArea;      // [NB][3][128]
-  unsigned char* pd = qd + NB * 384;                            // [NVG][4][32]
+  unsigned char* pd = qd + NB * kQdBytes;                            // [NVG][4][32]
   float* ow = reinterpret_cast<float*>(pd + NVG * 128);         // [128]
-  unsigned char* ring = smem + kMHeaderBytes + 4 * kArea;
+  unsigned char* ring = smem + ring_offset(NB, NVG);
   const int unit_i = blockIdx.x, split = blockIdx.y;
   const int h = unit_i / p.B, b = unit_i - h * p.B;
   const HeadInfo hd = p.heads[h];
@@ -103,7 +107,9 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
   const int n_b = p.deficit != nullptr ? p.n - __ldg(p.deficit + b) : p.n;      // this sequence's rows
   const int nq_b = p.qlens != nullptr ? __ldg(p.qlens + b) : p.nq;              // ... of which held as codes
   const int nqb = nq_b >> gshift;
-  const int nwk = hd.rp_k >> 3, nks = (hd.rp_k + 31) >> 5, nmt = (hd.rp_v + 15) >> 4, nvg = qh.nvg;
+  const int rp_k = FULL ? 16 * NMT : hd.rp_k, rp_v = FULL ? 16 * NMT : hd.rp_v;
+  const int nwk = rp_k >> 3, nks = FULL ? NKS : (rp_k + 31) >> 5, nmt = FULL ? NMT : (rp_v + 15) >> 4;
+  const int nvg = FULL ? NVG : qh.nvg;
   const int stage_stride = (bps * qh.block_bytes + 127) & ~127;
   const int nst_b = (nq_b + kMStageRows - 1) / kMStageRows;
   const int per = (nst_b + p.splits - 1) / p.splits;
@@ -202,6 +208,20 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
     m = mx;
   };
 
+  // what a lane's loads depend on besides the stage: word offsets of its key rows, its row, its digit positions
+  const int r0 = warp * 32, blk0 = r0 >> gshift;
+  const int rho = 8 * tig + gid;                   // the row of the warp's 32 this lane owns after the score products
+  int koff[2][2];                                  // [tile][row gid / gid + 8]: word offset in the block's key codes
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int ro = (r0 + 16 * t) & (G - 1);
+    koff[t][0] = tig * G + ((ro + gid + 8 * tig) & (G - 1));
+    koff[t][1] = tig * G + ((ro + gid + 8 + 8 * tig) & (G - 1));
+  }
+  const int kpos0 = ((lane & 1) << 4) | (((lane >> 3) & 3) << 2) | ((lane >> 1) & 3);   // channel lane + 32 k -> 32 k + kpos0
+  const int ppos = ((rho & 1) << 4) | ((rho >> 3) << 2) | ((rho >> 1) & 3);
+  const int dn = gid & 3;                          // operand columns 4..7 repeat 0..3
+
   for (int s = s_lo; s < s_hi; ++s) {
     const int it = s - s_lo, slot = it % kMStages;
     if (__any_sync(kFull, !mbar_wait(&hdr->full[slot], (it / kMStages) & 1, p.status))) {
@@ -210,21 +230,20 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
     }
     const unsigned char* st = ring + slot * stage_stride;
     const int nblk = min(bps, nqb - s * bps);
-    const int r0 = warp * 32, blk0 = r0 >> gshift;
     if (blk0 < nblk) {
       // ---- digits of x_c = q'_c s_c for the warp's block(s)
       int corr[NB];
       float delta[NB];
 #pragma unroll
       for (int i = 0; i < NB; ++i) {
-        const bool have = blk0 + i < nblk;
+        const bool have = i == 0 || blk0 + i < nblk;
         const __half* ks = reinterpret_cast<const __half*>(st + (blk0 + i) * qh.block_bytes + qh.ks_off);
         float x[NKS];
         uint32_t ab = 0;
 #pragma unroll
         for (int k = 0; k < NKS; ++k) {
           const int c = lane + 32 * k;
-          x[k] = (have && c < hd.rp_k) ? hdr->qp[c] * __half2float(ks[c]) : 0.f;
+          x[k] = (have && c < rp_k) ? hdr->qp[c] * __half2float(ks[c]) : 0.f;
           ab = max(ab, __float_as_uint(x[k]) & 0x7fffffffu);
         }
         ab = __reduce_max_sync(kFull, ab);
@@ -238,22 +257,20 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
           const int F = __float2int_rn(x[k] * sc);
           fs += F;
           const uint32_t u = static_cast<uint32_t>(F + 0x808080) ^ 0x808080u;      // three signed bytes
-          const int kpos = (c & ~31) | ((c & 1) << 4) | (((c >> 3) & 3) << 2) | ((c >> 1) & 3);
-          unsigned char* dst = qd + i * 384 + kpos;
+          unsigned char* dst = qd + i * kQdBytes + 32 * k + kpos0;
           dst[0] = static_cast<unsigned char>(u);
-          dst[128] = static_cast<unsigned char>(u >> 8);
-          dst[256] = static_cast<unsigned char>(u >> 16);
+          dst[kDigitStride] = static_cast<unsigned char>(u >> 8);
+          dst[2 * kDigitStride] = static_cast<unsigned char>(u >> 16);
         }
         corr[i] = 8 * __reduce_add_sync(kFull, fs);
       }
       __syncwarp();
       uint32_t bq[NB][NKS][2];
-      const int dn = gid & 3;                                             // columns 4..7 repeat 0..3
 #pragma unroll
       for (int i = 0; i < NB; ++i)
 #pragma unroll
         for (int k = 0; k < NKS; ++k) {
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(qd + i * 384 + (dn < 3 ? dn : 0) * 128 + 32 * k + 4 * tig);
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(qd + i * kQdBytes + (dn < 3 ? dn : 0) * kDigitStride + 32 * k + 4 * tig);
           bq[i][k][0] = dn < 3 ? src[0] : 0u;
           bq[i][k][1] = dn < 3 ? src[4] : 0u;
         }
@@ -263,16 +280,15 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
         const int bi = G == 16 ? t : 0;
-        const int ro = (r0 + 16 * t) & (G - 1);
         const uint32_t* kc = reinterpret_cast<const uint32_t*>(st + ((r0 + 16 * t) >> gshift) * qh.block_bytes);
         int acc[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int k = 0; k < NKS; ++k)
           if (k < nks) {
             const int j = 4 * k + tig;
-            const bool ok = j < nwk;
-            const uint32_t wa = ok ? kc[j * G + ((ro + gid + 8 * tig) & (G - 1))] : 0u;
-            const uint32_t wb = ok ? kc[j * G + ((ro + gid + 8 + 8 * tig) & (G - 1))] : 0u;
+            const bool ok = (FULL && 4 * k + 3 < 2 * NMT) || j < nwk;
+            const uint32_t wa = ok ? kc[4 * k * G + koff[t][0]] : 0u;
+            const uint32_t wb = ok ? kc[4 * k * G + koff[t][1]] : 0u;
             mma_u8s8(acc, wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, bq[bi][k][0], bq[bi][k][1]);
           }
         // even lanes of a pair hold digits 0 and 1 of rows gid and gid + 8, odd lanes digit 2 (and a zero column)
@@ -284,11 +300,10 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         tot[t][1] = v1 - corr[bi];
       }
       // lane (gid, tig) owns row rho = 8 tig + gid of the warp's 32: tile tig >> 1, half tig & 1
-      const int rho = 8 * tig + gid;
       const int mine = (tig & 2) ? ((tig & 1) ? tot[1][1] : tot[1][0]) : ((tig & 1) ? tot[0][1] : tot[0][0]);
       const float dl = (G == 16 && (tig & 2)) ? delta[NB - 1] : delta[0];
       const int rblk = (r0 + rho) >> gshift, ri = (r0 + rho) & (G - 1);
-      const bool valid = rblk < nblk;
+      const bool valid = NB == 1 || rblk < nblk;
       const int j_abs = s * kMStageRows + r0 + rho;
       const float score = valid ? fmaf(slope2, static_cast<float>(j_abs - pos_q), static_cast<float>(mine) * dl) : -INFINITY;
       if (__any_sync(kFull, score > m + kRaise)) rescale(warp_max(score));
@@ -301,7 +316,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
       float smax = 0.f;
 #pragma unroll
       for (int g = 0; g < NVG; ++g) {
-        const float sv = (valid && g < nvg) ? __half2float(vs[g * G]) : 0.f;
+        const float sv = (valid && (FULL || g < nvg)) ? __half2float(vs[g * G]) : 0.f;
         smax = fmaxf(smax, sv);
         wv[g] = pr * sv;
       }
@@ -313,10 +328,9 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         kappa = 1073740800.f / S;                  // 2^30 - 1024: p <= 4 keeps p s kappa below 2^32
         unit = S / 1073740800.f;
       }
-      const int ppos = ((rho & 1) << 4) | ((rho >> 3) << 2) | ((rho >> 1) & 3);
 #pragma unroll
       for (int g = 0; g < NVG; ++g)
-        if (g < nvg) {
+        if (FULL || g < nvg) {
           const uint32_t F = __float2uint_rn(wv[g] * kappa);
           sig[g] += static_cast<float>(F);
           unsigned char* dst = pd + g * 128 + ppos;
@@ -330,8 +344,8 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
 #pragma unroll
       for (int g = 0; g < NVG; ++g) {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(pd + g * 128 + dn * 32 + 4 * tig);
-        pb[g][0] = g < nvg ? src[0] : 0u;
-        pb[g][1] = g < nvg ? src[4] : 0u;
+        pb[g][0] = (FULL || g < nvg) ? src[0] : 0u;
+        pb[g][1] = (FULL || g < nvg) ? src[4] : 0u;
       }
 
       // ---- weighted sums: tiles of 16 channels, contraction over the 32 rows
@@ -342,7 +356,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         wstride = 2;
         woff = tig & 1;
       } else {
-        vw = reinterpret_cast<const uint32_t*>(st + blk0 * qh.block_bytes + qh.vc_off) + ((r0 & (G - 1)) >> 5) * hd.rp_v * 4;
+        vw = reinterpret_cast<const uint32_t*>(st + blk0 * qh.block_bytes + qh.vc_off) + ((r0 & (G - 1)) >> 5) * rp_v * 4;
         wstride = 4;
         woff = tig;
       }
@@ -351,8 +365,8 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         if (mt < nmt) {
           const int g = (16 * mt) >> gshift;
           const int c = 16 * mt + gid;
-          const uint32_t wa = c < hd.rp_v ? vw[c * wstride + woff] : 0u;
-          const uint32_t wb = c + 8 < hd.rp_v ? vw[(c + 8) * wstride + woff] : 0u;
+          const uint32_t wa = (FULL || c < rp_v) ? vw[c * wstride + woff] : 0u;
+          const uint32_t wb = (FULL || c + 8 < rp_v) ? vw[(c + 8) * wstride + woff] : 0u;
           mma_u8u8(oacc[mt], wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, pb[g][0], pb[g][1]);
         }
       if (++since_flush >= kFlushBlocks) flush();
@@ -409,7 +423,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
     if (!aborted)
 #pragma unroll
       for (int w = 0; w < 4; ++w)
-        acc = fmaf(reinterpret_cast<const float*>(smem + kMHeaderBytes + w * kArea + NB * 384 + NVG * 128)[tid], hdr->wfac[w], acc);
+        acc = fmaf(reinterpret_cast<const float*>(smem + kMHeaderBytes + w * kArea + NB * kQdBytes + NVG * 128)[tid], hdr->wfac[w], acc);
     part[4 + tid] = acc;
   }
   if (tid == 0) {
@@ -418,21 +432,21 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
   }
 }
 
-template <int NKS, int NMT, int G>
+template <int NKS, int NMT, int G, bool FULL>
 cudaError_t launch_mma_variant(const QuantParams& p, size_t smem, cudaStream_t s) {
   static size_t configured[kMaxDevices] = {};
-  const cudaError_t ec = ensure_dynamic_smem(decode_quant_mma_kernel<NKS, NMT, G>, smem, configured);
+  const cudaError_t ec = ensure_dynamic_smem(decode_quant_mma_kernel<NKS, NMT, G, FULL>, smem, configured);
   if (ec != cudaSuccess) return ec;
-  decode_quant_mma_kernel<NKS, NMT, G><<<dim3(p.B * p.H, p.splits), kMThreads, smem, s>>>(p);
+  decode_quant_mma_kernel<NKS, NMT, G, FULL><<<dim3(p.B * p.H, p.splits), kMThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 template <int NKS, int NMT>
-cudaError_t launch_mma_group(const QuantParams& p, size_t smem, cudaStream_t s) {
+cudaError_t launch_mma_group(const QuantParams& p, bool full, size_t smem, cudaStream_t s) {
   switch (p.group) {
-    case 16: return launch_mma_variant<NKS, NMT, 16>(p, smem, s);
-    case 32: return launch_mma_variant<NKS, NMT, 32>(p, smem, s);
-    case 64: return launch_mma_variant<NKS, NMT, 64>(p, smem, s);
-    default: return launch_mma_variant<NKS, NMT, 128>(p, smem, s);
+    case 16: return full ? launch_mma_variant<NKS, NMT, 16, true>(p, smem, s) : launch_mma_variant<NKS, NMT, 16, false>(p, smem, s);
+    case 32: return full ? launch_mma_variant<NKS, NMT, 32, true>(p, smem, s) : launch_mma_variant<NKS, NMT, 32, false>(p, smem, s);
+    case 64: return full ? launch_mma_variant<NKS, NMT, 64, true>(p, smem, s) : launch_mma_variant<NKS, NMT, 64, false>(p, smem, s);
+    default: return full ? launch_mma_variant<NKS, NMT, 128, true>(p, smem, s) : launch_mma_variant<NKS, NMT, 128, false>(p, smem, s);
   }
 }
 // the template arguments a layer's widest padded rank selects
@@ -448,15 +462,15 @@ size_t decode_quant_mma_smem_bytes(int max_stage_bytes, int max_rp, int group) {
   int nks, nmt;
   mma_shape(max_rp, &nks, &nmt);
   const int nvg = (16 * nmt + group - 1) / group, nb = group == 16 ? 2 : 1;
-  return kMHeaderBytes + 4 * static_cast<size_t>(warp_area_bytes(nb, nvg)) +
-         static_cast<size_t>(kMStages) * ((max_stage_bytes + 127) & ~127);
+  return ring_offset(nb, nvg) + static_cast<size_t>(kMStages) * ((max_stage_bytes + 127) & ~127);
 }
 
-cudaError_t launch_decode_quant_mma(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches) {
+cudaError_t launch_decode_quant_mma(const QuantParams& p, int max_rp, int min_rp, size_t smem, cudaStream_t s,
+                                    uint64_t* launches) {
   cudaError_t e;
-  if (max_rp <= 64) e = launch_mma_group<2, 4>(p, smem, s);
-  else if (max_rp <= 80) e = launch_mma_group<3, 5>(p, smem, s);
-  else e = launch_mma_group<4, 8>(p, smem, s);
+  if (max_rp <= 64) e = launch_mma_group<2, 4>(p, min_rp == 64, smem, s);
+  else if (max_rp <= 80) e = launch_mma_group<3, 5>(p, min_rp == 80, smem, s);
+  else e = launch_mma_group<4, 8>(p, min_rp == 128, smem, s);
   if (e != cudaSuccess) return e;
   ++*launches;
   return launch_quant_combine(p, s, launches);

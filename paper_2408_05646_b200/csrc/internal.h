@@ -317,7 +317,8 @@ cudaError_t launch_decode_quant(const QuantParams& p, int max_rp, int min_rp, si
                                 uint64_t* launches);   // min_rp: narrowest padded rank over heads and K/V
 // 4-bit codes: the integer tensor-core kernel
 size_t decode_quant_mma_smem_bytes(int max_stage_bytes, int max_rp, int group);
-cudaError_t launch_decode_quant_mma(const QuantParams& p, int max_rp, size_t smem, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_decode_quant_mma(const QuantParams& p, int max_rp, int min_rp, size_t smem, cudaStream_t s,
+                                    uint64_t* launches);   // min_rp: narrowest padded rank over heads and K/V
 cudaError_t launch_quant_combine(const QuantParams& p, cudaStream_t s, uint64_t* launches);
 
 // Built-in scratch for eigen_attn_decode_static: device address and capacity (in floats) of the
