@@ -1461,7 +1461,7 @@ ea_status eigen_attn_decode_quant(eigen_attn_t h, const void* d_q, int64_t strid
   // CTAs per unit: waves of (SMs x resident CTAs), a start-up worth a few stages per CTA, and room for
   // units x splits partials in the workspace
   int ctas_per_sm = static_cast<int>(static_cast<size_t>(228 * 1024) / (smem + 1024));
-  const int reg_limit = mma ? 4 : max_rp <= 80 ? 3 : 2;
+  const int reg_limit = mma ? 5 : max_rp <= 80 ? 3 : 2;
   if (ctas_per_sm > reg_limit) ctas_per_sm = reg_limit;
   if (ctas_per_sm < 1) ctas_per_sm = 1;
   const int64_t units = static_cast<int64_t>(p.B) * p.H;

@@ -5,9 +5,10 @@
 //   o'_c    = sum_i (n_ic - 8) s_ig p_i          s_ig = value scale of row i and channel group g, p_i = 2^(score_i - m)
 //
 // Both sums are 8-bit integer products with 32-bit accumulators (mma.sync m16n8k32).  A nibble word becomes two
-// operand registers with one shift and two masks (w & 0x0F0F0F0F holds nibbles 0, 2, 4, 6 as bytes, (w >> 4) & ...
-// nibbles 1, 3, 5, 7).  The real-valued factor goes into the other operand as fixed-point digits, one digit per
-// operand column:
+// operand registers with two masks and no shift: w & 0x0F0F0F0F holds nibbles 0, 2, 4, 6 as bytes, w & 0xF0F0F0F0
+// holds 16 times nibbles 1, 3, 5, 7; the factor 16 is taken out of the other operand (the fixed-point value of an
+// odd channel, or of an odd row in the second product, is formed with a 16 times smaller scale, so it has four bits
+// fewer).  The real-valued factor goes into the other operand as fixed-point digits, one digit per operand column:
 //   keys:   x_c = q'_c s_c of a block -> F_c = rint(x_c 2^19 / 2^E) with 2^E above the block's largest |x_c|;
 //           the three signed bytes of F_c are columns 0..2, score = 2^(E-19) (sum_n 256^n D_n - 8 sum_c F_c).
 //   values: w_ig = p_i s_ig -> F = rint(w_ig kappa), an unsigned 32-bit integer whose four bytes are columns 0..3;
@@ -36,12 +37,12 @@ namespace {
 using namespace tc;
 
 constexpr int kMThreads = 128;
-constexpr int kMStages = 4;
+constexpr int kMStages = 3;
 constexpr int kMStageRows = 128;
-constexpr uint32_t kNib = 0x0F0F0F0Fu;
+constexpr uint32_t kNib = 0x0F0F0F0Fu, kNibHi = 0xF0F0F0F0u;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kRaise = 2.f;            // the running maximum is raised when a score exceeds it by this much
-constexpr int kFlushBlocks = 2048;       // 2048 x 32 rows x 15 x 255 < 2^31
+constexpr int kFlushBlocks = 1024;       // 1024 blocks x (16 rows x 240 + 16 rows x 15) x 255 < 2^30
 
 struct __align__(16) MmaSmemHeader {
   unsigned long long full[kMStages];
@@ -86,7 +87,7 @@ __device__ __forceinline__ float warp_max(float v) {
 // NKS: 32-channel steps of the widest key row; NMT: 16-channel tiles of the widest value row; G: group size;
 // FULL: every head's padded key and value ranks are 16 NMT (no per-word, per-tile or per-group guards).
 template <int NKS, int NMT, int G, bool FULL>
-__global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const QuantParams p) {
+__global__ void __launch_bounds__(kMThreads, 5) decode_quant_mma_kernel(const QuantParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   constexpr int gshift = G == 16 ? 4 : G == 32 ? 5 : G == 64 ? 6 : 7;
   constexpr int bps = kMStageRows >> gshift;                    // blocks per stage
@@ -176,7 +177,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
     float sg[NVG];
 #pragma unroll
     for (int g = 0; g < NVG; ++g) {
-      sg[g] = warp_sum(sig[g]);
+      sg[g] = warp_sum((gid & 1) ? 16.f * sig[g] : sig[g]);
       sig[g] = 0.f;
     }
 #pragma unroll
@@ -221,6 +222,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
   const int kpos0 = ((lane & 1) << 4) | (((lane >> 3) & 3) << 2) | ((lane >> 1) & 3);   // channel lane + 32 k -> 32 k + kpos0
   const int ppos = ((rho & 1) << 4) | ((rho >> 3) << 2) | ((rho >> 1) & 3);
   const int dn = gid & 3;                          // operand columns 4..7 repeat 0..3
+  const int odd4 = (lane & 1) << 2;                // channel lane + 32 k is odd: its fixed-point value is 16 times coarser
 
   for (int s = s_lo; s < s_hi; ++s) {
     const int it = s - s_lo, slot = it % kMStages;
@@ -248,14 +250,15 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         }
         ab = __reduce_max_sync(kFull, ab);
         const int e = max(static_cast<int>(ab >> 23), 40);               // every |x| < 2^(e - 126)
-        const float sc = __uint_as_float(static_cast<uint32_t>(272 - e) << 23);    // 2^(19 - (e - 126))
+        // 2^(19 - (e - 126)); odd channels meet 16 n in the product and take 2^(15 - (e - 126))
+        const float sc = __uint_as_float(static_cast<uint32_t>(272 - e - odd4) << 23);
         delta[i] = __uint_as_float(static_cast<uint32_t>(e - 18) << 23);           // 2^((e - 126) - 19)
         int fs = 0;
 #pragma unroll
         for (int k = 0; k < NKS; ++k) {
           const int c = lane + 32 * k;
           const int F = __float2int_rn(x[k] * sc);
-          fs += F;
+          fs += F << odd4;
           const uint32_t u = static_cast<uint32_t>(F + 0x808080) ^ 0x808080u;      // three signed bytes
           unsigned char* dst = qd + i * kQdBytes + 32 * k + kpos0;
           dst[0] = static_cast<unsigned char>(u);
@@ -289,7 +292,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
             const bool ok = (FULL && 4 * k + 3 < 2 * NMT) || j < nwk;
             const uint32_t wa = ok ? kc[4 * k * G + koff[t][0]] : 0u;
             const uint32_t wb = ok ? kc[4 * k * G + koff[t][1]] : 0u;
-            mma_u8s8(acc, wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, bq[bi][k][0], bq[bi][k][1]);
+            mma_u8s8(acc, wa & kNib, wb & kNib, wa & kNibHi, wb & kNibHi, bq[bi][k][0], bq[bi][k][1]);
           }
         // even lanes of a pair hold digits 0 and 1 of rows gid and gid + 8, odd lanes digit 2 (and a zero column)
         const int ka = (tig & 1) ? 65536 : 1, kb = (tig & 1) ? 0 : 256;
@@ -325,7 +328,8 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
         flush();
         const uint32_t e = max(sb >> 23, 64u);
         S = __uint_as_float((e + 1u) << 23);       // a power of two above every scale so far
-        kappa = 1073740800.f / S;                  // 2^30 - 1024: p <= 4 keeps p s kappa below 2^32
+        // 2^30 - 1024: p <= 4 keeps p s kappa below 2^32; odd rows meet 16 n in the product and take kappa / 16
+        kappa = ((gid & 1) ? 67108800.f : 1073740800.f) / S;
         unit = S / 1073740800.f;
       }
 #pragma unroll
@@ -367,7 +371,7 @@ __global__ void __launch_bounds__(kMThreads, 4) decode_quant_mma_kernel(const Qu
           const int c = 16 * mt + gid;
           const uint32_t wa = (FULL || c < rp_v) ? vw[c * wstride + woff] : 0u;
           const uint32_t wb = (FULL || c + 8 < rp_v) ? vw[(c + 8) * wstride + woff] : 0u;
-          mma_u8u8(oacc[mt], wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, pb[g][0], pb[g][1]);
+          mma_u8u8(oacc[mt], wa & kNib, wb & kNib, wa & kNibHi, wb & kNibHi, pb[g][0], pb[g][1]);
         }
       if (++since_flush >= kFlushBlocks) flush();
     }
