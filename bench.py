@@ -639,7 +639,7 @@ def workload_table(device, binding, lay2, wl2, ranks2, q2, k2, v2, steps=30, war
         nq = n2 // G * G
         codes = wl2.batch * (nq // G) * sum(lay2.quant_layout(h)[1] for h in range(wl2.n_heads))
         tail = wl2.batch * (n2 + 1 - nq) * row_bytes
-        table[f"quant_{bits}bit_g{G}"] = table_entry("decode_quant_kernel", k_us, s_us, codes + tail, peak,
+        table[f"quant_{bits}bit_g{G}"] = table_entry("decode_quant_mma_kernel" if bits == 4 else "decode_quant_kernel", k_us, s_us, codes + tail, peak,
                                                      workload=wl2.name + f", {bits}-bit codes, group {G}",
                                                      bytes_16bit=algorithmic_bytes(wl2, ranks2, ranks2, n2 + 1))
         lay2.quant_detach()
@@ -1091,7 +1091,7 @@ def run_quant(args, wl):
                    "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "bits": 4, "group": G,
                    "quantised_rows": nq, "cache_gb": bytes_step / 1e9, "cache_gb_16bit": bytes_16bit / 1e9,
                    "l2": "inputs larger than L2: every step streams all codes"},
-        "roofline": {"bound": "hbm", "kernel": "decode_quant_kernel (+ combine)", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_quant_mma_kernel (+ combine)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "kernel_us": kern * 1e3,
                      "algorithmic_bytes": bytes_step, "traffic": None},
         "decode_16bit_us": ms_16bit * 1e3, "speedup_over_16bit": ms_16bit / (kern if kern > 0 else ms),

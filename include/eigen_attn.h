@@ -227,12 +227,17 @@ ea_status eigen_attn_set_rope(eigen_attn_t h, double base, int32_t interleaved, 
  *               codes and 16-bit tail.
  * quant_layout: where head `head` lives in the buffer: byte offset of its slab [B][n_max / group][block_bytes],
  *               and inside a block the offsets of the key scales [rp_k] halves, the value codes and the value
- *               scales [ceil(rp_v / group)][group] halves; key codes sit at offset 0.  A code area is [rp / 8][group]
- *               units, unit j of row i holding channels 8j..8j+7.  4-bit: a unit is a 32-bit word, channel 8j+k in
- *               bits 4k..4k+3 as c + 8.  3-bit: a unit is 24 bits, channel 8j+k in bits 3k..3k+2 as c + 4, kept as
- *               two planes: the low 16 bits of all units ([rp / 8][group] halfwords), then their high 8 bits
- *               ([rp / 8][group] bytes).  Keys therefore cost exactly bits + 16/group bits per (padded) element,
- *               the accounting behind Table 8; a value row pays one scale per started group of its rp_v channels. */
+ *               scales [ceil(rp_v / group)][group] halves; key codes sit at offset 0.
+ *               3-bit: a code area is [rp / 8][group] units, unit j of row i holding channels 8j..8j+7 in 24 bits,
+ *               channel 8j+k in bits 3k..3k+2 as c + 4, kept as two planes: the low 16 bits of all units
+ *               ([rp / 8][group] halfwords), then their high 8 bits ([rp / 8][group] bytes).
+ *               4-bit: units are 32-bit words of eight nibbles, each c + 8, ordered for the operand fragments of the
+ *               integer tensor-core products of decode_quant.  Keys: word j of row i holds channels 8j..8j+7
+ *               (channel 8j+k in bits 4k..4k+3) and sits at word j * group + ((i + 8 * (j mod 4)) mod group).
+ *               Values: chunks of min(group, 32) rows; a chunk is [rp_v][rows / 8] words, word (c, o) holding rows
+ *               8o..8o+7 of channel c (row 8o+k in bits 4k..4k+3).
+ *               Keys therefore cost exactly bits + 16/group bits per (padded) element, the accounting behind
+ *               Table 8; a value row pays one scale per started group of its rp_v channels. */
 ea_status eigen_attn_quant_bytes(eigen_attn_t h, int32_t bits, int32_t group, size_t* bytes);
 ea_status eigen_attn_quant_attach(eigen_attn_t h, int32_t bits, int32_t group, void* d_qcache, size_t bytes,
                                   void* cuda_stream);

@@ -207,6 +207,55 @@ def test_decode_quant_with_peaked_attention_and_alibi(B, bits):
     assert_close(out, want, BF16, "peaked + alibi")
 
 
+def scaled_case(B, B_, H, d, r, n, seed, G, k_gain, v_gain, q_scale=1.0):
+    """A layer whose rank-space rows are those of rank_space_case times per-channel key gains [r] and per-row
+    value gains [n] (exact powers of two, so the 16-bit rows stay exact), on both sides."""
+    U_k, U_v, q, kp, vp, _ = rank_space_case(B_, H, d, [r] * H, [r] * H, n, seed, q_scale)
+    kg = torch.tensor(k_gain, dtype=torch.float32).cuda()
+    vg = torch.tensor(v_gain, dtype=torch.float32).cuda()
+    kp = (kp.float() * kg.repeat(H)[None, None, :]).to(BF16)
+    vp = (vp.float() * vg[None, :, None]).to(BF16)
+    lay = B.EigenAttnLayer(B_, H, d, n, BF16, U_k, U_v)
+    lay.append_kv(kp, vp, preprojected=True)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    for b in range(B_):
+        for h in range(H):
+            ref.Kp[(b, h)] = kp[b, :, h * r:(h + 1) * r].double().cpu().numpy()
+            ref.Vp[(b, h)] = vp[b, :, h * r:(h + 1) * r].double().cpu().numpy()
+    ref.set_len(n)
+    lay.quant_attach(4, G)
+    lay.quant_sync()
+    return lay, ref, q
+
+
+def test_decode_quant_scales_that_grow_and_spread(B):
+    """Value scales that grow by 2^14 along the sequence (the fixed-point unit of the weights has to follow them,
+    folding what was accumulated under the old unit) and key channels whose scales spread over 2^10 (the digits of
+    q' s are taken relative to the largest channel of a block)."""
+    B_, H, d, r, G, n = 2, 2, 128, 80, 32, 2048 + 64
+    k_gain = [2.0 ** -(c // 8) for c in range(r)]
+    v_gain = [2.0 ** (i // 150 - 14) for i in range(n)]          # the last rows, which carry the output, have gain 1
+    lay, ref, q = scaled_case(B, B_, H, d, r, n, 177, G, k_gain, v_gain)
+    out = lay.decode_quant(q)
+    lay.poll_status()
+    res = ref.decode_quant(to_np(q), 4, G)
+    want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out, want, BF16, "growing value scales, spread key scales")
+
+
+def test_decode_quant_one_cta_over_more_blocks_than_one_fold(B):
+    """One CTA per unit over 140 000 rows: every warp meets more blocks than the integer accumulators may take
+    before they are folded into fp32, so the periodic fold runs."""
+    B_, H, d, r, G, n = 1, 1, 128, 80, 32, 140000
+    lay, ref, q = scaled_case(B, B_, H, d, r, n, 178, G, [1.0] * r, [1.0] * n)
+    lay.set_option(B.EA_OPT_DECODE_CTAS, 1)
+    out = lay.decode_quant(q)
+    lay.poll_status()
+    res = ref.decode_quant(to_np(q), 4, G)
+    want = np.stack([np.stack([res[(b, h)] for h in range(H)]) for b in range(B_)])[:, None]
+    assert_close(out, want, BF16, "one CTA, 1094 stages")
+
+
 def test_decode_quant_merged_weight_flags(B):
     B_, H, d, G, n = 2, 2, 128, 32, 500
     lay, ref, q, _ = fill_both(B, B_, H, d, [80, 56], [72, 80], n, n, 175, G)
