@@ -700,7 +700,7 @@ def workload_table_own_layers(device, binding, steps=30, warmup=3):
     def step_gqa():
         lay.set_len(wl.context); lay.append_kv(kn, vn); lay.decode_gqa(q, g, out=out)
     k_us, s_us = timed_kernel(lay, device, step_gqa, steps, warmup)
-    table[wl.name] = table_entry("decode_gqa_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
+    table[wl.name] = table_entry("decode_gqa_mma_kernel", k_us, s_us, algorithmic_bytes(wl, ranks, ranks, wl.context + 1), peak,
                                  group=g)
     # the same layer with the rotary embedding these models use (the bytes counted are the rows of the cache, read once)
     lay.set_rope(10000.0)
@@ -993,7 +993,7 @@ def run_gqa(args, wl):
         "config": {"workload": wl.name, "batch": wl.batch, "kv_heads": wl.n_heads, "group": g, "d_head": wl.d_head,
                    "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "cache_gb": bytes_step / 1e9,
                    "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
-        "roofline": {"bound": "hbm", "kernel": "decode_gqa_rope_kernel" if rope else "decode_gqa_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "decode_gqa_rope_kernel" if rope else "decode_gqa_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "kernel_us": kern * 1e3,
                      "algorithmic_bytes": bytes_step, "traffic": None},
         "one_query_head_at_a_time_us": ms_one_by_one * 1e3,

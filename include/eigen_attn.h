@@ -326,6 +326,9 @@ typedef enum {
   EA_OPT_DECODE_MIN_COPY_BYTES = 8, /* split-KV decode: heads whose K' or V' tile is smaller than this many bytes
                                  put up to four consecutive tiles into one ring slot, i.e. one bulk copy;
                                  -1 = the default (16 KiB), 0 = always one tile per slot                     */
+  EA_OPT_GQA_IMPL = 9,        /* eigen_attn_decode_gqa without a rotary embedding: 0 = automatic (warp-level mma.sync
+                                 products where every padded key rank is a multiple of 16 and d_head <= 128, else the
+                                 tcgen05 kernel), 1 = always the tcgen05 kernel                              */
   EA_OPT_TEST_WAIT_GIVES_UP = 7 /* failure-path test hook.  1 arms it for the NEXT eigen_attn_decode /
                                  _decode_step / _decode_static launch only: one warp of one CTA treats its
                                  first wait for a tile as having exceeded the bound.  The launch then ends the

@@ -27,6 +27,7 @@ EA_OPT_DECODE_FUSED = 5
 EA_OPT_PREFILL_PROJECT = 6
 EA_OPT_TEST_WAIT_GIVES_UP = 7
 EA_OPT_DECODE_MIN_COPY_BYTES = 8
+EA_OPT_GQA_IMPL = 9
 
 STATUS_NAMES = {0: "EA_OK", -1: "EA_ERR_INVALID_ARG", -2: "EA_ERR_SHAPE", -3: "EA_ERR_CAPACITY",
                 -4: "EA_ERR_UNSUPPORTED", -5: "EA_ERR_CUDA", -6: "EA_ERR_TIMEOUT",

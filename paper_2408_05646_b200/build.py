@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libeigenattn.so")
-SOURCES = ["api.cu", "append.cu", "decode.cu", "decode_gqa.cu", "decode_rope.cu", "decode_quant_mma.cu", "kv_quant.cu", "prefill_simt.cu", "prefill_rope.cu", "prefill_tc.cu", "prefill_tc_ws.cu", "project_tc.cu", "project_tc_stream.cu", "rope_lift_tc.cu"]
+SOURCES = ["api.cu", "append.cu", "decode.cu", "decode_gqa.cu", "decode_gqa_mma.cu", "decode_rope.cu", "decode_quant_mma.cu", "kv_quant.cu", "prefill_simt.cu", "prefill_rope.cu", "prefill_tc.cu", "prefill_tc_ws.cu", "project_tc.cu", "project_tc_stream.cu", "rope_lift_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

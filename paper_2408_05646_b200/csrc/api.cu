@@ -250,6 +250,7 @@ struct eigen_attn {
   std::vector<int32_t> page_cap;      // [B]: rows sequence b can hold = leading mapped pages * page_rows
   int64_t opt_min_copy = -1;  // EA_OPT_DECODE_MIN_COPY_BYTES; < 0 = the built-in default
   int64_t opt_give_up = 0;   // EA_OPT_TEST_WAIT_GIVES_UP: armed for the next split-KV decode launch
+  int64_t opt_gqa_impl = 0;  // EA_OPT_GQA_IMPL
   uint64_t launches = 0;
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   // quantised copy of the cache (Section 5.3), attached by the caller
@@ -1212,7 +1213,20 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table (without a rotary embedding)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
-  const size_t smem = rope_tc ? ea::decode_gqa_rope_smem_bytes(L.max_rp_k, h->desc.d_head) : ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
+  // without a rotary embedding: warp-level products where every rank is a multiple of 16 (EA_OPT_GQA_IMPL = 1 keeps
+  // the tcgen05 kernel)
+  const int max_rp = L.max_rp_k > L.max_rp_v ? L.max_rp_k : L.max_rp_v;
+  int min_rp = max_rp;
+  bool ranks16 = true;
+  for (const HeadInfo& hi : L.heads) {
+    if (hi.rp_k < min_rp) min_rp = hi.rp_k;
+    if (hi.rp_v < min_rp) min_rp = hi.rp_v;
+    if (hi.rp_k % 16) ranks16 = false;
+  }
+  const bool warp_mma = !rope_tc && h->opt_gqa_impl != 1 && ranks16 && h->desc.d_head <= 128 &&
+                        ea::decode_gqa_mma_smem_bytes(max_rp, max_rp) != 0;
+  const size_t smem = rope_tc ? ea::decode_gqa_rope_smem_bytes(L.max_rp_k, h->desc.d_head)
+                      : warp_mma ? ea::decode_gqa_mma_smem_bytes(max_rp, max_rp) : ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
   if (smem > static_cast<size_t>(kSmemLimit)) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: tiles do not fit");
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   ea::GqaDecodeParams p{};
@@ -1256,7 +1270,8 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
     p.interleaved = h->rope_interleaved;
   }
   const cudaError_t e = rope_tc ? ea::launch_decode_gqa_rope(p, L.max_rp_k, s, &h->launches)
-                                : ea::launch_decode_gqa(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
+                        : warp_mma ? ea::launch_decode_gqa_mma(p, max_rp, min_rp, s, &h->launches)
+                                   : ea::launch_decode_gqa(p, L.max_rp_k, L.max_rp_v, s, &h->launches);
   if (h->ev_stop) cudaEventRecord(h->ev_stop, s);
   if (e != cudaSuccess) return cuda_fail(h, e, "decode_gqa launch");
   return EA_OK;
@@ -1530,6 +1545,10 @@ ea_status eigen_attn_set_option(eigen_attn_t h, int32_t option, int64_t value) {
     case EA_OPT_DECODE_MIN_COPY_BYTES:
       if (value < -1 || value > (1 << 20)) return fail(h, EA_ERR_INVALID_ARG, "DECODE_MIN_COPY_BYTES %lld", static_cast<long long>(value));
       h->opt_min_copy = value;
+      return EA_OK;
+    case EA_OPT_GQA_IMPL:
+      if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "GQA_IMPL %lld", static_cast<long long>(value));
+      h->opt_gqa_impl = value;
       return EA_OK;
     case EA_OPT_TEST_WAIT_GIVES_UP:
       if (value < 0 || value > 1) return fail(h, EA_ERR_INVALID_ARG, "TEST_WAIT_GIVES_UP %lld", static_cast<long long>(value));

@@ -886,6 +886,12 @@ cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp
 
 // Shared memory of decode_gqa_rope_kernel; 0 where it does not fit (wide ranks: the caller then serves every query
 // head as a unit of the multi-head rotary kernel).
+cudaError_t launch_gqa_combine(const GqaDecodeParams& p, cudaStream_t s, uint64_t* launches) {
+  gqa_combine_kernel<<<p.B * p.H * p.group, 128, 0, s>>>(p);
+  ++*launches;
+  return cudaGetLastError();
+}
+
 size_t decode_gqa_rope_smem_bytes(int max_rp_k, int d_head) {
   const int k16 = (max_rp_k + 15) & ~15;
   const size_t bytes = kGrHeader + static_cast<size_t>(gr_kb(kMaxGroup * d_head * 2)) + 2 * kMaxGroup * kTile * 2 +

@@ -293,6 +293,10 @@ size_t decode_gqa_smem_bytes(int max_rp_k, int max_rp_v);
 size_t decode_gqa_rope_smem_bytes(int max_rp_k, int d_head);
 cudaError_t launch_decode_gqa_rope(const GqaDecodeParams& p, int max_rp_k, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_decode_gqa(const GqaDecodeParams& p, int max_rp_k, int max_rp_v, cudaStream_t s, uint64_t* launches);
+// grouped queries with warp-level products (ranks that are multiples of 16, d_head <= 128); 0 bytes = does not fit
+size_t decode_gqa_mma_smem_bytes(int max_rp_k, int max_rp_v);
+cudaError_t launch_decode_gqa_mma(const GqaDecodeParams& p, int max_rp, int min_rp, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_gqa_combine(const GqaDecodeParams& p, cudaStream_t s, uint64_t* launches);
 size_t decode_rope_smem_bytes(int max_rp_k, int max_rp_v, int d_head);
 // bytes of the rotary constants a layer keeps: inverse frequencies (64 doubles), per-tile steps (64 float2),
 // the row-offset table (32 x 128 float4)

@@ -33,11 +33,13 @@ def group_queries(B_, H, g, d, seed):
     (2, 1, 128, [64, 64], [64, 64], 3000),                          # group 1 = multi-head attention
     (2, 5, 128, [80, 80], [80, 80], 9000),                          # a group that is not a power of two
 ])
-def test_gqa_decode_matches_oracle(B, H, g, d, rk, rv, n):
+@pytest.mark.parametrize("impl", [0, 1])               # 0: warp-level products where the ranks allow, 1: the tcgen05 kernel
+def test_gqa_decode_matches_oracle(B, H, g, d, rk, rv, n, impl):
     B_ = 2
     U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n, BF16, seed_cfg=161)
     q = group_queries(B_, H, g, d, 161)
     lay = B.EigenAttnLayer(B_, H, d, n + 4, BF16, U_k, U_v)
+    lay.set_option(B.EA_OPT_GQA_IMPL, impl)
     lay.append_kv(k, v)
     ref = oracle_layer(B_, H, d, U_k, U_v)
     ref.append_kv(to_np(k), to_np(v))
@@ -52,7 +54,8 @@ def test_gqa_decode_matches_oracle(B, H, g, d, rk, rv, n):
     lay.poll_status()
 
 
-def test_gqa_peaked_attention_and_steps(B):
+@pytest.mark.parametrize("impl", [0, 1])
+def test_gqa_peaked_attention_and_steps(B, impl):
     """Sharply peaked weights (queries scaled by 6) over several appended tokens: an error in a handful of rows
     or in one query of the group shows up here."""
     from helpers import OraclePair
@@ -60,6 +63,7 @@ def test_gqa_peaked_attention_and_steps(B):
     rk, rv = [80, 48], [64, 80]
     U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n + steps, BF16, seed_cfg=163)
     lay = B.EigenAttnLayer(B_, H, d, n + steps, BF16, U_k, U_v)
+    lay.set_option(B.EA_OPT_GQA_IMPL, impl)
     lay.append_kv(k[:, :n], v[:, :n])
     ref = OraclePair(B_, H, d, U_k, U_v, BF16)
     ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
