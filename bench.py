@@ -929,6 +929,8 @@ def run_gqa(args, wl):
     rope = {"base": 10000.0, "interleaved": False} if args.rope else None
     if rope:                                       # Section 4.3 for the group: the form the Llama-3 models run
         lay.set_rope(rope["base"])
+    lay.set_option(binding.EA_OPT_GQA_IMPL, args.gqa_impl)
+    gqa_kernel = "decode_gqa_rope_kernel" if rope else "decode_gqa_kernel" if args.gqa_impl == 1 else "decode_gqa_mma_kernel"
 
     def step():
         lay.set_len(n0)
@@ -993,7 +995,7 @@ def run_gqa(args, wl):
         "config": {"workload": wl.name, "batch": wl.batch, "kv_heads": wl.n_heads, "group": g, "d_head": wl.d_head,
                    "rank": sorted(set(ranks)), "context": n0, "new_tokens": 1, "cache_gb": bytes_step / 1e9,
                    "l2": "inputs larger than L2: every step streams the whole rank-r cache"},
-        "roofline": {"bound": "hbm", "kernel": "decode_gqa_rope_kernel" if rope else "decode_gqa_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": gqa_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "kernel_us": kern * 1e3,
                      "algorithmic_bytes": bytes_step, "traffic": None},
         "one_query_head_at_a_time_us": ms_one_by_one * 1e3,
@@ -1119,6 +1121,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaled-down profiling case)")
     ap.add_argument("--context", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--prefill-impl", type=int, default=0, help="prefill workload: 0 auto, 1 CUDA-core, 2 tcgen05 kernel")
+    ap.add_argument("--gqa-impl", type=int, default=0, choices=[0, 1],
+                    help="grouped-query workload: 0 auto (warp-level products), 1 the tcgen05 kernel")
     args = ap.parse_args()
     VARIANT["alibi"] = bool(args.alibi)
     VARIANT["rope"] = bool(args.rope)
