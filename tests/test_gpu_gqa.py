@@ -32,6 +32,8 @@ def group_queries(B_, H, g, d, seed):
     (1, 16, 128, [80], [80], 17),                                   # largest group, shorter than a tile
     (2, 1, 128, [64, 64], [64, 64], 3000),                          # group 1 = multi-head attention
     (2, 5, 128, [80, 80], [80, 80], 9000),                          # a group that is not a power of two
+    (3, 3, 64, [32, 64, 16], [16, 48, 64], 2100),                   # small d_head, ranks that are multiples of 16, per head
+    (1, 12, 128, [128], [128], 1500),                               # more than 8 queries on the widest rank
 ])
 @pytest.mark.parametrize("impl", [0, 1])               # 0: warp-level products where the ranks allow, 1: the tcgen05 kernel
 def test_gqa_decode_matches_oracle(B, H, g, d, rk, rv, n, impl):
