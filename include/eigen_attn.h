@@ -177,8 +177,11 @@ ea_status eigen_attn_set_alibi(eigen_attn_t h, const float* slopes, void* cuda_s
  * otherwise).  With a rotary embedding set (the Llama models: Section 4.3 per query head) the keys of a tile are
  * lifted and turned once for the whole group and scored on the tensor cores (fp16 operand tiles: turned keys and
  * scaled queries must stay below 65504); where the tiles do not fit shared memory (r_k above 96 at d_head 128) or a
- * page table is set, every query head is served as its own unit of the multi-head rotary kernel.  The partials of batch x n_heads x group x splits must fit the workspace
- * (EA_ERR_CAPACITY).  Attends over the rows the cache holds: append the new token's rows first. */
+ * page table is set, every query head is served as its own unit of the multi-head rotary kernel.  Without a rotary
+ * embedding a page table is followed where every padded key rank is a multiple of 16 and d_head <= 128 (the
+ * warp-level kernel, see EA_OPT_GQA_IMPL; EA_ERR_UNSUPPORTED otherwise).  The partials of batch x n_heads x group x
+ * splits must fit the workspace (EA_ERR_CAPACITY).  Attends over the rows the cache holds: append the new token's
+ * rows first. */
 ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_b_q, int32_t group, void* d_out,
                                 int64_t stride_b_out, void* cuda_stream);
 

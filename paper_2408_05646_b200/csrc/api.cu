@@ -1210,7 +1210,6 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   const bool rope_tc = h->rope && !h->paged && group > 1 && ea::decode_gqa_rope_smem_bytes(h->L.max_rp_k, h->desc.d_head) != 0;
   if (h->rope && !rope_tc)
     return do_decode_rope(h, d_q, stride_b_q, d_out, stride_b_out, 0u, static_cast<cudaStream_t>(cuda_stream), group);
-  if (h->paged) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: not available with a page table (without a rotary embedding)");
   const Layout& L = h->L;
   const int B = h->desc.batch, H = h->desc.n_heads, n = h->len;
   // without a rotary embedding: warp-level products where every rank is a multiple of 16 (EA_OPT_GQA_IMPL = 1 keeps
@@ -1225,6 +1224,9 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   }
   const bool warp_mma = !rope_tc && h->opt_gqa_impl != 1 && ranks16 && h->desc.d_head <= 128 &&
                         ea::decode_gqa_mma_smem_bytes(max_rp, max_rp) != 0;
+  if (h->paged && !warp_mma)
+    return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: with a page table the ranks must be multiples of 16 and d_head <= 128 "
+                                       "(EA_OPT_GQA_IMPL = 0)");
   const size_t smem = rope_tc ? ea::decode_gqa_rope_smem_bytes(L.max_rp_k, h->desc.d_head)
                       : warp_mma ? ea::decode_gqa_mma_smem_bytes(max_rp, max_rp) : ea::decode_gqa_smem_bytes(L.max_rp_k, L.max_rp_v);
   if (smem > static_cast<size_t>(kSmemLimit)) return fail(h, EA_ERR_UNSUPPORTED, "decode_gqa: tiles do not fit");
@@ -1236,6 +1238,7 @@ ea_status eigen_attn_decode_gqa(eigen_attn_t h, const void* d_q, int64_t stride_
   p.status = dev_status(h);
   p.tmaps = h->ws + L.off_tmaps;
   p.deficit = dev_deficit(h);
+  p.pages = dev_pages(h);
   p.part_stride = L.part_stride;
   p.B = B; p.H = H; p.d_head = h->desc.d_head; p.n = n; p.n_max = h->desc.n_max;
   p.nt = (n + 127) / 128;

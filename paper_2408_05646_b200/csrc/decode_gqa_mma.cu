@@ -4,7 +4,8 @@
 // With at most 16 queries per K/V head the two products of a tile are thin: S^T has 16 rows, of which `group`
 // are real.  The kernel is bound by the bytes of K' and V', so what matters is that the tiles stream without a
 // stall; a product per warp, issued by the warp that consumes it, has no hand-over between threads at all:
-//   * K' and V' tiles of 128 rows arrive row-major, as they lie in the cache, through a ring of bulk copies;
+//   * K' and V' tiles of 128 rows arrive row-major, as they lie in the cache (or in the page that holds them),
+//     through a ring of bulk copies;
 //   * a warp owns 32 rows of every tile: S = Q' K'^T (A = Q' fragments, loaded once per CTA; B = K' rows, ldmatrix),
 //     online softmax on the accumulator fragments, which are at the same time the A fragments of the second
 //     product, O' += P V' (B = V' rows through ldmatrix.trans);
@@ -86,8 +87,8 @@ __global__ void __launch_bounds__(kGmThreads, 2) decode_gqa_mma_kernel(const Gqa
   const int nt_b = (n_b + kGmTile - 1) / kGmTile;
   const int per = (nt_b + p.splits - 1) / p.splits;
   const int t_lo = min(nt_b, split * per), t_hi = min(nt_b, t_lo + per);
-  const char* k_rows = p.cache + hd.k_off + static_cast<int64_t>(b) * p.n_max * kb;
-  const char* v_rows = p.cache + hd.v_off + static_cast<int64_t>(b) * p.n_max * vb;
+  const char* k_slab = p.cache + hd.k_off;
+  const char* v_slab = p.cache + hd.v_off;
 
   if (tid == 0) {
     for (int s = 0; s < kGmMaxStages; ++s) {
@@ -103,9 +104,9 @@ __global__ void __launch_bounds__(kGmThreads, 2) decode_gqa_mma_kernel(const Gqa
     const int rows = min(kGmTile, n_b - t * kGmTile);
     unsigned char* dst = ring + slot * stage_bytes;
     mbar_arrive_expect_tx(&hdr->full[slot], static_cast<uint32_t>(rows) * (kb + vb));
-    bulk_load(dst, k_rows + static_cast<int64_t>(t) * kGmTile * kb, static_cast<uint32_t>(rows) * kb, &hdr->full[slot], policy);
-    bulk_load(dst + k_tile, v_rows + static_cast<int64_t>(t) * kGmTile * vb, static_cast<uint32_t>(rows) * vb, &hdr->full[slot],
-              policy);
+    const int64_t row0 = physical_row(p.pages, b, p.n_max, t * kGmTile);     // a tile lies inside one page
+    bulk_load(dst, k_slab + row0 * kb, static_cast<uint32_t>(rows) * kb, &hdr->full[slot], policy);
+    bulk_load(dst + k_tile, v_slab + row0 * vb, static_cast<uint32_t>(rows) * vb, &hdr->full[slot], policy);
   };
   if (tid == 0)
     for (int i = 0; i < stages && t_lo + i < t_hi; ++i) issue(t_lo + i, i);

@@ -15,7 +15,7 @@
 //           kappa = (2^30 - 1024) / S with S a power of two above every value scale met so far, and p <= 4 because the
 //           running maximum is raised as soon as a score exceeds it by 2.  The accumulators stay integers from
 //           block to block; they are folded into fp32 (o' += sum_n 256^n D_n - 8 sum_i F_i, times 1/kappa) only when
-//           the maximum or S is raised, every 2048 blocks, and at the end.
+//           the maximum or S is raised, every 1024 blocks, and at the end.
 // A warp owns 32 rows of every 128-row stage and walks the stages on its own; the stages arrive through a ring of
 // bulk copies.  Code layout of a block (written by quantize_blocks_kernel for 4-bit codes):
 //   keys:   [rp_k/8][G] words, word j of row i (channels 8j..8j+7) at j G + ((i + 8 (j & 3)) mod G): the rotation by

@@ -224,6 +224,7 @@ struct GqaDecodeParams {     // grouped-query decode (bf16 layers): `group` quer
   const float2* tile_step;  // [64]: cos, sin of -128 phi_i
   const float4* el_table;   // [32][128]: cos, cos, sin, sin of l phi for pairs 2k, 2k + 1 and row offset l
   int32_t interleaved;
+  PageMap pages;            // paged cache (decode_gqa_mma_kernel): a tile of 128 rows lies inside one page
 };
 
 // Quantised copy of the cache (Section 5.3 of the paper): per head a slab [B][blocks_max][block_bytes]; a block

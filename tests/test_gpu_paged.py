@@ -132,9 +132,13 @@ def test_page_table_argument_checks(B):
     with pytest.raises(B.EigenAttnError) as e:
         lay.quant_attach(4, 32)
     assert e.value.status == B.EA_ERR_UNSUPPORTED
+    # grouped queries follow the page table in the warp-level kernel; the tcgen05 kernel reads contiguous slabs only
+    assert float((lay.decode_gqa(q, 1).float() - lay.decode(q).float()).abs().max()) < 2e-2
+    lay.set_option(B.EA_OPT_GQA_IMPL, 1)
     with pytest.raises(B.EigenAttnError) as e:
         lay.decode_gqa(q, 1)
     assert e.value.status == B.EA_ERR_UNSUPPORTED
+    lay.set_option(B.EA_OPT_GQA_IMPL, 0)
     with pytest.raises(B.EigenAttnError) as e:         # the rows held must stay mapped
         lay.set_page_table([[2, -1], [-1, -1]], 128)
     assert e.value.status == B.EA_ERR_CAPACITY
@@ -193,3 +197,41 @@ def test_paged_layer_with_rotary_embedding_equals_contiguous_layer(B, interleave
     with pytest.raises(B.EigenAttnError) as e:
         odd.decode(q[:2, :1, :1].contiguous())
     assert e.value.status == B.EA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("g,rk,rv", [(4, [80, 80], [80, 80]), (12, [48, 128], [96, 64])])
+def test_grouped_queries_over_a_paged_cache(B, g, rk, rv):
+    """Grouped queries (no rotary embedding) of a paged layer: the warp-level kernel fetches every tile of 128 rows
+    from the page that holds it and returns what the contiguous layer returns, bit for bit, through several CTA counts
+    and a decode step; both agree with the oracle.  The tcgen05 kernel reads contiguous slabs only and is refused."""
+    B_, H, d, n_max, page_rows = 3, 2, 128, 1536, 128
+    n = 1100
+    U_k, U_v, _, k, v = make_case(B_, H, d, rk, rv, n + 1, BF16, seed_cfg=191)
+    W_q = synth.mixing_matrices(H * g, 16, d, 191, "W_Q")
+    qg = synth.lowrank_rows(W_q, B_, 1, 0.1, 191, "Q", dtype=BF16, device="cuda:0")
+    flat = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v)
+    paged = B.EigenAttnLayer(B_, H, d, n_max, BF16, U_k, U_v)
+    per_seq = n_max // page_rows
+    perm = np.random.default_rng(11).permutation(B_ * per_seq)
+    paged.set_page_table([[int(x) for x in perm[b * per_seq:(b + 1) * per_seq]] for b in range(B_)], page_rows)
+    ref = oracle_layer(B_, H, d, U_k, U_v)
+    for lay in (flat, paged):
+        lay.append_kv(k[:, :n], v[:, :n])
+    ref.append_kv(to_np(k[:, :n]), to_np(v[:, :n]))
+    expect = ref.decode_gqa(to_np(qg), g)
+    for ctas in (0, 1, 9, 300):
+        for lay in (flat, paged):
+            lay.set_option(B.EA_OPT_DECODE_CTAS, ctas)
+        want = flat.decode_gqa(qg, g)
+        assert torch.equal(paged.decode_gqa(qg, g), want), f"paged grouped decode differs, ctas={ctas}"
+        assert_close(want, expect, BF16, f"grouped queries, paged, ctas={ctas}")
+    for lay in (flat, paged):
+        lay.append_kv(k[:, n:], v[:, n:])
+    ref.append_kv(to_np(k[:, n:]), to_np(v[:, n:]))
+    want = flat.decode_gqa(qg, g)
+    assert torch.equal(paged.decode_gqa(qg, g), want)
+    assert_close(want, ref.decode_gqa(to_np(qg), g), BF16, "grouped queries, paged, after an append")
+    paged.poll_status(); flat.poll_status()
+    paged.set_option(B.EA_OPT_GQA_IMPL, 1)
+    with pytest.raises(B.EigenAttnError):
+        paged.decode_gqa(qg, g)
